@@ -1,0 +1,292 @@
+"""CPU oracle for one windowed denoising step (Window-Diffusion).
+
+TEST INFRASTRUCTURE ONLY.  This is a plain, slow, float64 numpy statement of
+what the step computes, written from the paper's text.  It shares no code with
+the CUDA library and must never be on a product path: only the tests, the
+smoke check and the benchmark's CPU-baseline leg may import it.
+
+What each part follows
+  * planner            Section 4.2 (dual-window sets, the buffer-set equation),
+                       Section 4.3 (one refresh step then normal steps per
+                       phase; newly decoded tokens keep being recomputed for a
+                       few steps), Section 5.3 "Effect of Cache Refresh Cycle"
+                       (in the authors' implementation that transient lasts
+                       until the next refresh).
+  * forward            Section 3.1 (bidirectional transformer forward, no
+                       causal mask) restricted to the rows Section 4.3 says
+                       are computed, reading K/V written at the refresh step
+                       (the cache-write equation of Section 4.3) for the rest.
+  * unmask             Section 3.2 Observation 1 / Section 4.1: decoding is
+                       decided by prediction confidence on the active tokens.
+
+The paper uses the pretrained models unmodified and does not restate their
+internals, so the block structure is the benchmark configurations' reading:
+pre-norm residual blocks, RMSNorm, rotary embedding at the absolute position
+(half-split pairing), grouped-query bidirectional attention with scale
+1/sqrt(dh), SwiGLU feed-forward, final RMSNorm, untied LM head, no biases.
+
+Parity pins: the forward is pinned to an independently written dense
+full-sequence forward (``dense_ref.py``) through the paper's reduction "window
+covers everything and every step is a refresh"; attention, RoPE, RMSNorm and
+the unmask rule are pinned to closed forms and brute force; the planner is
+pinned to the set identities of Section 4.2 and to a hand-traced trajectory.
+The readings the paper does not fix (transient length capped by T and reset at
+a refresh, forced early refresh when the window is exhausted, every model
+constant) are **parity unpinned against the paper**: they are only checked for
+internal consistency.
+"""
+from __future__ import annotations
+
+from dataclasses import dataclass, field
+
+import numpy as np
+
+NEVER = -(1 << 30)          # decode step of tokens that were given, not generated
+
+
+# ---------------------------------------------------------------------------
+# sequence state and planner (Sections 4.2 and 4.3)
+# ---------------------------------------------------------------------------
+
+@dataclass
+class SeqState:
+    """x^(t) of Section 3.1 plus the phase bookkeeping of Section 4.3."""
+    ids: np.ndarray                       # [S] token ids (mask id where undecoded)
+    decoded: np.ndarray                   # [S] bool
+    dec_step: np.ndarray = None           # [S] step at which a token was unmasked
+    t: int = 0                            # diffusion step index
+    since: int = 0                        # steps since the last refresh
+    phase_start: int = 0
+    wex: list = field(default_factory=list)   # external window of the current phase
+
+    def __post_init__(self):
+        self.ids = np.array(self.ids, dtype=np.int64)
+        self.decoded = np.array(self.decoded, dtype=bool)
+        if self.dec_step is None:
+            self.dec_step = np.full(self.ids.shape, NEVER, dtype=np.int64)
+
+
+def oracle_plan(st: SeqState, A: int, B: int, R: int, T: int) -> dict:
+    """Index sets for the step that comes next.  Does not modify ``st``.
+
+    Section 4.2: the external window is a fixed-length prefix of the undecoded
+    region, fixed within a phase; the internal (active) window is the front of
+    what is still undecoded inside it; buffer = external \\ (active ∪ decoded in
+    phase); undecoded tokens outside the external window are far-field.
+    Section 4.3: a phase is one refresh step followed by normal steps.
+    """
+    if A < 1 or B < 0 or R < 1 or T < 0:
+        raise ValueError("bad window parameters")
+    S = len(st.ids)
+    U = [i for i in range(S) if not st.decoded[i]]
+    if not U:
+        return dict(done=True)
+    Uset = set(U)
+    refresh = (st.t == 0) or (st.since >= R) or not any(i in Uset for i in st.wex)
+    if refresh:
+        wex = U[: min(A + B, len(U))]
+        phase_start = st.t
+    else:
+        wex = list(st.wex)
+        phase_start = st.phase_start
+    W = [i for i in wex if i in Uset]                    # still undecoded part
+    act = W[: min(A, len(W))]
+    buf = W[len(act):]
+    dp = [i for i in wex if i not in Uset]               # decoded within this phase
+    trans = [i for i in dp if 1 <= st.t - int(st.dec_step[i]) <= T]
+    wexset = set(wex)
+    far = [i for i in U if i not in wexset]
+    dec = [i for i in range(S) if st.decoded[i]]
+    vis = sorted(set(dec) | set(W))
+    rows = list(vis) if refresh else sorted(set(act) | set(trans))
+    return dict(done=False, refresh=refresh, wex=wex, phase_start=phase_start,
+                active=act, buffer=buf, in_phase_decoded=dp, transient=trans,
+                far_field=far, decoded=dec, vis=vis, rows=rows)
+
+
+def oracle_commit(st: SeqState, plan: dict, positions, token_ids) -> None:
+    """Apply the step's update set U^(t) (Section 3.1) and advance the phase
+    counters (Section 4.3)."""
+    if plan["refresh"]:
+        st.wex = list(plan["wex"])
+        st.phase_start = plan["phase_start"]
+        st.since = 0
+    for p, v in zip(positions, token_ids):
+        st.ids[p] = v
+        st.decoded[p] = True
+        st.dec_step[p] = st.t
+    st.t += 1
+    st.since += 1
+
+
+# ---------------------------------------------------------------------------
+# model pieces
+# ---------------------------------------------------------------------------
+
+def rmsnorm(x: np.ndarray, g: np.ndarray, eps: float) -> np.ndarray:
+    ms = np.mean(x * x, axis=-1, keepdims=True)
+    return g * x / np.sqrt(ms + eps)
+
+
+def rope(x: np.ndarray, pos: np.ndarray, theta: float) -> np.ndarray:
+    """x: [n, H, dh]; rotate pair (j, j + dh/2) by pos * theta^(-2j/dh)."""
+    n, H, dh = x.shape
+    half = dh // 2
+    j = np.arange(half, dtype=np.float64)
+    ang = np.asarray(pos, dtype=np.float64)[:, None] * theta ** (-2.0 * j / dh)[None, :]
+    c, s = np.cos(ang)[:, None, :], np.sin(ang)[:, None, :]
+    a, b = x[..., :half], x[..., half:]
+    return np.concatenate([a * c - b * s, b * c + a * s], axis=-1)
+
+
+def silu(z: np.ndarray) -> np.ndarray:
+    return z / (1.0 + np.exp(-z))
+
+
+def attention_rows(q: np.ndarray, K: np.ndarray, V: np.ndarray, group: int):
+    """Bidirectional attention of n query rows over m visible positions.
+
+    q: [n, Hq, dh]; K, V: [m, Hkv, dh].  Query head h uses KV head h // group.
+    Returns (out [n, Hq, dh], probs [n, Hq, m]).  No mask (Section 3.1).
+    """
+    n, Hq, dh = q.shape
+    out = np.empty_like(q)
+    probs = np.empty((n, Hq, K.shape[0]), dtype=np.float64)
+    for h in range(Hq):
+        kv = h // group
+        s = q[:, h, :] @ K[:, kv, :].T / np.sqrt(dh)
+        s = s - s.max(axis=-1, keepdims=True)
+        p = np.exp(s)
+        p /= p.sum(axis=-1, keepdims=True)
+        probs[:, h, :] = p
+        out[:, h, :] = p @ V[:, kv, :]
+    return out, probs
+
+
+@dataclass
+class KVCache:
+    """Per-sequence fp64 K/V of every layer, indexed by absolute position."""
+    K: np.ndarray      # [L, S, Hkv, dh]
+    V: np.ndarray
+
+    @staticmethod
+    def empty(dims: dict, S: int, fill=np.nan) -> "KVCache":
+        shape = (dims["L"], S, dims["Hkv"], dims["dh"])
+        return KVCache(np.full(shape, fill), np.full(shape, fill))
+
+
+def oracle_layer(dims: dict, lw: dict, x: np.ndarray, pos, vis, cache: KVCache, l: int,
+                 want_probs: bool = False) -> dict:
+    """One transformer block over the computed rows ``pos`` (ascending
+    positions) whose inputs are ``x`` [n, d].  All fresh K/V are written to the
+    cache before any row attends; attention then reads every visible position
+    from the cache (fresh rows included).  Returns the block output and the
+    attention output (before the output projection)."""
+    Hq, Hkv, dh = dims["Hq"], dims["Hkv"], dims["dh"]
+    n = x.shape[0]
+    pos = np.asarray(pos, dtype=np.int64)
+    a = rmsnorm(x, lw["attn_norm"], dims["eps"])
+    q = (a @ lw["wq"].T).reshape(n, Hq, dh)
+    k = (a @ lw["wk"].T).reshape(n, Hkv, dh)
+    v = (a @ lw["wv"].T).reshape(n, Hkv, dh)
+    q = rope(q, pos, dims["theta"])
+    k = rope(k, pos, dims["theta"])
+    cache.K[l, pos] = k
+    cache.V[l, pos] = v
+    vis = np.asarray(vis, dtype=np.int64)
+    o, probs = attention_rows(q, cache.K[l, vis], cache.V[l, vis], Hq // Hkv)
+    o = o.reshape(n, Hq * dh)
+    h = x + o @ lw["wo"].T
+    f = rmsnorm(h, lw["ffn_norm"], dims["eps"])
+    y = h + (silu(f @ lw["w_gate"].T) * (f @ lw["w_up"].T)) @ lw["w_down"].T
+    res = dict(out=y, attn=o)
+    if want_probs:
+        res["probs"] = probs
+    return res
+
+
+# ---------------------------------------------------------------------------
+# unmask rule
+# ---------------------------------------------------------------------------
+
+def oracle_unmask(logits: np.ndarray, positions, k: int) -> dict:
+    """Choose which active positions to unmask.
+
+    Per row: token = lowest index among the maximal logits, confidence = the
+    softmax probability of that token = 1 / sum_v exp(logit_v - max).  Rows are
+    ranked by confidence (descending), equal confidence by position
+    (ascending); the first min(k, rows) are unmasked.
+    """
+    logits = np.asarray(logits, dtype=np.float64)
+    n = logits.shape[0]
+    ids = np.empty(n, dtype=np.int64)
+    conf = np.empty(n, dtype=np.float64)
+    for r in range(n):
+        m = logits[r].max()
+        ids[r] = int(np.flatnonzero(logits[r] == m)[0])
+        conf[r] = 1.0 / np.exp(logits[r] - m).sum()
+    order = sorted(range(n), key=lambda r: (-conf[r], positions[r]))
+    chosen = order[: min(k, n)]
+    return dict(ids=ids, conf=conf, order=order,
+                positions=[int(positions[r]) for r in chosen],
+                token_ids=[int(ids[r]) for r in chosen],
+                confidence=[float(conf[r]) for r in chosen])
+
+
+# ---------------------------------------------------------------------------
+# one step
+# ---------------------------------------------------------------------------
+
+def oracle_step(model, states, caches, A: int, B: int, R: int, T: int, k: int,
+                forced=None, want_probs: bool = False, commit: bool = True) -> list:
+    """One windowed denoising step for a batch of independent sequences.
+
+    ``model`` supplies float64 weights (``dims``, ``embed_rows``, ``layer``,
+    ``final_norm``, ``lm_head``).  ``forced[i]`` = (positions, token_ids)
+    replaces sequence i's own unmask choice (teacher forcing).  Returns one
+    dict per sequence: the plan, per-layer outputs, attention outputs, logits
+    of the active rows, confidences and the chosen update set.
+    """
+    dims = model.dims
+    plans = [oracle_plan(st, A, B, R, T) for st in states]
+    outs = []
+    xs = []
+    for st, pl in zip(states, plans):
+        if pl["done"]:
+            outs.append(dict(plan=pl, done=True))
+            xs.append(None)
+            continue
+        rows = pl["rows"]
+        xs.append(model.embed_rows(st.ids[rows]))
+        outs.append(dict(plan=pl, done=False, layer_out=[], attn_out=[], probs=[]))
+    for l in range(dims["L"]):
+        lw = model.layer(l)
+        for i, (pl, cache) in enumerate(zip(plans, caches)):
+            if pl["done"]:
+                continue
+            r = oracle_layer(dims, lw, xs[i], pl["rows"], pl["vis"], cache, l, want_probs)
+            xs[i] = r["out"]
+            outs[i]["layer_out"].append(r["out"])
+            outs[i]["attn_out"].append(r["attn"])
+            if want_probs:
+                outs[i]["probs"].append(r["probs"])
+    g_final = model.final_norm()
+    w_lm = None
+    for i, (st, pl) in enumerate(zip(states, plans)):
+        if pl["done"]:
+            continue
+        if w_lm is None:
+            w_lm = model.lm_head()
+        rows = pl["rows"]
+        sel = [rows.index(p) for p in pl["active"]]
+        logits = rmsnorm(xs[i][sel], g_final, dims["eps"]) @ w_lm.T
+        um = oracle_unmask(logits, pl["active"], k)
+        outs[i].update(logits=logits, unmask=um)
+        if forced is not None and forced[i] is not None:
+            pos, tok = forced[i]
+        else:
+            pos, tok = um["positions"], um["token_ids"]
+        outs[i]["committed"] = (list(pos), list(tok))
+        if commit:
+            oracle_commit(st, pl, pos, tok)
+    return outs

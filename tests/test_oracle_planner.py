@@ -1,0 +1,171 @@
+"""Pins for the oracle's planner: the set identities of Section 4.2, the phase
+structure of Section 4.3 and a hand-traced trajectory."""
+import os
+
+import numpy as np
+import pytest
+
+from oracle.wd_oracle import SeqState, oracle_plan, oracle_commit
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden", "planner_trace.txt")
+
+
+def _state(P, G, mask_id=99):
+    ids = np.array([1] * P + [mask_id] * G)
+    dec = np.array([True] * P + [False] * G)
+    return SeqState(ids=ids, decoded=dec)
+
+
+def _parse(field):
+    field = field.strip()
+    return [] if field == "-" else [int(v) for v in field.split()]
+
+
+def test_hand_traced_trajectory():
+    st = _state(4, 10)
+    A, B, R, T = 3, 3, 3, 1
+    rows = [l for l in open(GOLDEN).read().splitlines() if l and not l.startswith("#")]
+    assert len(rows) == 4
+    for line in rows:
+        f = [c.strip() for c in line.split("|")]
+        pl = oracle_plan(st, A, B, R, T)
+        assert st.t == int(f[0])
+        assert pl["refresh"] == (f[1] == "refresh")
+        for name, col in (("wex", 2), ("active", 3), ("buffer", 4), ("in_phase_decoded", 5),
+                          ("transient", 6), ("far_field", 7), ("vis", 8), ("rows", 9)):
+            assert pl[name] == _parse(f[col]), (f[0], name)
+        oracle_commit(st, pl, [int(f[10])], [7])
+
+
+def _random_walk(seed, S, frac, A, B, R, T, k, prefix):
+    rng = np.random.default_rng(seed)
+    if prefix:
+        P = int(S * frac)
+        dec = np.arange(S) < P
+    else:
+        dec = rng.random(S) < frac
+    st = SeqState(ids=np.zeros(S, dtype=np.int64), decoded=dec)
+    trace = []
+    while True:
+        pl = oracle_plan(st, A, B, R, T)
+        if pl["done"]:
+            break
+        trace.append((st.t, st.since, pl, st.decoded.copy()))
+        n = min(k, len(pl["active"]))
+        pick = list(rng.choice(pl["active"], size=n, replace=False))
+        oracle_commit(st, pl, pick, [5] * n)
+    return st, trace
+
+
+CASES = [  # seed, S, frac, A, B, R, T, k, prefix
+    (0, 40, 0.3, 4, 6, 3, 1, 1, True),
+    (1, 64, 0.25, 8, 16, 4, 2, 1, True),
+    (2, 64, 0.5, 8, 0, 1, 0, 2, True),
+    (3, 50, 0.4, 3, 5, 5, 9, 2, False),
+    (4, 50, 0.1, 6, 2, 16, 3, 3, False),
+    (5, 30, 0.0, 30, 0, 1, 0, 4, True),
+    (6, 45, 0.3, 2, 1, 8, 2, 1, False),     # k*R > A+B: window exhausted mid-phase
+]
+
+
+@pytest.mark.parametrize("case", CASES)
+def test_set_invariants(case):
+    seed, S, frac, A, B, R, T, k, prefix = case
+    st, trace = _random_walk(*case)
+    assert st.decoded.all()
+    prev_min_act, prev_max_wex, prev_vis, prev_refresh_t = -1, -1, None, None
+    for t, since, pl, decoded in trace:
+        U = set(np.flatnonzero(~decoded).tolist())
+        D = set(np.flatnonzero(decoded).tolist())
+        act, buf, far = set(pl["active"]), set(pl["buffer"]), set(pl["far_field"])
+        # partition of the undecoded region (Section 4.2)
+        assert act | buf | far == U
+        assert not (act & buf) and not (act & far) and not (buf & far)
+        assert len(act) + len(buf) + len(far) == len(U)
+        assert set(pl["decoded"]) == D and D | U == set(range(S))
+        wex = set(pl["wex"])
+        # B = W_ex \ (A u D_p)
+        assert buf == wex - (act | set(pl["in_phase_decoded"]))
+        assert act <= wex and far == U - wex
+        assert set(pl["transient"]) <= set(pl["in_phase_decoded"]) <= D
+        # the internal window is the front of the undecoded prefix and keeps its size
+        assert min(U) in act
+        assert len(act) == min(A, len(wex & U))
+        assert max(act) < min(buf | far | {S})
+        # lists are ascending
+        for name in ("active", "buffer", "far_field", "decoded", "vis", "rows", "transient"):
+            assert pl[name] == sorted(pl[name])
+        # window slides monotonically to the right
+        # (the right edge is that of the visible set: near the end the external
+        #  window is "whatever is left", whose maximum may lie left of an earlier one)
+        assert min(act) >= prev_min_act and max(pl["vis"]) >= prev_max_wex
+        prev_min_act, prev_max_wex = min(act), max(pl["vis"])
+        assert len(pl["transient"]) <= k * min(T, since)
+        if pl["refresh"]:
+            assert pl["rows"] == pl["vis"] and not pl["in_phase_decoded"]
+            assert len(wex) == min(A + B, len(U))
+            prev_refresh_t = t
+        else:
+            assert set(pl["rows"]) == act | set(pl["transient"])
+            assert pl["vis"] == prev_vis            # |vis| constant within a phase
+            assert t - prev_refresh_t < R           # one refresh then at most R-1 normal steps
+        prev_vis = pl["vis"]
+        assert set(pl["vis"]) == D | (wex & U)
+        # contiguity: with a decoded prefix the visible set is a range [0, hi]
+        if prefix:
+            assert pl["vis"] == list(range(len(pl["vis"])))
+
+
+def test_phase_is_one_refresh_then_normal_steps():
+    st, trace = _random_walk(7, 200, 0.2, 8, 24, 4, 2, 1, True)
+    kinds = [pl["refresh"] for _, _, pl, _ in trace]
+    # k*R <= A+B so no forced refresh: the pattern is strictly periodic
+    assert kinds[:12] == [True, False, False, False] * 3
+
+
+def test_paper_transient_mode():
+    """Section 5.3: in the authors' implementation tokens decoded inside the
+    window are recomputed until the next refresh, i.e. T >= R-1 makes the
+    transient set equal the in-phase decoded set."""
+    _, trace = _random_walk(8, 120, 0.25, 8, 24, 6, 5, 2, True)
+    seen = 0
+    for _, _, pl, _ in trace:
+        assert pl["transient"] == pl["in_phase_decoded"]
+        seen += len(pl["transient"])
+    assert seen > 0
+
+
+def test_transient_ages_out_and_resets_at_refresh():
+    st = _state(2, 20)
+    A, B, R, T = 4, 4, 5, 2
+    ages = []
+    for step in range(5):
+        pl = oracle_plan(st, A, B, R, T)
+        ages.append(sorted(st.t - int(st.dec_step[i]) for i in pl["transient"]))
+        oracle_commit(st, pl, [pl["active"][0]], [3])
+    assert ages == [[], [1], [1, 2], [1, 2], [1, 2]]
+    pl = oracle_plan(st, A, B, R, T)
+    assert pl["refresh"] and pl["transient"] == []
+
+
+def test_forced_refresh_when_window_exhausted():
+    st = _state(1, 12)
+    A, B, R, T = 2, 0, 8, 1
+    kinds = []
+    for _ in range(4):
+        pl = oracle_plan(st, A, B, R, T)
+        kinds.append(pl["refresh"])
+        oracle_commit(st, pl, pl["active"], [3] * len(pl["active"]))
+    assert kinds == [True, True, True, True]
+
+
+def test_plan_is_pure_and_done():
+    st = _state(3, 2)
+    before = (st.ids.copy(), st.decoded.copy(), st.t, st.since, list(st.wex))
+    oracle_plan(st, 2, 2, 2, 1)
+    assert (st.ids == before[0]).all() and (st.decoded == before[1]).all()
+    assert (st.t, st.since, st.wex) == (before[2], before[3], before[4])
+    done = SeqState(ids=np.zeros(3), decoded=np.ones(3, dtype=bool))
+    assert oracle_plan(done, 2, 2, 2, 1)["done"]
+    with pytest.raises(ValueError):
+        oracle_plan(st, 0, 2, 2, 1)
