@@ -1,0 +1,328 @@
+#!/usr/bin/env python
+"""Benchmark of the windowed denoising step on B200.
+
+Default workload: the LLaDA-8B-shaped bf16 configuration (32 layers, d 4096,
+32 heads x 128, FFN 12288, vocab 126464; prompt 256 + 256 masks; A=32, B=64,
+R=8, T=2, one token per step, batch 1) with seeded random-init weights and
+uniform-random prompt ids.  A "step" is one wd_step + wd_step_sync of the
+generation trajectory (one refresh step then R-1 normal steps per phase).
+
+Prints ONE JSON line.  `value` is generated tokens/s with the state resident
+on the GPU; `e2e` is the same loop timed on the host clock from host buffers
+(ids uploaded inside the timed region, per-step index lists up and results
+down); `roofline` is the tensor-core GEMM kernel's algorithmic bytes over its
+CUDA-event time; `cpu_baseline` is the fp64 oracle timed on the host cores.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config NAME]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+from paper_2601_20332_b200 import synth
+
+METRIC = "generated tokens/s (windowed denoising steps, LLaDA-8B shape, 1 B200)"
+UNIT = "tokens/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons sampled while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu, self.proc, self.path = gpu_index, None, None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            os.close(fd)
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.Q}",
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=open(self.path, "w"), stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        try:
+            for line in open(self.path):
+                f = [c.strip() for c in line.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def algorithmic_step(cfg, rows, n_act, vis, batch=1):
+    """Bytes and FLOPs the method itself must move / compute in one step
+    (weights once, K/V of the visible positions read, fresh K/V written)."""
+    L, d, Hq, Hkv, dh, F, V = (cfg[k] for k in ("L", "d", "Hq", "Hkv", "dh", "F", "V"))
+    w = 2 if cfg["dtype"] == "bf16" else 4
+    per_layer = d * (Hq + 2 * Hkv) * dh + Hq * dh * d + 3 * d * F
+    kv_tok = 2 * Hkv * dh * w * L
+    by = per_layer * L * w + V * d * w + vis * kv_tok + rows * kv_tok
+    fl = 2 * rows * per_layer * L + 2 * n_act * d * V + 4 * rows * (vis / max(batch, 1)) * Hq * dh * L
+    return by, fl
+
+
+def run_ours(args, rank, world):
+    from paper_2601_20332_b200 import binding as wd
+    from paper_2601_20332_b200 import build as wd_build
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = f"cuda:{local}"
+    wd_build.build()
+    wd.lib()
+    cfg = synth.get_config(args.config)
+    A, B, R, T, k, batch = (cfg[x] for x in ("A", "B", "R", "T", "k", "batch"))
+    S = cfg["P"] + cfg["G"]
+    K, W = args.steps, args.warmup
+    assert W + K <= cfg["G"] // k, "steps + warmup exceed the generation length"
+    w = synth.make_weights(cfg, dev)
+    ids = synth.make_prompts(cfg)
+    ctx = wd.Context(cfg, w, batch, S, batch * S, batch * max(A, cfg["G"]))
+    stream = torch.cuda.Stream(device=dev)
+    peaks = measured_peaks()
+
+    def trajectory(n_warm, n_timed, state, timed_cb=None):
+        infos, per_step = [], []
+        for i in range(n_warm):
+            state.step(A, B, R, T, k, stream)
+            state.sync()
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(n_timed + 1)]
+        t0 = time.perf_counter()
+        ev[0].record(stream)
+        for i in range(n_timed):
+            _, info = state.step(A, B, R, T, k, stream)
+            ev[i + 1].record(stream)
+            state.sync()
+            infos.append(info)
+        torch.cuda.synchronize()
+        wall = time.perf_counter() - t0
+        if world > 1:
+            torch.distributed.barrier()
+        per_step = [ev[i].elapsed_time(ev[i + 1]) for i in range(n_timed)]
+        return infos, per_step, ev[0].elapsed_time(ev[n_timed]), wall
+
+    # ---- device-resident run: the headline value
+    state = wd.State(ctx, ids)
+    sampler = ClockSampler(local)
+    sampler.start()
+    infos, per_step, total_ms, _ = trajectory(W, K, state)
+    # ---- same trajectory again with GEMM events: roofline of the dominant kernel
+    state.reset(ids, None, stream)
+    ctx.profile_enable(True)
+    p_infos, _, _, _ = trajectory(W, K, state)
+    prof = ctx.profile_read()
+    ctx.profile_enable(False)
+    clocks = sampler.stop()
+    # ---- end to end from host buffers on the host clock
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    state.reset(ids, None, stream)
+    for i in range(W + K):
+        state.step(A, B, R, T, k, stream)
+        state.sync()
+    torch.cuda.synchronize()
+    e2e_wall = time.perf_counter() - t0
+    # ---- the full-sequence no-pruning step at the same starting state, for context
+    state.reset(ids, None, stream)
+    full_ms = []
+    for i in range(4):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        state.step(cfg["G"], 0, 1, 0, k, stream)
+        e1.record(stream)
+        state.sync()
+        torch.cuda.synchronize()
+        full_ms.append(e0.elapsed_time(e1))
+    state.close()
+
+    t_total = torch.tensor([total_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        torch.distributed.all_reduce(t_total, op=torch.distributed.ReduceOp.MAX)
+    total_ms = float(t_total.item())
+    tokens = batch * k * K * world
+    value = tokens / (total_ms * 1e-3)
+    normal = [t for t, i in zip(per_step, infos) if not i["is_refresh"]]
+    refresh = [t for t, i in zip(per_step, infos) if i["is_refresh"]]
+    # roofline of the GEMM kernel: algorithmic bytes per launch / average launch time
+    n_l = max(prof["gemm_launches"], 1)
+    gemm_gbs = prof["gemm_bytes"] / (prof["gemm_ms"] * 1e-3) / 1e9 if prof["gemm_ms"] > 0 else 0.0
+    # whole-step roofline for the normal step (HBM bound)
+    ni = [i for i in infos if not i["is_refresh"]]
+    step_by, step_fl = algorithmic_step(cfg, np.mean([i["n_rows"] for i in ni]) if ni else 0,
+                                        np.mean([i["n_active"] for i in ni]) if ni else 0,
+                                        np.mean([i["n_vis"] for i in ni]) if ni else 0, batch)
+    normal_ms = float(np.median(normal)) if normal else None
+    plan_ints = np.mean([2 * i["n_rows"] + 2 * i["n_active"] + 2 * (batch + 1) + i["n_vis"] for i in infos])
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
+        "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": cfg["dtype"], "data": "synthetic",
+        "config": {"workload": f"{args.config}: LLaDA-8B-shaped bf16, prompt {cfg['P']} + {cfg['G']} masks, A={A} B={B} R={R} "
+                               f"T={T} k={k} batch {batch}; steps {W}..{W + K - 1} of the generation; replicas only at N>1",
+                   "l2": "inputs larger than L2: every step streams 15 GB of weights",
+                   "normal_step_ms": normal_ms, "refresh_step_ms": float(np.median(refresh)) if refresh else None,
+                   "normal_step_algorithmic_gb": step_by / 1e9,
+                   "normal_step_frac_of_hbm_roofline_measured": (step_by / (normal_ms * 1e-3) / 1e9 / peaks["hbm_gbs"])
+                   if normal_ms else None,
+                   "normal_step_frac_of_hbm_roofline_nominal_8TBs": (step_by / (normal_ms * 1e-3) / 8e12) if normal_ms else None,
+                   "full_sequence_step_ms": float(np.median(full_ms)),
+                   "rows_normal": float(np.mean([i["n_rows"] for i in ni])) if ni else None,
+                   "gemm_impl": infos[-1]["gemm_impl"]},
+        "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
+                   "samples": clocks["samples"]},
+        "e2e": {"value": batch * k * (W + K) * world / e2e_wall, "unit": UNIT,
+                "h2d_bytes_per_step": float(plan_ints * 4 + batch * S * 4 / (W + K)),
+                "d2h_bytes_per_step": float((1 + batch + 3 * batch * k) * 4)},
+        "gpu_launches": int(sum(i["n_launches"] for i in infos)),
+        "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel", "achieved": gemm_gbs, "peak": peaks["hbm_gbs"],
+                     "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+                     "traffic": None, "launches": int(prof["gemm_launches"]),
+                     "avg_launch_us": prof["gemm_ms"] * 1e3 / n_l, "bytes_per_launch": prof["gemm_bytes"] / n_l},
+    }
+    if rank == 0:
+        line["cpu_baseline"] = cpu_baseline(cfg, w, ids, budget_s=args.cpu_seconds)
+        print(json.dumps(line))
+    ctx.close()
+
+
+def cpu_baseline(cfg, w, ids, budget_s=25.0):
+    """The oracle as it stands, timed on the host cores on a bounded sample:
+    one refresh step and one normal step of the same workload truncated to 1
+    and to 2 layers, extrapolated linearly in depth to the full model."""
+    from oracle import wd_oracle as wo
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = os.cpu_count() or 1
+    S = cfg["P"] + cfg["G"]
+    A, B, R, T, k = (cfg[x] for x in ("A", "B", "R", "T", "k"))
+
+    class Truncated(synth.OracleModelView):
+        def __init__(self, w, n_layers):
+            super().__init__(w)
+            self.dims = dict(self.dims, L=n_layers)
+
+    times = {}
+    for nl in (1, 2):
+        model = Truncated(w, nl)
+        st = [wo.SeqState(ids=ids[0], decoded=np.arange(S) < cfg["P"])]
+        cache = [wo.KVCache.empty(model.dims, S)]
+        t0 = time.perf_counter()
+        wo.oracle_step(model, st, cache, A, B, R, T, k)
+        t1 = time.perf_counter()
+        wo.oracle_step(model, st, cache, A, B, R, T, k)
+        t2 = time.perf_counter()
+        times[nl] = (t1 - t0, t2 - t1)
+    L = cfg["L"]
+    per_layer_r, per_layer_n = times[2][0] - times[1][0], times[2][1] - times[1][1]
+    t_refresh = times[1][0] + (L - 1) * max(per_layer_r, 0.0)
+    t_normal = times[1][1] + (L - 1) * max(per_layer_n, 0.0)
+    phase = t_refresh + (R - 1) * t_normal
+    return {"value": k * R / phase, "unit": UNIT, "cores": int(cores), "kind": "oracle",
+            "sample": f"one refresh + one normal step of batch-1 sequence 0 at 1 and 2 of {L} layers, extrapolated linearly "
+                      f"in depth; refresh {t_refresh:.1f} s, normal {t_normal:.1f} s per step"}
+
+
+def run_reference(args, rank, world):
+    """The reference arm is the CPU oracle (there is no reference implementation)."""
+    if rank != 0:
+        return
+    cfg = synth.get_config(args.config)
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    w = synth.make_weights(cfg, dev)
+    ids = synth.make_prompts(cfg)
+    vals = []
+    for i in range(args.warmup + args.steps):
+        cb = cpu_baseline(cfg, w, ids)
+        if i >= args.warmup:
+            vals.append(cb["value"])
+    v = float(np.mean(vals))
+    R, k = cfg["R"], cfg["k"]
+    cb["value"] = v
+    print(json.dumps({"impl": "reference", "metric": METRIC, "value": v, "unit": UNIT, "n_gpus": world,
+                      "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * k / v, "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+                      "config": {"workload": f"{args.config}: fp64 CPU oracle on a bounded sample of the same workload"},
+                      "cpu_baseline": cb,
+                      "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--config", default="llada8b")
+    ap.add_argument("--cpu-seconds", type=float, default=25.0)
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if args.impl == "reference":
+        args.steps = 1 if args.steps is None else min(args.steps, 3)
+        args.warmup = 0 if args.warmup is None else min(args.warmup, 1)
+        run_reference(args, rank, world)
+        return
+    args.steps = 64 if args.steps is None else args.steps
+    args.warmup = 8 if args.warmup is None else max(args.warmup, 3)
+    if world > 1:
+        torch.distributed.init_process_group("nccl", device_id=torch.device(f"cuda:{int(os.environ.get('LOCAL_RANK', 0))}"))
+    try:
+        run_ours(args, rank, world)
+    finally:
+        if world > 1:
+            torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

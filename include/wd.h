@@ -1,0 +1,312 @@
+/*
+ * wd.h — C ABI of the windowed denoising step (Window-Diffusion) for NVIDIA B200.
+ *
+ * One call of wd_step() runs one diffusion step of a masked diffusion language
+ * model over only the tokens the method says must be computed:
+ *   - the sequence is a fixed-length state of decoded tokens and [MASK]
+ *     placeholders (paper Section 3.1);
+ *   - undecoded tokens are split into an external window (a fixed-length prefix
+ *     of the undecoded region), its front part the internal window of ACTIVE
+ *     tokens, the BUFFER tokens (external minus active minus tokens decoded in
+ *     this phase) and the pruned FAR-FIELD tokens (Section 4.2);
+ *   - steps are grouped into phases of one REFRESH step (full forward over the
+ *     decoded tokens and the external window, all K/V written to the cache)
+ *     followed by NORMAL steps (only active tokens and recently decoded tokens
+ *     are computed; buffer and earlier decoded tokens are read from the cache)
+ *     (Section 4.3);
+ *   - logits exist only for active tokens, and the step ends by unmasking the
+ *     k active tokens with the highest prediction confidence (Section 4.1,
+ *     Observation 1 of Section 3.2).
+ *
+ * Conventions
+ *   - Every function returns a wd_status (0 = WD_OK, positive = informational,
+ *     negative = error).  Nothing aborts, traps or throws across this boundary.
+ *   - "device" pointers are CUDA device memory of the current device, "host"
+ *     pointers are ordinary host memory.  The library never allocates device
+ *     memory: the caller passes workspaces whose sizes the *_bytes functions
+ *     report.  All device pointers must be 256-byte aligned.
+ *   - Borrowed memory (weights, workspaces, debug taps) stays owned by the
+ *     caller and must outlive the object that borrows it.
+ *   - The library is sm_100a only and has no CPU fallback.
+ */
+#ifndef WD_H
+#define WD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define WD_API __attribute__((visibility("default")))
+#else
+#define WD_API
+#endif
+
+typedef int wd_status;
+
+enum {
+    WD_OK = 0,
+    WD_DONE = 1,                      /* no undecoded token left anywhere      */
+    WD_ERR_NULL = -1,                 /* a required pointer is NULL            */
+    WD_ERR_INVALID_DIMS = -2,
+    WD_ERR_WORKSPACE_TOO_SMALL = -3,
+    WD_ERR_UNSUPPORTED_ARCH = -4,     /* current device is not sm_100          */
+    WD_ERR_BAD_PARAM = -5,            /* A<1, B<0, R<1, T<0, k<0, bad index... */
+    WD_ERR_CAPACITY = -6,             /* a caller-sized buffer is too short    */
+    WD_ERR_PENDING = -7,              /* wd_step without wd_step_sync before   */
+    WD_ERR_CUDA = -8,                 /* a CUDA runtime/driver call failed     */
+    WD_ERR_DEVICE_TIMEOUT = -9,       /* a bounded device-side wait ran out    */
+    WD_ERR_BOUNDS = -10,              /* a device-side index check failed      */
+    WD_ERR_NOT_PENDING = -11,         /* wd_step_sync without wd_step before   */
+    WD_ERR_MISALIGNED = -12
+};
+
+enum { WD_F32 = 0, WD_BF16 = 1 };     /* element type of weights, activations, K/V cache */
+
+/* GEMM implementation selector (wd_set_gemm_impl, wd_op_gemm). */
+enum {
+    WD_GEMM_AUTO = 0,                 /* tensor-core kernel for bf16, plain for f32 */
+    WD_GEMM_PLAIN = 1,                /* CUDA-core kernel (any dtype)               */
+    WD_GEMM_TCGEN05 = 2               /* tcgen05/TMEM/TMA kernel (bf16 only)        */
+};
+
+/* Model shape.  The paper runs the pretrained model unmodified (Section 4.1),
+ * so the block is the usual one: pre-norm residual blocks with RMSNorm, rotary
+ * embedding at the absolute position, bidirectional grouped-query attention,
+ * SwiGLU feed-forward, final RMSNorm, untied LM head, no biases. */
+typedef struct wd_model_dims {
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ffn, vocab;
+    float   rope_theta, rms_eps;
+    int32_t dtype;                    /* WD_F32 or WD_BF16                                  */
+    int32_t mask_id;                  /* id of the [MASK] placeholder (Section 3.1)         */
+    int32_t max_batch;                /* sequences per state                                */
+    int32_t max_seq;                  /* S: positions per sequence                          */
+    int32_t max_rows;                 /* most rows computed in one step, whole batch        */
+    int32_t max_active;               /* most active rows in one step, whole batch          */
+} wd_model_dims;
+
+/* Device pointers to the weights, row-major with the reduction dimension
+ * contiguous ("[out, in]").  Per-layer members are HOST arrays of n_layers
+ * device pointers.  Matrices have the model dtype; norm gains are float.
+ * Borrowed, never written. */
+typedef struct wd_weights {
+    const void*         tok_embed;    /* [vocab, d_model]                     */
+    const void* const*  wq;           /* [n_q_heads*head_dim, d_model]        */
+    const void* const*  wk;           /* [n_kv_heads*head_dim, d_model]       */
+    const void* const*  wv;           /* [n_kv_heads*head_dim, d_model]       */
+    const void* const*  wo;           /* [d_model, n_q_heads*head_dim]        */
+    const void* const*  w_gate;       /* [d_ffn, d_model]                     */
+    const void* const*  w_up;         /* [d_ffn, d_model]                     */
+    const void* const*  w_down;       /* [d_model, d_ffn]                     */
+    const float* const* attn_norm;    /* [d_model]                            */
+    const float* const* ffn_norm;     /* [d_model]                            */
+    const float*        final_norm;   /* [d_model]                            */
+    const void*         lm_head;      /* [vocab, d_model]                     */
+} wd_weights;
+
+typedef struct wd_ctx wd_ctx;         /* model + step workspace               */
+typedef struct wd_state wd_state;     /* a batch of sequences + their K/V cache */
+
+/* Index sets of one sequence for the next step (Section 4.2; the buffer-set
+ * equation; Section 4.3 for which rows are computed).  The caller allocates
+ * every list with `capacity` entries (capacity >= sequence length is always
+ * enough); lists come back ascending. */
+typedef struct wd_index_sets {
+    int32_t  capacity;
+    int32_t* active;       int32_t n_active;      /* internal window A^(t)                       */
+    int32_t* buffer;       int32_t n_buffer;      /* B^(t): undecoded context read from the cache */
+    int32_t* decoded;      int32_t n_decoded;     /* every decoded position                      */
+    int32_t* transient;    int32_t n_transient;   /* decoded in this phase and still recomputed  */
+    int32_t* far_field;    int32_t n_far_field;   /* pruned undecoded positions                  */
+    int32_t* rows;         int32_t n_rows;        /* positions computed this step                */
+    int32_t* vis;          int32_t n_vis;         /* positions whose K/V are attended            */
+    int32_t* ext_window;   int32_t n_ext_window;  /* W_ex^(p) as fixed at the phase start        */
+    int32_t  is_refresh;                          /* 1 = refresh step, 0 = normal step           */
+    int32_t  vis_contiguous;                      /* 1 if vis == [0, n_vis)                      */
+    int32_t  done;                                /* 1 if the sequence has no undecoded token    */
+} wd_index_sets;
+
+/* Result of a step, host memory, caller-allocated: n_unmasked[batch];
+ * positions / token_ids / confidence [batch * k] with sequence i at offset i*k,
+ * ranked by confidence (highest first; equal confidence: lowest position). */
+typedef struct wd_step_out {
+    int32_t* n_unmasked;
+    int32_t* positions;
+    int32_t* token_ids;
+    float*   confidence;
+} wd_step_out;
+
+/* Optional device buffers that receive intermediate values of the next steps
+ * (for parity tests; leave unset in timed runs).  Any member may be NULL.
+ * With n_rows computed rows and n_act active rows in the step (whole batch,
+ * sequences concatenated in order, positions ascending inside a sequence):
+ *   layer_out [n_layers][n_rows][d_model]   block outputs (residual stream)
+ *   attn_out  [n_layers][n_rows][n_q_heads*head_dim]   attention outputs before
+ *             the output projection
+ *   logits    [n_act][vocab]   logits of the active rows
+ * all float.  Capacities are for max_rows / max_active. */
+typedef struct wd_debug_taps {
+    float* layer_out;
+    float* attn_out;
+    float* logits;
+} wd_debug_taps;
+
+/* Per-step counters filled by wd_step (host). */
+typedef struct wd_step_info {
+    int32_t is_refresh;      /* any sequence refreshed (sequences of a state share the phase clock) */
+    int32_t n_rows;          /* rows computed, whole batch   */
+    int32_t n_active;        /* active rows, whole batch     */
+    int32_t n_vis;           /* visible positions, summed    */
+    int32_t n_launches;      /* kernels enqueued by the step */
+    int32_t gemm_impl;       /* WD_GEMM_PLAIN or WD_GEMM_TCGEN05 actually used */
+} wd_step_info;
+
+/* ---- sizes -------------------------------------------------------------- */
+
+/* Bytes of device workspace wd_create needs for these dims (0 if invalid). */
+WD_API size_t wd_workspace_bytes(const wd_model_dims* dims);
+/* Bytes of device memory one state of `batch` sequences of `seq_len` positions
+ * needs (token ids + K/V cache of every layer; 0 if invalid). */
+WD_API size_t wd_state_bytes(const wd_model_dims* dims, int32_t batch, int32_t seq_len);
+/* Library version: major*10000 + minor*100 + patch. */
+WD_API int32_t wd_version(void);
+/* Static text for a status code. */
+WD_API const char* wd_status_string(wd_status s);
+
+/* ---- context ------------------------------------------------------------ */
+
+/* Build a context on the current CUDA device.  Validates dims (head_dim even,
+ * n_q_heads a multiple of n_kv_heads, bf16 needs d_model, d_ffn and
+ * n_q_heads*head_dim to be multiples of 64, ...), borrows weights and
+ * workspace, creates the TMA descriptors of the weights.
+ * Errors: WD_ERR_NULL, WD_ERR_INVALID_DIMS, WD_ERR_WORKSPACE_TOO_SMALL,
+ * WD_ERR_MISALIGNED, WD_ERR_UNSUPPORTED_ARCH, WD_ERR_CUDA. */
+WD_API wd_status wd_create(const wd_model_dims* dims, const wd_weights* weights,
+                    void* workspace /*device*/, size_t workspace_bytes, wd_ctx** out);
+/* Frees host objects only. */
+WD_API wd_status wd_destroy(wd_ctx* ctx);
+/* Choose the GEMM kernel used by later steps (default WD_GEMM_AUTO). */
+WD_API wd_status wd_set_gemm_impl(wd_ctx* ctx, int32_t impl);
+
+/* GEMM timing for benchmarks.  While enabled, wd_step brackets every GEMM launch
+ * (one launch covers all weight matrices that share an input: q/k/v, gate/up)
+ * with CUDA events on the step's stream and wd_step_sync adds up their device
+ * time and their algorithmic bytes (weights once + activations in + result
+ * out).  Enabling resets the totals.  Off by default; leave it off in runs
+ * whose step time is reported. */
+WD_API wd_status wd_profile_enable(wd_ctx* ctx, int32_t on);
+WD_API wd_status wd_profile_read(const wd_ctx* ctx, double* gemm_ms, double* gemm_bytes, int64_t* gemm_launches);
+
+/* ---- sequence state (Section 3.1: the fixed-length state x^(t)) ---------- */
+
+/* token_ids: host [batch, seq_len].  decoded: host [batch, seq_len] of 0/1, or
+ * NULL meaning decoded = (id != mask_id).  Decoded-ness is tracked by these
+ * flags afterwards, never by comparing ids with mask_id.  state_mem is device
+ * memory of wd_state_bytes(); its K/V cache part is not initialised (the first
+ * step is a refresh and writes every row it reads).  Copies ids to the device
+ * on the legacy default stream and waits for it.
+ * Errors: WD_ERR_NULL, WD_ERR_BAD_PARAM (batch/seq_len out of range),
+ * WD_ERR_WORKSPACE_TOO_SMALL, WD_ERR_CUDA. */
+WD_API wd_status wd_state_create(wd_ctx* ctx, int32_t batch, int32_t seq_len,
+                          const int32_t* token_ids, const uint8_t* decoded,
+                          void* state_mem /*device*/, size_t state_mem_bytes, wd_state** out);
+/* Start over with new ids/flags (same batch and seq_len): step counter 0, next
+ * step is a refresh.  The host->device copy of the ids is enqueued on `stream`. */
+WD_API wd_status wd_state_reset(wd_state* st, const int32_t* token_ids, const uint8_t* decoded,
+                         void* stream /*cudaStream_t*/);
+WD_API wd_status wd_state_destroy(wd_state* st);
+/* Host mirror of one sequence: any of the outputs may be NULL.
+ * token_ids/decoded/dec_step have seq_len entries; dec_step is the step at
+ * which a token was unmasked, INT32_MIN for tokens that were given. */
+WD_API wd_status wd_state_read(const wd_state* st, int32_t seq, int32_t* token_ids, uint8_t* decoded,
+                        int32_t* dec_step, int32_t* step_index, int32_t* steps_since_refresh);
+WD_API wd_status wd_debug_taps_set(wd_state* st, const wd_debug_taps* taps /*NULL = off*/);
+
+/* ---- the step ----------------------------------------------------------- */
+
+/* Preview of the index sets the next wd_step(st, A, B, R, T, ...) will use for
+ * sequence `seq`.  Pure host function, no GPU work, does not change the state.
+ *   A  size of the internal (active) window, >= 1
+ *   B  number of buffer tokens: the external window holds A+B undecoded tokens
+ *   R  phase length in steps: 1 refresh + (R-1) normal steps, >= 1
+ *   T  a token unmasked at step s is recomputed at steps s+1..s+T of the same
+ *      phase (the post-decode transient of Section 4.3), >= 0
+ * Errors: WD_ERR_NULL, WD_ERR_BAD_PARAM, WD_ERR_CAPACITY. */
+WD_API wd_status wd_plan(const wd_state* st, int32_t seq, int32_t A, int32_t B, int32_t R, int32_t T,
+                  wd_index_sets* out);
+
+/* The same planner on explicit state arrays (no wd_state, no GPU, usable in a
+ * process without a CUDA device): decoded[seq_len] 0/1 flags, dec_step[seq_len]
+ * (step at which a token was unmasked, INT32_MIN if it was given), step_index
+ * t, steps_since_refresh, and the external window stored at the last refresh
+ * (ext_window[n_ext_window], ascending; empty before the first step).
+ * Errors: as wd_plan, plus WD_ERR_BAD_PARAM for an index outside the sequence. */
+WD_API wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, int32_t seq_len,
+                      int32_t step_index, int32_t steps_since_refresh,
+                      const int32_t* ext_window, int32_t n_ext_window,
+                      int32_t A, int32_t B, int32_t R, int32_t T, wd_index_sets* out);
+
+/* Enqueue one step for every sequence of the state on `stream` and return
+ * without waiting.  k = tokens unmasked per sequence (at most the number of
+ * active tokens; 0 = compute only).  Needs max_active >= batch * A.  The step
+ * must be completed with wd_step_sync before the next wd_step, wd_plan or
+ * wd_state_read.  `info` may be NULL.
+ * Returns WD_OK, WD_DONE (nothing left to decode: nothing enqueued),
+ * WD_ERR_PENDING, WD_ERR_BAD_PARAM, WD_ERR_CAPACITY (a dims.max_* limit),
+ * WD_ERR_CUDA. */
+WD_API wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int32_t T, int32_t k,
+                  void* stream /*cudaStream_t*/, wd_step_info* info);
+
+/* Wait for the enqueued step, read its result and the device status word,
+ * apply the update set to the host mirror of the state and advance the phase
+ * counters.  `out` (host) may be NULL.  Returns WD_OK, WD_ERR_NOT_PENDING,
+ * WD_ERR_DEVICE_TIMEOUT, WD_ERR_BOUNDS, WD_ERR_CUDA. */
+WD_API wd_status wd_step_sync(wd_state* st, wd_step_out* out);
+
+/* ---- single operations (unit parity tests, micro-benchmarks) -------------- */
+
+/* y[rows, n_out] (float, device) = x[rows, k_in] * w[n_out, k_in]^T, x and w of
+ * `dtype`, fp32 accumulation.  `scratch` (device, scratch_bytes) holds split-K
+ * partial sums for WD_GEMM_TCGEN05 (wd_op_gemm_scratch_bytes); unused for
+ * WD_GEMM_PLAIN.  Section 3.1's transformer forward is made of these.
+ * Errors: WD_ERR_NULL, WD_ERR_BAD_PARAM, WD_ERR_WORKSPACE_TOO_SMALL, WD_ERR_CUDA,
+ * WD_ERR_DEVICE_TIMEOUT (only after the caller synchronises: see wd_op_status). */
+WD_API wd_status wd_op_gemm(int32_t dtype, int32_t impl, const void* x, const void* w, float* y,
+                     int32_t rows, int32_t n_out, int32_t k_in,
+                     void* scratch, size_t scratch_bytes, void* stream);
+WD_API size_t wd_op_gemm_scratch_bytes(int32_t rows, int32_t n_out, int32_t k_in);
+
+/* Bidirectional grouped-query attention (Section 3.1: no causal mask) of
+ * n_rows query rows over n_vis cached positions of one sequence:
+ * out[r, h, :] = softmax_j(q[r,h,:] . K[kvh(h), vis[j], :] / sqrt(head_dim)) V[kvh(h), vis[j], :].
+ * q, out: [n_rows, n_q_heads, head_dim]; kcache, vcache: [n_kv_heads, seq_len, head_dim];
+ * vis: device int32 [n_vis], all of `dtype`. */
+WD_API wd_status wd_op_attention(int32_t dtype, const void* q, const void* kcache, const void* vcache,
+                          const int32_t* vis, void* out, int32_t n_rows, int32_t n_vis,
+                          int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t seq_len,
+                          void* stream);
+
+/* The unmask rule on given logits (device float [n, vocab]) of one sequence:
+ * token = lowest index of the maximal logit, confidence = its softmax
+ * probability; the min(k, n) rows of highest confidence are returned (equal
+ * confidence: lowest position).  positions: device int32 [n] ascending.
+ * Outputs are device arrays: row_token[n], row_sumexp[n] (sum_v exp(logit_v - max),
+ * the reciprocal of the confidence), row_conf[n], sel_pos[k], sel_token[k],
+ * sel_conf[k], n_sel[1]; none of them may overlap. */
+WD_API wd_status wd_op_unmask(const float* logits, const int32_t* positions, int32_t n, int32_t vocab,
+                       int32_t k, int32_t* row_token, float* row_sumexp, float* row_conf,
+                       int32_t* sel_pos, int32_t* sel_token, float* sel_conf, int32_t* n_sel,
+                       void* stream);
+
+/* Device status word shared by the single operations: 0, or the first
+ * WD_ERR_DEVICE_TIMEOUT / WD_ERR_BOUNDS raised by a kernel since the last
+ * call.  Synchronises the device. */
+WD_API wd_status wd_op_status(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WD_H */

@@ -1,0 +1,745 @@
+// C ABI of libwd.so: context, sequence state, the step driver and the single
+// operations.  Host code; every step of the path runs in the kernels it launches.
+#include <algorithm>
+#include <climits>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "wd_internal.h"
+#include "gemm_tc.h"
+
+// ---------------------------------------------------------------------------
+// error bookkeeping
+// ---------------------------------------------------------------------------
+static thread_local char g_last_cuda_error[256];
+
+void wd_note_cuda_error(cudaError_t e, const char* file, int line) {
+    snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "%s at %s:%d", cudaGetErrorString(e), file, line);
+    cudaGetLastError();   // clear the sticky-less error so later calls report their own
+}
+
+extern "C" const char* wd_status_string(wd_status s) {
+    switch (s) {
+        case WD_OK: return "ok";
+        case WD_DONE: return "done: no undecoded token left";
+        case WD_ERR_NULL: return "null pointer";
+        case WD_ERR_INVALID_DIMS: return "invalid model dims";
+        case WD_ERR_WORKSPACE_TOO_SMALL: return "workspace too small";
+        case WD_ERR_UNSUPPORTED_ARCH: return "device is not sm_100";
+        case WD_ERR_BAD_PARAM: return "bad parameter";
+        case WD_ERR_CAPACITY: return "capacity exceeded";
+        case WD_ERR_PENDING: return "a step is pending: call wd_step_sync first";
+        case WD_ERR_CUDA: return g_last_cuda_error[0] ? g_last_cuda_error : "CUDA error";
+        case WD_ERR_DEVICE_TIMEOUT: return "a bounded device-side wait ran out";
+        case WD_ERR_BOUNDS: return "a device-side index check failed";
+        case WD_ERR_NOT_PENDING: return "no step pending";
+        case WD_ERR_MISALIGNED: return "device pointer not 256-byte aligned";
+        default: return "unknown status";
+    }
+}
+
+extern "C" int32_t wd_version(void) { return 100; }
+
+// ---------------------------------------------------------------------------
+// context
+// ---------------------------------------------------------------------------
+struct wd_ctx {
+    wd_model_dims d;
+    const void* tok_embed;
+    const void* lm_head;
+    const float* final_norm;
+    std::vector<const void*> wq, wk, wv, wo, wg, wu, wd;
+    std::vector<const float*> attn_norm, ffn_norm;
+    int gemm_impl = WD_GEMM_AUTO;
+    int sm_count = 148;
+
+    // workspace carve-up (device)
+    float* x = nullptr;          // [max_rows, d] residual stream
+    void* xn = nullptr;          // [max_rows, d] normalised rows (model dtype)
+    void* q = nullptr;           // [max_rows, Hq*dh]
+    void* attn = nullptr;        // [max_rows, Hq*dh]
+    void* h = nullptr;           // [max_rows, F]
+    float* part = nullptr;       // split-K partial sums / GEMM outputs
+    size_t part_floats = 0;
+    float* logits = nullptr;     // [max_active, V]
+    int32_t* row_token = nullptr;
+    float* row_sumexp = nullptr;
+    float* row_conf = nullptr;
+    int32_t* plan = nullptr;     // packed index lists of the step
+    size_t plan_ints = 0;
+    int32_t* result = nullptr;   // [status | n_sel[batch] | pos | tok | conf]
+    size_t result_ints = 0;
+
+    WdTcWeights tc;              // tensor maps of the weights (bf16 only)
+
+    // optional GEMM timing (benchmarks): event pairs around every GEMM launch of a step
+    bool prof_on = false;
+    std::vector<cudaEvent_t> prof_events;
+    size_t prof_used = 0;
+    double prof_step_bytes = 0.0, prof_ms = 0.0, prof_bytes = 0.0;
+    long long prof_launches = 0;
+    ~wd_ctx() { for (cudaEvent_t e : prof_events) cudaEventDestroy(e); }
+};
+
+static bool dims_valid(const wd_model_dims* d) {
+    if (!d) return false;
+    if (d->n_layers < 1 || d->d_model < 1 || d->n_q_heads < 1 || d->n_kv_heads < 1 || d->head_dim < 2 ||
+        d->d_ffn < 1 || d->vocab < 2)
+        return false;
+    if (d->head_dim % 2 || d->n_q_heads % d->n_kv_heads) return false;
+    if (d->dtype != WD_F32 && d->dtype != WD_BF16) return false;
+    if (d->mask_id < 0 || d->mask_id >= d->vocab) return false;
+    if (d->max_batch < 1 || d->max_seq < 1 || d->max_rows < 1 || d->max_active < 1) return false;
+    if ((int64_t)d->max_rows > (int64_t)d->max_batch * d->max_seq) return false;
+    if (d->max_active > d->max_rows) return false;
+    if (!(d->rope_theta > 1.f) || !(d->rms_eps >= 0.f)) return false;
+    if (d->dtype == WD_BF16) {
+        // TMA tiles are 64 elements (128 bytes) along the reduction dimension
+        if (d->d_model % 64 || d->d_ffn % 64 || (d->n_q_heads * d->head_dim) % 64) return false;
+    }
+    return true;
+}
+
+struct Carve {
+    size_t off = 0;
+    size_t take(size_t bytes) { size_t o = off; off = wd_align_up(off + bytes, 256); return o; }
+};
+
+static size_t max_gemm_cols(const wd_model_dims* d) {
+    const size_t qkv = (size_t)(d->n_q_heads + 2 * d->n_kv_heads) * d->head_dim;
+    return std::max({qkv, (size_t)d->d_model, (size_t)2 * d->d_ffn});
+}
+
+// partial-sum buffer: split-K is only used while rows are few
+static size_t part_floats_for(const wd_model_dims* d) {
+    const size_t cols = max_gemm_cols(d);
+    const size_t small_rows = std::min<size_t>(d->max_rows, WD_TC_SPLITK_MAX_ROWS);
+    return std::max((size_t)d->max_rows * cols, (size_t)WD_TC_MAX_SPLIT * small_rows * cols);
+}
+
+static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[16]) {
+    const size_t e = wd_elt_size(d->dtype);
+    const size_t MR = d->max_rows, MA = d->max_active, hq = (size_t)d->n_q_heads * d->head_dim;
+    off[0] = c.take(MR * d->d_model * 4);                       // x
+    off[1] = c.take(MR * d->d_model * e);                       // xn
+    off[2] = c.take(MR * hq * e);                               // q
+    off[3] = c.take(MR * hq * e);                               // attn
+    off[4] = c.take(MR * d->d_ffn * e);                         // h
+    off[5] = c.take(part_floats_for(d) * 4);                    // part
+    off[6] = c.take(MA * d->vocab * 4);                         // logits
+    off[7] = c.take(MA * 4);                                    // row_token
+    off[8] = c.take(MA * 4);                                    // row_sumexp
+    off[9] = c.take(MA * 4);                                    // row_conf
+    const size_t plan_ints = 2 * MR + 2 * MA + 2 * ((size_t)d->max_batch + 1) + (size_t)d->max_batch * d->max_seq;
+    off[10] = c.take(plan_ints * 4);                            // plan
+    off[11] = c.take((1 + (size_t)d->max_batch + 3 * MA) * 4);  // result
+    off[12] = plan_ints;
+}
+
+extern "C" size_t wd_workspace_bytes(const wd_model_dims* dims) {
+    if (!dims_valid(dims)) return 0;
+    Carve c;
+    size_t off[16];
+    carve_ctx(dims, c, off);
+    return c.off;
+}
+
+extern "C" size_t wd_state_bytes(const wd_model_dims* d, int32_t batch, int32_t seq_len) {
+    if (!dims_valid(d) || batch < 1 || seq_len < 1 || batch > d->max_batch || seq_len > d->max_seq) return 0;
+    const size_t kv = (size_t)d->n_layers * batch * d->n_kv_heads * seq_len * d->head_dim * wd_elt_size(d->dtype);
+    return wd_align_up((size_t)batch * seq_len * 4, 256) + 2 * wd_align_up(kv, 256);
+}
+
+extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, void* workspace,
+                               size_t workspace_bytes, wd_ctx** out) {
+    if (!dims || !w || !workspace || !out) return WD_ERR_NULL;
+    *out = nullptr;
+    if (!dims_valid(dims)) return WD_ERR_INVALID_DIMS;
+    if (!w->tok_embed || !w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate || !w->w_up || !w->w_down ||
+        !w->attn_norm || !w->ffn_norm || !w->final_norm || !w->lm_head)
+        return WD_ERR_NULL;
+    for (int l = 0; l < dims->n_layers; ++l)
+        if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->w_gate[l] || !w->w_up[l] || !w->w_down[l] ||
+            !w->attn_norm[l] || !w->ffn_norm[l])
+            return WD_ERR_NULL;
+    if ((uintptr_t)workspace % 256) return WD_ERR_MISALIGNED;
+    if (workspace_bytes < wd_workspace_bytes(dims)) return WD_ERR_WORKSPACE_TOO_SMALL;
+
+    int dev = 0;
+    cudaDeviceProp prop;
+    WD_CUDA_TRY(cudaGetDevice(&dev));
+    WD_CUDA_TRY(cudaGetDeviceProperties(&prop, dev));
+    if (prop.major != 10) return WD_ERR_UNSUPPORTED_ARCH;
+
+    wd_ctx* c = new (std::nothrow) wd_ctx();
+    if (!c) return WD_ERR_CUDA;
+    c->d = *dims;
+    c->sm_count = prop.multiProcessorCount;
+    c->tok_embed = w->tok_embed;
+    c->lm_head = w->lm_head;
+    c->final_norm = w->final_norm;
+    for (int l = 0; l < dims->n_layers; ++l) {
+        c->wq.push_back(w->wq[l]); c->wk.push_back(w->wk[l]); c->wv.push_back(w->wv[l]);
+        c->wo.push_back(w->wo[l]); c->wg.push_back(w->w_gate[l]); c->wu.push_back(w->w_up[l]);
+        c->wd.push_back(w->w_down[l]);
+        c->attn_norm.push_back(w->attn_norm[l]); c->ffn_norm.push_back(w->ffn_norm[l]);
+    }
+    Carve cv;
+    size_t off[16];
+    carve_ctx(dims, cv, off);
+    char* base = (char*)workspace;
+    c->x = (float*)(base + off[0]);
+    c->xn = base + off[1];
+    c->q = base + off[2];
+    c->attn = base + off[3];
+    c->h = base + off[4];
+    c->part = (float*)(base + off[5]);
+    c->part_floats = part_floats_for(dims);
+    c->logits = (float*)(base + off[6]);
+    c->row_token = (int32_t*)(base + off[7]);
+    c->row_sumexp = (float*)(base + off[8]);
+    c->row_conf = (float*)(base + off[9]);
+    c->plan = (int32_t*)(base + off[10]);
+    c->plan_ints = off[12];
+    c->result = (int32_t*)(base + off[11]);
+    c->result_ints = 1 + (size_t)dims->max_batch + 3 * (size_t)dims->max_active;
+    WD_CUDA_TRY(cudaMemset(c->result, 0, 4));
+
+    if (dims->dtype == WD_BF16) {
+        wd_status s = wd_tc_weights_init(&c->tc, dims, c->tok_embed, c->lm_head, c->wq, c->wk, c->wv, c->wo,
+                                         c->wg, c->wu, c->wd, c->xn, c->attn, c->h);
+        if (s != WD_OK) { delete c; return s; }
+    }
+    *out = c;
+    return WD_OK;
+}
+
+extern "C" wd_status wd_destroy(wd_ctx* ctx) {
+    if (!ctx) return WD_ERR_NULL;
+    delete ctx;
+    return WD_OK;
+}
+
+extern "C" wd_status wd_set_gemm_impl(wd_ctx* ctx, int32_t impl) {
+    if (!ctx) return WD_ERR_NULL;
+    if (impl != WD_GEMM_AUTO && impl != WD_GEMM_PLAIN && impl != WD_GEMM_TCGEN05) return WD_ERR_BAD_PARAM;
+    if (impl == WD_GEMM_TCGEN05 && ctx->d.dtype != WD_BF16) return WD_ERR_BAD_PARAM;
+    ctx->gemm_impl = impl;
+    return WD_OK;
+}
+
+extern "C" wd_status wd_profile_enable(wd_ctx* ctx, int32_t on) {
+    if (!ctx) return WD_ERR_NULL;
+    ctx->prof_on = on != 0;
+    ctx->prof_ms = 0.0; ctx->prof_bytes = 0.0; ctx->prof_launches = 0;
+    return WD_OK;
+}
+
+extern "C" wd_status wd_profile_read(const wd_ctx* ctx, double* gemm_ms, double* gemm_bytes, int64_t* gemm_launches) {
+    if (!ctx) return WD_ERR_NULL;
+    if (gemm_ms) *gemm_ms = ctx->prof_ms;
+    if (gemm_bytes) *gemm_bytes = ctx->prof_bytes;
+    if (gemm_launches) *gemm_launches = ctx->prof_launches;
+    return WD_OK;
+}
+
+// ---------------------------------------------------------------------------
+// state
+// ---------------------------------------------------------------------------
+struct wd_state {
+    wd_ctx* ctx = nullptr;
+    int batch = 0, S = 0;
+    std::vector<WdSeq> seqs;
+    std::vector<WdSeqPlan> plans;       // of the pending step
+    int32_t* ids_dev = nullptr;
+    char* kcache = nullptr;             // [L][batch][Hkv][S][dh]
+    char* vcache = nullptr;
+    size_t kv_layer_bytes = 0;
+    int32_t* plan_host = nullptr;       // pinned
+    int32_t* result_host = nullptr;     // pinned
+    int32_t* ids_host = nullptr;        // pinned staging for ids
+    cudaEvent_t done = nullptr;
+    bool pending = false;
+    int k_pending = 0, k_user = 0;
+    wd_debug_taps taps = {nullptr, nullptr, nullptr};
+};
+
+static void load_host_mirror(wd_state* st, const int32_t* ids, const uint8_t* decoded) {
+    const int mask_id = st->ctx->d.mask_id;
+    for (int b = 0; b < st->batch; ++b) {
+        WdSeq& s = st->seqs[b];
+        s.ids.assign(ids + (size_t)b * st->S, ids + (size_t)(b + 1) * st->S);
+        s.decoded.resize(st->S);
+        for (int i = 0; i < st->S; ++i)
+            s.decoded[i] = decoded ? (decoded[(size_t)b * st->S + i] ? 1 : 0) : (s.ids[i] != mask_id ? 1 : 0);
+        s.dec_step.assign(st->S, INT32_MIN);
+        s.wex.clear();
+        s.t = 0; s.since = 0; s.phase_start = 0;
+    }
+    memcpy(st->ids_host, ids, (size_t)st->batch * st->S * 4);
+}
+
+extern "C" wd_status wd_state_create(wd_ctx* ctx, int32_t batch, int32_t seq_len, const int32_t* token_ids,
+                                     const uint8_t* decoded, void* state_mem, size_t state_mem_bytes,
+                                     wd_state** out) {
+    if (!ctx || !token_ids || !state_mem || !out) return WD_ERR_NULL;
+    *out = nullptr;
+    if (batch < 1 || seq_len < 1 || batch > ctx->d.max_batch || seq_len > ctx->d.max_seq) return WD_ERR_BAD_PARAM;
+    if ((uintptr_t)state_mem % 256) return WD_ERR_MISALIGNED;
+    const size_t need = wd_state_bytes(&ctx->d, batch, seq_len);
+    if (state_mem_bytes < need) return WD_ERR_WORKSPACE_TOO_SMALL;
+    for (size_t i = 0; i < (size_t)batch * seq_len; ++i)
+        if (token_ids[i] < 0 || token_ids[i] >= ctx->d.vocab) return WD_ERR_BAD_PARAM;
+
+    wd_state* st = new (std::nothrow) wd_state();
+    if (!st) return WD_ERR_CUDA;
+    st->ctx = ctx; st->batch = batch; st->S = seq_len;
+    st->seqs.resize(batch);
+    const wd_model_dims& d = ctx->d;
+    const size_t ids_bytes = wd_align_up((size_t)batch * seq_len * 4, 256);
+    st->kv_layer_bytes = (size_t)batch * d.n_kv_heads * seq_len * d.head_dim * wd_elt_size(d.dtype);
+    const size_t kv = wd_align_up(st->kv_layer_bytes * d.n_layers, 256);
+    st->ids_dev = (int32_t*)state_mem;
+    st->kcache = (char*)state_mem + ids_bytes;
+    st->vcache = st->kcache + kv;
+    cudaError_t e;
+    if ((e = cudaHostAlloc((void**)&st->plan_host, ctx->plan_ints * 4, cudaHostAllocDefault)) != cudaSuccess ||
+        (e = cudaHostAlloc((void**)&st->result_host, ctx->result_ints * 4, cudaHostAllocDefault)) != cudaSuccess ||
+        (e = cudaHostAlloc((void**)&st->ids_host, (size_t)batch * seq_len * 4, cudaHostAllocDefault)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&st->done, cudaEventDisableTiming)) != cudaSuccess) {
+        wd_note_cuda_error(e, __FILE__, __LINE__);
+        wd_state_destroy(st);
+        return WD_ERR_CUDA;
+    }
+    load_host_mirror(st, token_ids, decoded);
+    e = cudaMemcpy(st->ids_dev, st->ids_host, (size_t)batch * seq_len * 4, cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) { wd_note_cuda_error(e, __FILE__, __LINE__); wd_state_destroy(st); return WD_ERR_CUDA; }
+    *out = st;
+    return WD_OK;
+}
+
+extern "C" wd_status wd_state_reset(wd_state* st, const int32_t* token_ids, const uint8_t* decoded, void* stream) {
+    if (!st || !token_ids) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    for (size_t i = 0; i < (size_t)st->batch * st->S; ++i)
+        if (token_ids[i] < 0 || token_ids[i] >= st->ctx->d.vocab) return WD_ERR_BAD_PARAM;
+    load_host_mirror(st, token_ids, decoded);
+    WD_CUDA_TRY(cudaMemcpyAsync(st->ids_dev, st->ids_host, (size_t)st->batch * st->S * 4, cudaMemcpyHostToDevice,
+                                (cudaStream_t)stream));
+    return WD_OK;
+}
+
+extern "C" wd_status wd_state_destroy(wd_state* st) {
+    if (!st) return WD_ERR_NULL;
+    if (st->pending && st->done) cudaEventSynchronize(st->done);
+    if (st->plan_host) cudaFreeHost(st->plan_host);
+    if (st->result_host) cudaFreeHost(st->result_host);
+    if (st->ids_host) cudaFreeHost(st->ids_host);
+    if (st->done) cudaEventDestroy(st->done);
+    delete st;
+    return WD_OK;
+}
+
+extern "C" wd_status wd_state_read(const wd_state* st, int32_t seq, int32_t* token_ids, uint8_t* decoded,
+                                   int32_t* dec_step, int32_t* step_index, int32_t* steps_since_refresh) {
+    if (!st) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    if (seq < 0 || seq >= st->batch) return WD_ERR_BAD_PARAM;
+    const WdSeq& s = st->seqs[seq];
+    if (token_ids) memcpy(token_ids, s.ids.data(), (size_t)st->S * 4);
+    if (decoded) memcpy(decoded, s.decoded.data(), (size_t)st->S);
+    if (dec_step) memcpy(dec_step, s.dec_step.data(), (size_t)st->S * 4);
+    if (step_index) *step_index = s.t;
+    if (steps_since_refresh) *steps_since_refresh = s.since;
+    return WD_OK;
+}
+
+extern "C" wd_status wd_debug_taps_set(wd_state* st, const wd_debug_taps* taps) {
+    if (!st) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    if (taps) st->taps = *taps;
+    else st->taps = {nullptr, nullptr, nullptr};
+    return WD_OK;
+}
+
+// ---------------------------------------------------------------------------
+// wd_plan
+// ---------------------------------------------------------------------------
+static wd_status copy_list(const std::vector<int32_t>& v, int32_t* dst, int32_t* n, int32_t cap) {
+    *n = (int32_t)v.size();
+    if ((int32_t)v.size() > cap) return WD_ERR_CAPACITY;
+    if (!v.empty()) {
+        if (!dst) return WD_ERR_NULL;
+        memcpy(dst, v.data(), v.size() * 4);
+    }
+    return WD_OK;
+}
+
+static wd_status export_plan(const WdSeqPlan& p, wd_index_sets* out);
+
+extern "C" wd_status wd_plan(const wd_state* st, int32_t seq, int32_t A, int32_t B, int32_t R, int32_t T,
+                             wd_index_sets* out) {
+    if (!st || !out) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    if (seq < 0 || seq >= st->batch) return WD_ERR_BAD_PARAM;
+    WdSeqPlan p;
+    wd_status s = wd_plan_seq(st->seqs[seq], A, B, R, T, &p);
+    if (s != WD_OK) return s;
+    return export_plan(p, out);
+}
+
+extern "C" wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, int32_t seq_len, int32_t step_index,
+                                 int32_t steps_since_refresh, const int32_t* ext_window, int32_t n_ext_window,
+                                 int32_t A, int32_t B, int32_t R, int32_t T, wd_index_sets* out) {
+    if (!decoded || !dec_step || !out || (n_ext_window > 0 && !ext_window)) return WD_ERR_NULL;
+    if (seq_len < 1 || n_ext_window < 0 || step_index < 0 || steps_since_refresh < 0) return WD_ERR_BAD_PARAM;
+    WdSeq s;
+    s.ids.assign(seq_len, 0);
+    s.decoded.assign(decoded, decoded + seq_len);
+    s.dec_step.assign(dec_step, dec_step + seq_len);
+    for (int32_t i = 0; i < n_ext_window; ++i) {
+        if (ext_window[i] < 0 || ext_window[i] >= seq_len) return WD_ERR_BAD_PARAM;
+        s.wex.push_back(ext_window[i]);
+    }
+    s.t = step_index;
+    s.since = steps_since_refresh;
+    WdSeqPlan p;
+    wd_status r = wd_plan_seq(s, A, B, R, T, &p);
+    if (r != WD_OK) return r;
+    return export_plan(p, out);
+}
+
+static wd_status export_plan(const WdSeqPlan& p, wd_index_sets* out) {
+    out->done = p.done ? 1 : 0;
+    out->is_refresh = p.refresh ? 1 : 0;
+    out->vis_contiguous = p.vis_contiguous ? 1 : 0;
+    wd_status worst = WD_OK, r;
+    const int32_t cap = out->capacity;
+    if ((r = copy_list(p.active, out->active, &out->n_active, cap)) != WD_OK) worst = r;
+    if ((r = copy_list(p.buffer, out->buffer, &out->n_buffer, cap)) != WD_OK) worst = r;
+    if ((r = copy_list(p.decoded, out->decoded, &out->n_decoded, cap)) != WD_OK) worst = r;
+    if ((r = copy_list(p.transient, out->transient, &out->n_transient, cap)) != WD_OK) worst = r;
+    if ((r = copy_list(p.far_field, out->far_field, &out->n_far_field, cap)) != WD_OK) worst = r;
+    if ((r = copy_list(p.rows, out->rows, &out->n_rows, cap)) != WD_OK) worst = r;
+    if ((r = copy_list(p.vis, out->vis, &out->n_vis, cap)) != WD_OK) worst = r;
+    if ((r = copy_list(p.wex, out->ext_window, &out->n_ext_window, cap)) != WD_OK) worst = r;
+    return worst;
+}
+
+// ---------------------------------------------------------------------------
+// GEMM dispatch: y[rows, sum n_i] = x[rows, K] * [w_0; w_1; ...]^T into ctx->part
+// ---------------------------------------------------------------------------
+struct GemmOut { int n_split; size_t split_stride; int launches; int impl; };
+
+static bool use_tc(const wd_ctx* c) {
+    if (c->d.dtype != WD_BF16) return false;
+    return c->gemm_impl != WD_GEMM_PLAIN;
+}
+
+static wd_status run_gemm(wd_ctx* c, const void* x, const WdTcX* x_map, const WdTcSeg* segs, int nseg,
+                          int rows, int K, float* y, size_t y_floats, int32_t* status, cudaStream_t stream,
+                          GemmOut* go, bool single_split = false, bool force_tc = false) {
+    int ncol = 0;
+    for (int i = 0; i < nseg; ++i) ncol += segs[i].n;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (c->prof_on) {
+        while (c->prof_events.size() < c->prof_used + 2) {
+            cudaEvent_t e;
+            WD_CUDA_TRY(cudaEventCreate(&e));
+            c->prof_events.push_back(e);
+        }
+        e0 = c->prof_events[c->prof_used++];
+        e1 = c->prof_events[c->prof_used++];
+        // algorithmic bytes: weights once, activations in, result out
+        c->prof_step_bytes += (double)ncol * K * wd_elt_size(c->d.dtype) + (double)rows * K * wd_elt_size(c->d.dtype) +
+                              (double)rows * ncol * 4;
+        WD_CUDA_TRY(cudaEventRecord(e0, stream));
+    }
+    if (use_tc(c) || force_tc) {
+        int n_split = 1;
+        wd_status s = wd_tc_gemm(x_map, segs, nseg, rows, K, y, y_floats, c->sm_count, status, stream, &n_split,
+                                 single_split);
+        if (s != WD_OK) return s;
+        *go = {n_split, (size_t)rows * ncol, 1, WD_GEMM_TCGEN05};
+    } else {
+        if ((size_t)rows * ncol > y_floats) return WD_ERR_CAPACITY;
+        int col = 0;
+        for (int i = 0; i < nseg; ++i) {
+            wd_launch_gemm_plain(c->d.dtype, x, segs[i].w, y + col, rows, segs[i].n, K, ncol, stream);
+            col += segs[i].n;
+        }
+        *go = {1, (size_t)rows * ncol, nseg, WD_GEMM_PLAIN};
+    }
+    if (e1) WD_CUDA_TRY(cudaEventRecord(e1, stream));
+    return WD_OK;
+}
+
+// ---------------------------------------------------------------------------
+// wd_step
+// ---------------------------------------------------------------------------
+extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int32_t T, int32_t k, void* stream_,
+                             wd_step_info* info) {
+    if (!st) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    if (A < 1 || B < 0 || R < 1 || T < 0 || k < 0) return WD_ERR_BAD_PARAM;
+    wd_ctx* c = st->ctx;
+    const wd_model_dims& d = c->d;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const int batch = st->batch, S = st->S;
+
+    st->plans.assign(batch, WdSeqPlan());
+    bool all_done = true, any_refresh = false, all_contig = true;
+    size_t n_rows = 0, n_act = 0, n_vis = 0;
+    int max_vis = 0;
+    for (int b = 0; b < batch; ++b) {
+        wd_status s = wd_plan_seq(st->seqs[b], A, B, R, T, &st->plans[b]);
+        if (s != WD_OK) return s;
+        const WdSeqPlan& p = st->plans[b];
+        if (p.done) continue;
+        all_done = false;
+        any_refresh |= p.refresh;
+        all_contig &= p.vis_contiguous;
+        n_rows += p.rows.size(); n_act += p.active.size(); n_vis += p.vis.size();
+        max_vis = std::max(max_vis, (int)p.vis.size());
+    }
+    if (all_done) return WD_DONE;
+    const int k_eff = std::min<int64_t>(k, A);
+    if (n_rows > (size_t)d.max_rows || n_act > (size_t)d.max_active ||
+        (size_t)batch * std::max(k_eff, 1) > (size_t)d.max_active)
+        return WD_ERR_CAPACITY;
+
+    // ---- pack the index lists and send them in one copy
+    int32_t* ph = st->plan_host;
+    size_t o = 0;
+    const size_t o_row_seq = o; o += n_rows;
+    const size_t o_row_pos = o; o += n_rows;
+    const size_t o_act_row = o; o += n_act;
+    const size_t o_act_pos = o; o += n_act;
+    const size_t o_act_off = o; o += batch + 1;
+    const size_t o_vis_off = o; o += batch + 1;
+    const size_t o_vis_idx = o; o += n_vis;
+    if (o > c->plan_ints) return WD_ERR_CAPACITY;
+    {
+        size_t r = 0, a = 0, v = 0;
+        for (int b = 0; b < batch; ++b) {
+            const WdSeqPlan& p = st->plans[b];
+            ph[o_act_off + b] = (int32_t)a;
+            ph[o_vis_off + b] = (int32_t)v;
+            if (p.done) continue;
+            size_t ai = 0;
+            for (size_t i = 0; i < p.rows.size(); ++i) {
+                ph[o_row_seq + r] = b;
+                ph[o_row_pos + r] = p.rows[i];
+                if (ai < p.active.size() && p.active[ai] == p.rows[i]) {
+                    ph[o_act_row + a] = (int32_t)r;
+                    ph[o_act_pos + a] = p.rows[i];
+                    ++a; ++ai;
+                }
+                ++r;
+            }
+            memcpy(ph + o_vis_idx + v, p.vis.data(), p.vis.size() * 4);
+            v += p.vis.size();
+        }
+        ph[o_act_off + batch] = (int32_t)a;
+        ph[o_vis_off + batch] = (int32_t)v;
+    }
+    WD_CUDA_TRY(cudaMemcpyAsync(c->plan, ph, o * 4, cudaMemcpyHostToDevice, stream));
+    const int32_t* row_seq = c->plan + o_row_seq;
+    const int32_t* row_pos = c->plan + o_row_pos;
+    const int32_t* act_row = c->plan + o_act_row;
+    const int32_t* act_pos = c->plan + o_act_pos;
+    const int32_t* act_off = c->plan + o_act_off;
+    const int32_t* vis_off = c->plan + o_vis_off;
+    const int32_t* vis_idx = c->plan + o_vis_idx;
+    int32_t* status = c->result;
+
+    const int R_ = (int)n_rows, NA = (int)n_act;
+    const int Hq = d.n_q_heads, Hkv = d.n_kv_heads, dh = d.head_dim, D = d.d_model, F = d.d_ffn;
+    const int hq = Hq * dh, hkv = Hkv * dh;
+    const long long launches0 = wd_launch_counter;
+    int impl_used = WD_GEMM_PLAIN;
+    c->prof_used = 0;
+    c->prof_step_bytes = 0.0;
+    GemmOut go;
+    wd_status s;
+
+    wd_launch_embed(d.dtype, c->tok_embed, st->ids_dev, row_seq, row_pos, c->x, R_, D, S, d.vocab, status, stream);
+    bool down_pending = false;          // x still lacks the previous block's FFN output
+    GemmOut down_go = {1, 0, 0, 0};
+    for (int l = 0; l < d.n_layers; ++l) {
+        char* kc = st->kcache + (size_t)l * st->kv_layer_bytes;
+        char* vc = st->vcache + (size_t)l * st->kv_layer_bytes;
+        // attention half
+        wd_launch_rmsnorm(d.dtype, c->x, down_pending ? c->part : nullptr, down_go.n_split, down_go.split_stride,
+                          c->attn_norm[l], d.rms_eps, c->xn, nullptr, R_, D, stream);
+        down_pending = false;
+        WdTcSeg qkv[3] = {{c->wq[l], hq, c->tc.get(WD_TC_WQ, l)}, {c->wk[l], hkv, c->tc.get(WD_TC_WK, l)},
+                          {c->wv[l], hkv, c->tc.get(WD_TC_WV, l)}};
+        if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, qkv, 3, R_, D, c->part, c->part_floats, status, stream, &go)) != WD_OK)
+            return s;
+        impl_used = go.impl;
+        wd_launch_rope_scatter(d.dtype, c->part, go.n_split, go.split_stride, row_seq, row_pos, c->q, kc, vc, R_, Hq,
+                               Hkv, dh, S, d.rope_theta, stream);
+        float* attn_tap = st->taps.attn_out ? st->taps.attn_out + (size_t)l * R_ * hq : nullptr;
+        wd_launch_attention_plain(d.dtype, c->q, kc, vc, row_seq, vis_idx, vis_off, c->attn, attn_tap, R_, max_vis,
+                                  Hq, Hkv, dh, S, stream);
+        WdTcSeg wo[1] = {{c->wo[l], D, c->tc.get(WD_TC_WO, l)}};
+        if ((s = run_gemm(c, c->attn, &c->tc.x_map_attn, wo, 1, R_, hq, c->part, c->part_floats, status, stream, &go)) != WD_OK)
+            return s;
+        // feed-forward half
+        wd_launch_rmsnorm(d.dtype, c->x, c->part, go.n_split, go.split_stride, c->ffn_norm[l], d.rms_eps, c->xn,
+                          nullptr, R_, D, stream);
+        WdTcSeg gu[2] = {{c->wg[l], F, c->tc.get(WD_TC_WG, l)}, {c->wu[l], F, c->tc.get(WD_TC_WU, l)}};
+        if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, gu, 2, R_, D, c->part, c->part_floats, status, stream, &go)) != WD_OK)
+            return s;
+        wd_launch_swiglu(d.dtype, c->part, go.n_split, go.split_stride, c->h, R_, F, stream);
+        WdTcSeg wdn[1] = {{c->wd[l], D, c->tc.get(WD_TC_WD, l)}};
+        if ((s = run_gemm(c, c->h, &c->tc.x_map_h, wdn, 1, R_, F, c->part, c->part_floats, status, stream, &go)) != WD_OK)
+            return s;
+        if (st->taps.layer_out || l == d.n_layers - 1) {
+            float* tap = st->taps.layer_out ? st->taps.layer_out + (size_t)l * R_ * D : nullptr;
+            wd_launch_residual_add(c->x, c->part, go.n_split, go.split_stride, tap, R_, D, stream);
+        } else {
+            down_pending = true;     // folded into the next block's RMSNorm
+            down_go = go;
+        }
+    }
+    // logits for the active rows only, then the unmask reduction
+    if (NA > 0) {
+        wd_launch_rmsnorm(d.dtype, c->x, nullptr, 0, 0, c->final_norm, d.rms_eps, c->xn, act_row, NA, D, stream);
+        WdTcSeg lm[1] = {{c->lm_head, d.vocab, c->tc.get(WD_TC_LM, 0)}};
+        if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, lm, 1, NA, D, c->logits, (size_t)d.max_active * d.vocab, status,
+                          stream, &go, /*single_split=*/true)) != WD_OK)
+            return s;
+        wd_launch_rowstats(c->logits, NA, d.vocab, c->row_token, c->row_sumexp, stream);
+        if (st->taps.logits)
+            WD_CUDA_TRY(cudaMemcpyAsync(st->taps.logits, c->logits, (size_t)NA * d.vocab * 4, cudaMemcpyDeviceToDevice,
+                                        stream));
+    }
+    int32_t* n_sel = c->result + 1;
+    int32_t* sel_pos = n_sel + batch;
+    int32_t* sel_tok = sel_pos + (size_t)batch * std::max(k_eff, 1);
+    float* sel_conf = (float*)(sel_tok + (size_t)batch * std::max(k_eff, 1));
+    wd_launch_select(c->row_token, c->row_sumexp, act_pos, act_off, 0, batch, k_eff, st->ids_dev, S, n_sel, sel_pos,
+                     sel_tok, sel_conf, c->row_conf, stream);
+    const size_t res_ints = 1 + (size_t)batch + 3 * (size_t)batch * std::max(k_eff, 1);
+    WD_CUDA_TRY(cudaMemcpyAsync(st->result_host, c->result, res_ints * 4, cudaMemcpyDeviceToHost, stream));
+    WD_CUDA_TRY(cudaEventRecord(st->done, stream));
+    WD_CUDA_TRY(cudaGetLastError());
+    st->pending = true;
+    st->k_pending = k_eff;
+    st->k_user = k;
+    if (info) {
+        info->is_refresh = any_refresh ? 1 : 0;
+        info->n_rows = R_; info->n_active = NA; info->n_vis = (int32_t)n_vis;
+        info->n_launches = (int32_t)(wd_launch_counter - launches0); info->gemm_impl = impl_used;
+    }
+    (void)all_contig;
+    return WD_OK;
+}
+
+extern "C" wd_status wd_step_sync(wd_state* st, wd_step_out* out) {
+    if (!st) return WD_ERR_NULL;
+    if (!st->pending) return WD_ERR_NOT_PENDING;
+    st->pending = false;
+    WD_CUDA_TRY(cudaEventSynchronize(st->done));
+    if (st->ctx->prof_on) {
+        wd_ctx* c = st->ctx;
+        for (size_t i = 0; i + 1 < c->prof_used; i += 2) {
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, c->prof_events[i], c->prof_events[i + 1]) == cudaSuccess) c->prof_ms += ms;
+            c->prof_launches += 1;
+        }
+        c->prof_bytes += c->prof_step_bytes;
+    }
+    const int batch = st->batch, k = st->k_pending, kk = std::max(k, 1), ku = st->k_user;
+    const int32_t* res = st->result_host;
+    const int32_t dev_status = res[0];
+    const int32_t* n_sel = res + 1;
+    const int32_t* pos = n_sel + batch;
+    const int32_t* tok = pos + (size_t)batch * kk;
+    const float* conf = (const float*)(tok + (size_t)batch * kk);
+    if (dev_status != 0) {
+        cudaMemset(st->ctx->result, 0, 4);
+        return dev_status == WD_ERR_DEVICE_TIMEOUT ? WD_ERR_DEVICE_TIMEOUT : WD_ERR_BOUNDS;
+    }
+    for (int b = 0; b < batch; ++b) {
+        const WdSeqPlan& p = st->plans[b];
+        const int n = p.done ? 0 : std::min(n_sel[b], k);
+        if (!p.done) wd_commit_seq(st->seqs[b], p, pos + (size_t)b * k, tok + (size_t)b * k, n);
+        if (out) {
+            if (out->n_unmasked) out->n_unmasked[b] = n;
+            for (int i = 0; i < n; ++i) {
+                if (out->positions) out->positions[(size_t)b * ku + i] = pos[(size_t)b * k + i];
+                if (out->token_ids) out->token_ids[(size_t)b * ku + i] = tok[(size_t)b * k + i];
+                if (out->confidence) out->confidence[(size_t)b * ku + i] = conf[(size_t)b * k + i];
+            }
+        }
+    }
+    return WD_OK;
+}
+
+// ---------------------------------------------------------------------------
+// single operations
+// ---------------------------------------------------------------------------
+extern "C" size_t wd_op_gemm_scratch_bytes(int32_t rows, int32_t n_out, int32_t k_in) {
+    if (rows < 1 || n_out < 1 || k_in < 1) return 0;
+    return wd_tc_scratch_bytes(rows, n_out, k_in);
+}
+
+extern "C" wd_status wd_op_gemm(int32_t dtype, int32_t impl, const void* x, const void* w, float* y, int32_t rows,
+                                int32_t n_out, int32_t k_in, void* scratch, size_t scratch_bytes, void* stream) {
+    if (!x || !w || !y) return WD_ERR_NULL;
+    if (rows < 1 || n_out < 1 || k_in < 1) return WD_ERR_BAD_PARAM;
+    if (dtype != WD_F32 && dtype != WD_BF16) return WD_ERR_BAD_PARAM;
+    if (impl == WD_GEMM_AUTO) impl = dtype == WD_BF16 ? WD_GEMM_TCGEN05 : WD_GEMM_PLAIN;
+    if (impl == WD_GEMM_PLAIN) {
+        wd_launch_gemm_plain(dtype, x, w, y, rows, n_out, k_in, n_out, (cudaStream_t)stream);
+        WD_CUDA_TRY(cudaGetLastError());
+        return WD_OK;
+    }
+    if (impl != WD_GEMM_TCGEN05 || dtype != WD_BF16) return WD_ERR_BAD_PARAM;
+    return wd_tc_gemm_standalone(x, w, y, rows, n_out, k_in, scratch, scratch_bytes, (cudaStream_t)stream);
+}
+
+extern "C" wd_status wd_op_attention(int32_t dtype, const void* q, const void* kcache, const void* vcache,
+                                     const int32_t* vis, void* out, int32_t n_rows, int32_t n_vis,
+                                     int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t seq_len,
+                                     void* stream) {
+    if (!q || !kcache || !vcache || !vis || !out) return WD_ERR_NULL;
+    if (dtype != WD_F32 && dtype != WD_BF16) return WD_ERR_BAD_PARAM;
+    if (n_rows < 1 || n_vis < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads || head_dim < 1 ||
+        seq_len < n_vis)
+        return WD_ERR_BAD_PARAM;
+    if ((size_t)(n_vis + head_dim) * 4 > 200 * 1024) return WD_ERR_CAPACITY;
+    // one sequence: no row->sequence table and no offsets, every row sees vis[0, n_vis)
+    wd_launch_attention_plain(dtype, q, kcache, vcache, nullptr, vis, nullptr, out, nullptr, n_rows, n_vis, n_q_heads,
+                              n_kv_heads, head_dim, seq_len, (cudaStream_t)stream);
+    WD_CUDA_TRY(cudaGetLastError());
+    return WD_OK;
+}
+
+extern "C" wd_status wd_op_unmask(const float* logits, const int32_t* positions, int32_t n, int32_t vocab, int32_t k,
+                                  int32_t* row_token, float* row_sumexp, float* row_conf, int32_t* sel_pos,
+                                  int32_t* sel_token, float* sel_conf, int32_t* n_sel, void* stream) {
+    if (!logits || !positions || !row_token || !row_sumexp || !row_conf || !sel_pos || !sel_token || !sel_conf || !n_sel)
+        return WD_ERR_NULL;
+    if (n < 1 || vocab < 1 || k < 0) return WD_ERR_BAD_PARAM;
+    cudaStream_t st = (cudaStream_t)stream;
+    wd_launch_rowstats(logits, n, vocab, row_token, row_sumexp, st);
+    wd_launch_select(row_token, row_sumexp, positions, nullptr, n, 1, k, nullptr, 0, n_sel, sel_pos, sel_token,
+                     sel_conf, row_conf, st);
+    WD_CUDA_TRY(cudaGetLastError());
+    return WD_OK;
+}
+
+extern "C" wd_status wd_op_status(void) {
+    int32_t* p = wd_op_status_ptr();
+    if (!p) return WD_ERR_CUDA;
+    WD_CUDA_TRY(cudaDeviceSynchronize());
+    int32_t v = 0;
+    WD_CUDA_TRY(cudaMemcpy(&v, p, 4, cudaMemcpyDeviceToHost));
+    if (v != 0) cudaMemset(p, 0, 4);
+    return v;
+}

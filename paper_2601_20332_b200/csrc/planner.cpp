@@ -1,0 +1,90 @@
+// Host planner: which positions are active, buffer, transient, far-field,
+// computed and visible in the next step.  Integer logic only.
+//
+// Section 4.2 of the paper: the external window is a fixed-length prefix of
+// the undecoded region and stays put within a phase; the internal window is
+// the front of its still-undecoded part and slides right as tokens decode;
+// buffer = external \ (active U decoded-in-phase); undecoded tokens outside
+// the external window are pruned.  Section 4.3: a phase is one refresh step
+// (everything visible is computed) followed by normal steps (active tokens and
+// recently decoded tokens are computed).
+#include <algorithm>
+#include <climits>
+
+#include "wd_internal.h"
+
+wd_status wd_plan_seq(const WdSeq& s, int32_t A, int32_t B, int32_t R, int32_t T, WdSeqPlan* out) {
+    if (!out) return WD_ERR_NULL;
+    if (A < 1 || B < 0 || R < 1 || T < 0) return WD_ERR_BAD_PARAM;
+    WdSeqPlan& p = *out;
+    p = WdSeqPlan();
+    const int32_t S = (int32_t)s.ids.size();
+
+    int32_t n_undecoded = 0;
+    for (int32_t i = 0; i < S; ++i) n_undecoded += s.decoded[i] ? 0 : 1;
+    if (n_undecoded == 0) { p.done = true; return WD_OK; }
+
+    // does the stored external window still hold an undecoded token?
+    bool window_alive = false;
+    for (int32_t i : s.wex) if (!s.decoded[i]) { window_alive = true; break; }
+    p.refresh = (s.t == 0) || (s.since >= R) || !window_alive;
+
+    if (p.refresh) {
+        // long arithmetic: A + B may exceed int32 for "window = everything" callers
+        const int64_t want = std::min<int64_t>((int64_t)A + (int64_t)B, n_undecoded);
+        p.wex.reserve((size_t)want);
+        for (int32_t i = 0; i < S && (int64_t)p.wex.size() < want; ++i)
+            if (!s.decoded[i]) p.wex.push_back(i);
+    } else {
+        p.wex = s.wex;
+    }
+
+    // walk the external window once: undecoded members fill the internal
+    // window first, the rest is buffer; decoded members were decoded in this
+    // phase and are recomputed while young enough
+    for (int32_t i : p.wex) {
+        if (!s.decoded[i]) {
+            if ((int32_t)p.active.size() < A) p.active.push_back(i);
+            else p.buffer.push_back(i);
+        } else {
+            const int64_t age = (int64_t)s.t - (int64_t)s.dec_step[i];
+            if (age >= 1 && age <= T) p.transient.push_back(i);
+        }
+    }
+
+    // one pass over the sequence for the position-ordered lists
+    std::vector<uint8_t> in_wex((size_t)S, 0);
+    for (int32_t i : p.wex) in_wex[i] = 1;
+    for (int32_t i = 0; i < S; ++i) {
+        if (s.decoded[i]) { p.decoded.push_back(i); p.vis.push_back(i); }
+        else if (in_wex[i]) p.vis.push_back(i);
+        else p.far_field.push_back(i);
+    }
+    if (p.refresh) {
+        p.rows = p.vis;
+    } else {
+        p.rows.resize(p.active.size() + p.transient.size());
+        std::merge(p.active.begin(), p.active.end(), p.transient.begin(), p.transient.end(),
+                   p.rows.begin());
+    }
+    p.vis_contiguous = !p.vis.empty() && p.vis.back() == (int32_t)p.vis.size() - 1;
+    return WD_OK;
+}
+
+void wd_commit_seq(WdSeq& s, const WdSeqPlan& plan, const int32_t* positions,
+                   const int32_t* token_ids, int32_t n) {
+    if (plan.done) return;
+    if (plan.refresh) {
+        s.wex = plan.wex;
+        s.phase_start = s.t;
+        s.since = 0;
+    }
+    for (int32_t i = 0; i < n; ++i) {
+        const int32_t pos = positions[i];
+        s.ids[pos] = token_ids[i];
+        s.decoded[pos] = 1;
+        s.dec_step[pos] = s.t;
+    }
+    s.t += 1;
+    s.since += 1;
+}

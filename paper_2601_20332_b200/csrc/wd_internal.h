@@ -1,0 +1,108 @@
+// Internal declarations shared by the translation units of libwd.so.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <cuda.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <vector>
+
+#include "../../include/wd.h"
+
+#define WD_CUDA_TRY(expr)                               \
+    do {                                                \
+        cudaError_t _e = (expr);                        \
+        if (_e != cudaSuccess) { wd_note_cuda_error(_e, __FILE__, __LINE__); return WD_ERR_CUDA; } \
+    } while (0)
+
+void wd_note_cuda_error(cudaError_t e, const char* file, int line);
+
+// kernels launched by this thread so far (every launcher below counts itself)
+extern thread_local long long wd_launch_counter;
+
+static inline size_t wd_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+static inline int wd_ceil_div(int a, int b) { return (a + b - 1) / b; }
+static inline size_t wd_elt_size(int dtype) { return dtype == WD_F32 ? 4 : 2; }
+
+// ---------------------------------------------------------------------------
+// host planner (planner.cpp): pure integer logic, no CUDA
+// ---------------------------------------------------------------------------
+struct WdSeq {
+    std::vector<int32_t> ids;
+    std::vector<uint8_t> decoded;
+    std::vector<int32_t> dec_step;
+    std::vector<int32_t> wex;       // external window of the current phase
+    int32_t t = 0;                  // diffusion step index
+    int32_t since = 0;              // steps since the last refresh
+    int32_t phase_start = 0;
+};
+
+struct WdSeqPlan {
+    bool done = false, refresh = false, vis_contiguous = false;
+    std::vector<int32_t> wex, active, buffer, decoded, transient, far_field, rows, vis;
+};
+
+// Pure: does not modify `s`.
+wd_status wd_plan_seq(const WdSeq& s, int32_t A, int32_t B, int32_t R, int32_t T, WdSeqPlan* out);
+// Apply a step's update set and advance the phase counters.
+void wd_commit_seq(WdSeq& s, const WdSeqPlan& plan, const int32_t* positions,
+                   const int32_t* token_ids, int32_t n);
+
+// ---------------------------------------------------------------------------
+// kernel launchers.  Every pointer is a device pointer unless stated.
+// `status` is a device int32: kernels store WD_ERR_* there on a failed check.
+// ---------------------------------------------------------------------------
+
+// x[r,:] = embed[ids[row_seq[r]*S + row_pos[r]], :]  (float residual stream)
+void wd_launch_embed(int dtype, const void* embed, const int32_t* ids, const int32_t* row_seq,
+                     const int32_t* row_pos, float* x, int n_rows, int d, int S, int vocab,
+                     int32_t* status, cudaStream_t st);
+
+// x += sum_s part[s] (if part != null); xn = rmsnorm(x) * gain, written as `dtype`.
+// With row_idx != null the rows x[row_idx[i]] are read (no partial add, x not written)
+// and xn[i] is written: used for the final norm over the active rows only.
+void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size_t split_stride,
+                       const float* gain, float eps, void* xn, const int32_t* row_idx, int n_rows,
+                       int d, cudaStream_t st);
+
+// plain GEMM: y[rows, n] (float) = x[rows,k] * w[n,k]^T
+void wd_launch_gemm_plain(int dtype, const void* x, const void* w, float* y, int rows, int n, int k,
+                          int ldy, cudaStream_t st);
+
+// qkv partials -> RoPE -> q (dtype) and K/V cache rows.
+//   part: [n_split][n_rows][(Hq+2Hkv)*dh] float, columns = [q | k | v]
+//   kcache/vcache: [batch][Hkv][S][dh] (this layer's slice)
+void wd_launch_rope_scatter(int dtype, const float* part, int n_split, size_t split_stride,
+                            const int32_t* row_seq, const int32_t* row_pos, void* q, void* kcache,
+                            void* vcache, int n_rows, int Hq, int Hkv, int dh, int S, float theta,
+                            cudaStream_t st);
+
+// general (index-list) attention, CUDA cores.
+//   seq_row_off[batch+1]: rows of sequence b are [off[b], off[b+1])
+//   vis_idx: concatenated visible positions, sequence b at [vis_off[b], vis_off[b+1])
+void wd_launch_attention_plain(int dtype, const void* q, const void* kcache, const void* vcache,
+                               const int32_t* row_seq, const int32_t* vis_idx, const int32_t* vis_off,
+                               void* out, float* tap, int n_rows, int max_vis, int Hq, int Hkv, int dh,
+                               int S, cudaStream_t st);
+
+// h = silu(gate) * up from partials [n_split][n_rows][2F] (columns = [gate | up])
+void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_stride, void* h,
+                      int n_rows, int F, cudaStream_t st);
+
+// x += sum_s part[s]; optionally copy x to tap.
+void wd_launch_residual_add(float* x, const float* part, int n_split, size_t split_stride,
+                            float* tap, int n_rows, int d, cudaStream_t st);
+
+// per-row (max, lowest argmax, sum exp(l - max)) of logits [n, V]
+void wd_launch_rowstats(const float* logits, int n, int V, int32_t* row_token, float* row_sumexp,
+                        cudaStream_t st);
+
+// per sequence: rank active rows by (sumexp ascending, position ascending), emit the first
+// min(k, n_b); optionally write the chosen ids into ids[b*S + pos].  act_off == null means one
+// sequence holding rows [0, n_single).
+void wd_launch_select(const int32_t* row_token, const float* row_sumexp, const int32_t* act_pos,
+                      const int32_t* act_off, int n_single, int batch, int k, int32_t* ids, int S,
+                      int32_t* n_sel, int32_t* sel_pos, int32_t* sel_token, float* sel_conf,
+                      float* row_conf, cudaStream_t st);
+
+int32_t* wd_op_status_ptr();   // device address of the single-operation status word

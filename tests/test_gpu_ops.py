@@ -1,0 +1,126 @@
+"""Unit parity of single operations against the CPU oracle (GPU required)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import wd_oracle as wo
+from paper_2601_20332_b200 import binding as wd
+from paper_2601_20332_b200 import build as wd_build
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    wd_build.build()
+    assert wd.lib() is not None
+
+
+def _ref_gemm(x, w):
+    return x.double().cpu().numpy() @ w.double().cpu().numpy().T
+
+
+GEMM_SHAPES = [  # rows, n, k  (ragged token counts, several tiles, ragged weight-row tail)
+    (1, 128, 64), (7, 256, 128), (16, 128, 512), (34, 384, 1024), (35, 640, 4096), (68, 512, 2048),
+    (130, 256, 1024), (256, 384, 512), (300, 256, 1024), (352, 512, 768), (700, 384, 512), (34, 200, 256),
+    (10, 1000, 264),
+]
+
+
+@pytest.mark.parametrize("rows,n,k", GEMM_SHAPES)
+def test_gemm_tcgen05_vs_oracle(rows, n, k):
+    g = torch.Generator(device=DEV).manual_seed(rows * 1000 + n + k)
+    x = torch.randn(rows, k, device=DEV, generator=g).to(torch.bfloat16)
+    w = (torch.randn(n, k, device=DEV, generator=g) * 0.05).to(torch.bfloat16)
+    y = wd.op_gemm(x, w, wd.WD_GEMM_TCGEN05)
+    assert wd.op_status() == 0
+    ref = _ref_gemm(x, w)
+    got = y.cpu().numpy().astype(np.float64)
+    # bf16 inputs are exact on both sides; only the fp32 accumulation order differs
+    err = np.abs(got - ref).max() / np.abs(ref).max()
+    assert err < 2e-5, err
+    # without scratch: single K slice straight into y
+    y1 = wd.op_gemm(x, w, wd.WD_GEMM_TCGEN05, scratch=torch.empty(256, dtype=torch.uint8, device=DEV))
+    assert np.abs(y1.cpu().numpy() - ref).max() / np.abs(ref).max() < 2e-5
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("rows,n,k", [(1, 5, 3), (10, 70, 33), (34, 384, 256), (97, 130, 1000)])
+def test_gemm_plain_vs_oracle(dtype, rows, n, k):
+    g = torch.Generator(device=DEV).manual_seed(7)
+    x = torch.randn(rows, k, device=DEV, generator=g).to(dtype)
+    w = torch.randn(n, k, device=DEV, generator=g).to(dtype)
+    y = wd.op_gemm(x, w, wd.WD_GEMM_PLAIN)
+    ref = _ref_gemm(x, w)
+    assert np.abs(y.cpu().numpy() - ref).max() / np.abs(ref).max() < 2e-5
+
+
+def test_gemm_bad_arguments():
+    x = torch.zeros(4, 64, device=DEV, dtype=torch.bfloat16)
+    w = torch.zeros(128, 64, device=DEV, dtype=torch.bfloat16)
+    y = torch.zeros(4, 128, device=DEV)
+    L = wd.lib()
+    assert L.wd_op_gemm(wd.WD_BF16, wd.WD_GEMM_TCGEN05, None, w.data_ptr(), y.data_ptr(), 4, 128, 64, None, 0, None) == wd.WD_ERR_NULL
+    assert L.wd_op_gemm(wd.WD_BF16, wd.WD_GEMM_TCGEN05, x.data_ptr(), w.data_ptr(), y.data_ptr(), 0, 128, 64, None, 0, None) == wd.WD_ERR_BAD_PARAM
+    assert L.wd_op_gemm(wd.WD_F32, wd.WD_GEMM_TCGEN05, x.data_ptr(), w.data_ptr(), y.data_ptr(), 4, 128, 64, None, 0, None) == wd.WD_ERR_BAD_PARAM
+    # K must keep rows 16-byte aligned for TMA
+    assert L.wd_op_gemm(wd.WD_BF16, wd.WD_GEMM_TCGEN05, x.data_ptr(), w.data_ptr(), y.data_ptr(), 4, 128, 60, None, 0, None) == wd.WD_ERR_BAD_PARAM
+
+
+ATTN_CASES = [  # rows, n_vis, Hq, Hkv, dh, S
+    (1, 1, 4, 4, 64, 8), (3, 5, 4, 2, 64, 16), (10, 56, 4, 4, 64, 96), (34, 352, 8, 8, 128, 512),
+    (35, 333, 14, 2, 128, 400), (5, 1000, 7, 1, 128, 1024),
+]
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+@pytest.mark.parametrize("rows,nv,Hq,Hkv,dh,S", ATTN_CASES)
+def test_attention_vs_oracle(dtype, rows, nv, Hq, Hkv, dh, S):
+    g = torch.Generator(device=DEV).manual_seed(rows + nv)
+    q = (torch.randn(rows, Hq, dh, device=DEV, generator=g) * 1.5).to(dtype)
+    kc = torch.randn(Hkv, S, dh, device=DEV, generator=g).to(dtype)
+    vc = torch.randn(Hkv, S, dh, device=DEV, generator=g).to(dtype)
+    vis_np = np.sort(np.random.default_rng(nv).choice(S, size=nv, replace=False)).astype(np.int32)
+    # poison what must not be read
+    hidden = np.setdiff1d(np.arange(S), vis_np)
+    if len(hidden):
+        kc[:, torch.as_tensor(hidden, device=DEV)] = float("nan")
+        vc[:, torch.as_tensor(hidden, device=DEV)] = float("nan")
+    vis = torch.as_tensor(vis_np, device=DEV)
+    out = wd.op_attention(q, kc, vc, vis).float().cpu().numpy().astype(np.float64)
+    K = kc.double().cpu().numpy().transpose(1, 0, 2)[vis_np]
+    V = vc.double().cpu().numpy().transpose(1, 0, 2)[vis_np]
+    ref, _ = wo.attention_rows(q.double().cpu().numpy(), K, V, Hq // Hkv)
+    tol = 2e-2 if dtype == torch.bfloat16 else 1e-5
+    assert np.isfinite(out).all()
+    assert np.abs(out - ref).max() / np.abs(ref).max() < tol
+
+
+@pytest.mark.parametrize("n,V,k", [(1, 2, 1), (8, 1024, 1), (32, 126464, 1), (64, 126464, 2), (5, 1000, 9), (7, 333, 0)])
+def test_unmask_vs_oracle_bit_exact(n, V, k):
+    g = torch.Generator(device=DEV).manual_seed(n * V)
+    logits = torch.randn(n, V, device=DEV, generator=g) * 1.3
+    pos_np = np.sort(np.random.default_rng(n).choice(4096, size=n, replace=False)).astype(np.int32)
+    got = wd.op_unmask(logits, torch.as_tensor(pos_np, device=DEV), k)
+    um = wo.oracle_unmask(logits.cpu().numpy(), pos_np.tolist(), k)
+    assert got["row_token"].tolist() == um["ids"].tolist()
+    np.testing.assert_allclose(got["row_conf"], um["conf"], rtol=2e-5)
+    assert got["positions"] == um["positions"]
+    assert got["token_ids"] == um["token_ids"]
+
+
+def test_unmask_exact_ties():
+    V = 777
+    logits = torch.zeros(6, V, device=DEV)
+    logits[1, [50, 400]] = 3.0                      # two equal maxima -> lowest index
+    logits[4] = logits[1]                           # duplicated row -> equal confidence -> lowest position
+    logits[2, 9] = 50.0
+    pos = torch.tensor([3, 5, 8, 13, 21, 34], dtype=torch.int32, device=DEV)
+    got = wd.op_unmask(logits, pos, 4)
+    um = wo.oracle_unmask(logits.cpu().numpy(), pos.cpu().tolist(), 4)
+    assert got["row_token"].tolist() == um["ids"].tolist() == [0, 50, 9, 0, 50, 0]
+    assert got["positions"] == um["positions"] == [8, 5, 21, 3]
+    assert got["row_conf"][1] == got["row_conf"][4]                     # identical rows give identical bits
+    np.testing.assert_allclose(got["row_conf"][0], 1.0 / V, rtol=1e-6)  # all-equal logits: 1 / V
+    assert abs(got["row_conf"][2] - 1.0) < 1e-6

@@ -1,0 +1,151 @@
+"""Parity of the whole windowed step against the CPU oracle (GPU required)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2601_20332_b200 import binding as wd
+from paper_2601_20332_b200 import build as wd_build
+from paper_2601_20332_b200 import synth
+from wd_harness import Parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    wd_build.build()
+
+
+def run(cfg, n_steps, ids=None, decoded=None, impl=wd.WD_GEMM_AUTO, jitter=0.1, tol_layer=1e-2, tol_attn=2e-2,
+        oracle_seqs=None, weights=None):
+    w = synth.make_weights(cfg, DEV, gain_jitter=jitter) if weights is None else weights
+    ids = synth.make_prompts(cfg) if ids is None else ids
+    p = Parity(cfg, w, ids, decoded, gemm_impl=impl, oracle_seqs=oracle_seqs)
+    logs = []
+    for _ in range(n_steps):
+        r = p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"], tol_layer, tol_attn)
+        if r is None:
+            break
+        logs.append(r)
+    p.check_state_mirror()
+    p.close()
+    return logs
+
+
+def test_tiny_fp32_full_generation():
+    """cfg 1: the whole 64-step generation, every step compared."""
+    cfg = synth.get_config("tiny")
+    logs = run(cfg, 70, tol_layer=2e-5, tol_attn=2e-5)
+    assert len(logs) == 64
+    kinds = [l["info"]["is_refresh"] for l in logs]
+    assert kinds[:8] == [1, 0, 0, 0, 1, 0, 0, 0]
+    assert sum(l["worst"]["ambiguous"] for l in logs) == 0
+    assert max(l["info"]["n_rows"] for l in logs if not l["info"]["is_refresh"]) <= 8 + 2
+
+
+SMALL_BF16 = dict(L=3, d=512, Hq=8, Hkv=8, dh=64, F=1408, V=5000, P=40, G=80, A=8, B=24, R=4, T=2, k=1)
+
+
+@pytest.mark.parametrize("impl", [wd.WD_GEMM_PLAIN, wd.WD_GEMM_TCGEN05])
+def test_small_bf16_trajectory(impl):
+    cfg = synth.get_config("llada8b", **SMALL_BF16)
+    logs = run(cfg, 10, impl=impl)
+    assert [l["info"]["is_refresh"] for l in logs[:9]] == [1, 0, 0, 0, 1, 0, 0, 0, 1]
+    assert all(l["info"]["gemm_impl"] == impl for l in logs)
+    assert any(len(p["transient"]) == 2 for l in logs for p in l["plans"])
+
+
+def test_small_bf16_gqa_batch_two_tokens():
+    """GQA (7 query heads per KV head), batch of independent windows, k = 2, head_dim 128."""
+    cfg = synth.get_config("dream7b", L=2, d=896, Hq=7, Hkv=1, dh=128, F=1024, V=3000, P=20, G=50, batch=3,
+                           A=6, B=10, R=3, T=3, k=2)
+    logs = run(cfg, 8)
+    assert len(logs) == 8
+    # sequences got different prompts, so their choices differ
+    pos = np.array([l["res"]["positions"][:, 0] for l in logs])
+    assert pos.shape == (8, 3)
+
+
+def test_window_covering_everything_is_full_sequence_step():
+    """A >= number of masks, B = 0, R = 1: every step is the no-pruning full-sequence step."""
+    cfg = synth.get_config("llada8b", **dict(SMALL_BF16, A=80, B=0, R=1, T=0, k=4))
+    logs = run(cfg, 3)
+    assert all(l["info"]["is_refresh"] for l in logs)
+    assert logs[0]["info"]["n_rows"] == 120 and logs[0]["info"]["n_active"] == 80
+
+
+def test_non_prefix_decoded_pattern_uses_index_lists():
+    cfg = synth.get_config("llada8b", **SMALL_BF16)
+    ids = synth.make_prompts(cfg)
+    S = ids.shape[1]
+    dec = synth.random_decoded_pattern(S, 0.4, 5)[None, :]
+    rng = np.random.default_rng(3)
+    ids = np.where(dec == 1, rng.integers(0, cfg["V"] - 1, size=ids.shape), cfg["mask_id"]).astype(np.int32)
+    logs = run(cfg, 6, ids=ids, decoded=dec)
+    assert not logs[0]["plans"][0]["vis_contiguous"]
+
+
+def test_late_state_and_finish():
+    """Fast-forwarded state near the end: runs to WD_DONE, last phases have fewer tokens than A."""
+    cfg = synth.get_config("llada8b", **SMALL_BF16)
+    ids, dec = synth.fast_forward(cfg, synth.make_prompts(cfg), 70)
+    logs = run(cfg, 20, ids=ids, decoded=dec)
+    assert len(logs) == 10                          # 10 masks left, one per step
+    assert logs[-1]["info"]["n_active"] == 1
+
+
+def test_far_field_and_refresh_independence_on_gpu():
+    """Changing ids at far-field positions and poisoning the K/V cache before a refresh
+    changes nothing, bit for bit."""
+    cfg = synth.get_config("llada8b", **SMALL_BF16)
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    S = ids.shape[1]
+    outs = []
+    for variant in range(2):
+        ctx = wd.Context(cfg, w, 1, S, S, S)
+        ids_v = ids.copy()
+        if variant:
+            ids_v[0, cfg["P"] + cfg["A"] + cfg["B"]:] = 17
+        st = wd.State(ctx, ids_v, (ids != cfg["mask_id"]).astype(np.uint8))
+        st.mem.view(torch.int16)[S * 2 + 128:].fill_(0x7FC0 if variant else 0)      # NaN / zero K/V cache
+        lg = torch.zeros(S * cfg["V"], device=DEV)
+        st.set_taps(logits=lg)
+        res = []
+        for _ in range(3):
+            _, info = st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], 1)
+            r = st.sync()
+            res.append((lg[: info["n_active"] * cfg["V"]].clone(), r["positions"].copy(), r["token_ids"].copy()))
+        outs.append(res)
+        st.close(); ctx.close()
+    for a, b in zip(*outs):
+        assert torch.equal(a[0], b[0]) and (a[1] == b[1]).all() and (a[2] == b[2]).all()
+
+
+def test_step_error_codes():
+    cfg = synth.get_config("llada8b", **SMALL_BF16)
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    S = ids.shape[1]
+    ctx = wd.Context(cfg, w, 1, S, 64, 16)            # max_rows 64 < a refresh over 72 rows
+    st = wd.State(ctx, ids)
+    with pytest.raises(wd.WdError) as e:
+        st.step(8, 24, 4, 2, 1)
+    assert e.value.status == wd.WD_ERR_CAPACITY
+    with pytest.raises(wd.WdError) as e:
+        st.step(0, 24, 4, 2, 1)
+    assert e.value.status == wd.WD_ERR_BAD_PARAM
+    with pytest.raises(wd.WdError) as e:
+        st.sync()
+    assert e.value.status == wd.WD_ERR_NOT_PENDING
+    status, _ = st.step(8, 8, 4, 2, 1)                # 40 + 16 = 56 rows fits
+    assert status == wd.WD_OK
+    with pytest.raises(wd.WdError) as e:
+        st.step(8, 8, 4, 2, 1)
+    assert e.value.status == wd.WD_ERR_PENDING
+    st.sync()
+    st.close(); ctx.close()
+    with pytest.raises(wd.WdError) as e:
+        wd.Context(synth.get_config("llada8b", **dict(SMALL_BF16, d=500)), w, 1, S, S, S)
+    assert e.value.status == wd.WD_ERR_INVALID_DIMS
