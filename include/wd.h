@@ -293,11 +293,11 @@ WD_API wd_status wd_op_attention(int32_t dtype, const void* q, const void* kcach
  * token = lowest index of the maximal logit, confidence = its softmax
  * probability; the min(k, n) rows of highest confidence are returned (equal
  * confidence: lowest position).  positions: device int32 [n] ascending.
- * Outputs are device arrays: row_token[n], row_sumexp[n] (sum_v exp(logit_v - max),
- * the reciprocal of the confidence), row_conf[n], sel_pos[k], sel_token[k],
- * sel_conf[k], n_sel[1]; none of them may overlap. */
+ * Outputs are device arrays: row_token[n], row_sumexp[n] (sum_v exp(logit_v - max)
+ * accumulated in double, the reciprocal of the confidence and the ranking key),
+ * row_conf[n], sel_pos[k], sel_token[k], sel_conf[k], n_sel[1]; none may overlap. */
 WD_API wd_status wd_op_unmask(const float* logits, const int32_t* positions, int32_t n, int32_t vocab,
-                       int32_t k, int32_t* row_token, float* row_sumexp, float* row_conf,
+                       int32_t k, int32_t* row_token, double* row_sumexp, float* row_conf,
                        int32_t* sel_pos, int32_t* sel_token, float* sel_conf, int32_t* n_sel,
                        void* stream);
 

@@ -322,7 +322,7 @@ def op_unmask(logits, positions, k: int, stream=None) -> dict:
     dev = logits.device
     kk = max(k, 1)
     row_token = torch.empty(n, dtype=torch.int32, device=dev)
-    row_sumexp = torch.empty(n, dtype=torch.float32, device=dev)
+    row_sumexp = torch.empty(n, dtype=torch.float64, device=dev)
     row_conf = torch.empty(n, dtype=torch.float32, device=dev)
     sel_pos = torch.full((kk,), -1, dtype=torch.int32, device=dev)
     sel_tok = torch.full((kk,), -1, dtype=torch.int32, device=dev)

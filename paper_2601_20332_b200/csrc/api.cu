@@ -64,7 +64,7 @@ struct wd_ctx {
     size_t part_floats = 0;
     float* logits = nullptr;     // [max_active, V]
     int32_t* row_token = nullptr;
-    float* row_sumexp = nullptr;
+    double* row_sumexp = nullptr;
     float* row_conf = nullptr;
     int32_t* plan = nullptr;     // packed index lists of the step
     size_t plan_ints = 0;
@@ -129,7 +129,7 @@ static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[16]) {
     off[5] = c.take(part_floats_for(d) * 4);                    // part
     off[6] = c.take(MA * d->vocab * 4);                         // logits
     off[7] = c.take(MA * 4);                                    // row_token
-    off[8] = c.take(MA * 4);                                    // row_sumexp
+    off[8] = c.take(MA * 8);                                    // row_sumexp
     off[9] = c.take(MA * 4);                                    // row_conf
     const size_t plan_ints = 2 * MR + 2 * MA + 2 * ((size_t)d->max_batch + 1) + (size_t)d->max_batch * d->max_seq;
     off[10] = c.take(plan_ints * 4);                            // plan
@@ -198,7 +198,7 @@ extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, v
     c->part_floats = part_floats_for(dims);
     c->logits = (float*)(base + off[6]);
     c->row_token = (int32_t*)(base + off[7]);
-    c->row_sumexp = (float*)(base + off[8]);
+    c->row_sumexp = (double*)(base + off[8]);
     c->row_conf = (float*)(base + off[9]);
     c->plan = (int32_t*)(base + off[10]);
     c->plan_ints = off[12];
@@ -721,7 +721,7 @@ extern "C" wd_status wd_op_attention(int32_t dtype, const void* q, const void* k
 }
 
 extern "C" wd_status wd_op_unmask(const float* logits, const int32_t* positions, int32_t n, int32_t vocab, int32_t k,
-                                  int32_t* row_token, float* row_sumexp, float* row_conf, int32_t* sel_pos,
+                                  int32_t* row_token, double* row_sumexp, float* row_conf, int32_t* sel_pos,
                                   int32_t* sel_token, float* sel_conf, int32_t* n_sel, void* stream) {
     if (!logits || !positions || !row_token || !row_sumexp || !row_conf || !sel_pos || !sel_token || !sel_conf || !n_sel)
         return WD_ERR_NULL;

@@ -449,6 +449,7 @@ size_t wd_tc_scratch_bytes(int rows, int n_out, int k_in) {
 
 wd_status wd_tc_gemm_standalone(const void* x, const void* w, float* y, int rows, int n_out, int k_in, void* scratch,
                                 size_t scratch_bytes, cudaStream_t stream) {
+    if (k_in % 8) return WD_ERR_BAD_PARAM;      // TMA rows must be multiples of 16 bytes
     int32_t* status = wd_op_status_ptr();
     if (!status) return WD_ERR_CUDA;
     CUtensorMap mw;

@@ -260,10 +260,20 @@ __global__ void residual_add_kernel(float* __restrict__ x, const float* __restri
 // ---------------------------------------------------------------- unmask reduction
 // One block of 256 threads per active row, the same reduction order for every row:
 // thread-strided scan, warp-shuffle tree, then the 8 warp results in lane order.
+// The sum of exponentials is taken in double precision: it decides which rows are unmasked,
+// and in double the ranking agrees with an exact evaluation of the same float logits except
+// for gaps at the 1e-13 level (the work is a few million exps per step).
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
 __global__ void rowstats_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ row_token,
-                                float* __restrict__ row_sumexp) {
+                                double* __restrict__ row_sumexp) {
     __shared__ float s_val[8];
     __shared__ int s_idx[8];
+    __shared__ double s_sum[8];
     __shared__ float s_max;
     const float* lr = logits + (size_t)blockIdx.x * V;
     float best = -INFINITY;
@@ -290,23 +300,22 @@ __global__ void rowstats_kernel(const float* __restrict__ logits, int V, int32_t
         row_token[blockIdx.x] = i;
     }
     __syncthreads();
-    const float m = s_max;
-    float sum = 0.f;
-    for (int v = threadIdx.x; v < V; v += 256) sum += expf(lr[v] - m);
-    sum = warp_sum(sum);
-    __syncthreads();
-    if (lane == 0) s_val[w] = sum;
+    const double m = (double)s_max;
+    double sum = 0.0;
+    for (int v = threadIdx.x; v < V; v += 256) sum += exp((double)lr[v] - m);
+    sum = warp_sum_d(sum);
+    if (lane == 0) s_sum[w] = sum;
     __syncthreads();
     if (threadIdx.x == 0) {
-        float t = 0.f;
-        for (int j = 0; j < 8; ++j) t += s_val[j];
+        double t = 0.0;
+        for (int j = 0; j < 8; ++j) t += s_sum[j];
         row_sumexp[blockIdx.x] = t;
     }
 }
 
 // One block per sequence.  rank(i) = #{j : s_j < s_i or (s_j == s_i and pos_j < pos_i)}; positions
 // are ascending inside a sequence, so "pos_j < pos_i" is "j < i".
-__global__ void select_kernel(const int32_t* __restrict__ row_token, const float* __restrict__ row_sumexp,
+__global__ void select_kernel(const int32_t* __restrict__ row_token, const double* __restrict__ row_sumexp,
                               const int32_t* __restrict__ act_pos, const int32_t* __restrict__ act_off,
                               int n_single, int k, int32_t* __restrict__ ids, int S, int32_t* __restrict__ n_sel,
                               int32_t* __restrict__ sel_pos, int32_t* __restrict__ sel_token,
@@ -317,18 +326,19 @@ __global__ void select_kernel(const int32_t* __restrict__ row_token, const float
     const int kk = min(k, n);
     if (threadIdx.x == 0) n_sel[b] = kk;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
-        const float si = row_sumexp[a0 + i];
-        if (row_conf) row_conf[a0 + i] = 1.f / si;
+        const double si = row_sumexp[a0 + i];
+        const float conf = (float)(1.0 / si);
+        if (row_conf) row_conf[a0 + i] = conf;
         int rank = 0;
         for (int j = 0; j < n; ++j) {
-            const float sj = row_sumexp[a0 + j];
+            const double sj = row_sumexp[a0 + j];
             rank += (sj < si || (sj == si && j < i)) ? 1 : 0;
         }
         if (rank < kk) {
             const int pos = act_pos[a0 + i], tok = row_token[a0 + i];
             sel_pos[b * k + rank] = pos;
             sel_token[b * k + rank] = tok;
-            sel_conf[b * k + rank] = 1.f / si;
+            sel_conf[b * k + rank] = conf;
             if (ids) ids[(size_t)b * S + pos] = tok;
         }
     }
@@ -424,14 +434,14 @@ void wd_launch_residual_add(float* x, const float* part, int n_split, size_t spl
     residual_add_kernel<<<blocks, 256, 0, st>>>(x, part, n_split, split_stride, tap, total);
 }
 
-void wd_launch_rowstats(const float* logits, int n, int V, int32_t* row_token, float* row_sumexp,
+void wd_launch_rowstats(const float* logits, int n, int V, int32_t* row_token, double* row_sumexp,
                         cudaStream_t st) {
     if (n <= 0) return;
     ++wd_launch_counter;
     rowstats_kernel<<<n, 256, 0, st>>>(logits, V, row_token, row_sumexp);
 }
 
-void wd_launch_select(const int32_t* row_token, const float* row_sumexp, const int32_t* act_pos,
+void wd_launch_select(const int32_t* row_token, const double* row_sumexp, const int32_t* act_pos,
                       const int32_t* act_off, int n_single, int batch, int k, int32_t* ids, int S,
                       int32_t* n_sel, int32_t* sel_pos, int32_t* sel_token, float* sel_conf,
                       float* row_conf, cudaStream_t st) {

@@ -93,14 +93,14 @@ void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_st
 void wd_launch_residual_add(float* x, const float* part, int n_split, size_t split_stride,
                             float* tap, int n_rows, int d, cudaStream_t st);
 
-// per-row (max, lowest argmax, sum exp(l - max)) of logits [n, V]
-void wd_launch_rowstats(const float* logits, int n, int V, int32_t* row_token, float* row_sumexp,
+// per-row (max, lowest argmax, sum exp(l - max) in double) of logits [n, V]
+void wd_launch_rowstats(const float* logits, int n, int V, int32_t* row_token, double* row_sumexp,
                         cudaStream_t st);
 
 // per sequence: rank active rows by (sumexp ascending, position ascending), emit the first
 // min(k, n_b); optionally write the chosen ids into ids[b*S + pos].  act_off == null means one
 // sequence holding rows [0, n_single).
-void wd_launch_select(const int32_t* row_token, const float* row_sumexp, const int32_t* act_pos,
+void wd_launch_select(const int32_t* row_token, const double* row_sumexp, const int32_t* act_pos,
                       const int32_t* act_off, int n_single, int batch, int k, int32_t* ids, int S,
                       int32_t* n_sel, int32_t* sel_pos, int32_t* sel_token, float* sel_conf,
                       float* row_conf, cudaStream_t st);
