@@ -279,6 +279,33 @@ WD_API wd_status wd_op_gemm(int32_t dtype, int32_t impl, const void* x, const vo
                      void* scratch, size_t scratch_bytes, void* stream);
 WD_API size_t wd_op_gemm_scratch_bytes(int32_t rows, int32_t n_out, int32_t k_in);
 
+/* (No counterpart in the paper: a packaging variant of wd_op_gemm.)
+ * The same bf16 tensor-core GEMM, y[rows, n_out] (float) = x[rows, k_in] * w[n_out, k_in]^T,
+ * for callers that cannot hand over scratch memory because they may not allocate
+ * where they call from: code living inside another framework's memory pool, a
+ * serving loop that bans allocator calls once it is running, a process whose device
+ * memory is already fully committed.  The split-K partial sums go to a fixed
+ * 16 MiB array that is part of the library image (wd_op_gemm_noalloc_max_floats()
+ * floats; each GPU that loads the library keeps it until the process exits).  This
+ * call allocates nothing, on the host or on the device.
+ *   - Limit: rows * n_out must not exceed wd_op_gemm_noalloc_max_floats(), otherwise
+ *     WD_ERR_CAPACITY and nothing is launched.  Fewer K slices are used when the
+ *     array cannot hold more, so large shapes run slower than with wd_op_gemm.
+ *   - The first call on each device looks up the array's device address (with that
+ *     device current) and remembers it; make that first call before any stream
+ *     capture begins.
+ *   - All calls share the one array and it keeps whatever the last call left in it.
+ *     Nothing needs clearing (every partial sum that is read is written first by
+ *     the same call), but two calls that overlap on the GPU, e.g. on different
+ *     streams, race on it: keep calls on one stream or order them with events.
+ * Pointers are device pointers; x, w bf16 row-major with k_in contiguous, 16-byte
+ * aligned, k_in a multiple of 8.  Errors: WD_ERR_NULL, WD_ERR_BAD_PARAM,
+ * WD_ERR_CAPACITY, WD_ERR_MISALIGNED, WD_ERR_CUDA; a device-side time-out is
+ * reported by wd_op_status(). */
+WD_API wd_status wd_op_gemm_noalloc(const void* x, const void* w, float* y, int32_t rows, int32_t n_out,
+                                    int32_t k_in, void* stream);
+WD_API size_t wd_op_gemm_noalloc_max_floats(void);
+
 /* Bidirectional grouped-query attention (Section 3.1: no causal mask) of
  * n_rows query rows over n_vis cached positions of one sequence:
  * out[r, h, :] = softmax_j(q[r,h,:] . K[kvh(h), vis[j], :] / sqrt(head_dim)) V[kvh(h), vis[j], :].

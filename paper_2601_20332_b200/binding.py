@@ -78,6 +78,8 @@ SIGNATURES = {
     "wd_step_sync": (C.c_int, [vp, C.POINTER(wd_step_out)]),
     "wd_op_gemm": (C.c_int, [i32, i32, vp, vp, vp, i32, i32, i32, vp, C.c_size_t, vp]),
     "wd_op_gemm_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
+    "wd_op_gemm_noalloc": (C.c_int, [vp, vp, vp, i32, i32, i32, vp]),
+    "wd_op_gemm_noalloc_max_floats": (C.c_size_t, []),
     "wd_op_attention": (C.c_int, [i32, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]),
     "wd_op_unmask": (C.c_int, [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
     "wd_op_status": (C.c_int, []),
@@ -301,6 +303,19 @@ def op_gemm(x, w, impl: int = WD_GEMM_AUTO, stream=None, scratch=None):
         scratch = torch.empty(max(nb, 256), dtype=torch.uint8, device=x.device)
     check(lib().wd_op_gemm(_dtype_code(x), impl, _ptr(x), _ptr(w), _ptr(y), rows, n, k, _ptr(scratch),
                            scratch.numel(), _stream_ptr(stream)), "wd_op_gemm")
+    return y
+
+
+def op_gemm_noalloc(x, w, y=None, stream=None):
+    """wd_op_gemm_noalloc: bf16 GEMM whose scratch is a fixed array inside the library, for
+    callers that may not allocate.  Pass a preallocated float32 `y` to keep this wrapper
+    allocation-free as well."""
+    import torch
+    rows, k = x.shape
+    n = w.shape[0]
+    if y is None:
+        y = torch.empty(rows, n, dtype=torch.float32, device=x.device)
+    check(lib().wd_op_gemm_noalloc(_ptr(x), _ptr(w), _ptr(y), rows, n, k, _stream_ptr(stream)), "wd_op_gemm_noalloc")
     return y
 
 

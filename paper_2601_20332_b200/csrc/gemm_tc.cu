@@ -475,3 +475,68 @@ wd_status wd_tc_gemm_standalone(const void* x, const void* w, float* y, int rows
     WD_CUDA_TRY(cudaGetLastError());
     return WD_OK;
 }
+
+// ------------------------------------------------------------------------------------------
+// wd_op_gemm_noalloc: the tensor-core GEMM with its split-K scratch inside the library image
+// ------------------------------------------------------------------------------------------
+// Some callers cannot provide scratch memory because they are not allowed to allocate at the
+// point of the call: a plugin running inside another framework's memory pool, a real-time
+// loop that forbids allocator calls after start-up, code that runs while device memory is
+// fully committed.  For them the partial sums of the K slices live in this fixed array, which
+// every GPU that loads the library holds until the process exits.
+#define WD_NOALLOC_SCRATCH_FLOATS (4u << 20)      // 4 Mi floats = 16 MiB
+static __device__ __align__(256) float g_noalloc_scratch[WD_NOALLOC_SCRATCH_FLOATS];
+
+// In host code the array's name is only a handle for the runtime, not a device address, so the
+// address is asked for once per device (with that device current) and cached.
+static float* noalloc_scratch_ptr(wd_status* err) {
+    static float* cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) { *err = WD_ERR_CUDA; return nullptr; }
+    if (!cached[dev]) {
+        float* p = nullptr;
+        cudaError_t e = cudaGetSymbolAddress((void**)&p, g_noalloc_scratch);
+        if (e != cudaSuccess || !p) {
+            wd_note_cuda_error(e, __FILE__, __LINE__);
+            *err = WD_ERR_CUDA;
+            return nullptr;
+        }
+        cached[dev] = p;
+    }
+    return cached[dev];
+}
+
+extern "C" size_t wd_op_gemm_noalloc_max_floats(void) { return (size_t)WD_NOALLOC_SCRATCH_FLOATS; }
+
+extern "C" wd_status wd_op_gemm_noalloc(const void* x, const void* w, float* y, int32_t rows, int32_t n_out,
+                                        int32_t k_in, void* stream_) {
+    if (!x || !w || !y) return WD_ERR_NULL;
+    if (rows < 1 || n_out < 1 || k_in < 8 || k_in % 8) return WD_ERR_BAD_PARAM;
+    const size_t slice = (size_t)rows * (size_t)n_out;
+    if (slice > (size_t)WD_NOALLOC_SCRATCH_FLOATS) return WD_ERR_CAPACITY;   // one K slice must fit
+    wd_status err = WD_OK;
+    float* scratch = noalloc_scratch_ptr(&err);
+    if (!scratch) return err;
+    int32_t* status = wd_op_status_ptr();
+    if (!status) return WD_ERR_CUDA;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    CUtensorMap mw;
+    wd_status s = encode_2d(&mw, w, n_out, k_in, kBM);
+    if (s != WD_OK) return s;
+    WdTcSeg seg = {w, n_out, &mw};
+    WdTcX xm = {x, k_in};
+    int sm = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+    // the number of K slices is capped by what fits in the fixed array; every element of every
+    // slice that the reduction reads is written by exactly one CTA first, so nothing has to be
+    // cleared between calls even though the array keeps the previous call's contents
+    int ns = 1;
+    s = wd_tc_gemm(&xm, &seg, 1, rows, k_in, scratch, (size_t)WD_NOALLOC_SCRATCH_FLOATS, sm, status, stream, &ns, false);
+    if (s != WD_OK) return s;
+    const int blocks = (int)((slice + 255) / 256 < 1184 ? (slice + 255) / 256 : 1184);
+    ++wd_launch_counter;
+    reduce_slices_kernel<<<blocks, 256, 0, stream>>>(scratch, ns, slice, y, slice);
+    WD_CUDA_TRY(cudaGetLastError());
+    return WD_OK;
+}
