@@ -309,8 +309,10 @@ WD_API size_t wd_op_gemm_noalloc_max_floats(void);
 /* Bidirectional grouped-query attention (Section 3.1: no causal mask) of
  * n_rows query rows over n_vis cached positions of one sequence:
  * out[r, h, :] = softmax_j(q[r,h,:] . K[kvh(h), vis[j], :] / sqrt(head_dim)) V[kvh(h), vis[j], :].
- * q, out: [n_rows, n_q_heads, head_dim]; kcache, vcache: [n_kv_heads, seq_len, head_dim];
- * vis: device int32 [n_vis], all of `dtype`. */
+ * q, out: [n_rows, n_q_heads, head_dim]; kcache: [n_kv_heads, seq_len, head_dim];
+ * vcache TRANSPOSED: [n_kv_heads, head_dim, seq_len] (the layout the step keeps V in, so
+ * that V tiles are read with the key position contiguous); vis: device int32 [n_vis];
+ * all of `dtype`. */
 WD_API wd_status wd_op_attention(int32_t dtype, const void* q, const void* kcache, const void* vcache,
                           const int32_t* vis, void* out, int32_t n_rows, int32_t n_vis,
                           int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t seq_len,
@@ -326,7 +328,9 @@ WD_API wd_status wd_op_attention(int32_t dtype, const void* q, const void* kcach
 WD_API wd_status wd_op_unmask(const float* logits, const int32_t* positions, int32_t n, int32_t vocab,
                        int32_t k, int32_t* row_token, double* row_sumexp, float* row_conf,
                        int32_t* sel_pos, int32_t* sel_token, float* sel_conf, int32_t* n_sel,
-                       void* stream);
+                       void* scratch, size_t scratch_bytes, void* stream);
+/* Device scratch the unmask operation needs (per-chunk partial statistics), 8-byte aligned. */
+WD_API size_t wd_op_unmask_scratch_bytes(int32_t n, int32_t vocab);
 
 /* Device status word shared by the single operations: 0, or the first
  * WD_ERR_DEVICE_TIMEOUT / WD_ERR_BOUNDS raised by a kernel since the last

@@ -81,7 +81,8 @@ SIGNATURES = {
     "wd_op_gemm_noalloc": (C.c_int, [vp, vp, vp, i32, i32, i32, vp]),
     "wd_op_gemm_noalloc_max_floats": (C.c_size_t, []),
     "wd_op_attention": (C.c_int, [i32, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]),
-    "wd_op_unmask": (C.c_int, [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp]),
+    "wd_op_unmask": (C.c_int, [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]),
+    "wd_op_unmask_scratch_bytes": (C.c_size_t, [i32, i32]),
     "wd_op_status": (C.c_int, []),
 }
 
@@ -320,7 +321,7 @@ def op_gemm_noalloc(x, w, y=None, stream=None):
 
 
 def op_attention(q, kcache, vcache, vis, stream=None):
-    """q: [rows, Hq, dh]; kcache/vcache: [Hkv, S, dh]; vis: int32 [n_vis] (device)."""
+    """q: [rows, Hq, dh]; kcache: [Hkv, S, dh]; vcache transposed: [Hkv, dh, S]; vis: int32 [n_vis] (device)."""
     import torch
     rows, Hq, dh = q.shape
     Hkv, S, _ = kcache.shape
@@ -343,9 +344,10 @@ def op_unmask(logits, positions, k: int, stream=None) -> dict:
     sel_tok = torch.full((kk,), -1, dtype=torch.int32, device=dev)
     sel_conf = torch.zeros(kk, dtype=torch.float32, device=dev)
     n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    scratch = torch.empty(lib().wd_op_unmask_scratch_bytes(n, V), dtype=torch.uint8, device=dev)
     check(lib().wd_op_unmask(_ptr(logits), _ptr(positions), n, V, k, _ptr(row_token), _ptr(row_sumexp),
                              _ptr(row_conf), _ptr(sel_pos), _ptr(sel_tok), _ptr(sel_conf), _ptr(n_sel),
-                             _stream_ptr(stream)), "wd_op_unmask")
+                             _ptr(scratch), scratch.numel(), _stream_ptr(stream)), "wd_op_unmask")
     ns = int(n_sel.item())
     return dict(row_token=row_token.cpu().numpy(), row_sumexp=row_sumexp.cpu().numpy(),
                 row_conf=row_conf.cpu().numpy(), positions=sel_pos.cpu().numpy()[:ns].tolist(),

@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libwd.so")
-SOURCES = ["api.cu", "planner.cpp", "kernels_plain.cu", "gemm_tc.cu"]
+SOURCES = ["api.cu", "planner.cpp", "kernels_plain.cu", "gemm_tc.cu", "attention_tc.cu"]
 
 
 def _nvcc() -> str:

@@ -8,6 +8,7 @@
 
 #include "wd_internal.h"
 #include "gemm_tc.h"
+#include "attention_tc.h"
 
 // ---------------------------------------------------------------------------
 // error bookkeeping
@@ -52,6 +53,7 @@ struct wd_ctx {
     std::vector<const void*> wq, wk, wv, wo, wg, wu, wd;
     std::vector<const float*> attn_norm, ffn_norm;
     int gemm_impl = WD_GEMM_AUTO;
+    int attn_impl = WD_GEMM_AUTO;   // WD_GEMM_PLAIN forces the CUDA-core attention
     int sm_count = 148;
 
     // workspace carve-up (device)
@@ -66,6 +68,10 @@ struct wd_ctx {
     int32_t* row_token = nullptr;
     double* row_sumexp = nullptr;
     float* row_conf = nullptr;
+    float* ch_max = nullptr;     // [max_active][chunks] unmask stage-1 statistics
+    int32_t* ch_idx = nullptr;
+    double* ch_sum = nullptr;
+    float2* rope_tab = nullptr;  // [max_rows][dh/2] (cos, sin) of this step's rows
     int32_t* plan = nullptr;     // packed index lists of the step
     size_t plan_ints = 0;
     int32_t* result = nullptr;   // [status | n_sel[batch] | pos | tok | conf]
@@ -94,6 +100,7 @@ static bool dims_valid(const wd_model_dims* d) {
     if ((int64_t)d->max_rows > (int64_t)d->max_batch * d->max_seq) return false;
     if (d->max_active > d->max_rows) return false;
     if (!(d->rope_theta > 1.f) || !(d->rms_eps >= 0.f)) return false;
+    if (d->d_model % 4 || d->d_ffn % 4 || d->d_model > 32768) return false;   // float4 paths
     if (d->dtype == WD_BF16) {
         // TMA tiles are 64 elements (128 bytes) along the reduction dimension
         if (d->d_model % 64 || d->d_ffn % 64 || (d->n_q_heads * d->head_dim) % 64) return false;
@@ -118,7 +125,7 @@ static size_t part_floats_for(const wd_model_dims* d) {
     return std::max((size_t)d->max_rows * cols, (size_t)WD_TC_MAX_SPLIT * small_rows * cols);
 }
 
-static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[16]) {
+static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[20]) {
     const size_t e = wd_elt_size(d->dtype);
     const size_t MR = d->max_rows, MA = d->max_active, hq = (size_t)d->n_q_heads * d->head_dim;
     off[0] = c.take(MR * d->d_model * 4);                       // x
@@ -131,24 +138,34 @@ static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[16]) {
     off[7] = c.take(MA * 4);                                    // row_token
     off[8] = c.take(MA * 8);                                    // row_sumexp
     off[9] = c.take(MA * 4);                                    // row_conf
-    const size_t plan_ints = 2 * MR + 2 * MA + 2 * ((size_t)d->max_batch + 1) + (size_t)d->max_batch * d->max_seq;
+    const size_t plan_ints = 2 * MR + 2 * MA + 2 * ((size_t)d->max_batch + 1) + (size_t)d->max_batch * d->max_seq +
+                             3 * (MR / 128 + (size_t)d->max_batch + 1) + (size_t)d->max_batch;
     off[10] = c.take(plan_ints * 4);                            // plan
     off[11] = c.take((1 + (size_t)d->max_batch + 3 * MA) * 4);  // result
     off[12] = plan_ints;
+    const size_t nch = (size_t)wd_unmask_chunks(d->vocab);
+    off[13] = c.take(MA * nch * 4);                             // ch_max
+    off[14] = c.take(MA * nch * 4);                             // ch_idx
+    off[15] = c.take(MA * nch * 8);                             // ch_sum
+    off[16] = c.take(MR * (size_t)(d->head_dim / 2) * 8);       // rope_tab
 }
 
 extern "C" size_t wd_workspace_bytes(const wd_model_dims* dims) {
     if (!dims_valid(dims)) return 0;
     Carve c;
-    size_t off[16];
+    size_t off[20];
     carve_ctx(dims, c, off);
     return c.off;
 }
 
+// the transposed V cache keeps the position contiguous; rows padded to 16 bytes for TMA
+static inline int seq_pad(int S) { return (S + 7) / 8 * 8; }
+
 extern "C" size_t wd_state_bytes(const wd_model_dims* d, int32_t batch, int32_t seq_len) {
     if (!dims_valid(d) || batch < 1 || seq_len < 1 || batch > d->max_batch || seq_len > d->max_seq) return 0;
-    const size_t kv = (size_t)d->n_layers * batch * d->n_kv_heads * seq_len * d->head_dim * wd_elt_size(d->dtype);
-    return wd_align_up((size_t)batch * seq_len * 4, 256) + 2 * wd_align_up(kv, 256);
+    const size_t k = (size_t)d->n_layers * batch * d->n_kv_heads * seq_len * d->head_dim * wd_elt_size(d->dtype);
+    const size_t v = (size_t)d->n_layers * batch * d->n_kv_heads * seq_pad(seq_len) * d->head_dim * wd_elt_size(d->dtype);
+    return wd_align_up((size_t)batch * seq_len * 4, 256) + wd_align_up(k, 256) + wd_align_up(v, 256);
 }
 
 extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, void* workspace,
@@ -186,7 +203,7 @@ extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, v
         c->attn_norm.push_back(w->attn_norm[l]); c->ffn_norm.push_back(w->ffn_norm[l]);
     }
     Carve cv;
-    size_t off[16];
+    size_t off[20];
     carve_ctx(dims, cv, off);
     char* base = (char*)workspace;
     c->x = (float*)(base + off[0]);
@@ -204,6 +221,10 @@ extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, v
     c->plan_ints = off[12];
     c->result = (int32_t*)(base + off[11]);
     c->result_ints = 1 + (size_t)dims->max_batch + 3 * (size_t)dims->max_active;
+    c->ch_max = (float*)(base + off[13]);
+    c->ch_idx = (int32_t*)(base + off[14]);
+    c->ch_sum = (double*)(base + off[15]);
+    c->rope_tab = (float2*)(base + off[16]);
     WD_CUDA_TRY(cudaMemset(c->result, 0, 4));
 
     if (dims->dtype == WD_BF16) {
@@ -226,6 +247,7 @@ extern "C" wd_status wd_set_gemm_impl(wd_ctx* ctx, int32_t impl) {
     if (impl != WD_GEMM_AUTO && impl != WD_GEMM_PLAIN && impl != WD_GEMM_TCGEN05) return WD_ERR_BAD_PARAM;
     if (impl == WD_GEMM_TCGEN05 && ctx->d.dtype != WD_BF16) return WD_ERR_BAD_PARAM;
     ctx->gemm_impl = impl;
+    ctx->attn_impl = impl;          // the plain setting selects the CUDA-core kernels throughout
     return WD_OK;
 }
 
@@ -254,8 +276,9 @@ struct wd_state {
     std::vector<WdSeqPlan> plans;       // of the pending step
     int32_t* ids_dev = nullptr;
     char* kcache = nullptr;             // [L][batch][Hkv][S][dh]
-    char* vcache = nullptr;
-    size_t kv_layer_bytes = 0;
+    char* vcache = nullptr;             // [L][batch][Hkv][dh][Sp]  (transposed: position contiguous)
+    size_t kv_layer_bytes = 0, v_layer_bytes = 0;
+    int Sp = 0;
     int32_t* plan_host = nullptr;       // pinned
     int32_t* result_host = nullptr;     // pinned
     int32_t* ids_host = nullptr;        // pinned staging for ids
@@ -263,6 +286,8 @@ struct wd_state {
     bool pending = false;
     int k_pending = 0, k_user = 0;
     wd_debug_taps taps = {nullptr, nullptr, nullptr};
+    bool attn_tc = false;               // tensor-core attention usable (bf16, head_dim 128)
+    CUtensorMap map_k, map_vt;
 };
 
 static void load_host_mirror(wd_state* st, const int32_t* ids, const uint8_t* decoded) {
@@ -298,7 +323,9 @@ extern "C" wd_status wd_state_create(wd_ctx* ctx, int32_t batch, int32_t seq_len
     st->seqs.resize(batch);
     const wd_model_dims& d = ctx->d;
     const size_t ids_bytes = wd_align_up((size_t)batch * seq_len * 4, 256);
+    st->Sp = seq_pad(seq_len);
     st->kv_layer_bytes = (size_t)batch * d.n_kv_heads * seq_len * d.head_dim * wd_elt_size(d.dtype);
+    st->v_layer_bytes = (size_t)batch * d.n_kv_heads * st->Sp * d.head_dim * wd_elt_size(d.dtype);
     const size_t kv = wd_align_up(st->kv_layer_bytes * d.n_layers, 256);
     st->ids_dev = (int32_t*)state_mem;
     st->kcache = (char*)state_mem + ids_bytes;
@@ -313,6 +340,17 @@ extern "C" wd_status wd_state_create(wd_ctx* ctx, int32_t batch, int32_t seq_len
         return WD_ERR_CUDA;
     }
     load_host_mirror(st, token_ids, decoded);
+    // Far-field cache rows are never read as values, but tiles of the tensor-core attention
+    // cover them (masked): start from finite contents.
+    e = cudaMemset(st->kcache, 0, st->kv_layer_bytes * d.n_layers);
+    if (e == cudaSuccess) e = cudaMemset(st->vcache, 0, st->v_layer_bytes * d.n_layers);
+    if (e != cudaSuccess) { wd_note_cuda_error(e, __FILE__, __LINE__); wd_state_destroy(st); return WD_ERR_CUDA; }
+    if (d.dtype == WD_BF16 && d.head_dim == 128) {
+        wd_status ms = wd_attn_tc_encode_cache(&st->map_k, &st->map_vt, st->kcache, st->vcache, d.n_layers,
+                                               batch * d.n_kv_heads, seq_len, st->Sp, d.head_dim);
+        if (ms != WD_OK) { wd_state_destroy(st); return ms; }
+        st->attn_tc = true;
+    }
     e = cudaMemcpy(st->ids_dev, st->ids_host, (size_t)batch * seq_len * 4, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { wd_note_cuda_error(e, __FILE__, __LINE__); wd_state_destroy(st); return WD_ERR_CUDA; }
     *out = st;
@@ -519,14 +557,26 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     const size_t o_act_off = o; o += batch + 1;
     const size_t o_vis_off = o; o += batch + 1;
     const size_t o_vis_idx = o; o += n_vis;
+    size_t n_qtiles = 0;
+    for (int b = 0; b < batch; ++b) n_qtiles += st->plans[b].done ? 0 : (st->plans[b].rows.size() + 127) / 128;
+    const size_t o_qt_seq = o; o += n_qtiles;
+    const size_t o_qt_row0 = o; o += n_qtiles;
+    const size_t o_qt_n = o; o += n_qtiles;
+    const size_t o_nvis = o; o += batch;
     if (o > c->plan_ints) return WD_ERR_CAPACITY;
     {
-        size_t r = 0, a = 0, v = 0;
+        size_t r = 0, a = 0, v = 0, qt = 0;
         for (int b = 0; b < batch; ++b) {
             const WdSeqPlan& p = st->plans[b];
             ph[o_act_off + b] = (int32_t)a;
             ph[o_vis_off + b] = (int32_t)v;
+            ph[o_nvis + b] = p.done ? 0 : (int32_t)p.vis.size();
             if (p.done) continue;
+            for (size_t t0 = 0; t0 < p.rows.size(); t0 += 128, ++qt) {
+                ph[o_qt_seq + qt] = b;
+                ph[o_qt_row0 + qt] = (int32_t)(r + t0);
+                ph[o_qt_n + qt] = (int32_t)std::min<size_t>(128, p.rows.size() - t0);
+            }
             size_t ai = 0;
             for (size_t i = 0; i < p.rows.size(); ++i) {
                 ph[o_row_seq + r] = b;
@@ -564,12 +614,14 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     GemmOut go;
     wd_status s;
 
-    wd_launch_embed(d.dtype, c->tok_embed, st->ids_dev, row_seq, row_pos, c->x, R_, D, S, d.vocab, status, stream);
+    const int Sp = st->Sp;
+    wd_launch_embed(d.dtype, c->tok_embed, st->ids_dev, row_seq, row_pos, c->x, c->rope_tab, R_, D, S, d.vocab, dh,
+                    d.rope_theta, status, stream);
     bool down_pending = false;          // x still lacks the previous block's FFN output
     GemmOut down_go = {1, 0, 0, 0};
     for (int l = 0; l < d.n_layers; ++l) {
         char* kc = st->kcache + (size_t)l * st->kv_layer_bytes;
-        char* vc = st->vcache + (size_t)l * st->kv_layer_bytes;
+        char* vc = st->vcache + (size_t)l * st->v_layer_bytes;
         // attention half
         wd_launch_rmsnorm(d.dtype, c->x, down_pending ? c->part : nullptr, down_go.n_split, down_go.split_stride,
                           c->attn_norm[l], d.rms_eps, c->xn, nullptr, R_, D, stream);
@@ -579,11 +631,18 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, qkv, 3, R_, D, c->part, c->part_floats, status, stream, &go)) != WD_OK)
             return s;
         impl_used = go.impl;
-        wd_launch_rope_scatter(d.dtype, c->part, go.n_split, go.split_stride, row_seq, row_pos, c->q, kc, vc, R_, Hq,
-                               Hkv, dh, S, d.rope_theta, stream);
+        wd_launch_rope_scatter(d.dtype, c->part, go.n_split, go.split_stride, row_seq, row_pos, c->rope_tab, c->q, kc,
+                               vc, R_, Hq, Hkv, dh, S, Sp, stream);
         float* attn_tap = st->taps.attn_out ? st->taps.attn_out + (size_t)l * R_ * hq : nullptr;
-        wd_launch_attention_plain(d.dtype, c->q, kc, vc, row_seq, vis_idx, vis_off, c->attn, attn_tap, R_, max_vis,
-                                  Hq, Hkv, dh, S, stream);
+        if (st->attn_tc && all_contig && c->attn_impl != WD_GEMM_PLAIN) {
+            if ((s = wd_attn_tc_launch(c->q, R_, (int)n_qtiles, c->plan + o_qt_seq, c->plan + o_qt_row0, c->plan + o_qt_n,
+                                       c->plan + o_nvis, &st->map_k, &st->map_vt, c->attn, attn_tap, Hq, Hkv, dh, l,
+                                       status, stream)) != WD_OK)
+                return s;
+        } else {
+            wd_launch_attention_plain(d.dtype, c->q, kc, vc, row_seq, vis_idx, vis_off, c->attn, attn_tap, R_, max_vis,
+                                      Hq, Hkv, dh, S, Sp, stream);
+        }
         WdTcSeg wo[1] = {{c->wo[l], D, c->tc.get(WD_TC_WO, l)}};
         if ((s = run_gemm(c, c->attn, &c->tc.x_map_attn, wo, 1, R_, hq, c->part, c->part_floats, status, stream, &go)) != WD_OK)
             return s;
@@ -612,7 +671,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, lm, 1, NA, D, c->logits, (size_t)d.max_active * d.vocab, status,
                           stream, &go, /*single_split=*/true)) != WD_OK)
             return s;
-        wd_launch_rowstats(c->logits, NA, d.vocab, c->row_token, c->row_sumexp, stream);
+        wd_launch_rowstats(c->logits, NA, d.vocab, c->ch_max, c->ch_idx, c->ch_sum, stream);
         if (st->taps.logits)
             WD_CUDA_TRY(cudaMemcpyAsync(st->taps.logits, c->logits, (size_t)NA * d.vocab * 4, cudaMemcpyDeviceToDevice,
                                         stream));
@@ -621,8 +680,8 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     int32_t* sel_pos = n_sel + batch;
     int32_t* sel_tok = sel_pos + (size_t)batch * std::max(k_eff, 1);
     float* sel_conf = (float*)(sel_tok + (size_t)batch * std::max(k_eff, 1));
-    wd_launch_select(c->row_token, c->row_sumexp, act_pos, act_off, 0, batch, k_eff, st->ids_dev, S, n_sel, sel_pos,
-                     sel_tok, sel_conf, c->row_conf, stream);
+    wd_launch_select(c->ch_max, c->ch_idx, c->ch_sum, wd_unmask_chunks(d.vocab), c->row_token, c->row_sumexp, act_pos,
+                     act_off, 0, batch, k_eff, st->ids_dev, S, n_sel, sel_pos, sel_tok, sel_conf, c->row_conf, stream);
     const size_t res_ints = 1 + (size_t)batch + 3 * (size_t)batch * std::max(k_eff, 1);
     WD_CUDA_TRY(cudaMemcpyAsync(st->result_host, c->result, res_ints * 4, cudaMemcpyDeviceToHost, stream));
     WD_CUDA_TRY(cudaEventRecord(st->done, stream));
@@ -635,7 +694,6 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         info->n_rows = R_; info->n_active = NA; info->n_vis = (int32_t)n_vis;
         info->n_launches = (int32_t)(wd_launch_counter - launches0); info->gemm_impl = impl_used;
     }
-    (void)all_contig;
     return WD_OK;
 }
 
@@ -715,21 +773,34 @@ extern "C" wd_status wd_op_attention(int32_t dtype, const void* q, const void* k
     if ((size_t)(n_vis + head_dim) * 4 > 200 * 1024) return WD_ERR_CAPACITY;
     // one sequence: no row->sequence table and no offsets, every row sees vis[0, n_vis)
     wd_launch_attention_plain(dtype, q, kcache, vcache, nullptr, vis, nullptr, out, nullptr, n_rows, n_vis, n_q_heads,
-                              n_kv_heads, head_dim, seq_len, (cudaStream_t)stream);
+                              n_kv_heads, head_dim, seq_len, seq_len, (cudaStream_t)stream);
     WD_CUDA_TRY(cudaGetLastError());
     return WD_OK;
 }
 
+extern "C" size_t wd_op_unmask_scratch_bytes(int32_t n, int32_t vocab) {
+    if (n < 1 || vocab < 1) return 0;
+    return (size_t)n * wd_unmask_chunks(vocab) * 16;
+}
+
 extern "C" wd_status wd_op_unmask(const float* logits, const int32_t* positions, int32_t n, int32_t vocab, int32_t k,
                                   int32_t* row_token, double* row_sumexp, float* row_conf, int32_t* sel_pos,
-                                  int32_t* sel_token, float* sel_conf, int32_t* n_sel, void* stream) {
-    if (!logits || !positions || !row_token || !row_sumexp || !row_conf || !sel_pos || !sel_token || !sel_conf || !n_sel)
+                                  int32_t* sel_token, float* sel_conf, int32_t* n_sel, void* scratch,
+                                  size_t scratch_bytes, void* stream) {
+    if (!logits || !positions || !row_token || !row_sumexp || !row_conf || !sel_pos || !sel_token || !sel_conf ||
+        !n_sel || !scratch)
         return WD_ERR_NULL;
     if (n < 1 || vocab < 1 || k < 0) return WD_ERR_BAD_PARAM;
+    if (scratch_bytes < wd_op_unmask_scratch_bytes(n, vocab)) return WD_ERR_WORKSPACE_TOO_SMALL;
+    if ((uintptr_t)scratch % 8) return WD_ERR_MISALIGNED;
     cudaStream_t st = (cudaStream_t)stream;
-    wd_launch_rowstats(logits, n, vocab, row_token, row_sumexp, st);
-    wd_launch_select(row_token, row_sumexp, positions, nullptr, n, 1, k, nullptr, 0, n_sel, sel_pos, sel_token,
-                     sel_conf, row_conf, st);
+    const int nch = wd_unmask_chunks(vocab);
+    double* ch_sum = (double*)scratch;
+    float* ch_max = (float*)(ch_sum + (size_t)n * nch);
+    int32_t* ch_idx = (int32_t*)(ch_max + (size_t)n * nch);
+    wd_launch_rowstats(logits, n, vocab, ch_max, ch_idx, ch_sum, st);
+    wd_launch_select(ch_max, ch_idx, ch_sum, nch, row_token, row_sumexp, positions, nullptr, n, 1, k, nullptr, 0, n_sel,
+                     sel_pos, sel_token, sel_conf, row_conf, st);
     WD_CUDA_TRY(cudaGetLastError());
     return WD_OK;
 }

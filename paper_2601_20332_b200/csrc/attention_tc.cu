@@ -1,0 +1,351 @@
+// Windowed bidirectional attention on the tensor cores (sm_100a), head_dim 128, bf16.
+//
+//   out[r, h, :] = softmax_j( q[r,h,:] . K[kvh, j, :] / sqrt(dh) ) V[kvh, j, :],   j in [0, n_vis)
+//
+// for the rows computed this step.  With a decoded prompt prefix the visible set of a sequence
+// is always a range [0, n_vis) (decoded prefix | external window), so K and V tiles are plain
+// TMA boxes of the cache; arbitrary index lists go through the CUDA-core kernel instead.
+//
+// One CTA per (128-row query tile of one sequence, query head):
+//   warp 0    TMA: the Q tile once, then [128 keys x 128] K boxes and [128 x 128 keys] boxes of
+//             the transposed V cache into a two-stage ring
+//   warp 1    tcgen05.mma: S = Q K^T into TMEM, then O_tile = P V into TMEM
+//   warps 2-5 one thread per query row: tcgen05.ld of its S row, online softmax in fp32
+//             (exp2 with the scale folded in), P as bf16 into shared memory in the 128-byte
+//             swizzled operand layout, then tcgen05.ld of its O_tile row accumulated in
+//             registers with the running rescale; final O / l written as bf16
+// Query rows beyond the tile's valid rows are computed on whatever the box holds and discarded
+// (rows are independent).  Keys at or beyond n_vis are masked by selection, and their V
+// columns are zeroed in shared memory, so stale or poisoned cache rows cannot leak in.
+// Every wait is bounded; on expiry the CTA records WD_ERR_DEVICE_TIMEOUT and leaves.
+#include <cstring>
+
+#include "attention_tc.h"
+#include "device_utils.cuh"
+
+namespace {
+
+using namespace wdk;
+
+constexpr int kTile = 128;                 // query rows per CTA = keys per step = head_dim
+constexpr int kAtom = kTile * 64 * 2;      // one [128 x 64] bf16 swizzle-atom column: 16 KB
+constexpr int kOperand = 2 * kAtom;        // a [128 x 128] bf16 operand: 32 KB
+constexpr int kThreads = 192;
+constexpr int kTmemCols = 256;             // S: columns 0..127, O_tile: columns 128..255
+
+struct AttnParams {
+    const int32_t* qtile_seq;    // [n_tiles] sequence of the tile
+    const int32_t* qtile_row0;   // [n_tiles] first row (index into the step's row list)
+    const int32_t* qtile_n;      // [n_tiles] valid rows
+    const int32_t* seq_nvis;     // [batch] visible positions [0, n_vis)
+    __nv_bfloat16* out;          // [rows][Hq*dh]
+    float* tap;                  // optional fp32 copy
+    int Hq, Hkv, layer;
+    float scale_log2e;           // log2(e) / sqrt(dh)
+    int32_t* status;
+    uint32_t idesc;
+};
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                    const __grid_constant__ CUtensorMap map_vt, const AttnParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    uint8_t* sQ = smem;                          // 32 KB
+    uint8_t* sP = smem + kOperand;               // 32 KB
+    uint8_t* sKV = smem + 2 * kOperand;          // 2 stages x (K 32 KB + V^T 32 KB)
+    uint64_t* bars = (uint64_t*)(smem + 2 * kOperand + 4 * kOperand);
+    // 0 q_full | 1,2 kv_full | 3,4 kv_empty | 5 s_full | 6 p_full | 7 o_full
+    uint32_t* tmem_slot = (uint32_t*)(bars + 8);
+    volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int tile = blockIdx.x, h = blockIdx.y;
+    const int b = p.qtile_seq[tile], row0 = p.qtile_row0[tile], n_valid = p.qtile_n[tile];
+    const int kvh = h / (p.Hq / p.Hkv);
+
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < 8; ++i) mbar_init(smem_u32(&bars[i]), i == 6 ? 128u : 1u);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    pdl_wait();                                   // q and the cache rows come from the previous kernel
+    const int n_vis = p.seq_nvis[b];
+    const int n_kt = (n_vis + kTile - 1) / kTile;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------------------------------------------- TMA producer
+            const uint32_t qf = smem_u32(&bars[0]);
+            mbar_expect_tx(qf, kOperand);
+            tma_load_2d(smem_u32(sQ), &map_q, qf, h * kTile, row0);
+            tma_load_2d(smem_u32(sQ) + kAtom, &map_q, qf, h * kTile + 64, row0);
+            for (int i = 0; i < n_kt; ++i) {
+                const int s = i & 1;
+                const uint32_t ph = (uint32_t)(i >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&bars[3 + s]), ph ^ 1u, abort_flag)) {
+                    *abort_flag = 1;
+                    atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
+                    break;
+                }
+                const uint32_t full = smem_u32(&bars[1 + s]);
+                const uint32_t sk = smem_u32(sKV + (size_t)s * 2 * kOperand), sv = sk + kOperand;
+                mbar_expect_tx(full, 2 * kOperand);
+                const int kv0 = i * kTile, bh = b * p.Hkv + kvh;
+                tma_load_4d(sk, &map_k, full, 0, kv0, bh, p.layer);            // keys kv0.., dims 0..63
+                tma_load_4d(sk + kAtom, &map_k, full, 64, kv0, bh, p.layer);   // dims 64..127
+                tma_load_4d(sv, &map_vt, full, kv0, 0, bh, p.layer);           // all dims, keys kv0..kv0+63
+                tma_load_4d(sv + kAtom, &map_vt, full, kv0 + 64, 0, bh, p.layer);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------------------------------------------- MMA issuer
+            bool ok = mbar_wait(smem_u32(&bars[0]), 0, abort_flag);
+            const uint64_t qd0 = make_sdesc(smem_u32(sQ)), qd1 = make_sdesc(smem_u32(sQ) + kAtom);
+            const uint64_t pd0 = make_sdesc(smem_u32(sP)), pd1 = make_sdesc(smem_u32(sP) + kAtom);
+            for (int i = 0; i < n_kt && ok; ++i) {
+                const int s = i & 1;
+                const uint32_t ph = (uint32_t)(i >> 1) & 1u;
+                if (!(ok = mbar_wait(smem_u32(&bars[1 + s]), ph, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t sk = smem_u32(sKV + (size_t)s * 2 * kOperand), sv = sk + kOperand;
+                const uint64_t kd0 = make_sdesc(sk), kd1 = make_sdesc(sk + kAtom);
+                // S = Q K^T: reduction over head_dim, 8 steps of 16
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) umma_bf16(tmem_base, qd0 + 2 * kk, kd0 + 2 * kk, p.idesc, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) umma_bf16(tmem_base, qd1 + 2 * kk, kd1 + 2 * kk, p.idesc, 1u);
+                umma_commit(smem_u32(&bars[5]));
+                // wait for P (which also means S and the previous O_tile have been read)
+                if (!(ok = mbar_wait(smem_u32(&bars[6]), (uint32_t)i & 1u, abort_flag))) break;
+                tc_fence_after();
+                const uint64_t vd0 = make_sdesc(sv), vd1 = make_sdesc(sv + kAtom);
+                // O_tile = P V: reduction over the 128 keys of the tile
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) umma_bf16(tmem_base + kTile, pd0 + 2 * kk, vd0 + 2 * kk, p.idesc, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) umma_bf16(tmem_base + kTile, pd1 + 2 * kk, vd1 + 2 * kk, p.idesc, 1u);
+                umma_commit(smem_u32(&bars[3 + s]));       // K/V stage free
+                umma_commit(smem_u32(&bars[7]));           // O_tile ready
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
+            }
+        }
+        __syncwarp();
+    } else {
+        // -------------------------------------------------------- softmax + accumulate (one row per thread)
+        const int quarter = warp & 3;
+        const int r = quarter * 32 + lane;                 // query row of the tile = TMEM lane
+        const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
+        float o[kTile];
+#pragma unroll
+        for (int c = 0; c < kTile; ++c) o[c] = 0.f;
+        float m = -INFINITY, l = 0.f;
+        bool ok = true;
+        for (int i = 0; i < n_kt; ++i) {
+            const int s = i & 1;
+            ok = ok && mbar_wait(smem_u32(&bars[5]), (uint32_t)i & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const int n_keys = min(kTile, n_vis - i * kTile);          // valid keys in this tile
+            // keys past n_vis may hold anything: zero their V columns so that 0 * garbage stays 0.
+            // Thread r owns row r (a head dim) of the transposed V tile.
+            if (n_keys < kTile) {
+                uint8_t* vt = sKV + (size_t)s * 2 * kOperand + kOperand;
+                for (int kv = n_keys; kv < kTile; ++kv) {
+                    const int a = kv >> 6, c16 = (kv & 63) >> 3, e = kv & 7;
+                    *reinterpret_cast<uint16_t*>(vt + a * kAtom + r * 128 + ((c16 ^ (r & 7)) << 4) + e * 2) = 0;
+                }
+            }
+            // pass 1: row maximum of the scaled scores
+            float mx = m;
+#pragma unroll
+            for (int c0 = 0; c0 < kTile; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(t_row + (uint32_t)c0, v);
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    const float sv = (c0 + c < n_keys) ? __uint_as_float(v[c]) * p.scale_log2e : -INFINITY;
+                    mx = fmaxf(mx, sv);
+                }
+            }
+            const float alpha = exp2f(m - mx);             // m = -inf on the first tile gives 0
+            m = mx;
+            l *= alpha;
+            // pass 2: probabilities, row sum, P as bf16 into the swizzled A-operand tile
+#pragma unroll
+            for (int c0 = 0; c0 < kTile; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(t_row + (uint32_t)c0, v);
+                float pr[32];
+#pragma unroll
+                for (int c = 0; c < 32; ++c) {
+                    pr[c] = (c0 + c < n_keys) ? exp2f(__uint_as_float(v[c]) * p.scale_log2e - mx) : 0.f;
+                    l += pr[c];
+                }
+                uint8_t* prow = sP + (c0 >> 6) * kAtom + r * 128;
+#pragma unroll
+                for (int g = 0; g < 4; ++g) {              // four 16-byte chunks of 8 keys
+                    const int c16 = ((c0 & 63) >> 3) + g;
+                    uint4 u;
+                    u.x = pack_bf16(pr[8 * g + 0], pr[8 * g + 1]);
+                    u.y = pack_bf16(pr[8 * g + 2], pr[8 * g + 3]);
+                    u.z = pack_bf16(pr[8 * g + 4], pr[8 * g + 5]);
+                    u.w = pack_bf16(pr[8 * g + 6], pr[8 * g + 7]);
+                    *reinterpret_cast<uint4*>(prow + ((c16 ^ (r & 7)) << 4)) = u;
+                }
+            }
+            tc_fence_before();
+            fence_proxy_async_smem();                      // P and the zeroed V columns -> visible to the MMA
+            mbar_arrive(smem_u32(&bars[6]));
+            // O += O_tile with the running rescale
+            ok = mbar_wait(smem_u32(&bars[7]), (uint32_t)i & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < kTile; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(t_row + (uint32_t)(kTile + c0), v);
+#pragma unroll
+                for (int c = 0; c < 32; ++c) o[c0 + c] = o[c0 + c] * alpha + __uint_as_float(v[c]);
+            }
+            tc_fence_before();
+        }
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
+        }
+        if (ok && r < n_valid) {
+            const float inv = 1.f / l;
+            const size_t base = ((size_t)(row0 + r) * p.Hq + h) * kTile;
+            uint4* dst = reinterpret_cast<uint4*>(p.out + base);
+#pragma unroll
+            for (int g = 0; g < kTile / 8; ++g) {
+                uint4 u;
+                u.x = pack_bf16(o[8 * g + 0] * inv, o[8 * g + 1] * inv);
+                u.y = pack_bf16(o[8 * g + 2] * inv, o[8 * g + 3] * inv);
+                u.z = pack_bf16(o[8 * g + 4] * inv, o[8 * g + 5] * inv);
+                u.w = pack_bf16(o[8 * g + 6] * inv, o[8 * g + 7] * inv);
+                dst[g] = u;
+            }
+            if (p.tap) {
+#pragma unroll
+                for (int c = 0; c < kTile; ++c) p.tap[base + c] = o[c] * inv;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+}  // namespace
+
+// K cache [L][BH][S][dh] -> dims (dh, S, BH, L), box (64, 128, 1, 1);
+// transposed V cache [L][BH][dh][Sp] -> dims (Sp, dh, BH, L), box (64, 128, 1, 1)
+wd_status wd_attn_tc_encode_cache(CUtensorMap* map_k, CUtensorMap* map_vt, const void* kcache, const void* vcache,
+                                  int L, int BH, int S, int Sp, int dh) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return WD_ERR_CUDA;
+    if (dh != kTile) return WD_ERR_BAD_PARAM;
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)dh, (cuuint64_t)S, (cuuint64_t)BH, (cuuint64_t)L};
+        cuuint64_t strides[3] = {(cuuint64_t)dh * 2, (cuuint64_t)S * dh * 2, (cuuint64_t)BH * S * dh * 2};
+        cuuint32_t box[4] = {64, 128, 1, 1}, estr[4] = {1, 1, 1, 1};
+        if (enc(map_k, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(kcache), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return WD_ERR_CUDA;
+    }
+    {
+        cuuint64_t dims[4] = {(cuuint64_t)Sp, (cuuint64_t)dh, (cuuint64_t)BH, (cuuint64_t)L};
+        cuuint64_t strides[3] = {(cuuint64_t)Sp * 2, (cuuint64_t)dh * Sp * 2, (cuuint64_t)BH * dh * Sp * 2};
+        cuuint32_t box[4] = {64, 128, 1, 1}, estr[4] = {1, 1, 1, 1};
+        if (enc(map_vt, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(vcache), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return WD_ERR_CUDA;
+    }
+    return WD_OK;
+}
+
+wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_t* qtile_seq, const int32_t* qtile_row0,
+                            const int32_t* qtile_n, const int32_t* seq_nvis, const CUtensorMap* map_k,
+                            const CUtensorMap* map_vt, void* out, float* tap, int Hq, int Hkv, int dh, int layer,
+                            int32_t* status, cudaStream_t stream) {
+    if (dh != kTile) return WD_ERR_BAD_PARAM;
+    if (n_tiles <= 0) return WD_OK;
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return WD_ERR_CUDA;
+    CUtensorMap mq;
+    {
+        cuuint64_t dims[2] = {(cuuint64_t)Hq * dh, (cuuint64_t)n_rows};
+        cuuint64_t strides[1] = {(cuuint64_t)Hq * dh * 2};
+        cuuint32_t box[2] = {64, 128}, estr[2] = {1, 1};
+        if (enc(&mq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(q), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return WD_ERR_CUDA;
+    }
+    AttnParams p;
+    memset(&p, 0, sizeof(p));
+    p.qtile_seq = qtile_seq; p.qtile_row0 = qtile_row0; p.qtile_n = qtile_n; p.seq_nvis = seq_nvis;
+    p.out = (__nv_bfloat16*)out; p.tap = tap;
+    p.Hq = Hq; p.Hkv = Hkv; p.layer = layer;
+    p.scale_log2e = 1.4426950408889634f / sqrtf((float)dh);
+    p.status = status;
+    p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+    const size_t smem = 6 * (size_t)kOperand + 8 * 8 + 16 + 1024;
+    WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(n_tiles, Hq);
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = wd_pdl_enabled ? 1 : 0;
+    ++wd_launch_counter;
+    WD_CUDA_TRY(cudaLaunchKernelEx(&lc, attention_tc_kernel, mq, *map_k, *map_vt, p));
+    return WD_OK;
+}

@@ -22,14 +22,16 @@
 #include <cstring>
 
 #include "gemm_tc.h"
+#include "device_utils.cuh"
 
 namespace {
+
+using namespace wdk;
 
 constexpr int kBM = 128;            // weight rows per tile (MMA M)
 constexpr int kBK = 64;             // K elements per stage = one 128-byte swizzle row
 constexpr int kStageA = kBM * kBK * 2;
 constexpr int kThreads = 192;
-constexpr uint32_t kWaitLimit = 1u << 22;
 
 struct TcParams {
     int rows, K, bn, n_split, kb_total, n_stages, tmem_cols;
@@ -42,92 +44,6 @@ struct TcParams {
     int32_t* status;
     uint32_t idesc;
 };
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
-        "selp.u32 %0, 1, 0, p;\n"
-        "}\n"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-// Bounded wait.  Returns false if the limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    for (uint32_t it = 0; it < kWaitLimit; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (it >= 128) {
-            __nanosleep(64);
-            if ((it & 255) == 0 && *abort_flag) return false;
-        }
-    }
-    return false;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c0, int c1,
-                                                 uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%3, %4}], [%2], %5;"
-        ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "l"(policy)
-        : "memory");
-}
-
-// Shared-memory matrix descriptor: K-major tile whose rows are 128 bytes, 128-byte swizzle,
-// 8-row groups 1024 bytes apart.
-__device__ __forceinline__ uint64_t make_sdesc(uint32_t saddr) {
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFF) >> 4);          // start address
-    d |= (uint64_t)1 << 16;                           // leading byte offset (unused with swizzle)
-    d |= (uint64_t)(1024 >> 4) << 32;                 // stride byte offset between 8-row groups
-    d |= (uint64_t)1 << 46;                           // descriptor version of sm_100
-    d |= (uint64_t)2 << 61;                           // 128-byte swizzle
-    return d;
-}
-
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n"
-        ".reg .pred p;\n"
-        "setp.ne.b32 p, %4, 0;\n"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
-        "}\n"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr)
-        : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
 
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w0,
@@ -157,6 +73,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     const int kb_end = (int)(((long long)(z + 1) * p.kb_total) / p.n_split);
     const int n_kb = kb_end - kb_begin;
 
+    pdl_launch_dependents();      // the next kernel may start its own prologue / weight prefetch
     if (threadIdx.x == 0) {
         for (int s = 0; s < p.n_stages; ++s) {
             mbar_init(smem_u32(&bars[s]), 1);
@@ -185,7 +102,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             uint64_t pol_stream, pol_keep;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
-            for (int i = 0; i < n_kb; ++i) {
+            // Weights never depend on earlier kernels of the stream: fill the ring with weight
+            // boxes first, then wait for the producer of the activations, then add their boxes.
+            const int n_pre = n_kb < p.n_stages ? n_kb : p.n_stages;
+            for (int i = 0; i < n_pre; ++i) {
+                const uint32_t full = smem_u32(&bars[i]);
+                mbar_expect_tx(full, (uint32_t)stage_bytes);
+                tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes), map_w, full, (kb_begin + i) * kBK, n0, pol_stream);
+            }
+            pdl_wait();
+            for (int i = 0; i < n_pre; ++i)
+                tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes) + kStageA, &map_x, smem_u32(&bars[i]),
+                                 (kb_begin + i) * kBK, tok0, pol_keep);
+            for (int i = n_pre; i < n_kb; ++i) {
                 const int s = i % p.n_stages;
                 const uint32_t ph = (uint32_t)(i / p.n_stages) & 1u;
                 if (!mbar_wait(smem_u32(&bars[p.n_stages + s]), ph ^ 1u, abort_flag)) {
@@ -244,6 +173,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         ok = __all_sync(0xffffffffu, ok);
         tc_fence_after();
+        pdl_wait();      // the previous consumer of y has finished (already implied by the data flow)
         float* yb = p.y + (size_t)z * p.split_stride + p.seg_col[seg] + n;
         for (int c = 0; c < p.bn; c += 16) {
             if (tok0 + c >= p.rows) break;
@@ -435,7 +365,17 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     const CUtensorMap& m1 = *segs[nseg > 1 ? 1 : 0].map;
     const CUtensorMap& m2 = *segs[nseg > 2 ? 2 : 0].map;
     ++wd_launch_counter;
-    gemm_tc_kernel<<<grid, kThreads, cfg.smem, stream>>>(mx, m0, m1, m2, p);
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = grid;
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = cfg.smem;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = wd_pdl_enabled ? 1 : 0;
+    WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel, mx, m0, m1, m2, p));
     WD_CUDA_TRY(cudaGetLastError());
     if (n_split_out) *n_split_out = p.n_split;
     return WD_OK;

@@ -5,9 +5,35 @@
 // plus CUDA-core versions of the GEMM and of attention that work for any dtype
 // and any index list; the fp32 configuration runs on them entirely and the
 // bf16 tensor-core kernels are cross-checked against them.
+#include <utility>
+
 #include "wd_internal.h"
+#include "device_utils.cuh"
+
+bool wd_pdl_enabled = true;
 
 namespace {
+
+using wdk::pdl_launch_dependents;
+using wdk::pdl_wait;
+
+// Launch with programmatic stream serialization: the kernel may start while its predecessor
+// is still draining; it calls pdl_wait() before touching anything the predecessor wrote.
+template <typename... KArgs, typename... Args>
+void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = wd_pdl_enabled ? 1 : 0;
+    ++wd_launch_counter;
+    cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 template <typename T> __device__ __forceinline__ float to_f(T v);
 template <> __device__ __forceinline__ float to_f<float>(float v) { return v; }
@@ -47,13 +73,26 @@ __device__ __forceinline__ float block_max(float v, float* red) {
     return warp_max(t);
 }
 
-// ---------------------------------------------------------------- embedding gather
+// ---------------------------------------------------------------- embedding gather + RoPE table
+// One block per computed row.  Also fills this step's rotary table: (cos, sin) of
+// pos * theta^(-2j/dh) for j < dh/2, evaluated in double so that the angle of a late position
+// is not limited by float rounding of the frequency.
 template <typename T>
 __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restrict__ ids,
                              const int32_t* __restrict__ row_seq, const int32_t* __restrict__ row_pos,
-                             float* __restrict__ x, int d, int S, int vocab, int32_t* status) {
+                             float* __restrict__ x, float2* __restrict__ rope_tab, int d, int S, int vocab, int dh,
+                             double log2_theta, int32_t* status) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int r = blockIdx.x;
-    const int id = ids[(size_t)row_seq[r] * S + row_pos[r]];
+    const int pos = row_pos[r];
+    for (int j = threadIdx.x; j < dh / 2; j += blockDim.x) {
+        const double ang = (double)pos * exp2(-2.0 * (double)j / (double)dh * log2_theta);
+        double sn, cs;
+        sincos(ang, &sn, &cs);
+        rope_tab[(size_t)r * (dh / 2) + j] = make_float2((float)cs, (float)sn);
+    }
+    const int id = ids[(size_t)row_seq[r] * S + pos];
     if (id < 0 || id >= vocab) {           // checked, never dereferenced
         if (threadIdx.x == 0) atomicCAS(status, 0, WD_ERR_BOUNDS);
         for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)r * d + c] = 0.f;
@@ -64,27 +103,64 @@ __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restr
 }
 
 // ---------------------------------------------------------------- RMSNorm (+ partial-sum add)
-template <typename T>
+// One block per row; columns in groups of four (float4 loads, all slices of a group in flight
+// together).  d must be a multiple of 4.
+template <typename T> struct Vec4;
+template <> struct Vec4<float> {
+    static __device__ __forceinline__ void store(float* p, float a, float b, float c, float d) {
+        *reinterpret_cast<float4*>(p) = make_float4(a, b, c, d);
+    }
+};
+template <> struct Vec4<__nv_bfloat16> {
+    static __device__ __forceinline__ void store(__nv_bfloat16* p, float a, float b, float c, float d) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+        uint2 u;
+        u.x = *reinterpret_cast<uint32_t*>(&lo);
+        u.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(p) = u;
+    }
+};
+
+template <typename T, int MAXV>
 __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
                                size_t split_stride, const float* __restrict__ gain, float eps,
                                T* __restrict__ xn, const int32_t* __restrict__ row_idx, int d) {
     __shared__ float red[32];
+    pdl_launch_dependents();
+    pdl_wait();
     const int i = blockIdx.x;
     const int r = row_idx ? row_idx[i] : i;
     float* xr = x + (size_t)r * d;
+    const int nv = d >> 2;
+    float4 v[MAXV];
     float ss = 0.f;
-    for (int c = threadIdx.x; c < d; c += blockDim.x) {
-        float v = xr[c];
-        if (part) {
-            for (int s = 0; s < n_split; ++s) v += part[s * split_stride + (size_t)r * d + c];
-            xr[c] = v;
+#pragma unroll
+    for (int u = 0; u < MAXV; ++u) {
+        const int c4 = threadIdx.x + u * blockDim.x;
+        if (c4 < nv) {
+            float4 a = reinterpret_cast<const float4*>(xr)[c4];
+            if (part) {
+                for (int s = 0; s < n_split; ++s) {
+                    const float4 b = reinterpret_cast<const float4*>(part + s * split_stride + (size_t)r * d)[c4];
+                    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
+                }
+                reinterpret_cast<float4*>(xr)[c4] = a;
+            }
+            v[u] = a;
+            ss += a.x * a.x + a.y * a.y + a.z * a.z + a.w * a.w;
         }
-        ss += v * v;
     }
     ss = block_sum(ss, red);
     const float inv = rsqrtf(ss / (float)d + eps);
-    for (int c = threadIdx.x; c < d; c += blockDim.x)
-        xn[(size_t)i * d + c] = from_f<T>(xr[c] * inv * gain[c]);
+#pragma unroll
+    for (int u = 0; u < MAXV; ++u) {
+        const int c4 = threadIdx.x + u * blockDim.x;
+        if (c4 < nv) {
+            const float4 g = reinterpret_cast<const float4*>(gain)[c4];
+            Vec4<T>::store(xn + (size_t)i * d + 4 * c4, v[u].x * inv * g.x, v[u].y * inv * g.y, v[u].z * inv * g.z,
+                           v[u].w * inv * g.w);
+        }
+    }
 }
 
 // ---------------------------------------------------------------- CUDA-core GEMM
@@ -94,6 +170,8 @@ __global__ void gemm_plain_kernel(const T* __restrict__ x, const T* __restrict__
                                   int rows, int n, int k, int ldy) {
     __shared__ float xs[32][33];
     __shared__ float ws[64][33];
+    pdl_launch_dependents();
+    pdl_wait();
     const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;          // 16 x 16
     const int r0 = blockIdx.y * 32, n0 = blockIdx.x * 64;
     float acc[2][4] = {};
@@ -132,46 +210,42 @@ __global__ void gemm_plain_kernel(const T* __restrict__ x, const T* __restrict__
 }
 
 // ---------------------------------------------------------------- RoPE + K/V scatter
-// One block per row.  Rotation pairs (j, j + dh/2) by pos * theta^(-2j/dh), fp32 math.
+// grid (row, group of 4 heads); 256 threads.  Adds the split-K slices of the fused q/k/v
+// projection, rotates q and k heads by the row's table, writes q and the K/V cache rows.
+// K cache [batch][Hkv][S][dh]; V cache transposed [batch][Hkv][dh][Sp] so that attention can
+// read V tiles with the key position contiguous.
 template <typename T>
 __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
                                     const int32_t* __restrict__ row_seq, const int32_t* __restrict__ row_pos,
-                                    T* __restrict__ q, T* __restrict__ kcache, T* __restrict__ vcache,
-                                    int Hq, int Hkv, int dh, int S, float log2_theta) {
+                                    const float2* __restrict__ rope_tab, T* __restrict__ q, T* __restrict__ kcache,
+                                    T* __restrict__ vcache, int Hq, int Hkv, int dh, int S, int Sp) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int r = blockIdx.x;
     const int pos = row_pos[r], b = row_seq[r];
     const int half = dh >> 1;
     const int ncol = (Hq + 2 * Hkv) * dh;
     const float* pr = part + (size_t)r * ncol;
-    auto col = [&](int c) {
-        float v = 0.f;
-        for (int s = 0; s < n_split; ++s) v += pr[s * split_stride + c];
-        return v;
-    };
-    // q and k heads: (Hq + Hkv) * half pairs
-    const int n_pairs = (Hq + Hkv) * half;
-    for (int i = threadIdx.x; i < n_pairs; i += blockDim.x) {
-        const int h = i / half, j = i - h * half;
-        const float inv_freq = exp2f(-2.f * (float)j / (float)dh * log2_theta);
-        float sn, cs;
-        sincosf((float)pos * inv_freq, &sn, &cs);
-        const float a = col(h * dh + j), bb = col(h * dh + j + half);
-        const float ra = a * cs - bb * sn, rb = bb * cs + a * sn;
-        if (h < Hq) {
-            T* dst = q + ((size_t)r * Hq + h) * dh;
+    const int h0 = blockIdx.y * 4;
+    for (int i = threadIdx.x; i < 4 * half; i += blockDim.x) {
+        const int h = h0 + i / half, j = i % half;
+        if (h >= Hq + 2 * Hkv) break;
+        float a = 0.f, bb = 0.f;
+        for (int s = 0; s < n_split; ++s) {
+            a += pr[s * split_stride + h * dh + j];
+            bb += pr[s * split_stride + h * dh + j + half];
+        }
+        if (h < Hq + Hkv) {
+            const float2 cs = rope_tab[(size_t)r * half + j];
+            const float ra = a * cs.x - bb * cs.y, rb = bb * cs.x + a * cs.y;
+            T* dst = h < Hq ? q + ((size_t)r * Hq + h) * dh : kcache + (((size_t)b * Hkv + (h - Hq)) * S + pos) * dh;
             dst[j] = from_f<T>(ra);
             dst[j + half] = from_f<T>(rb);
         } else {
-            const int kh = h - Hq;
-            T* dst = kcache + (((size_t)b * Hkv + kh) * S + pos) * dh;
-            dst[j] = from_f<T>(ra);
-            dst[j + half] = from_f<T>(rb);
+            T* dst = vcache + ((size_t)b * Hkv + (h - Hq - Hkv)) * dh * Sp + pos;
+            dst[(size_t)j * Sp] = from_f<T>(a);
+            dst[(size_t)(j + half) * Sp] = from_f<T>(bb);
         }
-    }
-    const int v0 = (Hq + Hkv) * dh;
-    for (int i = threadIdx.x; i < Hkv * dh; i += blockDim.x) {
-        const int kh = i / dh, c = i - kh * dh;
-        vcache[(((size_t)b * Hkv + kh) * S + pos) * dh + c] = from_f<T>(col(v0 + i));
     }
 }
 
@@ -183,16 +257,18 @@ __global__ void attention_plain_kernel(const T* __restrict__ q, const T* __restr
                                        const T* __restrict__ vcache, const int32_t* __restrict__ row_seq,
                                        const int32_t* __restrict__ vis_idx, const int32_t* __restrict__ vis_off,
                                        T* __restrict__ out, float* __restrict__ tap, int nv_single, int Hq,
-                                       int Hkv, int dh, int S) {
+                                       int Hkv, int dh, int S, int Sp) {
     extern __shared__ float sc[];                 // [n_vis] scores, then dh floats of q
     __shared__ float red[32];
+    pdl_launch_dependents();
+    pdl_wait();
     const int r = blockIdx.x, h = blockIdx.y;
     const int b = row_seq ? row_seq[r] : 0;
     const int v0 = vis_off ? vis_off[b] : 0;
     const int nv = vis_off ? vis_off[b + 1] - v0 : nv_single;
     const int kvh = h / (Hq / Hkv);
     const T* kb = kcache + ((size_t)b * Hkv + kvh) * S * dh;
-    const T* vb = vcache + ((size_t)b * Hkv + kvh) * S * dh;
+    const T* vb = vcache + ((size_t)b * Hkv + kvh) * dh * Sp;     // [dh][Sp]
     float* qs = sc + nv;
     for (int c = threadIdx.x; c < dh; c += blockDim.x) qs[c] = to_f(q[((size_t)r * Hq + h) * dh + c]);
     __syncthreads();
@@ -218,36 +294,49 @@ __global__ void attention_plain_kernel(const T* __restrict__ q, const T* __restr
     sum = block_sum(sum, red);
     __syncthreads();
     const float inv = 1.f / sum;
-    for (int c = threadIdx.x; c < dh; c += blockDim.x) {
+    // V is stored transposed ([dh][Sp]): each warp takes head dims c = wid, wid + nw, ... and its
+    // lanes stride over the visible positions, so consecutive lanes read consecutive positions
+    for (int c = wid; c < dh; c += nw) {
+        const T* vr = vb + (size_t)c * Sp;
         float a = 0.f;
-        for (int j = 0; j < nv; ++j) a += sc[j] * to_f(vb[(size_t)vis_idx[v0 + j] * dh + c]);
-        a *= inv;
-        const size_t o = ((size_t)r * Hq + h) * dh + c;
-        out[o] = from_f<T>(a);
-        if (tap) tap[o] = a;
+        for (int j = lane; j < nv; j += 32) a += sc[j] * to_f(vr[vis_idx[v0 + j]]);
+        a = warp_sum(a) * inv;
+        if (lane == 0) {
+            const size_t o = ((size_t)r * Hq + h) * dh + c;
+            out[o] = from_f<T>(a);
+            if (tap) tap[o] = a;
+        }
     }
 }
 
 // ---------------------------------------------------------------- SwiGLU
+// four columns per thread; F must be a multiple of 4
 template <typename T>
 __global__ void swiglu_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
                               T* __restrict__ h, int n_rows, int F) {
-    const size_t total = (size_t)n_rows * F;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int f4 = F >> 2;
+    const size_t total = (size_t)n_rows * f4;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (size_t)gridDim.x * blockDim.x) {
-        const size_t r = i / F, c = i - r * F;
-        float g = 0.f, u = 0.f;
+        const size_t r = i / f4, c4 = i - r * f4;
+        float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
         for (int s = 0; s < n_split; ++s) {
-            const float* p = part + s * split_stride + r * 2 * F;
-            g += p[c];
-            u += p[F + c];
+            const float4* p = reinterpret_cast<const float4*>(part + s * split_stride + r * 2 * F);
+            const float4 a = p[c4], b = p[f4 + c4];
+            g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w;
+            u.x += b.x; u.y += b.y; u.z += b.z; u.w += b.w;
         }
-        h[i] = from_f<T>(g / (1.f + __expf(-g)) * u);
+        Vec4<T>::store(h + r * F + 4 * c4, g.x / (1.f + __expf(-g.x)) * u.x, g.y / (1.f + __expf(-g.y)) * u.y,
+                       g.z / (1.f + __expf(-g.z)) * u.z, g.w / (1.f + __expf(-g.w)) * u.w);
     }
 }
 
 __global__ void residual_add_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
                                     size_t split_stride, float* __restrict__ tap, size_t total) {
+    pdl_launch_dependents();
+    pdl_wait();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (size_t)gridDim.x * blockDim.x) {
         float v = x[i];
@@ -258,27 +347,31 @@ __global__ void residual_add_kernel(float* __restrict__ x, const float* __restri
 }
 
 // ---------------------------------------------------------------- unmask reduction
-// One block of 256 threads per active row, the same reduction order for every row:
-// thread-strided scan, warp-shuffle tree, then the 8 warp results in lane order.
-// The sum of exponentials is taken in double precision: it decides which rows are unmasked,
-// and in double the ranking agrees with an exact evaluation of the same float logits except
-// for gaps at the 1e-13 level (the work is a few million exps per step).
+// Stage 1: grid (active row, vocabulary chunk).  Per chunk: maximum with the lowest index
+// (thread-strided scan, warp-shuffle tree, 8 warp results in order) and the sum of
+// exp(l - chunk max) in double.  Stage 2 (select_kernel) merges the chunks of a row in chunk
+// order, which is the same fixed order for every row, so identical logit rows give identical
+// bits.  The sums are in double because they decide which rows are unmasked: in double the
+// ranking agrees with an exact evaluation of the same float logits down to 1e-13 gaps.
 __device__ __forceinline__ double warp_sum_d(double v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
 
-__global__ void rowstats_kernel(const float* __restrict__ logits, int V, int32_t* __restrict__ row_token,
-                                double* __restrict__ row_sumexp) {
+__global__ void rowstats_kernel(const float* __restrict__ logits, int V, int chunk, float* __restrict__ ch_max,
+                                int32_t* __restrict__ ch_idx, double* __restrict__ ch_sum) {
     __shared__ float s_val[8];
     __shared__ int s_idx[8];
     __shared__ double s_sum[8];
     __shared__ float s_max;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int v0 = blockIdx.y * chunk, v1 = min(V, v0 + chunk);
     const float* lr = logits + (size_t)blockIdx.x * V;
     float best = -INFINITY;
     int bi = 0x7fffffff;
-    for (int v = threadIdx.x; v < V; v += 256) {
+    for (int v = v0 + threadIdx.x; v < v1; v += 256) {
         const float l = lr[v];
         if (l > best) { best = l; bi = v; }       // strictly greater keeps the lowest index
     }
@@ -297,38 +390,55 @@ __global__ void rowstats_kernel(const float* __restrict__ logits, int V, int32_t
         for (int j = 1; j < 8; ++j)
             if (s_val[j] > b || (s_val[j] == b && s_idx[j] < i)) { b = s_val[j]; i = s_idx[j]; }
         s_max = b;
-        row_token[blockIdx.x] = i;
+        ch_max[(size_t)blockIdx.x * gridDim.y + blockIdx.y] = b;
+        ch_idx[(size_t)blockIdx.x * gridDim.y + blockIdx.y] = i;
     }
     __syncthreads();
     const double m = (double)s_max;
     double sum = 0.0;
-    for (int v = threadIdx.x; v < V; v += 256) sum += exp((double)lr[v] - m);
+    for (int v = v0 + threadIdx.x; v < v1; v += 256) sum += exp((double)lr[v] - m);
     sum = warp_sum_d(sum);
     if (lane == 0) s_sum[w] = sum;
     __syncthreads();
     if (threadIdx.x == 0) {
         double t = 0.0;
         for (int j = 0; j < 8; ++j) t += s_sum[j];
-        row_sumexp[blockIdx.x] = t;
+        ch_sum[(size_t)blockIdx.x * gridDim.y + blockIdx.y] = t;
     }
 }
 
-// One block per sequence.  rank(i) = #{j : s_j < s_i or (s_j == s_i and pos_j < pos_i)}; positions
-// are ascending inside a sequence, so "pos_j < pos_i" is "j < i".
-__global__ void select_kernel(const int32_t* __restrict__ row_token, const double* __restrict__ row_sumexp,
-                              const int32_t* __restrict__ act_pos, const int32_t* __restrict__ act_off,
-                              int n_single, int k, int32_t* __restrict__ ids, int S, int32_t* __restrict__ n_sel,
-                              int32_t* __restrict__ sel_pos, int32_t* __restrict__ sel_token,
-                              float* __restrict__ sel_conf, float* __restrict__ row_conf) {
+// One block per sequence.  Merge the chunk statistics of every active row, then
+// rank(i) = #{j : s_j < s_i or (s_j == s_i and pos_j < pos_i)}; positions are ascending inside a
+// sequence, so "pos_j < pos_i" is "j < i".
+__global__ void select_kernel(const float* __restrict__ ch_max, const int32_t* __restrict__ ch_idx,
+                              const double* __restrict__ ch_sum, int n_chunks, int32_t* __restrict__ row_token,
+                              double* __restrict__ row_sumexp, const int32_t* __restrict__ act_pos,
+                              const int32_t* __restrict__ act_off, int n_single, int k, int32_t* __restrict__ ids,
+                              int S, int32_t* __restrict__ n_sel, int32_t* __restrict__ sel_pos,
+                              int32_t* __restrict__ sel_token, float* __restrict__ sel_conf,
+                              float* __restrict__ row_conf) {
+    pdl_launch_dependents();
+    pdl_wait();
     const int b = blockIdx.x;
     const int a0 = act_off ? act_off[b] : 0;
     const int n = act_off ? act_off[b + 1] - a0 : n_single;
     const int kk = min(k, n);
     if (threadIdx.x == 0) n_sel[b] = kk;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const size_t base = (size_t)(a0 + i) * n_chunks;
+        float m = ch_max[base];
+        int tok = ch_idx[base];
+        for (int c = 1; c < n_chunks; ++c)
+            if (ch_max[base + c] > m) { m = ch_max[base + c]; tok = ch_idx[base + c]; }   // chunks ascend in index
+        double s = 0.0;
+        for (int c = 0; c < n_chunks; ++c) s += ch_sum[base + c] * exp((double)ch_max[base + c] - (double)m);
+        row_token[a0 + i] = tok;
+        row_sumexp[a0 + i] = s;
+        if (row_conf) row_conf[a0 + i] = (float)(1.0 / s);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
         const double si = row_sumexp[a0 + i];
-        const float conf = (float)(1.0 / si);
-        if (row_conf) row_conf[a0 + i] = conf;
         int rank = 0;
         for (int j = 0; j < n; ++j) {
             const double sj = row_sumexp[a0 + j];
@@ -338,7 +448,7 @@ __global__ void select_kernel(const int32_t* __restrict__ row_token, const doubl
             const int pos = act_pos[a0 + i], tok = row_token[a0 + i];
             sel_pos[b * k + rank] = pos;
             sel_token[b * k + rank] = tok;
-            sel_conf[b * k + rank] = conf;
+            sel_conf[b * k + rank] = (float)(1.0 / si);
             if (ids) ids[(size_t)b * S + pos] = tok;
         }
     }
@@ -348,81 +458,89 @@ __device__ int32_t g_op_status;
 
 }  // namespace
 
+thread_local long long wd_launch_counter = 0;
+
 // ---------------------------------------------------------------- launchers
 
 #define WD_DISPATCH(dtype, ...)                                   \
     do {                                                          \
-        ++wd_launch_counter;                                      \
         if ((dtype) == WD_F32) { using T = float; __VA_ARGS__; }  \
         else { using T = __nv_bfloat16; __VA_ARGS__; }            \
     } while (0)
 
-thread_local long long wd_launch_counter = 0;
-
 void wd_launch_embed(int dtype, const void* embed, const int32_t* ids, const int32_t* row_seq,
-                     const int32_t* row_pos, float* x, int n_rows, int d, int S, int vocab,
-                     int32_t* status, cudaStream_t st) {
+                     const int32_t* row_pos, float* x, float2* rope_tab, int n_rows, int d, int S, int vocab, int dh,
+                     float theta, int32_t* status, cudaStream_t st) {
     if (n_rows <= 0) return;
-    WD_DISPATCH(dtype, embed_kernel<T><<<n_rows, 256, 0, st>>>((const T*)embed, ids, row_seq, row_pos, x, d,
-                                                               S, vocab, status));
+    const double l2 = log2((double)theta);
+    WD_DISPATCH(dtype, launch_pdl(embed_kernel<T>, dim3(n_rows), dim3(256), 0, st, (const T*)embed, ids, row_seq,
+                                  row_pos, x, rope_tab, d, S, vocab, dh, l2, status));
 }
 
 void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size_t split_stride,
                        const float* gain, float eps, void* xn, const int32_t* row_idx, int n_rows,
                        int d, cudaStream_t st) {
     if (n_rows <= 0) return;
-    WD_DISPATCH(dtype, rmsnorm_kernel<T><<<n_rows, 256, 0, st>>>(x, part, n_split, split_stride, gain, eps,
-                                                                 (T*)xn, row_idx, d));
+    // 256 threads x MAXV float4 per thread cover d; pick the smallest MAXV that fits
+    const int nv = d >> 2;
+    if (nv <= 256 * 2) {
+        WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 2>, dim3(n_rows), dim3(256), 0, st, x, part, n_split,
+                                      split_stride, gain, eps, (T*)xn, row_idx, d));
+    } else if (nv <= 256 * 4) {
+        WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 4>, dim3(n_rows), dim3(256), 0, st, x, part, n_split,
+                                      split_stride, gain, eps, (T*)xn, row_idx, d));
+    } else {
+        WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 8>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split,
+                                      split_stride, gain, eps, (T*)xn, row_idx, d));
+    }
 }
 
 void wd_launch_gemm_plain(int dtype, const void* x, const void* w, float* y, int rows, int n, int k,
                           int ldy, cudaStream_t st) {
     if (rows <= 0 || n <= 0) return;
     dim3 grid(wd_ceil_div(n, 64), wd_ceil_div(rows, 32));
-    WD_DISPATCH(dtype, gemm_plain_kernel<T><<<grid, 256, 0, st>>>((const T*)x, (const T*)w, y, rows, n, k, ldy));
+    WD_DISPATCH(dtype, launch_pdl(gemm_plain_kernel<T>, grid, dim3(256), 0, st, (const T*)x, (const T*)w, y, rows, n,
+                                  k, ldy));
 }
 
 void wd_launch_rope_scatter(int dtype, const float* part, int n_split, size_t split_stride,
-                            const int32_t* row_seq, const int32_t* row_pos, void* q, void* kcache,
-                            void* vcache, int n_rows, int Hq, int Hkv, int dh, int S, float theta,
+                            const int32_t* row_seq, const int32_t* row_pos, const float2* rope_tab, void* q,
+                            void* kcache, void* vcache, int n_rows, int Hq, int Hkv, int dh, int S, int Sp,
                             cudaStream_t st) {
     if (n_rows <= 0) return;
-    const float l2 = log2f(theta);
-    WD_DISPATCH(dtype, rope_scatter_kernel<T><<<n_rows, 256, 0, st>>>(part, n_split, split_stride, row_seq,
-                                                                      row_pos, (T*)q, (T*)kcache, (T*)vcache,
-                                                                      Hq, Hkv, dh, S, l2));
+    dim3 grid(n_rows, wd_ceil_div(Hq + 2 * Hkv, 4));
+    WD_DISPATCH(dtype, launch_pdl(rope_scatter_kernel<T>, grid, dim3(256), 0, st, part, n_split, split_stride,
+                                  row_seq, row_pos, rope_tab, (T*)q, (T*)kcache, (T*)vcache, Hq, Hkv, dh, S, Sp));
 }
 
 void wd_launch_attention_plain(int dtype, const void* q, const void* kcache, const void* vcache,
                                const int32_t* row_seq, const int32_t* vis_idx, const int32_t* vis_off,
                                void* out, float* tap, int n_rows, int max_vis, int Hq, int Hkv, int dh,
-                               int S, cudaStream_t st) {
+                               int S, int Sp, cudaStream_t st) {
     if (n_rows <= 0) return;
     const size_t smem = (size_t)(max_vis + dh) * sizeof(float);
     dim3 grid(n_rows, Hq);
-    ++wd_launch_counter;
     if (dtype == WD_F32) {
         if (smem > 48 * 1024)
             cudaFuncSetAttribute(attention_plain_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attention_plain_kernel<float><<<grid, 128, smem, st>>>((const float*)q, (const float*)kcache,
-                                                               (const float*)vcache, row_seq, vis_idx, vis_off,
-                                                               (float*)out, tap, max_vis, Hq, Hkv, dh, S);
+        launch_pdl(attention_plain_kernel<float>, grid, dim3(128), smem, st, (const float*)q, (const float*)kcache,
+                   (const float*)vcache, row_seq, vis_idx, vis_off, (float*)out, tap, max_vis, Hq, Hkv, dh, S, Sp);
     } else {
         using T = __nv_bfloat16;
         if (smem > 48 * 1024)
             cudaFuncSetAttribute(attention_plain_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        attention_plain_kernel<T><<<grid, 128, smem, st>>>((const T*)q, (const T*)kcache, (const T*)vcache,
-                                                           row_seq, vis_idx, vis_off, (T*)out, tap, max_vis, Hq, Hkv, dh,
-                                                           S);
+        launch_pdl(attention_plain_kernel<T>, grid, dim3(128), smem, st, (const T*)q, (const T*)kcache,
+                   (const T*)vcache, row_seq, vis_idx, vis_off, (T*)out, tap, max_vis, Hq, Hkv, dh, S, Sp);
     }
 }
 
 void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_stride, void* h,
                       int n_rows, int F, cudaStream_t st) {
     if (n_rows <= 0) return;
-    const size_t total = (size_t)n_rows * F;
-    const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
-    WD_DISPATCH(dtype, swiglu_kernel<T><<<blocks, 256, 0, st>>>(part, n_split, split_stride, (T*)h, n_rows, F));
+    const size_t total = (size_t)n_rows * (F >> 2);
+    const int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
+    WD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, dim3(blocks), dim3(256), 0, st, part, n_split, split_stride,
+                                  (T*)h, n_rows, F));
 }
 
 void wd_launch_residual_add(float* x, const float* part, int n_split, size_t split_stride,
@@ -430,25 +548,31 @@ void wd_launch_residual_add(float* x, const float* part, int n_split, size_t spl
     if (n_rows <= 0) return;
     const size_t total = (size_t)n_rows * d;
     const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
-    ++wd_launch_counter;
-    residual_add_kernel<<<blocks, 256, 0, st>>>(x, part, n_split, split_stride, tap, total);
+    launch_pdl(residual_add_kernel, dim3(blocks), dim3(256), 0, st, x, part, n_split, split_stride, tap, total);
 }
 
-void wd_launch_rowstats(const float* logits, int n, int V, int32_t* row_token, double* row_sumexp,
+int wd_unmask_chunks(int V) {
+    int n = (V + 4095) / 4096;            // about 4096 logits per block
+    if (n < 1) n = 1;
+    if (n > WD_UNMASK_MAX_CHUNKS) n = WD_UNMASK_MAX_CHUNKS;
+    return n;
+}
+
+void wd_launch_rowstats(const float* logits, int n, int V, float* ch_max, int32_t* ch_idx, double* ch_sum,
                         cudaStream_t st) {
     if (n <= 0) return;
-    ++wd_launch_counter;
-    rowstats_kernel<<<n, 256, 0, st>>>(logits, V, row_token, row_sumexp);
+    const int nch = wd_unmask_chunks(V);
+    const int chunk = (V + nch - 1) / nch;
+    launch_pdl(rowstats_kernel, dim3(n, nch), dim3(256), 0, st, logits, V, chunk, ch_max, ch_idx, ch_sum);
 }
 
-void wd_launch_select(const int32_t* row_token, const double* row_sumexp, const int32_t* act_pos,
-                      const int32_t* act_off, int n_single, int batch, int k, int32_t* ids, int S,
-                      int32_t* n_sel, int32_t* sel_pos, int32_t* sel_token, float* sel_conf,
-                      float* row_conf, cudaStream_t st) {
+void wd_launch_select(const float* ch_max, const int32_t* ch_idx, const double* ch_sum, int n_chunks,
+                      int32_t* row_token, double* row_sumexp, const int32_t* act_pos, const int32_t* act_off,
+                      int n_single, int batch, int k, int32_t* ids, int S, int32_t* n_sel, int32_t* sel_pos,
+                      int32_t* sel_token, float* sel_conf, float* row_conf, cudaStream_t st) {
     if (batch <= 0) return;
-    ++wd_launch_counter;
-    select_kernel<<<batch, 256, 0, st>>>(row_token, row_sumexp, act_pos, act_off, n_single, k, ids, S, n_sel,
-                                         sel_pos, sel_token, sel_conf, row_conf);
+    launch_pdl(select_kernel, dim3(batch), dim3(256), 0, st, ch_max, ch_idx, ch_sum, n_chunks, row_token, row_sumexp,
+               act_pos, act_off, n_single, k, ids, S, n_sel, sel_pos, sel_token, sel_conf, row_conf);
 }
 
 int32_t* wd_op_status_ptr() {

@@ -53,14 +53,15 @@ void wd_commit_seq(WdSeq& s, const WdSeqPlan& plan, const int32_t* positions,
 // `status` is a device int32: kernels store WD_ERR_* there on a failed check.
 // ---------------------------------------------------------------------------
 
-// x[r,:] = embed[ids[row_seq[r]*S + row_pos[r]], :]  (float residual stream)
+// x[r,:] = embed[ids[row_seq[r]*S + row_pos[r]], :]  (float residual stream); also fills the
+// rotary table rope_tab[r][j] = (cos, sin)(row_pos[r] * theta^(-2j/dh)), j < dh/2
 void wd_launch_embed(int dtype, const void* embed, const int32_t* ids, const int32_t* row_seq,
-                     const int32_t* row_pos, float* x, int n_rows, int d, int S, int vocab,
-                     int32_t* status, cudaStream_t st);
+                     const int32_t* row_pos, float* x, float2* rope_tab, int n_rows, int d, int S, int vocab, int dh,
+                     float theta, int32_t* status, cudaStream_t st);
 
 // x += sum_s part[s] (if part != null); xn = rmsnorm(x) * gain, written as `dtype`.
 // With row_idx != null the rows x[row_idx[i]] are read (no partial add, x not written)
-// and xn[i] is written: used for the final norm over the active rows only.
+// and xn[i] is written: used for the final norm over the active rows only.  d % 4 == 0.
 void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size_t split_stride,
                        const float* gain, float eps, void* xn, const int32_t* row_idx, int n_rows,
                        int d, cudaStream_t st);
@@ -71,21 +72,22 @@ void wd_launch_gemm_plain(int dtype, const void* x, const void* w, float* y, int
 
 // qkv partials -> RoPE -> q (dtype) and K/V cache rows.
 //   part: [n_split][n_rows][(Hq+2Hkv)*dh] float, columns = [q | k | v]
-//   kcache/vcache: [batch][Hkv][S][dh] (this layer's slice)
+//   kcache: [batch][Hkv][S][dh]; vcache: [batch][Hkv][dh][Sp] (this layer's slices)
 void wd_launch_rope_scatter(int dtype, const float* part, int n_split, size_t split_stride,
-                            const int32_t* row_seq, const int32_t* row_pos, void* q, void* kcache,
-                            void* vcache, int n_rows, int Hq, int Hkv, int dh, int S, float theta,
+                            const int32_t* row_seq, const int32_t* row_pos, const float2* rope_tab, void* q,
+                            void* kcache, void* vcache, int n_rows, int Hq, int Hkv, int dh, int S, int Sp,
                             cudaStream_t st);
 
 // general (index-list) attention, CUDA cores.
-//   seq_row_off[batch+1]: rows of sequence b are [off[b], off[b+1])
+//   row_seq[r]: sequence of row r (null: one sequence)
 //   vis_idx: concatenated visible positions, sequence b at [vis_off[b], vis_off[b+1])
+//            (vis_off null: one sequence seeing vis_idx[0, max_vis))
 void wd_launch_attention_plain(int dtype, const void* q, const void* kcache, const void* vcache,
                                const int32_t* row_seq, const int32_t* vis_idx, const int32_t* vis_off,
                                void* out, float* tap, int n_rows, int max_vis, int Hq, int Hkv, int dh,
-                               int S, cudaStream_t st);
+                               int S, int Sp, cudaStream_t st);
 
-// h = silu(gate) * up from partials [n_split][n_rows][2F] (columns = [gate | up])
+// h = silu(gate) * up from partials [n_split][n_rows][2F] (columns = [gate | up]); F % 4 == 0
 void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_stride, void* h,
                       int n_rows, int F, cudaStream_t st);
 
@@ -93,16 +95,20 @@ void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_st
 void wd_launch_residual_add(float* x, const float* part, int n_split, size_t split_stride,
                             float* tap, int n_rows, int d, cudaStream_t st);
 
-// per-row (max, lowest argmax, sum exp(l - max) in double) of logits [n, V]
-void wd_launch_rowstats(const float* logits, int n, int V, int32_t* row_token, double* row_sumexp,
+// unmask stage 1: per (row, vocabulary chunk) maximum, lowest argmax, sum exp(l - max) in double;
+// outputs are [n][wd_unmask_chunks(V)]
+#define WD_UNMASK_MAX_CHUNKS 64
+int wd_unmask_chunks(int V);
+void wd_launch_rowstats(const float* logits, int n, int V, float* ch_max, int32_t* ch_idx, double* ch_sum,
                         cudaStream_t st);
 
-// per sequence: rank active rows by (sumexp ascending, position ascending), emit the first
-// min(k, n_b); optionally write the chosen ids into ids[b*S + pos].  act_off == null means one
-// sequence holding rows [0, n_single).
-void wd_launch_select(const int32_t* row_token, const double* row_sumexp, const int32_t* act_pos,
-                      const int32_t* act_off, int n_single, int batch, int k, int32_t* ids, int S,
-                      int32_t* n_sel, int32_t* sel_pos, int32_t* sel_token, float* sel_conf,
-                      float* row_conf, cudaStream_t st);
+// unmask stage 2, per sequence: merge the chunks of each row into (token, sum exp), rank the
+// rows by (sum exp ascending, position ascending), emit the first min(k, n_b); optionally write
+// the chosen ids into ids[b*S + pos].  act_off == null: one sequence holding rows [0, n_single).
+void wd_launch_select(const float* ch_max, const int32_t* ch_idx, const double* ch_sum, int n_chunks,
+                      int32_t* row_token, double* row_sumexp, const int32_t* act_pos, const int32_t* act_off,
+                      int n_single, int batch, int k, int32_t* ids, int S, int32_t* n_sel, int32_t* sel_pos,
+                      int32_t* sel_token, float* sel_conf, float* row_conf, cudaStream_t st);
 
 int32_t* wd_op_status_ptr();   // device address of the single-operation status word
+extern bool wd_pdl_enabled;    // programmatic dependent launch on every kernel (default on)

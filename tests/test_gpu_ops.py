@@ -88,7 +88,7 @@ def test_attention_vs_oracle(dtype, rows, nv, Hq, Hkv, dh, S):
         kc[:, torch.as_tensor(hidden, device=DEV)] = float("nan")
         vc[:, torch.as_tensor(hidden, device=DEV)] = float("nan")
     vis = torch.as_tensor(vis_np, device=DEV)
-    out = wd.op_attention(q, kc, vc, vis).float().cpu().numpy().astype(np.float64)
+    out = wd.op_attention(q, kc, vc.transpose(1, 2).contiguous(), vis).float().cpu().numpy().astype(np.float64)
     K = kc.double().cpu().numpy().transpose(1, 0, 2)[vis_np]
     V = vc.double().cpu().numpy().transpose(1, 0, 2)[vis_np]
     ref, _ = wo.attention_rows(q.double().cpu().numpy(), K, V, Hq // Hkv)

@@ -67,6 +67,44 @@ def test_small_bf16_gqa_batch_two_tokens():
     assert pos.shape == (8, 3)
 
 
+DH128 = dict(L=2, d=512, Hq=4, Hkv=4, dh=128, F=1024, V=4000, P=200, G=150, A=16, B=40, R=3, T=2, k=2)
+
+
+@pytest.mark.parametrize("Hkv,batch", [(4, 1), (2, 2), (1, 1)])
+def test_bf16_head_dim_128_tensor_core_attention(Hkv, batch):
+    """head_dim 128 takes the tcgen05 attention: two query tiles at the refresh (256 visible
+    rows), three key tiles with a ragged tail, MHA and GQA, batch of independent windows."""
+    cfg = synth.get_config("llada8b", **dict(DH128, Hkv=Hkv, batch=batch))
+    logs = run(cfg, 7)
+    assert [l["info"]["is_refresh"] for l in logs] == [1, 0, 0, 1, 0, 0, 1]
+    assert logs[0]["info"]["n_rows"] == batch * 256
+
+
+def test_plain_and_tensor_core_paths_agree():
+    """The CUDA-core kernels and the tensor-core kernels compute the same step."""
+    cfg = synth.get_config("llada8b", **DH128)
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    S = ids.shape[1]
+    outs = []
+    for impl in (wd.WD_GEMM_PLAIN, wd.WD_GEMM_TCGEN05):
+        ctx = wd.Context(cfg, w, 1, S, S, S)
+        ctx.set_gemm_impl(impl)
+        st = wd.State(ctx, ids)
+        lay = torch.zeros(cfg["L"] * S * cfg["d"], device=DEV)
+        st.set_taps(layer_out=lay)
+        res = []
+        for _ in range(3):
+            _, info = st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], 0)      # k = 0: same state on both paths
+            st.sync()
+            res.append(lay[: cfg["L"] * info["n_rows"] * cfg["d"]].clone())
+        outs.append(res)
+        st.close(); ctx.close()
+    for a, b in zip(*outs):
+        rel = (a - b).norm() / b.norm()
+        assert rel < 5e-3, rel
+
+
 def test_window_covering_everything_is_full_sequence_step():
     """A >= number of masks, B = 0, R = 1: every step is the no-pruning full-sequence step."""
     cfg = synth.get_config("llada8b", **dict(SMALL_BF16, A=80, B=0, R=1, T=0, k=4))
@@ -95,10 +133,12 @@ def test_late_state_and_finish():
     assert logs[-1]["info"]["n_active"] == 1
 
 
-def test_far_field_and_refresh_independence_on_gpu():
+@pytest.mark.parametrize("shape", [SMALL_BF16, DH128])
+def test_far_field_and_refresh_independence_on_gpu(shape):
     """Changing ids at far-field positions and poisoning the K/V cache before a refresh
-    changes nothing, bit for bit."""
-    cfg = synth.get_config("llada8b", **SMALL_BF16)
+    changes nothing, bit for bit (with head_dim 128 the attention tiles cover poisoned
+    far-field cache rows, which must stay masked)."""
+    cfg = synth.get_config("llada8b", **shape)
     w = synth.make_weights(cfg, DEV)
     ids = synth.make_prompts(cfg)
     S = ids.shape[1]
@@ -110,6 +150,7 @@ def test_far_field_and_refresh_independence_on_gpu():
             ids_v[0, cfg["P"] + cfg["A"] + cfg["B"]:] = 17
         st = wd.State(ctx, ids_v, (ids != cfg["mask_id"]).astype(np.uint8))
         st.mem.view(torch.int16)[S * 2 + 128:].fill_(0x7FC0 if variant else 0)      # NaN / zero K/V cache
+        torch.cuda.synchronize()
         lg = torch.zeros(S * cfg["V"], device=DEV)
         st.set_taps(logits=lg)
         res = []
