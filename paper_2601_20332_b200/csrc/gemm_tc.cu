@@ -19,6 +19,7 @@
 // consumes the GEMM output adds them, which keeps the result deterministic.
 // Every wait is bounded: on expiry the CTA records WD_ERR_DEVICE_TIMEOUT and leaves.
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 
 #include "gemm_tc.h"
@@ -34,17 +35,37 @@ constexpr int kStageA = kBM * kBK * 2;
 constexpr int kThreads = 192;
 
 struct TcParams {
-    int rows, K, bn, n_split, kb_total, n_stages, tmem_cols;
+    int rows, bn, kb_total, tok_tiles, n_units, n_stages, buf_cols, n_slices, aligned;
     int nseg, ncol;
-    int seg_tile0[4];               // first tile index of each segment (+ end)
+    int seg_tile0[4];               // first tile index of each weight matrix (+ end)
     int seg_n[3];
     int seg_col[3];
+    long long W;                    // total K blocks of the launch = n_units * kb_total
     float* y;
     size_t split_stride;
     int32_t* status;
     uint32_t idesc;
 };
 
+// A unit is one [128 weight rows x BN tokens] output tile; unit u = tile * tok_tiles + token tile.
+struct UnitInfo { int seg, n0, tok0; };
+__device__ __forceinline__ UnitInfo decode_unit(const TcParams& p, int unit) {
+    UnitInfo u;
+    const int tile = unit / p.tok_tiles;
+    u.tok0 = (unit - tile * p.tok_tiles) * p.bn;
+    u.seg = 0;
+    if (p.nseg > 1 && tile >= p.seg_tile0[1]) u.seg = 1;
+    if (p.nseg > 2 && tile >= p.seg_tile0[2]) u.seg = 2;
+    u.n0 = (tile - p.seg_tile0[u.seg]) * kBM;
+    return u;
+}
+
+// Persistent, stream-K: the K blocks of all output tiles form one line of W blocks and CTA c
+// takes the contiguous piece [c W / G, (c+1) W / G).  Every CTA therefore streams the same
+// number of weight bytes whatever the shape, the TMA ring never drains between tiles, and the
+// epilogue of one piece overlaps the MMAs of the next (two accumulators in TMEM).  A tile cut
+// by piece boundaries gets one partial sum per CTA that touched it, written to slice
+// (CTA - first CTA of the tile); the CTA that finishes the tile zero-fills the unused slices.
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w0,
                const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2,
@@ -52,72 +73,91 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: required by the 128-byte swizzle atoms
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const int stage_b = p.bn * kBK * 2;
-    const int stage_bytes = kStageA + stage_b;
-    uint64_t* bars = (uint64_t*)(smem + (size_t)p.n_stages * stage_bytes);
-    // bars[0..NS) full, bars[NS..2NS) empty, bars[2NS] accumulator ready
-    uint32_t* tmem_slot = (uint32_t*)(bars + 2 * p.n_stages + 1);
+    const int NS = p.n_stages;
+    const int stage_bytes = kStageA + p.bn * kBK * 2;
+    uint64_t* bars = (uint64_t*)(smem + (size_t)NS * stage_bytes);
+    // bars[0..NS) full | [NS..2NS) empty | [2NS, 2NS+1] accumulator full | [2NS+2, 2NS+3] accumulator empty
+    uint32_t* tmem_slot = (uint32_t*)(bars + 2 * NS + 4);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    // token tile fastest: CTAs that share a weight tile run together and share it through L2
-    const int tile = blockIdx.y, tok0 = blockIdx.x * p.bn, z = blockIdx.z;
-
-    // which weight matrix does this tile belong to
-    int seg = 0;
-    if (p.nseg > 1 && tile >= p.seg_tile0[1]) seg = 1;
-    if (p.nseg > 2 && tile >= p.seg_tile0[2]) seg = 2;
-    const CUtensorMap* map_w = seg == 0 ? &map_w0 : (seg == 1 ? &map_w1 : &map_w2);
-    const int n0 = (tile - p.seg_tile0[seg]) * kBM;           // first weight row of the tile
-    const int kb_begin = (int)(((long long)z * p.kb_total) / p.n_split);
-    const int kb_end = (int)(((long long)(z + 1) * p.kb_total) / p.n_split);
-    const int n_kb = kb_end - kb_begin;
+    const long long c = blockIdx.x, G = gridDim.x;
+    long long g_begin, g_end;
+    if (p.aligned) {
+        g_begin = (c * p.n_units / G) * p.kb_total;
+        g_end = ((c + 1) * p.n_units / G) * p.kb_total;
+    } else {
+        g_begin = c * p.W / G;
+        g_end = (c + 1) * p.W / G;
+    }
+    const int n_total = (int)(g_end - g_begin);
 
     pdl_launch_dependents();      // the next kernel may start its own prologue / weight prefetch
     if (threadIdx.x == 0) {
-        for (int s = 0; s < p.n_stages; ++s) {
+        for (int s = 0; s < NS; ++s) {
             mbar_init(smem_u32(&bars[s]), 1);
-            mbar_init(smem_u32(&bars[p.n_stages + s]), 1);
+            mbar_init(smem_u32(&bars[NS + s]), 1);
         }
-        mbar_init(smem_u32(&bars[2 * p.n_stages]), 1);
+        mbar_init(smem_u32(&bars[2 * NS]), 1);
+        mbar_init(smem_u32(&bars[2 * NS + 1]), 1);
+        mbar_init(smem_u32(&bars[2 * NS + 2]), 128);
+        mbar_init(smem_u32(&bars[2 * NS + 3]), 128);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
-        asm volatile("prefetch.tensormap [%0];" ::"l"(map_w) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w0) : "memory");
     }
-    if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
-                     "r"((uint32_t)p.tmem_cols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 2u * (uint32_t)p.buf_cols);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
     if (warp == 0) {
-        if (lane == 0) {
+        if (lane == 0 && n_total > 0) {
             // ------------------------------------------------ TMA producer
-            uint64_t pol_stream, pol_keep;
+            uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-            asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_keep));
+            // walks the K blocks of this CTA's piece of the line without divisions
+            struct Walk {
+                int unit, kb, n0, tok0;
+                const CUtensorMap* mw;
+            };
+            auto decode = [&](Walk& w) {
+                const UnitInfo u = decode_unit(p, w.unit);
+                w.n0 = u.n0;
+                w.tok0 = u.tok0;
+                w.mw = u.seg == 0 ? &map_w0 : (u.seg == 1 ? &map_w1 : &map_w2);
+            };
+            auto advance = [&](Walk& w) {
+                if (++w.kb == p.kb_total) {
+                    w.kb = 0;
+                    ++w.unit;
+                    decode(w);
+                }
+            };
+            Walk w0;
+            w0.unit = (int)(g_begin / p.kb_total);
+            w0.kb = (int)(g_begin - (long long)w0.unit * p.kb_total);
+            decode(w0);
             // Weights never depend on earlier kernels of the stream: fill the ring with weight
             // boxes first, then wait for the producer of the activations, then add their boxes.
-            const int n_pre = n_kb < p.n_stages ? n_kb : p.n_stages;
-            for (int i = 0; i < n_pre; ++i) {
-                const uint32_t full = smem_u32(&bars[i]);
-                mbar_expect_tx(full, (uint32_t)stage_bytes);
-                tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes), map_w, full, (kb_begin + i) * kBK, n0, pol_stream);
+            const int n_pre = n_total < NS ? n_total : NS;
+            Walk w = w0;
+            for (int i = 0; i < n_pre; ++i, advance(w)) {
+                mbar_expect_tx(smem_u32(&bars[i]), (uint32_t)stage_bytes);
+                tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes), w.mw, smem_u32(&bars[i]), w.kb * kBK, w.n0,
+                                 pol_stream);
             }
             pdl_wait();
-            for (int i = 0; i < n_pre; ++i)
-                tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes) + kStageA, &map_x, smem_u32(&bars[i]),
-                                 (kb_begin + i) * kBK, tok0, pol_keep);
-            for (int i = n_pre; i < n_kb; ++i) {
-                const int s = i % p.n_stages;
-                const uint32_t ph = (uint32_t)(i / p.n_stages) & 1u;
-                if (!mbar_wait(smem_u32(&bars[p.n_stages + s]), ph ^ 1u, abort_flag)) {
+            Walk wx = w0;
+            for (int i = 0; i < n_pre; ++i, advance(wx))
+                tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + kStageA, &map_x, smem_u32(&bars[i]), wx.kb * kBK,
+                            wx.tok0);
+            int s = n_pre % NS;
+            uint32_t ph = (uint32_t)(n_pre / NS) & 1u;
+            for (int i = n_pre; i < n_total; ++i, advance(w)) {
+                if (!mbar_wait(smem_u32(&bars[NS + s]), ph ^ 1u, abort_flag)) {
                     *abort_flag = 1;
                     atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
                     break;
@@ -125,9 +165,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const uint32_t full = smem_u32(&bars[s]);
                 const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
                 mbar_expect_tx(full, (uint32_t)stage_bytes);
-                const int kc = (kb_begin + i) * kBK;
-                tma_load_2d_hint(sa, map_w, full, kc, n0, pol_stream);
-                tma_load_2d_hint(sa + kStageA, &map_x, full, kc, tok0, pol_keep);
+                tma_load_2d_hint(sa, w.mw, full, w.kb * kBK, w.n0, pol_stream);
+                tma_load_2d(sa + kStageA, &map_x, full, w.kb * kBK, w.tok0);
+                if (++s == NS) { s = 0; ph ^= 1u; }
             }
         }
         __syncwarp();
@@ -135,70 +175,100 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         if (lane == 0) {
             // ------------------------------------------------ MMA issuer
             bool ok = true;
-            for (int i = 0; i < n_kb && ok; ++i) {
-                const int s = i % p.n_stages;
-                const uint32_t ph = (uint32_t)(i / p.n_stages) & 1u;
-                if (!mbar_wait(smem_u32(&bars[s]), ph, abort_flag)) {
-                    *abort_flag = 1;
-                    atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
-                    ok = false;
-                    break;
-                }
+            int piece = 0, s = 0;
+            uint32_t ph = 0;
+            long long g = g_begin;
+            while (g < g_end && ok) {
+                const int unit = (int)(g / p.kb_total), kb0 = (int)(g - (long long)unit * p.kb_total);
+                const int len = (int)((long long)(p.kb_total - kb0) < g_end - g ? (p.kb_total - kb0) : g_end - g);
+                const int buf = piece & 1;
+                // the epilogue has drained this accumulator (free at the start)
+                if (!(ok = mbar_wait(smem_u32(&bars[2 * NS + 2 + buf]), ((uint32_t)(piece >> 1) & 1u) ^ 1u, abort_flag))) break;
                 tc_fence_after();
-                const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-                const uint64_t adesc = make_sdesc(sa);
-                const uint64_t bdesc = make_sdesc(sa + kStageA);
+                const uint32_t acc = tmem_base + (uint32_t)(buf * p.buf_cols);
+                for (int j = 0; j < len; ++j) {
+                    if (!(ok = mbar_wait(smem_u32(&bars[s]), ph, abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+                    const uint64_t adesc = make_sdesc(sa);
+                    const uint64_t bdesc = make_sdesc(sa + kStageA);
 #pragma unroll
-                for (int kk = 0; kk < kBK / 16; ++kk) {
-                    // 16 bf16 = 32 bytes further along K inside the swizzle row: +2 in 16-byte units
-                    umma_bf16(tmem_base, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
-                              (i > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < kBK / 16; ++kk) {
+                        // 16 bf16 = 32 bytes further along K inside the swizzle row: +2 in 16-byte units
+                        umma_bf16(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
+                                  (j > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    umma_commit(smem_u32(&bars[NS + s]));          // stage free once these MMAs have read it
+                    if (++s == NS) { s = 0; ph ^= 1u; }
                 }
-                umma_commit(smem_u32(&bars[p.n_stages + s]));     // stage free once these MMAs have read it
+                if (ok) umma_commit(smem_u32(&bars[2 * NS + buf]));  // this piece's accumulator complete
+                g += len;
+                ++piece;
             }
-            if (ok) umma_commit(smem_u32(&bars[2 * p.n_stages]));  // accumulator complete
+            if (!ok) {
+                *abort_flag = 1;
+                atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
+            }
         }
         __syncwarp();
     } else {
         // ---------------------------------------------------- epilogue (warps 2..5)
         const int quarter = warp & 3;                  // TMEM lanes 32*quarter .. +31
         const int n_local = quarter * 32 + lane;
-        const int n = n0 + n_local;
-        const bool n_ok = n < p.seg_n[seg];
-        bool ok = n_kb > 0;
-        if (ok) ok = mbar_wait(smem_u32(&bars[2 * p.n_stages]), 0, abort_flag);
-        if (!ok && n_kb > 0 && lane == 0) {
-            *abort_flag = 1;
-            atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
-        }
-        ok = __all_sync(0xffffffffu, ok);
-        tc_fence_after();
-        pdl_wait();      // the previous consumer of y has finished (already implied by the data flow)
-        float* yb = p.y + (size_t)z * p.split_stride + p.seg_col[seg] + n;
-        for (int c = 0; c < p.bn; c += 16) {
-            if (tok0 + c >= p.rows) break;
-            uint32_t v[16];
-            if (ok) {
-                tmem_ld16(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)c, v);
-            } else {
+        pdl_wait();      // the previous reader of y has finished (already implied by the data flow)
+        bool ok = true;
+        int piece = 0;
+        long long g = g_begin;
+        while (g < g_end) {
+            const int unit = (int)(g / p.kb_total), kb0 = (int)(g - (long long)unit * p.kb_total);
+            const int len = (int)((long long)(p.kb_total - kb0) < g_end - g ? (p.kb_total - kb0) : g_end - g);
+            const UnitInfo u = decode_unit(p, unit);
+            const int buf = piece & 1;
+            const int n = u.n0 + n_local;
+            const bool n_ok = n < p.seg_n[u.seg];
+            int ord = 0;
+            if (!p.aligned) ord = (int)(c - (((long long)unit * p.kb_total + 1) * G - 1) / p.W);
+            ok = ok && mbar_wait(smem_u32(&bars[2 * NS + buf]), (uint32_t)(piece >> 1) & 1u, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            float* yb = p.y + p.seg_col[u.seg] + n;
+            const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.buf_cols);
+            for (int cc = 0; cc < p.bn; cc += 16) {
+                if (u.tok0 + cc >= p.rows) break;
+                uint32_t v[16];
+                tmem_ld16(t_acc + (uint32_t)cc, v);
+                if (n_ok) {
+                    float* ys = yb + (size_t)ord * p.split_stride;
 #pragma unroll
-                for (int t = 0; t < 16; ++t) v[t] = 0u;
-            }
-            if (n_ok) {
-#pragma unroll
-                for (int t = 0; t < 16; ++t) {
-                    const int tok = tok0 + c + t;
-                    if (tok < p.rows) yb[(size_t)tok * p.ncol] = __uint_as_float(v[t]);
+                    for (int t = 0; t < 16; ++t) {
+                        const int tok = u.tok0 + cc + t;
+                        if (tok < p.rows) ys[(size_t)tok * p.ncol] = __uint_as_float(v[t]);
+                    }
                 }
             }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars[2 * NS + 2 + buf]));       // accumulator may be overwritten
+            if (kb0 + len == p.kb_total && n_ok) {
+                // this CTA finished the tile: slices nobody wrote must read as zero
+                for (int sl = ord + 1; sl < p.n_slices; ++sl) {
+                    float* ys = yb + (size_t)sl * p.split_stride;
+                    for (int tok = u.tok0; tok < u.tok0 + p.bn && tok < p.rows; ++tok) ys[(size_t)tok * p.ncol] = 0.f;
+                }
+            }
+            g += len;
+            ++piece;
+        }
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
         }
         tc_fence_before();
     }
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)p.tmem_cols)
-                     : "memory");
+        tmem_dealloc(tmem_base, 2u * (uint32_t)p.buf_cols);
     }
 }
 
@@ -248,7 +318,12 @@ wd_status encode_2d(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_
     return r == CUDA_SUCCESS ? WD_OK : WD_ERR_CUDA;
 }
 
-struct TcConfig { int bn, tok_tiles, n_stages, tmem_cols, ctas_per_sm; size_t smem; };
+struct TcConfig { int bn, tok_tiles, n_stages, buf_cols, ctas_per_sm; size_t smem; };
+
+int env_int(const char* name, int dflt) {
+    const char* v = getenv(name);
+    return v && *v ? atoi(v) : dflt;
+}
 
 TcConfig pick_config(int rows) {
     TcConfig c;
@@ -256,32 +331,26 @@ TcConfig pick_config(int rows) {
     c.bn = ((rows + c.tok_tiles - 1) / c.tok_tiles + 15) / 16 * 16;     // balanced token tiles, <= 256
     int cols = 32;
     while (cols < c.bn) cols <<= 1;
-    c.tmem_cols = cols;
+    c.buf_cols = cols;                                                   // two accumulators: 2 * cols <= 512
     const int stage = kStageA + c.bn * kBK * 2;
-    // two CTAs per SM while the token tile is narrow, so one CTA's epilogue overlaps the
-    // other's streaming; one CTA with a deeper ring otherwise
-    c.ctas_per_sm = c.bn <= 96 ? 2 : 1;
-    const int budget = c.ctas_per_sm == 2 ? 108 * 1024 : 208 * 1024;
-    c.n_stages = budget / stage;
-    if (c.n_stages > 8) c.n_stages = 8;
+    static const int want2 = env_int("WD_GEMM_CTAS_PER_SM", 1);
+    c.ctas_per_sm = (want2 == 2 && c.bn <= 64) ? 2 : 1;
+    c.n_stages = ((c.ctas_per_sm == 2 ? 104 : 200) * 1024) / stage;
+    if (c.n_stages > 10) c.n_stages = 10;
     if (c.n_stages < 2) c.n_stages = 2;
-    c.smem = (size_t)c.n_stages * stage + (2 * c.n_stages + 1) * 8 + 16 + 1024;
+    c.smem = (size_t)c.n_stages * stage + (2 * c.n_stages + 4) * 8 + 16 + 1024;
     return c;
 }
 
-int pick_split(int tiles, int kb_total, int slots, int rows, bool force_single, size_t y_floats, size_t slice_floats) {
-    if (force_single || rows > WD_TC_SPLITK_MAX_ROWS) return 1;
-    int best = 1;
-    double best_eff = 0.0;
-    for (int s = 1; s <= WD_TC_MAX_SPLIT; ++s) {
-        if (s > 1 && kb_total / s < 4) break;                 // keep at least 4 K blocks per CTA
-        if ((size_t)s * slice_floats > y_floats) break;
-        const long long ctas = (long long)tiles * s;
-        const long long waves = (ctas + slots - 1) / slots;
-        const double eff = (double)ctas / (double)(waves * slots);
-        if (eff > best_eff + 0.02) { best_eff = eff; best = s; }
+// most CTAs that contribute to one output tile when W K-blocks are cut into G equal pieces
+int count_slices(int n_units, int kb_total, long long W, long long G) {
+    int n = 1;
+    for (long long u = 0; u < n_units; ++u) {
+        const long long first = ((u * kb_total + 1) * G - 1) / W;
+        const long long last = (((u + 1) * kb_total) * G - 1) / W;
+        if ((int)(last - first + 1) > n) n = (int)(last - first + 1);
     }
-    return best;
+    return n;
 }
 
 uint32_t make_idesc(int bn) {
@@ -342,14 +411,27 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     p.seg_tile0[nseg] = tiles;
     p.nseg = nseg;
     p.ncol = col;
-    p.rows = rows; p.K = K; p.bn = cfg.bn;
+    p.rows = rows; p.bn = cfg.bn;
     p.kb_total = (K + kBK - 1) / kBK;
+    p.tok_tiles = cfg.tok_tiles;
+    p.n_units = tiles * cfg.tok_tiles;
+    p.W = (long long)p.n_units * p.kb_total;
     p.n_stages = cfg.n_stages;
-    p.tmem_cols = cfg.tmem_cols;
+    p.buf_cols = cfg.buf_cols;
     const size_t slice = (size_t)rows * col;
     if (slice > y_floats) return WD_ERR_CAPACITY;
-    p.n_split = pick_split(tiles * cfg.tok_tiles, p.kb_total, sm_count * cfg.ctas_per_sm, rows, force_single_split,
-                           y_floats, slice);
+    // stream-K over all SMs when the partial sums fit, whole tiles per CTA otherwise
+    long long G = (long long)sm_count * cfg.ctas_per_sm;
+    if (G > p.W / 2) G = p.W / 2 > 0 ? p.W / 2 : 1;           // at least two K blocks per CTA
+    int n_slices = count_slices(p.n_units, p.kb_total, p.W, G);
+    p.aligned = 0;
+    if (force_single_split || (size_t)n_slices * slice > y_floats || n_slices > WD_TC_MAX_SPLIT) {
+        p.aligned = 1;
+        n_slices = 1;
+        G = (long long)sm_count * cfg.ctas_per_sm;
+        if (G > p.n_units) G = p.n_units;
+    }
+    p.n_slices = n_slices;
     p.y = y;
     p.split_stride = slice;
     p.status = status;
@@ -360,13 +442,12 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     if (s != WD_OK) return s;
 
     WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
-    dim3 grid(cfg.tok_tiles, tiles, p.n_split);
     const CUtensorMap& m0 = *segs[0].map;
     const CUtensorMap& m1 = *segs[nseg > 1 ? 1 : 0].map;
     const CUtensorMap& m2 = *segs[nseg > 2 ? 2 : 0].map;
     ++wd_launch_counter;
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = grid;
+    lc.gridDim = dim3((unsigned)G);
     lc.blockDim = dim3(kThreads);
     lc.dynamicSmemBytes = cfg.smem;
     lc.stream = stream;
@@ -376,8 +457,7 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     lc.attrs = attr;
     lc.numAttrs = wd_pdl_enabled ? 1 : 0;
     WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel, mx, m0, m1, m2, p));
-    WD_CUDA_TRY(cudaGetLastError());
-    if (n_split_out) *n_split_out = p.n_split;
+    if (n_split_out) *n_split_out = p.n_slices;
     return WD_OK;
 }
 
