@@ -191,6 +191,12 @@ WD_API wd_status wd_destroy(wd_ctx* ctx);
 /* Choose the GEMM kernel used by later steps (default WD_GEMM_AUTO). */
 WD_API wd_status wd_set_gemm_impl(wd_ctx* ctx, int32_t impl);
 
+/* Experimental (default off): let the GEMM CTA that completes an output tile also do the
+ * consumer's element-wise work (1/rms scaling, RoPE + cache scatter, SwiGLU, residual add), which
+ * shortens a block from nine kernels to five.  Only taken for bf16 with head_dim 128 and d_model,
+ * d_ffn multiples of 128; same results within rounding.  Currently slower than separate kernels. */
+WD_API wd_status wd_set_fusion(wd_ctx* ctx, int32_t on);
+
 /* GEMM timing for benchmarks.  While enabled, wd_step brackets every GEMM launch
  * (one launch covers all weight matrices that share an input: q/k/v, gate/up)
  * with CUDA events on the step's stream and wd_step_sync adds up their device

@@ -65,6 +65,7 @@ SIGNATURES = {
     "wd_create": (C.c_int, [C.POINTER(wd_model_dims), C.POINTER(wd_weights), vp, C.c_size_t, C.POINTER(vp)]),
     "wd_destroy": (C.c_int, [vp]),
     "wd_set_gemm_impl": (C.c_int, [vp, i32]),
+    "wd_set_fusion": (C.c_int, [vp, i32]),
     "wd_profile_enable": (C.c_int, [vp, i32]),
     "wd_profile_read": (C.c_int, [vp, C.POINTER(C.c_double), C.POINTER(C.c_double), C.POINTER(C.c_int64)]),
     "wd_state_create": (C.c_int, [vp, i32, i32, i32p, u8p, vp, C.c_size_t, C.POINTER(vp)]),
@@ -189,6 +190,9 @@ class Context:
 
     def set_gemm_impl(self, impl: int):
         check(lib().wd_set_gemm_impl(self.handle, impl), "wd_set_gemm_impl")
+
+    def set_fusion(self, on: bool):
+        check(lib().wd_set_fusion(self.handle, 1 if on else 0), "wd_set_fusion")
 
     def profile_enable(self, on: bool):
         check(lib().wd_profile_enable(self.handle, 1 if on else 0), "wd_profile_enable")

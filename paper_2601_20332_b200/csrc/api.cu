@@ -3,6 +3,7 @@
 #include <algorithm>
 #include <climits>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -72,6 +73,12 @@ struct wd_ctx {
     int32_t* ch_idx = nullptr;
     double* ch_sum = nullptr;
     float2* rope_tab = nullptr;  // [max_rows][dh/2] (cos, sin) of this step's rows
+    float* sumsq = nullptr;      // [d/128][max_rows] partial sums of squares of the residual rows
+    float* attn_scratch = nullptr;     // parts of the attention's split over keys
+    int32_t* attn_counters = nullptr;
+    int32_t* tile_counters = nullptr;  // arrival counters of the fused GEMM epilogues (kept zero)
+    size_t n_tile_counters = 0;
+    bool fuse = false;           // fused GEMM epilogues (experimental: slower than separate kernels so far)
     int32_t* plan = nullptr;     // packed index lists of the step
     size_t plan_ints = 0;
     int32_t* result = nullptr;   // [status | n_sel[batch] | pos | tok | conf]
@@ -125,7 +132,7 @@ static size_t part_floats_for(const wd_model_dims* d) {
     return std::max((size_t)d->max_rows * cols, (size_t)WD_TC_MAX_SPLIT * small_rows * cols);
 }
 
-static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[20]) {
+static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[24]) {
     const size_t e = wd_elt_size(d->dtype);
     const size_t MR = d->max_rows, MA = d->max_active, hq = (size_t)d->n_q_heads * d->head_dim;
     off[0] = c.take(MR * d->d_model * 4);                       // x
@@ -148,12 +155,17 @@ static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[20]) {
     off[14] = c.take(MA * nch * 4);                             // ch_idx
     off[15] = c.take(MA * nch * 8);                             // ch_sum
     off[16] = c.take(MR * (size_t)(d->head_dim / 2) * 8);       // rope_tab
+    off[17] = c.take(((size_t)d->d_model / 128 + 1) * MR * 4);  // sumsq
+    off[18] = c.take(((max_gemm_cols(d) + 127) / 128) * (MR / 256 + 2) * 4);   // tile counters
+    off[19] = ((max_gemm_cols(d) + 127) / 128) * (MR / 256 + 2);
+    off[20] = c.take(wd_attn_tc_scratch_floats() * 4);          // attention split parts
+    off[21] = c.take(WD_ATTN_SPLIT_SLOTS * 4);                  // attention counters
 }
 
 extern "C" size_t wd_workspace_bytes(const wd_model_dims* dims) {
     if (!dims_valid(dims)) return 0;
     Carve c;
-    size_t off[20];
+    size_t off[24];
     carve_ctx(dims, c, off);
     return c.off;
 }
@@ -192,6 +204,10 @@ extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, v
     wd_ctx* c = new (std::nothrow) wd_ctx();
     if (!c) return WD_ERR_CUDA;
     c->d = *dims;
+    // debugging switches: WD_FUSE=1 moves the element-wise work into the GEMM epilogues,
+    // WD_NO_PDL=1 launches every kernel fully serialised
+    if (const char* e = getenv("WD_FUSE")) c->fuse = (e[0] == '1');
+    if (const char* e = getenv("WD_NO_PDL")) wd_pdl_enabled = !(e[0] == '1');
     c->sm_count = prop.multiProcessorCount;
     c->tok_embed = w->tok_embed;
     c->lm_head = w->lm_head;
@@ -203,7 +219,7 @@ extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, v
         c->attn_norm.push_back(w->attn_norm[l]); c->ffn_norm.push_back(w->ffn_norm[l]);
     }
     Carve cv;
-    size_t off[20];
+    size_t off[24];
     carve_ctx(dims, cv, off);
     char* base = (char*)workspace;
     c->x = (float*)(base + off[0]);
@@ -225,6 +241,13 @@ extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, v
     c->ch_idx = (int32_t*)(base + off[14]);
     c->ch_sum = (double*)(base + off[15]);
     c->rope_tab = (float2*)(base + off[16]);
+    c->sumsq = (float*)(base + off[17]);
+    c->tile_counters = (int32_t*)(base + off[18]);
+    c->n_tile_counters = off[19];
+    WD_CUDA_TRY(cudaMemset(c->tile_counters, 0, c->n_tile_counters * 4));
+    c->attn_scratch = (float*)(base + off[20]);
+    c->attn_counters = (int32_t*)(base + off[21]);
+    WD_CUDA_TRY(cudaMemset(c->attn_counters, 0, WD_ATTN_SPLIT_SLOTS * 4));
     WD_CUDA_TRY(cudaMemset(c->result, 0, 4));
 
     if (dims->dtype == WD_BF16) {
@@ -248,6 +271,12 @@ extern "C" wd_status wd_set_gemm_impl(wd_ctx* ctx, int32_t impl) {
     if (impl == WD_GEMM_TCGEN05 && ctx->d.dtype != WD_BF16) return WD_ERR_BAD_PARAM;
     ctx->gemm_impl = impl;
     ctx->attn_impl = impl;          // the plain setting selects the CUDA-core kernels throughout
+    return WD_OK;
+}
+
+extern "C" wd_status wd_set_fusion(wd_ctx* ctx, int32_t on) {
+    if (!ctx) return WD_ERR_NULL;
+    ctx->fuse = on != 0;
     return WD_OK;
 }
 
@@ -477,7 +506,7 @@ static bool use_tc(const wd_ctx* c) {
 
 static wd_status run_gemm(wd_ctx* c, const void* x, const WdTcX* x_map, const WdTcSeg* segs, int nseg,
                           int rows, int K, float* y, size_t y_floats, int32_t* status, cudaStream_t stream,
-                          GemmOut* go, bool single_split = false, bool force_tc = false) {
+                          GemmOut* go, bool single_split = false, const WdTcFuse* fuse = nullptr) {
     int ncol = 0;
     for (int i = 0; i < nseg; ++i) ncol += segs[i].n;
     cudaEvent_t e0 = nullptr, e1 = nullptr;
@@ -494,10 +523,10 @@ static wd_status run_gemm(wd_ctx* c, const void* x, const WdTcX* x_map, const Wd
                               (double)rows * ncol * 4;
         WD_CUDA_TRY(cudaEventRecord(e0, stream));
     }
-    if (use_tc(c) || force_tc) {
+    if (use_tc(c)) {
         int n_split = 1;
         wd_status s = wd_tc_gemm(x_map, segs, nseg, rows, K, y, y_floats, c->sm_count, status, stream, &n_split,
-                                 single_split);
+                                 single_split, fuse);
         if (s != WD_OK) return s;
         *go = {n_split, (size_t)rows * ncol, 1, WD_GEMM_TCGEN05};
     } else {
@@ -615,6 +644,70 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     wd_status s;
 
     const int Sp = st->Sp;
+    const bool fused = use_tc(c) && c->fuse && dh == 128 && D % 128 == 0 && F % 128 == 0;
+    auto attention = [&](int l, char* kc, char* vc) -> wd_status {
+        float* attn_tap = st->taps.attn_out ? st->taps.attn_out + (size_t)l * R_ * hq : nullptr;
+        if (st->attn_tc && all_contig && c->attn_impl != WD_GEMM_PLAIN)
+            return wd_attn_tc_launch(c->q, R_, (int)n_qtiles, c->plan + o_qt_seq, c->plan + o_qt_row0, c->plan + o_qt_n,
+                                     c->plan + o_nvis, &st->map_k, &st->map_vt, c->attn, attn_tap, Hq, Hkv, dh, l, max_vis,
+                                     c->sm_count, c->attn_scratch, c->attn_counters, status, stream);
+        wd_launch_attention_plain(d.dtype, c->q, kc, vc, row_seq, vis_idx, vis_off, c->attn, attn_tap, R_, max_vis, Hq,
+                                  Hkv, dh, S, Sp, stream);
+        return WD_OK;
+    };
+    if (fused) {
+        // Five kernels per block.  The GEMM input is bf16(x * gain) without the 1/rms factor; the CTA
+        // that completes an output tile applies it (from per-block sums of squares written by the
+        // previous GEMM) together with RoPE + cache scatter, SwiGLU, or the residual add.
+        wd_launch_embed_fused(c->tok_embed, st->ids_dev, row_seq, row_pos, c->x, c->xn, c->attn_norm[0], c->sumsq,
+                              c->rope_tab, R_, D, S, d.vocab, dh, d.rope_theta, status, stream);
+        WdTcFuse base;
+        base.counters = c->tile_counters;
+        base.rows_total = R_;
+        base.n_prev_tiles = D / 128;
+        base.inv_d = 1.f / (float)D;
+        base.eps = d.rms_eps;
+        for (int l = 0; l < d.n_layers; ++l) {
+            char* kc = st->kcache + (size_t)l * st->kv_layer_bytes;
+            char* vc = st->vcache + (size_t)l * st->v_layer_bytes;
+            WdTcFuse fq = base;
+            fq.mode = WD_FUSE_QKV;
+            fq.sumsq_in = c->sumsq;
+            fq.row_seq = row_seq; fq.row_pos = row_pos; fq.rope_tab = c->rope_tab;
+            fq.q = (__nv_bfloat16*)c->q; fq.kcache = (__nv_bfloat16*)kc; fq.vcache = (__nv_bfloat16*)vc;
+            fq.Hq = Hq; fq.Hkv = Hkv; fq.S = S; fq.Sp = Sp;
+            WdTcSeg qkv[3] = {{c->wq[l], hq, c->tc.get(WD_TC_WQ, l)}, {c->wk[l], hkv, c->tc.get(WD_TC_WK, l)},
+                              {c->wv[l], hkv, c->tc.get(WD_TC_WV, l)}};
+            if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, qkv, 3, R_, D, c->part, c->part_floats, status, stream, &go, false,
+                              &fq)) != WD_OK)
+                return s;
+            impl_used = go.impl;
+            if ((s = attention(l, kc, vc)) != WD_OK) return s;
+            WdTcFuse fo = base;
+            fo.mode = WD_FUSE_RESID;
+            fo.x = c->x; fo.gain_next = c->ffn_norm[l]; fo.xg = (__nv_bfloat16*)c->xn; fo.sumsq_out = c->sumsq;
+            WdTcSeg wo[1] = {{c->wo[l], D, c->tc.get(WD_TC_WO, l)}};
+            if ((s = run_gemm(c, c->attn, &c->tc.x_map_attn, wo, 1, R_, hq, c->part, c->part_floats, status, stream, &go,
+                              false, &fo)) != WD_OK)
+                return s;
+            WdTcFuse fg = base;
+            fg.mode = WD_FUSE_SWIGLU;
+            fg.sumsq_in = c->sumsq; fg.h = (__nv_bfloat16*)c->h; fg.F = F;
+            WdTcSeg gu[2] = {{c->wg[l], F, c->tc.get(WD_TC_WG, l)}, {c->wu[l], F, c->tc.get(WD_TC_WU, l)}};
+            if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, gu, 2, R_, D, c->part, c->part_floats, status, stream, &go, false,
+                              &fg)) != WD_OK)
+                return s;
+            WdTcFuse fd = base;
+            fd.mode = WD_FUSE_RESID;
+            fd.x = c->x; fd.xg = (__nv_bfloat16*)c->xn; fd.sumsq_out = c->sumsq;
+            fd.gain_next = l + 1 < d.n_layers ? c->attn_norm[l + 1] : nullptr;
+            fd.tap = st->taps.layer_out ? st->taps.layer_out + (size_t)l * R_ * D : nullptr;
+            WdTcSeg wdn[1] = {{c->wd[l], D, c->tc.get(WD_TC_WD, l)}};
+            if ((s = run_gemm(c, c->h, &c->tc.x_map_h, wdn, 1, R_, F, c->part, c->part_floats, status, stream, &go, false,
+                              &fd)) != WD_OK)
+                return s;
+        }
+    } else {
     wd_launch_embed(d.dtype, c->tok_embed, st->ids_dev, row_seq, row_pos, c->x, c->rope_tab, R_, D, S, d.vocab, dh,
                     d.rope_theta, status, stream);
     bool down_pending = false;          // x still lacks the previous block's FFN output
@@ -633,16 +726,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         impl_used = go.impl;
         wd_launch_rope_scatter(d.dtype, c->part, go.n_split, go.split_stride, row_seq, row_pos, c->rope_tab, c->q, kc,
                                vc, R_, Hq, Hkv, dh, S, Sp, stream);
-        float* attn_tap = st->taps.attn_out ? st->taps.attn_out + (size_t)l * R_ * hq : nullptr;
-        if (st->attn_tc && all_contig && c->attn_impl != WD_GEMM_PLAIN) {
-            if ((s = wd_attn_tc_launch(c->q, R_, (int)n_qtiles, c->plan + o_qt_seq, c->plan + o_qt_row0, c->plan + o_qt_n,
-                                       c->plan + o_nvis, &st->map_k, &st->map_vt, c->attn, attn_tap, Hq, Hkv, dh, l,
-                                       status, stream)) != WD_OK)
-                return s;
-        } else {
-            wd_launch_attention_plain(d.dtype, c->q, kc, vc, row_seq, vis_idx, vis_off, c->attn, attn_tap, R_, max_vis,
-                                      Hq, Hkv, dh, S, Sp, stream);
-        }
+        if ((s = attention(l, kc, vc)) != WD_OK) return s;
         WdTcSeg wo[1] = {{c->wo[l], D, c->tc.get(WD_TC_WO, l)}};
         if ((s = run_gemm(c, c->attn, &c->tc.x_map_attn, wo, 1, R_, hq, c->part, c->part_floats, status, stream, &go)) != WD_OK)
             return s;
@@ -663,6 +747,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
             down_pending = true;     // folded into the next block's RMSNorm
             down_go = go;
         }
+    }
     }
     // logits for the active rows only, then the unmask reduction
     if (NA > 0) {

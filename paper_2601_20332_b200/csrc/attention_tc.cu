@@ -17,6 +17,9 @@
 // Query rows beyond the tile's valid rows are computed on whatever the box holds and discarded
 // (rows are independent).  Keys at or beyond n_vis are masked by selection, and their V
 // columns are zeroed in shared memory, so stale or poisoned cache rows cannot leak in.
+// When there are few (tile, head) pairs, as in a normal step, the keys are also split across
+// CTAs (grid.z) so that the machine is filled: each CTA leaves its running maximum, sum and
+// unnormalised output in scratch and the last one to arrive merges them in a fixed order.
 // Every wait is bounded; on expiry the CTA records WD_ERR_DEVICE_TIMEOUT and leaves.
 #include <cstring>
 
@@ -44,6 +47,13 @@ struct AttnParams {
     float scale_log2e;           // log2(e) / sqrt(dh)
     int32_t* status;
     uint32_t idesc;
+    // split over the keys: CTA z of (tile, head) takes key tiles [z * tiles_per_split, ...) and, when a
+    // sequence needs more than one CTA, leaves (m, l, unnormalised O) in scratch; the CTA that arrives
+    // last merges the parts in order of z
+    int tiles_per_split, max_parts;
+    float* part_o;               // [(tile * Hq + h) * max_parts + z][128 rows][128]
+    float* part_ml;              // [(tile * Hq + h) * max_parts + z][128 rows][2]
+    int32_t* counters;           // [n_tiles * Hq], zero between launches
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
@@ -70,6 +80,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int kvh = h / (p.Hq / p.Hkv);
 
     pdl_launch_dependents();
+    // the index lists were copied before the first kernel of the step: safe to read right away
+    const int n_vis = p.seq_nvis[b];
+    const int n_kt_all = (n_vis + kTile - 1) / kTile;
+    const int n_parts = (n_kt_all + p.tiles_per_split - 1) / p.tiles_per_split;
+    const int kt_begin = (int)blockIdx.z * p.tiles_per_split;
+    if (kt_begin >= n_kt_all) return;                       // nothing for this CTA (uniform exit)
+    const int n_kt = min(p.tiles_per_split, n_kt_all - kt_begin);
     if (threadIdx.x == 0) {
         for (int i = 0; i < 8; ++i) mbar_init(smem_u32(&bars[i]), i == 6 ? 128u : 1u);
         *abort_flag = 0;
@@ -81,8 +98,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     pdl_wait();                                   // q and the cache rows come from the previous kernel
-    const int n_vis = p.seq_nvis[b];
-    const int n_kt = (n_vis + kTile - 1) / kTile;
 
     if (warp == 0) {
         if (lane == 0) {
@@ -102,7 +117,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 const uint32_t full = smem_u32(&bars[1 + s]);
                 const uint32_t sk = smem_u32(sKV + (size_t)s * 2 * kOperand), sv = sk + kOperand;
                 mbar_expect_tx(full, 2 * kOperand);
-                const int kv0 = i * kTile, bh = b * p.Hkv + kvh;
+                const int kv0 = (kt_begin + i) * kTile, bh = b * p.Hkv + kvh;
                 tma_load_4d(sk, &map_k, full, 0, kv0, bh, p.layer);            // keys kv0.., dims 0..63
                 tma_load_4d(sk + kAtom, &map_k, full, 64, kv0, bh, p.layer);   // dims 64..127
                 tma_load_4d(sv, &map_vt, full, kv0, 0, bh, p.layer);           // all dims, keys kv0..kv0+63
@@ -163,7 +178,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int n_keys = min(kTile, n_vis - i * kTile);          // valid keys in this tile
+            const int n_keys = min(kTile, n_vis - (kt_begin + i) * kTile);   // valid keys in this tile
             // keys past n_vis may hold anything: zero their V columns so that 0 * garbage stays 0.
             // Thread r owns row r (a head dim) of the transposed V tile.
             if (n_keys < kTile) {
@@ -232,22 +247,67 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             *abort_flag = 1;
             atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
         }
-        if (ok && r < n_valid) {
-            const float inv = 1.f / l;
-            const size_t base = ((size_t)(row0 + r) * p.Hq + h) * kTile;
-            uint4* dst = reinterpret_cast<uint4*>(p.out + base);
+        if (n_parts == 1) {
+            if (ok && r < n_valid) {
+                const float inv = 1.f / l;
+                const size_t base = ((size_t)(row0 + r) * p.Hq + h) * kTile;
+                uint4* dst = reinterpret_cast<uint4*>(p.out + base);
 #pragma unroll
-            for (int g = 0; g < kTile / 8; ++g) {
-                uint4 u;
-                u.x = pack_bf16(o[8 * g + 0] * inv, o[8 * g + 1] * inv);
-                u.y = pack_bf16(o[8 * g + 2] * inv, o[8 * g + 3] * inv);
-                u.z = pack_bf16(o[8 * g + 4] * inv, o[8 * g + 5] * inv);
-                u.w = pack_bf16(o[8 * g + 6] * inv, o[8 * g + 7] * inv);
-                dst[g] = u;
+                for (int g = 0; g < kTile / 8; ++g) {
+                    uint4 u;
+                    u.x = pack_bf16(o[8 * g + 0] * inv, o[8 * g + 1] * inv);
+                    u.y = pack_bf16(o[8 * g + 2] * inv, o[8 * g + 3] * inv);
+                    u.z = pack_bf16(o[8 * g + 4] * inv, o[8 * g + 5] * inv);
+                    u.w = pack_bf16(o[8 * g + 6] * inv, o[8 * g + 7] * inv);
+                    dst[g] = u;
+                }
+                if (p.tap) {
+#pragma unroll
+                    for (int c = 0; c < kTile; ++c) p.tap[base + c] = o[c] * inv;
+                }
             }
-            if (p.tap) {
+        } else {
+            // leave this CTA's part in scratch, count the arrival, the last CTA merges
+            const size_t slot = ((size_t)tile * p.Hq + h) * p.max_parts;
+            if (ok && r < n_valid) {
+                float4* dst = reinterpret_cast<float4*>(p.part_o + ((slot + blockIdx.z) * kTile + r) * kTile);
 #pragma unroll
-                for (int c = 0; c < kTile; ++c) p.tap[base + c] = o[c] * inv;
+                for (int g = 0; g < kTile / 4; ++g) dst[g] = make_float4(o[4 * g], o[4 * g + 1], o[4 * g + 2], o[4 * g + 3]);
+                *reinterpret_cast<float2*>(p.part_ml + ((slot + blockIdx.z) * kTile + r) * 2) = make_float2(m, l);
+            }
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            int* last_flag = (int*)(tmem_slot + 2);
+            if (threadIdx.x == 64) {
+                const int old = atomicAdd(p.counters + tile * p.Hq + h, 1);
+                const int last = old + 1 == n_parts ? 1 : 0;
+                if (last) p.counters[tile * p.Hq + h] = 0;
+                *last_flag = last;
+                __threadfence();
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (*last_flag) {
+                // warp `quarter` merges rows quarter, quarter + 4, ...; lanes hold 4 columns each
+                for (int rr = quarter; rr < n_valid; rr += 4) {
+                    float mx = -INFINITY;
+                    for (int z = 0; z < n_parts; ++z) mx = fmaxf(mx, __ldcg(p.part_ml + ((slot + z) * kTile + rr) * 2));
+                    float lsum = 0.f;
+                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    for (int z = 0; z < n_parts; ++z) {
+                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot + z) * kTile + rr) * 2));
+                        const float wgt = exp2f(ml.x - mx);
+                        const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_o + ((slot + z) * kTile + rr) * kTile) + lane);
+                        lsum += ml.y * wgt;
+                        acc.x += v.x * wgt; acc.y += v.y * wgt; acc.z += v.z * wgt; acc.w += v.w * wgt;
+                    }
+                    const float inv = 1.f / lsum;
+                    const size_t base = ((size_t)(row0 + rr) * p.Hq + h) * kTile + 4 * lane;
+                    uint2 u;
+                    u.x = pack_bf16(acc.x * inv, acc.y * inv);
+                    u.y = pack_bf16(acc.z * inv, acc.w * inv);
+                    *reinterpret_cast<uint2*>(p.out + base) = u;
+                    if (p.tap) *reinterpret_cast<float4*>(p.tap + base) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+                }
             }
         }
     }
@@ -310,7 +370,8 @@ wd_status wd_attn_tc_encode_cache(CUtensorMap* map_k, CUtensorMap* map_vt, const
 wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_t* qtile_seq, const int32_t* qtile_row0,
                             const int32_t* qtile_n, const int32_t* seq_nvis, const CUtensorMap* map_k,
                             const CUtensorMap* map_vt, void* out, float* tap, int Hq, int Hkv, int dh, int layer,
-                            int32_t* status, cudaStream_t stream) {
+                            int max_vis, int sm_count, float* scratch, int32_t* counters, int32_t* status,
+                            cudaStream_t stream) {
     if (dh != kTile) return WD_ERR_BAD_PARAM;
     if (n_tiles <= 0) return WD_OK;
     EncodeTiledFn enc = get_encode();
@@ -333,10 +394,21 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     p.scale_log2e = 1.4426950408889634f / sqrtf((float)dh);
     p.status = status;
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
+    // split the keys across CTAs while (tile, head) pairs alone would leave SMs idle
+    const int max_kt = (max_vis + kTile - 1) / kTile;
+    int want = sm_count / (n_tiles * Hq);
+    if (want < 1 || !scratch || !counters || n_tiles * Hq > WD_ATTN_SPLIT_SLOTS / 2) want = 1;
+    if (want > max_kt) want = max_kt;
+    p.tiles_per_split = (max_kt + want - 1) / want;
+    p.max_parts = (max_kt + p.tiles_per_split - 1) / p.tiles_per_split;
+    if ((long long)n_tiles * Hq * p.max_parts > WD_ATTN_SPLIT_SLOTS) { p.tiles_per_split = max_kt; p.max_parts = 1; }
+    p.part_o = scratch;
+    p.part_ml = scratch ? scratch + (size_t)WD_ATTN_SPLIT_SLOTS * kTile * kTile : nullptr;
+    p.counters = counters;
     const size_t smem = 6 * (size_t)kOperand + 8 * 8 + 16 + 1024;
     WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3(n_tiles, Hq);
+    lc.gridDim = dim3(n_tiles, Hq, p.max_parts);
     lc.blockDim = dim3(kThreads);
     lc.dynamicSmemBytes = smem;
     lc.stream = stream;

@@ -45,6 +45,7 @@ struct TcParams {
     size_t split_stride;
     int32_t* status;
     uint32_t idesc;
+    WdTcFuse f;
 };
 
 // A unit is one [128 weight rows x BN tokens] output tile; unit u = tile * tok_tiles + token tile.
@@ -58,6 +59,231 @@ __device__ __forceinline__ UnitInfo decode_unit(const TcParams& p, int unit) {
     if (p.nseg > 2 && tile >= p.seg_tile0[2]) u.seg = 2;
     u.n0 = (tile - p.seg_tile0[u.seg]) * kBM;
     return u;
+}
+
+// The pieces of one CTA's share [g_begin, g_end) of the K-block line, in the order they are
+// processed: first the partial tile at the front of the share, then the partial tile at its
+// back, then the whole tiles in between.  Partial tiles are the ones other CTAs also work on;
+// doing them first lets those tiles complete (and their fused epilogue run) in the middle of the
+// kernel instead of all at its end.
+struct Sched {
+    long long g_begin, g_end;
+    int kb_total, head_len, tail_len, n_full, n_pieces;
+    long long full_begin;
+    __device__ void init(long long gb, long long ge, int kb) {
+        g_begin = gb; g_end = ge; kb_total = kb;
+        const long long total = ge - gb;
+        const int off = (int)(gb % kb);
+        head_len = off ? (int)((long long)(kb - off) < total ? (kb - off) : total) : 0;
+        const long long rest_begin = gb + head_len;
+        const long long rest = ge - rest_begin;
+        n_full = (int)(rest / kb);
+        tail_len = (int)(rest - (long long)n_full * kb);
+        full_begin = rest_begin;
+        n_pieces = (head_len ? 1 : 0) + (tail_len ? 1 : 0) + n_full;
+    }
+    // piece i -> first K block on the line and length
+    __device__ void piece(int i, long long& g, int& len) const {
+        if (head_len) { if (i == 0) { g = g_begin; len = head_len; return; } --i; }
+        if (tail_len) { if (i == 0) { g = g_end - tail_len; len = tail_len; return; } --i; }
+        g = full_begin + (long long)i * kb_total;
+        len = kb_total;
+    }
+};
+
+// number of CTAs whose piece of the line touches unit u
+__device__ __forceinline__ int n_contrib(const TcParams& p, long long G, int unit) {
+    if (p.aligned) return 1;
+    const long long first = ((long long)unit * p.kb_total + 1) * G - 1;
+    const long long last = ((long long)(unit + 1) * p.kb_total) * G - 1;
+    return (int)(last / p.W - first / p.W) + 1;
+}
+
+__device__ __forceinline__ float4 ldcg4(const float* p) { return __ldcg(reinterpret_cast<const float4*>(p)); }
+__device__ __forceinline__ void add4(float4& a, const float4 b) { a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
+__device__ __forceinline__ void store_bf16x4(__nv_bfloat16* p, float a, float b, float c, float d) {
+    __nv_bfloat162 lo = __floats2bfloat162_rn(a, b), hi = __floats2bfloat162_rn(c, d);
+    uint2 u;
+    u.x = *reinterpret_cast<uint32_t*>(&lo);
+    u.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p) = u;
+}
+__device__ __forceinline__ float warp_sum_f(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ void epi_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
+// Adds slices [0, nc) of UN rows into acc, MS slices at a time: all loads of a group are issued
+// before the first add, so their L2 round trips overlap; the adds keep slice order.
+template <int UN, int MS>
+__device__ __forceinline__ void add_slices(float4 (&acc)[UN], const float* const (&base)[UN], const bool (&valid)[UN],
+                                           int nc, size_t stride) {
+    for (int s0 = 0; s0 < nc; s0 += MS) {
+        float4 tmp[UN][MS];
+#pragma unroll
+        for (int i = 0; i < UN; ++i)
+#pragma unroll
+            for (int k = 0; k < MS; ++k)
+                tmp[i][k] = (valid[i] && s0 + k < nc) ? ldcg4(base[i] + (size_t)(s0 + k) * stride) : make_float4(0, 0, 0, 0);
+#pragma unroll
+        for (int i = 0; i < UN; ++i)
+#pragma unroll
+            for (int k = 0; k < MS; ++k) add4(acc[i], tmp[i][k]);
+    }
+}
+
+// this lane's share of row r's sum of squares (the previous GEMM's per-block partial sums)
+__device__ __forceinline__ float sumsq_lane(const TcParams& p, int r, int lane) {
+    float ss = 0.f;
+    for (int i = lane; i < p.f.n_prev_tiles; i += 32) ss += __ldcg(p.f.sumsq_in + (size_t)i * p.f.rows_total + r);
+    return ss;
+}
+
+// Run by the 128 epilogue threads of the CTA that completed `unit` (e = 0..127).  Every
+// partial slice of the tile is in y; sums are taken in slice order, so the result does not
+// depend on which CTA arrived last.  A warp handles one token at a time, its lanes the tile's
+// 128 columns as float4; the loads of several tokens and slices are issued together so that
+// their L2 round trips overlap, and only then reduced.
+__device__ void finalize_unit(const TcParams& p, long long G, int unit, int e) {
+    const UnitInfo u = decode_unit(p, unit);
+    const int nt = min(p.bn, p.rows - u.tok0);
+    const int lane = e & 31, wq = e >> 5;
+    if (p.f.mode == WD_FUSE_RESID) {
+        // x += tile; xg = bf16(x * gain); per-row sum of squares over this tile's 128 columns
+        constexpr int UN = 3;
+        const int nc = n_contrib(p, G, unit);
+        const int col = u.n0 + 4 * lane, d = p.ncol;
+        const float4 g = p.f.gain_next ? *reinterpret_cast<const float4*>(p.f.gain_next + col) : make_float4(0, 0, 0, 0);
+        for (int t0 = wq; t0 < nt; t0 += 4 * UN) {
+            float4 v[UN];
+            const float* base[UN];
+            bool valid[UN];
+#pragma unroll
+            for (int i = 0; i < UN; ++i) {
+                const int t = t0 + 4 * i;
+                valid[i] = t < nt;
+                const size_t o = (size_t)(u.tok0 + (valid[i] ? t : 0)) * d + col;
+                base[i] = p.y + o;
+                v[i] = valid[i] ? *reinterpret_cast<const float4*>(p.f.x + o) : make_float4(0, 0, 0, 0);
+            }
+            add_slices<UN, 3>(v, base, valid, nc, p.split_stride);
+#pragma unroll
+            for (int i = 0; i < UN; ++i) {
+                const int t = t0 + 4 * i;
+                if (valid[i]) {
+                    const size_t o = (size_t)(u.tok0 + t) * d + col;
+                    *reinterpret_cast<float4*>(p.f.x + o) = v[i];
+                    if (p.f.gain_next) store_bf16x4(p.f.xg + o, v[i].x * g.x, v[i].y * g.y, v[i].z * g.z, v[i].w * g.w);
+                    if (p.f.tap) *reinterpret_cast<float4*>(p.f.tap + o) = v[i];
+                    const float ss = warp_sum_f(v[i].x * v[i].x + v[i].y * v[i].y + v[i].z * v[i].z + v[i].w * v[i].w);
+                    if (lane == 0) p.f.sumsq_out[(size_t)(u.n0 >> 7) * p.f.rows_total + u.tok0 + t] = ss;
+                }
+            }
+        }
+    } else if (p.f.mode == WD_FUSE_QKV) {
+        // one tile = one head (head_dim 128): scale by 1/rms, rotate q and k, write q / K / V^T.
+        // Half a warp per token: lane quad q4 holds columns 4*q4.. and their rotation partners +64.
+        constexpr int UN = 2;
+        const int nc = n_contrib(p, G, unit);
+        const int head = (p.seg_col[u.seg] + u.n0) >> 7;            // index among q | k | v heads
+        const int q4 = lane & 15, tsel = lane >> 4;
+        const size_t col = (size_t)p.seg_col[u.seg] + u.n0 + 4 * q4;
+        for (int t0 = 2 * wq; t0 < nt; t0 += 8 * UN) {
+            float4 a[UN], b[UN];
+            const float* base_a[UN];
+            const float* base_b[UN];
+            bool valid[UN];
+            float ss0[UN], ss1[UN];
+#pragma unroll
+            for (int i = 0; i < UN; ++i) {
+                const int tb = t0 + 8 * i;                          // this warp's token pair: tb, tb + 1
+                const int t = tb + tsel;
+                valid[i] = t < nt;
+                a[i] = b[i] = make_float4(0, 0, 0, 0);
+                base_a[i] = p.y + (size_t)(u.tok0 + (valid[i] ? t : 0)) * p.ncol + col;
+                base_b[i] = base_a[i] + 64;
+                // every lane loads its share of both rows' sums of squares (full-warp reductions below)
+                ss0[i] = tb < nt ? sumsq_lane(p, u.tok0 + tb, lane) : 0.f;
+                ss1[i] = tb + 1 < nt ? sumsq_lane(p, u.tok0 + tb + 1, lane) : 0.f;
+            }
+            add_slices<UN, 3>(a, base_a, valid, nc, p.split_stride);
+            add_slices<UN, 3>(b, base_b, valid, nc, p.split_stride);
+#pragma unroll
+            for (int i = 0; i < UN; ++i) {
+                const float s0 = warp_sum_f(ss0[i]), s1 = warp_sum_f(ss1[i]);
+                const int t = t0 + 8 * i + tsel;
+                if (!valid[i]) continue;
+                const float inv = rsqrtf((tsel ? s1 : s0) * p.f.inv_d + p.f.eps);
+                const int r = u.tok0 + t;
+                const float av[4] = {a[i].x * inv, a[i].y * inv, a[i].z * inv, a[i].w * inv};
+                const float bv[4] = {b[i].x * inv, b[i].y * inv, b[i].z * inv, b[i].w * inv};
+                const int pos = p.f.row_pos[r], sq = p.f.row_seq[r];
+                if (head < p.f.Hq + p.f.Hkv) {
+                    const float4 c01 = *reinterpret_cast<const float4*>(p.f.rope_tab + (size_t)r * 64 + 4 * q4);
+                    const float4 c23 = *reinterpret_cast<const float4*>(p.f.rope_tab + (size_t)r * 64 + 4 * q4 + 2);
+                    const float cs[4] = {c01.x, c01.z, c23.x, c23.z}, sn[4] = {c01.y, c01.w, c23.y, c23.w};
+                    float ra[4], rb[4];
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        ra[k] = av[k] * cs[k] - bv[k] * sn[k];
+                        rb[k] = bv[k] * cs[k] + av[k] * sn[k];
+                    }
+                    __nv_bfloat16* dst = head < p.f.Hq
+                        ? p.f.q + ((size_t)r * p.f.Hq + head) * 128
+                        : p.f.kcache + (((size_t)sq * p.f.Hkv + (head - p.f.Hq)) * p.f.S + pos) * 128;
+                    store_bf16x4(dst + 4 * q4, ra[0], ra[1], ra[2], ra[3]);
+                    store_bf16x4(dst + 64 + 4 * q4, rb[0], rb[1], rb[2], rb[3]);
+                } else {
+                    __nv_bfloat16* dst = p.f.vcache + ((size_t)sq * p.f.Hkv + (head - p.f.Hq - p.f.Hkv)) * 128 * p.f.Sp + pos;
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) {
+                        dst[(size_t)(4 * q4 + k) * p.f.Sp] = __float2bfloat16_rn(av[k]);
+                        dst[(size_t)(64 + 4 * q4 + k) * p.f.Sp] = __float2bfloat16_rn(bv[k]);
+                    }
+                }
+            }
+        }
+    } else if (p.f.mode == WD_FUSE_SWIGLU) {
+        // gate tile t and up tile t (same columns of the two matrices): h = silu(g) * u
+        constexpr int UN = 3;
+        const int tile = unit / p.tok_tiles, tokt = unit - tile * p.tok_tiles;
+        const int t_in = tile - p.seg_tile0[u.seg];
+        const int ug = (p.seg_tile0[0] + t_in) * p.tok_tiles + tokt, uu = (p.seg_tile0[1] + t_in) * p.tok_tiles + tokt;
+        const int ncg = n_contrib(p, G, ug), ncu = n_contrib(p, G, uu);
+        const int col = u.n0 + 4 * lane;
+        for (int t0 = wq; t0 < nt; t0 += 4 * UN) {
+            float4 gv[UN], uv[UN];
+            const float* base_g[UN];
+            const float* base_u[UN];
+            bool valid[UN];
+            float ss[UN];
+#pragma unroll
+            for (int i = 0; i < UN; ++i) {
+                const int t = t0 + 4 * i;
+                valid[i] = t < nt;
+                gv[i] = uv[i] = make_float4(0, 0, 0, 0);
+                base_g[i] = p.y + (size_t)(u.tok0 + (valid[i] ? t : 0)) * p.ncol + col;
+                base_u[i] = base_g[i] + p.f.F;
+                ss[i] = valid[i] ? sumsq_lane(p, u.tok0 + t, lane) : 0.f;
+            }
+            add_slices<UN, 2>(gv, base_g, valid, ncg, p.split_stride);
+            add_slices<UN, 2>(uv, base_u, valid, ncu, p.split_stride);
+#pragma unroll
+            for (int i = 0; i < UN; ++i) {
+                const int t = t0 + 4 * i;
+                if (valid[i]) {            // uniform across the warp
+                    const float inv = rsqrtf(warp_sum_f(ss[i]) * p.f.inv_d + p.f.eps);
+                    const float g0 = gv[i].x * inv, g1 = gv[i].y * inv, g2 = gv[i].z * inv, g3 = gv[i].w * inv;
+                    store_bf16x4(p.f.h + (size_t)(u.tok0 + t) * p.f.F + col,
+                                 g0 / (1.f + __expf(-g0)) * (uv[i].x * inv), g1 / (1.f + __expf(-g1)) * (uv[i].y * inv),
+                                 g2 / (1.f + __expf(-g2)) * (uv[i].z * inv), g3 / (1.f + __expf(-g3)) * (uv[i].w * inv));
+                }
+            }
+        }
+    }
 }
 
 // Persistent, stream-K: the K blocks of all output tiles form one line of W blocks and CTA c
@@ -79,6 +305,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // bars[0..NS) full | [NS..2NS) empty | [2NS, 2NS+1] accumulator full | [2NS+2, 2NS+3] accumulator empty
     uint32_t* tmem_slot = (uint32_t*)(bars + 2 * NS + 4);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+    int* last_flag = (int*)(tmem_slot + 2);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long c = blockIdx.x, G = gridDim.x;
@@ -91,6 +318,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         g_end = (c + 1) * p.W / G;
     }
     const int n_total = (int)(g_end - g_begin);
+    Sched sch;
+    sch.init(g_begin, g_end, p.kb_total);
 
     pdl_launch_dependents();      // the next kernel may start its own prologue / weight prefetch
     if (threadIdx.x == 0) {
@@ -118,28 +347,30 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             // ------------------------------------------------ TMA producer
             uint64_t pol_stream;
             asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
-            // walks the K blocks of this CTA's piece of the line without divisions
+            // walks the K blocks of this CTA's pieces in schedule order without per-block divisions
             struct Walk {
-                int unit, kb, n0, tok0;
+                int piece, left, kb, n0, tok0;
                 const CUtensorMap* mw;
             };
-            auto decode = [&](Walk& w) {
-                const UnitInfo u = decode_unit(p, w.unit);
+            auto enter = [&](Walk& w) {                    // position on the first block of piece w.piece
+                long long g;
+                int len;
+                sch.piece(w.piece, g, len);
+                const int unit = (int)(g / p.kb_total);
+                w.kb = (int)(g - (long long)unit * p.kb_total);
+                w.left = len;
+                const UnitInfo u = decode_unit(p, unit);
                 w.n0 = u.n0;
                 w.tok0 = u.tok0;
                 w.mw = u.seg == 0 ? &map_w0 : (u.seg == 1 ? &map_w1 : &map_w2);
             };
             auto advance = [&](Walk& w) {
-                if (++w.kb == p.kb_total) {
-                    w.kb = 0;
-                    ++w.unit;
-                    decode(w);
-                }
+                ++w.kb;
+                if (--w.left == 0 && ++w.piece < sch.n_pieces) enter(w);
             };
             Walk w0;
-            w0.unit = (int)(g_begin / p.kb_total);
-            w0.kb = (int)(g_begin - (long long)w0.unit * p.kb_total);
-            decode(w0);
+            w0.piece = 0;
+            enter(w0);
             // Weights never depend on earlier kernels of the stream: fill the ring with weight
             // boxes first, then wait for the producer of the activations, then add their boxes.
             const int n_pre = n_total < NS ? n_total : NS;
@@ -175,12 +406,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         if (lane == 0) {
             // ------------------------------------------------ MMA issuer
             bool ok = true;
-            int piece = 0, s = 0;
+            int s = 0;
             uint32_t ph = 0;
-            long long g = g_begin;
-            while (g < g_end && ok) {
-                const int unit = (int)(g / p.kb_total), kb0 = (int)(g - (long long)unit * p.kb_total);
-                const int len = (int)((long long)(p.kb_total - kb0) < g_end - g ? (p.kb_total - kb0) : g_end - g);
+            for (int piece = 0; piece < sch.n_pieces && ok; ++piece) {
+                long long g;
+                int len;
+                sch.piece(piece, g, len);
                 const int buf = piece & 1;
                 // the epilogue has drained this accumulator (free at the start)
                 if (!(ok = mbar_wait(smem_u32(&bars[2 * NS + 2 + buf]), ((uint32_t)(piece >> 1) & 1u) ^ 1u, abort_flag))) break;
@@ -202,8 +433,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     if (++s == NS) { s = 0; ph ^= 1u; }
                 }
                 if (ok) umma_commit(smem_u32(&bars[2 * NS + buf]));  // this piece's accumulator complete
-                g += len;
-                ++piece;
             }
             if (!ok) {
                 *abort_flag = 1;
@@ -217,11 +446,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         const int n_local = quarter * 32 + lane;
         pdl_wait();      // the previous reader of y has finished (already implied by the data flow)
         bool ok = true;
-        int piece = 0;
-        long long g = g_begin;
-        while (g < g_end) {
+        for (int piece = 0; piece < sch.n_pieces; ++piece) {
+            long long g;
+            int len;
+            sch.piece(piece, g, len);
             const int unit = (int)(g / p.kb_total), kb0 = (int)(g - (long long)unit * p.kb_total);
-            const int len = (int)((long long)(p.kb_total - kb0) < g_end - g ? (p.kb_total - kb0) : g_end - g);
             const UnitInfo u = decode_unit(p, unit);
             const int buf = piece & 1;
             const int n = u.n0 + n_local;
@@ -249,15 +478,38 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             }
             tc_fence_before();
             mbar_arrive(smem_u32(&bars[2 * NS + 2 + buf]));       // accumulator may be overwritten
-            if (kb0 + len == p.kb_total && n_ok) {
+            if (p.f.mode != WD_FUSE_NONE) {
+                // count this piece's arrival at its tile; the CTA that arrives last finishes the tile
+                const int e = (int)threadIdx.x - 64;
+                __threadfence();
+                epi_sync();
+                if (e == 0) {
+                    int idx = unit, expected;
+                    if (p.f.mode == WD_FUSE_SWIGLU) {
+                        const int tile = unit / p.tok_tiles, tokt = unit - tile * p.tok_tiles;
+                        const int t_in = tile - p.seg_tile0[u.seg];
+                        idx = t_in * p.tok_tiles + tokt;
+                        expected = n_contrib(p, G, (p.seg_tile0[0] + t_in) * p.tok_tiles + tokt) +
+                                   n_contrib(p, G, (p.seg_tile0[1] + t_in) * p.tok_tiles + tokt);
+                    } else {
+                        expected = n_contrib(p, G, unit);
+                    }
+                    const int old = atomicAdd(p.f.counters + idx, 1);
+                    const int last = (old + 1 == expected) ? 1 : 0;
+                    if (last) p.f.counters[idx] = 0;               // ready for the next launch
+                    *last_flag = last;
+                    __threadfence();
+                }
+                epi_sync();
+                if (*last_flag) finalize_unit(p, G, unit, e);
+                epi_sync();
+            } else if (kb0 + len == p.kb_total && n_ok) {
                 // this CTA finished the tile: slices nobody wrote must read as zero
                 for (int sl = ord + 1; sl < p.n_slices; ++sl) {
                     float* ys = yb + (size_t)sl * p.split_stride;
                     for (int tok = u.tok0; tok < u.tok0 + p.bn && tok < p.rows; ++tok) ys[(size_t)tok * p.ncol] = 0.f;
                 }
             }
-            g += len;
-            ++piece;
         }
         if (!ok && lane == 0) {
             *abort_flag = 1;
@@ -335,10 +587,10 @@ TcConfig pick_config(int rows) {
     const int stage = kStageA + c.bn * kBK * 2;
     static const int want2 = env_int("WD_GEMM_CTAS_PER_SM", 1);
     c.ctas_per_sm = (want2 == 2 && c.bn <= 64) ? 2 : 1;
-    c.n_stages = ((c.ctas_per_sm == 2 ? 104 : 200) * 1024) / stage;
+    c.n_stages = ((c.ctas_per_sm == 2 ? 100 : 196) * 1024) / stage;
     if (c.n_stages > 10) c.n_stages = 10;
     if (c.n_stages < 2) c.n_stages = 2;
-    c.smem = (size_t)c.n_stages * stage + (2 * c.n_stages + 4) * 8 + 16 + 1024;
+    c.smem = (size_t)c.n_stages * stage + (2 * c.n_stages + 4) * 8 + 16 + 4096 + 1024;
     return c;
 }
 
@@ -393,7 +645,8 @@ wd_status wd_tc_weights_init(WdTcWeights* tc, const wd_model_dims* d, const void
 }
 
 wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, int K, float* y, size_t y_floats,
-                     int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out, bool force_single_split) {
+                     int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out, bool force_single_split,
+                     const WdTcFuse* fuse) {
     if (!x || !segs || !y || !status || nseg < 1 || nseg > 3) return WD_ERR_BAD_PARAM;
     if (rows < 1 || K < 8 || K % 8) return WD_ERR_BAD_PARAM;
     TcParams p;
@@ -436,6 +689,12 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     p.split_stride = slice;
     p.status = status;
     p.idesc = make_idesc(cfg.bn);
+    if (fuse) {
+        p.f = *fuse;
+        if (fuse->mode != WD_FUSE_NONE && !fuse->counters) return WD_ERR_NULL;
+        if (fuse->mode == WD_FUSE_SWIGLU && (nseg != 2 || segs[0].n != segs[1].n)) return WD_ERR_BAD_PARAM;
+        if (fuse->mode != WD_FUSE_NONE && col % kBM) return WD_ERR_BAD_PARAM;      // whole tiles only
+    }
 
     CUtensorMap mx;
     wd_status s = encode_2d(&mx, x->ptr, rows, K, cfg.bn);

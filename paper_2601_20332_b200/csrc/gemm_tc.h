@@ -38,11 +38,43 @@ wd_status wd_tc_weights_init(WdTcWeights* tc, const wd_model_dims* d, const void
                              const std::vector<const void*>& wg, const std::vector<const void*>& wu,
                              const std::vector<const void*>& wd, const void* xn, const void* attn, const void* h);
 
+// What the CTA that completes an output tile does with the summed tile ("fused epilogue").
+// The tile sums still pass through the partial-sum slices in y; these modes only add the
+// consumer's work to the GEMM so that no separate kernel (and no dependency bubble) follows.
+enum { WD_FUSE_NONE = 0, WD_FUSE_QKV = 1, WD_FUSE_RESID = 2, WD_FUSE_SWIGLU = 3 };
+
+struct WdTcFuse {
+    int mode = WD_FUSE_NONE;
+    int32_t* counters = nullptr;      // zeroed ints, one per output tile (left zeroed again on return)
+    int rows_total = 0;
+    // QKV and SWIGLU: the input rows were not normalised; scale by 1/rms from these partial sums of squares
+    const float* sumsq_in = nullptr;  // [n_prev_tiles][rows_total]
+    int n_prev_tiles = 0;
+    float inv_d = 0.f, eps = 0.f;
+    // QKV: rotate q/k heads, write q and the K / transposed-V cache rows (head_dim 128 = one tile per head)
+    const int32_t* row_seq = nullptr;
+    const int32_t* row_pos = nullptr;
+    const float2* rope_tab = nullptr;
+    __nv_bfloat16* q = nullptr;
+    __nv_bfloat16* kcache = nullptr;
+    __nv_bfloat16* vcache = nullptr;
+    int Hq = 0, Hkv = 0, S = 0, Sp = 0;
+    // RESID: x += tile; xg = bf16(x * gain_next) for the next GEMM; partial sums of squares of the new x
+    float* x = nullptr;
+    const float* gain_next = nullptr; // null: no xg (after the last block)
+    __nv_bfloat16* xg = nullptr;
+    float* sumsq_out = nullptr;       // [d/128][rows_total]
+    float* tap = nullptr;
+    // SWIGLU: h = silu(gate) * up, gate tile t and up tile t complete together
+    __nv_bfloat16* h = nullptr;
+    int F = 0;
+};
+
 // y[split][rows][sum n_i] = x * [w_0; w_1; ...]^T, split-K partial sums side by side
 // (split_stride = rows * sum n_i floats).  The consumer adds the slices.
 wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, int K, float* y, size_t y_floats,
                      int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out,
-                     bool force_single_split = false);
+                     bool force_single_split = false, const WdTcFuse* fuse = nullptr);
 
 size_t wd_tc_scratch_bytes(int rows, int n_out, int k_in);
 wd_status wd_tc_gemm_standalone(const void* x, const void* w, float* y, int rows, int n_out, int k_in, void* scratch,

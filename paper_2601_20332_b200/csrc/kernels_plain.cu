@@ -73,6 +73,33 @@ __device__ __forceinline__ float block_max(float v, float* red) {
     return warp_max(t);
 }
 
+// Sum of n_split partial-sum slices at one float4 position.  Slices are loaded four at a time
+// before the first add so that their L2 round trips overlap; the adds keep slice order.
+__device__ __forceinline__ float4 sum_slices4(const float* __restrict__ p, int n_split, size_t stride) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s0 = 0; s0 < n_split; s0 += 4) {
+        float4 t[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k)
+            t[k] = s0 + k < n_split ? *reinterpret_cast<const float4*>(p + (size_t)(s0 + k) * stride)
+                                    : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) { acc.x += t[k].x; acc.y += t[k].y; acc.z += t[k].z; acc.w += t[k].w; }
+    }
+    return acc;
+}
+__device__ __forceinline__ float sum_slices1(const float* __restrict__ p, int n_split, size_t stride) {
+    float acc = 0.f;
+    for (int s0 = 0; s0 < n_split; s0 += 4) {
+        float t[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) t[k] = s0 + k < n_split ? p[(size_t)(s0 + k) * stride] : 0.f;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) acc += t[k];
+    }
+    return acc;
+}
+
 // ---------------------------------------------------------------- embedding gather + RoPE table
 // One block per computed row.  Also fills this step's rotary table: (cos, sin) of
 // pos * theta^(-2j/dh) for j < dh/2, evaluated in double so that the angle of a late position
@@ -100,6 +127,48 @@ __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restr
     }
     const T* src = embed + (size_t)id * d;
     for (int c = threadIdx.x; c < d; c += blockDim.x) x[(size_t)r * d + c] = to_f(src[c]);
+}
+
+// Same gather for the fused pipeline: besides x it writes xg = bf16(x * gain) (the un-normalised
+// GEMM input; the 1/rms factor is applied by the GEMM's consumer) and the per-row sums of
+// squares of every 128-column block, sumsq[block][row].  Warp w owns blocks w, w+8, ...; the
+// sum inside a block is a fixed shuffle tree, so the result is reproducible bit for bit.
+__global__ void embed_fused_kernel(const __nv_bfloat16* __restrict__ embed, const int32_t* __restrict__ ids,
+                                   const int32_t* __restrict__ row_seq, const int32_t* __restrict__ row_pos,
+                                   float* __restrict__ x, __nv_bfloat16* __restrict__ xg, const float* __restrict__ gain,
+                                   float* __restrict__ sumsq, float2* __restrict__ rope_tab, int n_rows, int d, int S,
+                                   int vocab, int dh, double log2_theta, int32_t* status) {
+    pdl_launch_dependents();
+    pdl_wait();
+    const int r = blockIdx.x;
+    const int pos = row_pos[r];
+    for (int j = threadIdx.x; j < dh / 2; j += blockDim.x) {
+        const double ang = (double)pos * exp2(-2.0 * (double)j / (double)dh * log2_theta);
+        double sn, cs;
+        sincos(ang, &sn, &cs);
+        rope_tab[(size_t)r * (dh / 2) + j] = make_float2((float)cs, (float)sn);
+    }
+    int id = ids[(size_t)row_seq[r] * S + pos];
+    const bool bad = id < 0 || id >= vocab;
+    if (bad) {
+        if (threadIdx.x == 0) atomicCAS(status, 0, WD_ERR_BOUNDS);
+        id = 0;
+    }
+    const __nv_bfloat16* src = embed + (size_t)id * d;
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    for (int blk = w; blk < d / 128; blk += nw) {
+        float ss = 0.f;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = blk * 128 + lane * 4 + i;
+            const float v = bad ? 0.f : __bfloat162float(src[c]);
+            x[(size_t)r * d + c] = v;
+            xg[(size_t)r * d + c] = __float2bfloat16_rn(v * gain[c]);
+            ss += v * v;
+        }
+        ss = warp_sum(ss);
+        if (lane == 0) sumsq[(size_t)blk * n_rows + r] = ss;
+    }
 }
 
 // ---------------------------------------------------------------- RMSNorm (+ partial-sum add)
@@ -132,18 +201,23 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ 
     const int r = row_idx ? row_idx[i] : i;
     float* xr = x + (size_t)r * d;
     const int nv = d >> 2;
-    float4 v[MAXV];
+    float4 v[MAXV], add[MAXV];
     float ss = 0.f;
+#pragma unroll
+    for (int u = 0; u < MAXV; ++u) {             // all loads first: x and every slice of every group
+        const int c4 = threadIdx.x + u * blockDim.x;
+        if (c4 < nv) {
+            v[u] = reinterpret_cast<const float4*>(xr)[c4];
+            if (part) add[u] = sum_slices4(part + (size_t)r * d + 4 * c4, n_split, split_stride);
+        }
+    }
 #pragma unroll
     for (int u = 0; u < MAXV; ++u) {
         const int c4 = threadIdx.x + u * blockDim.x;
         if (c4 < nv) {
-            float4 a = reinterpret_cast<const float4*>(xr)[c4];
+            float4 a = v[u];
             if (part) {
-                for (int s = 0; s < n_split; ++s) {
-                    const float4 b = reinterpret_cast<const float4*>(part + s * split_stride + (size_t)r * d)[c4];
-                    a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w;
-                }
+                a.x += add[u].x; a.y += add[u].y; a.z += add[u].z; a.w += add[u].w;
                 reinterpret_cast<float4*>(xr)[c4] = a;
             }
             v[u] = a;
@@ -230,11 +304,8 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
     for (int i = threadIdx.x; i < 4 * half; i += blockDim.x) {
         const int h = h0 + i / half, j = i % half;
         if (h >= Hq + 2 * Hkv) break;
-        float a = 0.f, bb = 0.f;
-        for (int s = 0; s < n_split; ++s) {
-            a += pr[s * split_stride + h * dh + j];
-            bb += pr[s * split_stride + h * dh + j + half];
-        }
+        const float a = sum_slices1(pr + h * dh + j, n_split, split_stride);
+        const float bb = sum_slices1(pr + h * dh + j + half, n_split, split_stride);
         if (h < Hq + Hkv) {
             const float2 cs = rope_tab[(size_t)r * half + j];
             const float ra = a * cs.x - bb * cs.y, rb = bb * cs.x + a * cs.y;
@@ -321,13 +392,8 @@ __global__ void swiglu_kernel(const float* __restrict__ part, int n_split, size_
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (size_t)gridDim.x * blockDim.x) {
         const size_t r = i / f4, c4 = i - r * f4;
-        float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
-        for (int s = 0; s < n_split; ++s) {
-            const float4* p = reinterpret_cast<const float4*>(part + s * split_stride + r * 2 * F);
-            const float4 a = p[c4], b = p[f4 + c4];
-            g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w;
-            u.x += b.x; u.y += b.y; u.z += b.z; u.w += b.w;
-        }
+        const float4 g = sum_slices4(part + r * 2 * F + 4 * c4, n_split, split_stride);
+        const float4 u = sum_slices4(part + r * 2 * F + F + 4 * c4, n_split, split_stride);
         Vec4<T>::store(h + r * F + 4 * c4, g.x / (1.f + __expf(-g.x)) * u.x, g.y / (1.f + __expf(-g.y)) * u.y,
                        g.z / (1.f + __expf(-g.z)) * u.z, g.w / (1.f + __expf(-g.w)) * u.w);
     }
@@ -339,8 +405,7 @@ __global__ void residual_add_kernel(float* __restrict__ x, const float* __restri
     pdl_wait();
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
          i += (size_t)gridDim.x * blockDim.x) {
-        float v = x[i];
-        for (int s = 0; s < n_split; ++s) v += part[s * split_stride + i];
+        const float v = x[i] + sum_slices1(part + i, n_split, split_stride);
         x[i] = v;
         if (tap) tap[i] = v;
     }
@@ -475,6 +540,14 @@ void wd_launch_embed(int dtype, const void* embed, const int32_t* ids, const int
     const double l2 = log2((double)theta);
     WD_DISPATCH(dtype, launch_pdl(embed_kernel<T>, dim3(n_rows), dim3(256), 0, st, (const T*)embed, ids, row_seq,
                                   row_pos, x, rope_tab, d, S, vocab, dh, l2, status));
+}
+
+void wd_launch_embed_fused(const void* embed, const int32_t* ids, const int32_t* row_seq, const int32_t* row_pos,
+                           float* x, void* xg, const float* gain, float* sumsq, float2* rope_tab, int n_rows, int d, int S,
+                           int vocab, int dh, float theta, int32_t* status, cudaStream_t st) {
+    if (n_rows <= 0) return;
+    launch_pdl(embed_fused_kernel, dim3(n_rows), dim3(256), 0, st, (const __nv_bfloat16*)embed, ids, row_seq, row_pos, x,
+               (__nv_bfloat16*)xg, gain, sumsq, rope_tab, n_rows, d, S, vocab, dh, log2((double)theta), status);
 }
 
 void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size_t split_stride,

@@ -59,6 +59,11 @@ void wd_launch_embed(int dtype, const void* embed, const int32_t* ids, const int
                      const int32_t* row_pos, float* x, float2* rope_tab, int n_rows, int d, int S, int vocab, int dh,
                      float theta, int32_t* status, cudaStream_t st);
 
+// fused pipeline (bf16): x, xg = bf16(x * gain), sumsq[d/128][n_rows] partial sums of squares, rope_tab
+void wd_launch_embed_fused(const void* embed, const int32_t* ids, const int32_t* row_seq, const int32_t* row_pos,
+                           float* x, void* xg, const float* gain, float* sumsq, float2* rope_tab, int n_rows, int d, int S,
+                           int vocab, int dh, float theta, int32_t* status, cudaStream_t st);
+
 // x += sum_s part[s] (if part != null); xn = rmsnorm(x) * gain, written as `dtype`.
 // With row_idx != null the rows x[row_idx[i]] are read (no partial add, x not written)
 // and xn[i] is written: used for the final norm over the active rows only.  d % 4 == 0.

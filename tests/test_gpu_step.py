@@ -18,10 +18,10 @@ def built():
 
 
 def run(cfg, n_steps, ids=None, decoded=None, impl=wd.WD_GEMM_AUTO, jitter=0.1, tol_layer=1e-2, tol_attn=2e-2,
-        oracle_seqs=None, weights=None):
+        oracle_seqs=None, weights=None, fusion=False):
     w = synth.make_weights(cfg, DEV, gain_jitter=jitter) if weights is None else weights
     ids = synth.make_prompts(cfg) if ids is None else ids
-    p = Parity(cfg, w, ids, decoded, gemm_impl=impl, oracle_seqs=oracle_seqs)
+    p = Parity(cfg, w, ids, decoded, gemm_impl=impl, oracle_seqs=oracle_seqs, fusion=fusion)
     logs = []
     for _ in range(n_steps):
         r = p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"], tol_layer, tol_attn)
@@ -70,12 +70,13 @@ def test_small_bf16_gqa_batch_two_tokens():
 DH128 = dict(L=2, d=512, Hq=4, Hkv=4, dh=128, F=1024, V=4000, P=200, G=150, A=16, B=40, R=3, T=2, k=2)
 
 
-@pytest.mark.parametrize("Hkv,batch", [(4, 1), (2, 2), (1, 1)])
-def test_bf16_head_dim_128_tensor_core_attention(Hkv, batch):
+@pytest.mark.parametrize("Hkv,batch,fusion", [(4, 1, False), (2, 2, False), (1, 1, False), (4, 1, True), (2, 2, True)])
+def test_bf16_head_dim_128_tensor_core_attention(Hkv, batch, fusion):
     """head_dim 128 takes the tcgen05 attention: two query tiles at the refresh (256 visible
-    rows), three key tiles with a ragged tail, MHA and GQA, batch of independent windows."""
+    rows), key tiles with a ragged tail split across CTAs, MHA and GQA, batch of independent
+    windows; with and without the fused GEMM epilogues."""
     cfg = synth.get_config("llada8b", **dict(DH128, Hkv=Hkv, batch=batch))
-    logs = run(cfg, 7)
+    logs = run(cfg, 7, fusion=fusion)
     assert [l["info"]["is_refresh"] for l in logs] == [1, 0, 0, 1, 0, 0, 1]
     assert logs[0]["info"]["n_rows"] == batch * 256
 

@@ -33,7 +33,7 @@ def max_rel(a, b):
 
 class Parity:
     def __init__(self, cfg, weights, ids, decoded=None, gemm_impl=wd.WD_GEMM_AUTO, oracle_seqs=None,
-                 max_rows=None, max_active=None):
+                 max_rows=None, max_active=None, fusion=False):
         self.cfg = cfg
         self.batch, self.S = ids.shape
         dev = weights.tok_embed.device
@@ -41,6 +41,7 @@ class Parity:
         max_active = max_rows if max_active is None else max_active
         self.ctx = wd.Context(cfg, weights, self.batch, self.S, max_rows, max_active)
         self.ctx.set_gemm_impl(gemm_impl)
+        self.ctx.set_fusion(fusion)
         self.st = wd.State(self.ctx, ids, decoded)
         L, d, hq, V = cfg["L"], cfg["d"], cfg["Hq"] * cfg["dh"], cfg["V"]
         self.t_layer = torch.zeros(L * max_rows * d, dtype=torch.float32, device=dev)
