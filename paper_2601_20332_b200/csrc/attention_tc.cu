@@ -10,10 +10,11 @@
 //   warp 0    TMA: the Q tile once, then [128 keys x 128] K boxes and [128 x 128 keys] boxes of
 //             the transposed V cache into a two-stage ring
 //   warp 1    tcgen05.mma: S = Q K^T into TMEM, then O_tile = P V into TMEM
-//   warps 2-5 one thread per query row: tcgen05.ld of its S row, online softmax in fp32
-//             (exp2 with the scale folded in), P as bf16 into shared memory in the 128-byte
-//             swizzled operand layout, then tcgen05.ld of its O_tile row accumulated in
-//             registers with the running rescale; final O / l written as bf16
+//   warps 2-9 two threads per query row (each takes 64 of the tile's 128 columns): tcgen05.ld of
+//             its half of the S row, online softmax in fp32 (exp2 with the scale folded in; the
+//             two halves exchange their row maxima through shared memory), P as bf16 into shared
+//             memory in the 128-byte swizzled operand layout, then tcgen05.ld of its half of the
+//             O_tile row accumulated in registers with the running rescale; final O / l as bf16
 // Query rows beyond the tile's valid rows are computed on whatever the box holds and discarded
 // (rows are independent).  Keys at or beyond n_vis are masked by selection, and their V
 // columns are zeroed in shared memory, so stale or poisoned cache rows cannot leak in.
@@ -33,7 +34,7 @@ using namespace wdk;
 constexpr int kTile = 128;                 // query rows per CTA = keys per step = head_dim
 constexpr int kAtom = kTile * 64 * 2;      // one [128 x 64] bf16 swizzle-atom column: 16 KB
 constexpr int kOperand = 2 * kAtom;        // a [128 x 128] bf16 operand: 32 KB
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;            // TMA warp, MMA warp, 8 softmax warps
 constexpr int kTmemCols = 256;             // S: columns 0..127, O_tile: columns 128..255
 
 struct AttnParams {
@@ -88,7 +89,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     if (kt_begin >= n_kt_all) return;                       // nothing for this CTA (uniform exit)
     const int n_kt = min(p.tiles_per_split, n_kt_all - kt_begin);
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 8; ++i) mbar_init(smem_u32(&bars[i]), i == 6 ? 128u : 1u);
+        for (int i = 0; i < 8; ++i) mbar_init(smem_u32(&bars[i]), i == 6 ? 256u : 1u);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -163,97 +164,100 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         }
         __syncwarp();
     } else {
-        // -------------------------------------------------------- softmax + accumulate (one row per thread)
-        const int quarter = warp & 3;
+        // -------------------------------------------------------- softmax + accumulate (two threads per row)
+        const int quarter = warp & 3;                      // TMEM lanes 32*quarter .. +31
+        const int hf = (warp - 2) >> 2;                    // which 64 columns of a 128-wide tile
         const int r = quarter * 32 + lane;                 // query row of the tile = TMEM lane
+        const int c_off = 64 * hf;
         const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        float o[kTile];
+        float* xch = (float*)(tmem_slot + 4);              // [2][128] exchange between the two halves
+        float o[64];
 #pragma unroll
-        for (int c = 0; c < kTile; ++c) o[c] = 0.f;
+        for (int c = 0; c < 64; ++c) o[c] = 0.f;
         float m = -INFINITY, l = 0.f;
         bool ok = true;
         for (int i = 0; i < n_kt; ++i) {
             const int s = i & 1;
-            ok = ok && mbar_wait(smem_u32(&bars[5]), (uint32_t)i & 1u, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+            // A failed wait must not leave the loop before the named barrier below (the other
+            // warps would wait there for ever): it raises the CTA's abort flag, every thread still
+            // reaches the barrier, and all of them leave together right after it.
+            if (!mbar_wait(smem_u32(&bars[5]), (uint32_t)i & 1u, abort_flag)) *abort_flag = 1;
             tc_fence_after();
             const int n_keys = min(kTile, n_vis - (kt_begin + i) * kTile);   // valid keys in this tile
             // keys past n_vis may hold anything: zero their V columns so that 0 * garbage stays 0.
-            // Thread r owns row r (a head dim) of the transposed V tile.
-            if (n_keys < kTile) {
-                uint8_t* vt = sKV + (size_t)s * 2 * kOperand + kOperand;
-                for (int kv = n_keys; kv < kTile; ++kv) {
-                    const int a = kv >> 6, c16 = (kv & 63) >> 3, e = kv & 7;
-                    *reinterpret_cast<uint16_t*>(vt + a * kAtom + r * 128 + ((c16 ^ (r & 7)) << 4) + e * 2) = 0;
-                }
+            // Thread (r, hf) owns row r (a head dim) of atom hf (keys 64*hf..) of the transposed V tile.
+            if (n_keys < c_off + 64) {
+                uint8_t* vt = sKV + (size_t)s * 2 * kOperand + kOperand + hf * kAtom + r * 128;
+                for (int kv = max(n_keys - c_off, 0); kv < 64; ++kv)
+                    *reinterpret_cast<uint16_t*>(vt + (((kv >> 3) ^ (r & 7)) << 4) + (kv & 7) * 2) = 0;
             }
-            // pass 1: row maximum of the scaled scores
-            float mx = m;
+            // scaled scores of this thread's 64 keys, kept in registers for both passes
+            float sc[64];
+            float mx = -INFINITY;
 #pragma unroll
-            for (int c0 = 0; c0 < kTile; c0 += 32) {
+            for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
-                tmem_ld32(t_row + (uint32_t)c0, v);
+                tmem_ld32(t_row + (uint32_t)(c_off + c0), v);
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
-                    const float sv = (c0 + c < n_keys) ? __uint_as_float(v[c]) * p.scale_log2e : -INFINITY;
-                    mx = fmaxf(mx, sv);
+                    sc[c0 + c] = (c_off + c0 + c < n_keys) ? __uint_as_float(v[c]) * p.scale_log2e : -INFINITY;
+                    mx = fmaxf(mx, sc[c0 + c]);
                 }
             }
+            xch[hf * kTile + r] = mx;
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            if (*abort_flag) { ok = false; break; }
+            mx = fmaxf(fmaxf(mx, xch[(hf ^ 1) * kTile + r]), m);
             const float alpha = exp2f(m - mx);             // m = -inf on the first tile gives 0
             m = mx;
             l *= alpha;
-            // pass 2: probabilities, row sum, P as bf16 into the swizzled A-operand tile
+            uint8_t* prow = sP + hf * kAtom + r * 128;
 #pragma unroll
-            for (int c0 = 0; c0 < kTile; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(t_row + (uint32_t)c0, v);
-                float pr[32];
+            for (int g = 0; g < 8; ++g) {                  // eight 16-byte chunks of 8 keys
+                float pr[8];
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    pr[c] = (c0 + c < n_keys) ? exp2f(__uint_as_float(v[c]) * p.scale_log2e - mx) : 0.f;
+                for (int c = 0; c < 8; ++c) {
+                    pr[c] = exp2f(sc[8 * g + c] - mx);     // masked keys: exp2(-inf) = 0
                     l += pr[c];
                 }
-                uint8_t* prow = sP + (c0 >> 6) * kAtom + r * 128;
-#pragma unroll
-                for (int g = 0; g < 4; ++g) {              // four 16-byte chunks of 8 keys
-                    const int c16 = ((c0 & 63) >> 3) + g;
-                    uint4 u;
-                    u.x = pack_bf16(pr[8 * g + 0], pr[8 * g + 1]);
-                    u.y = pack_bf16(pr[8 * g + 2], pr[8 * g + 3]);
-                    u.z = pack_bf16(pr[8 * g + 4], pr[8 * g + 5]);
-                    u.w = pack_bf16(pr[8 * g + 6], pr[8 * g + 7]);
-                    *reinterpret_cast<uint4*>(prow + ((c16 ^ (r & 7)) << 4)) = u;
-                }
+                uint4 u;
+                u.x = pack_bf16(pr[0], pr[1]);
+                u.y = pack_bf16(pr[2], pr[3]);
+                u.z = pack_bf16(pr[4], pr[5]);
+                u.w = pack_bf16(pr[6], pr[7]);
+                *reinterpret_cast<uint4*>(prow + ((g ^ (r & 7)) << 4)) = u;
             }
             tc_fence_before();
             fence_proxy_async_smem();                      // P and the zeroed V columns -> visible to the MMA
             mbar_arrive(smem_u32(&bars[6]));
-            // O += O_tile with the running rescale
-            ok = mbar_wait(smem_u32(&bars[7]), (uint32_t)i & 1u, abort_flag);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
+            // O += O_tile with the running rescale (a failed wait is picked up at the next barrier)
+            if (!mbar_wait(smem_u32(&bars[7]), (uint32_t)i & 1u, abort_flag)) { *abort_flag = 1; ok = false; }
             tc_fence_after();
 #pragma unroll
-            for (int c0 = 0; c0 < kTile; c0 += 32) {
+            for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
-                tmem_ld32(t_row + (uint32_t)(kTile + c0), v);
+                tmem_ld32(t_row + (uint32_t)(kTile + c_off + c0), v);
 #pragma unroll
                 for (int c = 0; c < 32; ++c) o[c0 + c] = o[c0 + c] * alpha + __uint_as_float(v[c]);
             }
             tc_fence_before();
         }
-        if (!ok && lane == 0) {
-            *abort_flag = 1;
-            atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
+        // row sum = sum of the two halves (same running maximum on both sides)
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (*abort_flag) {
+            ok = false;
+            if (threadIdx.x == 64) atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
         }
+        xch[hf * kTile + r] = l;
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        l += xch[(hf ^ 1) * kTile + r];
         if (n_parts == 1) {
             if (ok && r < n_valid) {
                 const float inv = 1.f / l;
-                const size_t base = ((size_t)(row0 + r) * p.Hq + h) * kTile;
+                const size_t base = ((size_t)(row0 + r) * p.Hq + h) * kTile + c_off;
                 uint4* dst = reinterpret_cast<uint4*>(p.out + base);
 #pragma unroll
-                for (int g = 0; g < kTile / 8; ++g) {
+                for (int g = 0; g < 8; ++g) {
                     uint4 u;
                     u.x = pack_bf16(o[8 * g + 0] * inv, o[8 * g + 1] * inv);
                     u.y = pack_bf16(o[8 * g + 2] * inv, o[8 * g + 3] * inv);
@@ -263,20 +267,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 }
                 if (p.tap) {
 #pragma unroll
-                    for (int c = 0; c < kTile; ++c) p.tap[base + c] = o[c] * inv;
+                    for (int c = 0; c < 64; ++c) p.tap[base + c] = o[c] * inv;
                 }
             }
         } else {
             // leave this CTA's part in scratch, count the arrival, the last CTA merges
             const size_t slot = ((size_t)tile * p.Hq + h) * p.max_parts;
             if (ok && r < n_valid) {
-                float4* dst = reinterpret_cast<float4*>(p.part_o + ((slot + blockIdx.z) * kTile + r) * kTile);
+                float4* dst = reinterpret_cast<float4*>(p.part_o + ((slot + blockIdx.z) * kTile + r) * kTile + c_off);
 #pragma unroll
-                for (int g = 0; g < kTile / 4; ++g) dst[g] = make_float4(o[4 * g], o[4 * g + 1], o[4 * g + 2], o[4 * g + 3]);
-                *reinterpret_cast<float2*>(p.part_ml + ((slot + blockIdx.z) * kTile + r) * 2) = make_float2(m, l);
+                for (int g = 0; g < 16; ++g) dst[g] = make_float4(o[4 * g], o[4 * g + 1], o[4 * g + 2], o[4 * g + 3]);
+                if (hf == 0)
+                    *reinterpret_cast<float2*>(p.part_ml + ((slot + blockIdx.z) * kTile + r) * 2) = make_float2(m, l);
             }
             __threadfence();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             int* last_flag = (int*)(tmem_slot + 2);
             if (threadIdx.x == 64) {
                 const int old = atomicAdd(p.counters + tile * p.Hq + h, 1);
@@ -285,17 +290,17 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 *last_flag = last;
                 __threadfence();
             }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             if (*last_flag) {
-                // warp `quarter` merges rows quarter, quarter + 4, ...; lanes hold 4 columns each
-                for (int rr = quarter; rr < n_valid; rr += 4) {
-                    float mx = -INFINITY;
-                    for (int z = 0; z < n_parts; ++z) mx = fmaxf(mx, __ldcg(p.part_ml + ((slot + z) * kTile + rr) * 2));
+                // warp w merges rows w, w + 8, ...; lanes hold 4 columns each
+                for (int rr = warp - 2; rr < n_valid; rr += 8) {
+                    float mxx = -INFINITY;
+                    for (int z = 0; z < n_parts; ++z) mxx = fmaxf(mxx, __ldcg(p.part_ml + ((slot + z) * kTile + rr) * 2));
                     float lsum = 0.f;
                     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
                     for (int z = 0; z < n_parts; ++z) {
                         const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot + z) * kTile + rr) * 2));
-                        const float wgt = exp2f(ml.x - mx);
+                        const float wgt = exp2f(ml.x - mxx);
                         const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_o + ((slot + z) * kTile + rr) * kTile) + lane);
                         lsum += ml.y * wgt;
                         acc.x += v.x * wgt; acc.y += v.y * wgt; acc.z += v.z * wgt; acc.w += v.w * wgt;
@@ -405,7 +410,7 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     p.part_o = scratch;
     p.part_ml = scratch ? scratch + (size_t)WD_ATTN_SPLIT_SLOTS * kTile * kTile : nullptr;
     p.counters = counters;
-    const size_t smem = 6 * (size_t)kOperand + 8 * 8 + 16 + 1024;
+    const size_t smem = 6 * (size_t)kOperand + 8 * 8 + 16 + 2 * kTile * 4 + 1024;
     WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(n_tiles, Hq, p.max_parts);

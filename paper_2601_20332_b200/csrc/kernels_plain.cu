@@ -284,39 +284,59 @@ __global__ void gemm_plain_kernel(const T* __restrict__ x, const T* __restrict__
 }
 
 // ---------------------------------------------------------------- RoPE + K/V scatter
-// grid (row, group of 4 heads); 256 threads.  Adds the split-K slices of the fused q/k/v
-// projection, rotates q and k heads by the row's table, writes q and the K/V cache rows.
-// K cache [batch][Hkv][S][dh]; V cache transposed [batch][Hkv][dh][Sp] so that attention can
-// read V tiles with the key position contiguous.
+// Adds the split-K slices of the fused q/k/v projection, rotates q and k heads by the row's
+// table, writes q and the K/V cache rows.  K cache [batch][Hkv][S][dh]; V cache transposed
+// [batch][Hkv][dh][Sp] so that attention can read V tiles with the key position contiguous.
+// One 1-D grid, two kinds of 256-thread blocks:
+//   blocks [0, n_qk):  (row, group of 4 q/k heads), one rotation pair per thread
+//   blocks [n_qk, ..): (v head, 32 head dims, 32 rows): slices summed with the dims contiguous,
+//                      transposed through shared memory and written with the rows (normally
+//                      consecutive positions) contiguous, so neighbouring lanes share sectors
 template <typename T>
 __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
                                     const int32_t* __restrict__ row_seq, const int32_t* __restrict__ row_pos,
                                     const float2* __restrict__ rope_tab, T* __restrict__ q, T* __restrict__ kcache,
-                                    T* __restrict__ vcache, int Hq, int Hkv, int dh, int S, int Sp) {
+                                    T* __restrict__ vcache, int n_rows, int Hq, int Hkv, int dh, int S, int Sp,
+                                    int n_qk, int qk_groups) {
+    __shared__ float tile[32][33];
     pdl_launch_dependents();
     pdl_wait();
-    const int r = blockIdx.x;
-    const int pos = row_pos[r], b = row_seq[r];
     const int half = dh >> 1;
     const int ncol = (Hq + 2 * Hkv) * dh;
-    const float* pr = part + (size_t)r * ncol;
-    const int h0 = blockIdx.y * 4;
-    for (int i = threadIdx.x; i < 4 * half; i += blockDim.x) {
-        const int h = h0 + i / half, j = i % half;
-        if (h >= Hq + 2 * Hkv) break;
-        const float a = sum_slices1(pr + h * dh + j, n_split, split_stride);
-        const float bb = sum_slices1(pr + h * dh + j + half, n_split, split_stride);
-        if (h < Hq + Hkv) {
+    if ((int)blockIdx.x < n_qk) {
+        const int r = blockIdx.x / qk_groups, h0 = (blockIdx.x - r * qk_groups) * 4;
+        const int pos = row_pos[r], b = row_seq[r];
+        const float* pr = part + (size_t)r * ncol;
+        for (int i = threadIdx.x; i < 4 * half; i += blockDim.x) {
+            const int h = h0 + i / half, j = i % half;
+            if (h >= Hq + Hkv) break;
+            const float a = sum_slices1(pr + h * dh + j, n_split, split_stride);
+            const float bb = sum_slices1(pr + h * dh + j + half, n_split, split_stride);
             const float2 cs = rope_tab[(size_t)r * half + j];
             const float ra = a * cs.x - bb * cs.y, rb = bb * cs.x + a * cs.y;
             T* dst = h < Hq ? q + ((size_t)r * Hq + h) * dh : kcache + (((size_t)b * Hkv + (h - Hq)) * S + pos) * dh;
             dst[j] = from_f<T>(ra);
             dst[j + half] = from_f<T>(rb);
-        } else {
-            T* dst = vcache + ((size_t)b * Hkv + (h - Hq - Hkv)) * dh * Sp + pos;
-            dst[(size_t)j * Sp] = from_f<T>(a);
-            dst[(size_t)(j + half) * Sp] = from_f<T>(bb);
         }
+        return;
+    }
+    const int vb = blockIdx.x - n_qk;
+    const int dchunks = (dh + 31) / 32, rchunks = (n_rows + 31) / 32;
+    const int kh = vb / (dchunks * rchunks), rem = vb - kh * dchunks * rchunks;
+    const int d0 = (rem / rchunks) * 32, r0 = (rem % rchunks) * 32;
+    const int lx = threadIdx.x & 31, ly = threadIdx.x >> 5;
+    const int vcol = (Hq + Hkv) * dh + kh * dh + d0;
+    for (int rr = ly; rr < 32; rr += 8) {
+        const int r = r0 + rr;
+        tile[rr][lx] = (r < n_rows && d0 + lx < dh)
+            ? sum_slices1(part + (size_t)r * ncol + vcol + lx, n_split, split_stride) : 0.f;
+    }
+    __syncthreads();
+    const int r = r0 + lx;
+    if (r < n_rows) {
+        const int pos = row_pos[r], b = row_seq[r];
+        T* dst = vcache + ((size_t)b * Hkv + kh) * dh * Sp + pos;
+        for (int dd = ly; dd < 32 && d0 + dd < dh; dd += 8) dst[(size_t)(d0 + dd) * Sp] = from_f<T>(tile[lx][dd]);
     }
 }
 
@@ -554,13 +574,15 @@ void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size
                        const float* gain, float eps, void* xn, const int32_t* row_idx, int n_rows,
                        int d, cudaStream_t st) {
     if (n_rows <= 0) return;
-    // 256 threads x MAXV float4 per thread cover d; pick the smallest MAXV that fits
+    // one float4 per thread where the row allows it: the kernel is a chain of dependent L2 round
+    // trips, so short per-thread work matters more than occupancy
     const int nv = d >> 2;
-    if (nv <= 256 * 2) {
-        WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 2>, dim3(n_rows), dim3(256), 0, st, x, part, n_split,
+    if (nv <= 1024) {
+        const int threads = (nv + 31) / 32 * 32;
+        WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 1>, dim3(n_rows), dim3(threads), 0, st, x, part, n_split,
                                       split_stride, gain, eps, (T*)xn, row_idx, d));
-    } else if (nv <= 256 * 4) {
-        WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 4>, dim3(n_rows), dim3(256), 0, st, x, part, n_split,
+    } else if (nv <= 2048) {
+        WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 2>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split,
                                       split_stride, gain, eps, (T*)xn, row_idx, d));
     } else {
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 8>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split,
@@ -581,9 +603,12 @@ void wd_launch_rope_scatter(int dtype, const float* part, int n_split, size_t sp
                             void* kcache, void* vcache, int n_rows, int Hq, int Hkv, int dh, int S, int Sp,
                             cudaStream_t st) {
     if (n_rows <= 0) return;
-    dim3 grid(n_rows, wd_ceil_div(Hq + 2 * Hkv, 4));
-    WD_DISPATCH(dtype, launch_pdl(rope_scatter_kernel<T>, grid, dim3(256), 0, st, part, n_split, split_stride,
-                                  row_seq, row_pos, rope_tab, (T*)q, (T*)kcache, (T*)vcache, Hq, Hkv, dh, S, Sp));
+    const int qk_groups = wd_ceil_div(Hq + Hkv, 4);
+    const int n_qk = n_rows * qk_groups;
+    const int n_v = Hkv * wd_ceil_div(dh, 32) * wd_ceil_div(n_rows, 32);
+    WD_DISPATCH(dtype, launch_pdl(rope_scatter_kernel<T>, dim3(n_qk + n_v), dim3(256), 0, st, part, n_split,
+                                  split_stride, row_seq, row_pos, rope_tab, (T*)q, (T*)kcache, (T*)vcache, n_rows, Hq,
+                                  Hkv, dh, S, Sp, n_qk, qk_groups));
 }
 
 void wd_launch_attention_plain(int dtype, const void* q, const void* kcache, const void* vcache,
