@@ -1,0 +1,80 @@
+"""Parity at the benchmark configurations' full widths (GPU required).
+
+The five configurations are run with their real model width, head layout, FFN
+width, vocabulary, sequence lengths, window sizes and batch, but with ONE
+transformer block instead of 28/32: the fp64 oracle needs 5-110 TFLOP for a
+full-depth refresh step, and depth only repeats the same kernels with the same
+launch configuration.  Steps compared per config: the first refresh, the normal
+steps of the phase (transients appear), the next refresh; for batches the
+oracle follows a subset of the sequences (they are independent)."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2601_20332_b200 import binding as wd
+from paper_2601_20332_b200 import build as wd_build
+from paper_2601_20332_b200 import synth
+from wd_harness import Parity
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda:0"
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    wd_build.build()
+
+
+def run_cfg(cfg, n_steps, oracle_seqs=None, ids=None, decoded=None):
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg) if ids is None else ids
+    batch, S = ids.shape
+    p = Parity(cfg, w, ids, decoded, oracle_seqs=oracle_seqs, max_rows=batch * S, max_active=batch * cfg["A"])
+    logs = []
+    for _ in range(n_steps):
+        logs.append(p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"]))
+    p.check_state_mirror()
+    p.close()
+    del w
+    torch.cuda.empty_cache()
+    return logs
+
+
+def test_cfg2_llada8b_shape():
+    """LLaDA-8B width, prompt 256 + 256 masks, A=32 B=64 R=8 T=2, one token per step."""
+    cfg = synth.get_config("llada8b", L=1)
+    logs = run_cfg(cfg, 9)
+    assert [l["info"]["is_refresh"] for l in logs] == [1, 0, 0, 0, 0, 0, 0, 0, 1]
+    assert logs[0]["info"]["n_rows"] == 352 and logs[3]["info"]["n_rows"] == 34
+    assert sum(l["worst"]["ambiguous"] for l in logs) == 0
+
+
+def test_cfg3_llada8b_long_two_tokens_and_full_sequence_step():
+    """prompt 512 + 1024 masks, A=64 B=128, two tokens per step; then the no-pruning step."""
+    cfg = synth.get_config("llada8b_long", L=1)
+    logs = run_cfg(cfg, 3)
+    assert logs[0]["info"]["n_rows"] == 704 and logs[1]["info"]["n_rows"] == 64 + 2
+    assert all(l["res"]["n_unmasked"][0] == 2 for l in logs)
+    full = dict(cfg, A=cfg["G"], B=0, R=1, T=0)
+    logs = run_cfg(full, 1)
+    assert logs[0]["info"]["n_rows"] == 1536 and logs[0]["info"]["n_active"] == 1024
+
+
+def test_cfg4_dream7b_shape_gqa_batch8():
+    """Dream-7B width (28 query heads over 4 KV heads), batch 8 with independent windows."""
+    cfg = synth.get_config("dream7b", L=1)
+    logs = run_cfg(cfg, 5, oracle_seqs=[0, 5])
+    assert [l["info"]["is_refresh"] for l in logs] == [1, 0, 0, 0, 1]
+    assert logs[0]["info"]["n_rows"] == 8 * 672 and logs[3]["info"]["n_rows"] == 8 * 35
+    pos = logs[0]["res"]["positions"][:, 0]
+    assert len(set(pos.tolist())) > 1                     # the windows really are independent
+
+
+def test_cfg5_sweep_corner_late_state():
+    """Window sweep corner A=128 B=256 R=4, prompt 1024 + 2048 masks, batch 2, from a
+    half-decoded state (2048 visible positions)."""
+    cfg = synth.get_config("llada8b_sweep", L=1, A=128, B=256, R=4, batch=2)
+    ids, dec = synth.fast_forward(cfg, synth.make_prompts(cfg), 640)
+    logs = run_cfg(cfg, 3, oracle_seqs=[1], ids=ids, decoded=dec)
+    assert logs[0]["info"]["n_rows"] == 2 * (1024 + 640 + 384)
+    assert logs[1]["info"]["n_rows"] == 2 * 129 and logs[1]["info"]["n_vis"] == 2 * 2048
