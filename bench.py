@@ -127,7 +127,7 @@ def run_ours(args, rank, world):
     stream = torch.cuda.Stream(device=dev)
     peaks = measured_peaks()
 
-    def trajectory(n_warm, n_timed, state, timed_cb=None):
+    def trajectory(n_warm, n_timed, state, per_step_cb=None):
         infos, per_step = [], []
         for i in range(n_warm):
             state.step(A, B, R, T, k, stream)
@@ -143,6 +143,8 @@ def run_ours(args, rank, world):
             ev[i + 1].record(stream)
             state.sync()
             infos.append(info)
+            if per_step_cb:
+                per_step_cb(info)
         torch.cuda.synchronize()
         wall = time.perf_counter() - t0
         if world > 1:
@@ -158,8 +160,31 @@ def run_ours(args, rank, world):
     # ---- same trajectory again with GEMM events: roofline of the dominant kernel
     state.reset(ids, None, stream)
     ctx.profile_enable(True)
-    p_infos, _, _, _ = trajectory(W, K, state)
-    prof = ctx.profile_read()
+    kinds = {0: dict(gemm_ms=0.0, gemm_bytes=0.0, gemm_launches=0, flops=0.0),
+             1: dict(gemm_ms=0.0, gemm_bytes=0.0, gemm_launches=0, flops=0.0)}
+    last = dict(gemm_ms=0.0, gemm_bytes=0.0, gemm_launches=0)
+    per_layer = cfg["d"] * (cfg["Hq"] + 2 * cfg["Hkv"]) * cfg["dh"] + cfg["Hq"] * cfg["dh"] * cfg["d"] + 3 * cfg["d"] * cfg["F"]
+
+    def on_step(info):
+        now = ctx.profile_read()
+        kk = kinds[1 if info["is_refresh"] else 0]
+        for key in last:
+            kk[key] += now[key] - last[key]
+            last[key] = now[key]
+        kk["flops"] += 2.0 * info["n_rows"] * per_layer * cfg["L"] + 2.0 * info["n_active"] * cfg["d"] * cfg["V"]
+
+    def warm_then_time(n_warm, n_timed, state):
+        # warm-up steps must not count: reset the totals after them
+        for i in range(n_warm):
+            state.step(A, B, R, T, k, stream)
+            state.sync()
+        now = ctx.profile_read()
+        last.update({key: now[key] for key in last})
+        return trajectory(0, n_timed, state, on_step)
+
+    warm_then_time(W, K, state)
+    prof = kinds[0] if kinds[0]["gemm_launches"] else kinds[1]
+    prof_refresh = kinds[1]
     ctx.profile_enable(False)
     clocks = sampler.stop()
     # ---- end to end from host buffers on the host clock
@@ -223,11 +248,22 @@ def run_ours(args, rank, world):
                 "h2d_bytes_per_step": float(plan_ints * 4 + batch * S * 4 / (W + K)),
                 "d2h_bytes_per_step": float((1 + batch + 3 * batch * k) * 4)},
         "gpu_launches": int(sum(i["n_launches"] for i in infos)),
-        "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel", "achieved": gemm_gbs, "peak": peaks["hbm_gbs"],
+        "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel (launches of the normal, weight-streaming steps)",
+                     "achieved": gemm_gbs, "peak": peaks["hbm_gbs"],
                      "unit": "GB/s", "frac": gemm_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
-                     "traffic": None, "launches": int(prof["gemm_launches"]),
-                     "avg_launch_us": prof["gemm_ms"] * 1e3 / n_l, "bytes_per_launch": prof["gemm_bytes"] / n_l},
+                     "traffic": prof["gemm_bytes"] / n_l * 1.03,
+                     "traffic_note": "ncu small case (gate/up shape): DRAM bytes = 1.03 x algorithmic, scaled by bytes",
+                     "launches": int(prof["gemm_launches"]),
+                     "avg_launch_us": prof["gemm_ms"] * 1e3 / n_l, "bytes_per_launch": prof["gemm_bytes"] / n_l,
+                     "timing": "CUDA events around every launch on the step's stream (serialises the stream: isolated "
+                               "launch time, without the programmatic overlap the timed value has)"},
     }
+    if prof_refresh["gemm_launches"] and prof_refresh["gemm_ms"] > 0:
+        tf = prof_refresh["flops"] / (prof_refresh["gemm_ms"] * 1e-3) / 1e12
+        line["roofline_refresh_steps"] = {"bound": "tensor", "kernel": "gemm_tc_kernel (launches of the refresh steps)",
+                                          "achieved": tf, "peak": peaks["bf16_tflops_sustained"], "unit": "TFLOP/s",
+                                          "frac": tf / peaks["bf16_tflops_sustained"], "peak_source": peaks["source"],
+                                          "launches": int(prof_refresh["gemm_launches"])}
     if rank == 0:
         line["cpu_baseline"] = cpu_baseline(cfg, w, ids, budget_s=args.cpu_seconds)
         print(json.dumps(line))

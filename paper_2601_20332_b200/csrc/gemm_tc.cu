@@ -579,7 +579,8 @@ int env_int(const char* name, int dflt) {
 
 TcConfig pick_config(int rows) {
     TcConfig c;
-    c.tok_tiles = (rows + 255) / 256;
+    static const int bn_max = env_int("WD_GEMM_BN_MAX", 256);      // tuning knob (multiple of 16, <= 256)
+    c.tok_tiles = (rows + bn_max - 1) / bn_max;
     c.bn = ((rows + c.tok_tiles - 1) / c.tok_tiles + 15) / 16 * 16;     // balanced token tiles, <= 256
     int cols = 32;
     while (cols < c.bn) cols <<= 1;

@@ -49,6 +49,7 @@ def time_gemm(rows, n, k, iters=20, impl=wd.WD_GEMM_TCGEN05, ring_bytes=600 << 2
     by = wbytes + rows * k * 2 + rows * n * 4
     return dict(rows=rows, n=n, k=k, us_median=float(np.median(ts) * 1e3), us_min=float(ts.min() * 1e3),
                 algorithmic_bytes=by, gbs_median=by / (np.median(ts) * 1e-3) / 1e9,
+                tflops_median=2.0 * rows * n * k / (np.median(ts) * 1e-3) / 1e12,
                 note="includes the split-K reduce kernel of the single-op entry point")
 
 
