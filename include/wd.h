@@ -230,6 +230,13 @@ WD_API wd_status wd_state_destroy(wd_state* st);
 WD_API wd_status wd_state_read(const wd_state* st, int32_t seq, int32_t* token_ids, uint8_t* decoded,
                         int32_t* dec_step, int32_t* step_index, int32_t* steps_since_refresh);
 WD_API wd_status wd_debug_taps_set(wd_state* st, const wd_debug_taps* taps /*NULL = off*/);
+/* Adaptive termination (Section 4.2, "Adaptive termination"): once a step has unmasked the
+ * token `eos_id` at some position, undecoded positions after the first such position are never
+ * activated again (they stay far-field and are ignored) and a sequence is done when nothing
+ * undecoded is left before it.  An eos id that was part of the given tokens does not count.
+ * eos_id < 0 switches it off (the default; the paper's main results also run with a fixed
+ * length).  Kept across wd_state_reset.  Errors: WD_ERR_NULL, WD_ERR_PENDING, WD_ERR_BAD_PARAM. */
+WD_API wd_status wd_state_set_eos(wd_state* st, int32_t eos_id);
 
 /* ---- the step ----------------------------------------------------------- */
 
@@ -246,14 +253,16 @@ WD_API wd_status wd_plan(const wd_state* st, int32_t seq, int32_t A, int32_t B, 
 
 /* The same planner on explicit state arrays (no wd_state, no GPU, usable in a
  * process without a CUDA device): decoded[seq_len] 0/1 flags, dec_step[seq_len]
- * (step at which a token was unmasked, INT32_MIN if it was given), step_index
- * t, steps_since_refresh, and the external window stored at the last refresh
- * (ext_window[n_ext_window], ascending; empty before the first step).
+ * (step at which a token was unmasked, INT32_MIN if it was given), token_ids and
+ * eos_id for adaptive termination (see wd_state_set_eos; token_ids may be NULL
+ * when eos_id < 0), step_index t, steps_since_refresh, and the external window
+ * stored at the last refresh (ext_window[n_ext_window], ascending; empty before
+ * the first step).
  * Errors: as wd_plan, plus WD_ERR_BAD_PARAM for an index outside the sequence. */
-WD_API wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, int32_t seq_len,
-                      int32_t step_index, int32_t steps_since_refresh,
-                      const int32_t* ext_window, int32_t n_ext_window,
-                      int32_t A, int32_t B, int32_t R, int32_t T, wd_index_sets* out);
+WD_API wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, const int32_t* token_ids,
+                             int32_t eos_id, int32_t seq_len, int32_t step_index,
+                             int32_t steps_since_refresh, const int32_t* ext_window, int32_t n_ext_window,
+                             int32_t A, int32_t B, int32_t R, int32_t T, wd_index_sets* out);
 
 /* Enqueue one step for every sequence of the state on `stream` and return
  * without waiting.  k = tokens unmasked per sequence (at most the number of

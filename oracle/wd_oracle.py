@@ -58,6 +58,7 @@ class SeqState:
     since: int = 0                        # steps since the last refresh
     phase_start: int = 0
     wex: list = field(default_factory=list)   # external window of the current phase
+    eos_id: int = None                    # adaptive termination (Section 4.2), None = off
 
     def __post_init__(self):
         self.ids = np.array(self.ids, dtype=np.int64)
@@ -78,7 +79,19 @@ def oracle_plan(st: SeqState, A: int, B: int, R: int, T: int) -> dict:
     if A < 1 or B < 0 or R < 1 or T < 0:
         raise ValueError("bad window parameters")
     S = len(st.ids)
-    U = [i for i in range(S) if not st.decoded[i]]
+    # Adaptive termination (Section 4.2): once an end-of-sequence token has been generated the
+    # internal window stops advancing: undecoded positions after it are never activated again,
+    # they stay in the far field, and generation ends when nothing undecoded is left before it.
+    # (Reading: "generated" = unmasked by a step; an eos id inside the given prompt does not count,
+    # and the first generated eos in position order is the one that ends the text.)
+    limit = S
+    if st.eos_id is not None:
+        for i in range(S):
+            if st.decoded[i] and st.ids[i] == st.eos_id and st.dec_step[i] != NEVER:
+                limit = i
+                break
+    undecoded_all = [i for i in range(S) if not st.decoded[i]]
+    U = [i for i in undecoded_all if i < limit]
     if not U:
         return dict(done=True)
     Uset = set(U)
@@ -94,8 +107,8 @@ def oracle_plan(st: SeqState, A: int, B: int, R: int, T: int) -> dict:
     buf = W[len(act):]
     dp = [i for i in wex if i not in Uset]               # decoded within this phase
     trans = [i for i in dp if 1 <= st.t - int(st.dec_step[i]) <= T]
-    wexset = set(wex)
-    far = [i for i in U if i not in wexset]
+    live = set(W)
+    far = [i for i in undecoded_all if i not in live]
     dec = [i for i in range(S) if st.decoded[i]]
     vis = sorted(set(dec) | set(W))
     rows = list(vis) if refresh else sorted(set(act) | set(trans))

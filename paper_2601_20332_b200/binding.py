@@ -74,7 +74,9 @@ SIGNATURES = {
     "wd_state_read": (C.c_int, [vp, i32, i32p, u8p, i32p, i32p, i32p]),
     "wd_debug_taps_set": (C.c_int, [vp, C.POINTER(wd_debug_taps)]),
     "wd_plan": (C.c_int, [vp, i32, i32, i32, i32, i32, C.POINTER(wd_index_sets)]),
-    "wd_plan_raw": (C.c_int, [u8p, i32p, i32, i32, i32, i32p, i32, i32, i32, i32, i32, C.POINTER(wd_index_sets)]),
+    "wd_plan_raw": (C.c_int, [u8p, i32p, i32p, i32, i32, i32, i32, i32p, i32, i32, i32, i32, i32,
+                              C.POINTER(wd_index_sets)]),
+    "wd_state_set_eos": (C.c_int, [vp, i32]),
     "wd_step": (C.c_int, [vp, i32, i32, i32, i32, i32, vp, C.POINTER(wd_step_info)]),
     "wd_step_sync": (C.c_int, [vp, C.POINTER(wd_step_out)]),
     "wd_op_gemm": (C.c_int, [i32, i32, vp, vp, vp, i32, i32, i32, vp, C.c_size_t, vp]),
@@ -153,14 +155,17 @@ def _index_sets_dict(s, bufs) -> dict:
     return out
 
 
-def plan_raw(decoded, dec_step, t: int, since: int, ext_window, A: int, B: int, R: int, T: int) -> dict:
+def plan_raw(decoded, dec_step, t: int, since: int, ext_window, A: int, B: int, R: int, T: int,
+             token_ids=None, eos_id: int = -1) -> dict:
     """wd_plan_raw: the host planner on explicit state arrays (needs no GPU)."""
     dec = np.ascontiguousarray(decoded, dtype=np.uint8)
     ds = np.ascontiguousarray(dec_step, dtype=np.int32)
     wex = np.ascontiguousarray(ext_window, dtype=np.int32)
+    ids = None if token_ids is None else np.ascontiguousarray(token_ids, dtype=np.int32)
     s, bufs = _index_sets(len(dec))
-    check(lib().wd_plan_raw(dec.ctypes.data_as(u8p), _np_i32p(ds), len(dec), t, since,
-                            _np_i32p(wex) if len(wex) else None, len(wex), A, B, R, T, C.byref(s)), "wd_plan_raw")
+    check(lib().wd_plan_raw(dec.ctypes.data_as(u8p), _np_i32p(ds), None if ids is None else _np_i32p(ids), eos_id,
+                            len(dec), t, since, _np_i32p(wex) if len(wex) else None, len(wex), A, B, R, T,
+                            C.byref(s)), "wd_plan_raw")
     return _index_sets_dict(s, bufs)
 
 
@@ -251,6 +256,10 @@ class State:
         s, bufs = _index_sets(self.S)
         check(lib().wd_plan(self.handle, seq, A, B, R, T, C.byref(s)), "wd_plan")
         return _index_sets_dict(s, bufs)
+
+    def set_eos(self, eos_id: int):
+        """Adaptive termination: stop extending the window past a generated eos token (-1 = off)."""
+        check(lib().wd_state_set_eos(self.handle, eos_id), "wd_state_set_eos")
 
     def set_taps(self, layer_out=None, attn_out=None, logits=None):
         """Device float tensors that receive intermediates of later steps (None = off)."""

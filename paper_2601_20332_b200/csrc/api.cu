@@ -329,7 +329,7 @@ static void load_host_mirror(wd_state* st, const int32_t* ids, const uint8_t* de
             s.decoded[i] = decoded ? (decoded[(size_t)b * st->S + i] ? 1 : 0) : (s.ids[i] != mask_id ? 1 : 0);
         s.dec_step.assign(st->S, INT32_MIN);
         s.wex.clear();
-        s.t = 0; s.since = 0; s.phase_start = 0;
+        s.t = 0; s.since = 0; s.phase_start = 0;          // eos_id is kept across resets
     }
     memcpy(st->ids_host, ids, (size_t)st->batch * st->S * 4);
 }
@@ -422,6 +422,14 @@ extern "C" wd_status wd_state_read(const wd_state* st, int32_t seq, int32_t* tok
     return WD_OK;
 }
 
+extern "C" wd_status wd_state_set_eos(wd_state* st, int32_t eos_id) {
+    if (!st) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    if (eos_id >= st->ctx->d.vocab) return WD_ERR_BAD_PARAM;
+    for (WdSeq& s : st->seqs) s.eos_id = eos_id < 0 ? -1 : eos_id;
+    return WD_OK;
+}
+
 extern "C" wd_status wd_debug_taps_set(wd_state* st, const wd_debug_taps* taps) {
     if (!st) return WD_ERR_NULL;
     if (st->pending) return WD_ERR_PENDING;
@@ -456,13 +464,17 @@ extern "C" wd_status wd_plan(const wd_state* st, int32_t seq, int32_t A, int32_t
     return export_plan(p, out);
 }
 
-extern "C" wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, int32_t seq_len, int32_t step_index,
-                                 int32_t steps_since_refresh, const int32_t* ext_window, int32_t n_ext_window,
-                                 int32_t A, int32_t B, int32_t R, int32_t T, wd_index_sets* out) {
+extern "C" wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, const int32_t* token_ids,
+                                 int32_t eos_id, int32_t seq_len, int32_t step_index, int32_t steps_since_refresh,
+                                 const int32_t* ext_window, int32_t n_ext_window, int32_t A, int32_t B, int32_t R,
+                                 int32_t T, wd_index_sets* out) {
     if (!decoded || !dec_step || !out || (n_ext_window > 0 && !ext_window)) return WD_ERR_NULL;
+    if (eos_id >= 0 && !token_ids) return WD_ERR_NULL;
     if (seq_len < 1 || n_ext_window < 0 || step_index < 0 || steps_since_refresh < 0) return WD_ERR_BAD_PARAM;
     WdSeq s;
-    s.ids.assign(seq_len, 0);
+    if (token_ids) s.ids.assign(token_ids, token_ids + seq_len);
+    else s.ids.assign(seq_len, 0);
+    s.eos_id = eos_id < 0 ? -1 : eos_id;
     s.decoded.assign(decoded, decoded + seq_len);
     s.dec_step.assign(dec_step, dec_step + seq_len);
     for (int32_t i = 0; i < n_ext_window; ++i) {

@@ -7,7 +7,9 @@
 // buffer = external \ (active U decoded-in-phase); undecoded tokens outside
 // the external window are pruned.  Section 4.3: a phase is one refresh step
 // (everything visible is computed) followed by normal steps (active tokens and
-// recently decoded tokens are computed).
+// recently decoded tokens are computed).  Adaptive termination (Section 4.2): once an
+// end-of-sequence token has been generated, undecoded positions after it are never activated
+// again (they stay far-field) and the sequence is done when nothing undecoded precedes it.
 #include <algorithm>
 #include <climits>
 
@@ -20,20 +22,26 @@ wd_status wd_plan_seq(const WdSeq& s, int32_t A, int32_t B, int32_t R, int32_t T
     p = WdSeqPlan();
     const int32_t S = (int32_t)s.ids.size();
 
+    // first generated end-of-sequence token in position order (tokens that were given do not count)
+    int32_t limit = S;
+    if (s.eos_id >= 0)
+        for (int32_t i = 0; i < S; ++i)
+            if (s.decoded[i] && s.ids[i] == s.eos_id && s.dec_step[i] != INT32_MIN) { limit = i; break; }
+
     int32_t n_undecoded = 0;
-    for (int32_t i = 0; i < S; ++i) n_undecoded += s.decoded[i] ? 0 : 1;
+    for (int32_t i = 0; i < limit; ++i) n_undecoded += s.decoded[i] ? 0 : 1;
     if (n_undecoded == 0) { p.done = true; return WD_OK; }
 
-    // does the stored external window still hold an undecoded token?
+    // does the stored external window still hold an undecoded token (before the limit)?
     bool window_alive = false;
-    for (int32_t i : s.wex) if (!s.decoded[i]) { window_alive = true; break; }
+    for (int32_t i : s.wex) if (!s.decoded[i] && i < limit) { window_alive = true; break; }
     p.refresh = (s.t == 0) || (s.since >= R) || !window_alive;
 
     if (p.refresh) {
         // long arithmetic: A + B may exceed int32 for "window = everything" callers
         const int64_t want = std::min<int64_t>((int64_t)A + (int64_t)B, n_undecoded);
         p.wex.reserve((size_t)want);
-        for (int32_t i = 0; i < S && (int64_t)p.wex.size() < want; ++i)
+        for (int32_t i = 0; i < limit && (int64_t)p.wex.size() < want; ++i)
             if (!s.decoded[i]) p.wex.push_back(i);
     } else {
         p.wex = s.wex;
@@ -42,8 +50,11 @@ wd_status wd_plan_seq(const WdSeq& s, int32_t A, int32_t B, int32_t R, int32_t T
     // walk the external window once: undecoded members fill the internal
     // window first, the rest is buffer; decoded members were decoded in this
     // phase and are recomputed while young enough
+    std::vector<uint8_t> live((size_t)S, 0);            // undecoded window members still in play
     for (int32_t i : p.wex) {
         if (!s.decoded[i]) {
+            if (i >= limit) continue;                       // cut off by an end-of-sequence token
+            live[i] = 1;
             if ((int32_t)p.active.size() < A) p.active.push_back(i);
             else p.buffer.push_back(i);
         } else {
@@ -53,11 +64,9 @@ wd_status wd_plan_seq(const WdSeq& s, int32_t A, int32_t B, int32_t R, int32_t T
     }
 
     // one pass over the sequence for the position-ordered lists
-    std::vector<uint8_t> in_wex((size_t)S, 0);
-    for (int32_t i : p.wex) in_wex[i] = 1;
     for (int32_t i = 0; i < S; ++i) {
         if (s.decoded[i]) { p.decoded.push_back(i); p.vis.push_back(i); }
-        else if (in_wex[i]) p.vis.push_back(i);
+        else if (live[i]) p.vis.push_back(i);
         else p.far_field.push_back(i);
     }
     if (p.refresh) {

@@ -35,6 +35,7 @@ struct WdSeq {
     int32_t t = 0;                  // diffusion step index
     int32_t since = 0;              // steps since the last refresh
     int32_t phase_start = 0;
+    int32_t eos_id = -1;            // adaptive termination: id of the end-of-sequence token, -1 = off
 };
 
 struct WdSeqPlan {

@@ -134,6 +134,30 @@ def test_late_state_and_finish():
     assert logs[-1]["info"]["n_active"] == 1
 
 
+def test_adaptive_termination_on_gpu():
+    """Take the id the model generates at the third step as the end-of-sequence id: the rerun
+    must follow the oracle step by step and finish early (Section 4.2, adaptive termination)."""
+    cfg = synth.get_config("llada8b", **SMALL_BF16)
+    w = synth.make_weights(cfg, DEV, gain_jitter=0.1)
+    ids = synth.make_prompts(cfg)
+    p = Parity(cfg, w, ids)
+    toks = [p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], 1)["res"] for _ in range(3)]
+    p.close()
+    eos = int(toks[2]["token_ids"][0, 0])
+    first = next(i for i, t in enumerate(toks) if int(t["token_ids"][0, 0]) == eos)   # may already occur earlier
+    p = Parity(cfg, w, ids, eos_id=eos)
+    n = 0
+    while p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], 1) is not None:
+        n += 1
+        assert n <= cfg["G"]
+    p.check_state_mirror()
+    st = p.st.read(0)
+    p.close()
+    e = int(toks[first]["positions"][0, 0])
+    assert n < cfg["G"] and st["decoded"][: e + 1].all()
+    assert not st["decoded"][e + 1:].all()                   # the tail was never decoded
+
+
 @pytest.mark.parametrize("shape", [SMALL_BF16, DH128])
 def test_far_field_and_refresh_independence_on_gpu(shape):
     """Changing ids at far-field positions and poisoning the K/V cache before a refresh

@@ -48,18 +48,23 @@ def test_sizes_and_dims_validation():
     assert wd.lib().wd_create(None, None, None, 0, C.byref(out)) == wd.WD_ERR_NULL
 
 
-def _walk(seed, S, frac, A, B, R, T, k, prefix):
+def _walk(seed, S, frac, A, B, R, T, k, prefix, eos_id=None, eos_prob=0.0):
     rng = np.random.default_rng(seed)
     dec = (np.arange(S) < int(S * frac)) if prefix else (rng.random(S) < frac)
-    st = SeqState(ids=np.zeros(S, dtype=np.int64), decoded=dec)
+    ids0 = np.where(dec, 3, 0)
+    if eos_id is not None:
+        ids0[: max(1, S // 8)] = np.where(dec[: max(1, S // 8)], eos_id, 0)     # eos ids among the GIVEN tokens
+    st = SeqState(ids=ids0.astype(np.int64), decoded=dec, eos_id=eos_id)
     # mirror of the state kept by the test for the raw planner
     m_dec = dec.astype(np.uint8).copy()
+    m_ids = ids0.astype(np.int32).copy()
     m_step = np.full(S, INT32_MIN, np.int32)
     m_t, m_since, m_wex = 0, 0, []
     steps = 0
     while True:
         want = oracle_plan(st, A, B, R, T)
-        got = wd.plan_raw(m_dec, m_step, m_t, m_since, m_wex, A, B, R, T)
+        got = wd.plan_raw(m_dec, m_step, m_t, m_since, m_wex, A, B, R, T, token_ids=m_ids,
+                          eos_id=-1 if eos_id is None else eos_id)
         assert got["done"] == want["done"]
         if want["done"]:
             break
@@ -71,11 +76,13 @@ def _walk(seed, S, frac, A, B, R, T, k, prefix):
         assert got["vis_contiguous"] == (want["vis"] == list(range(len(want["vis"]))))
         n = min(k, len(want["active"]))
         pick = sorted(rng.choice(want["active"], size=n, replace=False).tolist())
-        oracle_commit(st, want, pick, [1] * n)
+        toks = [eos_id if (eos_id is not None and rng.random() < eos_prob) else 1 for _ in pick]
+        oracle_commit(st, want, pick, toks)
         if got["refresh"]:
             m_wex, m_since = got["ext_window"], 0
-        for p in pick:
+        for p, tk in zip(pick, toks):
             m_dec[p] = 1
+            m_ids[p] = tk
             m_step[p] = m_t
         m_t += 1
         m_since += 1
@@ -92,6 +99,16 @@ def test_host_planner_matches_oracle_bit_exact(case):
     assert _walk(*case) > 0
 
 
+@pytest.mark.parametrize("case", [
+    (10, 60, 0.3, 4, 6, 3, 1, 1, True), (11, 96, 0.3, 8, 16, 4, 2, 2, True), (12, 70, 0.4, 3, 5, 5, 9, 2, False),
+    (13, 200, 0.2, 16, 48, 8, 2, 1, True),
+])
+def test_host_planner_matches_oracle_with_adaptive_termination(case):
+    full = _walk(*case)
+    short = _walk(*case, eos_id=7, eos_prob=0.15)
+    assert 0 < short < full                       # an eos token ended generation early
+
+
 def test_plan_raw_errors():
     dec = np.zeros(8, np.uint8)
     ds = np.full(8, INT32_MIN, np.int32)
@@ -106,8 +123,8 @@ def test_plan_raw_errors():
     import ctypes as C
     s, bufs = wd._index_sets(8)
     s.capacity = 2
-    r = wd.lib().wd_plan_raw(dec.ctypes.data_as(wd.u8p), ds.ctypes.data_as(wd.i32p), 8, 0, 0, None, 0, 4, 2, 2, 1,
-                             C.byref(s))
+    r = wd.lib().wd_plan_raw(dec.ctypes.data_as(wd.u8p), ds.ctypes.data_as(wd.i32p), None, -1, 8, 0, 0, None, 0, 4, 2,
+                             2, 1, C.byref(s))
     assert r == wd.WD_ERR_CAPACITY
     # huge window parameters must not overflow
     p = wd.plan_raw(dec, ds, 0, 0, [], 2**31 - 1, 2**31 - 1, 1, 0)

@@ -169,3 +169,54 @@ def test_plan_is_pure_and_done():
     assert oracle_plan(done, 2, 2, 2, 1)["done"]
     with pytest.raises(ValueError):
         oracle_plan(st, 0, 2, 2, 1)
+
+
+def _run_with_eos(eos_picks, eos_id=42, P=3, G=30, A=4, B=4, R=3, T=1, prompt_has_eos=False):
+    """Decode the first active position every step; positions in eos_picks get the eos id."""
+    ids = np.array(([eos_id] if prompt_has_eos else [1]) + [1] * (P - 1) + [99] * G)
+    st = SeqState(ids=ids, decoded=np.arange(P + G) < P, eos_id=eos_id)
+    plans = []
+    while True:
+        pl = oracle_plan(st, A, B, R, T)
+        if pl["done"]:
+            break
+        plans.append(pl)
+        pos = pl["active"][0]
+        oracle_commit(st, pl, [pos], [eos_id if pos in eos_picks else 5])
+    return st, plans
+
+
+def test_adaptive_termination_stops_the_window():
+    """Section 4.2, adaptive termination: after an eos token is generated the internal window
+    stops advancing, later positions stay far-field, and generation ends early."""
+    st, plans = _run_with_eos({12})
+    # positions 3..12 are decoded one by one, then everything after 12 is ignored for good
+    assert len(plans) == 10
+    assert st.decoded[:13].all() and not st.decoded[13:].any()
+    for pl in plans:
+        assert max(pl["active"] + pl["buffer"]) <= 12 + 8          # window never ran ahead of A + B
+    # once the eos is in, a sequence with undecoded tokens only after it is done
+    assert oracle_plan(st, 4, 4, 3, 1)["done"]
+    # without an eos the same schedule runs through all 30 masks
+    st2, plans2 = _run_with_eos(set())
+    assert len(plans2) == 30 and st2.decoded.all()
+    # and the plans before the eos appears are identical
+    for a, b in zip(plans[:9], plans2[:9]):
+        assert a == b
+
+
+def test_adaptive_termination_ignores_given_eos_and_takes_the_first_in_position_order():
+    st, plans = _run_with_eos(set(), prompt_has_eos=True)
+    assert len(plans) == 30                                   # an eos id inside the prompt does not count
+    # out-of-order decoding: eos generated at 20 first, then another at 10 moves the limit left
+    ids = np.array([1] * 2 + [99] * 30)
+    st = SeqState(ids=ids, decoded=np.arange(32) < 2, eos_id=42)
+    pl = oracle_plan(st, 24, 0, 1, 0)
+    oracle_commit(st, pl, [20], [42])
+    pl = oracle_plan(st, 24, 0, 1, 0)
+    assert max(pl["active"]) == 19 and set(range(21, 32)) <= set(pl["far_field"])
+    oracle_commit(st, pl, [10], [42])
+    pl = oracle_plan(st, 24, 0, 1, 0)
+    assert pl["active"] == list(range(2, 10))
+    assert set(pl["far_field"]) == set(range(11, 20)) | set(range(21, 32))
+    assert 20 in pl["vis"] and 10 in pl["vis"]                 # decoded tokens stay visible context
