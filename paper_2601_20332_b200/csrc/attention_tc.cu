@@ -280,10 +280,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 if (hf == 0)
                     *reinterpret_cast<float2*>(p.part_ml + ((slot + blockIdx.z) * kTile + r) * 2) = make_float2(m, l);
             }
-            __threadfence();
+            // one fence after the barrier publishes every thread's part (fences are cumulative)
             asm volatile("bar.sync 1, 256;" ::: "memory");
             int* last_flag = (int*)(tmem_slot + 2);
             if (threadIdx.x == 64) {
+                __threadfence();
                 const int old = atomicAdd(p.counters + tile * p.Hq + h, 1);
                 const int last = old + 1 == n_parts ? 1 : 0;
                 if (last) p.counters[tile * p.Hq + h] = 0;
@@ -381,8 +382,11 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     if (n_tiles <= 0) return WD_OK;
     EncodeTiledFn enc = get_encode();
     if (!enc) return WD_ERR_CUDA;
-    CUtensorMap mq;
-    {
+    // the query descriptor depends only on (buffer, rows, heads): the same for every layer of a step
+    static CUtensorMap mq;
+    static const void* mq_ptr = nullptr;
+    static int mq_rows = -1, mq_hq = -1;
+    if (mq_ptr != q || mq_rows != n_rows || mq_hq != Hq) {
         cuuint64_t dims[2] = {(cuuint64_t)Hq * dh, (cuuint64_t)n_rows};
         cuuint64_t strides[1] = {(cuuint64_t)Hq * dh * 2};
         cuuint32_t box[2] = {64, 128}, estr[2] = {1, 1};
@@ -390,6 +394,7 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return WD_ERR_CUDA;
+        mq_ptr = q; mq_rows = n_rows; mq_hq = Hq;
     }
     AttnParams p;
     memset(&p, 0, sizeof(p));
@@ -411,7 +416,11 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     p.part_ml = scratch ? scratch + (size_t)WD_ATTN_SPLIT_SLOTS * kTile * kTile : nullptr;
     p.counters = counters;
     const size_t smem = 6 * (size_t)kOperand + 8 * 8 + 16 + 2 * kTile * 4 + 1024;
-    WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    static bool attr_done = false;      // one device per process
+    if (!attr_done) {
+        WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_done = true;
+    }
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(n_tiles, Hq, p.max_parts);
     lc.blockDim = dim3(kThreads);

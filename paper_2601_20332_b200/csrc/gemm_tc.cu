@@ -32,10 +32,13 @@ using namespace wdk;
 constexpr int kBM = 128;            // weight rows per tile (MMA M)
 constexpr int kBK = 64;             // K elements per stage = one 128-byte swizzle row
 constexpr int kStageA = kBM * kBK * 2;
-constexpr int kThreads = 192;
+constexpr int kThreads = 192;         // TMA warp, MMA warp, 4 epilogue warps
+constexpr int kThreadsWide = 320;     // ... 8 epilogue warps when a CTA carries two weight halves
 
 struct TcParams {
     int rows, bn, kb_total, tok_tiles, n_units, n_stages, buf_cols, n_slices, aligned;
+    int wide;                       // 1: a tile is 256 weight rows = two MMA halves sharing each activation box
+    int tile_rows;                  // 128, or 256 when wide
     int nseg, ncol;
     int seg_tile0[4];               // first tile index of each weight matrix (+ end)
     int seg_n[3];
@@ -57,7 +60,7 @@ __device__ __forceinline__ UnitInfo decode_unit(const TcParams& p, int unit) {
     u.seg = 0;
     if (p.nseg > 1 && tile >= p.seg_tile0[1]) u.seg = 1;
     if (p.nseg > 2 && tile >= p.seg_tile0[2]) u.seg = 2;
-    u.n0 = (tile - p.seg_tile0[u.seg]) * kBM;
+    u.n0 = (tile - p.seg_tile0[u.seg]) * p.tile_rows;
     return u;
 }
 
@@ -292,7 +295,8 @@ __device__ void finalize_unit(const TcParams& p, long long G, int unit, int e) {
 // epilogue of one piece overlaps the MMAs of the next (two accumulators in TMEM).  A tile cut
 // by piece boundaries gets one partial sum per CTA that touched it, written to slice
 // (CTA - first CTA of the tile); the CTA that finishes the tile zero-fills the unused slices.
-__global__ void __launch_bounds__(kThreads)
+template <bool kWide>
+__global__ void __launch_bounds__(kWide ? kThreadsWide : kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w0,
                const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2,
                const TcParams p) {
@@ -300,7 +304,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     // 1024-byte alignment: required by the 128-byte swizzle atoms
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int NS = p.n_stages;
-    const int stage_bytes = kStageA + p.bn * kBK * 2;
+    const int stage_a = p.tile_rows * kBK * 2;            // 16 KB, or 32 KB when wide
+    const int stage_bytes = stage_a + p.bn * kBK * 2;
     uint64_t* bars = (uint64_t*)(smem + (size_t)NS * stage_bytes);
     // bars[0..NS) full | [NS..2NS) empty | [2NS, 2NS+1] accumulator full | [2NS+2, 2NS+3] accumulator empty
     uint32_t* tmem_slot = (uint32_t*)(bars + 2 * NS + 4);
@@ -329,8 +334,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         mbar_init(smem_u32(&bars[2 * NS]), 1);
         mbar_init(smem_u32(&bars[2 * NS + 1]), 1);
-        mbar_init(smem_u32(&bars[2 * NS + 2]), 128);
-        mbar_init(smem_u32(&bars[2 * NS + 3]), 128);
+        mbar_init(smem_u32(&bars[2 * NS + 2]), kWide ? 256 : 128);
+        mbar_init(smem_u32(&bars[2 * NS + 3]), kWide ? 256 : 128);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
@@ -379,11 +384,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 mbar_expect_tx(smem_u32(&bars[i]), (uint32_t)stage_bytes);
                 tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes), w.mw, smem_u32(&bars[i]), w.kb * kBK, w.n0,
                                  pol_stream);
+                if (kWide)
+                    tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes) + kStageA, w.mw, smem_u32(&bars[i]),
+                                     w.kb * kBK, w.n0 + kBM, pol_stream);
             }
             pdl_wait();
             Walk wx = w0;
             for (int i = 0; i < n_pre; ++i, advance(wx))
-                tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + kStageA, &map_x, smem_u32(&bars[i]), wx.kb * kBK,
+                tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + stage_a, &map_x, smem_u32(&bars[i]), wx.kb * kBK,
                             wx.tok0);
             int s = n_pre % NS;
             uint32_t ph = (uint32_t)(n_pre / NS) & 1u;
@@ -397,7 +405,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
                 mbar_expect_tx(full, (uint32_t)stage_bytes);
                 tma_load_2d_hint(sa, w.mw, full, w.kb * kBK, w.n0, pol_stream);
-                tma_load_2d(sa + kStageA, &map_x, full, w.kb * kBK, w.tok0);
+                if (kWide) tma_load_2d_hint(sa + kStageA, w.mw, full, w.kb * kBK, w.n0 + kBM, pol_stream);
+                tma_load_2d(sa + stage_a, &map_x, full, w.kb * kBK, w.tok0);
                 if (++s == NS) { s = 0; ph ^= 1u; }
             }
         }
@@ -412,9 +421,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 long long g;
                 int len;
                 sch.piece(piece, g, len);
-                const int buf = piece & 1;
+                // normal: two accumulators used alternately; wide: one accumulator pair (both weight halves)
+                const int buf = kWide ? 0 : (piece & 1);
+                const uint32_t par = kWide ? ((uint32_t)piece & 1u) : ((uint32_t)(piece >> 1) & 1u);
                 // the epilogue has drained this accumulator (free at the start)
-                if (!(ok = mbar_wait(smem_u32(&bars[2 * NS + 2 + buf]), ((uint32_t)(piece >> 1) & 1u) ^ 1u, abort_flag))) break;
+                if (!(ok = mbar_wait(smem_u32(&bars[2 * NS + 2 + buf]), par ^ 1u, abort_flag))) break;
                 tc_fence_after();
                 const uint32_t acc = tmem_base + (uint32_t)(buf * p.buf_cols);
                 for (int j = 0; j < len; ++j) {
@@ -422,12 +433,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     tc_fence_after();
                     const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
                     const uint64_t adesc = make_sdesc(sa);
-                    const uint64_t bdesc = make_sdesc(sa + kStageA);
+                    const uint64_t bdesc = make_sdesc(sa + stage_a);
+                    const uint64_t adesc1 = make_sdesc(sa + kStageA);   // second weight half (wide)
 #pragma unroll
                     for (int kk = 0; kk < kBK / 16; ++kk) {
                         // 16 bf16 = 32 bytes further along K inside the swizzle row: +2 in 16-byte units
                         umma_bf16(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
                                   (j > 0 || kk > 0) ? 1u : 0u);
+                        if (kWide)
+                            umma_bf16(acc + (uint32_t)p.buf_cols, adesc1 + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk),
+                                      p.idesc, (j > 0 || kk > 0) ? 1u : 0u);
                     }
                     umma_commit(smem_u32(&bars[NS + s]));          // stage free once these MMAs have read it
                     if (++s == NS) { s = 0; ph ^= 1u; }
@@ -441,9 +456,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         __syncwarp();
     } else {
-        // ---------------------------------------------------- epilogue (warps 2..5)
+        // ---------------------------------------------------- epilogue (warps 2..5; wide: 2..9)
         const int quarter = warp & 3;                  // TMEM lanes 32*quarter .. +31
-        const int n_local = quarter * 32 + lane;
+        const int half_sel = (warp - 2) >> 2;          // wide: which weight half this warp drains
+        const int n_local = half_sel * kBM + quarter * 32 + lane;
         pdl_wait();      // the previous reader of y has finished (already implied by the data flow)
         bool ok = true;
         for (int piece = 0; piece < sch.n_pieces; ++piece) {
@@ -452,17 +468,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             sch.piece(piece, g, len);
             const int unit = (int)(g / p.kb_total), kb0 = (int)(g - (long long)unit * p.kb_total);
             const UnitInfo u = decode_unit(p, unit);
-            const int buf = piece & 1;
+            const int buf = kWide ? 0 : (piece & 1);
+            const uint32_t par = kWide ? ((uint32_t)piece & 1u) : ((uint32_t)(piece >> 1) & 1u);
             const int n = u.n0 + n_local;
             const bool n_ok = n < p.seg_n[u.seg];
             int ord = 0;
             if (!p.aligned) ord = (int)(c - (((long long)unit * p.kb_total + 1) * G - 1) / p.W);
-            ok = ok && mbar_wait(smem_u32(&bars[2 * NS + buf]), (uint32_t)(piece >> 1) & 1u, abort_flag);
+            ok = ok && mbar_wait(smem_u32(&bars[2 * NS + buf]), par, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             float* yb = p.y + p.seg_col[u.seg] + n;
-            const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.buf_cols);
+            const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf + half_sel) * p.buf_cols);
             for (int cc = 0; cc < p.bn; cc += 16) {
                 if (u.tok0 + cc >= p.rows) break;
                 uint32_t v[16];
@@ -570,24 +587,29 @@ wd_status encode_2d(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_
     return r == CUDA_SUCCESS ? WD_OK : WD_ERR_CUDA;
 }
 
-struct TcConfig { int bn, tok_tiles, n_stages, buf_cols, ctas_per_sm; size_t smem; };
+struct TcConfig { int bn, tok_tiles, n_stages, buf_cols, ctas_per_sm, wide, tile_rows; size_t smem; };
 
 int env_int(const char* name, int dflt) {
     const char* v = getenv(name);
     return v && *v ? atoi(v) : dflt;
 }
 
-TcConfig pick_config(int rows) {
+TcConfig pick_config(int rows, bool allow_wide) {
     TcConfig c;
+    // Many tokens: the GEMM is bound by operand traffic from L2 into shared memory, so a CTA
+    // carries two 128-row weight halves that share every activation box ([256 x BN] per CTA).
+    static const int wide_from = env_int("WD_GEMM_WIDE_FROM", 512);
+    c.wide = (allow_wide && rows >= wide_from) ? 1 : 0;
+    c.tile_rows = c.wide ? 2 * kBM : kBM;
     static const int bn_max = env_int("WD_GEMM_BN_MAX", 256);      // tuning knob (multiple of 16, <= 256)
     c.tok_tiles = (rows + bn_max - 1) / bn_max;
     c.bn = ((rows + c.tok_tiles - 1) / c.tok_tiles + 15) / 16 * 16;     // balanced token tiles, <= 256
     int cols = 32;
     while (cols < c.bn) cols <<= 1;
     c.buf_cols = cols;                                                   // two accumulators: 2 * cols <= 512
-    const int stage = kStageA + c.bn * kBK * 2;
+    const int stage = c.tile_rows * kBK * 2 + c.bn * kBK * 2;
     static const int want2 = env_int("WD_GEMM_CTAS_PER_SM", 1);
-    c.ctas_per_sm = (want2 == 2 && c.bn <= 64) ? 2 : 1;
+    c.ctas_per_sm = (want2 == 2 && c.bn <= 64 && !c.wide) ? 2 : 1;
     c.n_stages = ((c.ctas_per_sm == 2 ? 100 : 196) * 1024) / stage;
     if (c.n_stages > 10) c.n_stages = 10;
     if (c.n_stages < 2) c.n_stages = 2;
@@ -652,14 +674,22 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     if (rows < 1 || K < 8 || K % 8) return WD_ERR_BAD_PARAM;
     TcParams p;
     memset(&p, 0, sizeof(p));
-    const TcConfig cfg = pick_config(rows);
+    const bool fused = fuse && fuse->mode != WD_FUSE_NONE;
+    // The wide tile halves the operand traffic per flop but has a shallower ring and an epilogue
+    // that does not overlap the next tile: it pays once every CTA gets at least one whole tile.
+    long long wide_units = 0;
+    for (int i = 0; i < nseg; ++i) wide_units += (segs[i].n + 2 * kBM - 1) / (2 * kBM);
+    wide_units *= (rows + 255) / 256;
+    const TcConfig cfg = pick_config(rows, !fused && wide_units >= sm_count);
+    p.wide = cfg.wide;
+    p.tile_rows = cfg.tile_rows;
     int tiles = 0, col = 0;
     for (int i = 0; i < nseg; ++i) {
         if (!segs[i].map) return WD_ERR_NULL;
         p.seg_tile0[i] = tiles;
         p.seg_n[i] = segs[i].n;
         p.seg_col[i] = col;
-        tiles += (segs[i].n + kBM - 1) / kBM;
+        tiles += (segs[i].n + cfg.tile_rows - 1) / cfg.tile_rows;
         col += segs[i].n;
     }
     p.seg_tile0[nseg] = tiles;
@@ -698,17 +728,28 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     }
 
     CUtensorMap mx;
-    wd_status s = encode_2d(&mx, x->ptr, rows, K, cfg.bn);
-    if (s != WD_OK) return s;
-
-    WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+    bool hit = false;
+    for (const WdTcX::Entry& e : x->cache)
+        if (e.rows == rows && e.bn == cfg.bn) { mx = e.map; hit = true; break; }
+    if (!hit) {
+        wd_status s = encode_2d(&mx, x->ptr, rows, K, cfg.bn);
+        if (s != WD_OK) return s;
+        if (x->cache.size() >= 16) x->cache.erase(x->cache.begin());
+        x->cache.push_back({rows, cfg.bn, mx});
+    }
+    static bool attr_done = false;      // one device per process
+    if (!attr_done) {
+        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        attr_done = true;
+    }
     const CUtensorMap& m0 = *segs[0].map;
     const CUtensorMap& m1 = *segs[nseg > 1 ? 1 : 0].map;
     const CUtensorMap& m2 = *segs[nseg > 2 ? 2 : 0].map;
     ++wd_launch_counter;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3((unsigned)G);
-    lc.blockDim = dim3(kThreads);
+    lc.blockDim = dim3(cfg.wide ? kThreadsWide : kThreads);
     lc.dynamicSmemBytes = cfg.smem;
     lc.stream = stream;
     cudaLaunchAttribute attr[1];
@@ -716,7 +757,8 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = wd_pdl_enabled ? 1 : 0;
-    WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel, mx, m0, m1, m2, p));
+    if (cfg.wide) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<true>, mx, m0, m1, m2, p));
+    else WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<false>, mx, m0, m1, m2, p));
     if (n_split_out) *n_split_out = p.n_slices;
     return WD_OK;
 }

@@ -21,6 +21,10 @@ struct WdTcSeg {
 struct WdTcX {
     const void* ptr = nullptr;
     int K = 0;
+    // descriptors already encoded for this operand, keyed by (rows, token tile): the same few
+    // shapes come back every step
+    struct Entry { int rows, bn; CUtensorMap map; };
+    mutable std::vector<Entry> cache;
 };
 
 struct WdTcWeights {

@@ -492,7 +492,8 @@ __global__ void rowstats_kernel(const float* __restrict__ logits, int V, int chu
     }
 }
 
-// One block per sequence.  Merge the chunk statistics of every active row, then
+// One block per sequence.  A warp merges the chunk statistics of one active row at a time (lanes
+// over chunks, then a fixed shuffle tree, so identical rows give identical bits); then
 // rank(i) = #{j : s_j < s_i or (s_j == s_i and pos_j < pos_i)}; positions are ascending inside a
 // sequence, so "pos_j < pos_i" is "j < i".
 __global__ void select_kernel(const float* __restrict__ ch_max, const int32_t* __restrict__ ch_idx,
@@ -509,17 +510,31 @@ __global__ void select_kernel(const float* __restrict__ ch_max, const int32_t* _
     const int n = act_off ? act_off[b + 1] - a0 : n_single;
     const int kk = min(k, n);
     if (threadIdx.x == 0) n_sel[b] = kk;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    for (int i = w; i < n; i += nw) {
         const size_t base = (size_t)(a0 + i) * n_chunks;
-        float m = ch_max[base];
-        int tok = ch_idx[base];
-        for (int c = 1; c < n_chunks; ++c)
-            if (ch_max[base + c] > m) { m = ch_max[base + c]; tok = ch_idx[base + c]; }   // chunks ascend in index
+        // row maximum and its lowest index: chunks ascend in index, so on equal maxima the lower chunk wins
+        float m = -INFINITY;
+        int tok = 0x7fffffff;
+        for (int c = lane; c < n_chunks; c += 32) {
+            const float cm = ch_max[base + c];
+            const int ci = ch_idx[base + c];
+            if (cm > m || (cm == m && ci < tok)) { m = cm; tok = ci; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, m, o);
+            const int oi = __shfl_xor_sync(0xffffffffu, tok, o);
+            if (om > m || (om == m && oi < tok)) { m = om; tok = oi; }
+        }
         double s = 0.0;
-        for (int c = 0; c < n_chunks; ++c) s += ch_sum[base + c] * exp((double)ch_max[base + c] - (double)m);
-        row_token[a0 + i] = tok;
-        row_sumexp[a0 + i] = s;
-        if (row_conf) row_conf[a0 + i] = (float)(1.0 / s);
+        for (int c = lane; c < n_chunks; c += 32) s += ch_sum[base + c] * exp((double)ch_max[base + c] - (double)m);
+        s = warp_sum_d(s);
+        if (lane == 0) {
+            row_token[a0 + i] = tok;
+            row_sumexp[a0 + i] = s;
+            if (row_conf) row_conf[a0 + i] = (float)(1.0 / s);
+        }
     }
     __syncthreads();
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
