@@ -9,7 +9,9 @@
 // One CTA per (128-row query tile of one sequence, query head):
 //   warp 0    TMA: the Q tile once, then [128 keys x 128] K boxes and [128 x 128 keys] boxes of
 //             the transposed V cache into a two-stage ring
-//   warp 1    tcgen05.mma: S = Q K^T into TMEM, then O_tile = P V into TMEM
+//   warp 1    tcgen05.mma: S = Q K^T into TMEM, then O_tile = P V into TMEM; software-pipelined:
+//             S and O_tile are double-buffered, Q K^T of the next key tile is issued before P V
+//             of the current one, so the tensor core works while the softmax threads are busy
 //   warps 2-9 two threads per query row (each takes 64 of the tile's 128 columns): tcgen05.ld of
 //             its half of the S row, online softmax in fp32 (exp2 with the scale folded in; the
 //             two halves exchange their row maxima through shared memory), P as bf16 into shared
@@ -35,7 +37,8 @@ constexpr int kTile = 128;                 // query rows per CTA = keys per step
 constexpr int kAtom = kTile * 64 * 2;      // one [128 x 64] bf16 swizzle-atom column: 16 KB
 constexpr int kOperand = 2 * kAtom;        // a [128 x 128] bf16 operand: 32 KB
 constexpr int kThreads = 320;            // TMA warp, MMA warp, 8 softmax warps
-constexpr int kTmemCols = 256;             // S: columns 0..127, O_tile: columns 128..255
+constexpr int kTmemCols = 512;             // S0, S1: columns 0..255; O_tile0, O_tile1: columns 256..511
+constexpr int kBars = 15;
 
 struct AttnParams {
     const int32_t* qtile_seq;    // [n_tiles] sequence of the tile
@@ -71,8 +74,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     uint8_t* sP = smem + kOperand;               // 32 KB
     uint8_t* sKV = smem + 2 * kOperand;          // 2 stages x (K 32 KB + V^T 32 KB)
     uint64_t* bars = (uint64_t*)(smem + 2 * kOperand + 4 * kOperand);
-    // 0 q_full | 1,2 kv_full | 3,4 kv_empty | 5 s_full | 6 p_full | 7 o_full
-    uint32_t* tmem_slot = (uint32_t*)(bars + 8);
+    // 0 q_full | 1,2 kv_full | 3,4 kv_empty | 5,6 s_full | 7,8 s_empty | 9 p_full | 10 p_empty |
+    // 11,12 o_full | 13,14 o_empty.  "empty" barriers that the softmax threads signal count 256.
+    uint32_t* tmem_slot = (uint32_t*)(bars + kBars + 1);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -89,7 +93,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     if (kt_begin >= n_kt_all) return;                       // nothing for this CTA (uniform exit)
     const int n_kt = min(p.tiles_per_split, n_kt_all - kt_begin);
     if (threadIdx.x == 0) {
-        for (int i = 0; i < 8; ++i) mbar_init(smem_u32(&bars[i]), i == 6 ? 256u : 1u);
+        for (int i = 0; i < kBars; ++i)
+            mbar_init(smem_u32(&bars[i]), (i == 7 || i == 8 || i == 9 || i == 13 || i == 14) ? 256u : 1u);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -129,33 +134,46 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------------------------------------------- MMA issuer
+            // tile i uses K/V stage i&1, S buffer i&1, O_tile buffer i&1; every barrier that is
+            // completed once per two tiles has parity (i>>1)&1 for tile i
             bool ok = mbar_wait(smem_u32(&bars[0]), 0, abort_flag);
             const uint64_t qd0 = make_sdesc(smem_u32(sQ)), qd1 = make_sdesc(smem_u32(sQ) + kAtom);
             const uint64_t pd0 = make_sdesc(smem_u32(sP)), pd1 = make_sdesc(smem_u32(sP) + kAtom);
+            auto issue_qk = [&](int j) -> bool {           // S[j&1] = Q K(j)^T
+                const int s = j & 1;
+                const uint32_t ph = (uint32_t)(j >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&bars[1 + s]), ph, abort_flag)) return false;        // K(j), V(j) landed
+                if (!mbar_wait(smem_u32(&bars[7 + s]), ph ^ 1u, abort_flag)) return false;   // S(j-2) has been read
+                tc_fence_after();
+                const uint32_t sk = smem_u32(sKV + (size_t)s * 2 * kOperand);
+                const uint64_t kd0 = make_sdesc(sk), kd1 = make_sdesc(sk + kAtom);
+                const uint32_t acc = tmem_base + (uint32_t)(s * kTile);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, qd0 + 2 * kk, kd0 + 2 * kk, p.idesc, kk > 0);
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, qd1 + 2 * kk, kd1 + 2 * kk, p.idesc, 1u);
+                umma_commit(smem_u32(&bars[5 + s]));
+                return true;
+            };
+            ok = ok && issue_qk(0);
             for (int i = 0; i < n_kt && ok; ++i) {
                 const int s = i & 1;
                 const uint32_t ph = (uint32_t)(i >> 1) & 1u;
-                if (!(ok = mbar_wait(smem_u32(&bars[1 + s]), ph, abort_flag))) break;
+                if (i + 1 < n_kt && !(ok = issue_qk(i + 1))) break;                           // runs ahead of the softmax
+                if (!(ok = mbar_wait(smem_u32(&bars[9]), (uint32_t)i & 1u, abort_flag))) break;      // P(i) written
+                if (!(ok = mbar_wait(smem_u32(&bars[13 + s]), ph ^ 1u, abort_flag))) break;         // O_tile(i-2) folded
                 tc_fence_after();
-                const uint32_t sk = smem_u32(sKV + (size_t)s * 2 * kOperand), sv = sk + kOperand;
-                const uint64_t kd0 = make_sdesc(sk), kd1 = make_sdesc(sk + kAtom);
-                // S = Q K^T: reduction over head_dim, 8 steps of 16
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) umma_bf16(tmem_base, qd0 + 2 * kk, kd0 + 2 * kk, p.idesc, kk > 0);
-#pragma unroll
-                for (int kk = 0; kk < 4; ++kk) umma_bf16(tmem_base, qd1 + 2 * kk, kd1 + 2 * kk, p.idesc, 1u);
-                umma_commit(smem_u32(&bars[5]));
-                // wait for P (which also means S and the previous O_tile have been read)
-                if (!(ok = mbar_wait(smem_u32(&bars[6]), (uint32_t)i & 1u, abort_flag))) break;
-                tc_fence_after();
+                const uint32_t sv = smem_u32(sKV + (size_t)s * 2 * kOperand) + kOperand;
                 const uint64_t vd0 = make_sdesc(sv), vd1 = make_sdesc(sv + kAtom);
+                const uint32_t acc = tmem_base + (uint32_t)(2 * kTile + s * kTile);
                 // O_tile = P V: reduction over the 128 keys of the tile
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) umma_bf16(tmem_base + kTile, pd0 + 2 * kk, vd0 + 2 * kk, p.idesc, kk > 0);
+                for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, pd0 + 2 * kk, vd0 + 2 * kk, p.idesc, kk > 0);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) umma_bf16(tmem_base + kTile, pd1 + 2 * kk, vd1 + 2 * kk, p.idesc, 1u);
+                for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, pd1 + 2 * kk, vd1 + 2 * kk, p.idesc, 1u);
                 umma_commit(smem_u32(&bars[3 + s]));       // K/V stage free
-                umma_commit(smem_u32(&bars[7]));           // O_tile ready
+                umma_commit(smem_u32(&bars[10]));          // P buffer free
+                umma_commit(smem_u32(&bars[11 + s]));      // O_tile(i) ready
             }
             if (!ok) {
                 *abort_flag = 1;
@@ -174,14 +192,30 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         float o[64];
 #pragma unroll
         for (int c = 0; c < 64; ++c) o[c] = 0.f;
-        float m = -INFINITY, l = 0.f;
+        float m = -INFINITY, l = 0.f, alpha_prev = 0.f;
         bool ok = true;
+        // o += O_tile(j) with tile j's rescale factor; done one tile late so that P V(j) has had
+        // time to finish while this thread was busy with the next tile's softmax
+        auto fold = [&](int j, float alpha) {
+            const int s = j & 1;
+            if (!mbar_wait(smem_u32(&bars[11 + s]), (uint32_t)(j >> 1) & 1u, abort_flag)) { *abort_flag = 1; ok = false; }
+            tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < 64; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld32(t_row + (uint32_t)(2 * kTile + s * kTile + c_off + c0), v);
+#pragma unroll
+                for (int c = 0; c < 32; ++c) o[c0 + c] = o[c0 + c] * alpha + __uint_as_float(v[c]);
+            }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars[13 + s]));          // O_tile buffer may be overwritten
+        };
         for (int i = 0; i < n_kt; ++i) {
             const int s = i & 1;
             // A failed wait must not leave the loop before the named barrier below (the other
             // warps would wait there for ever): it raises the CTA's abort flag, every thread still
             // reaches the barrier, and all of them leave together right after it.
-            if (!mbar_wait(smem_u32(&bars[5]), (uint32_t)i & 1u, abort_flag)) *abort_flag = 1;
+            if (!mbar_wait(smem_u32(&bars[5 + s]), (uint32_t)(i >> 1) & 1u, abort_flag)) *abort_flag = 1;
             tc_fence_after();
             const int n_keys = min(kTile, n_vis - (kt_begin + i) * kTile);   // valid keys in this tile
             // keys past n_vis may hold anything: zero their V columns so that 0 * garbage stays 0.
@@ -197,13 +231,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
             for (int c0 = 0; c0 < 64; c0 += 32) {
                 uint32_t v[32];
-                tmem_ld32(t_row + (uint32_t)(c_off + c0), v);
+                tmem_ld32(t_row + (uint32_t)(s * kTile + c_off + c0), v);
 #pragma unroll
                 for (int c = 0; c < 32; ++c) {
                     sc[c0 + c] = (c_off + c0 + c < n_keys) ? __uint_as_float(v[c]) * p.scale_log2e : -INFINITY;
                     mx = fmaxf(mx, sc[c0 + c]);
                 }
             }
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars[7 + s]));           // S buffer may be overwritten
             xch[hf * kTile + r] = mx;
             asm volatile("bar.sync 1, 256;" ::: "memory");
             if (*abort_flag) { ok = false; break; }
@@ -211,6 +247,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const float alpha = exp2f(m - mx);             // m = -inf on the first tile gives 0
             m = mx;
             l *= alpha;
+            // P V of the previous tile must have finished reading the P buffer
+            if (!mbar_wait(smem_u32(&bars[10]), ((uint32_t)i & 1u) ^ 1u, abort_flag)) { *abort_flag = 1; ok = false; }
             uint8_t* prow = sP + hf * kAtom + r * 128;
 #pragma unroll
             for (int g = 0; g < 8; ++g) {                  // eight 16-byte chunks of 8 keys
@@ -227,21 +265,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 u.w = pack_bf16(pr[6], pr[7]);
                 *reinterpret_cast<uint4*>(prow + ((g ^ (r & 7)) << 4)) = u;
             }
-            tc_fence_before();
             fence_proxy_async_smem();                      // P and the zeroed V columns -> visible to the MMA
-            mbar_arrive(smem_u32(&bars[6]));
-            // O += O_tile with the running rescale (a failed wait is picked up at the next barrier)
-            if (!mbar_wait(smem_u32(&bars[7]), (uint32_t)i & 1u, abort_flag)) { *abort_flag = 1; ok = false; }
-            tc_fence_after();
-#pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(t_row + (uint32_t)(kTile + c_off + c0), v);
-#pragma unroll
-                for (int c = 0; c < 32; ++c) o[c0 + c] = o[c0 + c] * alpha + __uint_as_float(v[c]);
-            }
-            tc_fence_before();
+            mbar_arrive(smem_u32(&bars[9]));
+            if (i > 0) fold(i - 1, alpha_prev);
+            alpha_prev = alpha;
         }
+        if (ok && n_kt > 0) fold(n_kt - 1, alpha_prev);
         // row sum = sum of the two halves (same running maximum on both sides)
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (*abort_flag) {
@@ -415,7 +444,7 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     p.part_o = scratch;
     p.part_ml = scratch ? scratch + (size_t)WD_ATTN_SPLIT_SLOTS * kTile * kTile : nullptr;
     p.counters = counters;
-    const size_t smem = 6 * (size_t)kOperand + 8 * 8 + 16 + 2 * kTile * 4 + 1024;
+    const size_t smem = 6 * (size_t)kOperand + (kBars + 1) * 8 + 16 + 2 * kTile * 4 + 1024;
     static bool attr_done = false;      // one device per process
     if (!attr_done) {
         WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
