@@ -598,7 +598,7 @@ TcConfig pick_config(int rows, bool allow_wide) {
     TcConfig c;
     // Many tokens: the GEMM is bound by operand traffic from L2 into shared memory, so a CTA
     // carries two 128-row weight halves that share every activation box ([256 x BN] per CTA).
-    static const int wide_from = env_int("WD_GEMM_WIDE_FROM", 512);
+    static const int wide_from = env_int("WD_GEMM_WIDE_FROM", 512);   // measured: pays from a few hundred rows when every CTA gets whole tiles
     c.wide = (allow_wide && rows >= wide_from) ? 1 : 0;
     c.tile_rows = c.wide ? 2 * kBM : kBM;
     static const int bn_max = env_int("WD_GEMM_BN_MAX", 256);      // tuning knob (multiple of 16, <= 256)
