@@ -150,7 +150,8 @@ static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[24]) {
     off[10] = c.take(plan_ints * 4);                            // plan
     off[11] = c.take((1 + (size_t)d->max_batch + 3 * MA) * 4);  // result
     off[12] = plan_ints;
-    const size_t nch = (size_t)wd_unmask_chunks(d->vocab);
+    // unmask statistics: per vocabulary chunk (CUDA-core path) or per 128-logit GEMM tile (LM-head epilogue)
+    const size_t nch = std::max<size_t>((size_t)wd_unmask_chunks(d->vocab), 256);   // or one per CTA of the LM head
     off[13] = c.take(MA * nch * 4);                             // ch_max
     off[14] = c.take(MA * nch * 4);                             // ch_idx
     off[15] = c.take(MA * nch * 8);                             // ch_sum
@@ -762,13 +763,23 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     }
     }
     // logits for the active rows only, then the unmask reduction
+    bool lm_fused = false;
+    int lm_chunks = wd_unmask_chunks(d.vocab);
     if (NA > 0) {
         wd_launch_rmsnorm(d.dtype, c->x, nullptr, 0, 0, c->final_norm, d.rms_eps, c->xn, act_row, NA, D, stream);
         WdTcSeg lm[1] = {{c->lm_head, d.vocab, c->tc.get(WD_TC_LM, 0)}};
+        // tensor-core path: the LM-head epilogue leaves per-tile (max, argmax, sum exp) instead of a separate
+        // pass over the logits, which then never have to be written (only for the parity tap)
+        WdTcFuse fl;
+        fl.mode = WD_FUSE_LMSTATS;
+        fl.st_max = c->ch_max; fl.st_idx = c->ch_idx; fl.st_sum = c->ch_sum;
+        fl.write_logits = st->taps.logits ? 1 : 0;
+        lm_fused = use_tc(c) && NA <= 256;
         if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, lm, 1, NA, D, c->logits, (size_t)d.max_active * d.vocab, status,
-                          stream, &go, /*single_split=*/true)) != WD_OK)
+                          stream, &go, /*single_split=*/true, lm_fused ? &fl : nullptr)) != WD_OK)
             return s;
-        wd_launch_rowstats(c->logits, NA, d.vocab, c->ch_max, c->ch_idx, c->ch_sum, stream);
+        if (lm_fused) lm_chunks = fl.n_chunks;
+        else wd_launch_rowstats(c->logits, NA, d.vocab, c->ch_max, c->ch_idx, c->ch_sum, stream);
         if (st->taps.logits)
             WD_CUDA_TRY(cudaMemcpyAsync(st->taps.logits, c->logits, (size_t)NA * d.vocab * 4, cudaMemcpyDeviceToDevice,
                                         stream));
@@ -777,7 +788,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     int32_t* sel_pos = n_sel + batch;
     int32_t* sel_tok = sel_pos + (size_t)batch * std::max(k_eff, 1);
     float* sel_conf = (float*)(sel_tok + (size_t)batch * std::max(k_eff, 1));
-    wd_launch_select(c->ch_max, c->ch_idx, c->ch_sum, wd_unmask_chunks(d.vocab), c->row_token, c->row_sumexp, act_pos,
+    wd_launch_select(c->ch_max, c->ch_idx, c->ch_sum, lm_chunks, c->row_token, c->row_sumexp, act_pos,
                      act_off, 0, batch, k_eff, st->ids_dev, S, n_sel, sel_pos, sel_tok, sel_conf, c->row_conf, stream);
     const size_t res_ints = 1 + (size_t)batch + 3 * (size_t)batch * std::max(k_eff, 1);
     WD_CUDA_TRY(cudaMemcpyAsync(st->result_host, c->result, res_ints * 4, cudaMemcpyDeviceToHost, stream));

@@ -295,7 +295,10 @@ __device__ void finalize_unit(const TcParams& p, long long G, int unit, int e) {
 // epilogue of one piece overlaps the MMAs of the next (two accumulators in TMEM).  A tile cut
 // by piece boundaries gets one partial sum per CTA that touched it, written to slice
 // (CTA - first CTA of the tile); the CTA that finishes the tile zero-fills the unused slices.
-template <bool kWide>
+// kWide: two weight halves per CTA (many tokens).  kLmStats: the LM-head epilogue that reduces
+// the logits to per-row statistics.  Separate instantiations keep the plain weight-streaming
+// kernel free of the other variants' code (its issue loops are sensitive to it).
+template <bool kWide, bool kLmStats>
 __global__ void __launch_bounds__(kWide ? kThreadsWide : kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w0,
                const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2,
@@ -311,6 +314,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     uint32_t* tmem_slot = (uint32_t*)(bars + 2 * NS + 4);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     int* last_flag = (int*)(tmem_slot + 2);
+    float* lm_scratch = (float*)(tmem_slot + 4);           // 1.5 KB for the LM-head statistics
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long c = blockIdx.x, G = gridDim.x;
@@ -480,11 +484,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             tc_fence_after();
             float* yb = p.y + p.seg_col[u.seg] + n;
             const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf + half_sel) * p.buf_cols);
+            constexpr bool lm_stats = kLmStats;
+            const bool store_y = !lm_stats || p.f.write_logits;
             for (int cc = 0; cc < p.bn; cc += 16) {
                 if (u.tok0 + cc >= p.rows) break;
                 uint32_t v[16];
                 tmem_ld16(t_acc + (uint32_t)cc, v);
-                if (n_ok) {
+                if (n_ok && store_y) {
                     float* ys = yb + (size_t)ord * p.split_stride;
 #pragma unroll
                     for (int t = 0; t < 16; ++t) {
@@ -492,10 +498,75 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         if (tok < p.rows) ys[(size_t)tok * p.ncol] = __uint_as_float(v[t]);
                     }
                 }
+                if (lm_stats) {
+                    // per token: maximum / lowest argmax / sum exp over this tile's 128 logits.
+                    // Thread = one vocabulary entry; warp shuffles, then the 4 warps through shared memory.
+                    float* sh_m = lm_scratch;                       // [4][16]
+                    int* sh_i = (int*)(lm_scratch + 64);            // [4][16]
+                    double* sh_s = (double*)(lm_scratch + 128);     // [4][16]
+                    float* sh_tm = lm_scratch + 256;                // [16] tile maxima
+                    int* sh_ti = (int*)(lm_scratch + 272);          // [16] their indices
+                    float* run_m = lm_scratch + 288;                // [256] running statistics of this CTA
+                    int* run_i = (int*)(lm_scratch + 544);
+                    double* run_s = (double*)(lm_scratch + 800);
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) {
+                        float bm = n_ok ? __uint_as_float(v[t]) : -INFINITY;
+                        int bi = n_ok ? n : 0x7fffffff;
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) {
+                            const float om = __shfl_xor_sync(0xffffffffu, bm, o);
+                            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+                            if (om > bm || (om == bm && oi < bi)) { bm = om; bi = oi; }
+                        }
+                        if (lane == 0) { sh_m[quarter * 16 + t] = bm; sh_i[quarter * 16 + t] = bi; }
+                    }
+                    epi_sync();
+                    const int e = (int)threadIdx.x - 64;
+                    if (e < 16) {
+                        float bm = sh_m[e];
+                        int bi = sh_i[e];
+                        for (int w = 1; w < 4; ++w) {
+                            const float om = sh_m[w * 16 + e];
+                            const int oi = sh_i[w * 16 + e];
+                            if (om > bm || (om == bm && oi < bi)) { bm = om; bi = oi; }
+                        }
+                        sh_tm[e] = bm;
+                        sh_ti[e] = bi;
+                    }
+                    epi_sync();
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) {
+                        // single-precision exp (1 ulp), double accumulation: the tile sum is good to ~1e-9
+                        double ex = n_ok ? (double)expf(__uint_as_float(v[t]) - sh_tm[t]) : 0.0;
+#pragma unroll
+                        for (int o = 16; o > 0; o >>= 1) ex += __shfl_xor_sync(0xffffffffu, ex, o);
+                        if (lane == 0) sh_s[quarter * 16 + t] = ex;
+                    }
+                    epi_sync();
+                    if (e < 16) {
+                        // fold this tile into the CTA's running statistics of the token (tiles ascend in
+                        // vocabulary index, so on equal maxima the earlier index stays)
+                        const int tl = cc + e;                       // token within the (single) token tile
+                        if (u.tok0 + tl < p.rows) {
+                            const double ts = sh_s[e] + sh_s[16 + e] + sh_s[32 + e] + sh_s[48 + e];
+                            const float tm = sh_tm[e];
+                            if (piece == 0) {
+                                run_m[tl] = tm; run_i[tl] = sh_ti[e]; run_s[tl] = ts;
+                            } else if (tm > run_m[tl]) {
+                                run_s[tl] = run_s[tl] * exp((double)run_m[tl] - (double)tm) + ts;
+                                run_m[tl] = tm; run_i[tl] = sh_ti[e];
+                            } else {
+                                run_s[tl] += ts * exp((double)tm - (double)run_m[tl]);
+                            }
+                        }
+                    }
+                    epi_sync();
+                }
             }
             tc_fence_before();
             mbar_arrive(smem_u32(&bars[2 * NS + 2 + buf]));       // accumulator may be overwritten
-            if (p.f.mode != WD_FUSE_NONE) {
+            if (p.f.mode != WD_FUSE_NONE && p.f.mode != WD_FUSE_LMSTATS) {
                 // count this piece's arrival at its tile; the CTA that arrives last finishes the tile
                 const int e = (int)threadIdx.x - 64;
                 __threadfence();
@@ -520,7 +591,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 epi_sync();
                 if (*last_flag) finalize_unit(p, G, unit, e);
                 epi_sync();
-            } else if (kb0 + len == p.kb_total && n_ok) {
+            } else if (kb0 + len == p.kb_total && n_ok && p.f.mode == WD_FUSE_NONE) {
                 // this CTA finished the tile: slices nobody wrote must read as zero
                 for (int sl = ord + 1; sl < p.n_slices; ++sl) {
                     float* ys = yb + (size_t)sl * p.split_stride;
@@ -531,6 +602,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         if (!ok && lane == 0) {
             *abort_flag = 1;
             atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
+        }
+        if (kLmStats && sch.n_pieces > 0) {
+            // one (max, argmax, sum exp) per token for all the vocabulary tiles this CTA covered
+            float* run_m = lm_scratch + 288;
+            int* run_i = (int*)(lm_scratch + 544);
+            double* run_s = (double*)(lm_scratch + 800);
+            epi_sync();
+            for (int t = (int)threadIdx.x - 64; t < p.rows; t += 128) {
+                const size_t si = (size_t)t * G + c;
+                p.f.st_max[si] = run_m[t];
+                p.f.st_idx[si] = run_i[t];
+                p.f.st_sum[si] = run_s[t];
+            }
         }
         tc_fence_before();
     }
@@ -610,10 +694,10 @@ TcConfig pick_config(int rows, bool allow_wide) {
     const int stage = c.tile_rows * kBK * 2 + c.bn * kBK * 2;
     static const int want2 = env_int("WD_GEMM_CTAS_PER_SM", 1);
     c.ctas_per_sm = (want2 == 2 && c.bn <= 64 && !c.wide) ? 2 : 1;
-    c.n_stages = ((c.ctas_per_sm == 2 ? 100 : 196) * 1024) / stage;
+    c.n_stages = ((c.ctas_per_sm == 2 ? 96 : 192) * 1024) / stage;
     if (c.n_stages > 10) c.n_stages = 10;
     if (c.n_stages < 2) c.n_stages = 2;
-    c.smem = (size_t)c.n_stages * stage + (2 * c.n_stages + 4) * 8 + 16 + 4096 + 1024;
+    c.smem = (size_t)c.n_stages * stage + (2 * c.n_stages + 4) * 8 + 16 + 8192 + 1024;
     return c;
 }
 
@@ -722,9 +806,13 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     p.idesc = make_idesc(cfg.bn);
     if (fuse) {
         p.f = *fuse;
-        if (fuse->mode != WD_FUSE_NONE && !fuse->counters) return WD_ERR_NULL;
+        if (fuse->mode != WD_FUSE_NONE && fuse->mode != WD_FUSE_LMSTATS && !fuse->counters) return WD_ERR_NULL;
+        if (fuse->mode == WD_FUSE_LMSTATS && (!p.aligned || cfg.wide || cfg.tok_tiles != 1 || nseg != 1 || !fuse->st_max ||
+                                              !fuse->st_idx || !fuse->st_sum))
+            return WD_ERR_BAD_PARAM;
+        fuse->n_chunks = (int)G;          // one statistics entry per (row, CTA)
         if (fuse->mode == WD_FUSE_SWIGLU && (nseg != 2 || segs[0].n != segs[1].n)) return WD_ERR_BAD_PARAM;
-        if (fuse->mode != WD_FUSE_NONE && col % kBM) return WD_ERR_BAD_PARAM;      // whole tiles only
+        if (fuse->mode != WD_FUSE_NONE && fuse->mode != WD_FUSE_LMSTATS && col % kBM) return WD_ERR_BAD_PARAM;   // whole tiles only
     }
 
     CUtensorMap mx;
@@ -739,8 +827,9 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     }
     static bool attr_done = false;      // one device per process
     if (!attr_done) {
-        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
-        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         attr_done = true;
     }
     const CUtensorMap& m0 = *segs[0].map;
@@ -757,8 +846,9 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = wd_pdl_enabled ? 1 : 0;
-    if (cfg.wide) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<true>, mx, m0, m1, m2, p));
-    else WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<false>, mx, m0, m1, m2, p));
+    if (cfg.wide) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<true, false>, mx, m0, m1, m2, p));
+    else if (p.f.mode == WD_FUSE_LMSTATS) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<false, true>, mx, m0, m1, m2, p));
+    else WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<false, false>, mx, m0, m1, m2, p));
     if (n_split_out) *n_split_out = p.n_slices;
     return WD_OK;
 }

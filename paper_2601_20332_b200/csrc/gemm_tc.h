@@ -45,7 +45,7 @@ wd_status wd_tc_weights_init(WdTcWeights* tc, const wd_model_dims* d, const void
 // What the CTA that completes an output tile does with the summed tile ("fused epilogue").
 // The tile sums still pass through the partial-sum slices in y; these modes only add the
 // consumer's work to the GEMM so that no separate kernel (and no dependency bubble) follows.
-enum { WD_FUSE_NONE = 0, WD_FUSE_QKV = 1, WD_FUSE_RESID = 2, WD_FUSE_SWIGLU = 3 };
+enum { WD_FUSE_NONE = 0, WD_FUSE_QKV = 1, WD_FUSE_RESID = 2, WD_FUSE_SWIGLU = 3, WD_FUSE_LMSTATS = 4 };
 
 struct WdTcFuse {
     int mode = WD_FUSE_NONE;
@@ -72,6 +72,15 @@ struct WdTcFuse {
     // SWIGLU: h = silu(gate) * up, gate tile t and up tile t complete together
     __nv_bfloat16* h = nullptr;
     int F = 0;
+    // LMSTATS (LM head, whole tiles per CTA, rows <= 256): per (row, CTA) maximum, lowest argmax and
+    // sum of exp(l - max) over the vocabulary tiles the CTA covered, [rows][n_chunks] with n_chunks
+    // (= grid size) filled in by wd_tc_gemm; the logits themselves are written only if write_logits
+    // is set (parity tests)
+    mutable int n_chunks = 0;
+    float* st_max = nullptr;
+    int32_t* st_idx = nullptr;
+    double* st_sum = nullptr;
+    int write_logits = 0;
 };
 
 // y[split][rows][sum n_i] = x * [w_0; w_1; ...]^T, split-K partial sums side by side
