@@ -61,7 +61,8 @@ enum {
     WD_ERR_DEVICE_TIMEOUT = -9,       /* a bounded device-side wait ran out    */
     WD_ERR_BOUNDS = -10,              /* a device-side index check failed      */
     WD_ERR_NOT_PENDING = -11,         /* wd_step_sync without wd_step before   */
-    WD_ERR_MISALIGNED = -12
+    WD_ERR_MISALIGNED = -12,
+    WD_ERR_INTERNAL = -13             /* host and device planners disagree (a bug)   */
 };
 
 enum { WD_F32 = 0, WD_BF16 = 1 };     /* element type of weights, activations, K/V cache */
@@ -266,20 +267,38 @@ WD_API wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, co
 
 /* Enqueue one step for every sequence of the state on `stream` and return
  * without waiting.  k = tokens unmasked per sequence (at most the number of
- * active tokens; 0 = compute only).  Needs max_active >= batch * A.  The step
- * must be completed with wd_step_sync before the next wd_step, wd_plan or
- * wd_state_read.  `info` may be NULL.
+ * active tokens; 0 = compute only).  Needs max_active >= batch * A.  `info` may
+ * be NULL.
+ *
+ * Steps may be enqueued back to back, up to 32 without a wd_step_sync in
+ * between, while the device can plan them itself: every sequence started from
+ * a decoded prefix (prompt then masks), at most 16 sequences, adaptive
+ * termination and GEMM profiling off.  A device kernel then builds the index
+ * lists from the device copy of the state (the sets of Section 4.2 and the
+ * phase structure of Section 4.3, the same planner as wd_plan, bit for bit) and
+ * the host only supplies counts, which do not depend on which tokens were
+ * unmasked.  Otherwise (arbitrary decoded patterns, adaptive termination) the
+ * host plans each step and wd_step_sync must come before the next wd_step.
+ * wd_plan, wd_state_read, wd_state_reset and the setters need an empty queue.
  * Returns WD_OK, WD_DONE (nothing left to decode: nothing enqueued),
- * WD_ERR_PENDING, WD_ERR_BAD_PARAM, WD_ERR_CAPACITY (a dims.max_* limit),
+ * WD_ERR_PENDING (queue full, or this state needs a sync between steps),
+ * WD_ERR_BAD_PARAM, WD_ERR_CAPACITY (a dims.max_* limit), WD_ERR_INTERNAL,
  * WD_ERR_CUDA. */
 WD_API wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int32_t T, int32_t k,
                   void* stream /*cudaStream_t*/, wd_step_info* info);
 
-/* Wait for the enqueued step, read its result and the device status word,
- * apply the update set to the host mirror of the state and advance the phase
- * counters.  `out` (host) may be NULL.  Returns WD_OK, WD_ERR_NOT_PENDING,
- * WD_ERR_DEVICE_TIMEOUT, WD_ERR_BOUNDS, WD_ERR_CUDA. */
+/* Wait for every enqueued step, read the results and the device status word,
+ * apply the update sets to the host mirror of the state in order and advance the
+ * phase counters.  `out` (host, may be NULL) receives the result of the NEWEST
+ * step.  Returns WD_OK, WD_ERR_NOT_PENDING, WD_ERR_DEVICE_TIMEOUT, WD_ERR_BOUNDS,
+ * WD_ERR_INTERNAL, WD_ERR_CUDA. */
 WD_API wd_status wd_step_sync(wd_state* st, wd_step_out* out);
+
+/* The same, returning every enqueued step's result: outs[0] is the oldest.
+ * `capacity` = entries of outs (0 with outs NULL just commits); WD_ERR_CAPACITY
+ * if more steps are pending (nothing is consumed then).  *n_steps (may be NULL)
+ * = steps completed. */
+WD_API wd_status wd_step_sync_all(wd_state* st, wd_step_out* outs, int32_t capacity, int32_t* n_steps);
 
 /* ---- single operations (unit parity tests, micro-benchmarks) -------------- */
 

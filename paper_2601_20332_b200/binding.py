@@ -15,7 +15,7 @@ LIB_PATH = os.path.join(HERE, "libwd.so")
 WD_OK, WD_DONE = 0, 1
 WD_ERR_NULL, WD_ERR_INVALID_DIMS, WD_ERR_WORKSPACE_TOO_SMALL, WD_ERR_UNSUPPORTED_ARCH = -1, -2, -3, -4
 WD_ERR_BAD_PARAM, WD_ERR_CAPACITY, WD_ERR_PENDING, WD_ERR_CUDA = -5, -6, -7, -8
-WD_ERR_DEVICE_TIMEOUT, WD_ERR_BOUNDS, WD_ERR_NOT_PENDING, WD_ERR_MISALIGNED = -9, -10, -11, -12
+WD_ERR_DEVICE_TIMEOUT, WD_ERR_BOUNDS, WD_ERR_NOT_PENDING, WD_ERR_MISALIGNED, WD_ERR_INTERNAL = -9, -10, -11, -12, -13
 WD_F32, WD_BF16 = 0, 1
 WD_GEMM_AUTO, WD_GEMM_PLAIN, WD_GEMM_TCGEN05 = 0, 1, 2
 
@@ -79,6 +79,7 @@ SIGNATURES = {
     "wd_state_set_eos": (C.c_int, [vp, i32]),
     "wd_step": (C.c_int, [vp, i32, i32, i32, i32, i32, vp, C.POINTER(wd_step_info)]),
     "wd_step_sync": (C.c_int, [vp, C.POINTER(wd_step_out)]),
+    "wd_step_sync_all": (C.c_int, [vp, C.POINTER(wd_step_out), i32, i32p]),
     "wd_op_gemm": (C.c_int, [i32, i32, vp, vp, vp, i32, i32, i32, vp, C.c_size_t, vp]),
     "wd_op_gemm_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
     "wd_op_gemm_noalloc": (C.c_int, [vp, vp, vp, i32, i32, i32, vp]),
@@ -286,6 +287,21 @@ class State:
         check(lib().wd_step_sync(self.handle, C.byref(out)), "wd_step_sync")
         return dict(n_unmasked=n, positions=pos.reshape(self.batch, k), token_ids=tok.reshape(self.batch, k),
                     confidence=conf.reshape(self.batch, k))
+
+    def sync_all(self, max_steps: int = 32) -> list:
+        """wd_step_sync_all: results of every enqueued step, oldest first (all enqueued with the same k)."""
+        k = max(self._k, 1)
+        bufs, outs = [], (wd_step_out * max_steps)()
+        for i in range(max_steps):
+            n = np.zeros(self.batch, np.int32)
+            pos = np.full(self.batch * k, -1, np.int32); tok = np.full(self.batch * k, -1, np.int32)
+            conf = np.zeros(self.batch * k, np.float32)
+            bufs.append((n, pos, tok, conf))
+            outs[i] = wd_step_out(_np_i32p(n), _np_i32p(pos), _np_i32p(tok), conf.ctypes.data_as(f32p))
+        done = i32()
+        check(lib().wd_step_sync_all(self.handle, outs, max_steps, C.byref(done)), "wd_step_sync_all")
+        return [dict(n_unmasked=n, positions=pos.reshape(self.batch, k), token_ids=tok.reshape(self.batch, k),
+                     confidence=conf.reshape(self.batch, k)) for (n, pos, tok, conf) in bufs[: done.value]]
 
     def close(self):
         if self.handle:

@@ -37,6 +37,7 @@ extern "C" const char* wd_status_string(wd_status s) {
         case WD_ERR_BOUNDS: return "a device-side index check failed";
         case WD_ERR_NOT_PENDING: return "no step pending";
         case WD_ERR_MISALIGNED: return "device pointer not 256-byte aligned";
+        case WD_ERR_INTERNAL: return "internal inconsistency between the host and device planners";
         default: return "unknown status";
     }
 }
@@ -146,7 +147,8 @@ static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[24]) {
     off[8] = c.take(MA * 8);                                    // row_sumexp
     off[9] = c.take(MA * 4);                                    // row_conf
     const size_t plan_ints = 2 * MR + 2 * MA + 2 * ((size_t)d->max_batch + 1) + (size_t)d->max_batch * d->max_seq +
-                             3 * (MR / 128 + (size_t)d->max_batch + 1) + (size_t)d->max_batch;
+                             3 * (MR / 128 + (size_t)d->max_batch + 1) + 2 * (size_t)d->max_batch +
+                             (size_t)d->max_batch * d->max_seq;      // + staging of the external windows
     off[10] = c.take(plan_ints * 4);                            // plan
     off[11] = c.take((1 + (size_t)d->max_batch + 3 * MA) * 4);  // result
     off[12] = plan_ints;
@@ -178,7 +180,8 @@ extern "C" size_t wd_state_bytes(const wd_model_dims* d, int32_t batch, int32_t 
     if (!dims_valid(d) || batch < 1 || seq_len < 1 || batch > d->max_batch || seq_len > d->max_seq) return 0;
     const size_t k = (size_t)d->n_layers * batch * d->n_kv_heads * seq_len * d->head_dim * wd_elt_size(d->dtype);
     const size_t v = (size_t)d->n_layers * batch * d->n_kv_heads * seq_pad(seq_len) * d->head_dim * wd_elt_size(d->dtype);
-    return wd_align_up((size_t)batch * seq_len * 4, 256) + wd_align_up(k, 256) + wd_align_up(v, 256);
+    const size_t plan_state = wd_align_up((size_t)batch * seq_len, 256) + 2 * wd_align_up((size_t)batch * seq_len * 4, 256);
+    return wd_align_up((size_t)batch * seq_len * 4, 256) + wd_align_up(k, 256) + wd_align_up(v, 256) + plan_state;
 }
 
 extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, void* workspace,
@@ -299,6 +302,8 @@ extern "C" wd_status wd_profile_read(const wd_ctx* ctx, double* gemm_ms, double*
 // ---------------------------------------------------------------------------
 // state
 // ---------------------------------------------------------------------------
+static const int kQueueCap = 32;        // most steps enqueued without wd_step_sync
+
 struct wd_state {
     wd_ctx* ctx = nullptr;
     int batch = 0, S = 0;
@@ -310,11 +315,29 @@ struct wd_state {
     size_t kv_layer_bytes = 0, v_layer_bytes = 0;
     int Sp = 0;
     int32_t* plan_host = nullptr;       // pinned
-    int32_t* result_host = nullptr;     // pinned
+    int32_t* result_host = nullptr;     // pinned: kQueueCap result blocks
     int32_t* ids_host = nullptr;        // pinned staging for ids
+    uint8_t* dec_host = nullptr;        // pinned staging for the decoded flags
     cudaEvent_t done = nullptr;
-    bool pending = false;
-    int k_pending = 0, k_user = 0;
+    bool pending = false;               // at least one step enqueued and not yet synced
+    // Device copy of the planner state, kept up to date by the unmask kernel, and the count-level
+    // shadow on the host: with them steps can be enqueued back to back (no host round trip), the
+    // index lists being built by plan_kernel.  Used while every sequence started from a decoded
+    // prefix and adaptive termination is off.
+    uint8_t* decoded_dev = nullptr;     // [batch][S]
+    int32_t* dec_step_dev = nullptr;    // [batch][S]  (0x80808080 = never)
+    int32_t* wex_dev = nullptr;         // [batch][S]
+    bool dev_mode = false;
+    std::vector<WdCount> counts;
+    struct Pending {
+        int32_t A, B, R, T, k_eff, k_user;
+        bool host_planned;
+        std::vector<WdCountPlan> cp;
+        std::vector<WdSeqPlan> plans;   // host-planned steps only
+    };
+    std::vector<Pending> queue;
+    size_t result_slot_ints = 0;
+    bool dev_plan_allowed = true;       // WD_HOST_PLAN=1 forces the host planner (debugging)
     wd_debug_taps taps = {nullptr, nullptr, nullptr};
     bool attn_tc = false;               // tensor-core attention usable (bf16, head_dim 128)
     CUtensorMap map_k, map_vt;
@@ -333,6 +356,32 @@ static void load_host_mirror(wd_state* st, const int32_t* ids, const uint8_t* de
         s.t = 0; s.since = 0; s.phase_start = 0;          // eos_id is kept across resets
     }
     memcpy(st->ids_host, ids, (size_t)st->batch * st->S * 4);
+    // device-side planning needs every sequence to start from a decoded prefix (then the visible
+    // set stays a range) and at most WD_PLAN_MAX_BATCH sequences; adaptive termination needs the
+    // host to see every result, so it keeps the host planner
+    bool prefix = st->batch <= WD_PLAN_MAX_BATCH;
+    st->counts.assign(st->batch, WdCount());
+    for (int b = 0; b < st->batch; ++b) {
+        const WdSeq& s = st->seqs[b];
+        bool seen_undecoded = false;
+        for (int i = 0; i < st->S; ++i) {
+            st->dec_host[(size_t)b * st->S + i] = s.decoded[i];
+            if (!s.decoded[i]) seen_undecoded = true;
+            else if (seen_undecoded) prefix = false;
+        }
+        if (s.eos_id >= 0) prefix = false;
+        wd_count_init(st->counts[b], s);
+    }
+    st->dev_mode = prefix && st->dev_plan_allowed;
+    st->queue.clear();
+}
+
+// uploads the device copy of the planner state (decoded flags; decode steps = "never")
+static cudaError_t upload_plan_state(wd_state* st, cudaStream_t stream) {
+    const size_t n = (size_t)st->batch * st->S;
+    cudaError_t e = cudaMemcpyAsync(st->decoded_dev, st->dec_host, n, cudaMemcpyHostToDevice, stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(st->dec_step_dev, 0x80, n * 4, stream);
+    return e;
 }
 
 extern "C" wd_status wd_state_create(wd_ctx* ctx, int32_t batch, int32_t seq_len, const int32_t* token_ids,
@@ -360,15 +409,24 @@ extern "C" wd_status wd_state_create(wd_ctx* ctx, int32_t batch, int32_t seq_len
     st->ids_dev = (int32_t*)state_mem;
     st->kcache = (char*)state_mem + ids_bytes;
     st->vcache = st->kcache + kv;
+    {
+        char* ps = st->vcache + wd_align_up(st->v_layer_bytes * d.n_layers, 256);
+        st->decoded_dev = (uint8_t*)ps;
+        st->dec_step_dev = (int32_t*)(ps + wd_align_up((size_t)batch * seq_len, 256));
+        st->wex_dev = (int32_t*)((char*)st->dec_step_dev + wd_align_up((size_t)batch * seq_len * 4, 256));
+    }
+    st->result_slot_ints = ctx->result_ints;
     cudaError_t e;
     if ((e = cudaHostAlloc((void**)&st->plan_host, ctx->plan_ints * 4, cudaHostAllocDefault)) != cudaSuccess ||
-        (e = cudaHostAlloc((void**)&st->result_host, ctx->result_ints * 4, cudaHostAllocDefault)) != cudaSuccess ||
+        (e = cudaHostAlloc((void**)&st->result_host, ctx->result_ints * 4 * kQueueCap, cudaHostAllocDefault)) != cudaSuccess ||
         (e = cudaHostAlloc((void**)&st->ids_host, (size_t)batch * seq_len * 4, cudaHostAllocDefault)) != cudaSuccess ||
+        (e = cudaHostAlloc((void**)&st->dec_host, (size_t)batch * seq_len, cudaHostAllocDefault)) != cudaSuccess ||
         (e = cudaEventCreateWithFlags(&st->done, cudaEventDisableTiming)) != cudaSuccess) {
         wd_note_cuda_error(e, __FILE__, __LINE__);
         wd_state_destroy(st);
         return WD_ERR_CUDA;
     }
+    if (const char* ev = getenv("WD_HOST_PLAN")) st->dev_plan_allowed = !(ev[0] == '1');
     load_host_mirror(st, token_ids, decoded);
     // Far-field cache rows are never read as values, but tiles of the tensor-core attention
     // cover them (masked): start from finite contents.
@@ -381,7 +439,8 @@ extern "C" wd_status wd_state_create(wd_ctx* ctx, int32_t batch, int32_t seq_len
         if (ms != WD_OK) { wd_state_destroy(st); return ms; }
         st->attn_tc = true;
     }
-    e = cudaMemcpy(st->ids_dev, st->ids_host, (size_t)batch * seq_len * 4, cudaMemcpyHostToDevice);
+    e = upload_plan_state(st, 0);
+    if (e == cudaSuccess) e = cudaMemcpy(st->ids_dev, st->ids_host, (size_t)batch * seq_len * 4, cudaMemcpyHostToDevice);
     if (e != cudaSuccess) { wd_note_cuda_error(e, __FILE__, __LINE__); wd_state_destroy(st); return WD_ERR_CUDA; }
     *out = st;
     return WD_OK;
@@ -393,6 +452,7 @@ extern "C" wd_status wd_state_reset(wd_state* st, const int32_t* token_ids, cons
     for (size_t i = 0; i < (size_t)st->batch * st->S; ++i)
         if (token_ids[i] < 0 || token_ids[i] >= st->ctx->d.vocab) return WD_ERR_BAD_PARAM;
     load_host_mirror(st, token_ids, decoded);
+    WD_CUDA_TRY(upload_plan_state(st, (cudaStream_t)stream));
     WD_CUDA_TRY(cudaMemcpyAsync(st->ids_dev, st->ids_host, (size_t)st->batch * st->S * 4, cudaMemcpyHostToDevice,
                                 (cudaStream_t)stream));
     return WD_OK;
@@ -404,6 +464,7 @@ extern "C" wd_status wd_state_destroy(wd_state* st) {
     if (st->plan_host) cudaFreeHost(st->plan_host);
     if (st->result_host) cudaFreeHost(st->result_host);
     if (st->ids_host) cudaFreeHost(st->ids_host);
+    if (st->dec_host) cudaFreeHost(st->dec_host);
     if (st->done) cudaEventDestroy(st->done);
     delete st;
     return WD_OK;
@@ -428,6 +489,7 @@ extern "C" wd_status wd_state_set_eos(wd_state* st, int32_t eos_id) {
     if (st->pending) return WD_ERR_PENDING;
     if (eos_id >= st->ctx->d.vocab) return WD_ERR_BAD_PARAM;
     for (WdSeq& s : st->seqs) s.eos_id = eos_id < 0 ? -1 : eos_id;
+    if (eos_id >= 0) st->dev_mode = false;      // every result must reach the host planner before the next step
     return WD_OK;
 }
 
@@ -561,30 +623,66 @@ static wd_status run_gemm(wd_ctx* c, const void* x, const WdTcX* x_map, const Wd
 extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int32_t T, int32_t k, void* stream_,
                              wd_step_info* info) {
     if (!st) return WD_ERR_NULL;
-    if (st->pending) return WD_ERR_PENDING;
     if (A < 1 || B < 0 || R < 1 || T < 0 || k < 0) return WD_ERR_BAD_PARAM;
     wd_ctx* c = st->ctx;
     const wd_model_dims& d = c->d;
     cudaStream_t stream = (cudaStream_t)stream_;
     const int batch = st->batch, S = st->S;
+    // Steps can queue up only while the device plans them (and no per-step profile is being taken)
+    const bool dev_mode = st->dev_mode && !c->prof_on;
+    if (!st->queue.empty() && (!dev_mode || (int)st->queue.size() >= kQueueCap)) return WD_ERR_PENDING;
+    const int k_eff = std::min<int64_t>(k, A);
 
-    st->plans.assign(batch, WdSeqPlan());
+    // ---- shape of the step: per-sequence counts, from the host planner or from the count shadow
+    wd_state::Pending pend;
+    pend.A = A; pend.B = B; pend.R = R; pend.T = T; pend.k_eff = k_eff; pend.k_user = k;
+    pend.host_planned = !dev_mode;
+    pend.cp.assign(batch, WdCountPlan());
     bool all_done = true, any_refresh = false, all_contig = true;
-    size_t n_rows = 0, n_act = 0, n_vis = 0;
+    size_t n_rows = 0, n_act = 0, n_vis = 0, n_qtiles = 0;
     int max_vis = 0;
+    if (!dev_mode) {
+        st->plans.assign(batch, WdSeqPlan());
+        for (int b = 0; b < batch; ++b) {
+            wd_status s = wd_plan_seq(st->seqs[b], A, B, R, T, &st->plans[b]);
+            if (s != WD_OK) return s;
+            const WdSeqPlan& p = st->plans[b];
+            WdCountPlan& cp = pend.cp[b];
+            cp.done = p.done; cp.refresh = p.refresh;
+            cp.n_active = (int32_t)p.active.size(); cp.n_transient = (int32_t)p.transient.size();
+            cp.n_vis = (int32_t)p.vis.size(); cp.n_rows = (int32_t)p.rows.size(); cp.n_wex = (int32_t)p.wex.size();
+            cp.n_unmask = std::min(k_eff, cp.n_active);
+            all_contig &= p.done || p.vis_contiguous;
+        }
+    } else {
+        for (int b = 0; b < batch; ++b) {
+            wd_status s = wd_count_plan(st->counts[b], A, B, R, T, k_eff, &pend.cp[b]);
+            if (s != WD_OK) return s;
+        }
+        if (st->queue.empty()) {
+            // the host mirror is current: cross-check the shadow's counts against the full planner
+            for (int b = 0; b < batch; ++b) {
+                WdSeqPlan p;
+                if (wd_plan_seq(st->seqs[b], A, B, R, T, &p) != WD_OK) return WD_ERR_INTERNAL;
+                const WdCountPlan& cp = pend.cp[b];
+                if (p.done != cp.done) return WD_ERR_INTERNAL;
+                if (!p.done && (p.refresh != cp.refresh || (int32_t)p.rows.size() != cp.n_rows ||
+                                (int32_t)p.active.size() != cp.n_active || (int32_t)p.vis.size() != cp.n_vis ||
+                                !p.vis_contiguous))
+                    return WD_ERR_INTERNAL;
+            }
+        }
+    }
     for (int b = 0; b < batch; ++b) {
-        wd_status s = wd_plan_seq(st->seqs[b], A, B, R, T, &st->plans[b]);
-        if (s != WD_OK) return s;
-        const WdSeqPlan& p = st->plans[b];
-        if (p.done) continue;
+        const WdCountPlan& cp = pend.cp[b];
+        if (cp.done) continue;
         all_done = false;
-        any_refresh |= p.refresh;
-        all_contig &= p.vis_contiguous;
-        n_rows += p.rows.size(); n_act += p.active.size(); n_vis += p.vis.size();
-        max_vis = std::max(max_vis, (int)p.vis.size());
+        any_refresh |= cp.refresh;
+        n_rows += cp.n_rows; n_act += cp.n_active; n_vis += cp.n_vis;
+        n_qtiles += (cp.n_rows + 127) / 128;
+        max_vis = std::max(max_vis, (int)cp.n_vis);
     }
     if (all_done) return WD_DONE;
-    const int k_eff = std::min<int64_t>(k, A);
     if (n_rows > (size_t)d.max_rows || n_act > (size_t)d.max_active ||
         (size_t)batch * std::max(k_eff, 1) > (size_t)d.max_active)
         return WD_ERR_CAPACITY;
@@ -599,20 +697,43 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     const size_t o_act_off = o; o += batch + 1;
     const size_t o_vis_off = o; o += batch + 1;
     const size_t o_vis_idx = o; o += n_vis;
-    size_t n_qtiles = 0;
-    for (int b = 0; b < batch; ++b) n_qtiles += st->plans[b].done ? 0 : (st->plans[b].rows.size() + 127) / 128;
     const size_t o_qt_seq = o; o += n_qtiles;
     const size_t o_qt_row0 = o; o += n_qtiles;
     const size_t o_qt_n = o; o += n_qtiles;
     const size_t o_nvis = o; o += batch;
+    const size_t o_tseq = o; o += batch;          // step index of each sequence (for the decode-step stamps)
     if (o > c->plan_ints) return WD_ERR_CAPACITY;
-    {
+    if (dev_mode) {
+        // the device builds the lists; the host passes counts and offsets as kernel arguments
+        WdPlanLaunch pl;
+        memset(&pl, 0, sizeof(pl));
+        pl.batch = batch; pl.S = S; pl.A = A; pl.T = T;
+        int32_t r = 0, a = 0, v = 0, qt = 0;
+        for (int b = 0; b < batch; ++b) {
+            const WdCountPlan& cp = pend.cp[b];
+            pl.row_off[b] = r; pl.act_off[b] = a; pl.vis_off[b] = v; pl.qt_off[b] = qt;
+            pl.done[b] = cp.done; pl.refresh[b] = cp.refresh; pl.n_wex[b] = cp.n_wex; pl.n_vis[b] = cp.n_vis;
+            pl.t[b] = st->counts[b].t;
+            if (cp.done) continue;
+            r += cp.n_rows; a += cp.n_active; v += cp.n_vis; qt += (cp.n_rows + 127) / 128;
+        }
+        pl.row_off[batch] = r; pl.act_off[batch] = a; pl.vis_off[batch] = v; pl.qt_off[batch] = qt;
+        pl.decoded = st->decoded_dev; pl.dec_step = st->dec_step_dev; pl.wex = st->wex_dev;
+        pl.row_seq = c->plan + o_row_seq; pl.row_pos = c->plan + o_row_pos;
+        pl.act_row = c->plan + o_act_row; pl.act_pos = c->plan + o_act_pos;
+        pl.act_off_dev = c->plan + o_act_off; pl.vis_off_dev = c->plan + o_vis_off; pl.vis_idx = c->plan + o_vis_idx;
+        pl.qt_seq = c->plan + o_qt_seq; pl.qt_row0 = c->plan + o_qt_row0; pl.qt_n = c->plan + o_qt_n;
+        pl.nvis_dev = c->plan + o_nvis; pl.tseq_dev = c->plan + o_tseq;
+        pl.status = c->result;
+        wd_launch_plan(pl, stream);
+    } else {
         size_t r = 0, a = 0, v = 0, qt = 0;
         for (int b = 0; b < batch; ++b) {
             const WdSeqPlan& p = st->plans[b];
             ph[o_act_off + b] = (int32_t)a;
             ph[o_vis_off + b] = (int32_t)v;
             ph[o_nvis + b] = p.done ? 0 : (int32_t)p.vis.size();
+            ph[o_tseq + b] = st->seqs[b].t;
             if (p.done) continue;
             for (size_t t0 = 0; t0 < p.rows.size(); t0 += 128, ++qt) {
                 ph[o_qt_seq + qt] = b;
@@ -635,8 +756,20 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         }
         ph[o_act_off + batch] = (int32_t)a;
         ph[o_vis_off + batch] = (int32_t)v;
+        WD_CUDA_TRY(cudaMemcpyAsync(c->plan, ph, o * 4, cudaMemcpyHostToDevice, stream));
+        // keep the device copy of the planner state complete (the unmask kernel maintains the flags
+        // and decode steps): a refreshed external window is uploaded, so that later steps may be
+        // planned on the device again
+        size_t w = o;
+        for (int b = 0; b < batch; ++b) {
+            const WdSeqPlan& p = st->plans[b];
+            if (p.done || !p.refresh || p.wex.empty()) continue;
+            if (w + p.wex.size() > c->plan_ints) return WD_ERR_CAPACITY;
+            memcpy(ph + w, p.wex.data(), p.wex.size() * 4);
+            WD_CUDA_TRY(cudaMemcpyAsync(st->wex_dev + (size_t)b * S, ph + w, p.wex.size() * 4, cudaMemcpyHostToDevice, stream));
+            w += p.wex.size();
+        }
     }
-    WD_CUDA_TRY(cudaMemcpyAsync(c->plan, ph, o * 4, cudaMemcpyHostToDevice, stream));
     const int32_t* row_seq = c->plan + o_row_seq;
     const int32_t* row_pos = c->plan + o_row_pos;
     const int32_t* act_row = c->plan + o_act_row;
@@ -789,14 +922,18 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     int32_t* sel_tok = sel_pos + (size_t)batch * std::max(k_eff, 1);
     float* sel_conf = (float*)(sel_tok + (size_t)batch * std::max(k_eff, 1));
     wd_launch_select(c->ch_max, c->ch_idx, c->ch_sum, lm_chunks, c->row_token, c->row_sumexp, act_pos,
-                     act_off, 0, batch, k_eff, st->ids_dev, S, n_sel, sel_pos, sel_tok, sel_conf, c->row_conf, stream);
+                     act_off, 0, batch, k_eff, st->ids_dev, S, n_sel, sel_pos, sel_tok, sel_conf, c->row_conf,
+                     st->decoded_dev, st->dec_step_dev, c->plan + o_tseq, stream);
+    // this step's result block goes to its own slot of the pinned ring
     const size_t res_ints = 1 + (size_t)batch + 3 * (size_t)batch * std::max(k_eff, 1);
-    WD_CUDA_TRY(cudaMemcpyAsync(st->result_host, c->result, res_ints * 4, cudaMemcpyDeviceToHost, stream));
+    int32_t* slot = st->result_host + st->queue.size() * st->result_slot_ints;
+    WD_CUDA_TRY(cudaMemcpyAsync(slot, c->result, res_ints * 4, cudaMemcpyDeviceToHost, stream));
     WD_CUDA_TRY(cudaEventRecord(st->done, stream));
     WD_CUDA_TRY(cudaGetLastError());
+    if (!dev_mode) pend.plans = st->plans;
+    else for (int b = 0; b < batch; ++b) wd_count_commit(st->counts[b], pend.cp[b]);
+    st->queue.push_back(std::move(pend));
     st->pending = true;
-    st->k_pending = k_eff;
-    st->k_user = k;
     if (info) {
         info->is_refresh = any_refresh ? 1 : 0;
         info->n_rows = R_; info->n_active = NA; info->n_vis = (int32_t)n_vis;
@@ -805,10 +942,9 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     return WD_OK;
 }
 
-extern "C" wd_status wd_step_sync(wd_state* st, wd_step_out* out) {
-    if (!st) return WD_ERR_NULL;
-    if (!st->pending) return WD_ERR_NOT_PENDING;
-    st->pending = false;
+// Completes every enqueued step, oldest first: reads its result block, re-plans it on the host
+// mirror (which the previous step's results have just brought up to date) and commits.
+static wd_status drain_queue(wd_state* st, wd_step_out* outs, bool every_step, int32_t* n_done) {
     WD_CUDA_TRY(cudaEventSynchronize(st->done));
     if (st->ctx->prof_on) {
         wd_ctx* c = st->ctx;
@@ -819,31 +955,74 @@ extern "C" wd_status wd_step_sync(wd_state* st, wd_step_out* out) {
         }
         c->prof_bytes += c->prof_step_bytes;
     }
-    const int batch = st->batch, k = st->k_pending, kk = std::max(k, 1), ku = st->k_user;
-    const int32_t* res = st->result_host;
-    const int32_t dev_status = res[0];
-    const int32_t* n_sel = res + 1;
-    const int32_t* pos = n_sel + batch;
-    const int32_t* tok = pos + (size_t)batch * kk;
-    const float* conf = (const float*)(tok + (size_t)batch * kk);
-    if (dev_status != 0) {
-        cudaMemset(st->ctx->result, 0, 4);
-        return dev_status == WD_ERR_DEVICE_TIMEOUT ? WD_ERR_DEVICE_TIMEOUT : WD_ERR_BOUNDS;
-    }
-    for (int b = 0; b < batch; ++b) {
-        const WdSeqPlan& p = st->plans[b];
-        const int n = p.done ? 0 : std::min(n_sel[b], k);
-        if (!p.done) wd_commit_seq(st->seqs[b], p, pos + (size_t)b * k, tok + (size_t)b * k, n);
-        if (out) {
-            if (out->n_unmasked) out->n_unmasked[b] = n;
-            for (int i = 0; i < n; ++i) {
-                if (out->positions) out->positions[(size_t)b * ku + i] = pos[(size_t)b * k + i];
-                if (out->token_ids) out->token_ids[(size_t)b * ku + i] = tok[(size_t)b * k + i];
-                if (out->confidence) out->confidence[(size_t)b * ku + i] = conf[(size_t)b * k + i];
+    const int batch = st->batch;
+    wd_status result = WD_OK;
+    int32_t done = 0;
+    for (size_t q = 0; q < st->queue.size(); ++q) {
+        const wd_state::Pending& pd = st->queue[q];
+        const int k = pd.k_eff, kk = std::max(k, 1), ku = pd.k_user;
+        const int32_t* res = st->result_host + q * st->result_slot_ints;
+        const int32_t* n_sel = res + 1;
+        const int32_t* pos = n_sel + batch;
+        const int32_t* tok = pos + (size_t)batch * kk;
+        const float* conf = (const float*)(tok + (size_t)batch * kk);
+        if (res[0] != 0) {
+            cudaMemset(st->ctx->result, 0, 4);
+            result = res[0] == WD_ERR_DEVICE_TIMEOUT ? WD_ERR_DEVICE_TIMEOUT : WD_ERR_BOUNDS;
+            break;
+        }
+        // which out block receives this step: all of them in order, or only the newest
+        wd_step_out* out = nullptr;
+        if (outs) out = every_step ? &outs[done] : (q + 1 == st->queue.size() ? outs : nullptr);
+        for (int b = 0; b < batch; ++b) {
+            WdSeqPlan replanned;
+            const WdSeqPlan* p = pd.host_planned ? &pd.plans[b] : &replanned;
+            if (!pd.host_planned) {
+                if (wd_plan_seq(st->seqs[b], pd.A, pd.B, pd.R, pd.T, &replanned) != WD_OK) { result = WD_ERR_INTERNAL; break; }
+                const WdCountPlan& cp = pd.cp[b];
+                if (replanned.done != cp.done ||
+                    (!cp.done && ((int32_t)replanned.rows.size() != cp.n_rows || replanned.refresh != cp.refresh))) {
+                    result = WD_ERR_INTERNAL;
+                    break;
+                }
+            }
+            const int n = p->done ? 0 : std::min(n_sel[b], k);
+            if (!p->done) wd_commit_seq(st->seqs[b], *p, pos + (size_t)b * k, tok + (size_t)b * k, n);
+            if (out) {
+                if (out->n_unmasked) out->n_unmasked[b] = n;
+                for (int i = 0; i < n; ++i) {
+                    if (out->positions) out->positions[(size_t)b * ku + i] = pos[(size_t)b * k + i];
+                    if (out->token_ids) out->token_ids[(size_t)b * ku + i] = tok[(size_t)b * k + i];
+                    if (out->confidence) out->confidence[(size_t)b * ku + i] = conf[(size_t)b * k + i];
+                }
             }
         }
+        if (result != WD_OK) break;
+        ++done;
     }
-    return WD_OK;
+    const bool host_planned = !st->queue.empty() && st->queue.back().host_planned;
+    st->queue.clear();
+    st->pending = false;
+    if (result != WD_OK)      // shadow and device state may be ahead of the mirror: plan on the host from here on
+        st->dev_mode = false;
+    else if (host_planned)    // the count shadow did not follow host-planned steps: rebuild it from the mirror
+        for (int b = 0; b < batch; ++b) wd_count_init(st->counts[b], st->seqs[b]);
+    if (n_done) *n_done = done;
+    return result;
+}
+
+extern "C" wd_status wd_step_sync(wd_state* st, wd_step_out* out) {
+    if (!st) return WD_ERR_NULL;
+    if (st->queue.empty()) return WD_ERR_NOT_PENDING;
+    return drain_queue(st, out, false, nullptr);
+}
+
+extern "C" wd_status wd_step_sync_all(wd_state* st, wd_step_out* outs, int32_t capacity, int32_t* n_steps) {
+    if (!st) return WD_ERR_NULL;
+    if (capacity < 0 || (capacity > 0 && !outs)) return WD_ERR_BAD_PARAM;
+    if (st->queue.empty()) return WD_ERR_NOT_PENDING;
+    if (capacity > 0 && (int32_t)st->queue.size() > capacity) return WD_ERR_CAPACITY;
+    return drain_queue(st, capacity > 0 ? outs : nullptr, true, n_steps);
 }
 
 // ---------------------------------------------------------------------------
@@ -908,7 +1087,7 @@ extern "C" wd_status wd_op_unmask(const float* logits, const int32_t* positions,
     int32_t* ch_idx = (int32_t*)(ch_max + (size_t)n * nch);
     wd_launch_rowstats(logits, n, vocab, ch_max, ch_idx, ch_sum, st);
     wd_launch_select(ch_max, ch_idx, ch_sum, nch, row_token, row_sumexp, positions, nullptr, n, 1, k, nullptr, 0, n_sel,
-                     sel_pos, sel_token, sel_conf, row_conf, st);
+                     sel_pos, sel_token, sel_conf, row_conf, nullptr, nullptr, nullptr, st);
     WD_CUDA_TRY(cudaGetLastError());
     return WD_OK;
 }

@@ -5,6 +5,7 @@
 // plus CUDA-core versions of the GEMM and of attention that work for any dtype
 // and any index list; the fp32 configuration runs on them entirely and the
 // bf16 tensor-core kernels are cross-checked against them.
+#include <cstring>
 #include <utility>
 
 #include "wd_internal.h"
@@ -98,6 +99,120 @@ __device__ __forceinline__ float sum_slices1(const float* __restrict__ p, int n_
         for (int k = 0; k < 4; ++k) acc += t[k];
     }
     return acc;
+}
+
+// ---------------------------------------------------------------- device-side planner
+// One block per sequence builds the step's index lists from the device-resident state (decoded
+// flags, decode steps, the external window of the phase), so that consecutive steps can be
+// enqueued without a host round trip.  The host passes only counts (which do not depend on
+// which tokens were unmasked).  Handles the states whose visible set is a prefix range.
+//   refresh:  external window = the first n_wex undecoded positions (ordered compaction),
+//             rows = visible positions = 0 .. n_vis-1, active = the first n_act of the window
+//   normal:   one pass over the window: undecoded members in order are active (the first A) or
+//             buffer, decoded members whose age is 1..T are the transient; rows = active and
+//             transient in position order
+struct PlanArgs {
+    int32_t refresh[WD_PLAN_MAX_BATCH], done[WD_PLAN_MAX_BATCH], n_wex[WD_PLAN_MAX_BATCH], n_vis[WD_PLAN_MAX_BATCH];
+    int32_t row_off[WD_PLAN_MAX_BATCH + 1], act_off[WD_PLAN_MAX_BATCH + 1], vis_off[WD_PLAN_MAX_BATCH + 1],
+        qt_off[WD_PLAN_MAX_BATCH + 1];
+    int32_t t[WD_PLAN_MAX_BATCH];
+    int32_t S, A, T, batch;
+    const uint8_t* decoded;
+    const int32_t* dec_step;
+    int32_t* wex;                 // [batch][S]
+    int32_t *row_seq, *row_pos, *act_row, *act_pos, *act_off_dev, *vis_off_dev, *vis_idx, *qt_seq, *qt_row0, *qt_n, *nvis_dev,
+        *tseq_dev;
+    int32_t* status;
+};
+
+// exclusive prefix sum of one flag per thread over the block; returns this thread's offset and the total
+__device__ __forceinline__ int block_scan_flag(int flag, int* total, int* warp_sums) {
+    const int lane = threadIdx.x & 31, w = threadIdx.x >> 5, nw = blockDim.x >> 5;
+    const unsigned bal = __ballot_sync(0xffffffffu, flag);
+    const int in_warp = __popc(bal & ((1u << lane) - 1u));
+    __syncthreads();
+    if (lane == 0) warp_sums[w] = __popc(bal);
+    __syncthreads();
+    int off = 0, tot = 0;
+    for (int i = 0; i < nw; ++i) {
+        const int v = warp_sums[i];
+        if (i < w) off += v;
+        tot += v;
+    }
+    *total = tot;
+    return off + in_warp;
+}
+
+__global__ void plan_kernel(const PlanArgs a) {
+    __shared__ int warp_sums[32];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int b = blockIdx.x;
+    if (threadIdx.x == 0) {
+        a.act_off_dev[b] = a.act_off[b];
+        a.vis_off_dev[b] = a.vis_off[b];
+        a.nvis_dev[b] = a.done[b] ? 0 : a.n_vis[b];
+        a.tseq_dev[b] = a.t[b];
+        if (b == a.batch - 1) { a.act_off_dev[a.batch] = a.act_off[a.batch]; a.vis_off_dev[a.batch] = a.vis_off[a.batch]; }
+    }
+    if (a.done[b]) return;
+    const int S = a.S, row0 = a.row_off[b], act0 = a.act_off[b];
+    const uint8_t* dec = a.decoded + (size_t)b * S;
+    const int32_t* dstep = a.dec_step + (size_t)b * S;
+    int32_t* wex = a.wex + (size_t)b * S;
+    const int n_wex = a.n_wex[b], n_vis = a.n_vis[b];
+    const int n_rows = a.row_off[b + 1] - row0, n_act = a.act_off[b + 1] - act0;
+    // visible range and query tiles follow from the counts alone
+    for (int j = threadIdx.x; j < n_vis; j += blockDim.x) a.vis_idx[a.vis_off[b] + j] = j;
+    for (int j = threadIdx.x; j < a.qt_off[b + 1] - a.qt_off[b]; j += blockDim.x) {
+        a.qt_seq[a.qt_off[b] + j] = b;
+        a.qt_row0[a.qt_off[b] + j] = row0 + 128 * j;
+        a.qt_n[a.qt_off[b] + j] = min(128, n_rows - 128 * j);
+    }
+    if (a.refresh[b]) {
+        // ordered compaction of the undecoded positions: the first n_wex form the window
+        int base = 0;
+        for (int i0 = 0; i0 < S && base < n_wex; i0 += blockDim.x) {
+            const int i = i0 + threadIdx.x;
+            const int und = (i < S && !dec[i]) ? 1 : 0;
+            int tot;
+            const int idx = base + block_scan_flag(und, &tot, warp_sums);
+            if (und && idx < n_wex) {
+                wex[idx] = i;
+                if (idx < n_act) { a.act_pos[act0 + idx] = i; a.act_row[act0 + idx] = row0 + i; }
+            }
+            base += tot;
+        }
+        if (base < n_wex && threadIdx.x == 0) atomicCAS(a.status, 0, WD_ERR_BOUNDS);   // counts and state disagree
+        for (int j = threadIdx.x; j < n_rows; j += blockDim.x) { a.row_seq[row0 + j] = b; a.row_pos[row0 + j] = j; }
+        return;
+    }
+    int n_und = 0, n_row = 0;
+    for (int j0 = 0; j0 < n_wex; j0 += blockDim.x) {
+        const int j = j0 + threadIdx.x;
+        int und = 0, trans = 0, pos = 0;
+        if (j < n_wex) {
+            pos = wex[j];
+            und = dec[pos] ? 0 : 1;
+            const long long age = (long long)a.t[b] - (long long)dstep[pos];
+            trans = (!und && age >= 1 && age <= a.T) ? 1 : 0;
+        }
+        int tot_u, tot_r;
+        const int rank_u = n_und + block_scan_flag(und, &tot_u, warp_sums);
+        const int act = und && rank_u < a.A;
+        const int rank_r = n_row + block_scan_flag(act | trans, &tot_r, warp_sums);
+        if (act | trans) {
+            if (rank_r < n_rows) { a.row_seq[row0 + rank_r] = b; a.row_pos[row0 + rank_r] = pos; }
+            else atomicCAS(a.status, 0, WD_ERR_BOUNDS);
+        }
+        if (act) {
+            if (rank_u < n_act) { a.act_pos[act0 + rank_u] = pos; a.act_row[act0 + rank_u] = row0 + rank_r; }
+            else atomicCAS(a.status, 0, WD_ERR_BOUNDS);
+        }
+        n_und += tot_u;
+        n_row += tot_r;
+    }
+    if (threadIdx.x == 0 && n_row != n_rows) atomicCAS(a.status, 0, WD_ERR_BOUNDS);
 }
 
 // ---------------------------------------------------------------- embedding gather + RoPE table
@@ -502,7 +617,8 @@ __global__ void select_kernel(const float* __restrict__ ch_max, const int32_t* _
                               const int32_t* __restrict__ act_off, int n_single, int k, int32_t* __restrict__ ids,
                               int S, int32_t* __restrict__ n_sel, int32_t* __restrict__ sel_pos,
                               int32_t* __restrict__ sel_token, float* __restrict__ sel_conf,
-                              float* __restrict__ row_conf) {
+                              float* __restrict__ row_conf, uint8_t* __restrict__ decoded,
+                              int32_t* __restrict__ dec_step, const int32_t* __restrict__ step_of_seq) {
     pdl_launch_dependents();
     pdl_wait();
     const int b = blockIdx.x;
@@ -550,6 +666,10 @@ __global__ void select_kernel(const float* __restrict__ ch_max, const int32_t* _
             sel_token[b * k + rank] = tok;
             sel_conf[b * k + rank] = (float)(1.0 / si);
             if (ids) ids[(size_t)b * S + pos] = tok;
+            if (decoded) {                                  // device-resident planner state
+                decoded[(size_t)b * S + pos] = 1;
+                dec_step[(size_t)b * S + pos] = step_of_seq[b];
+            }
         }
     }
 }
@@ -682,10 +802,31 @@ void wd_launch_rowstats(const float* logits, int n, int V, float* ch_max, int32_
 void wd_launch_select(const float* ch_max, const int32_t* ch_idx, const double* ch_sum, int n_chunks,
                       int32_t* row_token, double* row_sumexp, const int32_t* act_pos, const int32_t* act_off,
                       int n_single, int batch, int k, int32_t* ids, int S, int32_t* n_sel, int32_t* sel_pos,
-                      int32_t* sel_token, float* sel_conf, float* row_conf, cudaStream_t st) {
+                      int32_t* sel_token, float* sel_conf, float* row_conf, uint8_t* decoded, int32_t* dec_step,
+                      const int32_t* step_of_seq, cudaStream_t st) {
     if (batch <= 0) return;
     launch_pdl(select_kernel, dim3(batch), dim3(256), 0, st, ch_max, ch_idx, ch_sum, n_chunks, row_token, row_sumexp,
-               act_pos, act_off, n_single, k, ids, S, n_sel, sel_pos, sel_token, sel_conf, row_conf);
+               act_pos, act_off, n_single, k, ids, S, n_sel, sel_pos, sel_token, sel_conf, row_conf, decoded, dec_step,
+               step_of_seq);
+}
+
+void wd_launch_plan(const WdPlanLaunch& h, cudaStream_t st) {
+    PlanArgs a;
+    memset(&a, 0, sizeof(a));
+    for (int b = 0; b < h.batch; ++b) {
+        a.refresh[b] = h.refresh[b]; a.done[b] = h.done[b]; a.n_wex[b] = h.n_wex[b]; a.n_vis[b] = h.n_vis[b];
+        a.t[b] = h.t[b];
+    }
+    for (int b = 0; b <= h.batch; ++b) {
+        a.row_off[b] = h.row_off[b]; a.act_off[b] = h.act_off[b]; a.vis_off[b] = h.vis_off[b]; a.qt_off[b] = h.qt_off[b];
+    }
+    a.S = h.S; a.A = h.A; a.T = h.T; a.batch = h.batch;
+    a.decoded = h.decoded; a.dec_step = h.dec_step; a.wex = h.wex;
+    a.row_seq = h.row_seq; a.row_pos = h.row_pos; a.act_row = h.act_row; a.act_pos = h.act_pos;
+    a.act_off_dev = h.act_off_dev; a.vis_off_dev = h.vis_off_dev; a.vis_idx = h.vis_idx;
+    a.qt_seq = h.qt_seq; a.qt_row0 = h.qt_row0; a.qt_n = h.qt_n; a.nvis_dev = h.nvis_dev; a.tseq_dev = h.tseq_dev;
+    a.status = h.status;
+    launch_pdl(plan_kernel, dim3(h.batch), dim3(256), 0, st, a);
 }
 
 int32_t* wd_op_status_ptr() {

@@ -97,3 +97,60 @@ void wd_commit_seq(WdSeq& s, const WdSeqPlan& plan, const int32_t* positions,
     s.t += 1;
     s.since += 1;
 }
+
+// ---- count-level shadow (see WdCount) ----------------------------------------------------
+
+void wd_count_init(WdCount& c, const WdSeq& s) {
+    c = WdCount();
+    for (uint8_t d : s.decoded) (d ? c.decoded : c.undecoded) += 1;
+    c.t = s.t;
+    c.since = s.since;
+    c.wex_size = (int32_t)s.wex.size();
+    for (int32_t i : s.wex) c.w_alive += s.decoded[i] ? 0 : 1;
+    // tokens unmasked at each step of the running phase, oldest first
+    if (!s.wex.empty() && s.t > s.phase_start) {
+        c.hist.assign((size_t)(s.t - s.phase_start), 0);
+        for (int32_t i : s.wex)
+            if (s.decoded[i] && s.dec_step[i] >= s.phase_start) c.hist[(size_t)(s.dec_step[i] - s.phase_start)] += 1;
+    }
+}
+
+wd_status wd_count_plan(const WdCount& c, int32_t A, int32_t B, int32_t R, int32_t T, int32_t k, WdCountPlan* out) {
+    if (!out) return WD_ERR_NULL;
+    if (A < 1 || B < 0 || R < 1 || T < 0 || k < 0) return WD_ERR_BAD_PARAM;
+    WdCountPlan& p = *out;
+    p = WdCountPlan();
+    if (c.undecoded == 0) { p.done = true; return WD_OK; }
+    p.refresh = (c.t == 0) || (c.since >= R) || (c.w_alive == 0);
+    int32_t w_alive = c.w_alive;
+    if (p.refresh) {
+        p.n_wex = (int32_t)std::min<int64_t>((int64_t)A + (int64_t)B, c.undecoded);
+        w_alive = p.n_wex;
+    } else {
+        p.n_wex = c.wex_size;
+        // tokens unmasked at the last min(T, steps in this phase) steps are still recomputed
+        const int32_t n_hist = (int32_t)c.hist.size();
+        for (int32_t age = 1; age <= T && age <= n_hist; ++age) p.n_transient += c.hist[(size_t)(n_hist - age)];
+    }
+    p.n_active = std::min(A, w_alive);
+    p.n_vis = c.decoded + w_alive;
+    p.n_rows = p.refresh ? p.n_vis : p.n_active + p.n_transient;
+    p.n_unmask = std::min(k, p.n_active);
+    return WD_OK;
+}
+
+void wd_count_commit(WdCount& c, const WdCountPlan& p) {
+    if (p.done) return;
+    if (p.refresh) {
+        c.wex_size = p.n_wex;
+        c.w_alive = p.n_wex;
+        c.since = 0;
+        c.hist.clear();
+    }
+    c.undecoded -= p.n_unmask;
+    c.decoded += p.n_unmask;
+    c.w_alive -= p.n_unmask;
+    c.hist.push_back(p.n_unmask);
+    c.t += 1;
+    c.since += 1;
+}

@@ -49,6 +49,24 @@ wd_status wd_plan_seq(const WdSeq& s, int32_t A, int32_t B, int32_t R, int32_t T
 void wd_commit_seq(WdSeq& s, const WdSeqPlan& plan, const int32_t* positions,
                    const int32_t* token_ids, int32_t n);
 
+// Count-level shadow of a sequence's planner state.  Which positions a step unmasks is only
+// known on the device, but HOW MANY rows, active rows and visible positions the following steps
+// have does not depend on it (k tokens leave the window per step), so the host can size the
+// launches of several steps ahead while the device plans the index lists.
+struct WdCount {
+    int32_t undecoded = 0, decoded = 0;   // |U|, |Dec|
+    int32_t wex_size = 0, w_alive = 0;    // external window: size at phase start, still undecoded
+    int32_t t = 0, since = 0;
+    std::vector<int32_t> hist;            // tokens unmasked at each step of the current phase
+};
+struct WdCountPlan {
+    bool done = false, refresh = false;
+    int32_t n_active = 0, n_transient = 0, n_vis = 0, n_rows = 0, n_wex = 0, n_unmask = 0;
+};
+void wd_count_init(WdCount& c, const WdSeq& s);
+wd_status wd_count_plan(const WdCount& c, int32_t A, int32_t B, int32_t R, int32_t T, int32_t k, WdCountPlan* out);
+void wd_count_commit(WdCount& c, const WdCountPlan& p);
+
 // ---------------------------------------------------------------------------
 // kernel launchers.  Every pointer is a device pointer unless stated.
 // `status` is a device int32: kernels store WD_ERR_* there on a failed check.
@@ -114,7 +132,26 @@ void wd_launch_rowstats(const float* logits, int n, int V, float* ch_max, int32_
 void wd_launch_select(const float* ch_max, const int32_t* ch_idx, const double* ch_sum, int n_chunks,
                       int32_t* row_token, double* row_sumexp, const int32_t* act_pos, const int32_t* act_off,
                       int n_single, int batch, int k, int32_t* ids, int S, int32_t* n_sel, int32_t* sel_pos,
-                      int32_t* sel_token, float* sel_conf, float* row_conf, cudaStream_t st);
+                      int32_t* sel_token, float* sel_conf, float* row_conf, uint8_t* decoded, int32_t* dec_step,
+                      const int32_t* step_of_seq, cudaStream_t st);
+
+// Device-side planner (one block per sequence): builds the step's index lists from the device
+// copy of the state; the host supplies counts and offsets only.  Up to WD_PLAN_MAX_BATCH sequences.
+#define WD_PLAN_MAX_BATCH 16
+struct WdPlanLaunch {
+    int32_t batch, S, A, T;
+    int32_t refresh[WD_PLAN_MAX_BATCH], done[WD_PLAN_MAX_BATCH], n_wex[WD_PLAN_MAX_BATCH], n_vis[WD_PLAN_MAX_BATCH],
+        t[WD_PLAN_MAX_BATCH];
+    int32_t row_off[WD_PLAN_MAX_BATCH + 1], act_off[WD_PLAN_MAX_BATCH + 1], vis_off[WD_PLAN_MAX_BATCH + 1],
+        qt_off[WD_PLAN_MAX_BATCH + 1];
+    const uint8_t* decoded;       // [batch][S] device
+    const int32_t* dec_step;      // [batch][S] device
+    int32_t* wex;                 // [batch][S] device: external window of the phase
+    int32_t *row_seq, *row_pos, *act_row, *act_pos, *act_off_dev, *vis_off_dev, *vis_idx, *qt_seq, *qt_row0, *qt_n, *nvis_dev,
+        *tseq_dev;
+    int32_t* status;
+};
+void wd_launch_plan(const WdPlanLaunch& h, cudaStream_t st);
 
 int32_t* wd_op_status_ptr();   // device address of the single-operation status word
 extern bool wd_pdl_enabled;    // programmatic dependent launch on every kernel (default on)

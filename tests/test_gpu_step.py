@@ -176,7 +176,10 @@ def test_far_field_and_refresh_independence_on_gpu(shape):
         if variant:
             ids_v[0, cfg["P"] + cfg["A"] + cfg["B"]:] = 17
         st = wd.State(ctx, ids_v, (ids != cfg["mask_id"]).astype(np.uint8))
-        st.mem.view(torch.int16)[S * 2 + 128:].fill_(0x7FC0 if variant else 0)      # NaN / zero K/V cache
+        # state memory = ids | K cache | V cache | device planner state (flags, steps, window)
+        up = lambda v: (v + 255) // 256 * 256
+        tail = (up(S) + 2 * up(4 * S)) // 2
+        st.mem.view(torch.int16)[S * 2 + 128: -tail].fill_(0x7FC0 if variant else 0)      # NaN / zero K/V cache
         torch.cuda.synchronize()
         lg = torch.zeros(S * cfg["V"], device=DEV)
         st.set_taps(logits=lg)
@@ -189,6 +192,68 @@ def test_far_field_and_refresh_independence_on_gpu(shape):
         st.close(); ctx.close()
     for a, b in zip(*outs):
         assert torch.equal(a[0], b[0]) and (a[1] == b[1]).all() and (a[2] == b[2]).all()
+
+
+@pytest.mark.parametrize("shape,batch", [(SMALL_BF16, 1), (DH128, 2)])
+def test_steps_enqueued_back_to_back_match_stepwise_sync(shape, batch):
+    """With a prompt-prefix state the device plans the steps itself: a whole run enqueued without
+    a host round trip gives exactly the results of the same run with a sync after every step,
+    and the host mirror ends up identical."""
+    cfg = synth.get_config("llada8b", **dict(shape, batch=batch))
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    S = ids.shape[1]
+    n_steps = 11
+    ctx = wd.Context(cfg, w, batch, S, batch * S, batch * cfg["A"])
+    runs = []
+    for queued in (False, True):
+        st = wd.State(ctx, ids)
+        res = []
+        for i in range(n_steps):
+            st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])
+            if not queued:
+                res.append(st.sync())
+        if queued:
+            res = st.sync_all()
+            assert len(res) == n_steps
+        runs.append((res, [st.read(b) for b in range(batch)]))
+        st.close()
+    for a, b in zip(*[r[0] for r in runs]):
+        assert (a["n_unmasked"] == b["n_unmasked"]).all()
+        assert (a["positions"] == b["positions"]).all() and (a["token_ids"] == b["token_ids"]).all()
+        assert (a["confidence"] == b["confidence"]).all()
+    for ma, mb in zip(runs[0][1], runs[1][1]):
+        assert (ma["ids"] == mb["ids"]).all() and (ma["decoded"] == mb["decoded"]).all()
+        assert (ma["dec_step"] == mb["dec_step"]).all() and ma["t"] == mb["t"] == n_steps and ma["since"] == mb["since"]
+    # the queue holds 32 steps; the 33rd needs a sync first
+    st = wd.State(ctx, ids)
+    for i in range(32):
+        st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])
+    with pytest.raises(wd.WdError) as e:
+        st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])
+    assert e.value.status == wd.WD_ERR_PENDING
+    with pytest.raises(wd.WdError) as e:
+        st.plan(0, cfg["A"], cfg["B"], cfg["R"], cfg["T"])
+    assert e.value.status == wd.WD_ERR_PENDING
+    st.sync()
+    assert st.read(0)["t"] == 32
+    st.close(); ctx.close()
+
+
+def test_non_prefix_state_needs_a_sync_between_steps():
+    cfg = synth.get_config("llada8b", **SMALL_BF16)
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    S = ids.shape[1]
+    dec = synth.random_decoded_pattern(S, 0.4, 5)[None, :]
+    ctx = wd.Context(cfg, w, 1, S, S, S)
+    st = wd.State(ctx, ids, dec)
+    st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], 1)
+    with pytest.raises(wd.WdError) as e:
+        st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], 1)
+    assert e.value.status == wd.WD_ERR_PENDING
+    st.sync()
+    st.close(); ctx.close()
 
 
 def test_step_error_codes():
@@ -209,9 +274,6 @@ def test_step_error_codes():
     assert e.value.status == wd.WD_ERR_NOT_PENDING
     status, _ = st.step(8, 8, 4, 2, 1)                # 40 + 16 = 56 rows fits
     assert status == wd.WD_OK
-    with pytest.raises(wd.WdError) as e:
-        st.step(8, 8, 4, 2, 1)
-    assert e.value.status == wd.WD_ERR_PENDING
     st.sync()
     st.close(); ctx.close()
     with pytest.raises(wd.WdError) as e:
