@@ -75,8 +75,6 @@ struct wd_ctx {
     double* ch_sum = nullptr;
     float2* rope_tab = nullptr;  // [max_rows][dh/2] (cos, sin) of this step's rows
     float* sumsq = nullptr;      // [d/128][max_rows] partial sums of squares of the residual rows
-    float* attn_scratch = nullptr;     // parts of the attention's split over keys
-    int32_t* attn_counters = nullptr;
     int32_t* tile_counters = nullptr;  // arrival counters of the fused GEMM epilogues (kept zero)
     size_t n_tile_counters = 0;
     bool fuse = false;           // fused GEMM epilogues (experimental: slower than separate kernels so far)
@@ -161,8 +159,7 @@ static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[24]) {
     off[17] = c.take(((size_t)d->d_model / 128 + 1) * MR * 4);  // sumsq
     off[18] = c.take(((max_gemm_cols(d) + 127) / 128) * (MR / 256 + 2) * 4);   // tile counters
     off[19] = ((max_gemm_cols(d) + 127) / 128) * (MR / 256 + 2);
-    off[20] = c.take(wd_attn_tc_scratch_floats() * 4);          // attention split parts
-    off[21] = c.take(WD_ATTN_SPLIT_SLOTS * 4);                  // attention counters
+    off[20] = off[21] = c.off;                                   // (unused)
 }
 
 extern "C" size_t wd_workspace_bytes(const wd_model_dims* dims) {
@@ -249,9 +246,6 @@ extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, v
     c->tile_counters = (int32_t*)(base + off[18]);
     c->n_tile_counters = off[19];
     WD_CUDA_TRY(cudaMemset(c->tile_counters, 0, c->n_tile_counters * 4));
-    c->attn_scratch = (float*)(base + off[20]);
-    c->attn_counters = (int32_t*)(base + off[21]);
-    WD_CUDA_TRY(cudaMemset(c->attn_counters, 0, WD_ATTN_SPLIT_SLOTS * 4));
     WD_CUDA_TRY(cudaMemset(c->result, 0, 4));
 
     if (dims->dtype == WD_BF16) {
@@ -796,7 +790,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         if (st->attn_tc && all_contig && c->attn_impl != WD_GEMM_PLAIN)
             return wd_attn_tc_launch(c->q, R_, (int)n_qtiles, c->plan + o_qt_seq, c->plan + o_qt_row0, c->plan + o_qt_n,
                                      c->plan + o_nvis, &st->map_k, &st->map_vt, c->attn, attn_tap, Hq, Hkv, dh, l, max_vis,
-                                     c->sm_count, c->attn_scratch, c->attn_counters, status, stream);
+                                     c->sm_count, status, stream);
         wd_launch_attention_plain(d.dtype, c->q, kc, vc, row_seq, vis_idx, vis_off, c->attn, attn_tap, R_, max_vis, Hq,
                                   Hkv, dh, S, Sp, stream);
         return WD_OK;

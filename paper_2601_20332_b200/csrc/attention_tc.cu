@@ -21,8 +21,10 @@
 // (rows are independent).  Keys at or beyond n_vis are masked by selection, and their V
 // columns are zeroed in shared memory, so stale or poisoned cache rows cannot leak in.
 // When there are few (tile, head) pairs, as in a normal step, the keys are also split across
-// CTAs (grid.z) so that the machine is filled: each CTA leaves its running maximum, sum and
-// unnormalised output in scratch and the last one to arrive merges them in a fixed order.
+// the CTAs of a thread-block cluster (grid.z = cluster size <= 8) so that the machine is filled:
+// each CTA leaves its running maximum, sum and unnormalised output in its own shared memory, and
+// after a cluster barrier every CTA merges a share of the rows, reading the other parts through
+// distributed shared memory in a fixed order (no global round trip, no atomics).
 // Every wait is bounded; on expiry the CTA records WD_ERR_DEVICE_TIMEOUT and leaves.
 #include <cstring>
 
@@ -38,7 +40,8 @@ constexpr int kAtom = kTile * 64 * 2;      // one [128 x 64] bf16 swizzle-atom c
 constexpr int kOperand = 2 * kAtom;        // a [128 x 128] bf16 operand: 32 KB
 constexpr int kThreads = 320;            // TMA warp, MMA warp, 8 softmax warps
 constexpr int kTmemCols = 512;             // S0, S1: columns 0..255; O_tile0, O_tile1: columns 256..511
-constexpr int kBars = 15;
+constexpr int kBars = 17;
+constexpr int kMaxCluster = 8;             // portable cluster size
 
 struct AttnParams {
     const int32_t* qtile_seq;    // [n_tiles] sequence of the tile
@@ -51,14 +54,31 @@ struct AttnParams {
     float scale_log2e;           // log2(e) / sqrt(dh)
     int32_t* status;
     uint32_t idesc;
-    // split over the keys: CTA z of (tile, head) takes key tiles [z * tiles_per_split, ...) and, when a
-    // sequence needs more than one CTA, leaves (m, l, unnormalised O) in scratch; the CTA that arrives
-    // last merges the parts in order of z
+    // split over the keys: CTA z of (tile, head) takes key tiles [z * tiles_per_split, ...); the
+    // max_parts CTAs of a (tile, head) pair form one cluster
     int tiles_per_split, max_parts;
-    float* part_o;               // [(tile * Hq + h) * max_parts + z][128 rows][128]
-    float* part_ml;              // [(tile * Hq + h) * max_parts + z][128 rows][2]
-    int32_t* counters;           // [n_tiles * Hq], zero between launches
 };
+
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t dsmem_addr(uint32_t local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float4 dsmem_ld4(uint32_t a) {
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ float2 dsmem_ld2(uint32_t a) {
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(a));
+    return v;
+}
 
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
@@ -69,15 +89,19 @@ __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_vt, const AttnParams p) {
     extern __shared__ uint8_t smem_raw[];
+    // the same offset in every CTA of the cluster (the dynamic window starts at the same address)
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;                          // 32 KB
     uint8_t* sP = smem + kOperand;               // 32 KB
     uint8_t* sKV = smem + 2 * kOperand;          // 2 stages x (K 32 KB + V^T 32 KB)
     uint64_t* bars = (uint64_t*)(smem + 2 * kOperand + 4 * kOperand);
-    // 0 q_full | 1,2 kv_full | 3,4 kv_empty | 5,6 s_full | 7,8 s_empty | 9 p_full | 10 p_empty |
-    // 11,12 o_full | 13,14 o_empty.  "empty" barriers that the softmax threads signal count 256.
+    // 0 q_full | 1,2 k_full | 3,4 kv_empty | 5,6 s_full | 7,8 s_empty | 9 p_full | 10 p_empty |
+    // 11,12 o_full | 13,14 o_empty | 15,16 v_full.  "empty" barriers that the softmax threads signal count 256.
     uint32_t* tmem_slot = (uint32_t*)(bars + kBars + 1);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+    // after the last P V the K/V ring is free: this CTA's part of a split lives there
+    float* part_o = (float*)sKV;                           // [128 rows][128], 16-byte chunks XOR-swizzled by row
+    float* part_ml = (float*)(sKV + 2 * kOperand);         // [128 rows][2] running maximum, sum
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x, h = blockIdx.y;
@@ -85,27 +109,33 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int kvh = h / (p.Hq / p.Hkv);
 
     pdl_launch_dependents();
-    // the index lists were copied before the first kernel of the step: safe to read right away
+    // the index lists were written before the first kernel of the step: safe to read right away
     const int n_vis = p.seq_nvis[b];
     const int n_kt_all = (n_vis + kTile - 1) / kTile;
     const int n_parts = (n_kt_all + p.tiles_per_split - 1) / p.tiles_per_split;
     const int kt_begin = (int)blockIdx.z * p.tiles_per_split;
-    if (kt_begin >= n_kt_all) return;                       // nothing for this CTA (uniform exit)
-    const int n_kt = min(p.tiles_per_split, n_kt_all - kt_begin);
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < kBars; ++i)
-            mbar_init(smem_u32(&bars[i]), (i == 7 || i == 8 || i == 9 || i == 13 || i == 14) ? 256u : 1u);
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    // a CTA without key tiles still takes part in the cluster barriers below
+    const bool has_work = kt_begin < n_kt_all;
+    const int n_kt = has_work ? min(p.tiles_per_split, n_kt_all - kt_begin) : 0;
+    uint32_t tmem_base = 0;
+    if (has_work) {
+        if (threadIdx.x == 0) {
+            for (int i = 0; i < kBars; ++i)
+                mbar_init(smem_u32(&bars[i]), (i == 7 || i == 8 || i == 9 || i == 13 || i == 14) ? 256u : 1u);
+            *abort_flag = 0;
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        tc_fence_before();
+        __syncthreads();
+        tc_fence_after();
+        tmem_base = *tmem_slot;
     }
-    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
     pdl_wait();                                   // q and the cache rows come from the previous kernel
 
-    if (warp == 0) {
+    if (!has_work) {
+        // nothing to compute
+    } else if (warp == 0) {
         if (lane == 0) {
             // ---------------------------------------------------- TMA producer
             const uint32_t qf = smem_u32(&bars[0]);
@@ -120,14 +150,15 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
                     break;
                 }
-                const uint32_t full = smem_u32(&bars[1 + s]);
+                const uint32_t kfull = smem_u32(&bars[1 + s]), vfull = smem_u32(&bars[15 + s]);
                 const uint32_t sk = smem_u32(sKV + (size_t)s * 2 * kOperand), sv = sk + kOperand;
-                mbar_expect_tx(full, 2 * kOperand);
                 const int kv0 = (kt_begin + i) * kTile, bh = b * p.Hkv + kvh;
-                tma_load_4d(sk, &map_k, full, 0, kv0, bh, p.layer);            // keys kv0.., dims 0..63
-                tma_load_4d(sk + kAtom, &map_k, full, 64, kv0, bh, p.layer);   // dims 64..127
-                tma_load_4d(sv, &map_vt, full, kv0, 0, bh, p.layer);           // all dims, keys kv0..kv0+63
-                tma_load_4d(sv + kAtom, &map_vt, full, kv0 + 64, 0, bh, p.layer);
+                mbar_expect_tx(kfull, kOperand);
+                tma_load_4d(sk, &map_k, kfull, 0, kv0, bh, p.layer);            // keys kv0.., dims 0..63
+                tma_load_4d(sk + kAtom, &map_k, kfull, 64, kv0, bh, p.layer);   // dims 64..127
+                mbar_expect_tx(vfull, kOperand);
+                tma_load_4d(sv, &map_vt, vfull, kv0, 0, bh, p.layer);           // all dims, keys kv0..kv0+63
+                tma_load_4d(sv + kAtom, &map_vt, vfull, kv0 + 64, 0, bh, p.layer);
             }
         }
         __syncwarp();
@@ -142,7 +173,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             auto issue_qk = [&](int j) -> bool {           // S[j&1] = Q K(j)^T
                 const int s = j & 1;
                 const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-                if (!mbar_wait(smem_u32(&bars[1 + s]), ph, abort_flag)) return false;        // K(j), V(j) landed
+                if (!mbar_wait(smem_u32(&bars[1 + s]), ph, abort_flag)) return false;        // K(j) landed
                 if (!mbar_wait(smem_u32(&bars[7 + s]), ph ^ 1u, abort_flag)) return false;   // S(j-2) has been read
                 tc_fence_after();
                 const uint32_t sk = smem_u32(sKV + (size_t)s * 2 * kOperand);
@@ -160,6 +191,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 const int s = i & 1;
                 const uint32_t ph = (uint32_t)(i >> 1) & 1u;
                 if (i + 1 < n_kt && !(ok = issue_qk(i + 1))) break;                           // runs ahead of the softmax
+                if (!(ok = mbar_wait(smem_u32(&bars[15 + s]), ph, abort_flag))) break;              // V(i) landed
                 if (!(ok = mbar_wait(smem_u32(&bars[9]), (uint32_t)i & 1u, abort_flag))) break;      // P(i) written
                 if (!(ok = mbar_wait(smem_u32(&bars[13 + s]), ph ^ 1u, abort_flag))) break;         // O_tile(i-2) folded
                 tc_fence_after();
@@ -186,6 +218,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const int quarter = warp & 3;                      // TMEM lanes 32*quarter .. +31
         const int hf = (warp - 2) >> 2;                    // which 64 columns of a 128-wide tile
         const int r = quarter * 32 + lane;                 // query row of the tile = TMEM lane
+        // warps whose 32 rows are all beyond the valid ones only keep the barrier counts right.
+        // The test is per warp, not per row: tcgen05.ld is warp-collective and must not diverge.
+        const bool live = quarter * 32 < n_valid;
+        const bool valid = r < n_valid;
         const int c_off = 64 * hf;
         const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
         float* xch = (float*)(tmem_slot + 4);              // [2][128] exchange between the two halves
@@ -200,12 +236,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const int s = j & 1;
             if (!mbar_wait(smem_u32(&bars[11 + s]), (uint32_t)(j >> 1) & 1u, abort_flag)) { *abort_flag = 1; ok = false; }
             tc_fence_after();
+            if (live) {
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(t_row + (uint32_t)(2 * kTile + s * kTile + c_off + c0), v);
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(t_row + (uint32_t)(2 * kTile + s * kTile + c_off + c0), v);
 #pragma unroll
-                for (int c = 0; c < 32; ++c) o[c0 + c] = o[c0 + c] * alpha + __uint_as_float(v[c]);
+                    for (int c = 0; c < 32; ++c) o[c0 + c] = o[c0 + c] * alpha + __uint_as_float(v[c]);
+                }
             }
             tc_fence_before();
             mbar_arrive(smem_u32(&bars[13 + s]));          // O_tile buffer may be overwritten
@@ -221,6 +259,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             // keys past n_vis may hold anything: zero their V columns so that 0 * garbage stays 0.
             // Thread (r, hf) owns row r (a head dim) of atom hf (keys 64*hf..) of the transposed V tile.
             if (n_keys < c_off + 64) {
+                if (!mbar_wait(smem_u32(&bars[15 + s]), (uint32_t)(i >> 1) & 1u, abort_flag)) *abort_flag = 1;   // V landed
                 uint8_t* vt = sKV + (size_t)s * 2 * kOperand + kOperand + hf * kAtom + r * 128;
                 for (int kv = max(n_keys - c_off, 0); kv < 64; ++kv)
                     *reinterpret_cast<uint16_t*>(vt + (((kv >> 3) ^ (r & 7)) << 4) + (kv & 7) * 2) = 0;
@@ -228,14 +267,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             // scaled scores of this thread's 64 keys, kept in registers for both passes
             float sc[64];
             float mx = -INFINITY;
+            if (live) {
 #pragma unroll
-            for (int c0 = 0; c0 < 64; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld32(t_row + (uint32_t)(s * kTile + c_off + c0), v);
+                for (int c0 = 0; c0 < 64; c0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld32(t_row + (uint32_t)(s * kTile + c_off + c0), v);
 #pragma unroll
-                for (int c = 0; c < 32; ++c) {
-                    sc[c0 + c] = (c_off + c0 + c < n_keys) ? __uint_as_float(v[c]) * p.scale_log2e : -INFINITY;
-                    mx = fmaxf(mx, sc[c0 + c]);
+                    for (int c = 0; c < 32; ++c) {
+                        sc[c0 + c] = (c_off + c0 + c < n_keys) ? __uint_as_float(v[c]) * p.scale_log2e : -INFINITY;
+                        mx = fmaxf(mx, sc[c0 + c]);
+                    }
                 }
             }
             tc_fence_before();
@@ -243,27 +284,32 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             xch[hf * kTile + r] = mx;
             asm volatile("bar.sync 1, 256;" ::: "memory");
             if (*abort_flag) { ok = false; break; }
-            mx = fmaxf(fmaxf(mx, xch[(hf ^ 1) * kTile + r]), m);
-            const float alpha = exp2f(m - mx);             // m = -inf on the first tile gives 0
-            m = mx;
-            l *= alpha;
+            float alpha = 0.f;
+            if (live) {
+                mx = fmaxf(fmaxf(mx, xch[(hf ^ 1) * kTile + r]), m);
+                alpha = exp2f(m - mx);                     // m = -inf on the first tile gives 0
+                m = mx;
+                l *= alpha;
+            }
             // P V of the previous tile must have finished reading the P buffer
             if (!mbar_wait(smem_u32(&bars[10]), ((uint32_t)i & 1u) ^ 1u, abort_flag)) { *abort_flag = 1; ok = false; }
-            uint8_t* prow = sP + hf * kAtom + r * 128;
+            if (live) {
+                uint8_t* prow = sP + hf * kAtom + r * 128;
 #pragma unroll
-            for (int g = 0; g < 8; ++g) {                  // eight 16-byte chunks of 8 keys
-                float pr[8];
+                for (int g = 0; g < 8; ++g) {              // eight 16-byte chunks of 8 keys
+                    float pr[8];
 #pragma unroll
-                for (int c = 0; c < 8; ++c) {
-                    pr[c] = exp2f(sc[8 * g + c] - mx);     // masked keys: exp2(-inf) = 0
-                    l += pr[c];
+                    for (int c = 0; c < 8; ++c) {
+                        pr[c] = exp2f(sc[8 * g + c] - mx); // masked keys: exp2(-inf) = 0
+                        l += pr[c];
+                    }
+                    uint4 u;
+                    u.x = pack_bf16(pr[0], pr[1]);
+                    u.y = pack_bf16(pr[2], pr[3]);
+                    u.z = pack_bf16(pr[4], pr[5]);
+                    u.w = pack_bf16(pr[6], pr[7]);
+                    *reinterpret_cast<uint4*>(prow + ((g ^ (r & 7)) << 4)) = u;
                 }
-                uint4 u;
-                u.x = pack_bf16(pr[0], pr[1]);
-                u.y = pack_bf16(pr[2], pr[3]);
-                u.z = pack_bf16(pr[4], pr[5]);
-                u.w = pack_bf16(pr[6], pr[7]);
-                *reinterpret_cast<uint4*>(prow + ((g ^ (r & 7)) << 4)) = u;
             }
             fence_proxy_async_smem();                      // P and the zeroed V columns -> visible to the MMA
             mbar_arrive(smem_u32(&bars[9]));
@@ -281,7 +327,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         asm volatile("bar.sync 1, 256;" ::: "memory");
         l += xch[(hf ^ 1) * kTile + r];
         if (n_parts == 1) {
-            if (ok && r < n_valid) {
+            if (ok && valid) {
                 const float inv = 1.f / l;
                 const size_t base = ((size_t)(row0 + r) * p.Hq + h) * kTile + c_off;
                 uint4* dst = reinterpret_cast<uint4*>(p.out + base);
@@ -299,58 +345,97 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     for (int c = 0; c < 64; ++c) p.tap[base + c] = o[c] * inv;
                 }
             }
-        } else {
-            // leave this CTA's part in scratch, count the arrival, the last CTA merges
-            const size_t slot = ((size_t)tile * p.Hq + h) * p.max_parts;
-            if (ok && r < n_valid) {
-                float4* dst = reinterpret_cast<float4*>(p.part_o + ((slot + blockIdx.z) * kTile + r) * kTile + c_off);
+        } else if (valid) {
+            // this CTA's part: every tensor-core read of the K/V ring has completed (the last fold
+            // waited for the last P V), so the ring is reused.  Chunk c of row r sits at c ^ (r & 31).
+            float4* dst = reinterpret_cast<float4*>(part_o + (size_t)r * kTile);
 #pragma unroll
-                for (int g = 0; g < 16; ++g) dst[g] = make_float4(o[4 * g], o[4 * g + 1], o[4 * g + 2], o[4 * g + 3]);
-                if (hf == 0)
-                    *reinterpret_cast<float2*>(p.part_ml + ((slot + blockIdx.z) * kTile + r) * 2) = make_float2(m, l);
-            }
-            // one fence after the barrier publishes every thread's part (fences are cumulative)
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            int* last_flag = (int*)(tmem_slot + 2);
-            if (threadIdx.x == 64) {
-                __threadfence();
-                const int old = atomicAdd(p.counters + tile * p.Hq + h, 1);
-                const int last = old + 1 == n_parts ? 1 : 0;
-                if (last) p.counters[tile * p.Hq + h] = 0;
-                *last_flag = last;
-                __threadfence();
-            }
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            if (*last_flag) {
-                // warp w merges rows w, w + 8, ...; lanes hold 4 columns each
-                for (int rr = warp - 2; rr < n_valid; rr += 8) {
-                    float mxx = -INFINITY;
-                    for (int z = 0; z < n_parts; ++z) mxx = fmaxf(mxx, __ldcg(p.part_ml + ((slot + z) * kTile + rr) * 2));
-                    float lsum = 0.f;
-                    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-                    for (int z = 0; z < n_parts; ++z) {
-                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(p.part_ml + ((slot + z) * kTile + rr) * 2));
-                        const float wgt = exp2f(ml.x - mxx);
-                        const float4 v = __ldcg(reinterpret_cast<const float4*>(p.part_o + ((slot + z) * kTile + rr) * kTile) + lane);
-                        lsum += ml.y * wgt;
-                        acc.x += v.x * wgt; acc.y += v.y * wgt; acc.z += v.z * wgt; acc.w += v.w * wgt;
+            for (int g = 0; g < 16; ++g)
+                dst[(hf * 16 + g) ^ (r & 31)] = make_float4(o[4 * g], o[4 * g + 1], o[4 * g + 2], o[4 * g + 3]);
+            if (hf == 0) *reinterpret_cast<float2*>(part_ml + r * 2) = make_float2(m, l);
+        }
+    }
+    if (p.max_parts > 1) {
+        // ------------------------------------------------------------ merge across the cluster
+        cluster_sync_all();                                // every part is in place and visible
+        if (has_work && n_parts > 1 && warp >= 2) {
+            // CTA z merges rows [z * per, (z + 1) * per).  An item = (row, group of 4 columns); a
+            // thread takes items t, t + 256, ... and keeps kItems x kParts remote loads in flight.
+            constexpr int kItems = 2, kParts = 4;
+            const int per = (n_valid + n_parts - 1) / n_parts;
+            const int r_lo = min((int)blockIdx.z * per, n_valid), r_hi = min(r_lo + per, n_valid);
+            const int t = (int)threadIdx.x - 64, n_items = (r_hi - r_lo) * 32;
+            const uint32_t lo = smem_u32(part_o), lml = smem_u32(part_ml);
+            for (int it0 = t; it0 < n_items; it0 += 256 * kItems) {
+                float mxx[kItems], lsum[kItems];
+                float4 acc[kItems];
+#pragma unroll
+                for (int u = 0; u < kItems; ++u) {
+                    mxx[u] = -INFINITY;
+                    lsum[u] = 0.f;
+                    acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+                for (int z0 = 0; z0 < n_parts; z0 += kParts) {       // parts in order of z
+                    float2 ml[kItems][kParts];
+                    float4 v[kItems][kParts];
+#pragma unroll
+                    for (int u = 0; u < kItems; ++u) {
+                        const int item = it0 + u * 256, rr = r_lo + (item >> 5), cg = item & 31;
+#pragma unroll
+                        for (int zz = 0; zz < kParts; ++zz) {
+                            ml[u][zz] = make_float2(-INFINITY, 0.f);
+                            v[u][zz] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (item < n_items && z0 + zz < n_parts) {
+                                ml[u][zz] = dsmem_ld2(dsmem_addr(lml + (uint32_t)rr * 8u, (uint32_t)(z0 + zz)));
+                                v[u][zz] = dsmem_ld4(dsmem_addr(lo + (uint32_t)rr * 512u + (uint32_t)((cg ^ (rr & 31)) << 4),
+                                                                (uint32_t)(z0 + zz)));
+                            }
+                        }
                     }
-                    const float inv = 1.f / lsum;
-                    const size_t base = ((size_t)(row0 + rr) * p.Hq + h) * kTile + 4 * lane;
-                    uint2 u;
-                    u.x = pack_bf16(acc.x * inv, acc.y * inv);
-                    u.y = pack_bf16(acc.z * inv, acc.w * inv);
-                    *reinterpret_cast<uint2*>(p.out + base) = u;
-                    if (p.tap) *reinterpret_cast<float4*>(p.tap + base) = make_float4(acc.x * inv, acc.y * inv, acc.z * inv, acc.w * inv);
+#pragma unroll
+                    for (int u = 0; u < kItems; ++u) {
+                        if (it0 + u * 256 >= n_items) continue;
+                        float mnew = mxx[u];
+#pragma unroll
+                        for (int zz = 0; zz < kParts; ++zz) mnew = fmaxf(mnew, ml[u][zz].x);
+                        const float keep = exp2f(mxx[u] - mnew);       // -inf on the first chunk gives 0
+                        mxx[u] = mnew;
+                        lsum[u] *= keep;
+                        acc[u].x *= keep; acc[u].y *= keep; acc[u].z *= keep; acc[u].w *= keep;
+#pragma unroll
+                        for (int zz = 0; zz < kParts; ++zz) {
+                            const float wgt = exp2f(ml[u][zz].x - mnew);   // absent parts: exp2(-inf) = 0
+                            lsum[u] += ml[u][zz].y * wgt;
+                            acc[u].x += v[u][zz].x * wgt; acc[u].y += v[u][zz].y * wgt;
+                            acc[u].z += v[u][zz].z * wgt; acc[u].w += v[u][zz].w * wgt;
+                        }
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < kItems; ++u) {
+                    const int item = it0 + u * 256, rr = r_lo + (item >> 5), cg = item & 31;
+                    if (item >= n_items) continue;
+                    const float inv = 1.f / lsum[u];
+                    const size_t base = ((size_t)(row0 + rr) * p.Hq + h) * kTile + 4 * cg;
+                    uint2 w2;
+                    w2.x = pack_bf16(acc[u].x * inv, acc[u].y * inv);
+                    w2.y = pack_bf16(acc[u].z * inv, acc[u].w * inv);
+                    *reinterpret_cast<uint2*>(p.out + base) = w2;
+                    if (p.tap)
+                        *reinterpret_cast<float4*>(p.tap + base) =
+                            make_float4(acc[u].x * inv, acc[u].y * inv, acc[u].z * inv, acc[u].w * inv);
                 }
             }
         }
+        cluster_sync_all();                                // no CTA leaves while its part may still be read
     }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
+    if (has_work) {
+        tc_fence_before();
+        __syncthreads();
+        if (warp == 1) {
+            tc_fence_after();
+            tmem_dealloc(tmem_base, kTmemCols);
+        }
     }
 }
 
@@ -405,8 +490,7 @@ wd_status wd_attn_tc_encode_cache(CUtensorMap* map_k, CUtensorMap* map_vt, const
 wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_t* qtile_seq, const int32_t* qtile_row0,
                             const int32_t* qtile_n, const int32_t* seq_nvis, const CUtensorMap* map_k,
                             const CUtensorMap* map_vt, void* out, float* tap, int Hq, int Hkv, int dh, int layer,
-                            int max_vis, int sm_count, float* scratch, int32_t* counters, int32_t* status,
-                            cudaStream_t stream) {
+                            int max_vis, int sm_count, int32_t* status, cudaStream_t stream) {
     if (dh != kTile) return WD_ERR_BAD_PARAM;
     if (n_tiles <= 0) return WD_OK;
     EncodeTiledFn enc = get_encode();
@@ -433,17 +517,14 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     p.scale_log2e = 1.4426950408889634f / sqrtf((float)dh);
     p.status = status;
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
-    // split the keys across CTAs while (tile, head) pairs alone would leave SMs idle
+    // split the keys across the CTAs of a cluster while (tile, head) pairs alone would leave SMs idle
     const int max_kt = (max_vis + kTile - 1) / kTile;
     int want = sm_count / (n_tiles * Hq);
-    if (want < 1 || !scratch || !counters || n_tiles * Hq > WD_ATTN_SPLIT_SLOTS / 2) want = 1;
+    if (want < 1) want = 1;
+    if (want > kMaxCluster) want = kMaxCluster;
     if (want > max_kt) want = max_kt;
     p.tiles_per_split = (max_kt + want - 1) / want;
     p.max_parts = (max_kt + p.tiles_per_split - 1) / p.tiles_per_split;
-    if ((long long)n_tiles * Hq * p.max_parts > WD_ATTN_SPLIT_SLOTS) { p.tiles_per_split = max_kt; p.max_parts = 1; }
-    p.part_o = scratch;
-    p.part_ml = scratch ? scratch + (size_t)WD_ATTN_SPLIT_SLOTS * kTile * kTile : nullptr;
-    p.counters = counters;
     const size_t smem = 6 * (size_t)kOperand + (kBars + 1) * 8 + 16 + 2 * kTile * 4 + 1024;
     static bool attr_done = false;      // one device per process
     if (!attr_done) {
@@ -455,11 +536,22 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     lc.blockDim = dim3(kThreads);
     lc.dynamicSmemBytes = smem;
     lc.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cudaLaunchAttribute attr[2];
+    int n_attr = 0;
+    if (p.max_parts > 1) {
+        attr[n_attr].id = cudaLaunchAttributeClusterDimension;
+        attr[n_attr].val.clusterDim.x = 1;
+        attr[n_attr].val.clusterDim.y = 1;
+        attr[n_attr].val.clusterDim.z = (unsigned)p.max_parts;
+        ++n_attr;
+    }
+    if (wd_pdl_enabled) {
+        attr[n_attr].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n_attr].val.programmaticStreamSerializationAllowed = 1;
+        ++n_attr;
+    }
     lc.attrs = attr;
-    lc.numAttrs = wd_pdl_enabled ? 1 : 0;
+    lc.numAttrs = n_attr;
     ++wd_launch_counter;
     WD_CUDA_TRY(cudaLaunchKernelEx(&lc, attention_tc_kernel, mq, *map_k, *map_vt, p));
     return WD_OK;

@@ -14,11 +14,5 @@ wd_status wd_attn_tc_encode_cache(CUtensorMap* map_k, CUtensorMap* map_vt, const
 wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_t* qtile_seq, const int32_t* qtile_row0,
                             const int32_t* qtile_n, const int32_t* seq_nvis, const CUtensorMap* map_k,
                             const CUtensorMap* map_vt, void* out, float* tap, int Hq, int Hkv, int dh, int layer,
-                            int max_vis, int sm_count, float* scratch, int32_t* counters, int32_t* status,
-                            cudaStream_t stream);
-
-// Scratch for the split over keys: WD_ATTN_SPLIT_SLOTS parts of [128 rows][128] floats plus
-// their (max, sum) pairs; counters: WD_ATTN_SPLIT_SLOTS zeroed ints.  max_vis = most visible
-// positions of any sequence.
-#define WD_ATTN_SPLIT_SLOTS 320
-static inline size_t wd_attn_tc_scratch_floats() { return (size_t)WD_ATTN_SPLIT_SLOTS * (128 * 128 + 128 * 2); }
+                            int max_vis, int sm_count, int32_t* status, cudaStream_t stream);
+// max_vis = most visible positions of any sequence (sizes the split of the keys over a cluster).
