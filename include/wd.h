@@ -300,6 +300,22 @@ WD_API wd_status wd_step_sync(wd_state* st, wd_step_out* out);
  * = steps completed. */
 WD_API wd_status wd_step_sync_all(wd_state* st, wd_step_out* outs, int32_t capacity, int32_t* n_steps);
 
+/* Whole-generation driver: the decoding loop of Section 4 (repeat windowed
+ * denoising steps, a refresh step opening every phase, until no masked position
+ * is left inside the reach of the window) run by the library.  Steps are enqueued
+ * back to back on `stream` and drained in groups, so the host only waits when
+ * the queue is full; a state that needs a host plan per step (see wd_step) is
+ * stepped and synchronised one step at a time instead.  Stops when wd_step
+ * reports WD_DONE (with adaptive termination: once the end-of-sequence token is
+ * out and nothing before it is masked) or after max_steps steps (max_steps <= 0:
+ * no limit).  On return the queue is empty and the host mirror is current
+ * (wd_state_read gives the tokens).  *n_steps (may be NULL) = steps run,
+ * *n_tokens (may be NULL) = tokens unmasked over all sequences.  Needs an empty
+ * queue (WD_ERR_PENDING).  Returns WD_DONE when generation finished, WD_OK when
+ * max_steps stopped it, else the first error of wd_step / wd_step_sync. */
+WD_API wd_status wd_generate(wd_state* st, int32_t A, int32_t B, int32_t R, int32_t T, int32_t k,
+                      int32_t max_steps, void* stream /*cudaStream_t*/, int32_t* n_steps, int32_t* n_tokens);
+
 /* ---- single operations (unit parity tests, micro-benchmarks) -------------- */
 
 /* y[rows, n_out] (float, device) = x[rows, k_in] * w[n_out, k_in]^T, x and w of

@@ -80,6 +80,7 @@ SIGNATURES = {
     "wd_step": (C.c_int, [vp, i32, i32, i32, i32, i32, vp, C.POINTER(wd_step_info)]),
     "wd_step_sync": (C.c_int, [vp, C.POINTER(wd_step_out)]),
     "wd_step_sync_all": (C.c_int, [vp, C.POINTER(wd_step_out), i32, i32p]),
+    "wd_generate": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32p, i32p]),
     "wd_op_gemm": (C.c_int, [i32, i32, vp, vp, vp, i32, i32, i32, vp, C.c_size_t, vp]),
     "wd_op_gemm_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
     "wd_op_gemm_noalloc": (C.c_int, [vp, vp, vp, i32, i32, i32, vp]),
@@ -302,6 +303,13 @@ class State:
         check(lib().wd_step_sync_all(self.handle, outs, max_steps, C.byref(done)), "wd_step_sync_all")
         return [dict(n_unmasked=n, positions=pos.reshape(self.batch, k), token_ids=tok.reshape(self.batch, k),
                      confidence=conf.reshape(self.batch, k)) for (n, pos, tok, conf) in bufs[: done.value]]
+
+    def generate(self, A: int, B: int, R: int, T: int, k: int, max_steps: int = 0, stream=None) -> tuple:
+        """wd_generate: run steps until done (or max_steps).  Returns (status, steps, tokens unmasked)."""
+        n_steps, n_tok = i32(), i32()
+        st = check(lib().wd_generate(self.handle, A, B, R, T, k, max_steps, _stream_ptr(stream), C.byref(n_steps),
+                                     C.byref(n_tok)), "wd_generate")
+        return st, n_steps.value, n_tok.value
 
     def close(self):
         if self.handle:

@@ -1019,6 +1019,45 @@ extern "C" wd_status wd_step_sync_all(wd_state* st, wd_step_out* outs, int32_t c
     return drain_queue(st, capacity > 0 ? outs : nullptr, true, n_steps);
 }
 
+extern "C" wd_status wd_generate(wd_state* st, int32_t A, int32_t B, int32_t R, int32_t T, int32_t k, int32_t max_steps,
+                                 void* stream, int32_t* n_steps, int32_t* n_tokens) {
+    if (!st) return WD_ERR_NULL;
+    if (!st->queue.empty()) return WD_ERR_PENDING;
+    if (n_steps) *n_steps = 0;
+    if (n_tokens) *n_tokens = 0;
+    int32_t steps = 0;
+    long long before = 0, after = 0;
+    for (const WdSeq& s : st->seqs)
+        for (uint8_t d : s.decoded) before += d;
+    wd_status result = WD_OK;
+    bool finished = false;
+    while (max_steps <= 0 || steps < max_steps) {
+        wd_step_info info;
+        wd_status s = wd_step(st, A, B, R, T, k, stream, &info);
+        if (s == WD_ERR_PENDING && !st->queue.empty()) {        // queue full, or one host-planned step in flight
+            if ((s = drain_queue(st, nullptr, true, nullptr)) != WD_OK) { result = s; break; }
+            continue;
+        }
+        if (s == WD_DONE) {
+            // the count shadow says nothing is left; with steps still in flight the mirror confirms it below
+            finished = true;
+            break;
+        }
+        if (s != WD_OK) { result = s; break; }
+        ++steps;
+    }
+    if (!st->queue.empty()) {
+        const wd_status s = drain_queue(st, nullptr, true, nullptr);
+        if (result == WD_OK && s != WD_OK) result = s;
+    }
+    for (const WdSeq& s : st->seqs)
+        for (uint8_t d : s.decoded) after += d;
+    if (n_steps) *n_steps = steps;
+    if (n_tokens) *n_tokens = (int32_t)(after - before);
+    if (result != WD_OK) return result;
+    return finished ? WD_DONE : WD_OK;
+}
+
 // ---------------------------------------------------------------------------
 // single operations
 // ---------------------------------------------------------------------------

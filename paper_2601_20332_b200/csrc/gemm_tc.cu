@@ -764,7 +764,8 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     long long wide_units = 0;
     for (int i = 0; i < nseg; ++i) wide_units += (segs[i].n + 2 * kBM - 1) / (2 * kBM);
     wide_units *= (rows + 255) / 256;
-    const TcConfig cfg = pick_config(rows, !fused && wide_units >= sm_count);
+    static const int wide_min_units = env_int("WD_GEMM_WIDE_MIN_UNITS", 0);     // tuning knob; 0 = one unit per SM
+    const TcConfig cfg = pick_config(rows, !fused && wide_units >= (wide_min_units > 0 ? wide_min_units : sm_count));
     p.wide = cfg.wide;
     p.tile_rows = cfg.tile_rows;
     int tiles = 0, col = 0;

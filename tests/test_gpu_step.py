@@ -240,6 +240,48 @@ def test_steps_enqueued_back_to_back_match_stepwise_sync(shape, batch):
     st.close(); ctx.close()
 
 
+@pytest.mark.parametrize("eos", [False, True])
+def test_generate_runs_the_whole_decoding_loop(eos):
+    """wd_generate = the same steps as a hand-written loop of wd_step + wd_step_sync: identical
+    final tokens, decode steps and counters (device-planned queue without adaptive termination,
+    host-planned one step at a time with it)."""
+    cfg = synth.get_config("llada8b", **DH128)
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    S = ids.shape[1]
+    A, B, R, T, k = (cfg[x] for x in ("A", "B", "R", "T", "k"))
+    ctx = wd.Context(cfg, w, 1, S, S, A)
+    finals = []
+    for use_generate in (False, True):
+        st = wd.State(ctx, ids)
+        if eos:
+            st.set_eos(3)
+        if use_generate:
+            status, n_steps, n_tok = st.generate(A, B, R, T, k)
+            assert status == wd.WD_DONE
+        else:
+            n_steps = n_tok = 0
+            while True:
+                status, _ = st.step(A, B, R, T, k)
+                if status == wd.WD_DONE:
+                    break
+                n_tok += int(st.sync()["n_unmasked"].sum())
+                n_steps += 1
+        finals.append((st.read(0), n_steps, n_tok))
+        st.close()
+    (ma, sa, ta), (mb, sb, tb) = finals
+    assert sa == sb and ta == tb and sa > 0
+    assert (ma["ids"] == mb["ids"]).all() and (ma["decoded"] == mb["decoded"]).all()
+    assert (ma["dec_step"] == mb["dec_step"]).all() and ma["t"] == mb["t"] == sa
+    if not eos:
+        assert ma["decoded"].all() and ta == cfg["G"]
+    # max_steps stops early with WD_OK and leaves a consistent state
+    st = wd.State(ctx, ids)
+    status, n_steps, n_tok = st.generate(A, B, R, T, k, max_steps=5)
+    assert status == wd.WD_OK and n_steps == 5 and n_tok == 5 * k and st.read(0)["t"] == 5
+    st.close(); ctx.close()
+
+
 def test_non_prefix_state_needs_a_sync_between_steps():
     cfg = synth.get_config("llada8b", **SMALL_BF16)
     w = synth.make_weights(cfg, DEV)
