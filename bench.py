@@ -200,6 +200,14 @@ def run_ours(args, rank, world):
         state.sync()
     torch.cuda.synchronize()
     e2e_wall = time.perf_counter() - t0
+    # ---- a whole generation through the library's own driver: host prompt in, host tokens out
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    state.reset(ids, None, stream)
+    _, gen_steps, gen_tokens = state.generate(A, B, R, T, k, 0, stream)
+    final_ids = [state.read(b)["ids"] for b in range(batch)]
+    gen_wall = time.perf_counter() - t0
+    assert gen_tokens == batch * cfg["G"] and all((f != cfg["mask_id"]).all() for f in final_ids)
     # ---- the full-sequence no-pruning step at the same starting state, for context
     state.reset(ids, None, stream)
     full_ms = []
@@ -250,6 +258,9 @@ def run_ours(args, rank, world):
                    "samples": clocks["samples"]},
         "e2e": {"value": batch * k * (W + K) * world / e2e_wall, "unit": UNIT,
                 "stepping": "one wd_step + wd_step_sync per step (every step's tokens reach the host before the next)",
+                "whole_generation": {"value": gen_tokens * world / gen_wall, "unit": UNIT, "steps": gen_steps,
+                                     "tokens": gen_tokens, "seconds": gen_wall,
+                                     "call": "wd_state_reset + wd_generate + wd_state_read on the host clock"},
                 "h2d_bytes_per_step": float(batch * S * 5 / (W + K)),
                 "d2h_bytes_per_step": float((1 + batch + 3 * batch * k) * 4)},
         "gpu_launches": int(sum(i["n_launches"] for i in infos)),

@@ -314,7 +314,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     uint32_t* tmem_slot = (uint32_t*)(bars + 2 * NS + 4);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     int* last_flag = (int*)(tmem_slot + 2);
-    float* lm_scratch = (float*)(tmem_slot + 4);           // 1.5 KB for the LM-head statistics
+    float* lm_scratch = (float*)(tmem_slot + 4);           // 23 KB for the LM-head statistics
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const long long c = blockIdx.x, G = gridDim.x;
@@ -484,84 +484,85 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             tc_fence_after();
             float* yb = p.y + p.seg_col[u.seg] + n;
             const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf + half_sel) * p.buf_cols);
-            constexpr bool lm_stats = kLmStats;
-            const bool store_y = !lm_stats || p.f.write_logits;
-            for (int cc = 0; cc < p.bn; cc += 16) {
-                if (u.tok0 + cc >= p.rows) break;
-                uint32_t v[16];
-                tmem_ld16(t_acc + (uint32_t)cc, v);
-                if (n_ok && store_y) {
-                    float* ys = yb + (size_t)ord * p.split_stride;
+            if constexpr (!kLmStats) {
+                for (int cc = 0; cc < p.bn; cc += 16) {
+                    if (u.tok0 + cc >= p.rows) break;
+                    uint32_t v[16];
+                    tmem_ld16(t_acc + (uint32_t)cc, v);
+                    if (n_ok) {
+                        float* ys = yb + (size_t)ord * p.split_stride;
 #pragma unroll
-                    for (int t = 0; t < 16; ++t) {
-                        const int tok = u.tok0 + cc + t;
-                        if (tok < p.rows) ys[(size_t)tok * p.ncol] = __uint_as_float(v[t]);
+                        for (int t = 0; t < 16; ++t) {
+                            const int tok = u.tok0 + cc + t;
+                            if (tok < p.rows) ys[(size_t)tok * p.ncol] = __uint_as_float(v[t]);
+                        }
                     }
                 }
-                if (lm_stats) {
-                    // per token: maximum / lowest argmax / sum exp over this tile's 128 logits.
-                    // Thread = one vocabulary entry; warp shuffles, then the 4 warps through shared memory.
-                    float* sh_m = lm_scratch;                       // [4][16]
-                    int* sh_i = (int*)(lm_scratch + 64);            // [4][16]
-                    double* sh_s = (double*)(lm_scratch + 128);     // [4][16]
-                    float* sh_tm = lm_scratch + 256;                // [16] tile maxima
-                    int* sh_ti = (int*)(lm_scratch + 272);          // [16] their indices
-                    float* run_m = lm_scratch + 288;                // [256] running statistics of this CTA
-                    int* run_i = (int*)(lm_scratch + 544);
-                    double* run_s = (double*)(lm_scratch + 800);
+            } else {
+                // LM head: per token maximum / lowest argmax / sum exp over this tile's 128 logits, folded
+                // into the CTA's running statistics.  A thread holds one vocabulary entry for 32 tokens;
+                // the chunk is transposed through shared memory so that a thread then owns one token and
+                // a quarter of the tile's vocabulary entries, and the four quarters are merged per token.
+                float* run_m = lm_scratch;                          // [256] running statistics of this CTA
+                int* run_i = (int*)(lm_scratch + 256);
+                double* run_s = (double*)(lm_scratch + 512);
+                float* g_m = lm_scratch + 1024;                     // [4 quarters][32 tokens]
+                int* g_i = (int*)(lm_scratch + 1152);
+                double* g_s = (double*)(lm_scratch + 1280);
+                float* tr = lm_scratch + 1536;                      // [32 tokens][129]: padded against bank conflicts
+                const int e = (int)threadIdx.x - 64, tt = e & 31, gq = e >> 5;
+                for (int cc = 0; cc < p.bn; cc += 32) {
+                    if (cc >= p.rows) break;
+                    uint32_t v[32];
+                    tmem_ld32(t_acc + (uint32_t)cc, v);
+                    if (n_ok && p.f.write_logits) {
 #pragma unroll
-                    for (int t = 0; t < 16; ++t) {
-                        float bm = n_ok ? __uint_as_float(v[t]) : -INFINITY;
-                        int bi = n_ok ? n : 0x7fffffff;
+                        for (int t = 0; t < 32; ++t)
+                            if (cc + t < p.rows) yb[(size_t)(cc + t) * p.ncol] = __uint_as_float(v[t]);
+                    }
 #pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) {
-                            const float om = __shfl_xor_sync(0xffffffffu, bm, o);
-                            const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
-                            if (om > bm || (om == bm && oi < bi)) { bm = om; bi = oi; }
+                    for (int t = 0; t < 32; ++t) tr[t * 129 + n_local] = n_ok ? __uint_as_float(v[t]) : -INFINITY;
+                    epi_sync();
+                    float x[32];
+                    float bm = -INFINITY;
+                    int bj = 0;
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        x[j] = tr[tt * 129 + 32 * gq + j];
+                        if (x[j] > bm) { bm = x[j]; bj = j; }       // strict: the lowest index stays on ties
+                    }
+                    // single-precision exp (1 ulp) of each term, double accumulation: sums good to ~1e-9
+                    double sm = 0.0;
+                    if (bm > -INFINITY) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) sm += (double)expf(x[j] - bm);
+                    }
+                    g_m[gq * 32 + tt] = bm;
+                    g_i[gq * 32 + tt] = u.n0 + 32 * gq + bj;
+                    g_s[gq * 32 + tt] = sm;
+                    epi_sync();
+                    if (e < 32 && cc + e < p.rows) {
+                        // quarters ascend in vocabulary index, and so do the tiles of a CTA: on equal
+                        // maxima the earlier index stays
+                        float tm = g_m[e];
+                        int ti = g_i[e];
+                        for (int w = 1; w < 4; ++w)
+                            if (g_m[w * 32 + e] > tm) { tm = g_m[w * 32 + e]; ti = g_i[w * 32 + e]; }
+                        double ts = 0.0;
+                        for (int w = 0; w < 4; ++w)
+                            if (g_m[w * 32 + e] > -INFINITY) ts += g_s[w * 32 + e] * exp((double)g_m[w * 32 + e] - (double)tm);
+                        const int tl = cc + e;
+                        if (piece == 0) {
+                            run_m[tl] = tm; run_i[tl] = ti; run_s[tl] = ts;
+                        } else if (tm > run_m[tl]) {
+                            run_s[tl] = run_s[tl] * exp((double)run_m[tl] - (double)tm) + ts;
+                            run_m[tl] = tm; run_i[tl] = ti;
+                        } else {
+                            run_s[tl] += ts * exp((double)tm - (double)run_m[tl]);
                         }
-                        if (lane == 0) { sh_m[quarter * 16 + t] = bm; sh_i[quarter * 16 + t] = bi; }
                     }
-                    epi_sync();
-                    const int e = (int)threadIdx.x - 64;
-                    if (e < 16) {
-                        float bm = sh_m[e];
-                        int bi = sh_i[e];
-                        for (int w = 1; w < 4; ++w) {
-                            const float om = sh_m[w * 16 + e];
-                            const int oi = sh_i[w * 16 + e];
-                            if (om > bm || (om == bm && oi < bi)) { bm = om; bi = oi; }
-                        }
-                        sh_tm[e] = bm;
-                        sh_ti[e] = bi;
-                    }
-                    epi_sync();
-#pragma unroll
-                    for (int t = 0; t < 16; ++t) {
-                        // single-precision exp (1 ulp), double accumulation: the tile sum is good to ~1e-9
-                        double ex = n_ok ? (double)expf(__uint_as_float(v[t]) - sh_tm[t]) : 0.0;
-#pragma unroll
-                        for (int o = 16; o > 0; o >>= 1) ex += __shfl_xor_sync(0xffffffffu, ex, o);
-                        if (lane == 0) sh_s[quarter * 16 + t] = ex;
-                    }
-                    epi_sync();
-                    if (e < 16) {
-                        // fold this tile into the CTA's running statistics of the token (tiles ascend in
-                        // vocabulary index, so on equal maxima the earlier index stays)
-                        const int tl = cc + e;                       // token within the (single) token tile
-                        if (u.tok0 + tl < p.rows) {
-                            const double ts = sh_s[e] + sh_s[16 + e] + sh_s[32 + e] + sh_s[48 + e];
-                            const float tm = sh_tm[e];
-                            if (piece == 0) {
-                                run_m[tl] = tm; run_i[tl] = sh_ti[e]; run_s[tl] = ts;
-                            } else if (tm > run_m[tl]) {
-                                run_s[tl] = run_s[tl] * exp((double)run_m[tl] - (double)tm) + ts;
-                                run_m[tl] = tm; run_i[tl] = sh_ti[e];
-                            } else {
-                                run_s[tl] += ts * exp((double)tm - (double)run_m[tl]);
-                            }
-                        }
-                    }
-                    epi_sync();
+                    // the next chunk's writes to the transpose tile and to the quarter statistics come
+                    // after its own barrier, which every thread reaches only after the reads above
                 }
             }
             tc_fence_before();
@@ -605,9 +606,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         }
         if (kLmStats && sch.n_pieces > 0) {
             // one (max, argmax, sum exp) per token for all the vocabulary tiles this CTA covered
-            float* run_m = lm_scratch + 288;
-            int* run_i = (int*)(lm_scratch + 544);
-            double* run_s = (double*)(lm_scratch + 800);
+            float* run_m = lm_scratch;
+            int* run_i = (int*)(lm_scratch + 256);
+            double* run_s = (double*)(lm_scratch + 512);
             epi_sync();
             for (int t = (int)threadIdx.x - 64; t < p.rows; t += 128) {
                 const size_t si = (size_t)t * G + c;
@@ -678,7 +679,7 @@ int env_int(const char* name, int dflt) {
     return v && *v ? atoi(v) : dflt;
 }
 
-TcConfig pick_config(int rows, bool allow_wide) {
+TcConfig pick_config(int rows, bool allow_wide, bool lm_stats) {
     TcConfig c;
     // Many tokens: the GEMM is bound by operand traffic from L2 into shared memory, so a CTA
     // carries two 128-row weight halves that share every activation box ([256 x BN] per CTA).
@@ -697,7 +698,7 @@ TcConfig pick_config(int rows, bool allow_wide) {
     c.n_stages = ((c.ctas_per_sm == 2 ? 96 : 192) * 1024) / stage;
     if (c.n_stages > 10) c.n_stages = 10;
     if (c.n_stages < 2) c.n_stages = 2;
-    c.smem = (size_t)c.n_stages * stage + (2 * c.n_stages + 4) * 8 + 16 + 8192 + 1024;
+    c.smem = (size_t)c.n_stages * stage + (2 * c.n_stages + 4) * 8 + 16 + (lm_stats ? 24576 : 8192) + 1024;
     return c;
 }
 
@@ -765,7 +766,8 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     for (int i = 0; i < nseg; ++i) wide_units += (segs[i].n + 2 * kBM - 1) / (2 * kBM);
     wide_units *= (rows + 255) / 256;
     static const int wide_min_units = env_int("WD_GEMM_WIDE_MIN_UNITS", 0);     // tuning knob; 0 = one unit per SM
-    const TcConfig cfg = pick_config(rows, !fused && wide_units >= (wide_min_units > 0 ? wide_min_units : sm_count));
+    const TcConfig cfg = pick_config(rows, !fused && wide_units >= (wide_min_units > 0 ? wide_min_units : sm_count),
+                                     fuse && fuse->mode == WD_FUSE_LMSTATS);
     p.wide = cfg.wide;
     p.tile_rows = cfg.tile_rows;
     int tiles = 0, col = 0;
