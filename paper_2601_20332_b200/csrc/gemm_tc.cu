@@ -626,6 +626,225 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
 }
 
+// Two-CTA variant for many tokens (compute-bound shapes).  The CTA pair of a cluster works on one
+// [256 weight rows x BN tokens] tile with tcgen05.mma.cta_group::2: each CTA loads its own 128 weight
+// rows and HALF of the token rows of every K block (the tensor cores of both SMs read both halves),
+// so the operand traffic per flop into shared memory is two thirds of the one-CTA [128 x BN] tile's,
+// while the ring keeps its depth and both accumulators stay double-buffered.  Same persistent
+// stream-K schedule, same output layout; the pair is the scheduling unit (c = pair index).
+//   even CTA: expects the bytes of both CTAs on its "full" barriers (the odd CTA's TMA loads count
+//             on them through .cta_group::2), issues every MMA, releases the stages and publishes the
+//             accumulators in BOTH CTAs (tcgen05.commit with a CTA mask)
+//   both:     TMA producer for their own operand halves, epilogue for their own 128 weight rows;
+//             epilogue threads of both CTAs arrive on the even CTA's "accumulator empty" barriers
+__global__ void __launch_bounds__(kThreads)
+gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w0,
+                    const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2,
+                    const TcParams p) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int NS = p.n_stages;
+    const int half_bn = p.bn >> 1;                        // token rows this CTA loads per K block
+    const int stage_a = kStageA;                          // 16 KB: this CTA's 128 weight rows
+    const int stage_bytes = stage_a + half_bn * kBK * 2;
+    uint64_t* bars = (uint64_t*)(smem + (size_t)NS * stage_bytes);
+    // bars[0..NS) full (used in the even CTA) | [NS..2NS) empty | [2NS, 2NS+1] accumulator full |
+    // [2NS+2, 2NS+3] accumulator empty (used in the even CTA, 256 arrivals)
+    uint32_t* tmem_slot = (uint32_t*)(bars + 2 * NS + 4);
+    volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();              // 0: issues the MMAs
+    const long long c = blockIdx.x >> 1, G = gridDim.x >> 1;
+    long long g_begin, g_end;
+    if (p.aligned) {
+        g_begin = (c * p.n_units / G) * p.kb_total;
+        g_end = ((c + 1) * p.n_units / G) * p.kb_total;
+    } else {
+        g_begin = c * p.W / G;
+        g_end = (c + 1) * p.W / G;
+    }
+    const int n_total = (int)(g_end - g_begin);
+    Sched sch;
+    sch.init(g_begin, g_end, p.kb_total);
+
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(smem_u32(&bars[s]), 1);
+            mbar_init(smem_u32(&bars[NS + s]), 1);
+        }
+        mbar_init(smem_u32(&bars[2 * NS]), 1);
+        mbar_init(smem_u32(&bars[2 * NS + 1]), 1);
+        mbar_init(smem_u32(&bars[2 * NS + 2]), 256);
+        mbar_init(smem_u32(&bars[2 * NS + 3]), 256);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w0) : "memory");
+    }
+    if (warp == 1) tmem2_alloc(smem_u32(tmem_slot), 2u * (uint32_t)p.buf_cols);   // the same warp in both CTAs
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync();               // the peer's barriers exist before anything signals them
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0 && n_total > 0) {
+            // ------------------------------------------------ TMA producer (both CTAs, own halves)
+            uint64_t pol_stream;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            struct Walk {
+                int piece, left, kb, n0, tok0;
+                const CUtensorMap* mw;
+            };
+            auto enter = [&](Walk& w) {
+                long long g;
+                int len;
+                sch.piece(w.piece, g, len);
+                const int unit = (int)(g / p.kb_total);
+                w.kb = (int)(g - (long long)unit * p.kb_total);
+                w.left = len;
+                const UnitInfo u = decode_unit(p, unit);
+                w.n0 = u.n0 + (int)rank * kBM;
+                w.tok0 = u.tok0 + (int)rank * half_bn;
+                w.mw = u.seg == 0 ? &map_w0 : (u.seg == 1 ? &map_w1 : &map_w2);
+            };
+            auto advance = [&](Walk& w) {
+                ++w.kb;
+                if (--w.left == 0 && ++w.piece < sch.n_pieces) enter(w);
+            };
+            Walk w0;
+            w0.piece = 0;
+            enter(w0);
+            const int n_pre = n_total < NS ? n_total : NS;
+            Walk w = w0;
+            for (int i = 0; i < n_pre; ++i, advance(w)) {
+                if (rank == 0) mbar_expect_tx(smem_u32(&bars[i]), 2u * (uint32_t)stage_bytes);
+                tma2_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes), w.mw, cluster_map(smem_u32(&bars[i]), 0),
+                                  w.kb * kBK, w.n0, pol_stream);
+            }
+            pdl_wait();
+            Walk wx = w0;
+            for (int i = 0; i < n_pre; ++i, advance(wx))
+                tma2_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + stage_a, &map_x,
+                             cluster_map(smem_u32(&bars[i]), 0), wx.kb * kBK, wx.tok0);
+            int s = n_pre % NS;
+            uint32_t ph = (uint32_t)(n_pre / NS) & 1u;
+            for (int i = n_pre; i < n_total; ++i, advance(w)) {
+                if (!mbar_wait(smem_u32(&bars[NS + s]), ph ^ 1u, abort_flag)) {
+                    *abort_flag = 1;
+                    atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
+                    break;
+                }
+                const uint32_t full = cluster_map(smem_u32(&bars[s]), 0);
+                const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+                if (rank == 0) mbar_expect_tx(smem_u32(&bars[s]), 2u * (uint32_t)stage_bytes);
+                tma2_load_2d_hint(sa, w.mw, full, w.kb * kBK, w.n0, pol_stream);
+                tma2_load_2d(sa + stage_a, &map_x, full, w.kb * kBK, w.tok0);
+                if (++s == NS) { s = 0; ph ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0 && rank == 0) {
+            // ------------------------------------------------ MMA issuer (even CTA only)
+            bool ok = true;
+            int s = 0;
+            uint32_t ph = 0;
+            for (int piece = 0; piece < sch.n_pieces && ok; ++piece) {
+                long long g;
+                int len;
+                sch.piece(piece, g, len);
+                const int buf = piece & 1;
+                const uint32_t par = (uint32_t)(piece >> 1) & 1u;
+                // the epilogues of both CTAs have drained this accumulator (free at the start)
+                if (!(ok = mbar_wait(smem_u32(&bars[2 * NS + 2 + buf]), par ^ 1u, abort_flag))) break;
+                tc_fence_after();
+                const uint32_t acc = tmem_base + (uint32_t)(buf * p.buf_cols);
+                for (int j = 0; j < len; ++j) {
+                    if (!(ok = mbar_wait(smem_u32(&bars[s]), ph, abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+                    const uint64_t adesc = make_sdesc(sa);
+                    const uint64_t bdesc = make_sdesc(sa + stage_a);
+#pragma unroll
+                    for (int kk = 0; kk < kBK / 16; ++kk)
+                        umma2_bf16(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
+                                   (j > 0 || kk > 0) ? 1u : 0u);
+                    umma2_commit_mc(smem_u32(&bars[NS + s]), 3);          // stage free in both CTAs
+                    if (++s == NS) { s = 0; ph ^= 1u; }
+                }
+                if (ok) umma2_commit_mc(smem_u32(&bars[2 * NS + buf]), 3);  // accumulator complete in both CTAs
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------------------------------------------- epilogue (warps 2..5 of both CTAs)
+        const int quarter = warp & 3;
+        const int n_local = (int)rank * kBM + quarter * 32 + lane;
+        pdl_wait();
+        bool ok = true;
+        for (int piece = 0; piece < sch.n_pieces; ++piece) {
+            long long g;
+            int len;
+            sch.piece(piece, g, len);
+            const int unit = (int)(g / p.kb_total), kb0 = (int)(g - (long long)unit * p.kb_total);
+            const UnitInfo u = decode_unit(p, unit);
+            const int buf = piece & 1;
+            const uint32_t par = (uint32_t)(piece >> 1) & 1u;
+            const int n = u.n0 + n_local;
+            const bool n_ok = n < p.seg_n[u.seg];
+            int ord = 0;
+            if (!p.aligned) ord = (int)(c - (((long long)unit * p.kb_total + 1) * G - 1) / p.W);
+            ok = ok && mbar_wait(smem_u32(&bars[2 * NS + buf]), par, abort_flag);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            float* yb = p.y + p.seg_col[u.seg] + n;
+            const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.buf_cols);
+            for (int cc = 0; cc < p.bn; cc += 16) {
+                if (u.tok0 + cc >= p.rows) break;
+                uint32_t v[16];
+                tmem_ld16(t_acc + (uint32_t)cc, v);
+                if (n_ok) {
+                    float* ys = yb + (size_t)ord * p.split_stride;
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) {
+                        const int tok = u.tok0 + cc + t;
+                        if (tok < p.rows) ys[(size_t)tok * p.ncol] = __uint_as_float(v[t]);
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive_cluster(cluster_map(smem_u32(&bars[2 * NS + 2 + buf]), 0));   // accumulator may be overwritten
+            if (kb0 + len == p.kb_total && n_ok) {
+                // this pair finished the tile: slices nobody wrote must read as zero
+                for (int sl = ord + 1; sl < p.n_slices; ++sl) {
+                    float* ys = yb + (size_t)sl * p.split_stride;
+                    for (int tok = u.tok0; tok < u.tok0 + p.bn && tok < p.rows; ++tok) ys[(size_t)tok * p.ncol] = 0.f;
+                }
+            }
+        }
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    cluster_sync();               // neither CTA frees tensor memory or leaves while the other may still signal it
+    if (warp == 1) {
+        tc_fence_after();
+        tmem2_dealloc(tmem_base, 2u * (uint32_t)p.buf_cols);
+    }
+}
+
 // y = sum of split-K slices
 __global__ void reduce_slices_kernel(const float* __restrict__ part, int n_split, size_t stride, float* __restrict__ y,
                                      size_t total) {
@@ -713,15 +932,107 @@ int count_slices(int n_units, int kb_total, long long W, long long G) {
     return n;
 }
 
-uint32_t make_idesc(int bn) {
+uint32_t make_idesc(int bn, int m = kBM) {
     uint32_t d = 0;
     d |= 1u << 4;                      // D format: f32
     d |= 1u << 7;                      // A format: bf16
     d |= 1u << 10;                     // B format: bf16
     // bits 15 / 16: A and B are K-major (0)
     d |= (uint32_t)(bn >> 3) << 17;    // N
-    d |= (uint32_t)(kBM >> 4) << 24;   // M
+    d |= (uint32_t)(m >> 4) << 24;     // M (256: the two-CTA form)
     return d;
+}
+
+// launch of gemm_tc_pair_kernel: same contract as wd_tc_gemm
+wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, int K, float* y, size_t y_floats,
+                       int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out, bool force_single_split) {
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.tile_rows = 2 * kBM;
+    p.tok_tiles = (rows + 255) / 256;
+    p.bn = ((rows + p.tok_tiles - 1) / p.tok_tiles + 15) / 16 * 16;        // balanced token tiles, <= 256
+    int cols = 32;
+    while (cols < p.bn) cols <<= 1;
+    p.buf_cols = cols;
+    const int half_bn = p.bn / 2;
+    const int stage = kStageA + half_bn * kBK * 2;
+    p.n_stages = (192 * 1024) / stage;
+    if (p.n_stages > 10) p.n_stages = 10;
+    const size_t smem = (size_t)p.n_stages * stage + (2 * p.n_stages + 4) * 8 + 16 + 256 + 1024;
+    int tiles = 0, col = 0;
+    for (int i = 0; i < nseg; ++i) {
+        if (!segs[i].map) return WD_ERR_NULL;
+        p.seg_tile0[i] = tiles;
+        p.seg_n[i] = segs[i].n;
+        p.seg_col[i] = col;
+        tiles += (segs[i].n + p.tile_rows - 1) / p.tile_rows;
+        col += segs[i].n;
+    }
+    p.seg_tile0[nseg] = tiles;
+    p.nseg = nseg;
+    p.ncol = col;
+    p.rows = rows;
+    p.kb_total = (K + kBK - 1) / kBK;
+    p.n_units = tiles * p.tok_tiles;
+    p.W = (long long)p.n_units * p.kb_total;
+    const size_t slice = (size_t)rows * col;
+    if (slice > y_floats) return WD_ERR_CAPACITY;
+    long long G = sm_count / 2;                                            // CTA pairs
+    if (G > p.W / 2) G = p.W / 2 > 0 ? p.W / 2 : 1;
+    int n_slices = count_slices(p.n_units, p.kb_total, p.W, G);
+    p.aligned = 0;
+    // With several whole tiles per pair the imbalance of whole-tile scheduling is small, and one
+    // slice instead of two or three saves the consumers (and the zero fill) most of their traffic.
+    static const int aligned_from = env_int("WD_GEMM_ALIGNED_UNITS", 2);
+    if (force_single_split || (size_t)n_slices * slice > y_floats || n_slices > WD_TC_MAX_SPLIT ||
+        p.n_units >= aligned_from * G) {
+        p.aligned = 1;
+        n_slices = 1;
+        G = sm_count / 2;
+        if (G > p.n_units) G = p.n_units;
+    }
+    p.n_slices = n_slices;
+    p.y = y;
+    p.split_stride = slice;
+    p.status = status;
+    p.idesc = make_idesc(p.bn, 2 * kBM);
+
+    CUtensorMap mx;
+    bool hit = false;
+    for (const WdTcX::Entry& e : x->cache)
+        if (e.rows == rows && e.bn == half_bn) { mx = e.map; hit = true; break; }
+    if (!hit) {
+        wd_status s = encode_2d(&mx, x->ptr, rows, K, half_bn);
+        if (s != WD_OK) return s;
+        if (x->cache.size() >= 16) x->cache.erase(x->cache.begin());
+        x->cache.push_back({rows, half_bn, mx});
+    }
+    static bool attr_done = false;      // one device per process
+    if (!attr_done) {
+        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        attr_done = true;
+    }
+    const CUtensorMap& m0 = *segs[0].map;
+    const CUtensorMap& m1 = *segs[nseg > 1 ? 1 : 0].map;
+    const CUtensorMap& m2 = *segs[nseg > 2 ? 2 : 0].map;
+    ++wd_launch_counter;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)(2 * G));
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = smem;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = wd_pdl_enabled ? 2 : 1;
+    WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_pair_kernel, mx, m0, m1, m2, p));
+    if (n_split_out) *n_split_out = p.n_slices;
+    return WD_OK;
 }
 
 }  // namespace
@@ -760,6 +1071,10 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     TcParams p;
     memset(&p, 0, sizeof(p));
     const bool fused = fuse && fuse->mode != WD_FUSE_NONE;
+    // Many tokens: CTA pairs on [256 x BN] tiles (tcgen05 cta_group::2)
+    static const int pair_from = env_int("WD_GEMM_PAIR_FROM", 512);        // rows from which pairs are used; 0 = never
+    if (!fused && pair_from > 0 && rows >= pair_from && sm_count >= 2)
+        return tc_gemm_pair(x, segs, nseg, rows, K, y, y_floats, sm_count, status, stream, n_split_out, force_single_split);
     // The wide tile halves the operand traffic per flop but has a shallower ring and an epilogue
     // that does not overlap the next tile: it pays once every CTA gets at least one whole tile.
     long long wide_units = 0;

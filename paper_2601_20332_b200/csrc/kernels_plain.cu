@@ -403,7 +403,8 @@ __global__ void gemm_plain_kernel(const T* __restrict__ x, const T* __restrict__
 // table, writes q and the K/V cache rows.  K cache [batch][Hkv][S][dh]; V cache transposed
 // [batch][Hkv][dh][Sp] so that attention can read V tiles with the key position contiguous.
 // One 1-D grid, two kinds of 256-thread blocks:
-//   blocks [0, n_qk):  (row, group of 4 q/k heads), one rotation pair per thread
+//   blocks [0, n_qk):  (row, group of q/k heads), four rotation pairs per thread (one pair and
+//                      groups of 4 heads when head_dim / 2 is not a multiple of 4)
 //   blocks [n_qk, ..): (v head, 32 head dims, 32 rows): slices summed with the dims contiguous,
 //                      transposed through shared memory and written with the rows (normally
 //                      consecutive positions) contiguous, so neighbouring lanes share sectors
@@ -419,9 +420,27 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
     const int half = dh >> 1;
     const int ncol = (Hq + 2 * Hkv) * dh;
     if ((int)blockIdx.x < n_qk) {
-        const int r = blockIdx.x / qk_groups, h0 = (blockIdx.x - r * qk_groups) * 4;
+        const int r = blockIdx.x / qk_groups, grp = blockIdx.x - r * qk_groups;
         const int pos = row_pos[r], b = row_seq[r];
         const float* pr = part + (size_t)r * ncol;
+        if ((half & 3) == 0) {
+            // four rotation pairs per thread (float4 loads, 8-byte bf16 stores): half/4 threads per head
+            const int tph = half >> 2, hpb = blockDim.x / tph;
+            const int h = grp * hpb + (int)threadIdx.x / tph, j = ((int)threadIdx.x % tph) * 4;
+            if ((int)threadIdx.x < hpb * tph && h < Hq + Hkv) {
+                const float4 a = sum_slices4(pr + h * dh + j, n_split, split_stride);
+                const float4 bb = sum_slices4(pr + h * dh + half + j, n_split, split_stride);
+                const float4 c01 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j);       // (cos, sin) x 2
+                const float4 c23 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j + 2);
+                T* dst = h < Hq ? q + ((size_t)r * Hq + h) * dh : kcache + (((size_t)b * Hkv + (h - Hq)) * S + pos) * dh;
+                Vec4<T>::store(dst + j, a.x * c01.x - bb.x * c01.y, a.y * c01.z - bb.y * c01.w, a.z * c23.x - bb.z * c23.y,
+                               a.w * c23.z - bb.w * c23.w);
+                Vec4<T>::store(dst + j + half, bb.x * c01.x + a.x * c01.y, bb.y * c01.z + a.y * c01.w,
+                               bb.z * c23.x + a.z * c23.y, bb.w * c23.z + a.w * c23.w);
+            }
+            return;
+        }
+        const int h0 = grp * 4;
         for (int i = threadIdx.x; i < 4 * half; i += blockDim.x) {
             const int h = h0 + i / half, j = i % half;
             if (h >= Hq + Hkv) break;
@@ -441,10 +460,18 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
     const int d0 = (rem / rchunks) * 32, r0 = (rem % rchunks) * 32;
     const int lx = threadIdx.x & 31, ly = threadIdx.x >> 5;
     const int vcol = (Hq + Hkv) * dh + kh * dh + d0;
-    for (int rr = ly; rr < 32; rr += 8) {
-        const int r = r0 + rr;
-        tile[rr][lx] = (r < n_rows && d0 + lx < dh)
-            ? sum_slices1(part + (size_t)r * ncol + vcol + lx, n_split, split_stride) : 0.f;
+    if ((dh & 3) == 0) {
+        // one float4 (four head dims of one row) per thread
+        const int rr = threadIdx.x >> 3, d4 = (threadIdx.x & 7) * 4, r = r0 + rr;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (r < n_rows && d0 + d4 < dh) v = sum_slices4(part + (size_t)r * ncol + vcol + d4, n_split, split_stride);
+        tile[rr][d4] = v.x; tile[rr][d4 + 1] = v.y; tile[rr][d4 + 2] = v.z; tile[rr][d4 + 3] = v.w;
+    } else {
+        for (int rr = ly; rr < 32; rr += 8) {
+            const int r = r0 + rr;
+            tile[rr][lx] = (r < n_rows && d0 + lx < dh)
+                ? sum_slices1(part + (size_t)r * ncol + vcol + lx, n_split, split_stride) : 0.f;
+        }
     }
     __syncthreads();
     const int r = r0 + lx;
@@ -523,26 +550,53 @@ __global__ void swiglu_kernel(const float* __restrict__ part, int n_split, size_
     pdl_launch_dependents();
     pdl_wait();
     const int f4 = F >> 2;
-    const size_t total = (size_t)n_rows * f4;
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-         i += (size_t)gridDim.x * blockDim.x) {
-        const size_t r = i / f4, c4 = i - r * f4;
-        const float4 g = sum_slices4(part + r * 2 * F + 4 * c4, n_split, split_stride);
-        const float4 u = sum_slices4(part + r * 2 * F + F + 4 * c4, n_split, split_stride);
-        Vec4<T>::store(h + r * F + 4 * c4, g.x / (1.f + __expf(-g.x)) * u.x, g.y / (1.f + __expf(-g.y)) * u.y,
-                       g.z / (1.f + __expf(-g.z)) * u.z, g.w / (1.f + __expf(-g.w)) * u.w);
+    const size_t total = (size_t)n_rows * f4, stride = (size_t)gridDim.x * blockDim.x;
+    // two positions per iteration so that four (or more) loads are in flight per thread
+    for (size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < total; i0 += 2 * stride) {
+        const size_t i1 = i0 + stride;
+        const bool has1 = i1 < total;
+        const size_t ra = i0 / f4, ca = i0 - ra * f4, rb = has1 ? i1 / f4 : ra, cb = has1 ? i1 - rb * f4 : ca;
+        const float* pa = part + ra * 2 * F + 4 * ca;
+        const float* pb = part + rb * 2 * F + 4 * cb;
+        float4 ga, ua, gb, ub;
+        if (n_split == 1) {
+            ga = *reinterpret_cast<const float4*>(pa);
+            ua = *reinterpret_cast<const float4*>(pa + F);
+            gb = *reinterpret_cast<const float4*>(pb);
+            ub = *reinterpret_cast<const float4*>(pb + F);
+        } else {
+            ga = sum_slices4(pa, n_split, split_stride);
+            ua = sum_slices4(pa + F, n_split, split_stride);
+            gb = sum_slices4(pb, n_split, split_stride);
+            ub = sum_slices4(pb + F, n_split, split_stride);
+        }
+        Vec4<T>::store(h + ra * F + 4 * ca, ga.x / (1.f + __expf(-ga.x)) * ua.x, ga.y / (1.f + __expf(-ga.y)) * ua.y,
+                       ga.z / (1.f + __expf(-ga.z)) * ua.z, ga.w / (1.f + __expf(-ga.w)) * ua.w);
+        if (has1)
+            Vec4<T>::store(h + rb * F + 4 * cb, gb.x / (1.f + __expf(-gb.x)) * ub.x, gb.y / (1.f + __expf(-gb.y)) * ub.y,
+                           gb.z / (1.f + __expf(-gb.z)) * ub.z, gb.w / (1.f + __expf(-gb.w)) * ub.w);
     }
 }
 
+// total is a multiple of 4 (d is)
 __global__ void residual_add_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
                                     size_t split_stride, float* __restrict__ tap, size_t total) {
     pdl_launch_dependents();
     pdl_wait();
-    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total;
-         i += (size_t)gridDim.x * blockDim.x) {
-        const float v = x[i] + sum_slices1(part + i, n_split, split_stride);
-        x[i] = v;
-        if (tap) tap[i] = v;
+    const size_t n4 = total >> 2, stride = (size_t)gridDim.x * blockDim.x;
+    for (size_t i0 = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i0 < n4; i0 += 2 * stride) {
+        const size_t i1 = i0 + stride < n4 ? i0 + stride : i0;
+        float4 xa = reinterpret_cast<const float4*>(x)[i0], xb = reinterpret_cast<const float4*>(x)[i1];
+        const float4 pa = sum_slices4(part + 4 * i0, n_split, split_stride);
+        const float4 pb = sum_slices4(part + 4 * i1, n_split, split_stride);
+        xa.x += pa.x; xa.y += pa.y; xa.z += pa.z; xa.w += pa.w;
+        reinterpret_cast<float4*>(x)[i0] = xa;
+        if (tap) reinterpret_cast<float4*>(tap)[i0] = xa;
+        if (i1 != i0) {
+            xb.x += pb.x; xb.y += pb.y; xb.z += pb.z; xb.w += pb.w;
+            reinterpret_cast<float4*>(x)[i1] = xb;
+            if (tap) reinterpret_cast<float4*>(tap)[i1] = xb;
+        }
     }
 }
 
@@ -712,7 +766,12 @@ void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size
     // one float4 per thread where the row allows it: the kernel is a chain of dependent L2 round
     // trips, so short per-thread work matters more than occupancy
     const int nv = d >> 2;
-    if (nv <= 1024) {
+    if (n_rows >= 512 && nv >= 256 && nv <= 4096) {
+        // many rows: bandwidth matters, so more (smaller) blocks per SM with four float4 in flight per thread
+        const int threads = ((nv + 3) / 4 + 31) / 32 * 32;
+        WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 4>, dim3(n_rows), dim3(threads), 0, st, x, part, n_split,
+                                      split_stride, gain, eps, (T*)xn, row_idx, d));
+    } else if (nv <= 1024) {
         const int threads = (nv + 31) / 32 * 32;
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 1>, dim3(n_rows), dim3(threads), 0, st, x, part, n_split,
                                       split_stride, gain, eps, (T*)xn, row_idx, d));
@@ -738,7 +797,8 @@ void wd_launch_rope_scatter(int dtype, const float* part, int n_split, size_t sp
                             void* kcache, void* vcache, int n_rows, int Hq, int Hkv, int dh, int S, int Sp,
                             cudaStream_t st) {
     if (n_rows <= 0) return;
-    const int qk_groups = wd_ceil_div(Hq + Hkv, 4);
+    const int half = dh >> 1;
+    const int qk_groups = (half & 3) == 0 ? wd_ceil_div(Hq + Hkv, std::max(1, 256 / (half >> 2))) : wd_ceil_div(Hq + Hkv, 4);
     const int n_qk = n_rows * qk_groups;
     const int n_v = Hkv * wd_ceil_div(dh, 32) * wd_ceil_div(n_rows, 32);
     WD_DISPATCH(dtype, launch_pdl(rope_scatter_kernel<T>, dim3(n_qk + n_v), dim3(256), 0, st, part, n_split,
@@ -779,8 +839,8 @@ void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_st
 void wd_launch_residual_add(float* x, const float* part, int n_split, size_t split_stride,
                             float* tap, int n_rows, int d, cudaStream_t st) {
     if (n_rows <= 0) return;
-    const size_t total = (size_t)n_rows * d;
-    const int blocks = (int)((total + 255) / 256 < 148 * 8 ? (total + 255) / 256 : 148 * 8);
+    const size_t total = (size_t)n_rows * d, n4 = total >> 2;
+    const int blocks = (int)((n4 + 255) / 256 < 148 * 8 ? (n4 + 255) / 256 : 148 * 8);
     launch_pdl(residual_add_kernel, dim3(blocks), dim3(256), 0, st, x, part, n_split, split_stride, tap, total);
 }
 
