@@ -39,6 +39,10 @@ struct TcParams {
     int rows, bn, kb_total, tok_tiles, n_units, n_stages, buf_cols, n_slices, aligned;
     int wide;                       // 1: a tile is 256 weight rows = two MMA halves sharing each activation box
     int tile_rows;                  // 128, or 256 when wide
+    // > 1: the grid is tok_split groups of CTAs, group t working on token tile t only; the K-block
+    // line then holds the weight tiles once (n_units, W count weight tiles), and the groups walk it
+    // in step, so that a weight block fetched for one token tile is still in L2 for the others
+    int tok_split;
     int nseg, ncol;
     int seg_tile0[4];               // first tile index of each weight matrix (+ end)
     int seg_n[3];
@@ -53,10 +57,10 @@ struct TcParams {
 
 // A unit is one [128 weight rows x BN tokens] output tile; unit u = tile * tok_tiles + token tile.
 struct UnitInfo { int seg, n0, tok0; };
-__device__ __forceinline__ UnitInfo decode_unit(const TcParams& p, int unit) {
+__device__ __forceinline__ UnitInfo decode_unit(const TcParams& p, int unit, int tok_group = 0) {
     UnitInfo u;
-    const int tile = unit / p.tok_tiles;
-    u.tok0 = (unit - tile * p.tok_tiles) * p.bn;
+    const int tile = p.tok_split > 1 ? unit : unit / p.tok_tiles;
+    u.tok0 = p.tok_split > 1 ? tok_group * p.bn : (unit - tile * p.tok_tiles) * p.bn;
     u.seg = 0;
     if (p.nseg > 1 && tile >= p.seg_tile0[1]) u.seg = 1;
     if (p.nseg > 2 && tile >= p.seg_tile0[2]) u.seg = 2;
@@ -317,7 +321,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     float* lm_scratch = (float*)(tmem_slot + 4);           // 23 KB for the LM-head statistics
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const long long c = blockIdx.x, G = gridDim.x;
+    const long long G = gridDim.x / (p.tok_split > 1 ? p.tok_split : 1), c = blockIdx.x % G;
+    const int tok_group = (int)(blockIdx.x / G);
     long long g_begin, g_end;
     if (p.aligned) {
         g_begin = (c * p.n_units / G) * p.kb_total;
@@ -368,7 +373,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const int unit = (int)(g / p.kb_total);
                 w.kb = (int)(g - (long long)unit * p.kb_total);
                 w.left = len;
-                const UnitInfo u = decode_unit(p, unit);
+                const UnitInfo u = decode_unit(p, unit, tok_group);
                 w.n0 = u.n0;
                 w.tok0 = u.tok0;
                 w.mw = u.seg == 0 ? &map_w0 : (u.seg == 1 ? &map_w1 : &map_w2);
@@ -471,7 +476,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             int len;
             sch.piece(piece, g, len);
             const int unit = (int)(g / p.kb_total), kb0 = (int)(g - (long long)unit * p.kb_total);
-            const UnitInfo u = decode_unit(p, unit);
+            const UnitInfo u = decode_unit(p, unit, tok_group);
             const int buf = kWide ? 0 : (piece & 1);
             const uint32_t par = kWide ? ((uint32_t)piece & 1u) : ((uint32_t)(piece >> 1) & 1u);
             const int n = u.n0 + n_local;
@@ -1073,7 +1078,7 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     const bool fused = fuse && fuse->mode != WD_FUSE_NONE;
     // Many tokens: CTA pairs on [256 x BN] tiles (tcgen05 cta_group::2)
     static const int pair_from = env_int("WD_GEMM_PAIR_FROM", 512);        // rows from which pairs are used; 0 = never
-    if (!fused && pair_from > 0 && rows >= pair_from && sm_count >= 2)
+    if (!fused && pair_from > 0 && rows > pair_from && sm_count >= 2)
         return tc_gemm_pair(x, segs, nseg, rows, K, y, y_floats, sm_count, status, stream, n_split_out, force_single_split);
     // The wide tile halves the operand traffic per flop but has a shallower ring and an epilogue
     // that does not overlap the next tile: it pays once every CTA gets at least one whole tile.
@@ -1100,21 +1105,29 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     p.rows = rows; p.bn = cfg.bn;
     p.kb_total = (K + kBK - 1) / kBK;
     p.tok_tiles = cfg.tok_tiles;
-    p.n_units = tiles * cfg.tok_tiles;
+    // Two or four token tiles: one group of CTAs per token tile, all groups walking the same line of
+    // weight K blocks in step, so a weight block comes from HBM once and from L2 for the other groups
+    // (with one line over (weight tile, token tile) units the second visit came a whole pass later,
+    // after the block had left the L2: DRAM traffic was twice the weight bytes)
+    const int slots = sm_count * cfg.ctas_per_sm;
+    const int ts = (!fused && !cfg.wide && (cfg.tok_tiles == 2 || cfg.tok_tiles == 4) && slots % cfg.tok_tiles == 0) ? cfg.tok_tiles : 1;
+    p.tok_split = ts;
+    p.n_units = ts > 1 ? tiles : tiles * cfg.tok_tiles;
     p.W = (long long)p.n_units * p.kb_total;
     p.n_stages = cfg.n_stages;
     p.buf_cols = cfg.buf_cols;
     const size_t slice = (size_t)rows * col;
     if (slice > y_floats) return WD_ERR_CAPACITY;
     // stream-K over all SMs when the partial sums fit, whole tiles per CTA otherwise
-    long long G = (long long)sm_count * cfg.ctas_per_sm;
+    // (G = CTAs per token group)
+    long long G = (long long)slots / ts;
     if (G > p.W / 2) G = p.W / 2 > 0 ? p.W / 2 : 1;           // at least two K blocks per CTA
     int n_slices = count_slices(p.n_units, p.kb_total, p.W, G);
     p.aligned = 0;
     if (force_single_split || (size_t)n_slices * slice > y_floats || n_slices > WD_TC_MAX_SPLIT) {
         p.aligned = 1;
         n_slices = 1;
-        G = (long long)sm_count * cfg.ctas_per_sm;
+        G = (long long)slots / ts;
         if (G > p.n_units) G = p.n_units;
     }
     p.n_slices = n_slices;
@@ -1155,7 +1168,7 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     const CUtensorMap& m2 = *segs[nseg > 2 ? 2 : 0].map;
     ++wd_launch_counter;
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3((unsigned)G);
+    lc.gridDim = dim3((unsigned)(G * ts));
     lc.blockDim = dim3(cfg.wide ? kThreadsWide : kThreads);
     lc.dynamicSmemBytes = cfg.smem;
     lc.stream = stream;
