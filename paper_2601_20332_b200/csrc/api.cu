@@ -901,7 +901,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         fl.mode = WD_FUSE_LMSTATS;
         fl.st_max = c->ch_max; fl.st_idx = c->ch_idx; fl.st_sum = c->ch_sum;
         fl.write_logits = st->taps.logits ? 1 : 0;
-        lm_fused = use_tc(c) && NA <= 256;
+        lm_fused = use_tc(c) && NA <= 1024 && c->sm_count % 4 == 0;     // one CTA group per tile of <= 256 active rows
         if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, lm, 1, NA, D, c->logits, (size_t)d.max_active * d.vocab, status,
                           stream, &go, /*single_split=*/true, lm_fused ? &fl : nullptr)) != WD_OK)
             return s;

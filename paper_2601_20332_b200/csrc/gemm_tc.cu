@@ -517,13 +517,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 float* tr = lm_scratch + 1536;                      // [32 tokens][129]: padded against bank conflicts
                 const int e = (int)threadIdx.x - 64, tt = e & 31, gq = e >> 5;
                 for (int cc = 0; cc < p.bn; cc += 32) {
-                    if (cc >= p.rows) break;
+                    if (u.tok0 + cc >= p.rows) break;
                     uint32_t v[32];
                     tmem_ld32(t_acc + (uint32_t)cc, v);
                     if (n_ok && p.f.write_logits) {
 #pragma unroll
                         for (int t = 0; t < 32; ++t)
-                            if (cc + t < p.rows) yb[(size_t)(cc + t) * p.ncol] = __uint_as_float(v[t]);
+                            if (u.tok0 + cc + t < p.rows) yb[(size_t)(u.tok0 + cc + t) * p.ncol] = __uint_as_float(v[t]);
                     }
 #pragma unroll
                     for (int t = 0; t < 32; ++t) tr[t * 129 + n_local] = n_ok ? __uint_as_float(v[t]) : -INFINITY;
@@ -546,7 +546,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     g_i[gq * 32 + tt] = u.n0 + 32 * gq + bj;
                     g_s[gq * 32 + tt] = sm;
                     epi_sync();
-                    if (e < 32 && cc + e < p.rows) {
+                    if (e < 32 && u.tok0 + cc + e < p.rows) {
                         // quarters ascend in vocabulary index, and so do the tiles of a CTA: on equal
                         // maxima the earlier index stays
                         float tm = g_m[e];
@@ -615,8 +615,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             int* run_i = (int*)(lm_scratch + 256);
             double* run_s = (double*)(lm_scratch + 512);
             epi_sync();
-            for (int t = (int)threadIdx.x - 64; t < p.rows; t += 128) {
-                const size_t si = (size_t)t * G + c;
+            // this CTA's token tile: rows tok_group * bn .. ; entry c of the row's G statistics
+            for (int t = (int)threadIdx.x - 64; t < p.bn && tok_group * p.bn + t < p.rows; t += 128) {
+                const size_t si = (size_t)(tok_group * p.bn + t) * G + c;
                 p.f.st_max[si] = run_m[t];
                 p.f.st_idx[si] = run_i[t];
                 p.f.st_sum[si] = run_s[t];
@@ -912,6 +913,7 @@ TcConfig pick_config(int rows, bool allow_wide, bool lm_stats) {
     c.tile_rows = c.wide ? 2 * kBM : kBM;
     static const int bn_max = env_int("WD_GEMM_BN_MAX", 256);      // tuning knob (multiple of 16, <= 256)
     c.tok_tiles = (rows + bn_max - 1) / bn_max;
+    if (lm_stats && c.tok_tiles == 3) c.tok_tiles = 4;             // the LM head takes one CTA group per token tile
     c.bn = ((rows + c.tok_tiles - 1) / c.tok_tiles + 15) / 16 * 16;     // balanced token tiles, <= 256
     int cols = 32;
     while (cols < c.bn) cols <<= 1;
@@ -1110,7 +1112,9 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     // (with one line over (weight tile, token tile) units the second visit came a whole pass later,
     // after the block had left the L2: DRAM traffic was twice the weight bytes)
     const int slots = sm_count * cfg.ctas_per_sm;
-    const int ts = (!fused && !cfg.wide && (cfg.tok_tiles == 2 || cfg.tok_tiles == 4) && slots % cfg.tok_tiles == 0) ? cfg.tok_tiles : 1;
+    const bool lm = fuse && fuse->mode == WD_FUSE_LMSTATS;
+    const int ts = ((!fused || lm) && !cfg.wide && (cfg.tok_tiles == 2 || cfg.tok_tiles == 4) && slots % cfg.tok_tiles == 0)
+                       ? cfg.tok_tiles : 1;
     p.tok_split = ts;
     p.n_units = ts > 1 ? tiles : tiles * cfg.tok_tiles;
     p.W = (long long)p.n_units * p.kb_total;
@@ -1138,7 +1142,7 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     if (fuse) {
         p.f = *fuse;
         if (fuse->mode != WD_FUSE_NONE && fuse->mode != WD_FUSE_LMSTATS && !fuse->counters) return WD_ERR_NULL;
-        if (fuse->mode == WD_FUSE_LMSTATS && (!p.aligned || cfg.wide || cfg.tok_tiles != 1 || nseg != 1 || !fuse->st_max ||
+        if (fuse->mode == WD_FUSE_LMSTATS && (!p.aligned || cfg.wide || cfg.tok_tiles != ts || nseg != 1 || !fuse->st_max ||
                                               !fuse->st_idx || !fuse->st_sum))
             return WD_ERR_BAD_PARAM;
         fuse->n_chunks = (int)G;          // one statistics entry per (row, CTA)

@@ -81,6 +81,16 @@ def test_bf16_head_dim_128_tensor_core_attention(Hkv, batch, fusion):
     assert logs[0]["info"]["n_rows"] == batch * 256
 
 
+@pytest.mark.parametrize("batch,A", [(2, 160), (4, 150), (4, 250)])
+def test_lm_head_statistics_with_several_token_tiles(batch, A):
+    """More than 256 active rows: the LM-head epilogue runs one CTA group per token tile (two
+    tiles at 320 rows, three rounded up to four at 600, four at 1000); logits, per-row
+    statistics and the unmask choice stay exact for every row."""
+    cfg = synth.get_config("llada8b", **dict(DH128, L=1, P=30, G=260, A=A, B=8, R=2, T=1, k=3, batch=batch))
+    logs = run(cfg, 3, oracle_seqs=[0, batch - 1])
+    assert logs[0]["info"]["n_active"] == batch * A
+
+
 def test_plain_and_tensor_core_paths_agree():
     """The CUDA-core kernels and the tensor-core kernels compute the same step."""
     cfg = synth.get_config("llada8b", **DH128)
