@@ -108,6 +108,21 @@ def algorithmic_step(cfg, rows, n_act, vis, batch=1):
     return by, fl
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """A multi-rank run is as slow as its slowest rank: all-reduce MAX of the device-timed region
+    (NCCL between GPUs; the CPU tests run the same code over gloo)."""
+    if world <= 1:
+        return float(ms)
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(units_per_rank: float, world: int, total_ms: float) -> float:
+    """Replicas only: every rank processes the same number of units, no data-path collective."""
+    return units_per_rank * world / (total_ms * 1e-3)
+
+
 def run_ours(args, rank, world):
     from paper_2601_20332_b200 import binding as wd
     from paper_2601_20332_b200 import build as wd_build
@@ -221,12 +236,8 @@ def run_ours(args, rank, world):
         full_ms.append(e0.elapsed_time(e1))
     state.close()
 
-    t_total = torch.tensor([total_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        torch.distributed.all_reduce(t_total, op=torch.distributed.ReduceOp.MAX)
-    total_ms = float(t_total.item())
-    tokens = batch * k * K * world
-    value = tokens / (total_ms * 1e-3)
+    total_ms = max_over_ranks(total_ms, world, dev)
+    value = whole_job_value(batch * k * K, world, total_ms)
     normal = [t for t, i in zip(per_step, infos) if not i["is_refresh"]]
     refresh = [t for t, i in zip(per_step, infos) if i["is_refresh"]]
     # roofline of the GEMM kernel: algorithmic bytes per launch / average launch time
