@@ -661,7 +661,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();              // 0: issues the MMAs
-    const long long c = blockIdx.x >> 1, G = gridDim.x >> 1;
+    // pairs per token group, this pair's index in its group, its token group (see TcParams::tok_split)
+    const long long G = (gridDim.x >> 1) / (p.tok_split > 1 ? p.tok_split : 1), c = (blockIdx.x >> 1) % G;
+    const int tok_group = (int)((blockIdx.x >> 1) / G);
     long long g_begin, g_end;
     if (p.aligned) {
         g_begin = (c * p.n_units / G) * p.kb_total;
@@ -712,7 +714,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 const int unit = (int)(g / p.kb_total);
                 w.kb = (int)(g - (long long)unit * p.kb_total);
                 w.left = len;
-                const UnitInfo u = decode_unit(p, unit);
+                const UnitInfo u = decode_unit(p, unit, tok_group);
                 w.n0 = u.n0 + (int)rank * kBM;
                 w.tok0 = u.tok0 + (int)rank * half_bn;
                 w.mw = u.seg == 0 ? &map_w0 : (u.seg == 1 ? &map_w1 : &map_w2);
@@ -801,7 +803,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
             int len;
             sch.piece(piece, g, len);
             const int unit = (int)(g / p.kb_total), kb0 = (int)(g - (long long)unit * p.kb_total);
-            const UnitInfo u = decode_unit(p, unit);
+            const UnitInfo u = decode_unit(p, unit, tok_group);
             const int buf = piece & 1;
             const uint32_t par = (uint32_t)(piece >> 1) & 1u;
             const int n = u.n0 + n_local;
@@ -980,11 +982,14 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     p.ncol = col;
     p.rows = rows;
     p.kb_total = (K + kBK - 1) / kBK;
-    p.n_units = tiles * p.tok_tiles;
+    // two token tiles: one group of pairs per token tile, walking the weight K blocks in step
+    const int ts = (p.tok_tiles == 2 && (sm_count / 2) % 2 == 0) ? 2 : 1;
+    p.tok_split = ts;
+    p.n_units = ts > 1 ? tiles : tiles * p.tok_tiles;
     p.W = (long long)p.n_units * p.kb_total;
     const size_t slice = (size_t)rows * col;
     if (slice > y_floats) return WD_ERR_CAPACITY;
-    long long G = sm_count / 2;                                            // CTA pairs
+    long long G = sm_count / 2 / ts;                                       // CTA pairs (per token group)
     if (G > p.W / 2) G = p.W / 2 > 0 ? p.W / 2 : 1;
     int n_slices = count_slices(p.n_units, p.kb_total, p.W, G);
     p.aligned = 0;
@@ -995,7 +1000,7 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
         p.n_units >= aligned_from * G) {
         p.aligned = 1;
         n_slices = 1;
-        G = sm_count / 2;
+        G = sm_count / 2 / ts;
         if (G > p.n_units) G = p.n_units;
     }
     p.n_slices = n_slices;
@@ -1024,7 +1029,7 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     const CUtensorMap& m2 = *segs[nseg > 2 ? 2 : 0].map;
     ++wd_launch_counter;
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3((unsigned)(2 * G));
+    lc.gridDim = dim3((unsigned)(2 * G * ts));
     lc.blockDim = dim3(kThreads);
     lc.dynamicSmemBytes = smem;
     lc.stream = stream;
@@ -1079,7 +1084,7 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     memset(&p, 0, sizeof(p));
     const bool fused = fuse && fuse->mode != WD_FUSE_NONE;
     // Many tokens: CTA pairs on [256 x BN] tiles (tcgen05 cta_group::2)
-    static const int pair_from = env_int("WD_GEMM_PAIR_FROM", 512);        // rows from which pairs are used; 0 = never
+    static const int pair_from = env_int("WD_GEMM_PAIR_FROM", 256);        // rows from which pairs are used; 0 = never
     if (!fused && pair_from > 0 && rows > pair_from && sm_count >= 2)
         return tc_gemm_pair(x, segs, nseg, rows, K, y, y_floats, sm_count, status, stream, n_split_out, force_single_split);
     // The wide tile halves the operand traffic per flop but has a shallower ring and an epilogue
