@@ -59,6 +59,7 @@ class SeqState:
     phase_start: int = 0
     wex: list = field(default_factory=list)   # external window of the current phase
     eos_id: int = None                    # adaptive termination (Section 4.2), None = off
+    refresh_mode: int = 0                 # 0: the paper's refresh (Section 4.3); 1: window-only variant (see oracle_plan)
 
     def __post_init__(self):
         self.ids = np.array(self.ids, dtype=np.int64)
@@ -75,6 +76,12 @@ def oracle_plan(st: SeqState, A: int, B: int, R: int, T: int) -> dict:
     what is still undecoded inside it; buffer = external \\ (active ∪ decoded in
     phase); undecoded tokens outside the external window are far-field.
     Section 4.3: a phase is one refresh step followed by normal steps.
+
+    ``st.refresh_mode == 1`` selects a VARIANT that is not in the paper (Section 4.3 recomputes
+    everything visible at a refresh): from the second phase on, a refresh step computes only the
+    new external window and the tokens decoded during the phase that just ended; every other
+    visible position (prompt, tokens of earlier phases) keeps the K/V it already has in the
+    cache.  The first step of a state always computes everything (nothing is cached yet).
     """
     if A < 1 or B < 0 or R < 1 or T < 0:
         raise ValueError("bad window parameters")
@@ -111,7 +118,14 @@ def oracle_plan(st: SeqState, A: int, B: int, R: int, T: int) -> dict:
     far = [i for i in undecoded_all if i not in live]
     dec = [i for i in range(S) if st.decoded[i]]
     vis = sorted(set(dec) | set(W))
-    rows = list(vis) if refresh else sorted(set(act) | set(trans))
+    if not refresh:
+        rows = sorted(set(act) | set(trans))
+    elif st.refresh_mode == 1 and st.t > 0:
+        # st.phase_start is still the start of the phase that just ended
+        prev = [i for i in dec if st.dec_step[i] != NEVER and st.dec_step[i] >= st.phase_start]
+        rows = sorted(set(W) | set(prev))
+    else:
+        rows = list(vis)
     return dict(done=False, refresh=refresh, wex=wex, phase_start=phase_start,
                 active=act, buffer=buf, in_phase_decoded=dp, transient=trans,
                 far_field=far, decoded=dec, vis=vis, rows=rows)

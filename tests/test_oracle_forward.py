@@ -358,3 +358,55 @@ def test_teacher_forcing_and_tiny_config_runs():
     assert o["logits"].shape == (8, 1024)
     c = o["unmask"]["conf"]
     assert (c > 1.0 / 1024).all() and (c < 0.1).all()      # random init: near-uniform but not degenerate
+
+
+# ---------------------------------------------------------------- window-only refresh (variant, not in the paper)
+
+def _variant_traj(cfg, model, mode, n_steps):
+    states = fresh_states(cfg)
+    for st in states:
+        st.refresh_mode = mode
+    return run_traj(cfg, model, n_steps, states=states)
+
+
+def test_window_refresh_is_exact_for_a_one_layer_model():
+    """With ONE block the K/V of a position depend only on its token and its position, so keeping
+    the cached K/V of positions whose token did not change is the same as recomputing them: the
+    variant must reproduce the paper's refresh to rounding, step after step."""
+    cfg = small_cfg(L=1, G=24, T=2, R=3, k=2)
+    model = make(cfg)
+    full, _, cf = _variant_traj(cfg, model, 0, 9)
+    win, _, cw = _variant_traj(cfg, model, 1, 9)
+    n_fewer = 0
+    for f, w in zip(full, win):
+        f, w = f[0], w[0]
+        assert f["plan"]["refresh"] == w["plan"]["refresh"]
+        n_fewer += len(w["plan"]["rows"]) < len(f["plan"]["rows"])
+        np.testing.assert_allclose(w["logits"], f["logits"], rtol=1e-10, atol=1e-10)
+        assert w["committed"] == f["committed"]
+    assert n_fewer >= 2                                     # the later refreshes really computed fewer rows
+    vis = full[-1][0]["plan"]["vis"]
+    np.testing.assert_allclose(cw[0].K[:, vis], cf[0].K[:, vis], rtol=1e-10, atol=1e-10)
+    np.testing.assert_allclose(cw[0].V[:, vis], cf[0].V[:, vis], rtol=1e-10, atol=1e-10)
+
+
+def test_window_refresh_is_an_approximation_for_deeper_models():
+    """From the second block on, K/V depend on the context, so stale prefix entries change the
+    result: the variant must differ from the paper's refresh (it is not a no-op) while the first
+    layer's cache and the first phase stay identical."""
+    cfg = small_cfg(L=2, G=24, T=2, R=3, k=2)
+    model = make(cfg)
+    forced = []
+    full, _, cf = _variant_traj(cfg, model, 0, 4)
+    for o in full:
+        forced.append([o[0]["committed"]])
+    states = fresh_states(cfg)
+    states[0].refresh_mode = 1
+    win, _, cw = run_traj(cfg, model, 4, states=states, forced_seq=forced)
+    for s in range(3):                                      # first phase: the same steps
+        np.testing.assert_allclose(win[s][0]["logits"], full[s][0]["logits"], rtol=1e-10, atol=1e-10)
+    assert win[3][0]["plan"]["refresh"] and len(win[3][0]["plan"]["rows"]) < len(full[3][0]["plan"]["rows"])
+    assert np.abs(win[3][0]["logits"] - full[3][0]["logits"]).max() > 1e-6
+    assert np.isfinite(win[3][0]["logits"]).all()
+    vis = full[3][0]["plan"]["vis"]
+    np.testing.assert_allclose(cw[0].K[0][vis], cf[0].K[0][vis], rtol=1e-10, atol=1e-10)   # layer 0: context-free

@@ -220,3 +220,48 @@ def test_adaptive_termination_ignores_given_eos_and_takes_the_first_in_position_
     assert pl["active"] == list(range(2, 10))
     assert set(pl["far_field"]) == set(range(11, 20)) | set(range(21, 32))
     assert 20 in pl["vis"] and 10 in pl["vis"]                 # decoded tokens stay visible context
+
+
+# ---------------------------------------------------------------------------
+# window-only refresh (a variant outside the paper, flagged by SeqState.refresh_mode)
+# ---------------------------------------------------------------------------
+
+def _walk(mode, S=96, P=20, A=6, B=10, R=4, T=2, k=2, steps=30, seed=3):
+    rng = np.random.default_rng(seed)
+    ids = np.where(np.arange(S) < P, 5, 99)
+    st = SeqState(ids=ids, decoded=np.arange(S) < P, refresh_mode=mode)
+    trace = []
+    for _ in range(steps):
+        pl = oracle_plan(st, A, B, R, T)
+        if pl["done"]:
+            break
+        trace.append(pl)
+        chosen = sorted(rng.choice(pl["active"], size=min(k, len(pl["active"])), replace=False).tolist())
+        oracle_commit(st, pl, chosen, [7] * len(chosen))
+    return trace
+
+
+def test_window_refresh_rows_are_the_new_window_plus_the_previous_phase():
+    full, win = _walk(0), _walk(1)
+    assert len(full) == len(win) and sum(p["refresh"] for p in win) >= 4
+    for i, (f, w) in enumerate(zip(full, win)):
+        # the variant changes which rows a refresh computes and nothing else
+        for key in ("refresh", "wex", "active", "buffer", "transient", "far_field", "decoded", "vis"):
+            assert f[key] == w[key]
+        assert f["rows"] == (f["vis"] if f["refresh"] else sorted(set(f["active"]) | set(f["transient"])))
+        if not w["refresh"]:
+            assert w["rows"] == f["rows"]
+        elif i == 0:
+            assert w["rows"] == w["vis"]                                    # nothing cached yet: everything
+        else:
+            # decoded during the phase that just ended = difference of the decoded sets at the two refreshes
+            j = max(q for q in range(i) if win[q]["refresh"])
+            decoded_in_prev_phase = set(w["decoded"]) - set(win[j]["decoded"])
+            assert decoded_in_prev_phase
+            assert w["rows"] == sorted(set(w["wex"]) | decoded_in_prev_phase)
+            assert set(w["rows"]) < set(f["rows"])                          # strictly fewer rows than the paper's refresh
+
+
+def test_window_refresh_first_step_is_a_full_refresh():
+    w = _walk(1, steps=1)[0]
+    assert w["refresh"] and w["rows"] == w["vis"]
