@@ -67,6 +67,15 @@ enum {
 
 enum { WD_F32 = 0, WD_BF16 = 1 };     /* element type of weights, activations, K/V cache */
 
+/* What a refresh step computes (wd_state_set_refresh_mode, wd_plan_raw). */
+enum {
+    WD_REFRESH_FULL = 0,              /* every visible position: Section 4.3 of the paper           */
+    WD_REFRESH_WINDOW = 1             /* variant, NOT in the paper: only the new external window and
+                                         the tokens decoded during the phase that just ended; older
+                                         context keeps its cached K/V.  Exact for one block, an
+                                         approximation beyond.  The first step is always full.   */
+};
+
 /* GEMM implementation selector (wd_set_gemm_impl, wd_op_gemm). */
 enum {
     WD_GEMM_AUTO = 0,                 /* tensor-core kernel for bf16, plain for f32 */
@@ -238,6 +247,10 @@ WD_API wd_status wd_debug_taps_set(wd_state* st, const wd_debug_taps* taps /*NUL
  * eos_id < 0 switches it off (the default; the paper's main results also run with a fixed
  * length).  Kept across wd_state_reset.  Errors: WD_ERR_NULL, WD_ERR_PENDING, WD_ERR_BAD_PARAM. */
 WD_API wd_status wd_state_set_eos(wd_state* st, int32_t eos_id);
+/* What the refresh steps of this state compute: WD_REFRESH_FULL (default, the paper's refresh)
+ * or WD_REFRESH_WINDOW (the variant described at the enum; no counterpart in the paper).
+ * Kept across wd_state_reset.  Errors: WD_ERR_NULL, WD_ERR_PENDING, WD_ERR_BAD_PARAM. */
+WD_API wd_status wd_state_set_refresh_mode(wd_state* st, int32_t mode);
 
 /* ---- the step ----------------------------------------------------------- */
 
@@ -258,12 +271,12 @@ WD_API wd_status wd_plan(const wd_state* st, int32_t seq, int32_t A, int32_t B, 
  * eos_id for adaptive termination (see wd_state_set_eos; token_ids may be NULL
  * when eos_id < 0), step_index t, steps_since_refresh, and the external window
  * stored at the last refresh (ext_window[n_ext_window], ascending; empty before
- * the first step).
+ * the first step), and refresh_mode (WD_REFRESH_FULL or WD_REFRESH_WINDOW).
  * Errors: as wd_plan, plus WD_ERR_BAD_PARAM for an index outside the sequence. */
 WD_API wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, const int32_t* token_ids,
                              int32_t eos_id, int32_t seq_len, int32_t step_index,
                              int32_t steps_since_refresh, const int32_t* ext_window, int32_t n_ext_window,
-                             int32_t A, int32_t B, int32_t R, int32_t T, wd_index_sets* out);
+                             int32_t A, int32_t B, int32_t R, int32_t T, int32_t refresh_mode, wd_index_sets* out);
 
 /* Enqueue one step for every sequence of the state on `stream` and return
  * without waiting.  k = tokens unmasked per sequence (at most the number of

@@ -487,6 +487,15 @@ extern "C" wd_status wd_state_set_eos(wd_state* st, int32_t eos_id) {
     return WD_OK;
 }
 
+extern "C" wd_status wd_state_set_refresh_mode(wd_state* st, int32_t mode) {
+    if (!st) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    if (mode != WD_REFRESH_FULL && mode != WD_REFRESH_WINDOW) return WD_ERR_BAD_PARAM;
+    for (WdSeq& s : st->seqs) s.refresh_mode = mode;
+    for (WdCount& c : st->counts) c.refresh_mode = mode;
+    return WD_OK;
+}
+
 extern "C" wd_status wd_debug_taps_set(wd_state* st, const wd_debug_taps* taps) {
     if (!st) return WD_ERR_NULL;
     if (st->pending) return WD_ERR_PENDING;
@@ -524,10 +533,11 @@ extern "C" wd_status wd_plan(const wd_state* st, int32_t seq, int32_t A, int32_t
 extern "C" wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, const int32_t* token_ids,
                                  int32_t eos_id, int32_t seq_len, int32_t step_index, int32_t steps_since_refresh,
                                  const int32_t* ext_window, int32_t n_ext_window, int32_t A, int32_t B, int32_t R,
-                                 int32_t T, wd_index_sets* out) {
+                                 int32_t T, int32_t refresh_mode, wd_index_sets* out) {
     if (!decoded || !dec_step || !out || (n_ext_window > 0 && !ext_window)) return WD_ERR_NULL;
     if (eos_id >= 0 && !token_ids) return WD_ERR_NULL;
     if (seq_len < 1 || n_ext_window < 0 || step_index < 0 || steps_since_refresh < 0) return WD_ERR_BAD_PARAM;
+    if (refresh_mode != WD_REFRESH_FULL && refresh_mode != WD_REFRESH_WINDOW) return WD_ERR_BAD_PARAM;
     WdSeq s;
     if (token_ids) s.ids.assign(token_ids, token_ids + seq_len);
     else s.ids.assign(seq_len, 0);
@@ -540,6 +550,8 @@ extern "C" wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step
     }
     s.t = step_index;
     s.since = steps_since_refresh;
+    s.phase_start = step_index - steps_since_refresh;       // first step of the running phase
+    s.refresh_mode = refresh_mode;
     WdSeqPlan p;
     wd_status r = wd_plan_seq(s, A, B, R, T, &p);
     if (r != WD_OK) return r;
@@ -708,6 +720,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
             pl.row_off[b] = r; pl.act_off[b] = a; pl.vis_off[b] = v; pl.qt_off[b] = qt;
             pl.done[b] = cp.done; pl.refresh[b] = cp.refresh; pl.n_wex[b] = cp.n_wex; pl.n_vis[b] = cp.n_vis;
             pl.t[b] = st->counts[b].t;
+            pl.window_refresh[b] = cp.window_refresh ? 1 : 0; pl.prev_phase_start[b] = cp.prev_phase_start;
             if (cp.done) continue;
             r += cp.n_rows; a += cp.n_active; v += cp.n_vis; qt += (cp.n_rows + 127) / 128;
         }

@@ -108,6 +108,8 @@ __device__ __forceinline__ float sum_slices1(const float* __restrict__ p, int n_
 // which tokens were unmasked).  Handles the states whose visible set is a prefix range.
 //   refresh:  external window = the first n_wex undecoded positions (ordered compaction),
 //             rows = visible positions = 0 .. n_vis-1, active = the first n_act of the window
+//             (window-only variant: rows = the window and the positions decoded since the
+//             previous phase began, by a second ordered compaction over the visible range)
 //   normal:   one pass over the window: undecoded members in order are active (the first A) or
 //             buffer, decoded members whose age is 1..T are the transient; rows = active and
 //             transient in position order
@@ -116,6 +118,7 @@ struct PlanArgs {
     int32_t row_off[WD_PLAN_MAX_BATCH + 1], act_off[WD_PLAN_MAX_BATCH + 1], vis_off[WD_PLAN_MAX_BATCH + 1],
         qt_off[WD_PLAN_MAX_BATCH + 1];
     int32_t t[WD_PLAN_MAX_BATCH];
+    int32_t window_refresh[WD_PLAN_MAX_BATCH], prev_phase_start[WD_PLAN_MAX_BATCH];
     int32_t S, A, T, batch;
     const uint8_t* decoded;
     const int32_t* dec_step;
@@ -184,7 +187,29 @@ __global__ void plan_kernel(const PlanArgs a) {
             base += tot;
         }
         if (base < n_wex && threadIdx.x == 0) atomicCAS(a.status, 0, WD_ERR_BOUNDS);   // counts and state disagree
-        for (int j = threadIdx.x; j < n_rows; j += blockDim.x) { a.row_seq[row0 + j] = b; a.row_pos[row0 + j] = j; }
+        if (!a.window_refresh[b]) {
+            for (int j = threadIdx.x; j < n_rows; j += blockDim.x) { a.row_seq[row0 + j] = b; a.row_pos[row0 + j] = j; }
+            return;
+        }
+        // window-only refresh: inside the visible range every undecoded position belongs to the
+        // window; decoded positions are rows when they were unmasked during the phase that just ended
+        int n_und = 0, n_row = 0;
+        for (int i0 = 0; i0 < n_vis; i0 += blockDim.x) {
+            const int i = i0 + threadIdx.x;
+            const int und = (i < n_vis && !dec[i]) ? 1 : 0;
+            const int prev = (i < n_vis && dec[i] && dstep[i] >= a.prev_phase_start[b]) ? 1 : 0;   // "never" is a large negative step
+            int tot_u, tot_r;
+            const int rank_u = n_und + block_scan_flag(und, &tot_u, warp_sums);
+            const int rank_r = n_row + block_scan_flag(und | prev, &tot_r, warp_sums);
+            if (und | prev) {
+                if (rank_r < n_rows) { a.row_seq[row0 + rank_r] = b; a.row_pos[row0 + rank_r] = i; }
+                else atomicCAS(a.status, 0, WD_ERR_BOUNDS);
+            }
+            if (und && rank_u < n_act) a.act_row[act0 + rank_u] = row0 + rank_r;
+            n_und += tot_u;
+            n_row += tot_r;
+        }
+        if (threadIdx.x == 0 && n_row != n_rows) atomicCAS(a.status, 0, WD_ERR_BOUNDS);
         return;
     }
     int n_und = 0, n_row = 0;
@@ -876,6 +901,7 @@ void wd_launch_plan(const WdPlanLaunch& h, cudaStream_t st) {
     for (int b = 0; b < h.batch; ++b) {
         a.refresh[b] = h.refresh[b]; a.done[b] = h.done[b]; a.n_wex[b] = h.n_wex[b]; a.n_vis[b] = h.n_vis[b];
         a.t[b] = h.t[b];
+        a.window_refresh[b] = h.window_refresh[b]; a.prev_phase_start[b] = h.prev_phase_start[b];
     }
     for (int b = 0; b <= h.batch; ++b) {
         a.row_off[b] = h.row_off[b]; a.act_off[b] = h.act_off[b]; a.vis_off[b] = h.vis_off[b]; a.qt_off[b] = h.qt_off[b];

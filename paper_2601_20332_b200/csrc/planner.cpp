@@ -69,7 +69,12 @@ wd_status wd_plan_seq(const WdSeq& s, int32_t A, int32_t B, int32_t R, int32_t T
         else if (live[i]) p.vis.push_back(i);
         else p.far_field.push_back(i);
     }
-    if (p.refresh) {
+    if (p.refresh && s.refresh_mode == WD_REFRESH_WINDOW && s.t > 0) {
+        // variant (not in the paper): only the new window and the tokens decoded during the phase
+        // that just ended are recomputed; s.phase_start is still that phase's first step
+        for (int32_t i : p.vis)
+            if (!s.decoded[i] || (s.dec_step[i] != INT32_MIN && s.dec_step[i] >= s.phase_start)) p.rows.push_back(i);
+    } else if (p.refresh) {
         p.rows = p.vis;
     } else {
         p.rows.resize(p.active.size() + p.transient.size());
@@ -105,6 +110,7 @@ void wd_count_init(WdCount& c, const WdSeq& s) {
     for (uint8_t d : s.decoded) (d ? c.decoded : c.undecoded) += 1;
     c.t = s.t;
     c.since = s.since;
+    c.refresh_mode = s.refresh_mode;
     c.wex_size = (int32_t)s.wex.size();
     for (int32_t i : s.wex) c.w_alive += s.decoded[i] ? 0 : 1;
     // tokens unmasked at each step of the running phase, oldest first
@@ -134,7 +140,11 @@ wd_status wd_count_plan(const WdCount& c, int32_t A, int32_t B, int32_t R, int32
     }
     p.n_active = std::min(A, w_alive);
     p.n_vis = c.decoded + w_alive;
-    p.n_rows = p.refresh ? p.n_vis : p.n_active + p.n_transient;
+    p.window_refresh = p.refresh && c.refresh_mode == WD_REFRESH_WINDOW && c.t > 0;
+    p.prev_phase_start = c.t - c.since;
+    int32_t prev_phase_tokens = 0;
+    for (int32_t h : c.hist) prev_phase_tokens += h;
+    p.n_rows = p.window_refresh ? p.n_wex + prev_phase_tokens : (p.refresh ? p.n_vis : p.n_active + p.n_transient);
     p.n_unmask = std::min(k, p.n_active);
     return WD_OK;
 }

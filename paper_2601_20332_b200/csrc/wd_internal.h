@@ -36,6 +36,7 @@ struct WdSeq {
     int32_t since = 0;              // steps since the last refresh
     int32_t phase_start = 0;
     int32_t eos_id = -1;            // adaptive termination: id of the end-of-sequence token, -1 = off
+    int32_t refresh_mode = 0;       // WD_REFRESH_FULL (the paper's refresh) or WD_REFRESH_WINDOW (variant)
 };
 
 struct WdSeqPlan {
@@ -57,10 +58,13 @@ struct WdCount {
     int32_t undecoded = 0, decoded = 0;   // |U|, |Dec|
     int32_t wex_size = 0, w_alive = 0;    // external window: size at phase start, still undecoded
     int32_t t = 0, since = 0;
+    int32_t refresh_mode = 0;
     std::vector<int32_t> hist;            // tokens unmasked at each step of the current phase
 };
 struct WdCountPlan {
     bool done = false, refresh = false;
+    bool window_refresh = false;          // refresh that computes only the new window and the previous phase's tokens
+    int32_t prev_phase_start = 0;
     int32_t n_active = 0, n_transient = 0, n_vis = 0, n_rows = 0, n_wex = 0, n_unmask = 0;
 };
 void wd_count_init(WdCount& c, const WdSeq& s);
@@ -142,6 +146,7 @@ struct WdPlanLaunch {
     int32_t batch, S, A, T;
     int32_t refresh[WD_PLAN_MAX_BATCH], done[WD_PLAN_MAX_BATCH], n_wex[WD_PLAN_MAX_BATCH], n_vis[WD_PLAN_MAX_BATCH],
         t[WD_PLAN_MAX_BATCH];
+    int32_t window_refresh[WD_PLAN_MAX_BATCH], prev_phase_start[WD_PLAN_MAX_BATCH];   // the window-only refresh variant
     int32_t row_off[WD_PLAN_MAX_BATCH + 1], act_off[WD_PLAN_MAX_BATCH + 1], vis_off[WD_PLAN_MAX_BATCH + 1],
         qt_off[WD_PLAN_MAX_BATCH + 1];
     const uint8_t* decoded;       // [batch][S] device

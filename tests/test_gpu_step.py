@@ -18,10 +18,10 @@ def built():
 
 
 def run(cfg, n_steps, ids=None, decoded=None, impl=wd.WD_GEMM_AUTO, jitter=0.1, tol_layer=1e-2, tol_attn=2e-2,
-        oracle_seqs=None, weights=None, fusion=False):
+        oracle_seqs=None, weights=None, fusion=False, refresh_mode=0):
     w = synth.make_weights(cfg, DEV, gain_jitter=jitter) if weights is None else weights
     ids = synth.make_prompts(cfg) if ids is None else ids
-    p = Parity(cfg, w, ids, decoded, gemm_impl=impl, oracle_seqs=oracle_seqs, fusion=fusion)
+    p = Parity(cfg, w, ids, decoded, gemm_impl=impl, oracle_seqs=oracle_seqs, fusion=fusion, refresh_mode=refresh_mode)
     logs = []
     for _ in range(n_steps):
         r = p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"], tol_layer, tol_attn)
@@ -89,6 +89,21 @@ def test_lm_head_statistics_with_several_token_tiles(batch, A):
     cfg = synth.get_config("llada8b", **dict(DH128, L=1, P=30, G=260, A=A, B=8, R=2, T=1, k=3, batch=batch))
     logs = run(cfg, 3, oracle_seqs=[0, batch - 1])
     assert logs[0]["info"]["n_active"] == batch * A
+
+
+@pytest.mark.parametrize("shape,batch", [(SMALL_BF16, 1), (DH128, 2)])
+def test_window_only_refresh_variant_matches_its_oracle(shape, batch):
+    """WD_REFRESH_WINDOW (not in the paper): refresh steps after the first compute only the new
+    window and the previous phase's tokens; index sets, layer outputs, logits and unmask choices
+    follow the oracle run in the same mode, through three phases (device-planned steps)."""
+    cfg = synth.get_config("llada8b", **dict(shape, batch=batch))
+    logs = run(cfg, 3 * cfg["R"] + 1, refresh_mode=wd.WD_REFRESH_WINDOW)
+    refreshes = [l for l in logs if l["info"]["is_refresh"]]
+    assert len(refreshes) == 4
+    per_seq_window = cfg["A"] + cfg["B"] + cfg["k"] * cfg["R"]
+    assert refreshes[0]["info"]["n_rows"] == refreshes[0]["info"]["n_vis"]        # first step: everything
+    for r in refreshes[1:]:
+        assert r["info"]["n_rows"] == batch * per_seq_window < r["info"]["n_vis"]
 
 
 def test_plain_and_tensor_core_paths_agree():
@@ -204,8 +219,8 @@ def test_far_field_and_refresh_independence_on_gpu(shape):
         assert torch.equal(a[0], b[0]) and (a[1] == b[1]).all() and (a[2] == b[2]).all()
 
 
-@pytest.mark.parametrize("shape,batch", [(SMALL_BF16, 1), (DH128, 2)])
-def test_steps_enqueued_back_to_back_match_stepwise_sync(shape, batch):
+@pytest.mark.parametrize("shape,batch,mode", [(SMALL_BF16, 1, 0), (DH128, 2, 0), (DH128, 2, 1)])
+def test_steps_enqueued_back_to_back_match_stepwise_sync(shape, batch, mode):
     """With a prompt-prefix state the device plans the steps itself: a whole run enqueued without
     a host round trip gives exactly the results of the same run with a sync after every step,
     and the host mirror ends up identical."""
@@ -218,6 +233,7 @@ def test_steps_enqueued_back_to_back_match_stepwise_sync(shape, batch):
     runs = []
     for queued in (False, True):
         st = wd.State(ctx, ids)
+        st.set_refresh_mode(mode)
         res = []
         for i in range(n_steps):
             st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])

@@ -33,7 +33,7 @@ def max_rel(a, b):
 
 class Parity:
     def __init__(self, cfg, weights, ids, decoded=None, gemm_impl=wd.WD_GEMM_AUTO, oracle_seqs=None,
-                 max_rows=None, max_active=None, fusion=False, eos_id=None):
+                 max_rows=None, max_active=None, fusion=False, eos_id=None, refresh_mode=0):
         self.cfg = cfg
         self.batch, self.S = ids.shape
         dev = weights.tok_embed.device
@@ -45,6 +45,8 @@ class Parity:
         self.st = wd.State(self.ctx, ids, decoded)
         if eos_id is not None:
             self.st.set_eos(eos_id)
+        if refresh_mode:
+            self.st.set_refresh_mode(refresh_mode)
         L, d, hq, V = cfg["L"], cfg["d"], cfg["Hq"] * cfg["dh"], cfg["V"]
         self.t_layer = torch.zeros(L * max_rows * d, dtype=torch.float32, device=dev)
         self.t_attn = torch.zeros(L * max_rows * hq, dtype=torch.float32, device=dev)
@@ -53,7 +55,8 @@ class Parity:
         self.model = synth.OracleModelView(weights)
         self.oracle_seqs = list(range(self.batch)) if oracle_seqs is None else list(oracle_seqs)
         dec = (ids != cfg["mask_id"]) if decoded is None else decoded.astype(bool)
-        self.ost = [wo.SeqState(ids=ids[b], decoded=dec[b], eos_id=eos_id) for b in self.oracle_seqs]
+        self.ost = [wo.SeqState(ids=ids[b], decoded=dec[b], eos_id=eos_id, refresh_mode=refresh_mode)
+                    for b in self.oracle_seqs]
         self.oc = [wo.KVCache.empty(self.model.dims, self.S) for _ in self.oracle_seqs]
         self.log = []
 
