@@ -202,6 +202,47 @@ class KVCache:
         return KVCache(np.full(shape, fill), np.full(shape, fill))
 
 
+# ---------------------------------------------------------------------------
+# FP8 mode (an option outside the paper, which calls quantisation orthogonal to the method)
+# ---------------------------------------------------------------------------
+# With dims["fp8"] set, the projections q/k/v, gate/up, down and the LM head take both operands
+# in 8-bit floating point e4m3 (4 exponent bits, 3 mantissa bits, largest finite value 448, no
+# infinities): every weight row and every activation row is divided by its own scale
+# s = fl32(max |row| / 448) (1 for an all-zero row), rounded to the nearest e4m3 value (ties to
+# even), and the product is scaled back by the two row scales.  The output projection, attention,
+# the residual stream and the K/V cache are unchanged.
+
+E4M3_MAX = 448.0
+
+
+def e4m3_round(v32: np.ndarray) -> np.ndarray:
+    """Nearest e4m3 value of each float32 (round to nearest even), returned as float64."""
+    import torch
+    t = torch.from_numpy(np.ascontiguousarray(v32, dtype=np.float32)).to(torch.float8_e4m3fn)
+    return t.to(torch.float64).numpy()
+
+
+def fp8_quant_rows(x: np.ndarray):
+    """Per-row e4m3 quantisation of a [n, K] matrix: (values on the e4m3 grid as float64, float32 scales).
+    The value that is quantised is the float32 rounding of the input (what a float32 pipeline holds)."""
+    x32 = np.asarray(x).astype(np.float32)
+    amax = np.abs(x32).max(axis=1) if x32.shape[1] else np.zeros(x32.shape[0], np.float32)
+    s = np.where(amax > 0, (amax / np.float32(E4M3_MAX)).astype(np.float32), np.float32(1.0)).astype(np.float32)
+    q = e4m3_round((x32 / s[:, None]).astype(np.float32))
+    return q, s
+
+
+def fp8_matmul(x: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """x w^T with both operands quantised row by row (see above)."""
+    qx, sx = fp8_quant_rows(x)
+    qw, sw = fp8_quant_rows(w)
+    return (qx @ qw.T) * sx.astype(np.float64)[:, None] * sw.astype(np.float64)[None, :]
+
+
+def _proj(dims: dict, x: np.ndarray, w: np.ndarray) -> np.ndarray:
+    return fp8_matmul(x, w) if dims.get("fp8") else x @ w.T
+
+
 def oracle_layer(dims: dict, lw: dict, x: np.ndarray, pos, vis, cache: KVCache, l: int,
                  want_probs: bool = False) -> dict:
     """One transformer block over the computed rows ``pos`` (ascending
@@ -213,9 +254,9 @@ def oracle_layer(dims: dict, lw: dict, x: np.ndarray, pos, vis, cache: KVCache, 
     n = x.shape[0]
     pos = np.asarray(pos, dtype=np.int64)
     a = rmsnorm(x, lw["attn_norm"], dims["eps"])
-    q = (a @ lw["wq"].T).reshape(n, Hq, dh)
-    k = (a @ lw["wk"].T).reshape(n, Hkv, dh)
-    v = (a @ lw["wv"].T).reshape(n, Hkv, dh)
+    q = _proj(dims, a, lw["wq"]).reshape(n, Hq, dh)
+    k = _proj(dims, a, lw["wk"]).reshape(n, Hkv, dh)
+    v = _proj(dims, a, lw["wv"]).reshape(n, Hkv, dh)
     q = rope(q, pos, dims["theta"])
     k = rope(k, pos, dims["theta"])
     cache.K[l, pos] = k
@@ -225,7 +266,7 @@ def oracle_layer(dims: dict, lw: dict, x: np.ndarray, pos, vis, cache: KVCache, 
     o = o.reshape(n, Hq * dh)
     h = x + o @ lw["wo"].T
     f = rmsnorm(h, lw["ffn_norm"], dims["eps"])
-    y = h + (silu(f @ lw["w_gate"].T) * (f @ lw["w_up"].T)) @ lw["w_down"].T
+    y = h + _proj(dims, silu(_proj(dims, f, lw["w_gate"])) * _proj(dims, f, lw["w_up"]), lw["w_down"])
     res = dict(out=y, attn=o)
     if want_probs:
         res["probs"] = probs
@@ -306,7 +347,7 @@ def oracle_step(model, states, caches, A: int, B: int, R: int, T: int, k: int,
             w_lm = model.lm_head()
         rows = pl["rows"]
         sel = [rows.index(p) for p in pl["active"]]
-        logits = rmsnorm(xs[i][sel], g_final, dims["eps"]) @ w_lm.T
+        logits = _proj(dims, rmsnorm(xs[i][sel], g_final, dims["eps"]), w_lm)
         um = oracle_unmask(logits, pl["active"], k)
         outs[i].update(logits=logits, unmask=um)
         if forced is not None and forced[i] is not None:

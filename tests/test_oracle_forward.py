@@ -410,3 +410,72 @@ def test_window_refresh_is_an_approximation_for_deeper_models():
     assert np.isfinite(win[3][0]["logits"]).all()
     vis = full[3][0]["plan"]["vis"]
     np.testing.assert_allclose(cw[0].K[0][vis], cf[0].K[0][vis], rtol=1e-10, atol=1e-10)   # layer 0: context-free
+
+
+# ---------------------------------------------------------------- FP8 mode (option outside the paper)
+
+def _all_e4m3_values():
+    """Every finite e4m3 value from the format's definition: sign, 4 exponent bits (bias 7),
+    3 mantissa bits; exponent 0 is subnormal; exponent 15 with mantissa 7 is NaN."""
+    vals = set()
+    for e in range(16):
+        for m in range(8):
+            if e == 15 and m == 7:
+                continue
+            v = (m / 8.0) * 2.0 ** (-6) if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7)
+            vals.add(v)
+            vals.add(-v)
+    return np.array(sorted(vals))
+
+
+def test_e4m3_rounding_against_the_format_definition():
+    grid = _all_e4m3_values()
+    assert grid.max() == 448.0 and len(grid) == 2 * (16 * 8 - 1) - 1           # +0 and -0 coincide
+    np.testing.assert_array_equal(wo.e4m3_round(grid.astype(np.float32)), grid)   # representable values stay
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.uniform(-448, 448, 4000), rng.normal(0, 3, 4000), rng.normal(0, 0.01, 2000)]).astype(np.float32)
+    got = wo.e4m3_round(x)
+    # brute force: the nearest grid value; on a tie the one whose mantissa is even
+    for v, g in zip(x.astype(np.float64), got):
+        d = np.abs(grid - v)
+        best = np.flatnonzero(d == d.min())
+        if len(best) == 1:
+            assert g == grid[best[0]]
+        else:
+            lo, hi = grid[best[0]], grid[best[1]]
+            even = [c for c in (lo, hi) if (abs(c) / 2.0 ** np.floor(np.log2(max(abs(c), 2.0 ** -6))) * 8) % 2 == 0]
+            assert g in (lo, hi) and (not even or g in even)
+    # exact midpoints between neighbours round to the even mantissa: 1.0625 is halfway between 1.0 and 1.125
+    np.testing.assert_array_equal(wo.e4m3_round(np.array([1.0625, 1.1875, -1.0625], np.float32)), [1.0, 1.25, -1.0])
+
+
+def test_fp8_row_quantisation_and_product():
+    rng = np.random.default_rng(6)
+    x = rng.normal(0, 2, (5, 64))
+    q, s = wo.fp8_quant_rows(x)
+    assert s.dtype == np.float32 and np.abs(q).max(axis=1).tolist() == [448.0] * 5      # the row maximum maps to 448
+    assert np.abs(q * s[:, None] - x).max() <= np.abs(x).max() * 2.0 ** -4           # half a spacing of the top binade
+    zq, zs = wo.fp8_quant_rows(np.zeros((2, 8)))
+    assert (zq == 0).all() and (zs == 1).all()
+    # operands that are already on the grid (times a power of two) multiply exactly
+    grid = _all_e4m3_values()
+    # (row maximum 7 = 448 / 2^6 and 1.75 = 448 / 2^8: the scales are then powers of two)
+    a = rng.choice(grid[(np.abs(grid) <= 7) & (np.abs(grid) >= 2.0 ** -3)], size=(4, 32)); a[:, 0] = 7.0
+    b = rng.choice(grid[(np.abs(grid) <= 1.75) & (np.abs(grid) >= 2.0 ** -5)], size=(6, 32)); b[:, 0] = 1.75
+    np.testing.assert_allclose(wo.fp8_matmul(a, b), a @ b.T, rtol=1e-6)
+    # and the quantised product stays within the format's relative precision of the exact one
+    w = rng.normal(0, 0.02, (16, 256)); xx = rng.normal(0, 1, (7, 256))
+    err = np.linalg.norm(wo.fp8_matmul(xx, w) - xx @ w.T) / np.linalg.norm(xx @ w.T)
+    assert 1e-3 < err < 8e-2
+
+
+def test_fp8_mode_changes_only_the_quantised_projections():
+    cfg = small_cfg(G=12)
+    model = make(cfg)
+    base, _, _ = run_traj(cfg, model, 2)
+    model.dims = dict(model.dims, fp8=True)
+    f8, _, _ = run_traj(cfg, model, 2)
+    a, b = base[0][0], f8[0][0]
+    assert a["plan"] == b["plan"]
+    rel = np.linalg.norm(a["logits"] - b["logits"]) / np.linalg.norm(a["logits"])
+    assert 1e-4 < rel < 0.3 and np.isfinite(b["logits"]).all()
