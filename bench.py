@@ -222,6 +222,21 @@ def run_ours(args, rank, world):
     v_total_ms = max_over_ranks(v_total_ms, world, dev)
     v_refresh = [t for t, i in zip(v_per_step, v_infos) if i["is_refresh"]]
     state.set_refresh_mode(wd.WD_REFRESH_FULL)
+    # ---- FP8 projections (an option outside the paper; never the headline, which stays bf16)
+    fp8_line = None
+    if cfg["dtype"] == "bf16":
+        ctx.fp8_enable(stream)
+        state.reset(ids, None, stream)
+        f_infos, f_per_step, f_total_ms, _ = trajectory(W, K, state, queued=True)
+        f_total_ms = max_over_ranks(f_total_ms, world, dev)
+        f_normal = [t for t, i in zip(f_per_step, f_infos) if not i["is_refresh"]]
+        f_refresh = [t for t, i in zip(f_per_step, f_infos) if i["is_refresh"]]
+        fp8_line = {"note": "NOT the headline precision: e4m3 weights and activations with per-row scales for q/k/v, "
+                            "gate/up, down and the LM head (fp32 accumulation); everything else as in the bf16 run",
+                    "value": whole_job_value(batch * k * K, world, f_total_ms), "unit": UNIT,
+                    "normal_step_ms": float(np.median(f_normal)) if f_normal else None,
+                    "refresh_step_ms": float(np.median(f_refresh)) if f_refresh else None}
+        ctx.fp8_set(False)
     # ---- a whole generation through the library's own driver: host prompt in, host tokens out
     torch.cuda.synchronize()
     t0 = time.perf_counter()
@@ -272,6 +287,7 @@ def run_ours(args, rank, world):
                    "rows_normal": float(np.mean([i["n_rows"] for i in ni])) if ni else None,
                    "stepping": "queued: steps enqueued back to back, index lists planned on the device, drained every 16 steps",
                    "gemm_impl": infos[-1]["gemm_impl"],
+                   "variant_fp8_projections": fp8_line,
                    "variant_window_only_refresh": {
                        "note": "NOT the paper's refresh: after the first step a refresh recomputes only the new window "
                                "and the previous phase's tokens (an approximation beyond one block); same steps otherwise",

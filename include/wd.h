@@ -252,6 +252,24 @@ WD_API wd_status wd_state_set_eos(wd_state* st, int32_t eos_id);
  * Kept across wd_state_reset.  Errors: WD_ERR_NULL, WD_ERR_PENDING, WD_ERR_BAD_PARAM. */
 WD_API wd_status wd_state_set_refresh_mode(wd_state* st, int32_t mode);
 
+/* ---- FP8 mode (no counterpart in the paper, which calls quantisation orthogonal to the method) ----
+ * The projections q/k/v, gate/up, down and the LM head then take both operands in 8-bit floating
+ * point e4m3: every weight row once (wd_fp8_enable) and every activation row at every step is
+ * divided by its own scale s = max|row| / 448 (1 for a zero row), rounded to the nearest e4m3
+ * value (ties to even), multiplied on the tensor cores (tcgen05 kind::f8f6f4, fp32 accumulation)
+ * and scaled back by the two row scales.  The output projection, attention, the residual stream
+ * and the K/V cache stay as they are.  Halves the weight bytes a normal step streams; changes the
+ * numbers (relative error of a projection around 3-4 %).  bf16 models on the tensor-core path only.
+ *   wd_fp8_bytes   size of the device memory block wd_fp8_enable needs (0 for invalid dims / fp32)
+ *   wd_fp8_enable  quantises the weights on `stream` into `mem` (caller-owned, 256-byte aligned,
+ *                  must outlive the context) and switches the mode on for later steps.
+ *                  d_model and d_ffn must be multiples of 16, d_ffn <= 32768.
+ *   wd_fp8_set     switches the mode off / on again (on needs a prior wd_fp8_enable).
+ * Errors: WD_ERR_NULL, WD_ERR_BAD_PARAM, WD_ERR_MISALIGNED, WD_ERR_WORKSPACE_TOO_SMALL, WD_ERR_CUDA. */
+WD_API size_t wd_fp8_bytes(const wd_model_dims* dims);
+WD_API wd_status wd_fp8_enable(wd_ctx* ctx, void* mem, size_t mem_bytes, void* stream /*cudaStream_t*/);
+WD_API wd_status wd_fp8_set(wd_ctx* ctx, int32_t on);
+
 /* ---- the step ----------------------------------------------------------- */
 
 /* Preview of the index sets the next wd_step(st, A, B, R, T, ...) will use for
@@ -341,6 +359,14 @@ WD_API wd_status wd_op_gemm(int32_t dtype, int32_t impl, const void* x, const vo
                      int32_t rows, int32_t n_out, int32_t k_in,
                      void* scratch, size_t scratch_bytes, void* stream);
 WD_API size_t wd_op_gemm_scratch_bytes(int32_t rows, int32_t n_out, int32_t k_in);
+
+/* The FP8 projection of the FP8 mode as a single operation (see wd_fp8_enable): both bf16
+ * operands are quantised row by row to e4m3 (scale = max|row| / 448) into `scratch`, multiplied
+ * on the tensor cores and scaled back; y[rows, n_out] float.  k_in a multiple of 16; scratch
+ * 256-byte aligned, wd_op_gemm_fp8_scratch_bytes large.  Errors as wd_op_gemm. */
+WD_API wd_status wd_op_gemm_fp8(const void* x, const void* w, float* y, int32_t rows, int32_t n_out, int32_t k_in,
+                         void* scratch, size_t scratch_bytes, void* stream /*cudaStream_t*/);
+WD_API size_t wd_op_gemm_fp8_scratch_bytes(int32_t rows, int32_t n_out, int32_t k_in);
 
 /* (No counterpart in the paper: a packaging variant of wd_op_gemm.)
  * The same bf16 tensor-core GEMM, y[rows, n_out] (float) = x[rows, k_in] * w[n_out, k_in]^T,

@@ -76,6 +76,9 @@ SIGNATURES = {
     "wd_plan": (C.c_int, [vp, i32, i32, i32, i32, i32, C.POINTER(wd_index_sets)]),
     "wd_plan_raw": (C.c_int, [u8p, i32p, i32p, i32, i32, i32, i32, i32p, i32, i32, i32, i32, i32, i32,
                               C.POINTER(wd_index_sets)]),
+    "wd_fp8_bytes": (C.c_size_t, [C.POINTER(wd_model_dims)]),
+    "wd_fp8_enable": (C.c_int, [vp, vp, C.c_size_t, vp]),
+    "wd_fp8_set": (C.c_int, [vp, i32]),
     "wd_state_set_eos": (C.c_int, [vp, i32]),
     "wd_state_set_refresh_mode": (C.c_int, [vp, i32]),
     "wd_step": (C.c_int, [vp, i32, i32, i32, i32, i32, vp, C.POINTER(wd_step_info)]),
@@ -84,6 +87,8 @@ SIGNATURES = {
     "wd_generate": (C.c_int, [vp, i32, i32, i32, i32, i32, i32, vp, i32p, i32p]),
     "wd_op_gemm": (C.c_int, [i32, i32, vp, vp, vp, i32, i32, i32, vp, C.c_size_t, vp]),
     "wd_op_gemm_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
+    "wd_op_gemm_fp8": (C.c_int, [vp, vp, vp, i32, i32, i32, vp, C.c_size_t, vp]),
+    "wd_op_gemm_fp8_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
     "wd_op_gemm_noalloc": (C.c_int, [vp, vp, vp, i32, i32, i32, vp]),
     "wd_op_gemm_noalloc_max_floats": (C.c_size_t, []),
     "wd_op_attention": (C.c_int, [i32, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]),
@@ -207,6 +212,18 @@ class Context:
 
     def profile_enable(self, on: bool):
         check(lib().wd_profile_enable(self.handle, 1 if on else 0), "wd_profile_enable")
+
+    def fp8_enable(self, stream=None):
+        """wd_fp8_enable: quantise the weights to e4m3 and run the projections in FP8 from now on."""
+        import torch
+        nbytes = lib().wd_fp8_bytes(C.byref(self.dims))
+        if nbytes == 0:
+            raise WdError(WD_ERR_BAD_PARAM, "wd_fp8_bytes")
+        self._fp8_mem = torch.empty(nbytes, dtype=torch.uint8, device=self.workspace.device)
+        check(lib().wd_fp8_enable(self.handle, _ptr(self._fp8_mem), nbytes, _stream_ptr(stream)), "wd_fp8_enable")
+
+    def fp8_set(self, on: bool):
+        check(lib().wd_fp8_set(self.handle, 1 if on else 0), "wd_fp8_set")
 
     def profile_read(self) -> dict:
         ms, by, n = C.c_double(), C.c_double(), C.c_int64()
@@ -349,6 +366,18 @@ def op_gemm(x, w, impl: int = WD_GEMM_AUTO, stream=None, scratch=None):
         scratch = torch.empty(max(nb, 256), dtype=torch.uint8, device=x.device)
     check(lib().wd_op_gemm(_dtype_code(x), impl, _ptr(x), _ptr(w), _ptr(y), rows, n, k, _ptr(scratch),
                            scratch.numel(), _stream_ptr(stream)), "wd_op_gemm")
+    return y
+
+
+def op_gemm_fp8(x, w, stream=None):
+    """y[rows, n] (float32) = FP8 product of the bf16 operands (per-row e4m3 quantisation of both)."""
+    import torch
+    rows, k = x.shape
+    n = w.shape[0]
+    y = torch.empty(rows, n, dtype=torch.float32, device=x.device)
+    nb = lib().wd_op_gemm_fp8_scratch_bytes(rows, n, k)
+    scratch = torch.empty(max(nb, 256), dtype=torch.uint8, device=x.device)
+    check(lib().wd_op_gemm_fp8(_ptr(x), _ptr(w), _ptr(y), rows, n, k, _ptr(scratch), nb, _stream_ptr(stream)), "wd_op_gemm_fp8")
     return y
 
 

@@ -85,6 +85,18 @@ struct wd_ctx {
 
     WdTcWeights tc;              // tensor maps of the weights (bf16 only)
 
+    // FP8 mode (wd_fp8_enable): e4m3 copies of q/k/v, gate/up, down and the LM head with one scale
+    // per weight row, FP8 activation buffers with one scale per row, and their tensor maps
+    bool fp8_ready = false, fp8_on = false;
+    struct Fp8Mat { const uint8_t* q = nullptr; const float* s = nullptr; CUtensorMap map; };
+    std::vector<Fp8Mat> f8q, f8k, f8v, f8g, f8u, f8d;
+    Fp8Mat f8lm;
+    uint8_t* xn8 = nullptr;      // [max_rows, d]
+    uint8_t* h8 = nullptr;       // [max_rows, F]
+    float* sxn = nullptr;        // [max_rows]
+    float* sh = nullptr;         // [max_rows]
+    WdTcX x8_d, x8_h;
+
     // optional GEMM timing (benchmarks): event pairs around every GEMM launch of a step
     bool prof_on = false;
     std::vector<cudaEvent_t> prof_events;
@@ -254,6 +266,84 @@ extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, v
         if (s != WD_OK) { delete c; return s; }
     }
     *out = c;
+    return WD_OK;
+}
+
+// ---------------------------------------------------------------------------
+// FP8 mode
+// ---------------------------------------------------------------------------
+static size_t fp8_carve(const wd_model_dims* d, size_t* off /*[8]*/) {
+    const size_t hq = (size_t)d->n_q_heads * d->head_dim, hkv = (size_t)d->n_kv_heads * d->head_dim;
+    const size_t D = d->d_model, F = d->d_ffn, V = d->vocab, L = d->n_layers, MR = d->max_rows;
+    const size_t rows_per_layer = hq + 2 * hkv + 2 * F + D;                  // weight rows with a scale each
+    const size_t codes_per_layer = (hq + 2 * hkv) * D + 2 * F * D + D * F;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { const size_t at = o; o = wd_align_up(o + bytes, 256); return at; };
+    off[0] = take(L * codes_per_layer);          // layer weight codes
+    off[1] = take(L * rows_per_layer * 4);       // layer weight scales
+    off[2] = take(V * D);                        // LM head codes
+    off[3] = take(V * 4);                        // LM head scales
+    off[4] = take(MR * D);                       // xn8
+    off[5] = take(MR * F);                       // h8
+    off[6] = take(MR * 4);                       // sxn
+    off[7] = take(MR * 4);                       // sh
+    return o;
+}
+
+extern "C" size_t wd_fp8_bytes(const wd_model_dims* dims) {
+    if (!dims_valid(dims) || dims->dtype != WD_BF16) return 0;
+    size_t off[8];
+    return fp8_carve(dims, off);
+}
+
+extern "C" wd_status wd_fp8_enable(wd_ctx* c, void* mem, size_t mem_bytes, void* stream_) {
+    if (!c || !mem) return WD_ERR_NULL;
+    const wd_model_dims& d = c->d;
+    if (d.dtype != WD_BF16 || d.d_model % 16 || d.d_ffn % 16 || d.d_ffn > 32768) return WD_ERR_BAD_PARAM;
+    if ((uintptr_t)mem % 256) return WD_ERR_MISALIGNED;
+    size_t off[8];
+    if (mem_bytes < fp8_carve(&d, off)) return WD_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const int hq = d.n_q_heads * d.head_dim, hkv = d.n_kv_heads * d.head_dim, D = d.d_model, F = d.d_ffn, L = d.n_layers;
+    uint8_t* codes = (uint8_t*)mem + off[0];
+    float* scales = (float*)((char*)mem + off[1]);
+    auto quant = [&](const void* w, int n, int K, wd_ctx::Fp8Mat* m) -> wd_status {
+        wd_launch_quantize_rows(WD_BF16, w, n, K, codes, scales, stream);
+        m->q = codes; m->s = scales;
+        wd_status s = wd_tc_encode_fp8(&m->map, codes, n, K, 128);
+        codes += (size_t)n * K;
+        scales += n;
+        return s;
+    };
+    c->f8q.assign(L, {}); c->f8k.assign(L, {}); c->f8v.assign(L, {}); c->f8g.assign(L, {}); c->f8u.assign(L, {}); c->f8d.assign(L, {});
+    wd_status s;
+    for (int l = 0; l < L; ++l) {
+        if ((s = quant(c->wq[l], hq, D, &c->f8q[l])) != WD_OK) return s;
+        if ((s = quant(c->wk[l], hkv, D, &c->f8k[l])) != WD_OK) return s;
+        if ((s = quant(c->wv[l], hkv, D, &c->f8v[l])) != WD_OK) return s;
+        if ((s = quant(c->wg[l], F, D, &c->f8g[l])) != WD_OK) return s;
+        if ((s = quant(c->wu[l], F, D, &c->f8u[l])) != WD_OK) return s;
+        if ((s = quant(c->wd[l], D, F, &c->f8d[l])) != WD_OK) return s;
+    }
+    codes = (uint8_t*)mem + off[2];
+    scales = (float*)((char*)mem + off[3]);
+    if ((s = quant(c->lm_head, d.vocab, D, &c->f8lm)) != WD_OK) return s;
+    c->xn8 = (uint8_t*)mem + off[4];
+    c->h8 = (uint8_t*)mem + off[5];
+    c->sxn = (float*)((char*)mem + off[6]);
+    c->sh = (float*)((char*)mem + off[7]);
+    c->x8_d = WdTcX(); c->x8_d.ptr = c->xn8; c->x8_d.K = D; c->x8_d.fp8 = 1;
+    c->x8_h = WdTcX(); c->x8_h.ptr = c->h8; c->x8_h.K = F; c->x8_h.fp8 = 1;
+    WD_CUDA_TRY(cudaGetLastError());
+    c->fp8_ready = true;
+    c->fp8_on = true;
+    return WD_OK;
+}
+
+extern "C" wd_status wd_fp8_set(wd_ctx* c, int32_t on) {
+    if (!c) return WD_ERR_NULL;
+    if (on && !c->fp8_ready) return WD_ERR_BAD_PARAM;
+    c->fp8_on = on != 0;
     return WD_OK;
 }
 
@@ -587,7 +677,8 @@ static bool use_tc(const wd_ctx* c) {
 
 static wd_status run_gemm(wd_ctx* c, const void* x, const WdTcX* x_map, const WdTcSeg* segs, int nseg,
                           int rows, int K, float* y, size_t y_floats, int32_t* status, cudaStream_t stream,
-                          GemmOut* go, bool single_split = false, const WdTcFuse* fuse = nullptr) {
+                          GemmOut* go, bool single_split = false, const WdTcFuse* fuse = nullptr,
+                          const WdTcFp8* fp8 = nullptr) {
     int ncol = 0;
     for (int i = 0; i < nseg; ++i) ncol += segs[i].n;
     cudaEvent_t e0 = nullptr, e1 = nullptr;
@@ -600,14 +691,14 @@ static wd_status run_gemm(wd_ctx* c, const void* x, const WdTcX* x_map, const Wd
         e0 = c->prof_events[c->prof_used++];
         e1 = c->prof_events[c->prof_used++];
         // algorithmic bytes: weights once, activations in, result out
-        c->prof_step_bytes += (double)ncol * K * wd_elt_size(c->d.dtype) + (double)rows * K * wd_elt_size(c->d.dtype) +
-                              (double)rows * ncol * 4;
+        const double elt = fp8 ? 1.0 : (double)wd_elt_size(c->d.dtype);
+        c->prof_step_bytes += (double)ncol * K * elt + (double)rows * K * elt + (double)rows * ncol * 4;
         WD_CUDA_TRY(cudaEventRecord(e0, stream));
     }
     if (use_tc(c)) {
         int n_split = 1;
         wd_status s = wd_tc_gemm(x_map, segs, nseg, rows, K, y, y_floats, c->sm_count, status, stream, &n_split,
-                                 single_split, fuse);
+                                 single_split, fuse, fp8);
         if (s != WD_OK) return s;
         *go = {n_split, (size_t)rows * ncol, 1, WD_GEMM_TCGEN05};
     } else {
@@ -798,6 +889,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
 
     const int Sp = st->Sp;
     const bool fused = use_tc(c) && c->fuse && dh == 128 && D % 128 == 0 && F % 128 == 0;
+    const bool fp8 = c->fp8_on && use_tc(c) && !fused;      // FP8 projections (q/k/v, gate/up, down, LM head)
     auto attention = [&](int l, char* kc, char* vc) -> wd_status {
         float* attn_tap = st->taps.attn_out ? st->taps.attn_out + (size_t)l * R_ * hq : nullptr;
         if (st->attn_tc && all_contig && c->attn_impl != WD_GEMM_PLAIN)
@@ -868,14 +960,24 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     for (int l = 0; l < d.n_layers; ++l) {
         char* kc = st->kcache + (size_t)l * st->kv_layer_bytes;
         char* vc = st->vcache + (size_t)l * st->v_layer_bytes;
-        // attention half
+        // attention half (FP8 mode: the normalised rows leave the RMSNorm as e4m3 codes + row scales)
         wd_launch_rmsnorm(d.dtype, c->x, down_pending ? c->part : nullptr, down_go.n_split, down_go.split_stride,
-                          c->attn_norm[l], d.rms_eps, c->xn, nullptr, R_, D, stream);
+                          c->attn_norm[l], d.rms_eps, c->xn, nullptr, R_, D, stream, fp8 ? c->xn8 : nullptr, c->sxn);
         down_pending = false;
+        if (fp8) {
+            WdTcSeg qkv[3] = {{c->f8q[l].q, hq, &c->f8q[l].map}, {c->f8k[l].q, hkv, &c->f8k[l].map},
+                              {c->f8v[l].q, hkv, &c->f8v[l].map}};
+            WdTcFp8 f8;
+            f8.sw[0] = c->f8q[l].s; f8.sw[1] = c->f8k[l].s; f8.sw[2] = c->f8v[l].s; f8.sx = c->sxn;
+            if ((s = run_gemm(c, c->xn8, &c->x8_d, qkv, 3, R_, D, c->part, c->part_floats, status, stream, &go, false,
+                              nullptr, &f8)) != WD_OK)
+                return s;
+        } else {
         WdTcSeg qkv[3] = {{c->wq[l], hq, c->tc.get(WD_TC_WQ, l)}, {c->wk[l], hkv, c->tc.get(WD_TC_WK, l)},
                           {c->wv[l], hkv, c->tc.get(WD_TC_WV, l)}};
         if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, qkv, 3, R_, D, c->part, c->part_floats, status, stream, &go)) != WD_OK)
             return s;
+        }
         impl_used = go.impl;
         wd_launch_rope_scatter(d.dtype, c->part, go.n_split, go.split_stride, row_seq, row_pos, c->rope_tab, c->q, kc,
                                vc, R_, Hq, Hkv, dh, S, Sp, stream);
@@ -885,7 +987,22 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
             return s;
         // feed-forward half
         wd_launch_rmsnorm(d.dtype, c->x, c->part, go.n_split, go.split_stride, c->ffn_norm[l], d.rms_eps, c->xn,
-                          nullptr, R_, D, stream);
+                          nullptr, R_, D, stream, fp8 ? c->xn8 : nullptr, c->sxn);
+        if (fp8) {
+            WdTcSeg gu[2] = {{c->f8g[l].q, F, &c->f8g[l].map}, {c->f8u[l].q, F, &c->f8u[l].map}};
+            WdTcFp8 f8;
+            f8.sw[0] = c->f8g[l].s; f8.sw[1] = c->f8u[l].s; f8.sx = c->sxn;
+            if ((s = run_gemm(c, c->xn8, &c->x8_d, gu, 2, R_, D, c->part, c->part_floats, status, stream, &go, false, nullptr,
+                              &f8)) != WD_OK)
+                return s;
+            if ((s = wd_launch_swiglu_fp8(c->part, go.n_split, go.split_stride, c->h8, c->sh, R_, F, stream)) != WD_OK) return s;
+            WdTcSeg wdn[1] = {{c->f8d[l].q, D, &c->f8d[l].map}};
+            WdTcFp8 f8d;
+            f8d.sw[0] = c->f8d[l].s; f8d.sx = c->sh;
+            if ((s = run_gemm(c, c->h8, &c->x8_h, wdn, 1, R_, F, c->part, c->part_floats, status, stream, &go, false, nullptr,
+                              &f8d)) != WD_OK)
+                return s;
+        } else {
         WdTcSeg gu[2] = {{c->wg[l], F, c->tc.get(WD_TC_WG, l)}, {c->wu[l], F, c->tc.get(WD_TC_WU, l)}};
         if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, gu, 2, R_, D, c->part, c->part_floats, status, stream, &go)) != WD_OK)
             return s;
@@ -893,6 +1010,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         WdTcSeg wdn[1] = {{c->wd[l], D, c->tc.get(WD_TC_WD, l)}};
         if ((s = run_gemm(c, c->h, &c->tc.x_map_h, wdn, 1, R_, F, c->part, c->part_floats, status, stream, &go)) != WD_OK)
             return s;
+        }
         if (st->taps.layer_out || l == d.n_layers - 1) {
             float* tap = st->taps.layer_out ? st->taps.layer_out + (size_t)l * R_ * D : nullptr;
             wd_launch_residual_add(c->x, c->part, go.n_split, go.split_stride, tap, R_, D, stream);
@@ -906,8 +1024,14 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     bool lm_fused = false;
     int lm_chunks = wd_unmask_chunks(d.vocab);
     if (NA > 0) {
-        wd_launch_rmsnorm(d.dtype, c->x, nullptr, 0, 0, c->final_norm, d.rms_eps, c->xn, act_row, NA, D, stream);
+        wd_launch_rmsnorm(d.dtype, c->x, nullptr, 0, 0, c->final_norm, d.rms_eps, c->xn, act_row, NA, D, stream,
+                          fp8 ? c->xn8 : nullptr, c->sxn);
         WdTcSeg lm[1] = {{c->lm_head, d.vocab, c->tc.get(WD_TC_LM, 0)}};
+        WdTcFp8 f8lm;
+        if (fp8) {
+            lm[0] = {c->f8lm.q, d.vocab, &c->f8lm.map};
+            f8lm.sw[0] = c->f8lm.s; f8lm.sx = c->sxn;
+        }
         // tensor-core path: the LM-head epilogue leaves per-tile (max, argmax, sum exp) instead of a separate
         // pass over the logits, which then never have to be written (only for the parity tap)
         WdTcFuse fl;
@@ -915,8 +1039,9 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         fl.st_max = c->ch_max; fl.st_idx = c->ch_idx; fl.st_sum = c->ch_sum;
         fl.write_logits = st->taps.logits ? 1 : 0;
         lm_fused = use_tc(c) && NA <= 1024 && c->sm_count % 4 == 0;     // one CTA group per tile of <= 256 active rows
-        if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, lm, 1, NA, D, c->logits, (size_t)d.max_active * d.vocab, status,
-                          stream, &go, /*single_split=*/true, lm_fused ? &fl : nullptr)) != WD_OK)
+        if ((s = run_gemm(c, fp8 ? (const void*)c->xn8 : c->xn, fp8 ? &c->x8_d : &c->tc.x_map_d, lm, 1, NA, D, c->logits,
+                          (size_t)d.max_active * d.vocab, status, stream, &go, /*single_split=*/true,
+                          lm_fused ? &fl : nullptr, fp8 ? &f8lm : nullptr)) != WD_OK)
             return s;
         if (lm_fused) lm_chunks = fl.n_chunks;
         else wd_launch_rowstats(c->logits, NA, d.vocab, c->ch_max, c->ch_idx, c->ch_sum, stream);
@@ -1077,6 +1202,31 @@ extern "C" wd_status wd_generate(wd_state* st, int32_t A, int32_t B, int32_t R, 
 extern "C" size_t wd_op_gemm_scratch_bytes(int32_t rows, int32_t n_out, int32_t k_in) {
     if (rows < 1 || n_out < 1 || k_in < 1) return 0;
     return wd_tc_scratch_bytes(rows, n_out, k_in);
+}
+
+extern "C" size_t wd_op_gemm_fp8_scratch_bytes(int32_t rows, int32_t n_out, int32_t k_in) {
+    if (rows < 1 || n_out < 1 || k_in < 1) return 0;
+    return wd_align_up((size_t)rows * k_in, 256) + wd_align_up((size_t)rows * 4, 256) + wd_align_up((size_t)n_out * k_in, 256) +
+           wd_align_up((size_t)n_out * 4, 256) + wd_tc_scratch_bytes(rows, n_out, k_in);
+}
+
+extern "C" wd_status wd_op_gemm_fp8(const void* x, const void* w, float* y, int32_t rows, int32_t n_out, int32_t k_in,
+                                    void* scratch, size_t scratch_bytes, void* stream_) {
+    if (!x || !w || !y || !scratch) return WD_ERR_NULL;
+    if (rows < 1 || n_out < 1 || k_in < 16 || k_in % 16) return WD_ERR_BAD_PARAM;
+    if ((uintptr_t)scratch % 256) return WD_ERR_MISALIGNED;
+    if (scratch_bytes < wd_op_gemm_fp8_scratch_bytes(rows, n_out, k_in)) return WD_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    char* p = (char*)scratch;
+    uint8_t* xq = (uint8_t*)p; p += wd_align_up((size_t)rows * k_in, 256);
+    float* sx = (float*)p; p += wd_align_up((size_t)rows * 4, 256);
+    uint8_t* wq = (uint8_t*)p; p += wd_align_up((size_t)n_out * k_in, 256);
+    float* sw = (float*)p; p += wd_align_up((size_t)n_out * 4, 256);
+    wd_launch_quantize_rows(WD_BF16, x, rows, k_in, xq, sx, stream);
+    wd_launch_quantize_rows(WD_BF16, w, n_out, k_in, wq, sw, stream);
+    WD_CUDA_TRY(cudaGetLastError());
+    return wd_tc_gemm_standalone_fp8(xq, sx, wq, sw, y, rows, n_out, k_in, (float*)p, wd_tc_scratch_bytes(rows, n_out, k_in) / 4,
+                                     stream);
 }
 
 extern "C" wd_status wd_op_gemm(int32_t dtype, int32_t impl, const void* x, const void* w, float* y, int32_t rows,

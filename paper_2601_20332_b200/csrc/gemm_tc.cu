@@ -43,6 +43,10 @@ struct TcParams {
     // line then holds the weight tiles once (n_units, W count weight tiles), and the groups walk it
     // in step, so that a weight block fetched for one token tile is still in L2 for the others
     int tok_split;
+    // FP8 operands: K blocks of 128 elements, outputs scaled by sw[segment][n] * sx[token]
+    int fp8;
+    const float* sw[3];
+    const float* sx;
     int nseg, ncol;
     int seg_tile0[4];               // first tile index of each weight matrix (+ end)
     int seg_n[3];
@@ -302,11 +306,12 @@ __device__ void finalize_unit(const TcParams& p, long long G, int unit, int e) {
 // kWide: two weight halves per CTA (many tokens).  kLmStats: the LM-head epilogue that reduces
 // the logits to per-row statistics.  Separate instantiations keep the plain weight-streaming
 // kernel free of the other variants' code (its issue loops are sensitive to it).
-template <bool kWide, bool kLmStats>
+template <bool kWide, bool kLmStats, bool kFp8 = false>
 __global__ void __launch_bounds__(kWide ? kThreadsWide : kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w0,
                const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2,
                const TcParams p) {
+    constexpr int kKE = kFp8 ? 128 : kBK;                 // K elements per block: one 128-byte swizzle row
     extern __shared__ uint8_t smem_raw[];
     // 1024-byte alignment: required by the 128-byte swizzle atoms
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -391,16 +396,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             Walk w = w0;
             for (int i = 0; i < n_pre; ++i, advance(w)) {
                 mbar_expect_tx(smem_u32(&bars[i]), (uint32_t)stage_bytes);
-                tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes), w.mw, smem_u32(&bars[i]), w.kb * kBK, w.n0,
+                tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes), w.mw, smem_u32(&bars[i]), w.kb * kKE, w.n0,
                                  pol_stream);
                 if (kWide)
                     tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes) + kStageA, w.mw, smem_u32(&bars[i]),
-                                     w.kb * kBK, w.n0 + kBM, pol_stream);
+                                     w.kb * kKE, w.n0 + kBM, pol_stream);
             }
             pdl_wait();
             Walk wx = w0;
             for (int i = 0; i < n_pre; ++i, advance(wx))
-                tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + stage_a, &map_x, smem_u32(&bars[i]), wx.kb * kBK,
+                tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + stage_a, &map_x, smem_u32(&bars[i]), wx.kb * kKE,
                             wx.tok0);
             int s = n_pre % NS;
             uint32_t ph = (uint32_t)(n_pre / NS) & 1u;
@@ -413,9 +418,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 const uint32_t full = smem_u32(&bars[s]);
                 const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
                 mbar_expect_tx(full, (uint32_t)stage_bytes);
-                tma_load_2d_hint(sa, w.mw, full, w.kb * kBK, w.n0, pol_stream);
-                if (kWide) tma_load_2d_hint(sa + kStageA, w.mw, full, w.kb * kBK, w.n0 + kBM, pol_stream);
-                tma_load_2d(sa + stage_a, &map_x, full, w.kb * kBK, w.tok0);
+                tma_load_2d_hint(sa, w.mw, full, w.kb * kKE, w.n0, pol_stream);
+                if (kWide) tma_load_2d_hint(sa + kStageA, w.mw, full, w.kb * kKE, w.n0 + kBM, pol_stream);
+                tma_load_2d(sa + stage_a, &map_x, full, w.kb * kKE, w.tok0);
                 if (++s == NS) { s = 0; ph ^= 1u; }
             }
         }
@@ -447,8 +452,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 #pragma unroll
                     for (int kk = 0; kk < kBK / 16; ++kk) {
                         // 16 bf16 = 32 bytes further along K inside the swizzle row: +2 in 16-byte units
-                        umma_bf16(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
-                                  (j > 0 || kk > 0) ? 1u : 0u);
+                        if (kFp8)
+                            umma_f8(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
+                                    (j > 0 || kk > 0) ? 1u : 0u);
+                        else
+                            umma_bf16(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
+                                      (j > 0 || kk > 0) ? 1u : 0u);
                         if (kWide)
                             umma_bf16(acc + (uint32_t)p.buf_cols, adesc1 + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk),
                                       p.idesc, (j > 0 || kk > 0) ? 1u : 0u);
@@ -488,6 +497,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             if (!ok) break;
             tc_fence_after();
             float* yb = p.y + p.seg_col[u.seg] + n;
+            const float sw_n = (kFp8 && n_ok) ? p.sw[u.seg][n] : 1.f;      // FP8: scale of this weight row
             const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf + half_sel) * p.buf_cols);
             if constexpr (!kLmStats) {
                 for (int cc = 0; cc < p.bn; cc += 16) {
@@ -499,7 +509,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 #pragma unroll
                         for (int t = 0; t < 16; ++t) {
                             const int tok = u.tok0 + cc + t;
-                            if (tok < p.rows) ys[(size_t)tok * p.ncol] = __uint_as_float(v[t]);
+                            if (tok < p.rows)
+                                ys[(size_t)tok * p.ncol] = kFp8 ? __uint_as_float(v[t]) * sw_n * p.sx[tok] : __uint_as_float(v[t]);
                         }
                     }
                 }
@@ -520,6 +531,11 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     if (u.tok0 + cc >= p.rows) break;
                     uint32_t v[32];
                     tmem_ld32(t_acc + (uint32_t)cc, v);
+                    if (kFp8) {
+#pragma unroll
+                        for (int t = 0; t < 32; ++t)
+                            v[t] = __float_as_uint(__uint_as_float(v[t]) * sw_n * (u.tok0 + cc + t < p.rows ? p.sx[u.tok0 + cc + t] : 0.f));
+                    }
                     if (n_ok && p.f.write_logits) {
 #pragma unroll
                         for (int t = 0; t < 32; ++t)
@@ -643,10 +659,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 //             accumulators in BOTH CTAs (tcgen05.commit with a CTA mask)
 //   both:     TMA producer for their own operand halves, epilogue for their own 128 weight rows;
 //             epilogue threads of both CTAs arrive on the even CTA's "accumulator empty" barriers
+template <bool kFp8>
 __global__ void __launch_bounds__(kThreads)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w0,
                     const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2,
                     const TcParams p) {
+    constexpr int kKE = kFp8 ? 128 : kBK;                 // K elements per block
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int NS = p.n_stages;
@@ -731,13 +749,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
             for (int i = 0; i < n_pre; ++i, advance(w)) {
                 if (rank == 0) mbar_expect_tx(smem_u32(&bars[i]), 2u * (uint32_t)stage_bytes);
                 tma2_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes), w.mw, cluster_map(smem_u32(&bars[i]), 0),
-                                  w.kb * kBK, w.n0, pol_stream);
+                                  w.kb * kKE, w.n0, pol_stream);
             }
             pdl_wait();
             Walk wx = w0;
             for (int i = 0; i < n_pre; ++i, advance(wx))
                 tma2_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + stage_a, &map_x,
-                             cluster_map(smem_u32(&bars[i]), 0), wx.kb * kBK, wx.tok0);
+                             cluster_map(smem_u32(&bars[i]), 0), wx.kb * kKE, wx.tok0);
             int s = n_pre % NS;
             uint32_t ph = (uint32_t)(n_pre / NS) & 1u;
             for (int i = n_pre; i < n_total; ++i, advance(w)) {
@@ -749,8 +767,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 const uint32_t full = cluster_map(smem_u32(&bars[s]), 0);
                 const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
                 if (rank == 0) mbar_expect_tx(smem_u32(&bars[s]), 2u * (uint32_t)stage_bytes);
-                tma2_load_2d_hint(sa, w.mw, full, w.kb * kBK, w.n0, pol_stream);
-                tma2_load_2d(sa + stage_a, &map_x, full, w.kb * kBK, w.tok0);
+                tma2_load_2d_hint(sa, w.mw, full, w.kb * kKE, w.n0, pol_stream);
+                tma2_load_2d(sa + stage_a, &map_x, full, w.kb * kKE, w.tok0);
                 if (++s == NS) { s = 0; ph ^= 1u; }
             }
         }
@@ -778,9 +796,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                     const uint64_t adesc = make_sdesc(sa);
                     const uint64_t bdesc = make_sdesc(sa + stage_a);
 #pragma unroll
-                    for (int kk = 0; kk < kBK / 16; ++kk)
-                        umma2_bf16(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
-                                   (j > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < kBK / 16; ++kk) {
+                        if (kFp8)
+                            umma2_f8(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
+                                     (j > 0 || kk > 0) ? 1u : 0u);
+                        else
+                            umma2_bf16(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
+                                       (j > 0 || kk > 0) ? 1u : 0u);
+                    }
                     umma2_commit_mc(smem_u32(&bars[NS + s]), 3);          // stage free in both CTAs
                     if (++s == NS) { s = 0; ph ^= 1u; }
                 }
@@ -815,6 +838,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
             if (!ok) break;
             tc_fence_after();
             float* yb = p.y + p.seg_col[u.seg] + n;
+            const float sw_n = (kFp8 && n_ok) ? p.sw[u.seg][n] : 1.f;
             const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.buf_cols);
             for (int cc = 0; cc < p.bn; cc += 16) {
                 if (u.tok0 + cc >= p.rows) break;
@@ -825,7 +849,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 #pragma unroll
                     for (int t = 0; t < 16; ++t) {
                         const int tok = u.tok0 + cc + t;
-                        if (tok < p.rows) ys[(size_t)tok * p.ncol] = __uint_as_float(v[t]);
+                        if (tok < p.rows)
+                            ys[(size_t)tok * p.ncol] = kFp8 ? __uint_as_float(v[t]) * sw_n * p.sx[tok] : __uint_as_float(v[t]);
                     }
                 }
             }
@@ -899,6 +924,21 @@ wd_status encode_2d(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_
     return r == CUDA_SUCCESS ? WD_OK : WD_ERR_CUDA;
 }
 
+// [n_rows, K] bytes (e4m3 codes) row-major, box = 128 (K) x box_rows, 128-byte swizzle
+wd_status encode_2d8(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_rows) {
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return WD_ERR_CUDA;
+    if ((uintptr_t)ptr % 16 || K % 16) return WD_ERR_MISALIGNED;
+    cuuint64_t dims[2] = {(cuuint64_t)K, (cuuint64_t)n_rows};
+    cuuint64_t strides[1] = {(cuuint64_t)K};
+    cuuint32_t box[2] = {128u, (cuuint32_t)box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = enc(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                     CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? WD_OK : WD_ERR_CUDA;
+}
+
 struct TcConfig { int bn, tok_tiles, n_stages, buf_cols, ctas_per_sm, wide, tile_rows; size_t smem; };
 
 int env_int(const char* name, int dflt) {
@@ -941,11 +981,13 @@ int count_slices(int n_units, int kb_total, long long W, long long G) {
     return n;
 }
 
-uint32_t make_idesc(int bn, int m = kBM) {
+uint32_t make_idesc(int bn, int m = kBM, bool fp8 = false) {
     uint32_t d = 0;
     d |= 1u << 4;                      // D format: f32
-    d |= 1u << 7;                      // A format: bf16
-    d |= 1u << 10;                     // B format: bf16
+    if (!fp8) {
+        d |= 1u << 7;                  // A format: bf16 (kind::f8f6f4: 0 = e4m3)
+        d |= 1u << 10;                 // B format: bf16
+    }
     // bits 15 / 16: A and B are K-major (0)
     d |= (uint32_t)(bn >> 3) << 17;    // N
     d |= (uint32_t)(m >> 4) << 24;     // M (256: the two-CTA form)
@@ -954,9 +996,16 @@ uint32_t make_idesc(int bn, int m = kBM) {
 
 // launch of gemm_tc_pair_kernel: same contract as wd_tc_gemm
 wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, int K, float* y, size_t y_floats,
-                       int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out, bool force_single_split) {
+                       int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out, bool force_single_split,
+                       const WdTcFp8* fp8) {
     TcParams p;
     memset(&p, 0, sizeof(p));
+    if (fp8) {
+        p.fp8 = 1;
+        for (int i = 0; i < 3; ++i) p.sw[i] = fp8->sw[i < nseg ? i : 0];
+        p.sx = fp8->sx;
+    }
+    const int kke = fp8 ? 128 : kBK;
     p.tile_rows = 2 * kBM;
     p.tok_tiles = (rows + 255) / 256;
     p.bn = ((rows + p.tok_tiles - 1) / p.tok_tiles + 15) / 16 * 16;        // balanced token tiles, <= 256
@@ -981,7 +1030,7 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     p.nseg = nseg;
     p.ncol = col;
     p.rows = rows;
-    p.kb_total = (K + kBK - 1) / kBK;
+    p.kb_total = (K + kke - 1) / kke;
     // two token tiles: one group of pairs per token tile, walking the weight K blocks in step
     const int ts = (p.tok_tiles == 2 && (sm_count / 2) % 2 == 0) ? 2 : 1;
     p.tok_split = ts;
@@ -1007,21 +1056,22 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     p.y = y;
     p.split_stride = slice;
     p.status = status;
-    p.idesc = make_idesc(p.bn, 2 * kBM);
+    p.idesc = make_idesc(p.bn, 2 * kBM, fp8 != nullptr);
 
     CUtensorMap mx;
     bool hit = false;
     for (const WdTcX::Entry& e : x->cache)
         if (e.rows == rows && e.bn == half_bn) { mx = e.map; hit = true; break; }
     if (!hit) {
-        wd_status s = encode_2d(&mx, x->ptr, rows, K, half_bn);
+        wd_status s = fp8 ? encode_2d8(&mx, x->ptr, rows, K, half_bn) : encode_2d(&mx, x->ptr, rows, K, half_bn);
         if (s != WD_OK) return s;
         if (x->cache.size() >= 16) x->cache.erase(x->cache.begin());
         x->cache.push_back({rows, half_bn, mx});
     }
     static bool attr_done = false;      // one device per process
     if (!attr_done) {
-        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         attr_done = true;
     }
     const CUtensorMap& m0 = *segs[0].map;
@@ -1042,7 +1092,8 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     attr[1].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = wd_pdl_enabled ? 2 : 1;
-    WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_pair_kernel, mx, m0, m1, m2, p));
+    if (fp8) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_pair_kernel<true>, mx, m0, m1, m2, p));
+    else WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_pair_kernel<false>, mx, m0, m1, m2, p));
     if (n_split_out) *n_split_out = p.n_slices;
     return WD_OK;
 }
@@ -1077,23 +1128,34 @@ wd_status wd_tc_weights_init(WdTcWeights* tc, const wd_model_dims* d, const void
 
 wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, int K, float* y, size_t y_floats,
                      int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out, bool force_single_split,
-                     const WdTcFuse* fuse) {
+                     const WdTcFuse* fuse, const WdTcFp8* fp8) {
     if (!x || !segs || !y || !status || nseg < 1 || nseg > 3) return WD_ERR_BAD_PARAM;
     if (rows < 1 || K < 8 || K % 8) return WD_ERR_BAD_PARAM;
     TcParams p;
     memset(&p, 0, sizeof(p));
     const bool fused = fuse && fuse->mode != WD_FUSE_NONE;
+    if (fp8) {
+        if (K % 16 || !fp8->sx || (fused && fuse->mode != WD_FUSE_LMSTATS)) return WD_ERR_BAD_PARAM;
+        p.fp8 = 1;
+        for (int i = 0; i < 3; ++i) {
+            p.sw[i] = fp8->sw[i < nseg ? i : 0];
+            if (!p.sw[i]) return WD_ERR_NULL;
+        }
+        p.sx = fp8->sx;
+    }
+    const int kke = fp8 ? 128 : kBK;
     // Many tokens: CTA pairs on [256 x BN] tiles (tcgen05 cta_group::2)
     static const int pair_from = env_int("WD_GEMM_PAIR_FROM", 256);        // rows from which pairs are used; 0 = never
     if (!fused && pair_from > 0 && rows > pair_from && sm_count >= 2)
-        return tc_gemm_pair(x, segs, nseg, rows, K, y, y_floats, sm_count, status, stream, n_split_out, force_single_split);
+        return tc_gemm_pair(x, segs, nseg, rows, K, y, y_floats, sm_count, status, stream, n_split_out, force_single_split,
+                            fp8);
     // The wide tile halves the operand traffic per flop but has a shallower ring and an epilogue
     // that does not overlap the next tile: it pays once every CTA gets at least one whole tile.
     long long wide_units = 0;
     for (int i = 0; i < nseg; ++i) wide_units += (segs[i].n + 2 * kBM - 1) / (2 * kBM);
     wide_units *= (rows + 255) / 256;
     static const int wide_min_units = env_int("WD_GEMM_WIDE_MIN_UNITS", 0);     // tuning knob; 0 = one unit per SM
-    const TcConfig cfg = pick_config(rows, !fused && wide_units >= (wide_min_units > 0 ? wide_min_units : sm_count),
+    const TcConfig cfg = pick_config(rows, !fused && !fp8 && wide_units >= (wide_min_units > 0 ? wide_min_units : sm_count),
                                      fuse && fuse->mode == WD_FUSE_LMSTATS);
     p.wide = cfg.wide;
     p.tile_rows = cfg.tile_rows;
@@ -1110,7 +1172,7 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     p.nseg = nseg;
     p.ncol = col;
     p.rows = rows; p.bn = cfg.bn;
-    p.kb_total = (K + kBK - 1) / kBK;
+    p.kb_total = (K + kke - 1) / kke;
     p.tok_tiles = cfg.tok_tiles;
     // Two or four token tiles: one group of CTAs per token tile, all groups walking the same line of
     // weight K blocks in step, so a weight block comes from HBM once and from L2 for the other groups
@@ -1143,7 +1205,7 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     p.y = y;
     p.split_stride = slice;
     p.status = status;
-    p.idesc = make_idesc(cfg.bn);
+    p.idesc = make_idesc(cfg.bn, kBM, fp8 != nullptr);
     if (fuse) {
         p.f = *fuse;
         if (fuse->mode != WD_FUSE_NONE && fuse->mode != WD_FUSE_LMSTATS && !fuse->counters) return WD_ERR_NULL;
@@ -1160,7 +1222,7 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     for (const WdTcX::Entry& e : x->cache)
         if (e.rows == rows && e.bn == cfg.bn) { mx = e.map; hit = true; break; }
     if (!hit) {
-        wd_status s = encode_2d(&mx, x->ptr, rows, K, cfg.bn);
+        wd_status s = fp8 ? encode_2d8(&mx, x->ptr, rows, K, cfg.bn) : encode_2d(&mx, x->ptr, rows, K, cfg.bn);
         if (s != WD_OK) return s;
         if (x->cache.size() >= 16) x->cache.erase(x->cache.begin());
         x->cache.push_back({rows, cfg.bn, mx});
@@ -1170,6 +1232,8 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
         WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        WD_CUDA_TRY(cudaFuncSetAttribute((gemm_tc_kernel<false, false, true>), cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        WD_CUDA_TRY(cudaFuncSetAttribute((gemm_tc_kernel<false, true, true>), cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         attr_done = true;
     }
     const CUtensorMap& m0 = *segs[0].map;
@@ -1186,11 +1250,17 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = attr;
     lc.numAttrs = wd_pdl_enabled ? 1 : 0;
-    if (cfg.wide) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<true, false>, mx, m0, m1, m2, p));
+    if (fp8 && p.f.mode == WD_FUSE_LMSTATS) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, (gemm_tc_kernel<false, true, true>), mx, m0, m1, m2, p));
+    else if (fp8) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, (gemm_tc_kernel<false, false, true>), mx, m0, m1, m2, p));
+    else if (cfg.wide) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<true, false>, mx, m0, m1, m2, p));
     else if (p.f.mode == WD_FUSE_LMSTATS) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<false, true>, mx, m0, m1, m2, p));
     else WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<false, false>, mx, m0, m1, m2, p));
     if (n_split_out) *n_split_out = p.n_slices;
     return WD_OK;
+}
+
+wd_status wd_tc_encode_fp8(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_rows) {
+    return encode_2d8(m, ptr, n_rows, K, box_rows);
 }
 
 size_t wd_tc_scratch_bytes(int rows, int n_out, int k_in) {
@@ -1224,6 +1294,35 @@ wd_status wd_tc_gemm_standalone(const void* x, const void* w, float* y, int rows
     const int blocks = (int)((slice + 255) / 256 < 1184 ? (slice + 255) / 256 : 1184);
     ++wd_launch_counter;
     reduce_slices_kernel<<<blocks, 256, 0, stream>>>((const float*)scratch, ns, slice, y, slice);
+    WD_CUDA_TRY(cudaGetLastError());
+    return WD_OK;
+}
+
+// FP8 single operation: operands already quantised (codes + row scales); slices: room for the partial sums
+wd_status wd_tc_gemm_standalone_fp8(const uint8_t* xq, const float* sx, const uint8_t* wq, const float* sw, float* y,
+                                    int rows, int n_out, int k_in, float* slices, size_t slice_floats, cudaStream_t stream) {
+    if (k_in % 16) return WD_ERR_BAD_PARAM;
+    int32_t* status = wd_op_status_ptr();
+    if (!status) return WD_ERR_CUDA;
+    CUtensorMap mw;
+    wd_status s = encode_2d8(&mw, wq, n_out, k_in, kBM);
+    if (s != WD_OK) return s;
+    WdTcSeg seg = {wq, n_out, &mw};
+    WdTcX xm;
+    xm.ptr = xq; xm.K = k_in; xm.fp8 = 1;
+    WdTcFp8 f8;
+    f8.sw[0] = sw; f8.sx = sx;
+    int sm = 148, dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
+    const size_t slice = (size_t)rows * n_out;
+    if (slice_floats < slice) return WD_ERR_WORKSPACE_TOO_SMALL;
+    int ns = 1;
+    s = wd_tc_gemm(&xm, &seg, 1, rows, k_in, slices, slice_floats, sm, status, stream, &ns, false, nullptr, &f8);
+    if (s != WD_OK) return s;
+    const int blocks = (int)((slice + 255) / 256 < 1184 ? (slice + 255) / 256 : 1184);
+    ++wd_launch_counter;
+    reduce_slices_kernel<<<blocks, 256, 0, stream>>>(slices, ns, slice, y, slice);
     WD_CUDA_TRY(cudaGetLastError());
     return WD_OK;
 }

@@ -21,6 +21,7 @@ struct WdTcSeg {
 struct WdTcX {
     const void* ptr = nullptr;
     int K = 0;
+    int fp8 = 0;             // byte matrix of e4m3 codes
     // descriptors already encoded for this operand, keyed by (rows, token tile): the same few
     // shapes come back every step
     struct Entry { int rows, bn; CUtensorMap map; };
@@ -83,12 +84,24 @@ struct WdTcFuse {
     int write_logits = 0;
 };
 
+// FP8 operands (e4m3 codes, one float scale per weight row and per activation row): the maps of
+// the segments and of x then describe byte matrices (box 128 (K) x rows), K is still the number
+// of elements, and every output is multiplied by sw[segment][n] * sx[row] in the epilogue.
+struct WdTcFp8 {
+    const float* sw[3] = {nullptr, nullptr, nullptr};
+    const float* sx = nullptr;
+};
+
 // y[split][rows][sum n_i] = x * [w_0; w_1; ...]^T, split-K partial sums side by side
 // (split_stride = rows * sum n_i floats).  The consumer adds the slices.
 wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, int K, float* y, size_t y_floats,
                      int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out,
-                     bool force_single_split = false, const WdTcFuse* fuse = nullptr);
+                     bool force_single_split = false, const WdTcFuse* fuse = nullptr, const WdTcFp8* fp8 = nullptr);
+// TMA descriptor of a [n_rows, K] byte matrix for the FP8 path (box 128 x box_rows)
+wd_status wd_tc_encode_fp8(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_rows);
 
 size_t wd_tc_scratch_bytes(int rows, int n_out, int k_in);
 wd_status wd_tc_gemm_standalone(const void* x, const void* w, float* y, int rows, int n_out, int k_in, void* scratch,
                                 size_t scratch_bytes, cudaStream_t stream);
+wd_status wd_tc_gemm_standalone_fp8(const uint8_t* xq, const float* sx, const uint8_t* wq, const float* sw, float* y,
+                                    int rows, int n_out, int k_in, float* slices, size_t slice_floats, cudaStream_t stream);

@@ -8,6 +8,8 @@
 #include <cstring>
 #include <utility>
 
+#include <cuda_fp8.h>
+
 #include "wd_internal.h"
 #include "device_utils.cuh"
 
@@ -330,10 +332,19 @@ template <> struct Vec4<__nv_bfloat16> {
     }
 };
 
+// four floats -> four e4m3 codes (round to nearest even, saturating), lowest byte first
+__device__ __forceinline__ uint32_t pack_e4m3(float a, float b, float c, float d) {
+    return (uint32_t)__nv_cvt_float_to_fp8(a, __NV_SATFINITE, __NV_E4M3) |
+           ((uint32_t)__nv_cvt_float_to_fp8(b, __NV_SATFINITE, __NV_E4M3) << 8) |
+           ((uint32_t)__nv_cvt_float_to_fp8(c, __NV_SATFINITE, __NV_E4M3) << 16) |
+           ((uint32_t)__nv_cvt_float_to_fp8(d, __NV_SATFINITE, __NV_E4M3) << 24);
+}
+
 template <typename T, int MAXV>
 __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
                                size_t split_stride, const float* __restrict__ gain, float eps,
-                               T* __restrict__ xn, const int32_t* __restrict__ row_idx, int d) {
+                               T* __restrict__ xn, const int32_t* __restrict__ row_idx, int d,
+                               uint8_t* __restrict__ xq, float* __restrict__ sx) {
     __shared__ float red[32];
     pdl_launch_dependents();
     pdl_wait();
@@ -366,6 +377,28 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ 
     }
     ss = block_sum(ss, red);
     const float inv = rsqrtf(ss / (float)d + eps);
+    if (xq) {
+        // FP8 output: e4m3 codes of (value / s) with s = max |value| / 448 of this row (1 for a zero row)
+        float amax = 0.f;
+#pragma unroll
+        for (int u = 0; u < MAXV; ++u) {
+            const int c4 = threadIdx.x + u * blockDim.x;
+            if (c4 < nv) {
+                const float4 g = reinterpret_cast<const float4*>(gain)[c4];
+                v[u] = make_float4(v[u].x * inv * g.x, v[u].y * inv * g.y, v[u].z * inv * g.z, v[u].w * inv * g.w);
+                amax = fmaxf(fmaxf(fmaxf(amax, fabsf(v[u].x)), fmaxf(fabsf(v[u].y), fabsf(v[u].z))), fabsf(v[u].w));
+            }
+        }
+        amax = block_max(amax, red);
+        const float s = amax > 0.f ? amax / 448.f : 1.f;
+        if (threadIdx.x == 0) sx[i] = s;
+#pragma unroll
+        for (int u = 0; u < MAXV; ++u) {
+            const int c4 = threadIdx.x + u * blockDim.x;
+            if (c4 < nv) reinterpret_cast<uint32_t*>(xq + (size_t)i * d)[c4] = pack_e4m3(v[u].x / s, v[u].y / s, v[u].z / s, v[u].w / s);
+        }
+        return;
+    }
 #pragma unroll
     for (int u = 0; u < MAXV; ++u) {
         const int c4 = threadIdx.x + u * blockDim.x;
@@ -603,6 +636,55 @@ __global__ void swiglu_kernel(const float* __restrict__ part, int n_split, size_
     }
 }
 
+// FP8 variant: one block per row keeps the whole row h = silu(gate) * up in registers (up to kMaxV
+// float4 per thread), takes its maximum, and writes e4m3 codes and the row's scale.
+template <int kMaxV>
+__global__ void swiglu_fp8_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
+                                  uint8_t* __restrict__ hq, float* __restrict__ sh, int F) {
+    __shared__ float red[32];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int r = blockIdx.x, f4 = F >> 2;
+    const float* pr = part + (size_t)r * 2 * F;
+    float4 hv[kMaxV];
+    float amax = 0.f;
+#pragma unroll
+    for (int u = 0; u < kMaxV; ++u) {
+        const int c4 = threadIdx.x + u * blockDim.x;
+        hv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c4 < f4) {
+            const float4 g = sum_slices4(pr + 4 * c4, n_split, split_stride);
+            const float4 up = sum_slices4(pr + F + 4 * c4, n_split, split_stride);
+            hv[u] = make_float4(g.x / (1.f + __expf(-g.x)) * up.x, g.y / (1.f + __expf(-g.y)) * up.y,
+                                g.z / (1.f + __expf(-g.z)) * up.z, g.w / (1.f + __expf(-g.w)) * up.w);
+            amax = fmaxf(fmaxf(fmaxf(amax, fabsf(hv[u].x)), fmaxf(fabsf(hv[u].y), fabsf(hv[u].z))), fabsf(hv[u].w));
+        }
+    }
+    amax = block_max(amax, red);
+    const float s = amax > 0.f ? amax / 448.f : 1.f;
+    if (threadIdx.x == 0) sh[r] = s;
+#pragma unroll
+    for (int u = 0; u < kMaxV; ++u) {
+        const int c4 = threadIdx.x + u * blockDim.x;
+        if (c4 < f4) reinterpret_cast<uint32_t*>(hq + (size_t)r * F)[c4] = pack_e4m3(hv[u].x / s, hv[u].y / s, hv[u].z / s, hv[u].w / s);
+    }
+}
+
+// Per-row e4m3 quantisation of a [n_rows, K] matrix (weights once at set-up; K % 4 == 0): one block per row
+template <typename T>
+__global__ void quantize_rows_kernel(const T* __restrict__ w, int K, uint8_t* __restrict__ q, float* __restrict__ s_out) {
+    __shared__ float red[32];
+    const T* wr = w + (size_t)blockIdx.x * K;
+    float amax = 0.f;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) amax = fmaxf(amax, fabsf(to_f(wr[k])));
+    amax = block_max(amax, red);
+    const float s = amax > 0.f ? amax / 448.f : 1.f;
+    if (threadIdx.x == 0) s_out[blockIdx.x] = s;
+    for (int k4 = threadIdx.x; k4 < (K >> 2); k4 += blockDim.x)
+        reinterpret_cast<uint32_t*>(q + (size_t)blockIdx.x * K)[k4] =
+            pack_e4m3(to_f(wr[4 * k4]) / s, to_f(wr[4 * k4 + 1]) / s, to_f(wr[4 * k4 + 2]) / s, to_f(wr[4 * k4 + 3]) / s);
+}
+
 // total is a multiple of 4 (d is)
 __global__ void residual_add_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
                                     size_t split_stride, float* __restrict__ tap, size_t total) {
@@ -786,7 +868,7 @@ void wd_launch_embed_fused(const void* embed, const int32_t* ids, const int32_t*
 
 void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size_t split_stride,
                        const float* gain, float eps, void* xn, const int32_t* row_idx, int n_rows,
-                       int d, cudaStream_t st) {
+                       int d, cudaStream_t st, uint8_t* xq, float* sx) {
     if (n_rows <= 0) return;
     // one float4 per thread where the row allows it: the kernel is a chain of dependent L2 round
     // trips, so short per-thread work matters more than occupancy
@@ -795,17 +877,17 @@ void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size
         // many rows: bandwidth matters, so more (smaller) blocks per SM with four float4 in flight per thread
         const int threads = ((nv + 3) / 4 + 31) / 32 * 32;
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 4>, dim3(n_rows), dim3(threads), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
     } else if (nv <= 1024) {
         const int threads = (nv + 31) / 32 * 32;
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 1>, dim3(n_rows), dim3(threads), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
     } else if (nv <= 2048) {
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 2>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
     } else {
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 8>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
     }
 }
 
@@ -859,6 +941,23 @@ void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_st
     const int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     WD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, dim3(blocks), dim3(256), 0, st, part, n_split, split_stride,
                                   (T*)h, n_rows, F));
+}
+
+wd_status wd_launch_swiglu_fp8(const float* part, int n_split, size_t split_stride, uint8_t* hq, float* sh, int n_rows,
+                               int F, cudaStream_t st) {
+    if (n_rows <= 0) return WD_OK;
+    const int f4 = F >> 2;
+    if (F % 4 || f4 > 8 * 1024) return WD_ERR_BAD_PARAM;
+    int threads = ((f4 + 7) / 8 + 31) / 32 * 32;
+    if (threads < 256) threads = f4 < 256 ? (f4 + 31) / 32 * 32 : 256;
+    launch_pdl(swiglu_fp8_kernel<8>, dim3(n_rows), dim3(threads), 0, st, part, n_split, split_stride, hq, sh, F);
+    return WD_OK;
+}
+
+void wd_launch_quantize_rows(int dtype, const void* w, int n_rows, int K, uint8_t* q, float* s, cudaStream_t st) {
+    if (n_rows <= 0) return;
+    WD_DISPATCH(dtype, (quantize_rows_kernel<T><<<n_rows, 256, 0, st>>>((const T*)w, K, q, s)));
+    ++wd_launch_counter;
 }
 
 void wd_launch_residual_add(float* x, const float* part, int n_split, size_t split_stride,

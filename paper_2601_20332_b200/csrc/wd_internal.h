@@ -92,7 +92,8 @@ void wd_launch_embed_fused(const void* embed, const int32_t* ids, const int32_t*
 // and xn[i] is written: used for the final norm over the active rows only.  d % 4 == 0.
 void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size_t split_stride,
                        const float* gain, float eps, void* xn, const int32_t* row_idx, int n_rows,
-                       int d, cudaStream_t st);
+                       int d, cudaStream_t st, uint8_t* xq = nullptr, float* sx = nullptr);
+// (xq != null: FP8 output instead of xn: e4m3 codes [n_rows][d] and one scale per row)
 
 // plain GEMM: y[rows, n] (float) = x[rows,k] * w[n,k]^T
 void wd_launch_gemm_plain(int dtype, const void* x, const void* w, float* y, int rows, int n, int k,
@@ -118,6 +119,12 @@ void wd_launch_attention_plain(int dtype, const void* q, const void* kcache, con
 // h = silu(gate) * up from partials [n_split][n_rows][2F] (columns = [gate | up]); F % 4 == 0
 void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_stride, void* h,
                       int n_rows, int F, cudaStream_t st);
+
+// FP8: h as e4m3 codes [n_rows][F] with one scale per row (F <= 32768)
+wd_status wd_launch_swiglu_fp8(const float* part, int n_split, size_t split_stride, uint8_t* hq, float* sh, int n_rows,
+                               int F, cudaStream_t st);
+// per-row e4m3 quantisation of a [n_rows, K] matrix of `dtype` (K % 4 == 0): codes and scales
+void wd_launch_quantize_rows(int dtype, const void* w, int n_rows, int K, uint8_t* q, float* s, cudaStream_t st);
 
 // x += sum_s part[s]; optionally copy x to tap.
 void wd_launch_residual_add(float* x, const float* part, int n_split, size_t split_stride,

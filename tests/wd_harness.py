@@ -33,7 +33,7 @@ def max_rel(a, b):
 
 class Parity:
     def __init__(self, cfg, weights, ids, decoded=None, gemm_impl=wd.WD_GEMM_AUTO, oracle_seqs=None,
-                 max_rows=None, max_active=None, fusion=False, eos_id=None, refresh_mode=0):
+                 max_rows=None, max_active=None, fusion=False, eos_id=None, refresh_mode=0, fp8=False):
         self.cfg = cfg
         self.batch, self.S = ids.shape
         dev = weights.tok_embed.device
@@ -42,6 +42,8 @@ class Parity:
         self.ctx = wd.Context(cfg, weights, self.batch, self.S, max_rows, max_active)
         self.ctx.set_gemm_impl(gemm_impl)
         self.ctx.set_fusion(fusion)
+        if fp8:
+            self.ctx.fp8_enable()
         self.st = wd.State(self.ctx, ids, decoded)
         if eos_id is not None:
             self.st.set_eos(eos_id)
@@ -53,6 +55,8 @@ class Parity:
         self.t_logits = torch.zeros(max_active * V, dtype=torch.float32, device=dev)
         self.st.set_taps(self.t_layer, self.t_attn, self.t_logits)
         self.model = synth.OracleModelView(weights)
+        if fp8:
+            self.model.dims = dict(self.model.dims, fp8=True)
         self.oracle_seqs = list(range(self.batch)) if oracle_seqs is None else list(oracle_seqs)
         dec = (ids != cfg["mask_id"]) if decoded is None else decoded.astype(bool)
         self.ost = [wo.SeqState(ids=ids[b], decoded=dec[b], eos_id=eos_id, refresh_mode=refresh_mode)
