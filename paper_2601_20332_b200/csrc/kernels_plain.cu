@@ -636,37 +636,65 @@ __global__ void swiglu_kernel(const float* __restrict__ part, int n_split, size_
     }
 }
 
-// FP8 variant: one block per row keeps the whole row h = silu(gate) * up in registers (up to kMaxV
-// float4 per thread), takes its maximum, and writes e4m3 codes and the row's scale.
+// FP8 variant: a cluster of four 256-thread blocks per row (light blocks, so that they are resident
+// and waiting while the GEMM still runs); each keeps its quarter of h = silu(gate) * up in registers
+// (up to kMaxV float4 per thread), the four partial maxima meet through distributed shared memory,
+// then every block writes the e4m3 codes of its quarter (and block 0 the row's scale).
 template <int kMaxV>
 __global__ void swiglu_fp8_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
                                   uint8_t* __restrict__ hq, float* __restrict__ sh, int F) {
     __shared__ float red[32];
+    __shared__ float my_max;
     pdl_launch_dependents();
     pdl_wait();
-    const int r = blockIdx.x, f4 = F >> 2;
+    const int r = blockIdx.x >> 2, quarter = blockIdx.x & 3, f4 = F >> 2;
+    const int q4 = (f4 + 3) >> 2, c_lo = quarter * q4, c_hi = min(f4, c_lo + q4);     // this block's float4 columns
     const float* pr = part + (size_t)r * 2 * F;
-    float4 hv[kMaxV];
+    // slice by slice, all of this thread's positions at once: 2 * kMaxV loads in flight per round trip
+    float4 g[kMaxV], up[kMaxV];
+#pragma unroll
+    for (int u = 0; u < kMaxV; ++u) g[u] = up[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int sl = 0; sl < n_split; ++sl) {
+        const float* ps = pr + (size_t)sl * split_stride;
+        float4 tg[kMaxV], tu[kMaxV];
+#pragma unroll
+        for (int u = 0; u < kMaxV; ++u) {
+            const int c4 = c_lo + (int)threadIdx.x + u * (int)blockDim.x;
+            tg[u] = tu[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (c4 < c_hi) {
+                tg[u] = *reinterpret_cast<const float4*>(ps + 4 * c4);
+                tu[u] = *reinterpret_cast<const float4*>(ps + F + 4 * c4);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kMaxV; ++u) {
+            g[u].x += tg[u].x; g[u].y += tg[u].y; g[u].z += tg[u].z; g[u].w += tg[u].w;
+            up[u].x += tu[u].x; up[u].y += tu[u].y; up[u].z += tu[u].z; up[u].w += tu[u].w;
+        }
+    }
     float amax = 0.f;
 #pragma unroll
     for (int u = 0; u < kMaxV; ++u) {
-        const int c4 = threadIdx.x + u * blockDim.x;
-        hv[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (c4 < f4) {
-            const float4 g = sum_slices4(pr + 4 * c4, n_split, split_stride);
-            const float4 up = sum_slices4(pr + F + 4 * c4, n_split, split_stride);
-            hv[u] = make_float4(g.x / (1.f + __expf(-g.x)) * up.x, g.y / (1.f + __expf(-g.y)) * up.y,
-                                g.z / (1.f + __expf(-g.z)) * up.z, g.w / (1.f + __expf(-g.w)) * up.w);
-            amax = fmaxf(fmaxf(fmaxf(amax, fabsf(hv[u].x)), fmaxf(fabsf(hv[u].y), fabsf(hv[u].z))), fabsf(hv[u].w));
-        }
+        g[u] = make_float4(g[u].x / (1.f + __expf(-g[u].x)) * up[u].x, g[u].y / (1.f + __expf(-g[u].y)) * up[u].y,
+                           g[u].z / (1.f + __expf(-g[u].z)) * up[u].z, g[u].w / (1.f + __expf(-g[u].w)) * up[u].w);
+        amax = fmaxf(fmaxf(fmaxf(amax, fabsf(g[u].x)), fmaxf(fabsf(g[u].y), fabsf(g[u].z))), fabsf(g[u].w));
     }
     amax = block_max(amax, red);
+    if (threadIdx.x == 0) my_max = amax;
+    wdk::cluster_sync();                            // the four partial maxima are in place
+    const uint32_t local = wdk::smem_u32(&my_max);
+    for (uint32_t k = 0; k < 4; ++k) {
+        float v;
+        asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(wdk::cluster_map(local, k)));
+        amax = fmaxf(amax, v);
+    }
+    wdk::cluster_sync();                            // nobody leaves while its maximum may still be read
     const float s = amax > 0.f ? amax / 448.f : 1.f;
-    if (threadIdx.x == 0) sh[r] = s;
+    if (threadIdx.x == 0 && quarter == 0) sh[r] = s;
 #pragma unroll
     for (int u = 0; u < kMaxV; ++u) {
-        const int c4 = threadIdx.x + u * blockDim.x;
-        if (c4 < f4) reinterpret_cast<uint32_t*>(hq + (size_t)r * F)[c4] = pack_e4m3(hv[u].x / s, hv[u].y / s, hv[u].z / s, hv[u].w / s);
+        const int c4 = c_lo + (int)threadIdx.x + u * (int)blockDim.x;
+        if (c4 < c_hi) reinterpret_cast<uint32_t*>(hq + (size_t)r * F)[c4] = pack_e4m3(g[u].x / s, g[u].y / s, g[u].z / s, g[u].w / s);
     }
 }
 
@@ -948,9 +976,26 @@ wd_status wd_launch_swiglu_fp8(const float* part, int n_split, size_t split_stri
     if (n_rows <= 0) return WD_OK;
     const int f4 = F >> 2;
     if (F % 4 || f4 > 8 * 1024) return WD_ERR_BAD_PARAM;
-    int threads = ((f4 + 7) / 8 + 31) / 32 * 32;
-    if (threads < 256) threads = f4 < 256 ? (f4 + 31) / 32 * 32 : 256;
-    launch_pdl(swiglu_fp8_kernel<8>, dim3(n_rows), dim3(threads), 0, st, part, n_split, split_stride, hq, sh, F);
+    ++wd_launch_counter;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(4 * n_rows);
+    lc.blockDim = dim3(256);
+    lc.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 4;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = wd_pdl_enabled ? 2 : 1;
+    const int per_thread = ((f4 + 3) / 4 + 255) / 256;          // float4 per thread
+    cudaError_t e;
+    if (per_thread <= 3) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<3>, part, n_split, split_stride, hq, sh, F);
+    else if (per_thread <= 5) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<5>, part, n_split, split_stride, hq, sh, F);
+    else e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<8>, part, n_split, split_stride, hq, sh, F);
+    if (e != cudaSuccess) { wd_note_cuda_error(e, __FILE__, __LINE__); return WD_ERR_CUDA; }
     return WD_OK;
 }
 
