@@ -492,6 +492,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             const bool n_ok = n < p.seg_n[u.seg];
             int ord = 0;
             if (!p.aligned) ord = (int)(c - (((long long)unit * p.kb_total + 1) * G - 1) / p.W);
+            // FP8: the row scales of this token tile go to shared memory while the MMAs still run
+            float* sx_s = lm_scratch + (kLmStats ? 5664 : 0);
+            if (kFp8) {
+                epi_sync();                                        // the previous piece's readers are done
+                for (int i = (int)threadIdx.x - 64; i < ((p.bn + 31) & ~31); i += 128)
+                    sx_s[i] = (i < p.bn && u.tok0 + i < p.rows) ? p.sx[u.tok0 + i] : 0.f;
+                epi_sync();
+            }
             ok = ok && mbar_wait(smem_u32(&bars[2 * NS + buf]), par, abort_flag);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -510,7 +518,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                         for (int t = 0; t < 16; ++t) {
                             const int tok = u.tok0 + cc + t;
                             if (tok < p.rows)
-                                ys[(size_t)tok * p.ncol] = kFp8 ? __uint_as_float(v[t]) * sw_n * p.sx[tok] : __uint_as_float(v[t]);
+                                ys[(size_t)tok * p.ncol] = kFp8 ? __uint_as_float(v[t]) * sw_n * sx_s[cc + t] : __uint_as_float(v[t]);
                         }
                     }
                 }
@@ -534,7 +542,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     if (kFp8) {
 #pragma unroll
                         for (int t = 0; t < 32; ++t)
-                            v[t] = __float_as_uint(__uint_as_float(v[t]) * sw_n * (u.tok0 + cc + t < p.rows ? p.sx[u.tok0 + cc + t] : 0.f));
+                            v[t] = __float_as_uint(__uint_as_float(v[t]) * sw_n * sx_s[cc + t]);
                     }
                     if (n_ok && p.f.write_logits) {
 #pragma unroll
