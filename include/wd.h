@@ -259,7 +259,7 @@ WD_API wd_status wd_state_set_refresh_mode(wd_state* st, int32_t mode);
  * value (ties to even), multiplied on the tensor cores (tcgen05 kind::f8f6f4, fp32 accumulation)
  * and scaled back by the two row scales.  The output projection, attention, the residual stream
  * and the K/V cache stay as they are.  Halves the weight bytes a normal step streams; changes the
- * numbers (relative error of a projection around 3-4 %).  bf16 models on the tensor-core path only.
+ * numbers (relative error of a projection about 3-4 %).  bf16 models on the tensor-core path only.
  *   wd_fp8_bytes   size of the device memory block wd_fp8_enable needs (0 for invalid dims / fp32)
  *   wd_fp8_enable  quantises the weights on `stream` into `mem` (caller-owned, 256-byte aligned,
  *                  must outlive the context) and switches the mode on for later steps.
