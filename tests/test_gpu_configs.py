@@ -25,14 +25,18 @@ def built():
     wd_build.build()
 
 
-def run_cfg(cfg, n_steps, oracle_seqs=None, ids=None, decoded=None):
+def run_cfg(cfg, n_steps, oracle_seqs=None, ids=None, decoded=None, refresh_mode=0, fp8=False, tol=None):
     w = synth.make_weights(cfg, DEV)
     ids = synth.make_prompts(cfg) if ids is None else ids
     batch, S = ids.shape
-    p = Parity(cfg, w, ids, decoded, oracle_seqs=oracle_seqs, max_rows=batch * S, max_active=batch * cfg["A"])
+    p = Parity(cfg, w, ids, decoded, oracle_seqs=oracle_seqs, max_rows=batch * S, max_active=batch * cfg["A"],
+               refresh_mode=refresh_mode, fp8=fp8)
     logs = []
     for _ in range(n_steps):
-        logs.append(p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"]))
+        if tol is None:
+            logs.append(p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"]))
+        else:
+            logs.append(p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"], tol_layer=tol[0], tol_attn=tol[1]))
     p.check_state_mirror()
     p.close()
     del w
@@ -78,3 +82,22 @@ def test_cfg5_sweep_corner_late_state():
     logs = run_cfg(cfg, 3, oracle_seqs=[1], ids=ids, decoded=dec)
     assert logs[0]["info"]["n_rows"] == 2 * (1024 + 640 + 384)
     assert logs[1]["info"]["n_rows"] == 2 * 129 and logs[1]["info"]["n_vis"] == 2 * 2048
+
+
+def test_cfg2_window_only_refresh_variant_at_full_width():
+    """The variant outside the paper at the LLaDA-8B width: the second refresh computes the new
+    window and the previous phase's tokens only (104 rows instead of 360)."""
+    cfg = synth.get_config("llada8b", L=1)
+    logs = run_cfg(cfg, 9, refresh_mode=wd.WD_REFRESH_WINDOW)
+    assert [l["info"]["is_refresh"] for l in logs] == [1, 0, 0, 0, 0, 0, 0, 0, 1]
+    assert logs[0]["info"]["n_rows"] == 352 and logs[8]["info"]["n_rows"] == 96 + 8 and logs[8]["info"]["n_vis"] == 360
+
+
+def test_cfg2_and_cfg4_fp8_projections_at_full_width():
+    """FP8 mode (outside the paper) at the real widths: LLaDA-8B shape (vocabulary 126464 through
+    the FP8 LM-head epilogue) and the Dream-7B shape (GQA, batch 8, d_ffn 18944, two-CTA FP8
+    GEMMs at 5376 rows); tolerances as derived in test_gpu_step."""
+    logs = run_cfg(synth.get_config("llada8b", L=1), 3, fp8=True, tol=(5e-2, 1e-1))
+    assert logs[0]["info"]["n_rows"] == 352 and logs[1]["info"]["n_rows"] == 33
+    logs = run_cfg(synth.get_config("dream7b", L=1), 2, oracle_seqs=[3], fp8=True, tol=(5e-2, 1e-1))
+    assert logs[0]["info"]["n_rows"] == 8 * 672 and logs[1]["info"]["n_rows"] == 8 * 33
