@@ -135,7 +135,6 @@ def run_ours(args, rank, world):
     A, B, R, T, k, batch = (cfg[x] for x in ("A", "B", "R", "T", "k", "batch"))
     S = cfg["P"] + cfg["G"]
     K, W = args.steps, args.warmup
-    assert W + K <= cfg["G"] // k, "steps + warmup exceed the generation length"
     w = synth.make_weights(cfg, dev)
     ids = synth.make_prompts(cfg)
     ctx = wd.Context(cfg, w, batch, S, batch * S, batch * max(A, cfg["G"]))
@@ -147,9 +146,25 @@ def run_ours(args, rank, world):
         `QUEUE` steps; otherwise every step is followed by a sync."""
         QUEUE = 16
         infos, per_step = [], []
+        pending = [False]
+
+        def one_step():
+            # a generation that runs out of masks starts again from the prompt (the first step of
+            # the new generation is a refresh like any other)
+            status, info = state.step(A, B, R, T, k, stream)
+            if status == wd.WD_DONE:
+                if pending[0]:
+                    state.sync()
+                    pending[0] = False
+                state.reset(ids, None, stream)
+                status, info = state.step(A, B, R, T, k, stream)
+            pending[0] = True
+            return info
+
         for i in range(n_warm):
-            state.step(A, B, R, T, k, stream)
+            one_step()
             state.sync()
+            pending[0] = False
         if world > 1:
             torch.distributed.barrier()
         torch.cuda.synchronize()
@@ -157,10 +172,11 @@ def run_ours(args, rank, world):
         t0 = time.perf_counter()
         ev[0].record(stream)
         for i in range(n_timed):
-            _, info = state.step(A, B, R, T, k, stream)
+            info = one_step()
             ev[i + 1].record(stream)
             if not queued or (i + 1) % QUEUE == 0 or i + 1 == n_timed:
                 state.sync()
+                pending[0] = False
             infos.append(info)
             if per_step_cb:
                 per_step_cb(info)
@@ -192,11 +208,17 @@ def run_ours(args, rank, world):
             last[key] = now[key]
         kk["flops"] += 2.0 * info["n_rows"] * per_layer * cfg["L"] + 2.0 * info["n_active"] * cfg["d"] * cfg["V"]
 
+    def step_sync(state):
+        status, _ = state.step(A, B, R, T, k, stream)
+        if status == wd.WD_DONE:                      # out of masks: start again from the prompt
+            state.reset(ids, None, stream)
+            state.step(A, B, R, T, k, stream)
+        state.sync()
+
     def warm_then_time(n_warm, n_timed, state):
         # warm-up steps must not count: reset the totals after them
         for i in range(n_warm):
-            state.step(A, B, R, T, k, stream)
-            state.sync()
+            step_sync(state)
         now = ctx.profile_read()
         last.update({key: now[key] for key in last})
         return trajectory(0, n_timed, state, on_step)
@@ -211,8 +233,7 @@ def run_ours(args, rank, world):
     t0 = time.perf_counter()
     state.reset(ids, None, stream)
     for i in range(W + K):
-        state.step(A, B, R, T, k, stream)
-        state.sync()
+        step_sync(state)
     torch.cuda.synchronize()
     e2e_wall = time.perf_counter() - t0
     # ---- the window-only refresh variant (NOT the paper's method; reported beside the headline, never as it)
