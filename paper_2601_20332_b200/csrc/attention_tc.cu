@@ -40,7 +40,7 @@ constexpr int kAtom = kTile * 64 * 2;      // one [128 x 64] bf16 swizzle-atom c
 constexpr int kOperand = 2 * kAtom;        // a [128 x 128] bf16 operand: 32 KB
 constexpr int kThreads = 320;            // TMA warp, MMA warp, 8 softmax warps
 constexpr int kTmemCols = 512;             // S0, S1: columns 0..255; O_tile0, O_tile1: columns 256..511
-constexpr int kBars = 17;
+constexpr int kBars = 21;
 constexpr int kMaxCluster = 8;             // portable cluster size
 
 struct AttnParams {
@@ -85,6 +85,11 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
+// K stage ks of 3: stages 0 and 1 sit in front of their V stages, stage 2 behind both pairs
+__device__ __forceinline__ uint8_t* k_stage(uint8_t* sKV, int ks) {
+    return sKV + (size_t)(ks < 2 ? 2 * ks : 4) * kOperand;
+}
+
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                     const __grid_constant__ CUtensorMap map_vt, const AttnParams p) {
@@ -93,10 +98,13 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;                          // 32 KB
     uint8_t* sP = smem + kOperand;               // 32 KB
-    uint8_t* sKV = smem + 2 * kOperand;          // 2 stages x (K 32 KB + V^T 32 KB)
-    uint64_t* bars = (uint64_t*)(smem + 2 * kOperand + 4 * kOperand);
-    // 0 q_full | 1,2 k_full | 3,4 kv_empty | 5,6 s_full | 7,8 s_empty | 9 p_full | 10 p_empty |
-    // 11,12 o_full | 13,14 o_empty | 15,16 v_full.  "empty" barriers that the softmax threads signal count 256.
+    uint8_t* sKV = smem + 2 * kOperand;          // 2 stages x (K 32 KB + V^T 32 KB), then the third K stage
+    uint64_t* bars = (uint64_t*)(smem + 2 * kOperand + 5 * kOperand);
+    // 0 q_full | 1,2 k_full | 3,4 v_empty | 5,6 s_full | 7,8 s_empty | 9 p_full | 10 p_empty |
+    // 11,12 o_full | 13,14 o_empty | 15,16 v_full | 17,18 k_empty | 19 k_full of the third K stage | 20 its
+    // k_empty.  "empty" barriers that the softmax threads signal count 256.  K has three stages and V two,
+    // released separately: a K stage is free as soon as Q K^T has read it, long before P V frees the V stage,
+    // and the producer asks for K(i+1) before V(i), so that more bytes are in flight per SM.
     uint32_t* tmem_slot = (uint32_t*)(bars + kBars + 1);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     // after the last P V the K/V ring is free: this CTA's part of a split lives there
@@ -142,23 +150,35 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             mbar_expect_tx(qf, kOperand);
             tma_load_2d(smem_u32(sQ), &map_q, qf, h * kTile, row0);
             tma_load_2d(smem_u32(sQ) + kAtom, &map_q, qf, h * kTile + 64, row0);
-            for (int i = 0; i < n_kt; ++i) {
-                const int s = i & 1;
-                const uint32_t ph = (uint32_t)(i >> 1) & 1u;
-                if (!mbar_wait(smem_u32(&bars[3 + s]), ph ^ 1u, abort_flag)) {
-                    *abort_flag = 1;
-                    atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
-                    break;
-                }
-                const uint32_t kfull = smem_u32(&bars[1 + s]), vfull = smem_u32(&bars[15 + s]);
-                const uint32_t sk = smem_u32(sKV + (size_t)s * 2 * kOperand), sv = sk + kOperand;
-                const int kv0 = (kt_begin + i) * kTile, bh = b * p.Hkv + kvh;
+            const int bh = b * p.Hkv + kvh;
+            auto load_k = [&](int j) -> bool {
+                const int ks = j % 3;
+                const uint32_t ph = (uint32_t)(j / 3) & 1u;
+                const uint32_t kfull = smem_u32(&bars[ks < 2 ? 1 + ks : 19]);
+                if (!mbar_wait(smem_u32(&bars[ks < 2 ? 17 + ks : 20]), ph ^ 1u, abort_flag)) return false;   // stage free
+                const uint32_t sk = smem_u32(k_stage(sKV, ks));
+                const int kv0 = (kt_begin + j) * kTile;
                 mbar_expect_tx(kfull, kOperand);
                 tma_load_4d(sk, &map_k, kfull, 0, kv0, bh, p.layer);            // keys kv0.., dims 0..63
                 tma_load_4d(sk + kAtom, &map_k, kfull, 64, kv0, bh, p.layer);   // dims 64..127
+                return true;
+            };
+            bool ok = load_k(0);
+            for (int i = 0; i < n_kt && ok; ++i) {
+                if (i + 1 < n_kt && !(ok = load_k(i + 1))) break;
+                const int s = i & 1;
+                const uint32_t ph = (uint32_t)(i >> 1) & 1u;
+                const uint32_t vfull = smem_u32(&bars[15 + s]);
+                const uint32_t sv = smem_u32(sKV + (size_t)s * 2 * kOperand) + kOperand;
+                const int kv0 = (kt_begin + i) * kTile;
+                if (!(ok = mbar_wait(smem_u32(&bars[3 + s]), ph ^ 1u, abort_flag))) break;          // V stage free
                 mbar_expect_tx(vfull, kOperand);
                 tma_load_4d(sv, &map_vt, vfull, kv0, 0, bh, p.layer);           // all dims, keys kv0..kv0+63
                 tma_load_4d(sv + kAtom, &map_vt, vfull, kv0 + 64, 0, bh, p.layer);
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
             }
         }
         __syncwarp();
@@ -171,18 +191,19 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             const uint64_t qd0 = make_sdesc(smem_u32(sQ)), qd1 = make_sdesc(smem_u32(sQ) + kAtom);
             const uint64_t pd0 = make_sdesc(smem_u32(sP)), pd1 = make_sdesc(smem_u32(sP) + kAtom);
             auto issue_qk = [&](int j) -> bool {           // S[j&1] = Q K(j)^T
-                const int s = j & 1;
+                const int s = j & 1, ks = j % 3;
                 const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-                if (!mbar_wait(smem_u32(&bars[1 + s]), ph, abort_flag)) return false;        // K(j) landed
+                if (!mbar_wait(smem_u32(&bars[ks < 2 ? 1 + ks : 19]), (uint32_t)(j / 3) & 1u, abort_flag)) return false;   // K(j) landed
                 if (!mbar_wait(smem_u32(&bars[7 + s]), ph ^ 1u, abort_flag)) return false;   // S(j-2) has been read
                 tc_fence_after();
-                const uint32_t sk = smem_u32(sKV + (size_t)s * 2 * kOperand);
+                const uint32_t sk = smem_u32(k_stage(sKV, ks));
                 const uint64_t kd0 = make_sdesc(sk), kd1 = make_sdesc(sk + kAtom);
                 const uint32_t acc = tmem_base + (uint32_t)(s * kTile);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, qd0 + 2 * kk, kd0 + 2 * kk, p.idesc, kk > 0);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, qd1 + 2 * kk, kd1 + 2 * kk, p.idesc, 1u);
+                umma_commit(smem_u32(&bars[ks < 2 ? 17 + ks : 20]));   // K stage free once these MMAs have read it
                 umma_commit(smem_u32(&bars[5 + s]));
                 return true;
             };
@@ -203,7 +224,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, pd0 + 2 * kk, vd0 + 2 * kk, p.idesc, kk > 0);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, pd1 + 2 * kk, vd1 + 2 * kk, p.idesc, 1u);
-                umma_commit(smem_u32(&bars[3 + s]));       // K/V stage free
+                umma_commit(smem_u32(&bars[3 + s]));       // V stage free
                 umma_commit(smem_u32(&bars[10]));          // P buffer free
                 umma_commit(smem_u32(&bars[11 + s]));      // O_tile(i) ready
             }
@@ -525,7 +546,7 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     if (want > max_kt) want = max_kt;
     p.tiles_per_split = (max_kt + want - 1) / want;
     p.max_parts = (max_kt + p.tiles_per_split - 1) / p.tiles_per_split;
-    const size_t smem = 6 * (size_t)kOperand + (kBars + 1) * 8 + 16 + 2 * kTile * 4 + 1024;
+    const size_t smem = 7 * (size_t)kOperand + (kBars + 1) * 8 + 16 + 2 * kTile * 4 + 1024;
     static bool attr_done = false;      // one device per process
     if (!attr_done) {
         WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
