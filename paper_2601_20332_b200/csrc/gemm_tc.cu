@@ -43,6 +43,9 @@ struct TcParams {
     // line then holds the weight tiles once (n_units, W count weight tiles), and the groups walk it
     // in step, so that a weight block fetched for one token tile is still in L2 for the others
     int tok_split;
+    // pair kernel only, 1: a unit is [256 weight rows x 2*bn tokens] = two accumulators fed from the same
+    // weight stage (each CTA holds bn token rows per K block: half of either accumulator's tokens)
+    int dual;
     // FP8 operands: K blocks of 128 elements, outputs scaled by sw[segment][n] * sx[token]
     int fp8;
     const float* sw[3];
@@ -64,7 +67,7 @@ struct UnitInfo { int seg, n0, tok0; };
 __device__ __forceinline__ UnitInfo decode_unit(const TcParams& p, int unit, int tok_group = 0) {
     UnitInfo u;
     const int tile = p.tok_split > 1 ? unit : unit / p.tok_tiles;
-    u.tok0 = p.tok_split > 1 ? tok_group * p.bn : (unit - tile * p.tok_tiles) * p.bn;
+    u.tok0 = p.tok_split > 1 ? tok_group * p.bn : (unit - tile * p.tok_tiles) * p.bn * (p.dual ? 2 : 1);
     u.seg = 0;
     if (p.nseg > 1 && tile >= p.seg_tile0[1]) u.seg = 1;
     if (p.nseg > 2 && tile >= p.seg_tile0[2]) u.seg = 2;
@@ -676,9 +679,14 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int NS = p.n_stages;
-    const int half_bn = p.bn >> 1;                        // token rows this CTA loads per K block
+    const int half_bn = p.bn >> 1;                        // token rows of one accumulator held by this CTA
+    const int tok_rows = p.dual ? p.bn : half_bn;         // token rows this CTA loads per K block
     const int stage_a = kStageA;                          // 16 KB: this CTA's 128 weight rows
-    const int stage_bytes = stage_a + half_bn * kBK * 2;
+    const int stage_bytes = stage_a + tok_rows * kBK * 2;
+    // accumulator sets of (dual ? 2 : 1) * buf_cols columns: two sets (MMA of one tile overlaps the
+    // epilogue of the previous one) when they fit the 512 columns, else one
+    const int set_cols = (p.dual ? 2 : 1) * p.buf_cols;
+    const int n_sets = 2 * set_cols <= 512 ? 2 : 1;
     uint64_t* bars = (uint64_t*)(smem + (size_t)NS * stage_bytes);
     // bars[0..NS) full (used in the even CTA) | [NS..2NS) empty | [2NS, 2NS+1] accumulator full |
     // [2NS+2, 2NS+3] accumulator empty (used in the even CTA, 256 arrivals)
@@ -717,7 +725,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_w0) : "memory");
     }
-    if (warp == 1) tmem2_alloc(smem_u32(tmem_slot), 2u * (uint32_t)p.buf_cols);   // the same warp in both CTAs
+    if (warp == 1) tmem2_alloc(smem_u32(tmem_slot), (uint32_t)(n_sets * set_cols));   // the same warp in both CTAs
     tc_fence_before();
     __syncthreads();
     cluster_sync();               // the peer's barriers exist before anything signals them
@@ -742,7 +750,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 w.left = len;
                 const UnitInfo u = decode_unit(p, unit, tok_group);
                 w.n0 = u.n0 + (int)rank * kBM;
-                w.tok0 = u.tok0 + (int)rank * half_bn;
+                w.tok0 = u.tok0 + (int)rank * tok_rows;
                 w.mw = u.seg == 0 ? &map_w0 : (u.seg == 1 ? &map_w1 : &map_w2);
             };
             auto advance = [&](Walk& w) {
@@ -791,12 +799,12 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 long long g;
                 int len;
                 sch.piece(piece, g, len);
-                const int buf = piece & 1;
-                const uint32_t par = (uint32_t)(piece >> 1) & 1u;
-                // the epilogues of both CTAs have drained this accumulator (free at the start)
+                const int buf = n_sets == 2 ? piece & 1 : 0;
+                const uint32_t par = (uint32_t)(n_sets == 2 ? piece >> 1 : piece) & 1u;
+                // the epilogues of both CTAs have drained this accumulator set (free at the start)
                 if (!(ok = mbar_wait(smem_u32(&bars[2 * NS + 2 + buf]), par ^ 1u, abort_flag))) break;
                 tc_fence_after();
-                const uint32_t acc = tmem_base + (uint32_t)(buf * p.buf_cols);
+                const uint32_t acc = tmem_base + (uint32_t)(buf * set_cols);
                 for (int j = 0; j < len; ++j) {
                     if (!(ok = mbar_wait(smem_u32(&bars[s]), ph, abort_flag))) break;
                     tc_fence_after();
@@ -811,6 +819,20 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                         else
                             umma2_bf16(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), p.idesc,
                                        (j > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    if (p.dual) {
+                        // second accumulator: the same weight rows against the other half of the token rows
+                        const uint64_t bdesc1 = bdesc + (uint64_t)(half_bn * 8);      // half_bn rows of 128 bytes, in 16-byte units
+                        const uint32_t acc1 = acc + (uint32_t)p.buf_cols;
+#pragma unroll
+                        for (int kk = 0; kk < kBK / 16; ++kk) {
+                            if (kFp8)
+                                umma2_f8(acc1, adesc + (uint64_t)(2 * kk), bdesc1 + (uint64_t)(2 * kk), p.idesc,
+                                         (j > 0 || kk > 0) ? 1u : 0u);
+                            else
+                                umma2_bf16(acc1, adesc + (uint64_t)(2 * kk), bdesc1 + (uint64_t)(2 * kk), p.idesc,
+                                           (j > 0 || kk > 0) ? 1u : 0u);
+                        }
                     }
                     umma2_commit_mc(smem_u32(&bars[NS + s]), 3);          // stage free in both CTAs
                     if (++s == NS) { s = 0; ph ^= 1u; }
@@ -835,8 +857,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
             sch.piece(piece, g, len);
             const int unit = (int)(g / p.kb_total), kb0 = (int)(g - (long long)unit * p.kb_total);
             const UnitInfo u = decode_unit(p, unit, tok_group);
-            const int buf = piece & 1;
-            const uint32_t par = (uint32_t)(piece >> 1) & 1u;
+            const int buf = n_sets == 2 ? piece & 1 : 0;
+            const uint32_t par = (uint32_t)(n_sets == 2 ? piece >> 1 : piece) & 1u;
             const int n = u.n0 + n_local;
             const bool n_ok = n < p.seg_n[u.seg];
             int ord = 0;
@@ -847,18 +869,31 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
             tc_fence_after();
             float* yb = p.y + p.seg_col[u.seg] + n;
             const float sw_n = (kFp8 && n_ok) ? p.sw[u.seg][n] : 1.f;
-            const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p.buf_cols);
-            for (int cc = 0; cc < p.bn; cc += 16) {
-                if (u.tok0 + cc >= p.rows) break;
-                uint32_t v[16];
-                tmem_ld16(t_acc + (uint32_t)cc, v);
-                if (n_ok) {
-                    float* ys = yb + (size_t)ord * p.split_stride;
+            const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * set_cols);
+            float* ys = yb + (size_t)ord * p.split_stride;
+            // Accumulator a, column cc: columns [0, half_bn) are the token rows the even CTA holds,
+            // the rest the odd CTA's.  One accumulator: tokens tok0 + cc.  Two: the even CTA holds
+            // tokens [tok0, tok0 + bn), the odd one [tok0 + bn, tok0 + 2 bn), accumulator a the a-th
+            // half of each.
+            for (int a = 0; a < (p.dual ? 2 : 1); ++a) {
+                for (int cc = 0; cc < p.bn; cc += 16) {
+                    int tk[16];
 #pragma unroll
                     for (int t = 0; t < 16; ++t) {
-                        const int tok = u.tok0 + cc + t;
-                        if (tok < p.rows)
-                            ys[(size_t)tok * p.ncol] = kFp8 ? __uint_as_float(v[t]) * sw_n * p.sx[tok] : __uint_as_float(v[t]);
+                        const int col = cc + t;
+                        tk[t] = !p.dual ? u.tok0 + col
+                                        : (col < half_bn ? u.tok0 + a * half_bn + col : u.tok0 + p.bn + a * half_bn + col - half_bn);
+                    }
+                    if (tk[0] >= p.rows) continue;           // tk[0] is the chunk's smallest token (same for the whole warp)
+                    uint32_t v[16];
+                    tmem_ld16(t_acc + (uint32_t)(a * p.buf_cols + cc), v);
+                    if (n_ok) {
+#pragma unroll
+                        for (int t = 0; t < 16; ++t) {
+                            const int tok = tk[t];
+                            if (tok < p.rows)
+                                ys[(size_t)tok * p.ncol] = kFp8 ? __uint_as_float(v[t]) * sw_n * p.sx[tok] : __uint_as_float(v[t]);
+                        }
                     }
                 }
             }
@@ -868,7 +903,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 // this pair finished the tile: slices nobody wrote must read as zero
                 for (int sl = ord + 1; sl < p.n_slices; ++sl) {
                     float* ys = yb + (size_t)sl * p.split_stride;
-                    for (int tok = u.tok0; tok < u.tok0 + p.bn && tok < p.rows; ++tok) ys[(size_t)tok * p.ncol] = 0.f;
+                    for (int tok = u.tok0; tok < u.tok0 + (p.dual ? 2 : 1) * p.bn && tok < p.rows; ++tok)
+                        ys[(size_t)tok * p.ncol] = 0.f;
                 }
             }
         }
@@ -882,7 +918,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     cluster_sync();               // neither CTA frees tensor memory or leaves while the other may still signal it
     if (warp == 1) {
         tc_fence_after();
-        tmem2_dealloc(tmem_base, 2u * (uint32_t)p.buf_cols);
+        tmem2_dealloc(tmem_base, (uint32_t)(n_sets * set_cols));
     }
 }
 
@@ -1015,13 +1051,33 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     }
     const int kke = fp8 ? 128 : kBK;
     p.tile_rows = 2 * kBM;
-    p.tok_tiles = (rows + 255) / 256;
-    p.bn = ((rows + p.tok_tiles - 1) / p.tok_tiles + 15) / 16 * 16;        // balanced token tiles, <= 256
+    // Two accumulators per weight stage (token super-tiles of 2*bn rows): the weights enter shared memory
+    // once for up to 512 tokens, but the accumulators fill the tensor memory, so the epilogue no longer
+    // overlaps the next tile.  Measured: pays for the widest weight matrices (gate/up) once every pair
+    // gets at least two whole units, costs 10-25 % on the narrow ones.  0 = never, 1 = that rule, 2 = always.
+    static const int dual_mode = env_int("WD_GEMM_DUAL", 1);
+    {
+        int tiles_all = 0, ncol_all = 0;
+        for (int i = 0; i < nseg; ++i) {
+            tiles_all += (segs[i].n + p.tile_rows - 1) / p.tile_rows;
+            ncol_all += segs[i].n;
+        }
+        const long long dual_units = (long long)tiles_all * ((rows + 511) / 512);
+        p.dual = (dual_mode == 2 || (dual_mode == 1 && ncol_all >= 16384 && dual_units >= 2 * (sm_count / 2))) ? 1 : 0;
+    }
+    if (p.dual) {
+        p.tok_tiles = (rows + 511) / 512;                                   // super-tiles
+        p.bn = ((rows + 2 * p.tok_tiles - 1) / (2 * p.tok_tiles) + 15) / 16 * 16;   // balanced, <= 256
+    } else {
+        p.tok_tiles = (rows + 255) / 256;
+        p.bn = ((rows + p.tok_tiles - 1) / p.tok_tiles + 15) / 16 * 16;    // balanced token tiles, <= 256
+    }
     int cols = 32;
     while (cols < p.bn) cols <<= 1;
     p.buf_cols = cols;
     const int half_bn = p.bn / 2;
-    const int stage = kStageA + half_bn * kBK * 2;
+    const int tok_rows = p.dual ? p.bn : half_bn;                           // token rows per CTA and K block
+    const int stage = kStageA + tok_rows * kBK * 2;
     p.n_stages = (192 * 1024) / stage;
     if (p.n_stages > 10) p.n_stages = 10;
     const size_t smem = (size_t)p.n_stages * stage + (2 * p.n_stages + 4) * 8 + 16 + 256 + 1024;
@@ -1040,7 +1096,7 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     p.rows = rows;
     p.kb_total = (K + kke - 1) / kke;
     // two token tiles: one group of pairs per token tile, walking the weight K blocks in step
-    const int ts = (p.tok_tiles == 2 && (sm_count / 2) % 2 == 0) ? 2 : 1;
+    const int ts = (!p.dual && p.tok_tiles == 2 && (sm_count / 2) % 2 == 0) ? 2 : 1;
     p.tok_split = ts;
     p.n_units = ts > 1 ? tiles : tiles * p.tok_tiles;
     p.W = (long long)p.n_units * p.kb_total;
@@ -1069,12 +1125,12 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     CUtensorMap mx;
     bool hit = false;
     for (const WdTcX::Entry& e : x->cache)
-        if (e.rows == rows && e.bn == half_bn) { mx = e.map; hit = true; break; }
+        if (e.rows == rows && e.bn == tok_rows) { mx = e.map; hit = true; break; }
     if (!hit) {
-        wd_status s = fp8 ? encode_2d8(&mx, x->ptr, rows, K, half_bn) : encode_2d(&mx, x->ptr, rows, K, half_bn);
+        wd_status s = fp8 ? encode_2d8(&mx, x->ptr, rows, K, tok_rows) : encode_2d(&mx, x->ptr, rows, K, tok_rows);
         if (s != WD_OK) return s;
         if (x->cache.size() >= 16) x->cache.erase(x->cache.begin());
-        x->cache.push_back({rows, half_bn, mx});
+        x->cache.push_back({rows, tok_rows, mx});
     }
     static bool attr_done = false;      // one device per process
     if (!attr_done) {
