@@ -678,7 +678,7 @@ static bool use_tc(const wd_ctx* c) {
 static wd_status run_gemm(wd_ctx* c, const void* x, const WdTcX* x_map, const WdTcSeg* segs, int nseg,
                           int rows, int K, float* y, size_t y_floats, int32_t* status, cudaStream_t stream,
                           GemmOut* go, bool single_split = false, const WdTcFuse* fuse = nullptr,
-                          const WdTcFp8* fp8 = nullptr) {
+                          const WdTcFp8* fp8 = nullptr, const WdTcSwiglu* sg = nullptr) {
     int ncol = 0;
     for (int i = 0; i < nseg; ++i) ncol += segs[i].n;
     cudaEvent_t e0 = nullptr, e1 = nullptr;
@@ -698,8 +698,10 @@ static wd_status run_gemm(wd_ctx* c, const void* x, const WdTcX* x_map, const Wd
     if (use_tc(c)) {
         int n_split = 1;
         wd_status s = wd_tc_gemm(x_map, segs, nseg, rows, K, y, y_floats, c->sm_count, status, stream, &n_split,
-                                 single_split, fuse, fp8);
+                                 single_split, fuse, fp8, sg);
         if (s != WD_OK) return s;
+        // SwiGLU done by the GEMM: bf16 h instead of the fp32 gate/up sums
+        if (sg && sg->done && c->prof_on) c->prof_step_bytes -= (double)rows * ncol * 4 - (double)rows * (ncol / 2) * 2;
         *go = {n_split, (size_t)rows * ncol, 1, WD_GEMM_TCGEN05};
     } else {
         if ((size_t)rows * ncol > y_floats) return WD_ERR_CAPACITY;
@@ -1004,9 +1006,12 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
                 return s;
         } else {
         WdTcSeg gu[2] = {{c->wg[l], F, c->tc.get(WD_TC_WG, l)}, {c->wu[l], F, c->tc.get(WD_TC_WU, l)}};
-        if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, gu, 2, R_, D, c->part, c->part_floats, status, stream, &go)) != WD_OK)
+        WdTcSwiglu sg;
+        sg.h = use_tc(c) ? (__nv_bfloat16*)c->h : nullptr;
+        if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, gu, 2, R_, D, c->part, c->part_floats, status, stream, &go, false,
+                          nullptr, nullptr, &sg)) != WD_OK)
             return s;
-        wd_launch_swiglu(d.dtype, c->part, go.n_split, go.split_stride, c->h, R_, F, stream);
+        if (!sg.done) wd_launch_swiglu(d.dtype, c->part, go.n_split, go.split_stride, c->h, R_, F, stream);
         WdTcSeg wdn[1] = {{c->wd[l], D, c->tc.get(WD_TC_WD, l)}};
         if ((s = run_gemm(c, c->h, &c->tc.x_map_h, wdn, 1, R_, F, c->part, c->part_floats, status, stream, &go)) != WD_OK)
             return s;

@@ -34,6 +34,7 @@ constexpr int kBK = 64;             // K elements per stage = one 128-byte swizz
 constexpr int kStageA = kBM * kBK * 2;
 constexpr int kThreads = 192;         // TMA warp, MMA warp, 4 epilogue warps
 constexpr int kThreadsWide = 320;     // ... 8 epilogue warps when a CTA carries two weight halves
+constexpr int kThreadsPair = 320;     // two-CTA kernel: 8 epilogue warps, two per quarter of the accumulator rows
 
 struct TcParams {
     int rows, bn, kb_total, tok_tiles, n_units, n_stages, buf_cols, n_slices, aligned;
@@ -45,7 +46,14 @@ struct TcParams {
     int tok_split;
     // pair kernel only, 1: a unit is [256 weight rows x 2*bn tokens] = two accumulators fed from the same
     // weight stage (each CTA holds bn token rows per K block: half of either accumulator's tokens)
+    // 2: the two accumulators are the gate tile and the up tile of the same 256 FFN columns against one
+    // token tile (both weight blocks in every stage); the epilogue writes h = silu(gate) * up as bf16
     int dual;
+    // pair kernel, whole-tile schedule: > 0 = units are ordered (token group of tok_grp tiles, weight tile,
+    // token tile in the group) and dealt to the pairs round-robin, so that the pairs running at the same
+    // time share a few weight tiles and one group of token tiles (working set well inside the L2)
+    int tok_grp;
+    __nv_bfloat16* swiglu_h;        // dual == 2: [rows, ncol] with ncol = FFN width
     // FP8 operands: K blocks of 128 elements, outputs scaled by sw[segment][n] * sx[token]
     int fp8;
     const float* sw[3];
@@ -66,8 +74,21 @@ struct TcParams {
 struct UnitInfo { int seg, n0, tok0; };
 __device__ __forceinline__ UnitInfo decode_unit(const TcParams& p, int unit, int tok_group = 0) {
     UnitInfo u;
-    const int tile = p.tok_split > 1 ? unit : unit / p.tok_tiles;
-    u.tok0 = p.tok_split > 1 ? tok_group * p.bn : (unit - tile * p.tok_tiles) * p.bn * (p.dual ? 2 : 1);
+    int tile, tokt;
+    if (p.tok_grp > 0) {
+        const int per = p.seg_tile0[p.nseg] * p.tok_grp;            // units of a full token group
+        const int n_grp = (p.tok_tiles + p.tok_grp - 1) / p.tok_grp;
+        int grp = unit / per;
+        if (grp >= n_grp) grp = n_grp - 1;                          // the last group may be smaller
+        const int rem = unit - grp * per;
+        const int gsz = min(p.tok_grp, p.tok_tiles - grp * p.tok_grp);
+        tile = rem / gsz;
+        tokt = grp * p.tok_grp + rem % gsz;
+    } else {
+        tile = p.tok_split > 1 ? unit : unit / p.tok_tiles;
+        tokt = p.tok_split > 1 ? tok_group : unit - tile * p.tok_tiles;
+    }
+    u.tok0 = tokt * p.bn * (p.dual == 1 ? 2 : 1);
     u.seg = 0;
     if (p.nseg > 1 && tile >= p.seg_tile0[1]) u.seg = 1;
     if (p.nseg > 2 && tile >= p.seg_tile0[2]) u.seg = 2;
@@ -84,6 +105,16 @@ struct Sched {
     long long g_begin, g_end;
     int kb_total, head_len, tail_len, n_full, n_pieces;
     long long full_begin;
+    long long stride = 0;           // > 0: whole units first, first + stride, ... (K blocks on the line)
+    // whole units c, c + G, c + 2G, ... of n_units
+    __device__ void init_strided(long long c, long long G, int n_units, int kb) {
+        kb_total = kb;
+        head_len = tail_len = 0;
+        n_full = n_pieces = c < n_units ? (int)((n_units - c + G - 1) / G) : 0;
+        g_begin = full_begin = c * kb;
+        stride = G * kb;
+        g_end = g_begin;
+    }
     __device__ void init(long long gb, long long ge, int kb) {
         g_begin = gb; g_end = ge; kb_total = kb;
         const long long total = ge - gb;
@@ -98,6 +129,7 @@ struct Sched {
     }
     // piece i -> first K block on the line and length
     __device__ void piece(int i, long long& g, int& len) const {
+        if (stride > 0) { g = full_begin + (long long)i * stride; len = kb_total; return; }
         if (head_len) { if (i == 0) { g = g_begin; len = head_len; return; } --i; }
         if (tail_len) { if (i == 0) { g = g_end - tail_len; len = tail_len; return; } --i; }
         g = full_begin + (long long)i * kb_total;
@@ -671,7 +703,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 //   both:     TMA producer for their own operand halves, epilogue for their own 128 weight rows;
 //             epilogue threads of both CTAs arrive on the even CTA's "accumulator empty" barriers
 template <bool kFp8>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreadsPair)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w0,
                     const __grid_constant__ CUtensorMap map_w1, const __grid_constant__ CUtensorMap map_w2,
                     const TcParams p) {
@@ -680,8 +712,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     const int NS = p.n_stages;
     const int half_bn = p.bn >> 1;                        // token rows of one accumulator held by this CTA
-    const int tok_rows = p.dual ? p.bn : half_bn;         // token rows this CTA loads per K block
-    const int stage_a = kStageA;                          // 16 KB: this CTA's 128 weight rows
+    const int tok_rows = p.dual == 1 ? p.bn : half_bn;    // token rows this CTA loads per K block
+    const bool gate_up = p.dual == 2;                     // two weight blocks (gate, up) per stage
+    const int stage_a = gate_up ? 2 * kStageA : kStageA;  // this CTA's 128 weight rows (of gate and of up)
     const int stage_bytes = stage_a + tok_rows * kBK * 2;
     // accumulator sets of (dual ? 2 : 1) * buf_cols columns: two sets (MMA of one tile overlaps the
     // epilogue of the previous one) when they fit the 512 columns, else one
@@ -689,7 +722,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     const int n_sets = 2 * set_cols <= 512 ? 2 : 1;
     uint64_t* bars = (uint64_t*)(smem + (size_t)NS * stage_bytes);
     // bars[0..NS) full (used in the even CTA) | [NS..2NS) empty | [2NS, 2NS+1] accumulator full |
-    // [2NS+2, 2NS+3] accumulator empty (used in the even CTA, 256 arrivals)
+    // [2NS+2, 2NS+3] accumulator empty (used in the even CTA; every epilogue warp of both CTAs arrives once)
     uint32_t* tmem_slot = (uint32_t*)(bars + 2 * NS + 4);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
 
@@ -698,17 +731,23 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     // pairs per token group, this pair's index in its group, its token group (see TcParams::tok_split)
     const long long G = (gridDim.x >> 1) / (p.tok_split > 1 ? p.tok_split : 1), c = (blockIdx.x >> 1) % G;
     const int tok_group = (int)((blockIdx.x >> 1) / G);
-    long long g_begin, g_end;
-    if (p.aligned) {
-        g_begin = (c * p.n_units / G) * p.kb_total;
-        g_end = ((c + 1) * p.n_units / G) * p.kb_total;
-    } else {
-        g_begin = c * p.W / G;
-        g_end = (c + 1) * p.W / G;
-    }
-    const int n_total = (int)(g_end - g_begin);
     Sched sch;
-    sch.init(g_begin, g_end, p.kb_total);
+    int n_total;
+    if (p.aligned && p.tok_grp > 0) {
+        sch.init_strided(c, G, p.n_units, p.kb_total);
+        n_total = sch.n_pieces * p.kb_total;
+    } else {
+        long long g_begin, g_end;
+        if (p.aligned) {
+            g_begin = (c * p.n_units / G) * p.kb_total;
+            g_end = ((c + 1) * p.n_units / G) * p.kb_total;
+        } else {
+            g_begin = c * p.W / G;
+            g_end = (c + 1) * p.W / G;
+        }
+        n_total = (int)(g_end - g_begin);
+        sch.init(g_begin, g_end, p.kb_total);
+    }
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
@@ -718,8 +757,8 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         }
         mbar_init(smem_u32(&bars[2 * NS]), 1);
         mbar_init(smem_u32(&bars[2 * NS + 1]), 1);
-        mbar_init(smem_u32(&bars[2 * NS + 2]), 256);
-        mbar_init(smem_u32(&bars[2 * NS + 3]), 256);
+        mbar_init(smem_u32(&bars[2 * NS + 2]), 2 * (kThreadsPair / 32 - 2));
+        mbar_init(smem_u32(&bars[2 * NS + 3]), 2 * (kThreadsPair / 32 - 2));
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&map_x) : "memory");
@@ -766,6 +805,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 if (rank == 0) mbar_expect_tx(smem_u32(&bars[i]), 2u * (uint32_t)stage_bytes);
                 tma2_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes), w.mw, cluster_map(smem_u32(&bars[i]), 0),
                                   w.kb * kKE, w.n0, pol_stream);
+                if (gate_up)
+                    tma2_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes) + kStageA, &map_w1,
+                                      cluster_map(smem_u32(&bars[i]), 0), w.kb * kKE, w.n0, pol_stream);
             }
             pdl_wait();
             Walk wx = w0;
@@ -784,6 +826,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
                 if (rank == 0) mbar_expect_tx(smem_u32(&bars[s]), 2u * (uint32_t)stage_bytes);
                 tma2_load_2d_hint(sa, w.mw, full, w.kb * kKE, w.n0, pol_stream);
+                if (gate_up) tma2_load_2d_hint(sa + kStageA, &map_w1, full, w.kb * kKE, w.n0, pol_stream);
                 tma2_load_2d(sa + stage_a, &map_x, full, w.kb * kKE, w.tok0);
                 if (++s == NS) { s = 0; ph ^= 1u; }
             }
@@ -822,15 +865,18 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                     }
                     if (p.dual) {
                         // second accumulator: the same weight rows against the other half of the token rows
-                        const uint64_t bdesc1 = bdesc + (uint64_t)(half_bn * 8);      // half_bn rows of 128 bytes, in 16-byte units
+                        // (offset of half_bn rows of 128 bytes, in 16-byte units), or the up weights against
+                        // the same token rows
+                        const uint64_t adesc1 = gate_up ? adesc + (uint64_t)(kStageA >> 4) : adesc;
+                        const uint64_t bdesc1 = gate_up ? bdesc : bdesc + (uint64_t)(half_bn * 8);
                         const uint32_t acc1 = acc + (uint32_t)p.buf_cols;
 #pragma unroll
                         for (int kk = 0; kk < kBK / 16; ++kk) {
                             if (kFp8)
-                                umma2_f8(acc1, adesc + (uint64_t)(2 * kk), bdesc1 + (uint64_t)(2 * kk), p.idesc,
+                                umma2_f8(acc1, adesc1 + (uint64_t)(2 * kk), bdesc1 + (uint64_t)(2 * kk), p.idesc,
                                          (j > 0 || kk > 0) ? 1u : 0u);
                             else
-                                umma2_bf16(acc1, adesc + (uint64_t)(2 * kk), bdesc1 + (uint64_t)(2 * kk), p.idesc,
+                                umma2_bf16(acc1, adesc1 + (uint64_t)(2 * kk), bdesc1 + (uint64_t)(2 * kk), p.idesc,
                                            (j > 0 || kk > 0) ? 1u : 0u);
                         }
                     }
@@ -846,8 +892,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
         }
         __syncwarp();
     } else {
-        // ---------------------------------------------------- epilogue (warps 2..5 of both CTAs)
+        // ---------------------------------------------------- epilogue (warps 2..9 of both CTAs)
+        // Warp w reads the accumulator rows (TMEM lanes) of quarter w % 4; the two warps of a quarter
+        // take alternate 16-column chunks.  (Plain loops on purpose: a version that kept the next
+        // chunk's tcgen05.ld in flight behind lambdas compiled to twice the instructions per chunk.)
         const int quarter = warp & 3;
+        const int hf = (warp - 2) >> 2;
+        constexpr int n_hf = 2;
         const int n_local = (int)rank * kBM + quarter * 32 + lane;
         pdl_wait();
         bool ok = true;
@@ -871,18 +922,39 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
             const float sw_n = (kFp8 && n_ok) ? p.sw[u.seg][n] : 1.f;
             const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * set_cols);
             float* ys = yb + (size_t)ord * p.split_stride;
-            // Accumulator a, column cc: columns [0, half_bn) are the token rows the even CTA holds,
-            // the rest the odd CTA's.  One accumulator: tokens tok0 + cc.  Two: the even CTA holds
-            // tokens [tok0, tok0 + bn), the odd one [tok0 + bn, tok0 + 2 bn), accumulator a the a-th
-            // half of each.
-            for (int a = 0; a < (p.dual ? 2 : 1); ++a) {
-                for (int cc = 0; cc < p.bn; cc += 16) {
+            // Accumulator a, column col: columns [0, half_bn) are the token rows the even CTA holds,
+            // the rest the odd CTA's.  One accumulator (or gate/up): token tok0 + col.  Two token
+            // halves: the even CTA holds tokens [tok0, tok0 + bn), the odd one [tok0 + bn, tok0 + 2 bn),
+            // accumulator a the a-th half of each.
+            const int col_step = 16 * n_hf;
+            if (gate_up) {
+                // h = silu(gate) * up
+                __nv_bfloat16* hb = p.swiglu_h + n;
+                for (int cc = 16 * hf; cc < p.bn; cc += col_step) {
+                    if (u.tok0 + cc >= p.rows) break;
+                    uint32_t vg[16], vu[16];
+                    tmem_ld16_issue(t_acc + (uint32_t)cc, vg);
+                    tmem_ld16(t_acc + (uint32_t)(p.buf_cols + cc), vu);
+                    tmem_ld16_wait(vg);
+                    if (n_ok) {
+#pragma unroll
+                        for (int t = 0; t < 16; ++t) {
+                            const int tok = u.tok0 + cc + t;
+                            const float gv = __uint_as_float(vg[t]);
+                            if (tok < p.rows)
+                                hb[(size_t)tok * p.ncol] = __float2bfloat16(__fdividef(gv, 1.f + __expf(-gv)) * __uint_as_float(vu[t]));
+                        }
+                    }
+                }
+            }
+            for (int a = 0; a < (gate_up ? 0 : p.dual ? 2 : 1); ++a) {
+                for (int cc = 16 * hf; cc < p.bn; cc += col_step) {
                     int tk[16];
 #pragma unroll
                     for (int t = 0; t < 16; ++t) {
                         const int col = cc + t;
-                        tk[t] = !p.dual ? u.tok0 + col
-                                        : (col < half_bn ? u.tok0 + a * half_bn + col : u.tok0 + p.bn + a * half_bn + col - half_bn);
+                        tk[t] = p.dual != 1 ? u.tok0 + col
+                                            : (col < half_bn ? u.tok0 + a * half_bn + col : u.tok0 + p.bn + a * half_bn + col - half_bn);
                     }
                     if (tk[0] >= p.rows) continue;           // tk[0] is the chunk's smallest token (same for the whole warp)
                     uint32_t v[16];
@@ -898,12 +970,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                 }
             }
             tc_fence_before();
-            mbar_arrive_cluster(cluster_map(smem_u32(&bars[2 * NS + 2 + buf]), 0));   // accumulator may be overwritten
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(cluster_map(smem_u32(&bars[2 * NS + 2 + buf]), 0));   // accumulator may be overwritten
             if (kb0 + len == p.kb_total && n_ok) {
                 // this pair finished the tile: slices nobody wrote must read as zero
                 for (int sl = ord + 1; sl < p.n_slices; ++sl) {
                     float* ys = yb + (size_t)sl * p.split_stride;
-                    for (int tok = u.tok0; tok < u.tok0 + (p.dual ? 2 : 1) * p.bn && tok < p.rows; ++tok)
+                    for (int tok = u.tok0 + hf; tok < u.tok0 + (p.dual == 1 ? 2 : 1) * p.bn && tok < p.rows; tok += n_hf)
                         ys[(size_t)tok * p.ncol] = 0.f;
                 }
             }
@@ -1041,7 +1114,7 @@ uint32_t make_idesc(int bn, int m = kBM, bool fp8 = false) {
 // launch of gemm_tc_pair_kernel: same contract as wd_tc_gemm
 wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, int K, float* y, size_t y_floats,
                        int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out, bool force_single_split,
-                       const WdTcFp8* fp8) {
+                       const WdTcFp8* fp8, const WdTcSwiglu* sg) {
     TcParams p;
     memset(&p, 0, sizeof(p));
     if (fp8) {
@@ -1064,8 +1137,15 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
         }
         const long long dual_units = (long long)tiles_all * ((rows + 511) / 512);
         p.dual = (dual_mode == 2 || (dual_mode == 1 && ncol_all >= 16384 && dual_units >= 2 * (sm_count / 2))) ? 1 : 0;
+        // gate and up against the same tokens, h = silu(gate) * up written by the epilogue: needs whole
+        // tiles per pair (no partial sums), taken when every pair gets at least two of them
+        static const int swiglu_fused = env_int("WD_GEMM_SWIGLU", 1);
+        if (sg && sg->h && swiglu_fused && !fp8 && nseg == 2 && segs[0].n == segs[1].n && dual_mode != 0) {
+            const long long gu_units = (long long)((segs[0].n + p.tile_rows - 1) / p.tile_rows) * ((rows + 255) / 256);
+            if (gu_units >= 2 * (sm_count / 2)) p.dual = 2;
+        }
     }
-    if (p.dual) {
+    if (p.dual == 1) {
         p.tok_tiles = (rows + 511) / 512;                                   // super-tiles
         p.bn = ((rows + 2 * p.tok_tiles - 1) / (2 * p.tok_tiles) + 15) / 16 * 16;   // balanced, <= 256
     } else {
@@ -1076,19 +1156,32 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     while (cols < p.bn) cols <<= 1;
     p.buf_cols = cols;
     const int half_bn = p.bn / 2;
-    const int tok_rows = p.dual ? p.bn : half_bn;                           // token rows per CTA and K block
-    const int stage = kStageA + tok_rows * kBK * 2;
+    const int tok_rows = p.dual == 1 ? p.bn : half_bn;                      // token rows per CTA and K block
+    const int stage = (p.dual == 2 ? 2 : 1) * kStageA + tok_rows * kBK * 2;
     p.n_stages = (192 * 1024) / stage;
     if (p.n_stages > 10) p.n_stages = 10;
     const size_t smem = (size_t)p.n_stages * stage + (2 * p.n_stages + 4) * 8 + 16 + 256 + 1024;
     int tiles = 0, col = 0;
-    for (int i = 0; i < nseg; ++i) {
+    for (int i = 0; i < nseg; ++i)
         if (!segs[i].map) return WD_ERR_NULL;
-        p.seg_tile0[i] = tiles;
-        p.seg_n[i] = segs[i].n;
-        p.seg_col[i] = col;
-        tiles += (segs[i].n + p.tile_rows - 1) / p.tile_rows;
-        col += segs[i].n;
+    if (p.dual == 2) {
+        // one line of (gate tile, up tile) pairs; the output has the FFN width
+        nseg = 1;
+        p.seg_tile0[0] = 0;
+        p.seg_n[0] = segs[0].n;
+        p.seg_col[0] = 0;
+        tiles = (segs[0].n + p.tile_rows - 1) / p.tile_rows;
+        col = segs[0].n;
+        p.swiglu_h = sg->h;
+        force_single_split = true;
+    } else {
+        for (int i = 0; i < nseg; ++i) {
+            p.seg_tile0[i] = tiles;
+            p.seg_n[i] = segs[i].n;
+            p.seg_col[i] = col;
+            tiles += (segs[i].n + p.tile_rows - 1) / p.tile_rows;
+            col += segs[i].n;
+        }
     }
     p.seg_tile0[nseg] = tiles;
     p.nseg = nseg;
@@ -1101,7 +1194,7 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     p.n_units = ts > 1 ? tiles : tiles * p.tok_tiles;
     p.W = (long long)p.n_units * p.kb_total;
     const size_t slice = (size_t)rows * col;
-    if (slice > y_floats) return WD_ERR_CAPACITY;
+    if (p.dual != 2 && slice > y_floats) return WD_ERR_CAPACITY;
     long long G = sm_count / 2 / ts;                                       // CTA pairs (per token group)
     if (G > p.W / 2) G = p.W / 2 > 0 ? p.W / 2 : 1;
     int n_slices = count_slices(p.n_units, p.kb_total, p.W, G);
@@ -1116,6 +1209,8 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
         G = sm_count / 2 / ts;
         if (G > p.n_units) G = p.n_units;
     }
+    static const int tok_grp = env_int("WD_GEMM_TOK_GROUP", 16);          // 0 = contiguous units per pair
+    p.tok_grp = (p.aligned && ts == 1) ? tok_grp : 0;
     p.n_slices = n_slices;
     p.y = y;
     p.split_stride = slice;
@@ -1139,12 +1234,13 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
         attr_done = true;
     }
     const CUtensorMap& m0 = *segs[0].map;
-    const CUtensorMap& m1 = *segs[nseg > 1 ? 1 : 0].map;
+    const CUtensorMap& m1 = *segs[(nseg > 1 || p.dual == 2) ? 1 : 0].map;
     const CUtensorMap& m2 = *segs[nseg > 2 ? 2 : 0].map;
+    if (sg) sg->done = p.dual == 2;
     ++wd_launch_counter;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3((unsigned)(2 * G * ts));
-    lc.blockDim = dim3(kThreads);
+    lc.blockDim = dim3(kThreadsPair);
     lc.dynamicSmemBytes = smem;
     lc.stream = stream;
     cudaLaunchAttribute attr[2];
@@ -1192,8 +1288,9 @@ wd_status wd_tc_weights_init(WdTcWeights* tc, const wd_model_dims* d, const void
 
 wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, int K, float* y, size_t y_floats,
                      int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out, bool force_single_split,
-                     const WdTcFuse* fuse, const WdTcFp8* fp8) {
+                     const WdTcFuse* fuse, const WdTcFp8* fp8, const WdTcSwiglu* sg) {
     if (!x || !segs || !y || !status || nseg < 1 || nseg > 3) return WD_ERR_BAD_PARAM;
+    if (sg) sg->done = false;
     if (rows < 1 || K < 8 || K % 8) return WD_ERR_BAD_PARAM;
     TcParams p;
     memset(&p, 0, sizeof(p));
@@ -1212,7 +1309,7 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     static const int pair_from = env_int("WD_GEMM_PAIR_FROM", 256);        // rows from which pairs are used; 0 = never
     if (!fused && pair_from > 0 && rows > pair_from && sm_count >= 2)
         return tc_gemm_pair(x, segs, nseg, rows, K, y, y_floats, sm_count, status, stream, n_split_out, force_single_split,
-                            fp8);
+                            fp8, sg);
     // The wide tile halves the operand traffic per flop but has a shallower ring and an epilogue
     // that does not overlap the next tile: it pays once every CTA gets at least one whole tile.
     long long wide_units = 0;

@@ -92,11 +92,21 @@ struct WdTcFp8 {
     const float* sx = nullptr;
 };
 
+// Gate/up launches (two weight matrices of the same height): where the GEMM can keep the gate tile and
+// the up tile of the same columns in two accumulators, its epilogue writes h = silu(gate) * up as bf16
+// [rows, n] and nothing goes to y.  `done` tells the caller whether that happened; if not, y holds the
+// partial sums as usual and the caller runs the SwiGLU kernel.
+struct WdTcSwiglu {
+    __nv_bfloat16* h = nullptr;
+    mutable bool done = false;
+};
+
 // y[split][rows][sum n_i] = x * [w_0; w_1; ...]^T, split-K partial sums side by side
 // (split_stride = rows * sum n_i floats).  The consumer adds the slices.
 wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, int K, float* y, size_t y_floats,
                      int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out,
-                     bool force_single_split = false, const WdTcFuse* fuse = nullptr, const WdTcFp8* fp8 = nullptr);
+                     bool force_single_split = false, const WdTcFuse* fuse = nullptr, const WdTcFp8* fp8 = nullptr,
+                     const WdTcSwiglu* sg = nullptr);
 // TMA descriptor of a [n_rows, K] byte matrix for the FP8 path (box 128 x box_rows)
 wd_status wd_tc_encode_fp8(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_rows);
 

@@ -74,6 +74,28 @@ def test_cfg4_dream7b_shape_gqa_batch8():
     assert len(set(pos.tolist())) > 1                     # the windows really are independent
 
 
+def test_cfg4_gate_up_launch_writes_swiglu_itself():
+    """At the Dream-7B width every CTA pair gets two whole (gate tile, up tile) units, so the gate/up
+    GEMM's epilogue writes h = silu(gate) * up and no SwiGLU kernel runs: one launch fewer per block
+    than at the LLaDA-8B width with 352 rows (96 units for 74 pairs: partial sums + SwiGLU kernel).
+    The parity of that path is what test_cfg4_dream7b_shape_gqa_batch8 checks."""
+    counts = {}
+    for name in ("llada8b", "dream7b"):
+        cfg = synth.get_config(name, L=1)
+        w = synth.make_weights(cfg, DEV)
+        ids = synth.make_prompts(cfg)
+        batch, S = ids.shape
+        ctx = wd.Context(cfg, w, batch, S, batch * S, batch * cfg["A"])
+        st = wd.State(ctx, ids)
+        _, info = st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])
+        st.sync()
+        assert info["is_refresh"] == 1 and info["n_rows"] > 256
+        counts[name] = info["n_launches"]
+        del st, ctx, w
+        torch.cuda.empty_cache()
+    assert counts["dream7b"] == counts["llada8b"] - 1
+
+
 def test_cfg5_sweep_corner_late_state():
     """Window sweep corner A=128 B=256 R=4, prompt 1024 + 2048 masks, batch 2, from a
     half-decoded state (2048 visible positions)."""
