@@ -40,7 +40,7 @@ constexpr int kAtom = kTile * 64 * 2;      // one [128 x 64] bf16 swizzle-atom c
 constexpr int kOperand = 2 * kAtom;        // a [128 x 128] bf16 operand: 32 KB
 constexpr int kThreads = 320;            // TMA warp, MMA warp, 8 softmax warps
 constexpr int kTmemCols = 512;             // S0, S1: columns 0..255; O_tile0, O_tile1: columns 256..511
-constexpr int kBars = 21;
+constexpr int kBars = 20;
 constexpr int kMaxCluster = 8;             // portable cluster size
 
 struct AttnParams {
@@ -80,15 +80,22 @@ __device__ __forceinline__ float2 dsmem_ld2(uint32_t a) {
     return v;
 }
 
+// 2^x by the special-function unit alone (x <= 0 here: results in [0, 1], denormals flushed)
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
 }
 
-// K stage ks of 3: stages 0 and 1 sit in front of their V stages, stage 2 behind both pairs
-__device__ __forceinline__ uint8_t* k_stage(uint8_t* sKV, int ks) {
-    return sKV + (size_t)(ks < 2 ? 2 * ks : 4) * kOperand;
-}
+// barrier indices
+constexpr int kQFull = 0, kKFull = 1, kKEmpty = 4, kVFull = 7, kVEmpty = 10, kSFull = 13, kPFull = 15, kOFull = 16,
+              kOEmpty = 18;
+constexpr int kStages = 3;                 // K stages and V stages
 
 __global__ void __launch_bounds__(kThreads, 1)
 attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
@@ -97,19 +104,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     // the same offset in every CTA of the cluster (the dynamic window starts at the same address)
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;                          // 32 KB
-    uint8_t* sP = smem + kOperand;               // 32 KB
-    uint8_t* sKV = smem + 2 * kOperand;          // 2 stages x (K 32 KB + V^T 32 KB), then the third K stage
-    uint64_t* bars = (uint64_t*)(smem + 2 * kOperand + 5 * kOperand);
-    // 0 q_full | 1,2 k_full | 3,4 v_empty | 5,6 s_full | 7,8 s_empty | 9 p_full | 10 p_empty |
-    // 11,12 o_full | 13,14 o_empty | 15,16 v_full | 17,18 k_empty | 19 k_full of the third K stage | 20 its
-    // k_empty.  "empty" barriers that the softmax threads signal count 256.  K has three stages and V two,
-    // released separately: a K stage is free as soon as Q K^T has read it, long before P V frees the V stage,
-    // and the producer asks for K(i+1) before V(i), so that more bytes are in flight per SM.
+    uint8_t* sK = smem + kOperand;               // 3 stages x 32 KB
+    uint8_t* sV = sK + kStages * kOperand;       // 3 stages x 32 KB (transposed V tiles)
+    uint64_t* bars = (uint64_t*)(sV + kStages * kOperand);
+    // q_full | k_full[3] | k_empty[3] | v_full[3] | v_empty[3] | s_full[2] | p_full | o_full[2] | o_empty[2].
+    // p_full and o_empty count the 256 softmax threads.  P never touches shared memory: the softmax
+    // threads write it as bf16 over the S buffer they have just read (tcgen05.st) and P V takes its A
+    // operand from tensor memory.  No "S empty" / "P empty" barriers are needed: the tensor core runs the
+    // MMAs in issue order (Q K^T(i+1), P V(i), Q K^T(i+2), ...), so S buffer i & 1 is rewritten by
+    // Q K^T(i+2) only after P V(i) has read P(i) from it, and P V(i) was issued after P(i) was complete.
+    // K and V stages are released separately: a K stage as soon as Q K^T has read it, a V stage after P V.
     uint32_t* tmem_slot = (uint32_t*)(bars + kBars + 1);
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     // after the last P V the K/V ring is free: this CTA's part of a split lives there
-    float* part_o = (float*)sKV;                           // [128 rows][128], 16-byte chunks XOR-swizzled by row
-    float* part_ml = (float*)(sKV + 2 * kOperand);         // [128 rows][2] running maximum, sum
+    float* part_o = (float*)sK;                            // [128 rows][128], 16-byte chunks XOR-swizzled by row
+    float* part_ml = (float*)(sK + 2 * kOperand);          // [128 rows][2] running maximum, sum
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x, h = blockIdx.y;
@@ -129,7 +138,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     if (has_work) {
         if (threadIdx.x == 0) {
             for (int i = 0; i < kBars; ++i)
-                mbar_init(smem_u32(&bars[i]), (i == 7 || i == 8 || i == 9 || i == 13 || i == 14) ? 256u : 1u);
+                mbar_init(smem_u32(&bars[i]), (i == kPFull || i == kOEmpty || i == kOEmpty + 1) ? 256u : 1u);
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
@@ -146,32 +155,33 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     } else if (warp == 0) {
         if (lane == 0) {
             // ---------------------------------------------------- TMA producer
-            const uint32_t qf = smem_u32(&bars[0]);
+            const uint32_t qf = smem_u32(&bars[kQFull]);
             mbar_expect_tx(qf, kOperand);
             tma_load_2d(smem_u32(sQ), &map_q, qf, h * kTile, row0);
             tma_load_2d(smem_u32(sQ) + kAtom, &map_q, qf, h * kTile + 64, row0);
             const int bh = b * p.Hkv + kvh;
             auto load_k = [&](int j) -> bool {
-                const int ks = j % 3;
-                const uint32_t ph = (uint32_t)(j / 3) & 1u;
-                const uint32_t kfull = smem_u32(&bars[ks < 2 ? 1 + ks : 19]);
-                if (!mbar_wait(smem_u32(&bars[ks < 2 ? 17 + ks : 20]), ph ^ 1u, abort_flag)) return false;   // stage free
-                const uint32_t sk = smem_u32(k_stage(sKV, ks));
+                const int ks = j % kStages;
+                const uint32_t ph = (uint32_t)(j / kStages) & 1u;
+                const uint32_t kfull = smem_u32(&bars[kKFull + ks]);
+                if (!mbar_wait(smem_u32(&bars[kKEmpty + ks]), ph ^ 1u, abort_flag)) return false;   // stage free
+                const uint32_t sk = smem_u32(sK + (size_t)ks * kOperand);
                 const int kv0 = (kt_begin + j) * kTile;
                 mbar_expect_tx(kfull, kOperand);
                 tma_load_4d(sk, &map_k, kfull, 0, kv0, bh, p.layer);            // keys kv0.., dims 0..63
                 tma_load_4d(sk + kAtom, &map_k, kfull, 64, kv0, bh, p.layer);   // dims 64..127
                 return true;
             };
+            // order of need: K(0), K(1), V(0), K(2), V(1), ...
             bool ok = load_k(0);
             for (int i = 0; i < n_kt && ok; ++i) {
                 if (i + 1 < n_kt && !(ok = load_k(i + 1))) break;
-                const int s = i & 1;
-                const uint32_t ph = (uint32_t)(i >> 1) & 1u;
-                const uint32_t vfull = smem_u32(&bars[15 + s]);
-                const uint32_t sv = smem_u32(sKV + (size_t)s * 2 * kOperand) + kOperand;
+                const int vs = i % kStages;
+                const uint32_t ph = (uint32_t)(i / kStages) & 1u;
+                const uint32_t vfull = smem_u32(&bars[kVFull + vs]);
+                const uint32_t sv = smem_u32(sV + (size_t)vs * kOperand);
                 const int kv0 = (kt_begin + i) * kTile;
-                if (!(ok = mbar_wait(smem_u32(&bars[3 + s]), ph ^ 1u, abort_flag))) break;          // V stage free
+                if (!(ok = mbar_wait(smem_u32(&bars[kVEmpty + vs]), ph ^ 1u, abort_flag))) break;   // stage free
                 mbar_expect_tx(vfull, kOperand);
                 tma_load_4d(sv, &map_vt, vfull, kv0, 0, bh, p.layer);           // all dims, keys kv0..kv0+63
                 tma_load_4d(sv + kAtom, &map_vt, vfull, kv0 + 64, 0, bh, p.layer);
@@ -185,48 +195,44 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     } else if (warp == 1) {
         if (lane == 0) {
             // ---------------------------------------------------- MMA issuer
-            // tile i uses K/V stage i&1, S buffer i&1, O_tile buffer i&1; every barrier that is
-            // completed once per two tiles has parity (i>>1)&1 for tile i
-            bool ok = mbar_wait(smem_u32(&bars[0]), 0, abort_flag);
+            // tile i uses K/V stage i % 3, S buffer i & 1, O_tile buffer i & 1
+            bool ok = mbar_wait(smem_u32(&bars[kQFull]), 0, abort_flag);
             const uint64_t qd0 = make_sdesc(smem_u32(sQ)), qd1 = make_sdesc(smem_u32(sQ) + kAtom);
-            const uint64_t pd0 = make_sdesc(smem_u32(sP)), pd1 = make_sdesc(smem_u32(sP) + kAtom);
             auto issue_qk = [&](int j) -> bool {           // S[j&1] = Q K(j)^T
-                const int s = j & 1, ks = j % 3;
-                const uint32_t ph = (uint32_t)(j >> 1) & 1u;
-                if (!mbar_wait(smem_u32(&bars[ks < 2 ? 1 + ks : 19]), (uint32_t)(j / 3) & 1u, abort_flag)) return false;   // K(j) landed
-                if (!mbar_wait(smem_u32(&bars[7 + s]), ph ^ 1u, abort_flag)) return false;   // S(j-2) has been read
+                const int s = j & 1, ks = j % kStages;
+                if (!mbar_wait(smem_u32(&bars[kKFull + ks]), (uint32_t)(j / kStages) & 1u, abort_flag)) return false;   // K(j) landed
                 tc_fence_after();
-                const uint32_t sk = smem_u32(k_stage(sKV, ks));
+                const uint32_t sk = smem_u32(sK + (size_t)ks * kOperand);
                 const uint64_t kd0 = make_sdesc(sk), kd1 = make_sdesc(sk + kAtom);
                 const uint32_t acc = tmem_base + (uint32_t)(s * kTile);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, qd0 + 2 * kk, kd0 + 2 * kk, p.idesc, kk > 0);
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, qd1 + 2 * kk, kd1 + 2 * kk, p.idesc, 1u);
-                umma_commit(smem_u32(&bars[ks < 2 ? 17 + ks : 20]));   // K stage free once these MMAs have read it
-                umma_commit(smem_u32(&bars[5 + s]));
+                umma_commit(smem_u32(&bars[kKEmpty + ks]));    // K stage free once these MMAs have read it
+                umma_commit(smem_u32(&bars[kSFull + s]));
                 return true;
             };
             ok = ok && issue_qk(0);
             for (int i = 0; i < n_kt && ok; ++i) {
-                const int s = i & 1;
+                const int s = i & 1, vs = i % kStages;
                 const uint32_t ph = (uint32_t)(i >> 1) & 1u;
                 if (i + 1 < n_kt && !(ok = issue_qk(i + 1))) break;                           // runs ahead of the softmax
-                if (!(ok = mbar_wait(smem_u32(&bars[15 + s]), ph, abort_flag))) break;              // V(i) landed
-                if (!(ok = mbar_wait(smem_u32(&bars[9]), (uint32_t)i & 1u, abort_flag))) break;      // P(i) written
-                if (!(ok = mbar_wait(smem_u32(&bars[13 + s]), ph ^ 1u, abort_flag))) break;         // O_tile(i-2) folded
+                if (!(ok = mbar_wait(smem_u32(&bars[kVFull + vs]), (uint32_t)(i / kStages) & 1u, abort_flag))) break;   // V(i) landed
+                if (!(ok = mbar_wait(smem_u32(&bars[kPFull]), (uint32_t)i & 1u, abort_flag))) break;    // P(i) written
+                if (!(ok = mbar_wait(smem_u32(&bars[kOEmpty + s]), ph ^ 1u, abort_flag))) break;        // O_tile(i-2) folded
                 tc_fence_after();
-                const uint32_t sv = smem_u32(sKV + (size_t)s * 2 * kOperand) + kOperand;
+                const uint32_t sv = smem_u32(sV + (size_t)vs * kOperand);
                 const uint64_t vd0 = make_sdesc(sv), vd1 = make_sdesc(sv + kAtom);
                 const uint32_t acc = tmem_base + (uint32_t)(2 * kTile + s * kTile);
-                // O_tile = P V: reduction over the 128 keys of the tile
+                const uint32_t pa = tmem_base + (uint32_t)(s * kTile);       // P(i): 64 columns over S(i)
+                // O_tile = P V: reduction over the 128 keys of the tile, 16 keys = 8 columns of P per MMA
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, pd0 + 2 * kk, vd0 + 2 * kk, p.idesc, kk > 0);
+                for (int kk = 0; kk < 4; ++kk) umma_bf16_ta(acc, pa + 8 * kk, vd0 + 2 * kk, p.idesc, kk > 0);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) umma_bf16(acc, pd1 + 2 * kk, vd1 + 2 * kk, p.idesc, 1u);
-                umma_commit(smem_u32(&bars[3 + s]));       // V stage free
-                umma_commit(smem_u32(&bars[10]));          // P buffer free
-                umma_commit(smem_u32(&bars[11 + s]));      // O_tile(i) ready
+                for (int kk = 0; kk < 4; ++kk) umma_bf16_ta(acc, pa + 32 + 8 * kk, vd1 + 2 * kk, p.idesc, 1u);
+                umma_commit(smem_u32(&bars[kVEmpty + vs]));    // V stage free
+                umma_commit(smem_u32(&bars[kOFull + s]));      // O_tile(i) ready
             }
             if (!ok) {
                 *abort_flag = 1;
@@ -255,7 +261,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // time to finish while this thread was busy with the next tile's softmax
         auto fold = [&](int j, float alpha) {
             const int s = j & 1;
-            if (!mbar_wait(smem_u32(&bars[11 + s]), (uint32_t)(j >> 1) & 1u, abort_flag)) { *abort_flag = 1; ok = false; }
+            if (!mbar_wait(smem_u32(&bars[kOFull + s]), (uint32_t)(j >> 1) & 1u, abort_flag)) { *abort_flag = 1; ok = false; }
             tc_fence_after();
             if (live) {
 #pragma unroll
@@ -267,25 +273,28 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 }
             }
             tc_fence_before();
-            mbar_arrive(smem_u32(&bars[13 + s]));          // O_tile buffer may be overwritten
+            mbar_arrive(smem_u32(&bars[kOEmpty + s]));     // O_tile buffer may be overwritten
         };
         for (int i = 0; i < n_kt; ++i) {
             const int s = i & 1;
             // A failed wait must not leave the loop before the named barrier below (the other
             // warps would wait there for ever): it raises the CTA's abort flag, every thread still
             // reaches the barrier, and all of them leave together right after it.
-            if (!mbar_wait(smem_u32(&bars[5 + s]), (uint32_t)(i >> 1) & 1u, abort_flag)) *abort_flag = 1;
+            if (!mbar_wait(smem_u32(&bars[kSFull + s]), (uint32_t)(i >> 1) & 1u, abort_flag)) *abort_flag = 1;
             tc_fence_after();
             const int n_keys = min(kTile, n_vis - (kt_begin + i) * kTile);   // valid keys in this tile
             // keys past n_vis may hold anything: zero their V columns so that 0 * garbage stays 0.
             // Thread (r, hf) owns row r (a head dim) of atom hf (keys 64*hf..) of the transposed V tile.
             if (n_keys < c_off + 64) {
-                if (!mbar_wait(smem_u32(&bars[15 + s]), (uint32_t)(i >> 1) & 1u, abort_flag)) *abort_flag = 1;   // V landed
-                uint8_t* vt = sKV + (size_t)s * 2 * kOperand + kOperand + hf * kAtom + r * 128;
+                if (!mbar_wait(smem_u32(&bars[kVFull + i % kStages]), (uint32_t)(i / kStages) & 1u, abort_flag)) *abort_flag = 1;   // V landed
+                uint8_t* vt = sV + (size_t)(i % kStages) * kOperand + hf * kAtom + r * 128;
                 for (int kv = max(n_keys - c_off, 0); kv < 64; ++kv)
                     *reinterpret_cast<uint16_t*>(vt + (((kv >> 3) ^ (r & 7)) << 4) + (kv & 7) * 2) = 0;
             }
-            // scaled scores of this thread's 64 keys, kept in registers for both passes
+            // This thread's 64 raw scores stay in registers for both passes.  The softmax warps are
+            // bound by instruction issue, so the passes are kept to one FMNMX, then one FFMA + one MUFU
+            // + one FADD (+ half a pack) per score: the scale is folded into the exponent's FFMA
+            // (exp2(s * c - m * c)), and only the last, ragged key tile pays for the masking.
             float sc[64];
             float mx = -INFINITY;
             if (live) {
@@ -293,47 +302,53 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 for (int c0 = 0; c0 < 64; c0 += 32) {
                     uint32_t v[32];
                     tmem_ld32(t_row + (uint32_t)(s * kTile + c_off + c0), v);
+                    if (n_keys >= kTile) {
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) {
-                        sc[c0 + c] = (c_off + c0 + c < n_keys) ? __uint_as_float(v[c]) * p.scale_log2e : -INFINITY;
-                        mx = fmaxf(mx, sc[c0 + c]);
+                        for (int c = 0; c < 32; ++c) {
+                            sc[c0 + c] = __uint_as_float(v[c]);
+                            mx = fmaxf(mx, sc[c0 + c]);
+                        }
+                    } else {
+#pragma unroll
+                        for (int c = 0; c < 32; ++c) {
+                            sc[c0 + c] = (c_off + c0 + c < n_keys) ? __uint_as_float(v[c]) : -INFINITY;
+                            mx = fmaxf(mx, sc[c0 + c]);
+                        }
                     }
                 }
+                mx *= p.scale_log2e;                       // the scale is positive; -inf stays -inf
             }
-            tc_fence_before();
-            mbar_arrive(smem_u32(&bars[7 + s]));           // S buffer may be overwritten
             xch[hf * kTile + r] = mx;
             asm volatile("bar.sync 1, 256;" ::: "memory");
             if (*abort_flag) { ok = false; break; }
             float alpha = 0.f;
             if (live) {
                 mx = fmaxf(fmaxf(mx, xch[(hf ^ 1) * kTile + r]), m);
-                alpha = exp2f(m - mx);                     // m = -inf on the first tile gives 0
+                alpha = ex2_approx(m - mx);                // m = -inf on the first tile gives 0
                 m = mx;
                 l *= alpha;
             }
-            // P V of the previous tile must have finished reading the P buffer
-            if (!mbar_wait(smem_u32(&bars[10]), ((uint32_t)i & 1u) ^ 1u, abort_flag)) { *abort_flag = 1; ok = false; }
+            // P(i) as bf16 pairs over the S buffer: both threads of the row hold their scores in registers
+            // (the barrier above), and the tensor core is done with whatever these columns held before
             if (live) {
-                uint8_t* prow = sP + hf * kAtom + r * 128;
+                uint32_t pw[32];
+                const float neg_mx = -mx;
+                float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-                for (int g = 0; g < 8; ++g) {              // eight 16-byte chunks of 8 keys
-                    float pr[8];
-#pragma unroll
-                    for (int c = 0; c < 8; ++c) {
-                        pr[c] = exp2f(sc[8 * g + c] - mx); // masked keys: exp2(-inf) = 0
-                        l += pr[c];
-                    }
-                    uint4 u;
-                    u.x = pack_bf16(pr[0], pr[1]);
-                    u.y = pack_bf16(pr[2], pr[3]);
-                    u.z = pack_bf16(pr[4], pr[5]);
-                    u.w = pack_bf16(pr[6], pr[7]);
-                    *reinterpret_cast<uint4*>(prow + ((g ^ (r & 7)) << 4)) = u;
+                for (int g = 0; g < 32; ++g) {
+                    // masked keys: fma(-inf, c, -m) = -inf, exp2(-inf) = 0
+                    const float p0 = ex2_approx(fmaf(sc[2 * g], p.scale_log2e, neg_mx));
+                    const float p1 = ex2_approx(fmaf(sc[2 * g + 1], p.scale_log2e, neg_mx));
+                    l0 += p0;
+                    l1 += p1;
+                    pw[g] = pack_bf16(p0, p1);
                 }
+                l += l0 + l1;
+                tmem_st32(t_row + (uint32_t)(s * kTile + 32 * hf), pw);
             }
-            fence_proxy_async_smem();                      // P and the zeroed V columns -> visible to the MMA
-            mbar_arrive(smem_u32(&bars[9]));
+            fence_proxy_async_smem();                      // the zeroed V columns -> visible to the MMA
+            tc_fence_before();
+            mbar_arrive(smem_u32(&bars[kPFull]));
             if (i > 0) fold(i - 1, alpha_prev);
             alpha_prev = alpha;
         }
@@ -546,7 +561,7 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     if (want > max_kt) want = max_kt;
     p.tiles_per_split = (max_kt + want - 1) / want;
     p.max_parts = (max_kt + p.tiles_per_split - 1) / p.tiles_per_split;
-    const size_t smem = 7 * (size_t)kOperand + (kBars + 1) * 8 + 16 + 2 * kTile * 4 + 1024;
+    const size_t smem = (1 + 2 * kStages) * (size_t)kOperand + (kBars + 1) * 8 + 16 + 2 * kTile * 4 + 1024;
     static bool attr_done = false;      // one device per process
     if (!attr_done) {
         WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
