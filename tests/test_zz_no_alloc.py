@@ -6,6 +6,8 @@ calls once running).  It keeps its split-K partial sums in a fixed array inside
 the library, shared by all calls, so the checks here are: it agrees with the
 ordinary entry point, also on a second call that finds the first call's leftovers
 in the array, and it refuses shapes the array cannot hold."""
+import gc
+
 import numpy as np
 import pytest
 import torch
@@ -34,6 +36,7 @@ def test_noalloc_gemm_matches_ordinary_entry_point_twice_in_a_row():
     x2, w2 = _pair(7, 1000, 264, 2)
     y2 = torch.empty(7, 1000, dtype=torch.float32, device=DEV)
     ref2 = wd.op_gemm(x2, w2, wd.WD_GEMM_TCGEN05)
+    gc.collect()                       # tensors of earlier tests must not be freed between the two readings
     torch.cuda.synchronize()
     before = torch.cuda.memory_allocated()
     wd.op_gemm_noalloc(x1, w1, y1)
