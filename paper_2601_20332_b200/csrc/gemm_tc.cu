@@ -774,8 +774,13 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     if (warp == 0) {
         if (lane == 0 && n_total > 0) {
             // ------------------------------------------------ TMA producer (both CTAs, own halves)
+            // weights that one or two units use are streamed past the L2 (evict first); with more token
+            // tiles the same weight block is wanted again by the units that follow: keep it (evict last)
             uint64_t pol_stream;
-            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            if (p.tok_tiles > 2)
+                asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol_stream));
+            else
+                asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
             struct Walk {
                 int piece, left, kb, n0, tok0;
                 const CUtensorMap* mw;
