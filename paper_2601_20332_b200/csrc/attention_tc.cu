@@ -40,7 +40,7 @@ constexpr int kAtom = kTile * 64 * 2;      // one [128 x 64] bf16 swizzle-atom c
 constexpr int kOperand = 2 * kAtom;        // a [128 x 128] bf16 operand: 32 KB
 constexpr int kThreads = 320;            // TMA warp, MMA warp, 8 softmax warps
 constexpr int kTmemCols = 512;             // S0, S1: columns 0..255; O_tile0, O_tile1: columns 256..511
-constexpr int kBars = 20;
+constexpr int kBars = 21;
 constexpr int kMaxCluster = 8;             // portable cluster size
 
 struct AttnParams {
@@ -93,8 +93,8 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 }
 
 // barrier indices
-constexpr int kQFull = 0, kKFull = 1, kKEmpty = 4, kVFull = 7, kVEmpty = 10, kSFull = 13, kPFull = 15, kOFull = 16,
-              kOEmpty = 18;
+constexpr int kQFull = 0, kKFull = 1, kKEmpty = 4, kVFull = 7, kVEmpty = 10, kSFull = 13, kPFull = 15, kOFull = 17,
+              kOEmpty = 19;
 constexpr int kStages = 3;                 // K stages and V stages
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -107,8 +107,11 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     uint8_t* sK = smem + kOperand;               // 3 stages x 32 KB
     uint8_t* sV = sK + kStages * kOperand;       // 3 stages x 32 KB (transposed V tiles)
     uint64_t* bars = (uint64_t*)(sV + kStages * kOperand);
-    // q_full | k_full[3] | k_empty[3] | v_full[3] | v_empty[3] | s_full[2] | p_full | o_full[2] | o_empty[2].
-    // p_full and o_empty count the 256 softmax threads.  P never touches shared memory: the softmax
+    // q_full | k_full[3] | k_empty[3] | v_full[3] | v_empty[3] | s_full[2] | p_full[2] | o_full[2] | o_empty[2].
+    // p_full and o_empty count the 256 softmax threads.  p_full is one barrier per S buffer, not one for all
+    // tiles: the softmax threads can finish P(i+1) before the MMA thread has looked at P(i)'s barrier (it waits
+    // for V(i) first), and a single barrier would then have gone through two phases unseen; P(i+2) on the
+    // other hand needs S(i+2), which is issued only after the MMA thread has seen P(i).  P never touches shared memory: the softmax
     // threads write it as bf16 over the S buffer they have just read (tcgen05.st) and P V takes its A
     // operand from tensor memory.  No "S empty" / "P empty" barriers are needed: the tensor core runs the
     // MMAs in issue order (Q K^T(i+1), P V(i), Q K^T(i+2), ...), so S buffer i & 1 is rewritten by
@@ -138,7 +141,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     if (has_work) {
         if (threadIdx.x == 0) {
             for (int i = 0; i < kBars; ++i)
-                mbar_init(smem_u32(&bars[i]), (i == kPFull || i == kOEmpty || i == kOEmpty + 1) ? 256u : 1u);
+                mbar_init(smem_u32(&bars[i]), (i == kPFull || i == kPFull + 1 || i == kOEmpty || i == kOEmpty + 1) ? 256u : 1u);
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
@@ -219,7 +222,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 const uint32_t ph = (uint32_t)(i >> 1) & 1u;
                 if (i + 1 < n_kt && !(ok = issue_qk(i + 1))) break;                           // runs ahead of the softmax
                 if (!(ok = mbar_wait(smem_u32(&bars[kVFull + vs]), (uint32_t)(i / kStages) & 1u, abort_flag))) break;   // V(i) landed
-                if (!(ok = mbar_wait(smem_u32(&bars[kPFull]), (uint32_t)i & 1u, abort_flag))) break;    // P(i) written
+                if (!(ok = mbar_wait(smem_u32(&bars[kPFull + s]), ph, abort_flag))) break;              // P(i) written
                 if (!(ok = mbar_wait(smem_u32(&bars[kOEmpty + s]), ph ^ 1u, abort_flag))) break;        // O_tile(i-2) folded
                 tc_fence_after();
                 const uint32_t sv = smem_u32(sV + (size_t)vs * kOperand);
@@ -348,7 +351,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             }
             fence_proxy_async_smem();                      // the zeroed V columns -> visible to the MMA
             tc_fence_before();
-            mbar_arrive(smem_u32(&bars[kPFull]));
+            mbar_arrive(smem_u32(&bars[kPFull + s]));
             if (i > 0) fold(i - 1, alpha_prev);
             alpha_prev = alpha;
         }

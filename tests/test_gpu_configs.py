@@ -106,6 +106,16 @@ def test_cfg5_sweep_corner_late_state():
     assert logs[1]["info"]["n_rows"] == 2 * 129 and logs[1]["info"]["n_vis"] == 2 * 2048
 
 
+def test_cfg5_sweep_batch8_small_window_many_key_tiles():
+    """Sweep point A=16 B=64 R=16 at batch 8: 256 attention CTAs (two waves) of nine key tiles with 17
+    valid query rows each, K/V streamed from HBM.  The softmax warps run a tile ahead of the MMA thread
+    here (it waits for V first), which a single 'P written' barrier did not survive."""
+    cfg = synth.get_config("llada8b_sweep", L=1, A=16, B=64, R=16, batch=8)
+    logs = run_cfg(cfg, 3, oracle_seqs=[3])
+    assert [l["info"]["is_refresh"] for l in logs] == [1, 0, 0]
+    assert logs[1]["info"]["n_rows"] == 8 * 17 and logs[1]["info"]["n_vis"] == 8 * 1104
+
+
 def test_cfg2_window_only_refresh_variant_at_full_width():
     """The variant outside the paper at the LLaDA-8B width: the second refresh computes the new
     window and the previous phase's tokens only (104 rows instead of 360)."""
