@@ -701,7 +701,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 //             on them through .cta_group::2), issues every MMA, releases the stages and publishes the
 //             accumulators in BOTH CTAs (tcgen05.commit with a CTA mask)
 //   both:     TMA producer for their own operand halves, epilogue for their own 128 weight rows;
-//             epilogue threads of both CTAs arrive on the even CTA's "accumulator empty" barriers
+//             epilogue warps of both CTAs arrive on the even CTA's "accumulator empty" barriers
+// Two-accumulator modes (TcParams::dual): each weight stage feeds two MMA chains, either against two
+// halves of a 2*BN-token super-tile (the weights enter shared memory once per 512 tokens) or with the
+// gate and the up block of the same FFN columns against one token tile (the epilogue then writes
+// silu(gate) * up as bf16).  With BN > 128 the two accumulators fill the tensor memory, so there is one
+// accumulator set and the epilogue of a unit does not overlap the next unit's MMAs.
+// Whole-tile schedule: units are dealt round-robin in (token group, weight tile, token tile) order so
+// that the pairs running at one time share a few weight tiles and one token group in the L2.
 template <bool kFp8>
 __global__ void __launch_bounds__(kThreadsPair)
 gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w0,
