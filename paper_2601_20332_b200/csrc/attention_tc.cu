@@ -251,7 +251,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         // warps whose 32 rows are all beyond the valid ones only keep the barrier counts right.
         // The test is per warp, not per row: tcgen05.ld is warp-collective and must not diverge.
         const bool live = quarter * 32 < n_valid;
-        const bool fold_first = (quarter & 1) != 0;
         const bool valid = r < n_valid;
         const int c_off = 64 * hf;
         const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
@@ -332,9 +331,6 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 m = mx;
                 l *= alpha;
             }
-            // The exponentials below are bound by the special-function unit while the rescale of O does not
-            // use it: half of the warps (odd quarters) rescale first, so the two phases overlap across warps.
-            if (fold_first && i > 0) fold(i - 1, alpha_prev);
             // P(i) as bf16 pairs over the S buffer: both threads of the row hold their scores in registers
             // (the barrier above), and the tensor core is done with whatever these columns held before
             if (live) {
@@ -356,7 +352,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             fence_proxy_async_smem();                      // the zeroed V columns -> visible to the MMA
             tc_fence_before();
             mbar_arrive(smem_u32(&bars[kPFull + s]));
-            if (!fold_first && i > 0) fold(i - 1, alpha_prev);
+            if (i > 0) fold(i - 1, alpha_prev);
             alpha_prev = alpha;
         }
         if (ok && n_kt > 0) fold(n_kt - 1, alpha_prev);
