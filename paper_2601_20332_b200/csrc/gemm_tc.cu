@@ -1147,14 +1147,19 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
             tiles_all += (segs[i].n + p.tile_rows - 1) / p.tile_rows;
             ncol_all += segs[i].n;
         }
+        // whole units pay when every pair gets two or more, or when the one or two rounds are nearly full
+        const long long pairs = sm_count / 2;
+        auto full_rounds = [&](long long units) {
+            return units >= 2 * pairs || (units >= pairs && 10 * units >= 9 * pairs * ((units + pairs - 1) / pairs));
+        };
         const long long dual_units = (long long)tiles_all * ((rows + 511) / 512);
-        p.dual = (dual_mode == 2 || (dual_mode == 1 && ncol_all >= 16384 && dual_units >= 2 * (sm_count / 2))) ? 1 : 0;
+        p.dual = (dual_mode == 2 || (dual_mode == 1 && ncol_all >= 16384 && dual_units >= 2 * pairs)) ? 1 : 0;
         // gate and up against the same tokens, h = silu(gate) * up written by the epilogue: needs whole
-        // tiles per pair (no partial sums), taken when every pair gets at least two of them
+        // tiles per pair (no partial sums)
         static const int swiglu_fused = env_int("WD_GEMM_SWIGLU", 1);
         if (sg && sg->h && swiglu_fused && !fp8 && nseg == 2 && segs[0].n == segs[1].n && dual_mode != 0) {
             const long long gu_units = (long long)((segs[0].n + p.tile_rows - 1) / p.tile_rows) * ((rows + 255) / 256);
-            if (gu_units >= 2 * (sm_count / 2)) p.dual = 2;
+            if (full_rounds(gu_units)) p.dual = 2;
         }
     }
     if (p.dual == 1) {
