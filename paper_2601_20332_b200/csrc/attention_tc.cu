@@ -254,7 +254,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const bool valid = r < n_valid;
         const int c_off = 64 * hf;
         const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
-        float* xch = (float*)(tmem_slot + 4);              // [2][128] exchange between the two halves
+        float* xch = (float*)(tmem_slot + 4);              // [2][128] exchange between the two halves (row sums)
+        uint16_t* xm = (uint16_t*)xch;                     // the same 1 KB as [2 parities][2][128] bf16 row maxima
         float o[64];
 #pragma unroll
         for (int c = 0; c < 64; ++c) o[c] = 0.f;
@@ -321,12 +322,21 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 }
                 mx *= p.scale_log2e;                       // the scale is positive; -inf stays -inf
             }
-            xch[hf * kTile + r] = mx;
+            // The two halves of a row must use the same reference value, and any upper bound of the scores
+            // serves (softmax does not depend on it): each half rounds its maximum up to bf16 and both take
+            // the larger.  Sixteen bits per value leave room for one buffer per tile parity, so a thread
+            // that is already a tile ahead cannot overwrite what its partner has yet to read.
+            {
+                uint32_t mb = __float_as_uint(mx);
+                mb = (mb & 0x80000000u) ? (mb & 0xffff0000u) : ((mb + 0xffffu) & 0xffff0000u);
+                mx = __uint_as_float(mb);
+                xm[((i & 1) * 2 + hf) * kTile + r] = (uint16_t)(mb >> 16);
+            }
             asm volatile("bar.sync 1, 256;" ::: "memory");
             if (*abort_flag) { ok = false; break; }
             float alpha = 0.f;
             if (live) {
-                mx = fmaxf(fmaxf(mx, xch[(hf ^ 1) * kTile + r]), m);
+                mx = fmaxf(fmaxf(mx, __uint_as_float((uint32_t)xm[((i & 1) * 2 + (hf ^ 1)) * kTile + r] << 16)), m);
                 alpha = ex2_approx(m - mx);                // m = -inf on the first tile gives 0
                 m = mx;
                 l *= alpha;
