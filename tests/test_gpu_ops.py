@@ -25,6 +25,9 @@ GEMM_SHAPES = [  # rows, n, k  (ragged token counts, several tiles, ragged weigh
     (1, 128, 64), (7, 256, 128), (16, 128, 512), (34, 384, 1024), (35, 640, 4096), (68, 512, 2048),
     (130, 256, 1024), (256, 384, 512), (300, 256, 1024), (352, 512, 768), (700, 384, 512), (34, 200, 256),
     (10, 1000, 264), (512, 1000, 264), (1030, 256, 2048), (264, 130, 72),
+    # wide weight matrices with every CTA pair getting two units: two accumulators per weight stage
+    # (token super-tiles of 2 x 160 and 3 x 2 x 192 rows, ragged last weight tile)
+    (300, 38016, 128), (1100, 16640, 192),
 ]
 
 
