@@ -426,6 +426,15 @@ WD_API size_t wd_op_unmask_scratch_bytes(int32_t n, int32_t vocab);
  * call.  Synchronises the device. */
 WD_API wd_status wd_op_status(void);
 
+/* Exercises the library's error path for device-side waits without any fault: one
+ * thread waits, with the same bounded wait every kernel of the library uses, on a
+ * shared-memory barrier that nothing ever signals.  The wait gives up after its
+ * time limit (two seconds), the kernel records
+ * WD_ERR_DEVICE_TIMEOUT in the operations' status word and returns normally; the
+ * context stays usable.  wd_op_status() then reports and clears the code.
+ * `stream`: a CUDA stream handle or NULL.  Errors: WD_ERR_CUDA. */
+WD_API wd_status wd_debug_wait_expire(void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -95,6 +95,7 @@ SIGNATURES = {
     "wd_op_unmask": (C.c_int, [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]),
     "wd_op_unmask_scratch_bytes": (C.c_size_t, [i32, i32]),
     "wd_op_status": (C.c_int, []),
+    "wd_debug_wait_expire": (C.c_int, [vp]),
 }
 
 _lib = None
@@ -430,3 +431,8 @@ def op_unmask(logits, positions, k: int, stream=None) -> dict:
 
 def op_status() -> int:
     return lib().wd_op_status()
+
+
+def debug_wait_expire(stream=None) -> None:
+    """Launch the kernel whose bounded wait runs out (see wd_debug_wait_expire)."""
+    check(lib().wd_debug_wait_expire(_stream_ptr(stream)), "wd_debug_wait_expire")

@@ -1293,6 +1293,8 @@ extern "C" wd_status wd_op_unmask(const float* logits, const int32_t* positions,
     return WD_OK;
 }
 
+extern "C" wd_status wd_debug_wait_expire(void* stream) { return wd_launch_wait_expire((cudaStream_t)stream); }
+
 extern "C" wd_status wd_op_status(void) {
     int32_t* p = wd_op_status_ptr();
     if (!p) return WD_ERR_CUDA;

@@ -7,7 +7,10 @@
 
 namespace wdk {
 
-constexpr uint32_t kWaitLimit = 1u << 22;   // polls of one bounded wait before it gives up
+constexpr uint32_t kWaitLimit = 1u << 22;   // polls of one bounded wait before it gives up, whatever the clock says
+constexpr unsigned long long kWaitNs = 2000000000ull;   // ... and the time after which it gives up: 2 s.  The longest
+                                                        // legitimate wait is a dependent kernel, launched early, sitting
+                                                        // out its predecessor (tens of milliseconds at the largest shapes)
 
 // Programmatic dependent launch: let the next kernel of the stream start its prologue now /
 // wait until every kernel this one depends on has finished and its writes are visible.
@@ -36,13 +39,25 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
-// Bounded wait.  Returns false if the limit ran out or another role already gave up.
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false if the time or poll limit ran out or another role already gave up.
+// The clock is read only on the slow path (every 256th poll after the first 128).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    unsigned long long t0 = 0;
     for (uint32_t it = 0; it < kWaitLimit; ++it) {
         if (mbar_try_wait(bar, parity)) return true;
         if (it >= 128) {
             __nanosleep(64);
-            if ((it & 255) == 0 && *abort_flag) return false;
+            if ((it & 255) == 0) {
+                if (*abort_flag) return false;
+                const unsigned long long now = global_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > kWaitNs) return false;
+            }
         }
     }
     return false;

@@ -1059,6 +1059,26 @@ void wd_launch_plan(const WdPlanLaunch& h, cudaStream_t st) {
     launch_pdl(plan_kernel, dim3(h.batch), dim3(256), 0, st, a);
 }
 
+// A bounded wait that is never satisfied: the barrier expects one arrival and nobody arrives.
+__global__ void wait_expire_kernel(int32_t* status) {
+    __shared__ uint64_t bar;
+    __shared__ int abort_flag;
+    if (threadIdx.x == 0) {
+        abort_flag = 0;
+        wdk::mbar_init(wdk::smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (!wdk::mbar_wait(wdk::smem_u32(&bar), 0, &abort_flag)) atomicCAS(status, 0, WD_ERR_DEVICE_TIMEOUT);
+    }
+}
+
+wd_status wd_launch_wait_expire(cudaStream_t st) {
+    int32_t* status = wd_op_status_ptr();
+    if (!status) return WD_ERR_CUDA;
+    wait_expire_kernel<<<1, 32, 0, st>>>(status);
+    ++wd_launch_counter;
+    return cudaGetLastError() == cudaSuccess ? WD_OK : WD_ERR_CUDA;
+}
+
 int32_t* wd_op_status_ptr() {
     int32_t* p = nullptr;
     if (cudaGetSymbolAddress((void**)&p, g_op_status) != cudaSuccess) return nullptr;

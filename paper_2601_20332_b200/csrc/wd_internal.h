@@ -165,5 +165,6 @@ struct WdPlanLaunch {
 };
 void wd_launch_plan(const WdPlanLaunch& h, cudaStream_t st);
 
+wd_status wd_launch_wait_expire(cudaStream_t st);
 int32_t* wd_op_status_ptr();   // device address of the single-operation status word
 extern bool wd_pdl_enabled;    // programmatic dependent launch on every kernel (default on)

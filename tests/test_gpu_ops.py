@@ -144,3 +144,19 @@ def test_unmask_exact_ties():
     assert got["row_conf"][1] == got["row_conf"][4]                     # identical rows give identical bits
     np.testing.assert_allclose(got["row_conf"][0], 1.0 / V, rtol=1e-6)  # all-equal logits: 1 / V
     assert abs(got["row_conf"][2] - 1.0) < 1e-6
+
+
+def test_bounded_wait_runs_out_and_the_context_stays_usable():
+    """A device-side wait that nothing satisfies gives up after its iteration limit, the kernel
+    returns normally with WD_ERR_DEVICE_TIMEOUT in the status word (no trap, no hang), the word is
+    cleared by reading it, and the next operation on the same context works."""
+    assert wd.op_status() == 0
+    wd.debug_wait_expire()
+    assert wd.op_status() == wd.WD_ERR_DEVICE_TIMEOUT
+    assert wd.op_status() == 0
+    g = torch.Generator(device=DEV).manual_seed(5)
+    x = torch.randn(34, 256, device=DEV, generator=g).to(torch.bfloat16)
+    w = (torch.randn(384, 256, device=DEV, generator=g) * 0.05).to(torch.bfloat16)
+    y = wd.op_gemm(x, w, wd.WD_GEMM_TCGEN05)
+    assert wd.op_status() == 0
+    assert np.abs(y.cpu().numpy() - _ref_gemm(x, w)).max() / np.abs(_ref_gemm(x, w)).max() < 2e-5
