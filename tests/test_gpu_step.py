@@ -1,4 +1,6 @@
 """Parity of the whole windowed step against the CPU oracle (GPU required)."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -80,6 +82,21 @@ def test_bf16_head_dim_128_tensor_core_attention(Hkv, batch, fusion):
     logs = run(cfg, 7, fusion=fusion)
     assert [l["info"]["is_refresh"] for l in logs] == [1, 0, 0, 1, 0, 0, 1]
     assert logs[0]["info"]["n_rows"] == batch * 256
+
+
+def test_gate_up_swiglu_epilogue_with_ragged_ffn_width_and_token_tile():
+    """d_ffn 19008 = 74 whole 256-row tiles + 64 rows, 262 rows at the second refresh (token tiles of
+    144 and 118): every CTA pair gets two (gate tile, up tile) units, so the two-CTA GEMM writes
+    h = silu(gate) * up itself; the last weight tile and the second token tile are partial.  The
+    layer outputs (which h feeds through the down projection) follow the oracle."""
+    cfg = synth.get_config("llada8b", L=1, d=256, Hq=2, Hkv=2, dh=128, F=19008, V=2000, P=200, G=100, A=16, B=40,
+                           R=3, T=2, k=2)
+    logs = run(cfg, 4)
+    assert [l["info"]["is_refresh"] for l in logs] == [1, 0, 0, 1]
+    assert logs[0]["info"]["n_rows"] == 256 and logs[3]["info"]["n_rows"] > 256
+    if not any(os.environ.get(k) == "0" for k in ("WD_GEMM_DUAL", "WD_GEMM_SWIGLU", "WD_GEMM_PAIR_FROM")):
+        # no SwiGLU kernel in the second refresh: one launch fewer than in the first (256 rows, one-CTA GEMMs)
+        assert logs[3]["info"]["n_launches"] == logs[0]["info"]["n_launches"] - 1
 
 
 @pytest.mark.parametrize("batch,A", [(2, 160), (4, 150), (4, 250)])
