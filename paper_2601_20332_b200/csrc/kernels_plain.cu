@@ -471,48 +471,52 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
                                     const int32_t* __restrict__ row_seq, const int32_t* __restrict__ row_pos,
                                     const float2* __restrict__ rope_tab, T* __restrict__ q, T* __restrict__ kcache,
                                     T* __restrict__ vcache, int n_rows, int Hq, int Hkv, int dh, int S, int Sp,
-                                    int n_qk, int qk_groups) {
+                                    int n_qk, int qk_groups, int n_qk_blocks) {
     __shared__ float tile[32][33];
     pdl_launch_dependents();
     pdl_wait();
     const int half = dh >> 1;
     const int ncol = (Hq + 2 * Hkv) * dh;
-    if ((int)blockIdx.x < n_qk) {
-        const int r = blockIdx.x / qk_groups, grp = blockIdx.x - r * qk_groups;
-        const int pos = row_pos[r], b = row_seq[r];
-        const float* pr = part + (size_t)r * ncol;
-        if ((half & 3) == 0) {
-            // four rotation pairs per thread (float4 loads, 8-byte bf16 stores): half/4 threads per head
-            const int tph = half >> 2, hpb = blockDim.x / tph;
-            const int h = grp * hpb + (int)threadIdx.x / tph, j = ((int)threadIdx.x % tph) * 4;
-            if ((int)threadIdx.x < hpb * tph && h < Hq + Hkv) {
-                const float4 a = sum_slices4(pr + h * dh + j, n_split, split_stride);
-                const float4 bb = sum_slices4(pr + h * dh + half + j, n_split, split_stride);
-                const float4 c01 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j);       // (cos, sin) x 2
-                const float4 c23 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j + 2);
-                T* dst = h < Hq ? q + ((size_t)r * Hq + h) * dh : kcache + (((size_t)b * Hkv + (h - Hq)) * S + pos) * dh;
-                Vec4<T>::store(dst + j, a.x * c01.x - bb.x * c01.y, a.y * c01.z - bb.y * c01.w, a.z * c23.x - bb.z * c23.y,
-                               a.w * c23.z - bb.w * c23.w);
-                Vec4<T>::store(dst + j + half, bb.x * c01.x + a.x * c01.y, bb.y * c01.z + a.y * c01.w,
-                               bb.z * c23.x + a.z * c23.y, bb.w * c23.z + a.w * c23.w);
+    if ((int)blockIdx.x < n_qk_blocks) {
+        // a block walks (row, head group) items n_qk_blocks apart: with thousands of rows one item per block
+        // would be all launch overhead
+        for (int item = blockIdx.x; item < n_qk; item += n_qk_blocks) {
+            const int r = item / qk_groups, grp = item - r * qk_groups;
+            const int pos = row_pos[r], b = row_seq[r];
+            const float* pr = part + (size_t)r * ncol;
+            if ((half & 3) == 0) {
+                // four rotation pairs per thread (float4 loads, 8-byte bf16 stores): half/4 threads per head
+                const int tph = half >> 2, hpb = blockDim.x / tph;
+                const int h = grp * hpb + (int)threadIdx.x / tph, j = ((int)threadIdx.x % tph) * 4;
+                if ((int)threadIdx.x < hpb * tph && h < Hq + Hkv) {
+                    const float4 a = sum_slices4(pr + h * dh + j, n_split, split_stride);
+                    const float4 bb = sum_slices4(pr + h * dh + half + j, n_split, split_stride);
+                    const float4 c01 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j);       // (cos, sin) x 2
+                    const float4 c23 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j + 2);
+                    T* dst = h < Hq ? q + ((size_t)r * Hq + h) * dh : kcache + (((size_t)b * Hkv + (h - Hq)) * S + pos) * dh;
+                    Vec4<T>::store(dst + j, a.x * c01.x - bb.x * c01.y, a.y * c01.z - bb.y * c01.w, a.z * c23.x - bb.z * c23.y,
+                                   a.w * c23.z - bb.w * c23.w);
+                    Vec4<T>::store(dst + j + half, bb.x * c01.x + a.x * c01.y, bb.y * c01.z + a.y * c01.w,
+                                   bb.z * c23.x + a.z * c23.y, bb.w * c23.z + a.w * c23.w);
+                }
+                continue;
             }
-            return;
-        }
-        const int h0 = grp * 4;
-        for (int i = threadIdx.x; i < 4 * half; i += blockDim.x) {
-            const int h = h0 + i / half, j = i % half;
-            if (h >= Hq + Hkv) break;
-            const float a = sum_slices1(pr + h * dh + j, n_split, split_stride);
-            const float bb = sum_slices1(pr + h * dh + j + half, n_split, split_stride);
-            const float2 cs = rope_tab[(size_t)r * half + j];
-            const float ra = a * cs.x - bb * cs.y, rb = bb * cs.x + a * cs.y;
-            T* dst = h < Hq ? q + ((size_t)r * Hq + h) * dh : kcache + (((size_t)b * Hkv + (h - Hq)) * S + pos) * dh;
-            dst[j] = from_f<T>(ra);
-            dst[j + half] = from_f<T>(rb);
+            const int h0 = grp * 4;
+            for (int i = threadIdx.x; i < 4 * half; i += blockDim.x) {
+                const int h = h0 + i / half, j = i % half;
+                if (h >= Hq + Hkv) break;
+                const float a = sum_slices1(pr + h * dh + j, n_split, split_stride);
+                const float bb = sum_slices1(pr + h * dh + j + half, n_split, split_stride);
+                const float2 cs = rope_tab[(size_t)r * half + j];
+                const float ra = a * cs.x - bb * cs.y, rb = bb * cs.x + a * cs.y;
+                T* dst = h < Hq ? q + ((size_t)r * Hq + h) * dh : kcache + (((size_t)b * Hkv + (h - Hq)) * S + pos) * dh;
+                dst[j] = from_f<T>(ra);
+                dst[j + half] = from_f<T>(rb);
+            }
         }
         return;
     }
-    const int vb = blockIdx.x - n_qk;
+    const int vb = blockIdx.x - n_qk_blocks;
     const int dchunks = (dh + 31) / 32, rchunks = (n_rows + 31) / 32;
     const int kh = vb / (dchunks * rchunks), rem = vb - kh * dchunks * rchunks;
     const int d0 = (rem / rchunks) * 32, r0 = (rem % rchunks) * 32;
@@ -936,9 +940,10 @@ void wd_launch_rope_scatter(int dtype, const float* part, int n_split, size_t sp
     const int qk_groups = (half & 3) == 0 ? wd_ceil_div(Hq + Hkv, std::max(1, 256 / (half >> 2))) : wd_ceil_div(Hq + Hkv, 4);
     const int n_qk = n_rows * qk_groups;
     const int n_v = Hkv * wd_ceil_div(dh, 32) * wd_ceil_div(n_rows, 32);
-    WD_DISPATCH(dtype, launch_pdl(rope_scatter_kernel<T>, dim3(n_qk + n_v), dim3(256), 0, st, part, n_split,
+    const int n_qk_blocks = std::min(n_qk, 148 * 8);
+    WD_DISPATCH(dtype, launch_pdl(rope_scatter_kernel<T>, dim3(n_qk_blocks + n_v), dim3(256), 0, st, part, n_split,
                                   split_stride, row_seq, row_pos, rope_tab, (T*)q, (T*)kcache, (T*)vcache, n_rows, Hq,
-                                  Hkv, dh, S, Sp, n_qk, qk_groups));
+                                  Hkv, dh, S, Sp, n_qk, qk_groups, n_qk_blocks));
 }
 
 void wd_launch_attention_plain(int dtype, const void* q, const void* kcache, const void* vcache,
