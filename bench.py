@@ -96,6 +96,21 @@ class ClockSampler:
         return out
 
 
+def weight_bytes(cfg) -> float:
+    """Bytes of all matrices a step reads once: the transformer blocks and the LM head."""
+    L, d, Hq, Hkv, dh, F, V = (cfg[k] for k in ("L", "d", "Hq", "Hkv", "dh", "F", "V"))
+    w = 2 if cfg["dtype"] == "bf16" else 4
+    return float((d * (Hq + 2 * Hkv) * dh + Hq * dh * d + 3 * d * F) * L * w + V * d * w)
+
+
+def shape_name(cfg) -> str:
+    kind = {"llada8b": "LLaDA-8B-shaped", "llada8b_long": "LLaDA-8B-shaped", "llada8b_sweep": "LLaDA-8B-shaped",
+            "dream7b": "Dream-7B-shaped", "tiny": "tiny"}.get(cfg.get("name", ""), cfg.get("name", "model"))
+    heads = f"{cfg['Hq']} heads" if cfg["Hq"] == cfg["Hkv"] else f"{cfg['Hq']} query / {cfg['Hkv']} KV heads"
+    return (f"{kind} {cfg['dtype']} ({cfg['L']} layers, d {cfg['d']}, {heads} x {cfg['dh']}, FFN {cfg['F']}, "
+            f"vocab {cfg['V']})")
+
+
 def algorithmic_step(cfg, rows, n_act, vis, batch=1):
     """Bytes and FLOPs the method itself must move / compute in one step
     (weights once, K/V of the visible positions read, fresh K/V written)."""
@@ -106,6 +121,18 @@ def algorithmic_step(cfg, rows, n_act, vis, batch=1):
     by = per_layer * L * w + V * d * w + vis * kv_tok + rows * kv_tok
     fl = 2 * rows * per_layer * L + 2 * n_act * d * V + 4 * rows * (vis / max(batch, 1)) * Hq * dh * L
     return by, fl
+
+
+def phase_amortised(normal_ms, refresh_ms, R, tokens_per_step):
+    """A phase is one refresh step and R-1 normal steps; the K timed steps need not hold refresh steps in
+    that proportion, so the per-step time of a whole phase is also given: (refresh + (R-1) normal) / R
+    from the medians of the two kinds."""
+    if not refresh_ms or (R > 1 and not normal_ms):
+        return None
+    r = float(np.median(refresh_ms))
+    n = float(np.median(normal_ms)) if normal_ms else 0.0
+    ms = (r + (R - 1) * n) / R
+    return {"ms_per_step": ms, "value": tokens_per_step / (ms * 1e-3), "unit": UNIT}
 
 
 def max_over_ranks(ms: float, world: int, device) -> float:
@@ -296,14 +323,15 @@ def run_ours(args, rank, world):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": W,
         "ms_per_step": total_ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": cfg["dtype"], "data": "synthetic",
-        "config": {"workload": f"{args.config}: LLaDA-8B-shaped bf16, prompt {cfg['P']} + {cfg['G']} masks, A={A} B={B} R={R} "
+        "config": {"workload": f"{args.config}: {shape_name(cfg)}, prompt {cfg['P']} + {cfg['G']} masks, A={A} B={B} R={R} "
                                f"T={T} k={k} batch {batch}; steps {W}..{W + K - 1} of the generation; replicas only at N>1",
-                   "l2": "inputs larger than L2: every step streams 15 GB of weights",
+                   "l2": f"inputs larger than L2: every step streams {weight_bytes(cfg) / 1e9:.1f} GB of weights",
                    "normal_step_ms": normal_ms, "refresh_step_ms": float(np.median(refresh)) if refresh else None,
                    "normal_step_algorithmic_gb": step_by / 1e9,
                    "normal_step_frac_of_hbm_roofline_measured": (step_by / (normal_ms * 1e-3) / 1e9 / peaks["hbm_gbs"])
                    if normal_ms else None,
                    "normal_step_frac_of_hbm_roofline_nominal_8TBs": (step_by / (normal_ms * 1e-3) / 8e12) if normal_ms else None,
+                   "phase_amortised": phase_amortised(normal, refresh, R, batch * k * world),
                    "full_sequence_step_ms": float(np.median(full_ms)),
                    "rows_normal": float(np.mean([i["n_rows"] for i in ni])) if ni else None,
                    "stepping": "queued: steps enqueued back to back, index lists planned on the device, drained every 16 steps",
@@ -383,7 +411,9 @@ def cpu_baseline(cfg, w, ids, budget_s=25.0):
     phase = t_refresh + (R - 1) * t_normal
     return {"value": k * R / phase, "unit": UNIT, "cores": int(cores), "kind": "oracle",
             "sample": f"one refresh + one normal step of batch-1 sequence 0 at 1 and 2 of {L} layers, extrapolated linearly "
-                      f"in depth; refresh {t_refresh:.1f} s, normal {t_normal:.1f} s per step"}
+                      f"in depth; refresh {t_refresh:.1f} s, normal {t_normal:.1f} s per step; most of either is the oracle's "
+                      f"weight access (each layer's matrices copied from the device and widened bf16 -> fp64 every step), "
+                      f"not its arithmetic, which is why the normal step is not faster than the refresh"}
 
 
 def run_reference(args, rank, world):
@@ -410,6 +440,34 @@ def run_reference(args, rank, world):
                       "e2e": {"value": v, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
 
 
+def run_plumbing_check(args, rank, world):
+    """`--plumbing-check` (used by the CPU tests of the launcher): the rank plumbing of a run without its
+    GPU work.  Every rank joins the process group the launcher set up, contributes a made-up local
+    time, and rank 0 prints a line whose n_gpus is the world size and whose value is the work of all
+    ranks over the slowest rank's time."""
+    local_ms = 10.0 * (rank + 1)
+    total = max_over_ranks(local_ms, world, "cpu")
+    if world > 1:
+        torch.distributed.barrier()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": whole_job_value(args.steps, world, total), "unit": UNIT,
+                          "n_gpus": world, "steps": args.steps, "warmup": args.warmup, "ms_per_step": total / args.steps,
+                          "scaling": "weak", "config": {"workload": "plumbing check: no GPU work"}}))
+
+
+def launch_ranks(args, argv) -> int:
+    """`bench.py --gpus N` started as a plain process: start N ranks of this same command, one per
+    GPU, under torch.distributed.run on this node (rendezvous on 127.0.0.1, a free port) and hand
+    their output through.  Replicas only: NCCL carries the barrier and the MAX of the timings."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + list(argv)
+    return subprocess.call(cmd)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -418,9 +476,33 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--config", default="llada8b")
     ap.add_argument("--cpu-seconds", type=float, default=25.0)
+    ap.add_argument("--plumbing-check", action="store_true",
+                    help="rank plumbing only, over gloo, no GPU work (CPU test of the --gpus launcher)")
     args = ap.parse_args()
+    if args.gpus < 1:
+        ap.error("--gpus must be at least 1")
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        # not under a launcher yet: become N ranks (the reference arm too, whose ranks > 0 exit at once)
+        if not args.plumbing_check and torch.cuda.device_count() < args.gpus:
+            sys.stderr.write(f"bench.py: --gpus {args.gpus} but {torch.cuda.device_count()} CUDA devices are visible\n")
+            sys.exit(2)
+        sys.exit(launch_ranks(args, sys.argv[1:]))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        sys.stderr.write(f"bench.py: --gpus {args.gpus} disagrees with WORLD_SIZE={world}\n")
+        sys.exit(2)
+    if args.plumbing_check:
+        args.steps = 64 if args.steps is None else args.steps
+        args.warmup = 8 if args.warmup is None else args.warmup
+        if world > 1:
+            torch.distributed.init_process_group("gloo")
+        try:
+            run_plumbing_check(args, rank, world)
+        finally:
+            if world > 1:
+                torch.distributed.destroy_process_group()
+        return
     if args.impl == "reference":
         args.steps = 1 if args.steps is None else min(args.steps, 3)
         args.warmup = 0 if args.warmup is None else min(args.warmup, 1)

@@ -34,6 +34,14 @@ The readings the paper does not fix (transient length capped by T and reset at
 a refresh, forced early refresh when the window is exhausted, every model
 constant) are **parity unpinned against the paper**: they are only checked for
 internal consistency.
+
+Precision modes.  The default is plain float64 with no intermediate rounding.
+Two optional modes restate a reduced-precision pipeline's *storage formats* (and
+nothing else of it) so that a deep model can be compared layer by layer without
+the formats' own rounding noise hiding everything else: ``dims["fp8"]`` (e4m3
+projections) and ``SeqState.bf16_points`` (activations stored as bfloat16 at the
+points a "bf16 in, fp32 accumulate" pipeline stores them).  Both are pinned to
+the formats' definitions by brute force.
 """
 from __future__ import annotations
 
@@ -60,6 +68,7 @@ class SeqState:
     wex: list = field(default_factory=list)   # external window of the current phase
     eos_id: int = None                    # adaptive termination (Section 4.2), None = off
     refresh_mode: int = 0                 # 0: the paper's refresh (Section 4.3); 1: window-only variant (see oracle_plan)
+    bf16_points: bool = False             # activations rounded to bfloat16 where a bf16 pipeline stores them (see oracle_layer)
 
     def __post_init__(self):
         self.ids = np.array(self.ids, dtype=np.int64)
@@ -243,6 +252,32 @@ def _proj(dims: dict, x: np.ndarray, w: np.ndarray) -> np.ndarray:
     return fp8_matmul(x, w) if dims.get("fp8") else x @ w.T
 
 
+# ---------------------------------------------------------------------------
+# bfloat16 storage points (a precision mode, not part of the method)
+# ---------------------------------------------------------------------------
+# bfloat16: 1 sign bit, 8 exponent bits, 7 mantissa bits = the upper half of a float32.  A
+# "bf16 in, fp32 accumulate" pipeline holds a value in float32 and stores it as the nearest
+# bfloat16 (ties to even).  With dims["bf16_points"] the oracle rounds the same stored values
+# in the same way: the normalised rows that feed q/k/v and the feed-forward projections,
+# q and k after the rotation, v (i.e. the K/V cache), the attention output that feeds the
+# output projection, the SwiGLU product that feeds the down projection, and the normalised
+# active rows that feed the LM head.  Everything else stays float64: products, sums, softmax,
+# the residual stream, the logits.
+
+
+def bf16_round(x: np.ndarray) -> np.ndarray:
+    """Nearest bfloat16 (ties to even) of the float32 rounding of each value, as float64.
+    Written out on the bit pattern: add half of the dropped 16 bits' range minus one, plus the
+    lowest kept bit (which breaks ties towards an even mantissa), then clear the dropped bits."""
+    b = np.ascontiguousarray(np.asarray(x, dtype=np.float64).astype(np.float32)).view(np.uint32).astype(np.uint64)
+    r = ((b + np.uint64(0x7FFF) + ((b >> np.uint64(16)) & np.uint64(1))) & np.uint64(0xFFFF0000)).astype(np.uint32)
+    return r.view(np.float32).astype(np.float64).reshape(np.shape(x))
+
+
+def _store(dims: dict, x: np.ndarray) -> np.ndarray:
+    return bf16_round(x) if dims.get("bf16_points") else x
+
+
 def oracle_layer(dims: dict, lw: dict, x: np.ndarray, pos, vis, cache: KVCache, l: int,
                  want_probs: bool = False) -> dict:
     """One transformer block over the computed rows ``pos`` (ascending
@@ -253,20 +288,20 @@ def oracle_layer(dims: dict, lw: dict, x: np.ndarray, pos, vis, cache: KVCache, 
     Hq, Hkv, dh = dims["Hq"], dims["Hkv"], dims["dh"]
     n = x.shape[0]
     pos = np.asarray(pos, dtype=np.int64)
-    a = rmsnorm(x, lw["attn_norm"], dims["eps"])
+    a = _store(dims, rmsnorm(x, lw["attn_norm"], dims["eps"]))
     q = _proj(dims, a, lw["wq"]).reshape(n, Hq, dh)
     k = _proj(dims, a, lw["wk"]).reshape(n, Hkv, dh)
     v = _proj(dims, a, lw["wv"]).reshape(n, Hkv, dh)
-    q = rope(q, pos, dims["theta"])
-    k = rope(k, pos, dims["theta"])
+    q = _store(dims, rope(q, pos, dims["theta"]))
+    k = _store(dims, rope(k, pos, dims["theta"]))
     cache.K[l, pos] = k
-    cache.V[l, pos] = v
+    cache.V[l, pos] = _store(dims, v)
     vis = np.asarray(vis, dtype=np.int64)
     o, probs = attention_rows(q, cache.K[l, vis], cache.V[l, vis], Hq // Hkv)
-    o = o.reshape(n, Hq * dh)
+    o = _store(dims, o.reshape(n, Hq * dh))
     h = x + o @ lw["wo"].T
-    f = rmsnorm(h, lw["ffn_norm"], dims["eps"])
-    y = h + _proj(dims, silu(_proj(dims, f, lw["w_gate"])) * _proj(dims, f, lw["w_up"]), lw["w_down"])
+    f = _store(dims, rmsnorm(h, lw["ffn_norm"], dims["eps"]))
+    y = h + _proj(dims, _store(dims, silu(_proj(dims, f, lw["w_gate"])) * _proj(dims, f, lw["w_up"])), lw["w_down"])
     res = dict(out=y, attn=o)
     if want_probs:
         res["probs"] = probs
@@ -305,6 +340,11 @@ def oracle_unmask(logits: np.ndarray, positions, k: int) -> dict:
 # one step
 # ---------------------------------------------------------------------------
 
+def _seq_dims(dims: dict, st: SeqState) -> dict:
+    """The model dims with this sequence's precision mode switched on."""
+    return dict(dims, bf16_points=True) if st.bf16_points else dims
+
+
 def oracle_step(model, states, caches, A: int, B: int, R: int, T: int, k: int,
                 forced=None, want_probs: bool = False, commit: bool = True) -> list:
     """One windowed denoising step for a batch of independent sequences.
@@ -332,7 +372,7 @@ def oracle_step(model, states, caches, A: int, B: int, R: int, T: int, k: int,
         for i, (pl, cache) in enumerate(zip(plans, caches)):
             if pl["done"]:
                 continue
-            r = oracle_layer(dims, lw, xs[i], pl["rows"], pl["vis"], cache, l, want_probs)
+            r = oracle_layer(_seq_dims(dims, states[i]), lw, xs[i], pl["rows"], pl["vis"], cache, l, want_probs)
             xs[i] = r["out"]
             outs[i]["layer_out"].append(r["out"])
             outs[i]["attn_out"].append(r["attn"])
@@ -347,7 +387,8 @@ def oracle_step(model, states, caches, A: int, B: int, R: int, T: int, k: int,
             w_lm = model.lm_head()
         rows = pl["rows"]
         sel = [rows.index(p) for p in pl["active"]]
-        logits = _proj(dims, rmsnorm(xs[i][sel], g_final, dims["eps"]), w_lm)
+        sd = _seq_dims(dims, st)
+        logits = _proj(sd, _store(sd, rmsnorm(xs[i][sel], g_final, dims["eps"])), w_lm)
         um = oracle_unmask(logits, pl["active"], k)
         outs[i].update(logits=logits, unmask=um)
         if forced is not None and forced[i] is not None:

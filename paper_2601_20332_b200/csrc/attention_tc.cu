@@ -129,7 +129,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     const int kvh = h / (p.Hq / p.Hkv);
 
     pdl_launch_dependents();
-    // the index lists were written before the first kernel of the step: safe to read right away
+    // The index lists are complete before this kernel can start: a host-planned step copies them in
+    // front of its first kernel, and a device-planned step's embedding kernel (the planner kernel's
+    // successor) triggers its dependents only after its own wait, i.e. after the planner has finished.
     const int n_vis = p.seq_nvis[b];
     const int n_kt_all = (n_vis + kTile - 1) / kTile;
     const int n_parts = (n_kt_all + p.tiles_per_split - 1) / p.tiles_per_split;

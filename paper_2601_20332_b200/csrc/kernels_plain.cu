@@ -251,8 +251,13 @@ __global__ void embed_kernel(const T* __restrict__ embed, const int32_t* __restr
                              const int32_t* __restrict__ row_seq, const int32_t* __restrict__ row_pos,
                              float* __restrict__ x, float2* __restrict__ rope_tab, int d, int S, int vocab, int dh,
                              double log2_theta, int32_t* status) {
-    pdl_launch_dependents();
+    // Wait first, trigger second: programmatic launch orders a kernel only against its immediate
+    // predecessor's trigger, and every later kernel of the step triggers at its start.  With the
+    // trigger here after the wait, no later kernel starts before the planner kernel (this kernel's
+    // predecessor when the device plans the step) has finished, so they may all read the step's
+    // index lists before their own wait.
     pdl_wait();
+    pdl_launch_dependents();
     const int r = blockIdx.x;
     const int pos = row_pos[r];
     for (int j = threadIdx.x; j < dh / 2; j += blockDim.x) {
@@ -280,8 +285,8 @@ __global__ void embed_fused_kernel(const __nv_bfloat16* __restrict__ embed, cons
                                    float* __restrict__ x, __nv_bfloat16* __restrict__ xg, const float* __restrict__ gain,
                                    float* __restrict__ sumsq, float2* __restrict__ rope_tab, int n_rows, int d, int S,
                                    int vocab, int dh, double log2_theta, int32_t* status) {
+    pdl_wait();                   // wait first, trigger second: see embed_kernel
     pdl_launch_dependents();
-    pdl_wait();
     const int r = blockIdx.x;
     const int pos = row_pos[r];
     for (int j = threadIdx.x; j < dh / 2; j += blockDim.x) {

@@ -11,6 +11,8 @@ import contextlib
 import json
 import os
 import socket
+import subprocess
+import sys
 import types
 
 import torch
@@ -67,3 +69,24 @@ def test_reference_arm_line_on_the_tiny_config(capsys):
     assert line["impl"] == "reference" and line["unit"] == bench.UNIT and line["higher_is_better"] is True
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["value"] == line["value"] > 0
     assert line["e2e"] == {"value": line["value"], "unit": bench.UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}
+
+
+def test_gpus_flag_starts_the_ranks_itself():
+    """`python bench.py --gpus 2` run as a plain process (no launcher, no WORLD_SIZE) must itself become two
+    ranks.  `--plumbing-check` keeps the GPU work out: the ranks rendezvous over gloo on 127.0.0.1, take
+    the slowest rank's time, and rank 0 alone prints the line, with n_gpus = 2."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, bench.__file__, "--gpus", "2", "--steps", "4", "--warmup", "3", "--plumbing-check"],
+                         capture_output=True, text=True, env=env, timeout=300)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(l) for l in res.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1                                # rank 0 alone prints
+    assert lines[0]["n_gpus"] == 2 and lines[0]["steps"] == 4
+    assert abs(lines[0]["value"] - 2 * 4 / 0.020) < 1e-9  # work of both ranks over the slower rank's 20 ms
+
+
+def test_gpus_flag_must_agree_with_the_launcher():
+    env = dict(os.environ, WORLD_SIZE="1", RANK="0")
+    res = subprocess.run([sys.executable, bench.__file__, "--gpus", "2", "--plumbing-check"], capture_output=True, text=True,
+                         env=env, timeout=120)
+    assert res.returncode == 2 and "disagrees" in res.stderr

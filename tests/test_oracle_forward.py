@@ -479,3 +479,57 @@ def test_fp8_mode_changes_only_the_quantised_projections():
     assert a["plan"] == b["plan"]
     rel = np.linalg.norm(a["logits"] - b["logits"]) / np.linalg.norm(a["logits"])
     assert 1e-4 < rel < 0.3 and np.isfinite(b["logits"]).all()
+
+
+# ---------------------------------------------------------------- bfloat16 storage points (precision mode)
+
+def test_bf16_rounding_against_the_format_definition():
+    """bfloat16 = sign, 8 exponent bits, 7 mantissa bits.  Brute force: the nearest value of the form
+    m * 2^(e-7) with an 8-bit integer significand m in [128, 256), ties to the even m; then torch's cast."""
+    import torch
+    rng = np.random.default_rng(9)
+    x = np.concatenate([rng.normal(0, 1, 3000), rng.normal(0, 1e-3, 1000), rng.uniform(-300, 300, 1000)]).astype(np.float32)
+    got = wo.bf16_round(x)
+    for v, g in zip(x.astype(np.float64), got):
+        e = math.floor(math.log2(abs(v)))
+        ulp = 2.0 ** (e - 7)
+        lo = math.floor(abs(v) / ulp)
+        cands = [lo * ulp, (lo + 1) * ulp]
+        d = [abs(abs(v) - c) for c in cands]
+        want = cands[0] if d[0] < d[1] else cands[1] if d[1] < d[0] else (cands[0] if lo % 2 == 0 else cands[1])
+        assert g == math.copysign(want, v)
+    np.testing.assert_array_equal(got, torch.from_numpy(x).to(torch.bfloat16).to(torch.float64).numpy())
+    # representable values stay; exact midpoints go to the even mantissa: 1 + 2^-8 is halfway between 1 and 1 + 2^-7
+    np.testing.assert_array_equal(wo.bf16_round(np.array([1.0, 1.5, -0.0078125, 0.0])), [1.0, 1.5, -0.0078125, 0.0])
+    np.testing.assert_array_equal(wo.bf16_round(np.array([1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, -(1.0 + 2.0 ** -8)])),
+                                  [1.0, 1.0 + 2.0 ** -6, -1.0])
+    assert wo.bf16_round(np.zeros((2, 3))).shape == (2, 3)
+
+
+def test_bf16_points_mode_rounds_the_stored_activations_and_nothing_else():
+    cfg = small_cfg(G=12)
+    model = make(cfg)
+    states = fresh_states(cfg)
+    rounded = [wo.SeqState(ids=states[0].ids.copy(), decoded=states[0].decoded.copy(), bf16_points=True)]
+    c0, c1 = caches_for(cfg, model, 1), caches_for(cfg, model, 1)
+    a = wo.oracle_step(model, states, c0, cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])[0]
+    b = wo.oracle_step(model, rounded, c1, cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])[0]
+    assert a["plan"] == b["plan"]                                       # the planner is untouched
+    vis = a["plan"]["vis"]
+    # what the mode stores is on the bfloat16 grid: the cache and the attention output
+    for t in (c1[0].K[:, vis], c1[0].V[:, vis], b["attn_out"][0]):
+        np.testing.assert_array_equal(wo.bf16_round(t), t)
+    assert not np.array_equal(wo.bf16_round(c0[0].K[:, vis]), c0[0].K[:, vis])
+    # layer 0's cache is the rounding of the unrounded one up to the rounding of the normalised input
+    rel = np.linalg.norm(c1[0].K[0][vis] - c0[0].K[0][vis]) / np.linalg.norm(c0[0].K[0][vis])
+    assert 5e-4 < rel < 6e-3
+    # the residual stream and the logits are not rounded, and stay close to the float64 run
+    assert not np.array_equal(wo.bf16_round(b["layer_out"][-1]), b["layer_out"][-1])
+    rel = np.linalg.norm(b["logits"] - a["logits"]) / np.linalg.norm(a["logits"])
+    assert 1e-4 < rel < 5e-2
+    # a batch may mix the two modes: each sequence keeps its own
+    mixed = wo.oracle_step(model, fresh_states(cfg) + [wo.SeqState(ids=states[0].ids.copy() * 0 + fresh_states(cfg)[0].ids,
+                                                                   decoded=fresh_states(cfg)[0].decoded, bf16_points=True)],
+                           caches_for(cfg, model, 2), cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])
+    np.testing.assert_array_equal(mixed[0]["logits"], a["logits"])
+    np.testing.assert_array_equal(mixed[1]["logits"], b["logits"])

@@ -87,6 +87,7 @@ class Parity:
             forced.append((res["positions"][b, :nb].tolist(), res["token_ids"][b, :nb].tolist()))
         outs = wo.oracle_step(self.model, self.ost, self.oc, A, B, R, T, k, forced=forced)
         worst = dict(layer=0.0, attn=0.0, logits=0.0, ambiguous=0)
+        curve = dict(layer=[0.0] * L, attn=[0.0] * L)      # worst error of each block over the followed sequences
         for j, b in enumerate(self.oracle_seqs):
             o, p = outs[j], plans[b]
             assert p["done"] == o["done"]
@@ -106,6 +107,8 @@ class Parity:
                 e_a = max_rel(att[l, r0:r1], o["attn_out"][l])
                 worst["layer"] = max(worst["layer"], e_l)
                 worst["attn"] = max(worst["attn"], e_a)
+                curve["layer"][l] = max(curve["layer"][l], e_l)
+                curve["attn"][l] = max(curve["attn"][l], e_a)
                 if check:
                     assert np.isfinite(lay[l, r0:r1]).all()
                     assert e_l <= tol_layer, f"seq {b} layer {l}: rel-RMS {e_l:.3e}"
@@ -134,8 +137,8 @@ class Parity:
                 assert got_pos == um["positions"], (got_pos, um["positions"])
             np.testing.assert_allclose(res["confidence"][b, :nb], [um["conf"][op["active"].index(q)] for q in got_pos],
                                        rtol=1e-4)
-        self.log.append(dict(info=info, worst=worst))
-        return dict(info=info, res=res, worst=worst, plans=plans, outs=outs)
+        self.log.append(dict(info=info, worst=worst, curve=curve))
+        return dict(info=info, res=res, worst=worst, curve=curve, plans=plans, outs=outs)
 
     def check_state_mirror(self):
         """The library's host mirror equals the oracle's state."""
