@@ -62,7 +62,8 @@ enum {
     WD_ERR_BOUNDS = -10,              /* a device-side index check failed      */
     WD_ERR_NOT_PENDING = -11,         /* wd_step_sync without wd_step before   */
     WD_ERR_MISALIGNED = -12,
-    WD_ERR_INTERNAL = -13             /* host and device planners disagree (a bug)   */
+    WD_ERR_INTERNAL = -13,            /* host and device planners disagree (a bug)   */
+    WD_ERR_POISONED = -14             /* an earlier device-side error left this state inconsistent */
 };
 
 enum { WD_F32 = 0, WD_BF16 = 1 };     /* element type of weights, activations, K/V cache */
@@ -183,12 +184,22 @@ WD_API size_t wd_workspace_bytes(const wd_model_dims* dims);
 WD_API size_t wd_state_bytes(const wd_model_dims* dims, int32_t batch, int32_t seq_len);
 /* Library version: major*10000 + minor*100 + patch. */
 WD_API int32_t wd_version(void);
+/* Bytes of that state memory taken by the K/V cache of every layer (Section 4.3: the cache the
+ * refresh step writes and the normal steps read): K rows plus the transposed V rows, whose
+ * positions are padded to a multiple of 8.  0 if invalid. */
+WD_API size_t wd_kv_bytes(const wd_model_dims* dims, int32_t batch, int32_t seq_len);
 /* Static text for a status code. */
 WD_API const char* wd_status_string(wd_status s);
+/* Text of the last CUDA runtime / driver error a call of this thread ran into ("" if none), with
+ * the source line that saw it: the detail behind a WD_ERR_CUDA return.  Valid until the thread's
+ * next failing call. */
+WD_API const char* wd_last_error(void);
 
 /* ---- context ------------------------------------------------------------ */
 
-/* Build a context on the current CUDA device.  Validates dims (head_dim even,
+/* Build a context on the current CUDA device for the model whose forward pass the step runs
+ * (Section 3.1: a bidirectional transformer; Section 4.1: the pretrained model is used without
+ * architectural change, so `weights` are its matrices as they are).  Validates dims (head_dim even,
  * n_q_heads a multiple of n_kv_heads, bf16 needs d_model, d_ffn and
  * n_q_heads*head_dim to be multiples of 64, ...), borrows weights and
  * workspace, creates the TMA descriptors of the weights.
@@ -221,16 +232,22 @@ WD_API wd_status wd_profile_read(const wd_ctx* ctx, double* gemm_ms, double* gem
 /* token_ids: host [batch, seq_len].  decoded: host [batch, seq_len] of 0/1, or
  * NULL meaning decoded = (id != mask_id).  Decoded-ness is tracked by these
  * flags afterwards, never by comparing ids with mask_id.  state_mem is device
- * memory of wd_state_bytes(); its K/V cache part is not initialised (the first
- * step is a refresh and writes every row it reads).  Copies ids to the device
- * on the legacy default stream and waits for it.
+ * memory of wd_state_bytes(); its K/V cache part is set to zero here (the first
+ * step is a refresh and writes every row whose value it uses, but the key tiles
+ * of the tensor-core attention also cover far-field rows, masked, which must hold
+ * finite numbers).  Copies ids to the device on the legacy default stream and
+ * waits for it.
  * Errors: WD_ERR_NULL, WD_ERR_BAD_PARAM (batch/seq_len out of range),
  * WD_ERR_WORKSPACE_TOO_SMALL, WD_ERR_CUDA. */
 WD_API wd_status wd_state_create(wd_ctx* ctx, int32_t batch, int32_t seq_len,
                           const int32_t* token_ids, const uint8_t* decoded,
                           void* state_mem /*device*/, size_t state_mem_bytes, wd_state** out);
 /* Start over with new ids/flags (same batch and seq_len): step counter 0, next
- * step is a refresh.  The host->device copy of the ids is enqueued on `stream`. */
+ * step is a refresh.  The host->device copies of the ids and flags are enqueued on
+ * `stream` from pinned staging buffers inside the state: the steps that follow must
+ * be enqueued on the same stream (or be ordered after it by the caller), and a
+ * second reset first waits until the previous reset's copies have left the staging
+ * buffers.  Also clears WD_ERR_POISONED. */
 WD_API wd_status wd_state_reset(wd_state* st, const int32_t* token_ids, const uint8_t* decoded,
                          void* stream /*cudaStream_t*/);
 WD_API wd_status wd_state_destroy(wd_state* st);
@@ -240,6 +257,32 @@ WD_API wd_status wd_state_destroy(wd_state* st);
 WD_API wd_status wd_state_read(const wd_state* st, int32_t seq, int32_t* token_ids, uint8_t* decoded,
                         int32_t* dec_step, int32_t* step_index, int32_t* steps_since_refresh);
 WD_API wd_status wd_debug_taps_set(wd_state* st, const wd_debug_taps* taps /*NULL = off*/);
+
+/* Checkpoint / resume of the sequence state x^(t) of Section 3.1 with the phase bookkeeping of
+ * Section 4.3 (token ids, decoded flags, decode steps, step index, steps since the last refresh,
+ * the external window of the running phase, end-of-sequence id, refresh mode), as one flat host
+ * blob of wd_state_export_bytes().  The K/V cache is not part of the blob: it lives in the
+ * caller's own state memory (wd_kv_bytes() of it), which the caller may copy and restore itself.
+ *   wd_state_import(st, blob, bytes, cache_valid, stream): `st` must have the blob's batch and
+ *   seq_len.  cache_valid != 0: the caller has restored the state memory the blob was taken with,
+ *   and the trajectory continues exactly where it stopped.  cache_valid == 0: the cache is taken
+ *   as lost, the stored external window is dropped, and the next step is a refresh step, which
+ *   rewrites every cache row it reads (Section 4.3); the phase clock restarts there (only for
+ *   states in WD_REFRESH_FULL mode: the window-only variant's refresh does not rebuild the cache).  A resumed
+ *   state is planned on the host (one wd_step_sync per wd_step).  Copies are enqueued on `stream`
+ *   and waited for.  Clears WD_ERR_POISONED.
+ * Errors: WD_ERR_NULL, WD_ERR_PENDING, WD_ERR_CAPACITY (export buffer too short), WD_ERR_BAD_PARAM
+ * (foreign, damaged or mismatching blob: nothing is changed), WD_ERR_CUDA. */
+WD_API size_t wd_state_export_bytes(const wd_state* st);
+WD_API wd_status wd_state_export(const wd_state* st, void* blob /*host*/, size_t bytes);
+WD_API wd_status wd_state_import(wd_state* st, const void* blob /*host*/, size_t bytes, int32_t cache_valid,
+                          void* stream /*cudaStream_t*/);
+
+/* Test hook for the device-side index checks: overwrites ONE entry of the DEVICE copy of the
+ * token ids with `id`, unchecked, leaving the host mirror alone.  An id outside [0, vocab) makes
+ * the next step's embedding kernel skip that row's gather and record WD_ERR_BOUNDS, which
+ * wd_step_sync then reports (no fault: the bad index is never dereferenced). */
+WD_API wd_status wd_debug_poke_id(wd_state* st, int32_t seq, int32_t pos, int32_t id, void* stream /*cudaStream_t*/);
 /* Adaptive termination (Section 4.2, "Adaptive termination"): once a step has unmasked the
  * token `eos_id` at some position, undecoded positions after the first such position are never
  * activated again (they stay far-field and are ignored) and a sequence is done when nothing
@@ -319,10 +362,16 @@ WD_API wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int32_t 
                   void* stream /*cudaStream_t*/, wd_step_info* info);
 
 /* Wait for every enqueued step, read the results and the device status word,
- * apply the update sets to the host mirror of the state in order and advance the
- * phase counters.  `out` (host, may be NULL) receives the result of the NEWEST
- * step.  Returns WD_OK, WD_ERR_NOT_PENDING, WD_ERR_DEVICE_TIMEOUT, WD_ERR_BOUNDS,
- * WD_ERR_INTERNAL, WD_ERR_CUDA. */
+ * apply the update sets U^(t) (Section 3.1: the few positions a step changes) to the
+ * host mirror of the state in order and advance the phase counters (Section 4.3:
+ * steps since the refresh that opened the phase).  `out` (host, may be NULL)
+ * receives the result of the NEWEST step.  Returns WD_OK, WD_ERR_NOT_PENDING,
+ * WD_ERR_DEVICE_TIMEOUT, WD_ERR_BOUNDS, WD_ERR_INTERNAL, WD_ERR_CUDA.
+ * After WD_ERR_DEVICE_TIMEOUT or WD_ERR_BOUNDS the steps up to the failing one are
+ * committed, the rest of the queue is dropped, and, because queued steps behind the
+ * failing one have already run on the device, the state is marked inconsistent:
+ * wd_step, wd_plan and wd_generate return WD_ERR_POISONED until wd_state_reset or
+ * wd_state_import.  The context and other states stay usable. */
 WD_API wd_status wd_step_sync(wd_state* st, wd_step_out* out);
 
 /* The same, returning every enqueued step's result: outs[0] is the oldest.
@@ -376,13 +425,15 @@ WD_API size_t wd_op_gemm_fp8_scratch_bytes(int32_t rows, int32_t n_out, int32_t 
  * memory is already fully committed.  The split-K partial sums go to a fixed
  * 16 MiB array that is part of the library image (wd_op_gemm_noalloc_max_floats()
  * floats; each GPU that loads the library keeps it until the process exits).  This
- * call allocates nothing, on the host or on the device.
+ * call allocates nothing, on the host or on the device (the operands' TMA descriptors
+ * are built on the stack).
  *   - Limit: rows * n_out must not exceed wd_op_gemm_noalloc_max_floats(), otherwise
  *     WD_ERR_CAPACITY and nothing is launched.  Fewer K slices are used when the
  *     array cannot hold more, so large shapes run slower than with wd_op_gemm.
- *   - The first call on each device looks up the array's device address (with that
- *     device current) and remembers it; make that first call before any stream
- *     capture begins.
+ *   - The first call on each device does the set-up for that device, with that device
+ *     current: it looks up the device addresses of the array and of the operations'
+ *     status word and sets the kernels' shared-memory limit, and remembers all three
+ *     per device.  Make that first call before any stream capture begins.
  *   - All calls share the one array and it keeps whatever the last call left in it.
  *     Nothing needs clearing (every partial sum that is read is written first by
  *     the same call), but two calls that overlap on the GPU, e.g. on different
@@ -407,6 +458,24 @@ WD_API wd_status wd_op_attention(int32_t dtype, const void* q, const void* kcach
                           int32_t n_q_heads, int32_t n_kv_heads, int32_t head_dim, int32_t seq_len,
                           void* stream);
 
+/* The same attention (Section 3.1, no causal mask) through the tensor-core kernel the step uses when
+ * the visible set of a sequence is a range: n_rows query rows of one sequence over the cached
+ * positions [0, n_vis), bf16, head_dim 128.  q, out: [n_rows, n_q_heads, 128] bf16; kcache:
+ * [n_kv_heads, seq_len, 128]; vcache_t TRANSPOSED: [n_kv_heads, 128, seq_len], seq_len a multiple
+ * of 8; rows of the caches at or beyond n_vis are never used as values (they may hold anything,
+ * NaN included).  max_vis >= n_vis sizes the split of the keys over the CTAs of a thread-block
+ * cluster exactly as the step does for its longest sequence (max_vis = n_vis: this sequence is the
+ * longest; larger: some CTAs of a cluster get no key tile, as for the shorter sequences of a
+ * batch).  scratch: device, 4-byte aligned, wd_op_attention_tc_scratch_bytes(n_rows) (the query-tile
+ * lists, written by a small kernel on `stream`).  All pointers device, 16-byte aligned.
+ * Errors: WD_ERR_NULL, WD_ERR_BAD_PARAM, WD_ERR_MISALIGNED, WD_ERR_WORKSPACE_TOO_SMALL, WD_ERR_CUDA;
+ * a device-side time-out is reported by wd_op_status(). */
+WD_API wd_status wd_op_attention_tc(const void* q, const void* kcache, const void* vcache_t, void* out,
+                             int32_t n_rows, int32_t n_vis, int32_t max_vis, int32_t n_q_heads,
+                             int32_t n_kv_heads, int32_t seq_len, void* scratch, size_t scratch_bytes,
+                             void* stream /*cudaStream_t*/);
+WD_API size_t wd_op_attention_tc_scratch_bytes(int32_t n_rows);
+
 /* The unmask rule on given logits (device float [n, vocab]) of one sequence:
  * token = lowest index of the maximal logit, confidence = its softmax
  * probability; the min(k, n) rows of highest confidence are returned (equal
@@ -420,6 +489,23 @@ WD_API wd_status wd_op_unmask(const float* logits, const int32_t* positions, int
                        void* scratch, size_t scratch_bytes, void* stream);
 /* Device scratch the unmask operation needs (per-chunk partial statistics), 8-byte aligned. */
 WD_API size_t wd_op_unmask_scratch_bytes(int32_t n, int32_t vocab);
+
+/* Logits and the unmask rule in one pass, as the step does it for its active rows (Section 4.1:
+ * logits only for the active tokens, decoding decided by prediction confidence): logits[n, vocab]
+ * (float) = x[n, k_in] * w[vocab, k_in]^T on the tensor cores (x = the normalised active rows, w =
+ * the LM head, both bf16, k_in a multiple of 8), whose epilogue reduces every CTA's logits to
+ * per-row (maximum, lowest index of the maximum, sum of exp(logit - maximum) in double); a second
+ * kernel merges the CTAs' entries of a row in a fixed order and ranks the rows.  Same outputs and
+ * tie rules as wd_op_unmask; `logits` (device, required) also receives the logits themselves, so
+ * that a test can hand the very same numbers to another implementation of the rule.  n <= 1024.
+ * scratch: device, 8-byte aligned, wd_op_lm_unmask_scratch_bytes(n, vocab).
+ * Errors: WD_ERR_NULL, WD_ERR_BAD_PARAM, WD_ERR_CAPACITY (n), WD_ERR_MISALIGNED,
+ * WD_ERR_WORKSPACE_TOO_SMALL, WD_ERR_CUDA; device-side time-outs through wd_op_status(). */
+WD_API wd_status wd_op_lm_unmask(const void* x, const void* w, const int32_t* positions, int32_t n, int32_t vocab,
+                          int32_t k_in, int32_t k, float* logits, int32_t* row_token, double* row_sumexp,
+                          float* row_conf, int32_t* sel_pos, int32_t* sel_token, float* sel_conf, int32_t* n_sel,
+                          void* scratch, size_t scratch_bytes, void* stream /*cudaStream_t*/);
+WD_API size_t wd_op_lm_unmask_scratch_bytes(int32_t n, int32_t vocab);
 
 /* Device status word shared by the single operations: 0, or the first
  * WD_ERR_DEVICE_TIMEOUT / WD_ERR_BOUNDS raised by a kernel since the last

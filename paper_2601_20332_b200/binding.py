@@ -16,6 +16,7 @@ WD_OK, WD_DONE = 0, 1
 WD_ERR_NULL, WD_ERR_INVALID_DIMS, WD_ERR_WORKSPACE_TOO_SMALL, WD_ERR_UNSUPPORTED_ARCH = -1, -2, -3, -4
 WD_ERR_BAD_PARAM, WD_ERR_CAPACITY, WD_ERR_PENDING, WD_ERR_CUDA = -5, -6, -7, -8
 WD_ERR_DEVICE_TIMEOUT, WD_ERR_BOUNDS, WD_ERR_NOT_PENDING, WD_ERR_MISALIGNED, WD_ERR_INTERNAL = -9, -10, -11, -12, -13
+WD_ERR_POISONED = -14
 WD_F32, WD_BF16 = 0, 1
 WD_GEMM_AUTO, WD_GEMM_PLAIN, WD_GEMM_TCGEN05 = 0, 1, 2
 
@@ -61,6 +62,12 @@ SIGNATURES = {
     "wd_workspace_bytes": (C.c_size_t, [C.POINTER(wd_model_dims)]),
     "wd_state_bytes": (C.c_size_t, [C.POINTER(wd_model_dims), i32, i32]),
     "wd_version": (i32, []),
+    "wd_kv_bytes": (C.c_size_t, [C.POINTER(wd_model_dims), i32, i32]),
+    "wd_last_error": (C.c_char_p, []),
+    "wd_state_export_bytes": (C.c_size_t, [vp]),
+    "wd_state_export": (C.c_int, [vp, vp, C.c_size_t]),
+    "wd_state_import": (C.c_int, [vp, vp, C.c_size_t, i32, vp]),
+    "wd_debug_poke_id": (C.c_int, [vp, i32, i32, i32, vp]),
     "wd_status_string": (C.c_char_p, [C.c_int]),
     "wd_create": (C.c_int, [C.POINTER(wd_model_dims), C.POINTER(wd_weights), vp, C.c_size_t, C.POINTER(vp)]),
     "wd_destroy": (C.c_int, [vp]),
@@ -94,6 +101,10 @@ SIGNATURES = {
     "wd_op_attention": (C.c_int, [i32, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]),
     "wd_op_unmask": (C.c_int, [vp, vp, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]),
     "wd_op_unmask_scratch_bytes": (C.c_size_t, [i32, i32]),
+    "wd_op_attention_tc": (C.c_int, [vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp, C.c_size_t, vp]),
+    "wd_op_attention_tc_scratch_bytes": (C.c_size_t, [i32]),
+    "wd_op_lm_unmask": (C.c_int, [vp, vp, vp, i32, i32, i32, i32, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_size_t, vp]),
+    "wd_op_lm_unmask_scratch_bytes": (C.c_size_t, [i32, i32]),
     "wd_op_status": (C.c_int, []),
     "wd_debug_wait_expire": (C.c_int, [vp]),
 }
@@ -276,6 +287,22 @@ class State:
                                   C.byref(t), C.byref(since)), "wd_state_read")
         return dict(ids=ids, decoded=dec.astype(bool), dec_step=ds, t=t.value, since=since.value)
 
+    def export(self) -> bytes:
+        """wd_state_export: the sequence state and phase bookkeeping as one blob (the K/V cache is not in it)."""
+        n = lib().wd_state_export_bytes(self.handle)
+        buf = C.create_string_buffer(n)
+        check(lib().wd_state_export(self.handle, buf, n), "wd_state_export")
+        return buf.raw
+
+    def import_(self, blob: bytes, cache_valid: bool, stream=None):
+        """wd_state_import: resume from a blob; cache_valid=False makes the next step a refresh."""
+        check(lib().wd_state_import(self.handle, blob, len(blob), 1 if cache_valid else 0, _stream_ptr(stream)),
+              "wd_state_import")
+
+    def poke_id(self, seq: int, pos: int, token_id: int, stream=None):
+        """wd_debug_poke_id: overwrite one entry of the device copy of the ids, unchecked (test hook)."""
+        check(lib().wd_debug_poke_id(self.handle, seq, pos, token_id, _stream_ptr(stream)), "wd_debug_poke_id")
+
     def plan(self, seq: int, A: int, B: int, R: int, T: int) -> dict:
         s, bufs = _index_sets(self.S)
         check(lib().wd_plan(self.handle, seq, A, B, R, T, C.byref(s)), "wd_plan")
@@ -404,6 +431,48 @@ def op_attention(q, kcache, vcache, vis, stream=None):
     check(lib().wd_op_attention(_dtype_code(q), _ptr(q), _ptr(kcache), _ptr(vcache), _ptr(vis), _ptr(out), rows,
                                 vis.numel(), Hq, Hkv, dh, S, _stream_ptr(stream)), "wd_op_attention")
     return out
+
+
+def op_attention_tc(q, kcache, vcache_t, n_vis: int, max_vis: int = 0, stream=None):
+    """Tensor-core attention over positions [0, n_vis).  q: [rows, Hq, 128] bf16; kcache: [Hkv, S, 128];
+    vcache_t transposed: [Hkv, 128, S]; max_vis (default n_vis) sizes the key split."""
+    import torch
+    rows, Hq, dh = q.shape
+    Hkv, S, _ = kcache.shape
+    assert dh == 128
+    out = torch.empty_like(q)
+    nb = lib().wd_op_attention_tc_scratch_bytes(rows)
+    scratch = torch.empty(nb, dtype=torch.uint8, device=q.device)
+    check(lib().wd_op_attention_tc(_ptr(q), _ptr(kcache), _ptr(vcache_t), _ptr(out), rows, n_vis, max(max_vis, n_vis), Hq,
+                                   Hkv, S, _ptr(scratch), nb, _stream_ptr(stream)), "wd_op_attention_tc")
+    return out
+
+
+def op_lm_unmask(x, w, positions, k: int, stream=None) -> dict:
+    """x: bf16 [n, K] normalised rows; w: bf16 [V, K] LM head; positions: int32 [n] ascending (all device).
+    Returns the per-row statistics, the selection and the logits the tensor-core GEMM produced."""
+    import torch
+    n, K = x.shape
+    V = w.shape[0]
+    dev = x.device
+    kk = max(k, 1)
+    logits = torch.empty(n, V, dtype=torch.float32, device=dev)
+    row_token = torch.empty(n, dtype=torch.int32, device=dev)
+    row_sumexp = torch.empty(n, dtype=torch.float64, device=dev)
+    row_conf = torch.empty(n, dtype=torch.float32, device=dev)
+    sel_pos = torch.full((kk,), -1, dtype=torch.int32, device=dev)
+    sel_tok = torch.full((kk,), -1, dtype=torch.int32, device=dev)
+    sel_conf = torch.zeros(kk, dtype=torch.float32, device=dev)
+    n_sel = torch.zeros(1, dtype=torch.int32, device=dev)
+    nb = lib().wd_op_lm_unmask_scratch_bytes(n, V)
+    scratch = torch.empty(nb, dtype=torch.uint8, device=dev)
+    check(lib().wd_op_lm_unmask(_ptr(x), _ptr(w), _ptr(positions), n, V, K, k, _ptr(logits), _ptr(row_token),
+                                _ptr(row_sumexp), _ptr(row_conf), _ptr(sel_pos), _ptr(sel_tok), _ptr(sel_conf), _ptr(n_sel),
+                                _ptr(scratch), nb, _stream_ptr(stream)), "wd_op_lm_unmask")
+    ns = int(n_sel.item())
+    return dict(logits=logits, row_token=row_token.cpu().numpy(), row_sumexp=row_sumexp.cpu().numpy(),
+                row_conf=row_conf.cpu().numpy(), positions=sel_pos.cpu().numpy()[:ns].tolist(),
+                token_ids=sel_tok.cpu().numpy()[:ns].tolist(), confidence=sel_conf.cpu().numpy()[:ns].tolist())
 
 
 def op_unmask(logits, positions, k: int, stream=None) -> dict:

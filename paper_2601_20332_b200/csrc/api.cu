@@ -38,11 +38,14 @@ extern "C" const char* wd_status_string(wd_status s) {
         case WD_ERR_NOT_PENDING: return "no step pending";
         case WD_ERR_MISALIGNED: return "device pointer not 256-byte aligned";
         case WD_ERR_INTERNAL: return "internal inconsistency between the host and device planners";
+        case WD_ERR_POISONED: return "a device-side error left the state inconsistent: reset or import it first";
         default: return "unknown status";
     }
 }
 
-extern "C" int32_t wd_version(void) { return 100; }
+extern "C" const char* wd_last_error(void) { return g_last_cuda_error; }
+
+extern "C" int32_t wd_version(void) { return 200; }
 
 // ---------------------------------------------------------------------------
 // context
@@ -191,6 +194,12 @@ extern "C" size_t wd_state_bytes(const wd_model_dims* d, int32_t batch, int32_t 
     const size_t v = (size_t)d->n_layers * batch * d->n_kv_heads * seq_pad(seq_len) * d->head_dim * wd_elt_size(d->dtype);
     const size_t plan_state = wd_align_up((size_t)batch * seq_len, 256) + 2 * wd_align_up((size_t)batch * seq_len * 4, 256);
     return wd_align_up((size_t)batch * seq_len * 4, 256) + wd_align_up(k, 256) + wd_align_up(v, 256) + plan_state;
+}
+
+extern "C" size_t wd_kv_bytes(const wd_model_dims* d, int32_t batch, int32_t seq_len) {
+    if (!dims_valid(d) || batch < 1 || seq_len < 1 || batch > d->max_batch || seq_len > d->max_seq) return 0;
+    const size_t per = (size_t)d->n_layers * batch * d->n_kv_heads * d->head_dim * wd_elt_size(d->dtype);
+    return per * seq_len + per * seq_pad(seq_len);      // K rows + transposed V rows (positions padded to 8)
 }
 
 extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, void* workspace,
@@ -403,6 +412,9 @@ struct wd_state {
     int32_t* ids_host = nullptr;        // pinned staging for ids
     uint8_t* dec_host = nullptr;        // pinned staging for the decoded flags
     cudaEvent_t done = nullptr;
+    cudaEvent_t staged = nullptr;       // recorded after the copies that read the pinned staging buffers
+    bool staged_recorded = false;
+    bool poisoned = false;              // a queued step failed on the device: device state is ahead of the mirror
     bool pending = false;               // at least one step enqueued and not yet synced
     // Device copy of the planner state, kept up to date by the unmask kernel, and the count-level
     // shadow on the host: with them steps can be enqueued back to back (no host round trip), the
@@ -505,7 +517,8 @@ extern "C" wd_status wd_state_create(wd_ctx* ctx, int32_t batch, int32_t seq_len
         (e = cudaHostAlloc((void**)&st->result_host, ctx->result_ints * 4 * kQueueCap, cudaHostAllocDefault)) != cudaSuccess ||
         (e = cudaHostAlloc((void**)&st->ids_host, (size_t)batch * seq_len * 4, cudaHostAllocDefault)) != cudaSuccess ||
         (e = cudaHostAlloc((void**)&st->dec_host, (size_t)batch * seq_len, cudaHostAllocDefault)) != cudaSuccess ||
-        (e = cudaEventCreateWithFlags(&st->done, cudaEventDisableTiming)) != cudaSuccess) {
+        (e = cudaEventCreateWithFlags(&st->done, cudaEventDisableTiming)) != cudaSuccess ||
+        (e = cudaEventCreateWithFlags(&st->staged, cudaEventDisableTiming)) != cudaSuccess) {
         wd_note_cuda_error(e, __FILE__, __LINE__);
         wd_state_destroy(st);
         return WD_ERR_CUDA;
@@ -535,10 +548,136 @@ extern "C" wd_status wd_state_reset(wd_state* st, const int32_t* token_ids, cons
     if (st->pending) return WD_ERR_PENDING;
     for (size_t i = 0; i < (size_t)st->batch * st->S; ++i)
         if (token_ids[i] < 0 || token_ids[i] >= st->ctx->d.vocab) return WD_ERR_BAD_PARAM;
+    // the pinned staging buffers may still be the source of an earlier reset's copies
+    if (st->staged_recorded) WD_CUDA_TRY(cudaEventSynchronize(st->staged));
     load_host_mirror(st, token_ids, decoded);
+    st->poisoned = false;
     WD_CUDA_TRY(upload_plan_state(st, (cudaStream_t)stream));
     WD_CUDA_TRY(cudaMemcpyAsync(st->ids_dev, st->ids_host, (size_t)st->batch * st->S * 4, cudaMemcpyHostToDevice,
                                 (cudaStream_t)stream));
+    WD_CUDA_TRY(cudaEventRecord(st->staged, (cudaStream_t)stream));
+    st->staged_recorded = true;
+    return WD_OK;
+}
+
+// ---------------------------------------------------------------------------
+// checkpoint / resume of the sequence state (host side; the K/V cache lives in the caller's
+// state memory and is the caller's to copy)
+// ---------------------------------------------------------------------------
+namespace {
+struct BlobHeader { uint32_t magic, version; int32_t batch, S; };
+struct BlobSeq { int32_t t, since, phase_start, eos_id, refresh_mode, n_wex; };
+constexpr uint32_t kBlobMagic = 0x57445354u;     // "WDST"
+}
+
+extern "C" size_t wd_state_export_bytes(const wd_state* st) {
+    if (!st) return 0;
+    size_t n = sizeof(BlobHeader);
+    for (const WdSeq& s : st->seqs)
+        n += sizeof(BlobSeq) + (size_t)st->S * 8 + wd_align_up((size_t)st->S, 4) + s.wex.size() * 4;
+    return n;
+}
+
+extern "C" wd_status wd_state_export(const wd_state* st, void* buf, size_t bytes) {
+    if (!st || !buf) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    if (st->poisoned) return WD_ERR_BAD_PARAM;
+    if (bytes < wd_state_export_bytes(st)) return WD_ERR_CAPACITY;
+    char* p = (char*)buf;
+    BlobHeader h = {kBlobMagic, 1u, st->batch, st->S};
+    memcpy(p, &h, sizeof(h)); p += sizeof(h);
+    for (const WdSeq& s : st->seqs) {
+        BlobSeq bs = {s.t, s.since, s.phase_start, s.eos_id, s.refresh_mode, (int32_t)s.wex.size()};
+        memcpy(p, &bs, sizeof(bs)); p += sizeof(bs);
+        memcpy(p, s.ids.data(), (size_t)st->S * 4); p += (size_t)st->S * 4;
+        memcpy(p, s.dec_step.data(), (size_t)st->S * 4); p += (size_t)st->S * 4;
+        memset(p, 0, wd_align_up((size_t)st->S, 4));
+        memcpy(p, s.decoded.data(), (size_t)st->S); p += wd_align_up((size_t)st->S, 4);
+        if (!s.wex.empty()) memcpy(p, s.wex.data(), s.wex.size() * 4);
+        p += s.wex.size() * 4;
+    }
+    return WD_OK;
+}
+
+extern "C" wd_status wd_state_import(wd_state* st, const void* buf, size_t bytes, int32_t cache_valid, void* stream_) {
+    if (!st || !buf) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    const char* p = (const char*)buf;
+    const char* end = p + bytes;
+    BlobHeader h;
+    if (bytes < sizeof(h)) return WD_ERR_BAD_PARAM;
+    memcpy(&h, p, sizeof(h)); p += sizeof(h);
+    if (h.magic != kBlobMagic || h.version != 1u || h.batch != st->batch || h.S != st->S) return WD_ERR_BAD_PARAM;
+    const int S = st->S, vocab = st->ctx->d.vocab;
+    // parse and validate everything before anything is changed
+    std::vector<WdSeq> seqs((size_t)st->batch);
+    for (WdSeq& s : seqs) {
+        BlobSeq bs;
+        if ((size_t)(end - p) < sizeof(bs)) return WD_ERR_BAD_PARAM;
+        memcpy(&bs, p, sizeof(bs)); p += sizeof(bs);
+        const size_t need = (size_t)S * 8 + wd_align_up((size_t)S, 4);
+        if (bs.n_wex < 0 || bs.n_wex > S || bs.t < 0 || bs.since < 0 || bs.phase_start < 0 || bs.phase_start > bs.t ||
+            bs.eos_id >= vocab || (bs.refresh_mode != WD_REFRESH_FULL && bs.refresh_mode != WD_REFRESH_WINDOW) ||
+            (size_t)(end - p) < need + (size_t)bs.n_wex * 4)
+            return WD_ERR_BAD_PARAM;
+        s.t = bs.t; s.since = bs.since; s.phase_start = bs.phase_start;
+        s.eos_id = bs.eos_id < 0 ? -1 : bs.eos_id; s.refresh_mode = bs.refresh_mode;
+        s.ids.resize(S); s.dec_step.resize(S); s.decoded.resize(S); s.wex.resize((size_t)bs.n_wex);
+        memcpy(s.ids.data(), p, (size_t)S * 4); p += (size_t)S * 4;
+        memcpy(s.dec_step.data(), p, (size_t)S * 4); p += (size_t)S * 4;
+        memcpy(s.decoded.data(), p, (size_t)S); p += wd_align_up((size_t)S, 4);
+        if (bs.n_wex) memcpy(s.wex.data(), p, (size_t)bs.n_wex * 4);
+        p += (size_t)bs.n_wex * 4;
+        for (int i = 0; i < S; ++i)
+            if (s.ids[i] < 0 || s.ids[i] >= vocab || s.decoded[i] > 1) return WD_ERR_BAD_PARAM;
+        for (size_t i = 0; i < s.wex.size(); ++i)
+            if (s.wex[i] < 0 || s.wex[i] >= S || (i > 0 && s.wex[i] <= s.wex[i - 1])) return WD_ERR_BAD_PARAM;
+    }
+    // a lost cache is rebuilt by a refresh that computes every visible position: the paper's refresh
+    if (!cache_valid)
+        for (const WdSeq& s : seqs)
+            if (s.refresh_mode != WD_REFRESH_FULL) return WD_ERR_BAD_PARAM;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    if (st->staged_recorded) WD_CUDA_TRY(cudaEventSynchronize(st->staged));
+    st->seqs = std::move(seqs);
+    st->counts.assign(st->batch, WdCount());
+    for (int b = 0; b < st->batch; ++b) {
+        WdSeq& s = st->seqs[b];
+        // without its cache a state resumes with a refresh step (which rewrites every row it reads)
+        if (!cache_valid) s.wex.clear();
+        memcpy(st->ids_host + (size_t)b * S, s.ids.data(), (size_t)S * 4);
+        memcpy(st->dec_host + (size_t)b * S, s.decoded.data(), (size_t)S);
+        wd_count_init(st->counts[b], s);
+    }
+    // the device planner only takes states whose generation began from a decoded prefix; a resumed state
+    // cannot prove that, so it is planned on the host (identical index sets, one host round trip per step)
+    st->dev_mode = false;
+    st->queue.clear();
+    st->poisoned = false;
+    const size_t n = (size_t)st->batch * S;
+    WD_CUDA_TRY(cudaMemcpyAsync(st->decoded_dev, st->dec_host, n, cudaMemcpyHostToDevice, stream));
+    WD_CUDA_TRY(cudaMemcpyAsync(st->ids_dev, st->ids_host, n * 4, cudaMemcpyHostToDevice, stream));
+    // decode steps: reuse the pinned plan staging buffer when it is large enough, else copy per sequence from the mirror
+    for (int b = 0; b < st->batch; ++b)
+        WD_CUDA_TRY(cudaMemcpyAsync(st->dec_step_dev + (size_t)b * S, st->seqs[b].dec_step.data(), (size_t)S * 4,
+                                    cudaMemcpyHostToDevice, stream));
+    for (int b = 0; b < st->batch; ++b)
+        if (!st->seqs[b].wex.empty())
+            WD_CUDA_TRY(cudaMemcpyAsync(st->wex_dev + (size_t)b * S, st->seqs[b].wex.data(), st->seqs[b].wex.size() * 4,
+                                        cudaMemcpyHostToDevice, stream));
+    // the mirror's vectors are pageable sources: wait until the copies have read them
+    WD_CUDA_TRY(cudaEventRecord(st->staged, stream));
+    st->staged_recorded = true;
+    WD_CUDA_TRY(cudaEventSynchronize(st->staged));
+    return WD_OK;
+}
+
+extern "C" wd_status wd_debug_poke_id(wd_state* st, int32_t seq, int32_t pos, int32_t id, void* stream) {
+    if (!st) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    if (seq < 0 || seq >= st->batch || pos < 0 || pos >= st->S) return WD_ERR_BAD_PARAM;
+    WD_CUDA_TRY(cudaMemcpyAsync(st->ids_dev + (size_t)seq * st->S + pos, &id, 4, cudaMemcpyHostToDevice, (cudaStream_t)stream));
+    WD_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
     return WD_OK;
 }
 
@@ -550,6 +689,7 @@ extern "C" wd_status wd_state_destroy(wd_state* st) {
     if (st->ids_host) cudaFreeHost(st->ids_host);
     if (st->dec_host) cudaFreeHost(st->dec_host);
     if (st->done) cudaEventDestroy(st->done);
+    if (st->staged) cudaEventDestroy(st->staged);
     delete st;
     return WD_OK;
 }
@@ -613,6 +753,7 @@ extern "C" wd_status wd_plan(const wd_state* st, int32_t seq, int32_t A, int32_t
                              wd_index_sets* out) {
     if (!st || !out) return WD_ERR_NULL;
     if (st->pending) return WD_ERR_PENDING;
+    if (st->poisoned) return WD_ERR_POISONED;
     if (seq < 0 || seq >= st->batch) return WD_ERR_BAD_PARAM;
     WdSeqPlan p;
     wd_status s = wd_plan_seq(st->seqs[seq], A, B, R, T, &p);
@@ -723,6 +864,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
                              wd_step_info* info) {
     if (!st) return WD_ERR_NULL;
     if (A < 1 || B < 0 || R < 1 || T < 0 || k < 0) return WD_ERR_BAD_PARAM;
+    if (st->poisoned) return WD_ERR_POISONED;
     wd_ctx* c = st->ctx;
     const wd_model_dims& d = c->d;
     cudaStream_t stream = (cudaStream_t)stream_;
@@ -899,7 +1041,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
                                      c->plan + o_nvis, &st->map_k, &st->map_vt, c->attn, attn_tap, Hq, Hkv, dh, l, max_vis,
                                      c->sm_count, status, stream);
         wd_launch_attention_plain(d.dtype, c->q, kc, vc, row_seq, vis_idx, vis_off, c->attn, attn_tap, R_, max_vis, Hq,
-                                  Hkv, dh, S, Sp, stream);
+                                  Hkv, dh, S, Sp, batch, status, stream);
         return WD_OK;
     };
     if (fused) {
@@ -982,7 +1124,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         }
         impl_used = go.impl;
         wd_launch_rope_scatter(d.dtype, c->part, go.n_split, go.split_stride, row_seq, row_pos, c->rope_tab, c->q, kc,
-                               vc, R_, Hq, Hkv, dh, S, Sp, stream);
+                               vc, R_, Hq, Hkv, dh, S, Sp, batch, status, stream);
         if ((s = attention(l, kc, vc)) != WD_OK) return s;
         WdTcSeg wo[1] = {{c->wo[l], D, c->tc.get(WD_TC_WO, l)}};
         if ((s = run_gemm(c, c->attn, &c->tc.x_map_attn, wo, 1, R_, hq, c->part, c->part_floats, status, stream, &go)) != WD_OK)
@@ -1140,8 +1282,13 @@ static wd_status drain_queue(wd_state* st, wd_step_out* outs, bool every_step, i
     const bool host_planned = !st->queue.empty() && st->queue.back().host_planned;
     st->queue.clear();
     st->pending = false;
-    if (result != WD_OK)      // shadow and device state may be ahead of the mirror: plan on the host from here on
+    if (result != WD_OK) {
+        // Steps queued behind the failed one have already run on the device, so the device copy of the
+        // state (ids, flags, decode steps, K/V cache) may be ahead of the host mirror, or built on garbage:
+        // the state takes no more steps until wd_state_reset or wd_state_import gives it a consistent start.
         st->dev_mode = false;
+        st->poisoned = true;
+    }
     else if (host_planned)    // the count shadow did not follow host-planned steps: rebuild it from the mirror
         for (int b = 0; b < batch; ++b) wd_count_init(st->counts[b], st->seqs[b]);
     if (n_done) *n_done = done;
@@ -1166,6 +1313,7 @@ extern "C" wd_status wd_generate(wd_state* st, int32_t A, int32_t B, int32_t R, 
                                  void* stream, int32_t* n_steps, int32_t* n_tokens) {
     if (!st) return WD_ERR_NULL;
     if (!st->queue.empty()) return WD_ERR_PENDING;
+    if (st->poisoned) return WD_ERR_POISONED;
     if (n_steps) *n_steps = 0;
     if (n_tokens) *n_tokens = 0;
     int32_t steps = 0;
@@ -1259,9 +1407,90 @@ extern "C" wd_status wd_op_attention(int32_t dtype, const void* q, const void* k
         seq_len < n_vis)
         return WD_ERR_BAD_PARAM;
     if ((size_t)(n_vis + head_dim) * 4 > 200 * 1024) return WD_ERR_CAPACITY;
+    int32_t* op_status = wd_op_status_ptr();
+    if (!op_status) return WD_ERR_CUDA;
     // one sequence: no row->sequence table and no offsets, every row sees vis[0, n_vis)
     wd_launch_attention_plain(dtype, q, kcache, vcache, nullptr, vis, nullptr, out, nullptr, n_rows, n_vis, n_q_heads,
-                              n_kv_heads, head_dim, seq_len, seq_len, (cudaStream_t)stream);
+                              n_kv_heads, head_dim, seq_len, seq_len, 1, op_status, (cudaStream_t)stream);
+    WD_CUDA_TRY(cudaGetLastError());
+    return WD_OK;
+}
+
+extern "C" size_t wd_op_attention_tc_scratch_bytes(int32_t n_rows) {
+    if (n_rows < 1) return 0;
+    return wd_align_up((size_t)(3 * ((n_rows + 127) / 128) + 1) * 4, 256);
+}
+
+extern "C" wd_status wd_op_attention_tc(const void* q, const void* kcache, const void* vcache_t, void* out,
+                                        int32_t n_rows, int32_t n_vis, int32_t max_vis, int32_t n_q_heads,
+                                        int32_t n_kv_heads, int32_t seq_len, void* scratch, size_t scratch_bytes,
+                                        void* stream_) {
+    if (!q || !kcache || !vcache_t || !out || !scratch) return WD_ERR_NULL;
+    if (n_rows < 1 || n_vis < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads || seq_len < n_vis ||
+        max_vis < n_vis || seq_len % 8)
+        return WD_ERR_BAD_PARAM;
+    if (((uintptr_t)q | (uintptr_t)kcache | (uintptr_t)vcache_t | (uintptr_t)out) % 16 || (uintptr_t)scratch % 4)
+        return WD_ERR_MISALIGNED;
+    if (scratch_bytes < wd_op_attention_tc_scratch_bytes(n_rows)) return WD_ERR_WORKSPACE_TOO_SMALL;
+    int32_t* status = wd_op_status_ptr();
+    if (!status) return WD_ERR_CUDA;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int sm = 148, dev = 0;
+    WD_CUDA_TRY(cudaGetDevice(&dev));
+    WD_CUDA_TRY(cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev));
+    CUtensorMap map_k, map_vt;
+    wd_status s = wd_attn_tc_encode_cache(&map_k, &map_vt, kcache, vcache_t, 1, n_kv_heads, seq_len, seq_len, 128);
+    if (s != WD_OK) return s;
+    const int n_tiles = (n_rows + 127) / 128;
+    int32_t* lists = (int32_t*)scratch;
+    wd_launch_fill_qtiles(lists, n_rows, n_vis, stream);
+    WD_CUDA_TRY(cudaGetLastError());
+    return wd_attn_tc_launch(q, n_rows, n_tiles, lists, lists + n_tiles, lists + 2 * n_tiles, lists + 3 * n_tiles, &map_k,
+                             &map_vt, out, nullptr, n_q_heads, n_kv_heads, 128, 0, max_vis, sm, status, stream);
+}
+
+extern "C" size_t wd_op_lm_unmask_scratch_bytes(int32_t n, int32_t vocab) {
+    if (n < 1 || vocab < 1) return 0;
+    // one statistics entry per (row, CTA of the LM-head launch), at most 256 CTAs
+    return (size_t)n * 256 * 16;
+}
+
+extern "C" wd_status wd_op_lm_unmask(const void* x, const void* w, const int32_t* positions, int32_t n, int32_t vocab,
+                                     int32_t k_in, int32_t k, float* logits, int32_t* row_token, double* row_sumexp,
+                                     float* row_conf, int32_t* sel_pos, int32_t* sel_token, float* sel_conf,
+                                     int32_t* n_sel, void* scratch, size_t scratch_bytes, void* stream_) {
+    if (!x || !w || !positions || !logits || !row_token || !row_sumexp || !row_conf || !sel_pos || !sel_token ||
+        !sel_conf || !n_sel || !scratch)
+        return WD_ERR_NULL;
+    if (n < 1 || vocab < 1 || k < 0 || k_in < 8 || k_in % 8) return WD_ERR_BAD_PARAM;
+    if (n > 1024) return WD_ERR_CAPACITY;
+    if (scratch_bytes < wd_op_lm_unmask_scratch_bytes(n, vocab)) return WD_ERR_WORKSPACE_TOO_SMALL;
+    if ((uintptr_t)scratch % 8 || ((uintptr_t)x | (uintptr_t)w) % 16) return WD_ERR_MISALIGNED;
+    int32_t* status = wd_op_status_ptr();
+    if (!status) return WD_ERR_CUDA;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int sm = 148, dev = 0;
+    WD_CUDA_TRY(cudaGetDevice(&dev));
+    WD_CUDA_TRY(cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev));
+    if (sm % 4 || sm > 256) return WD_ERR_UNSUPPORTED_ARCH;     // the launch puts one CTA group on each of up to four token tiles
+    double* ch_sum = (double*)scratch;
+    float* ch_max = (float*)(ch_sum + (size_t)n * 256);
+    int32_t* ch_idx = (int32_t*)(ch_max + (size_t)n * 256);
+    CUtensorMap mw;
+    wd_status s = wd_tc_encode_bf16(&mw, w, vocab, k_in, 128);
+    if (s != WD_OK) return s;
+    WdTcSeg seg = {w, vocab, &mw};
+    WdTcX xm;
+    xm.ptr = x; xm.K = k_in; xm.keep = false;
+    WdTcFuse fl;
+    fl.mode = WD_FUSE_LMSTATS;
+    fl.st_max = ch_max; fl.st_idx = ch_idx; fl.st_sum = ch_sum;
+    fl.write_logits = 1;
+    int ns = 1;
+    s = wd_tc_gemm(&xm, &seg, 1, n, k_in, logits, (size_t)n * vocab, sm, status, stream, &ns, /*single split*/ true, &fl);
+    if (s != WD_OK) return s;
+    wd_launch_select(ch_max, ch_idx, ch_sum, fl.n_chunks, row_token, row_sumexp, positions, nullptr, n, 1, k, nullptr, 0,
+                     n_sel, sel_pos, sel_token, sel_conf, row_conf, nullptr, nullptr, nullptr, stream);
     WD_CUDA_TRY(cudaGetLastError());
     return WD_OK;
 }

@@ -549,8 +549,11 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     // the query descriptor depends only on (buffer, rows, heads): the same for every layer of a step
     static CUtensorMap mq;
     static const void* mq_ptr = nullptr;
-    static int mq_rows = -1, mq_hq = -1;
-    if (mq_ptr != q || mq_rows != n_rows || mq_hq != Hq) {
+    static int mq_rows = -1, mq_hq = -1, mq_dev = -1;
+    int dev = 0;
+    WD_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return WD_ERR_CUDA;
+    if (mq_ptr != q || mq_rows != n_rows || mq_hq != Hq || mq_dev != dev) {
         cuuint64_t dims[2] = {(cuuint64_t)Hq * dh, (cuuint64_t)n_rows};
         cuuint64_t strides[1] = {(cuuint64_t)Hq * dh * 2};
         cuuint32_t box[2] = {64, 128}, estr[2] = {1, 1};
@@ -558,7 +561,7 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return WD_ERR_CUDA;
-        mq_ptr = q; mq_rows = n_rows; mq_hq = Hq;
+        mq_ptr = q; mq_rows = n_rows; mq_hq = Hq; mq_dev = dev;
     }
     AttnParams p;
     memset(&p, 0, sizeof(p));
@@ -577,10 +580,10 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     p.tiles_per_split = (max_kt + want - 1) / want;
     p.max_parts = (max_kt + p.tiles_per_split - 1) / p.tiles_per_split;
     const size_t smem = (1 + 2 * kStages) * (size_t)kOperand + (kBars + 1) * 8 + 16 + 2 * kTile * 4 + 1024;
-    static bool attr_done = false;      // one device per process
-    if (!attr_done) {
+    static bool attr_done[64] = {};     // the attribute is per device
+    if (!attr_done[dev]) {
         WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_done = true;
+        attr_done[dev] = true;
     }
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(n_tiles, Hq, p.max_parts);

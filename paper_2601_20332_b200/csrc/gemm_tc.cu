@@ -1099,6 +1099,13 @@ TcConfig pick_config(int rows, bool allow_wide, bool lm_stats) {
     return c;
 }
 
+// index of the current device, or -1 (beyond the 64 the per-device tables hold, or on an error)
+int current_device() {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return -1;
+    return dev;
+}
+
 // most CTAs that contribute to one output tile when W K-blocks are cut into G equal pieces
 int count_slices(int n_units, int kb_total, long long W, long long G) {
     int n = 1;
@@ -1241,14 +1248,18 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     if (!hit) {
         wd_status s = fp8 ? encode_2d8(&mx, x->ptr, rows, K, tok_rows) : encode_2d(&mx, x->ptr, rows, K, tok_rows);
         if (s != WD_OK) return s;
-        if (x->cache.size() >= 16) x->cache.erase(x->cache.begin());
-        x->cache.push_back({rows, tok_rows, mx});
+        if (x->keep) {
+            if (x->cache.size() >= 16) x->cache.erase(x->cache.begin());
+            x->cache.push_back({rows, tok_rows, mx});
+        }
     }
-    static bool attr_done = false;      // one device per process
-    if (!attr_done) {
+    static bool attr_done[64] = {};     // the attribute belongs to the function on ONE device: set once per device
+    const int dev = current_device();
+    if (dev < 0) return WD_ERR_CUDA;
+    if (!attr_done[dev]) {
         WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_pair_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_pair_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
-        attr_done = true;
+        attr_done[dev] = true;
     }
     const CUtensorMap& m0 = *segs[0].map;
     const CUtensorMap& m1 = *segs[(nseg > 1 || p.dual == 2) ? 1 : 0].map;
@@ -1402,17 +1413,21 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     if (!hit) {
         wd_status s = fp8 ? encode_2d8(&mx, x->ptr, rows, K, cfg.bn) : encode_2d(&mx, x->ptr, rows, K, cfg.bn);
         if (s != WD_OK) return s;
-        if (x->cache.size() >= 16) x->cache.erase(x->cache.begin());
-        x->cache.push_back({rows, cfg.bn, mx});
+        if (x->keep) {
+            if (x->cache.size() >= 16) x->cache.erase(x->cache.begin());
+            x->cache.push_back({rows, cfg.bn, mx});
+        }
     }
-    static bool attr_done = false;      // one device per process
-    if (!attr_done) {
+    static bool attr_done[64] = {};     // set once per device
+    const int dev = current_device();
+    if (dev < 0) return WD_ERR_CUDA;
+    if (!attr_done[dev]) {
         WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         WD_CUDA_TRY(cudaFuncSetAttribute(gemm_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         WD_CUDA_TRY(cudaFuncSetAttribute((gemm_tc_kernel<false, false, true>), cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
         WD_CUDA_TRY(cudaFuncSetAttribute((gemm_tc_kernel<false, true, true>), cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
-        attr_done = true;
+        attr_done[dev] = true;
     }
     const CUtensorMap& m0 = *segs[0].map;
     const CUtensorMap& m1 = *segs[nseg > 1 ? 1 : 0].map;
@@ -1441,6 +1456,10 @@ wd_status wd_tc_encode_fp8(CUtensorMap* m, const void* ptr, int n_rows, int K, i
     return encode_2d8(m, ptr, n_rows, K, box_rows);
 }
 
+wd_status wd_tc_encode_bf16(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_rows) {
+    return encode_2d(m, ptr, n_rows, K, box_rows);
+}
+
 size_t wd_tc_scratch_bytes(int rows, int n_out, int k_in) {
     (void)k_in;
     const size_t r = rows <= WD_TC_SPLITK_MAX_ROWS ? WD_TC_MAX_SPLIT : 1;
@@ -1456,7 +1475,8 @@ wd_status wd_tc_gemm_standalone(const void* x, const void* w, float* y, int rows
     wd_status s = encode_2d(&mw, w, n_out, k_in, kBM);
     if (s != WD_OK) return s;
     WdTcSeg seg = {w, n_out, &mw};
-    WdTcX xm = {x, k_in};
+    WdTcX xm;
+    xm.ptr = x; xm.K = k_in; xm.keep = false;
     int sm = 148, dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);
@@ -1487,7 +1507,7 @@ wd_status wd_tc_gemm_standalone_fp8(const uint8_t* xq, const float* sx, const ui
     if (s != WD_OK) return s;
     WdTcSeg seg = {wq, n_out, &mw};
     WdTcX xm;
-    xm.ptr = xq; xm.K = k_in; xm.fp8 = 1;
+    xm.ptr = xq; xm.K = k_in; xm.fp8 = 1; xm.keep = false;
     WdTcFp8 f8;
     f8.sw[0] = sw; f8.sx = sx;
     int sm = 148, dev = 0;
@@ -1553,7 +1573,8 @@ extern "C" wd_status wd_op_gemm_noalloc(const void* x, const void* w, float* y, 
     wd_status s = encode_2d(&mw, w, n_out, k_in, kBM);
     if (s != WD_OK) return s;
     WdTcSeg seg = {w, n_out, &mw};
-    WdTcX xm = {x, k_in};
+    WdTcX xm;                       // one-off operand: its descriptor is encoded on the stack (no host allocation)
+    xm.ptr = x; xm.K = k_in; xm.keep = false;
     int sm = 148, dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev);

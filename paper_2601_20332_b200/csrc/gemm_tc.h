@@ -26,6 +26,7 @@ struct WdTcX {
     // shapes come back every step
     struct Entry { int rows, bn; CUtensorMap map; };
     mutable std::vector<Entry> cache;
+    bool keep = true;        // false: one-off operand (single operations): encode on the stack, remember nothing
 };
 
 struct WdTcWeights {
@@ -109,6 +110,8 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
                      const WdTcSwiglu* sg = nullptr);
 // TMA descriptor of a [n_rows, K] byte matrix for the FP8 path (box 128 x box_rows)
 wd_status wd_tc_encode_fp8(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_rows);
+// TMA descriptor of a [n_rows, K] bf16 matrix (box 64 x box_rows, 128-byte swizzle)
+wd_status wd_tc_encode_bf16(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_rows);
 
 size_t wd_tc_scratch_bytes(int rows, int n_out, int k_in);
 wd_status wd_tc_gemm_standalone(const void* x, const void* w, float* y, int rows, int n_out, int k_in, void* scratch,

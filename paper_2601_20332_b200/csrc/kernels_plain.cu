@@ -476,7 +476,7 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
                                     const int32_t* __restrict__ row_seq, const int32_t* __restrict__ row_pos,
                                     const float2* __restrict__ rope_tab, T* __restrict__ q, T* __restrict__ kcache,
                                     T* __restrict__ vcache, int n_rows, int Hq, int Hkv, int dh, int S, int Sp,
-                                    int n_qk, int qk_groups, int n_qk_blocks) {
+                                    int n_qk, int qk_groups, int n_qk_blocks, int batch, int32_t* __restrict__ status) {
     __shared__ float tile[32][33];
     pdl_launch_dependents();
     pdl_wait();
@@ -488,12 +488,15 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
         for (int item = blockIdx.x; item < n_qk; item += n_qk_blocks) {
             const int r = item / qk_groups, grp = item - r * qk_groups;
             const int pos = row_pos[r], b = row_seq[r];
+            // index check: a cache row outside the state is recorded and not written
+            const bool in_range = (unsigned)pos < (unsigned)S && (unsigned)b < (unsigned)batch;
+            if (!in_range && threadIdx.x == 0) atomicCAS(status, 0, WD_ERR_BOUNDS);
             const float* pr = part + (size_t)r * ncol;
             if ((half & 3) == 0) {
                 // four rotation pairs per thread (float4 loads, 8-byte bf16 stores): half/4 threads per head
                 const int tph = half >> 2, hpb = blockDim.x / tph;
                 const int h = grp * hpb + (int)threadIdx.x / tph, j = ((int)threadIdx.x % tph) * 4;
-                if ((int)threadIdx.x < hpb * tph && h < Hq + Hkv) {
+                if ((int)threadIdx.x < hpb * tph && h < Hq + Hkv && (h < Hq || in_range)) {
                     const float4 a = sum_slices4(pr + h * dh + j, n_split, split_stride);
                     const float4 bb = sum_slices4(pr + h * dh + half + j, n_split, split_stride);
                     const float4 c01 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j);       // (cos, sin) x 2
@@ -510,6 +513,7 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
             for (int i = threadIdx.x; i < 4 * half; i += blockDim.x) {
                 const int h = h0 + i / half, j = i % half;
                 if (h >= Hq + Hkv) break;
+                if (h >= Hq && !in_range) continue;
                 const float a = sum_slices1(pr + h * dh + j, n_split, split_stride);
                 const float bb = sum_slices1(pr + h * dh + j + half, n_split, split_stride);
                 const float2 cs = rope_tab[(size_t)r * half + j];
@@ -544,8 +548,12 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
     const int r = r0 + lx;
     if (r < n_rows) {
         const int pos = row_pos[r], b = row_seq[r];
-        T* dst = vcache + ((size_t)b * Hkv + kh) * dh * Sp + pos;
-        for (int dd = ly; dd < 32 && d0 + dd < dh; dd += 8) dst[(size_t)(d0 + dd) * Sp] = from_f<T>(tile[lx][dd]);
+        if ((unsigned)pos < (unsigned)S && (unsigned)b < (unsigned)batch) {
+            T* dst = vcache + ((size_t)b * Hkv + kh) * dh * Sp + pos;
+            for (int dd = ly; dd < 32 && d0 + dd < dh; dd += 8) dst[(size_t)(d0 + dd) * Sp] = from_f<T>(tile[lx][dd]);
+        } else if (ly == 0) {
+            atomicCAS(status, 0, WD_ERR_BOUNDS);
+        }
     }
 }
 
@@ -557,13 +565,17 @@ __global__ void attention_plain_kernel(const T* __restrict__ q, const T* __restr
                                        const T* __restrict__ vcache, const int32_t* __restrict__ row_seq,
                                        const int32_t* __restrict__ vis_idx, const int32_t* __restrict__ vis_off,
                                        T* __restrict__ out, float* __restrict__ tap, int nv_single, int Hq,
-                                       int Hkv, int dh, int S, int Sp) {
+                                       int Hkv, int dh, int S, int Sp, int batch, int32_t* __restrict__ status) {
     extern __shared__ float sc[];                 // [n_vis] scores, then dh floats of q
     __shared__ float red[32];
     pdl_launch_dependents();
     pdl_wait();
     const int r = blockIdx.x, h = blockIdx.y;
-    const int b = row_seq ? row_seq[r] : 0;
+    int b = row_seq ? row_seq[r] : 0;
+    if ((unsigned)b >= (unsigned)batch) {              // index check: recorded, the row reads sequence 0 instead
+        if (threadIdx.x == 0) atomicCAS(status, 0, WD_ERR_BOUNDS);
+        b = 0;
+    }
     const int v0 = vis_off ? vis_off[b] : 0;
     const int nv = vis_off ? vis_off[b + 1] - v0 : nv_single;
     const int kvh = h / (Hq / Hkv);
@@ -576,7 +588,12 @@ __global__ void attention_plain_kernel(const T* __restrict__ q, const T* __restr
     const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nw = blockDim.x >> 5;
     float mx = -INFINITY;
     for (int j = wid; j < nv; j += nw) {
-        const T* kr = kb + (size_t)vis_idx[v0 + j] * dh;
+        const int vi = vis_idx[v0 + j];
+        if ((unsigned)vi >= (unsigned)S) {             // index check: recorded, the position is left out (weight 0)
+            if (lane == 0) { atomicCAS(status, 0, WD_ERR_BOUNDS); sc[j] = -INFINITY; }
+            continue;
+        }
+        const T* kr = kb + (size_t)vi * dh;
         float a = 0.f;
         for (int c = lane; c < dh; c += 32) a += qs[c] * to_f(kr[c]);
         a = warp_sum(a) * scale;
@@ -599,7 +616,10 @@ __global__ void attention_plain_kernel(const T* __restrict__ q, const T* __restr
     for (int c = wid; c < dh; c += nw) {
         const T* vr = vb + (size_t)c * Sp;
         float a = 0.f;
-        for (int j = lane; j < nv; j += 32) a += sc[j] * to_f(vr[vis_idx[v0 + j]]);
+        for (int j = lane; j < nv; j += 32) {
+            const int vi = vis_idx[v0 + j];
+            if ((unsigned)vi < (unsigned)S) a += sc[j] * to_f(vr[vi]);
+        }
         a = warp_sum(a) * inv;
         if (lane == 0) {
             const size_t o = ((size_t)r * Hq + h) * dh + c;
@@ -939,7 +959,7 @@ void wd_launch_gemm_plain(int dtype, const void* x, const void* w, float* y, int
 void wd_launch_rope_scatter(int dtype, const float* part, int n_split, size_t split_stride,
                             const int32_t* row_seq, const int32_t* row_pos, const float2* rope_tab, void* q,
                             void* kcache, void* vcache, int n_rows, int Hq, int Hkv, int dh, int S, int Sp,
-                            cudaStream_t st) {
+                            int batch, int32_t* status, cudaStream_t st) {
     if (n_rows <= 0) return;
     const int half = dh >> 1;
     const int qk_groups = (half & 3) == 0 ? wd_ceil_div(Hq + Hkv, std::max(1, 256 / (half >> 2))) : wd_ceil_div(Hq + Hkv, 4);
@@ -948,13 +968,13 @@ void wd_launch_rope_scatter(int dtype, const float* part, int n_split, size_t sp
     const int n_qk_blocks = std::min(n_qk, 148 * 8);
     WD_DISPATCH(dtype, launch_pdl(rope_scatter_kernel<T>, dim3(n_qk_blocks + n_v), dim3(256), 0, st, part, n_split,
                                   split_stride, row_seq, row_pos, rope_tab, (T*)q, (T*)kcache, (T*)vcache, n_rows, Hq,
-                                  Hkv, dh, S, Sp, n_qk, qk_groups, n_qk_blocks));
+                                  Hkv, dh, S, Sp, n_qk, qk_groups, n_qk_blocks, batch, status));
 }
 
 void wd_launch_attention_plain(int dtype, const void* q, const void* kcache, const void* vcache,
                                const int32_t* row_seq, const int32_t* vis_idx, const int32_t* vis_off,
                                void* out, float* tap, int n_rows, int max_vis, int Hq, int Hkv, int dh,
-                               int S, int Sp, cudaStream_t st) {
+                               int S, int Sp, int batch, int32_t* status, cudaStream_t st) {
     if (n_rows <= 0) return;
     const size_t smem = (size_t)(max_vis + dh) * sizeof(float);
     dim3 grid(n_rows, Hq);
@@ -962,13 +982,13 @@ void wd_launch_attention_plain(int dtype, const void* q, const void* kcache, con
         if (smem > 48 * 1024)
             cudaFuncSetAttribute(attention_plain_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         launch_pdl(attention_plain_kernel<float>, grid, dim3(128), smem, st, (const float*)q, (const float*)kcache,
-                   (const float*)vcache, row_seq, vis_idx, vis_off, (float*)out, tap, max_vis, Hq, Hkv, dh, S, Sp);
+                   (const float*)vcache, row_seq, vis_idx, vis_off, (float*)out, tap, max_vis, Hq, Hkv, dh, S, Sp, batch, status);
     } else {
         using T = __nv_bfloat16;
         if (smem > 48 * 1024)
             cudaFuncSetAttribute(attention_plain_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         launch_pdl(attention_plain_kernel<T>, grid, dim3(128), smem, st, (const T*)q, (const T*)kcache,
-                   (const T*)vcache, row_seq, vis_idx, vis_off, (T*)out, tap, max_vis, Hq, Hkv, dh, S, Sp);
+                   (const T*)vcache, row_seq, vis_idx, vis_off, (T*)out, tap, max_vis, Hq, Hkv, dh, S, Sp, batch, status);
     }
 }
 
@@ -1089,8 +1109,33 @@ wd_status wd_launch_wait_expire(cudaStream_t st) {
     return cudaGetLastError() == cudaSuccess ? WD_OK : WD_ERR_CUDA;
 }
 
+// In host code the symbol's name is a handle, not a device address: looked up once per device
+// (with that device current) and remembered.
 int32_t* wd_op_status_ptr() {
-    int32_t* p = nullptr;
-    if (cudaGetSymbolAddress((void**)&p, g_op_status) != cudaSuccess) return nullptr;
-    return p;
+    static int32_t* cached[64] = {};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cached[dev]) {
+        int32_t* p = nullptr;
+        if (cudaGetSymbolAddress((void**)&p, g_op_status) != cudaSuccess) return nullptr;
+        cached[dev] = p;
+    }
+    return cached[dev];
+}
+
+// Query-tile lists of ONE sequence whose n_rows rows all see positions [0, n_vis): tile t covers
+// rows [128 t, 128 t + n).  Layout of `lists`: seq[n_tiles] | row0[n_tiles] | n[n_tiles] | n_vis[1].
+__global__ void fill_qtiles_kernel(int32_t* lists, int n_rows, int n_vis) {
+    const int n_tiles = (n_rows + 127) / 128;
+    for (int t = threadIdx.x; t < n_tiles; t += blockDim.x) {
+        lists[t] = 0;
+        lists[n_tiles + t] = 128 * t;
+        lists[2 * n_tiles + t] = min(128, n_rows - 128 * t);
+    }
+    if (threadIdx.x == 0) lists[3 * n_tiles] = n_vis;
+}
+
+void wd_launch_fill_qtiles(int32_t* lists, int n_rows, int n_vis, cudaStream_t st) {
+    fill_qtiles_kernel<<<1, 128, 0, st>>>(lists, n_rows, n_vis);
+    ++wd_launch_counter;
 }

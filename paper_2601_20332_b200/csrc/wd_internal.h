@@ -105,7 +105,8 @@ void wd_launch_gemm_plain(int dtype, const void* x, const void* w, float* y, int
 void wd_launch_rope_scatter(int dtype, const float* part, int n_split, size_t split_stride,
                             const int32_t* row_seq, const int32_t* row_pos, const float2* rope_tab, void* q,
                             void* kcache, void* vcache, int n_rows, int Hq, int Hkv, int dh, int S, int Sp,
-                            cudaStream_t st);
+                            int batch, int32_t* status, cudaStream_t st);
+// (a row whose position or sequence index is outside the state records WD_ERR_BOUNDS and writes no cache row)
 
 // general (index-list) attention, CUDA cores.
 //   row_seq[r]: sequence of row r (null: one sequence)
@@ -114,7 +115,8 @@ void wd_launch_rope_scatter(int dtype, const float* part, int n_split, size_t sp
 void wd_launch_attention_plain(int dtype, const void* q, const void* kcache, const void* vcache,
                                const int32_t* row_seq, const int32_t* vis_idx, const int32_t* vis_off,
                                void* out, float* tap, int n_rows, int max_vis, int Hq, int Hkv, int dh,
-                               int S, int Sp, cudaStream_t st);
+                               int S, int Sp, int batch, int32_t* status, cudaStream_t st);
+// (a visible index outside [0, S) or a sequence index outside [0, batch) records WD_ERR_BOUNDS and is not dereferenced)
 
 // h = silu(gate) * up from partials [n_split][n_rows][2F] (columns = [gate | up]); F % 4 == 0
 void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_stride, void* h,
@@ -164,6 +166,9 @@ struct WdPlanLaunch {
     int32_t* status;
 };
 void wd_launch_plan(const WdPlanLaunch& h, cudaStream_t st);
+
+// query-tile lists of one sequence for the tensor-core attention (single operation): see the kernel
+void wd_launch_fill_qtiles(int32_t* lists, int n_rows, int n_vis, cudaStream_t st);
 
 wd_status wd_launch_wait_expire(cudaStream_t st);
 int32_t* wd_op_status_ptr();   // device address of the single-operation status word

@@ -117,6 +117,73 @@ def test_attention_vs_oracle(dtype, rows, nv, Hq, Hkv, dh, S):
     assert np.abs(out - ref).max() / np.abs(ref).max() < tol
 
 
+# The tensor-core attention kernel alone: rows and visible lengths around the 128-wide tiles, MHA and a
+# 7:1 query group, mild and large score magnitudes (q scale 8 puts the row maxima of different key tiles
+# tens of units apart, so the running maximum moves and earlier tiles are rescaled), NaN in every cache
+# row that must not be read, and key splits that leave CTAs of a cluster without a key tile.
+ATTN_TC_CASES = [  # rows, n_vis, Hq, Hkv, S, q scale, max_vis (0 = n_vis)
+    (1, 1, 1, 1, 8, 1.5, 0), (1, 127, 1, 1, 128, 8.0, 0), (127, 128, 1, 1, 136, 1.5, 0), (128, 129, 1, 1, 256, 8.0, 0),
+    (129, 127, 7, 1, 128, 1.5, 0), (300, 1025, 1, 1, 1032, 8.0, 0), (34, 352, 8, 8, 512, 1.5, 0),
+    (35, 3072, 7, 1, 3072, 8.0, 0), (129, 1025, 14, 2, 1040, 1.5, 0), (5, 3072, 1, 1, 3072, 1.5, 0),
+    # max_vis > n_vis: the split is sized for 8 or 24 key tiles, this sequence has 1, 2 or 3
+    (34, 129, 1, 1, 1024, 8.0, 1024), (1, 1, 7, 1, 3072, 1.5, 3072), (130, 300, 2, 2, 1024, 1.5, 1000),
+]
+
+
+@pytest.mark.parametrize("rows,nv,Hq,Hkv,S,qs,mv", ATTN_TC_CASES)
+def test_attention_tc_kernel_vs_oracle(rows, nv, Hq, Hkv, S, qs, mv):
+    dh = 128
+    g = torch.Generator(device=DEV).manual_seed(rows * 7 + nv)
+    q = (torch.randn(rows, Hq, dh, device=DEV, generator=g) * qs).to(torch.bfloat16)
+    kc = torch.randn(Hkv, S, dh, device=DEV, generator=g).to(torch.bfloat16)
+    vc = torch.randn(Hkv, S, dh, device=DEV, generator=g).to(torch.bfloat16)
+    K = kc.double().cpu().numpy().transpose(1, 0, 2)[:nv]
+    V = vc.double().cpu().numpy().transpose(1, 0, 2)[:nv]
+    kc[:, nv:] = float("nan")                     # what must not be read as a value
+    vc[:, nv:] = float("nan")
+    out = wd.op_attention_tc(q, kc, vc.transpose(1, 2).contiguous(), nv, mv).float().cpu().numpy().astype(np.float64)
+    assert wd.op_status() == 0
+    ref, probs = wo.attention_rows(q.double().cpu().numpy(), K, V, Hq // Hkv)
+    assert np.isfinite(out).all()
+    assert np.abs(out - ref).max() / np.abs(ref).max() < 2e-2
+    if qs >= 8 and nv > 128:
+        assert probs.max() > 0.5                  # the large-scale cases really are peaked
+
+
+@pytest.mark.parametrize("n,V,K", [(6, 20000, 256), (34, 126464, 128), (130, 5001, 64), (300, 4099, 64)])
+def test_lm_head_epilogue_statistics_exact_ties(n, V, K):
+    """The LM-head GEMM's epilogue (per-CTA running maximum / lowest argmax / sum of exponentials, merged
+    by the selection kernel) on constructed ties: two identical LM-head rows in different 128-row tiles
+    and different CTAs (the token must be the lower id), an all-zero hidden row (every logit 0: token 0,
+    confidence 1 / V), and two identical hidden rows (equal confidence: the lower position ranks first).
+    The rule itself is checked on the GPU's own logits, which the operation also returns."""
+    g = torch.Generator(device=DEV).manual_seed(n + V)
+    x = torch.randn(n, K, device=DEV, generator=g).to(torch.bfloat16)
+    w = (torch.randn(V, K, device=DEV, generator=g) * 0.05).to(torch.bfloat16)
+    lo, hi = 77, V - 130                                   # far apart: different tiles, different CTAs
+    x[1] = 0                                               # all-zero hidden row
+    x[4] = x[2]                                            # duplicated hidden row
+    w[lo] = (x[2].float() * 0.25).to(torch.bfloat16)       # the largest logit of rows 2 and 4, twice
+    w[hi] = w[lo]
+    pos_np = (np.arange(n) * 3 + 5).astype(np.int32)
+    k = min(4, n)
+    got = wd.op_lm_unmask(x, w, torch.as_tensor(pos_np, device=DEV), k)
+    assert wd.op_status() == 0
+    logits = got["logits"].cpu().numpy()
+    exact = x.double().cpu().numpy() @ w.double().cpu().numpy().T
+    assert np.abs(logits - exact).max() <= 2e-5 * np.abs(exact).max()
+    um = wo.oracle_unmask(logits, pos_np.tolist(), k)
+    assert got["row_token"].tolist() == um["ids"].tolist()
+    assert logits[2, lo] == logits[2, hi] == logits[2].max() and got["row_token"][2] == lo and got["row_token"][4] == lo
+    assert got["row_token"][1] == 0
+    np.testing.assert_allclose(got["row_conf"][1], 1.0 / V, rtol=1e-6)
+    np.testing.assert_allclose(got["row_sumexp"], 1.0 / um["conf"], rtol=1e-7)
+    assert got["row_sumexp"][2] == got["row_sumexp"][4]                  # identical rows: identical bits
+    assert got["positions"] == um["positions"] and got["token_ids"] == um["token_ids"]
+    i2, i4 = got["positions"].index(int(pos_np[2])), got["positions"].index(int(pos_np[4]))
+    assert i4 == i2 + 1                                                  # rows 2 and 4 lead (their logit is huge), lower position first
+
+
 @pytest.mark.parametrize("n,V,k", [(1, 2, 1), (8, 1024, 1), (32, 126464, 1), (64, 126464, 2), (5, 1000, 9), (7, 333, 0)])
 def test_unmask_vs_oracle_bit_exact(n, V, k):
     g = torch.Generator(device=DEV).manual_seed(n * V)

@@ -407,3 +407,100 @@ def test_step_error_codes():
     with pytest.raises(wd.WdError) as e:
         wd.Context(synth.get_config("llada8b", **dict(SMALL_BF16, d=500)), w, 1, S, S, S)
     assert e.value.status == wd.WD_ERR_INVALID_DIMS
+
+
+def _small_state(cfg, w, ids):
+    S = ids.shape[1]
+    ctx = wd.Context(cfg, w, ids.shape[0], S, ids.shape[0] * S, ids.shape[0] * cfg["A"])
+    return ctx, wd.State(ctx, ids)
+
+
+def _steps(st, cfg, n, stream=None):
+    out = []
+    for _ in range(n):
+        status, info = st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"], stream)
+        if status == wd.WD_DONE:
+            break
+        r = st.sync()
+        out.append((info["is_refresh"], info["n_rows"], r["positions"].tolist(), r["token_ids"].tolist(),
+                    r["confidence"].tolist()))
+    return out
+
+
+@pytest.mark.parametrize("queued", [False, True])
+def test_device_index_check_reports_bounds_and_the_state_waits_for_a_reset(queued):
+    """A token id outside the vocabulary in the DEVICE copy of the ids (put there through the test hook; the
+    host entry points reject such ids) is never used as an index: the embedding kernel skips the row and
+    records WD_ERR_BOUNDS, wd_step_sync reports it, the state refuses further steps (WD_ERR_POISONED) until
+    it is reset, and after the reset the same context produces exactly what a fresh state produces."""
+    cfg = synth.get_config("llada8b", **SMALL_BF16)
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    ctx, st = _small_state(cfg, w, ids)
+    want = _steps(st, cfg, 6)
+    st.reset(ids)
+    _steps(st, cfg, 2)
+    first_active = st.plan(0, cfg["A"], cfg["B"], cfg["R"], cfg["T"])["active"][0]
+    st.poke_id(0, first_active, cfg["V"] + 5)
+    n_enq = 3 if queued else 1
+    for _ in range(n_enq):
+        st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])
+    with pytest.raises(wd.WdError) as e:
+        st.sync()
+    assert e.value.status == wd.WD_ERR_BOUNDS
+    for call in (lambda: st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"]),
+                 lambda: st.plan(0, cfg["A"], cfg["B"], cfg["R"], cfg["T"]),
+                 lambda: st.generate(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])):
+        with pytest.raises(wd.WdError) as e:
+            call()
+        assert e.value.status == wd.WD_ERR_POISONED
+    st.reset(ids)
+    assert _steps(st, cfg, 6) == want
+    st.close(); ctx.close()
+
+
+def test_state_export_import_resumes_the_trajectory():
+    """Checkpoint / resume: the blob holds the sequence state and phase bookkeeping, the caller copies the
+    state memory (K/V cache).  Resumed with its cache, a second state continues bit for bit; resumed without
+    it, the next step is a refresh step over the same index sets the oracle's planner gives for a state whose
+    external window was dropped, and generation runs to the end."""
+    from oracle import wd_oracle as wo
+    cfg = synth.get_config("llada8b", **dict(SMALL_BF16, batch=2, k=2))
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    ctx, st = _small_state(cfg, w, ids)
+    _steps(st, cfg, 6)                                    # stops mid-phase (R = 4: steps 4, 5 of the second phase done)
+    blob = st.export()
+    mem = st.mem.clone()
+    snap = [st.read(b) for b in range(2)]
+    rest = _steps(st, cfg, 7)
+    assert [r[0] for r in rest[:3]] == [0, 0, 1]
+    # with the cache: identical continuation
+    st2 = wd.State(ctx, ids)
+    st2.mem.copy_(mem)
+    st2.import_(blob, True)
+    for b in range(2):
+        got = st2.read(b)
+        assert all((got[k] == snap[b][k]).all() if hasattr(got[k], "all") else got[k] == snap[b][k] for k in got)
+    assert _steps(st2, cfg, 7) == rest
+    # without the cache: a refresh first, planned like the oracle plans a state without a stored window
+    st3 = wd.State(ctx, ids)
+    st3.import_(blob, False)
+    for b in range(2):
+        ost = wo.SeqState(ids=snap[b]["ids"], decoded=snap[b]["decoded"], t=snap[b]["t"], since=snap[b]["since"],
+                          dec_step=np.where(snap[b]["dec_step"] == -(1 << 31), wo.NEVER, snap[b]["dec_step"]), wex=[])
+        op = wo.oracle_plan(ost, cfg["A"], cfg["B"], cfg["R"], cfg["T"])
+        p = st3.plan(b, cfg["A"], cfg["B"], cfg["R"], cfg["T"])
+        assert p["refresh"] and op["refresh"] and p["rows"] == op["rows"] == op["vis"] and p["active"] == op["active"]
+        assert p["ext_window"] == op["wex"] and p["transient"] == []
+    tail = _steps(st3, cfg, 200)
+    assert tail[0][0] == 1 and tail[0][1] == sum(int(s["decoded"].sum()) + cfg["A"] + cfg["B"] for s in snap)
+    assert all((st3.read(b)["decoded"]).all() for b in range(2))
+    # foreign or damaged blobs change nothing
+    for bad in (blob[:40], b"x" * len(blob), blob[:-4]):
+        with pytest.raises(wd.WdError) as e:
+            st2.import_(bad, True)
+        assert e.value.status == wd.WD_ERR_BAD_PARAM
+    for s_ in (st, st2, st3):
+        s_.close()
+    ctx.close()

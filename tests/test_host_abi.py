@@ -46,6 +46,12 @@ def test_sizes_and_dims_validation():
     assert wd.lib().wd_state_bytes(C.byref(dims), 2, 512) == 0      # batch above max_batch
     out = C.c_void_p()
     assert wd.lib().wd_create(None, None, None, 0, C.byref(out)) == wd.WD_ERR_NULL
+    # the K/V cache inside the state memory: K rows + transposed V rows (positions padded to 8), all layers, bf16
+    assert wd.lib().wd_kv_bytes(C.byref(dims), 1, 512) == 2 * 32 * 32 * 128 * 512 * 2
+    assert wd.lib().wd_kv_bytes(C.byref(dims), 1, 509) == 32 * 32 * 128 * (509 + 512) * 2
+    assert wd.lib().wd_kv_bytes(C.byref(dims), 1, 512) < kv and wd.lib().wd_kv_bytes(C.byref(bad), 1, 512) == 0
+    assert isinstance(wd.lib().wd_last_error(), bytes)              # no CUDA call has failed in this thread
+    assert b"reset" in wd.lib().wd_status_string(wd.WD_ERR_POISONED)
 
 
 def _walk(seed, S, frac, A, B, R, T, k, prefix, eos_id=None, eos_prob=0.0, refresh_mode=0):

@@ -4,8 +4,9 @@ wd_op_gemm_noalloc serves callers that cannot allocate scratch memory where they
 call from (code inside another framework's memory pool, loops that ban allocator
 calls once running).  It keeps its split-K partial sums in a fixed array inside
 the library, shared by all calls, so the checks here are: it agrees with the
-ordinary entry point, also on a second call that finds the first call's leftovers
-in the array, and it refuses shapes the array cannot hold."""
+ordinary entry point and with the float64 product of the same operands, also on a
+second call that finds the first call's leftovers in the array, and it refuses
+shapes the array cannot hold."""
 import gc
 
 import numpy as np
@@ -44,10 +45,13 @@ def test_noalloc_gemm_matches_ordinary_entry_point_twice_in_a_row():
     torch.cuda.synchronize()
     assert torch.cuda.memory_allocated() == before
     assert wd.op_status() == 0
-    for y, ref in ((y1, ref1), (y2, ref2)):
+    for y, ref, (x, w) in ((y1, ref1, (x1, w1)), (y2, ref2, (x2, w2))):
         a, b = y.cpu().numpy().astype(np.float64), ref.cpu().numpy().astype(np.float64)
         assert np.isfinite(a).all()
         assert np.abs(a - b).max() / np.abs(b).max() < 2e-5
+        # and against the definition itself: the float64 product of the same bf16 operands
+        exact = x.double().cpu().numpy() @ w.double().cpu().numpy().T
+        assert np.abs(a - exact).max() / np.abs(exact).max() < 2e-5
     # and the first shape once more, now over the second call's leftovers
     y3 = torch.empty_like(y1)
     wd.op_gemm_noalloc(x1, w1, y3)

@@ -33,7 +33,12 @@ def max_rel(a, b):
 
 class Parity:
     def __init__(self, cfg, weights, ids, decoded=None, gemm_impl=wd.WD_GEMM_AUTO, oracle_seqs=None,
-                 max_rows=None, max_active=None, fusion=False, eos_id=None, refresh_mode=0, fp8=False):
+                 max_rows=None, max_active=None, fusion=False, eos_id=None, refresh_mode=0, fp8=False,
+                 follow_rounded=False):
+        """follow_rounded: a second oracle follower per sequence runs in the bfloat16 storage-points mode
+        (the same teacher-forced trajectory); `step` then also records, per block, the GPU's distance to it
+        and its own distance to the plain float64 follower: what the storage format alone costs at that
+        depth, the yardstick for the GPU's error in a deep model."""
         self.cfg = cfg
         self.batch, self.S = ids.shape
         dev = weights.tok_embed.device
@@ -61,10 +66,16 @@ class Parity:
         dec = (ids != cfg["mask_id"]) if decoded is None else decoded.astype(bool)
         self.ost = [wo.SeqState(ids=ids[b], decoded=dec[b], eos_id=eos_id, refresh_mode=refresh_mode)
                     for b in self.oracle_seqs]
-        self.oc = [wo.KVCache.empty(self.model.dims, self.S) for _ in self.oracle_seqs]
+        self.follow_rounded = follow_rounded
+        if follow_rounded:      # followers n .. 2n-1: the same sequences with bfloat16 storage points
+            self.ost += [wo.SeqState(ids=ids[b], decoded=dec[b], eos_id=eos_id, refresh_mode=refresh_mode, bf16_points=True)
+                         for b in self.oracle_seqs]
+        self.oc = [wo.KVCache.empty(self.model.dims, self.S) for _ in self.ost]
         self.log = []
 
-    def step(self, A, B, R, T, k, tol_layer=TOL_LAYER, tol_attn=TOL_ATTN, check=True):
+    def step(self, A, B, R, T, k, tol_layer=TOL_LAYER, tol_attn=TOL_ATTN, check=True, envelope=None):
+        """envelope: optional function block index -> (layer tolerance, attention tolerance) for the comparison
+        with the plain float64 oracle (default: tol_layer, tol_attn for every block)."""
         cfg = self.cfg
         L, d, hq, V = cfg["L"], cfg["d"], cfg["Hq"] * cfg["dh"], cfg["V"]
         plans = [self.st.plan(b, A, B, R, T) for b in range(self.batch)]
@@ -85,9 +96,13 @@ class Parity:
         for b in self.oracle_seqs:
             nb = int(res["n_unmasked"][b])
             forced.append((res["positions"][b, :nb].tolist(), res["token_ids"][b, :nb].tolist()))
+        if self.follow_rounded:
+            forced = forced + forced
         outs = wo.oracle_step(self.model, self.ost, self.oc, A, B, R, T, k, forced=forced)
-        worst = dict(layer=0.0, attn=0.0, logits=0.0, ambiguous=0)
-        curve = dict(layer=[0.0] * L, attn=[0.0] * L)      # worst error of each block over the followed sequences
+        worst = dict(layer=0.0, attn=0.0, logits=0.0, ambiguous=0, layer_rounded=0.0, attn_rounded=0.0, logits_rounded=0.0)
+        # worst error of each block over the followed sequences (and against the bf16 storage-points followers)
+        curve = dict(layer=[0.0] * L, attn=[0.0] * L, layer_rounded=[0.0] * L, attn_rounded=[0.0] * L,
+                     layer_format=[0.0] * L, attn_format=[0.0] * L)    # *_format: storage-points oracle against the plain one
         for j, b in enumerate(self.oracle_seqs):
             o, p = outs[j], plans[b]
             assert p["done"] == o["done"]
@@ -109,15 +124,29 @@ class Parity:
                 worst["attn"] = max(worst["attn"], e_a)
                 curve["layer"][l] = max(curve["layer"][l], e_l)
                 curve["attn"][l] = max(curve["attn"][l], e_a)
+                tl, ta = envelope(l) if envelope else (tol_layer, tol_attn)
                 if check:
                     assert np.isfinite(lay[l, r0:r1]).all()
-                    assert e_l <= tol_layer, f"seq {b} layer {l}: rel-RMS {e_l:.3e}"
-                    assert e_a <= tol_attn, f"seq {b} layer {l}: attention max-rel {e_a:.3e}"
+                    assert e_l <= tl, f"seq {b} layer {l}: rel-RMS {e_l:.3e}"
+                    assert e_a <= ta, f"seq {b} layer {l}: attention max-rel {e_a:.3e}"
+                if self.follow_rounded:
+                    orr = outs[len(self.oracle_seqs) + j]
+                    r_l = rel_rms(lay[l, r0:r1], orr["layer_out"][l])
+                    r_a = max_rel(att[l, r0:r1], orr["attn_out"][l])
+                    worst["layer_rounded"] = max(worst["layer_rounded"], r_l)
+                    worst["attn_rounded"] = max(worst["attn_rounded"], r_a)
+                    curve["layer_rounded"][l] = max(curve["layer_rounded"][l], r_l)
+                    curve["attn_rounded"][l] = max(curve["attn_rounded"][l], r_a)
+                    curve["layer_format"][l] = max(curve["layer_format"][l], rel_rms(orr["layer_out"][l], o["layer_out"][l]))
+                    curve["attn_format"][l] = max(curve["attn_format"][l], max_rel(orr["attn_out"][l], o["attn_out"][l]))
             glg = lg[a0:a1]
             e_lg = rel_rms(glg.astype(np.float64), o["logits"])
             worst["logits"] = max(worst["logits"], e_lg)
             if check:
-                assert e_lg <= 2 * tol_layer, f"seq {b}: logits rel-RMS {e_lg:.3e}"
+                assert e_lg <= 2 * (envelope(L - 1)[0] if envelope else tol_layer), f"seq {b}: logits rel-RMS {e_lg:.3e}"
+            if self.follow_rounded:
+                r_lg = rel_rms(glg.astype(np.float64), outs[len(self.oracle_seqs) + j]["logits"])
+                worst["logits_rounded"] = max(worst["logits_rounded"], r_lg)
             # the unmask rule on the GPU's own logits: token ids exact, ranking exact unless the
             # confidence gap at the cut is below rounding
             um = wo.oracle_unmask(glg, op["active"], k)
