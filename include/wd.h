@@ -212,11 +212,21 @@ WD_API wd_status wd_destroy(wd_ctx* ctx);
 /* Choose the GEMM kernel used by later steps (default WD_GEMM_AUTO). */
 WD_API wd_status wd_set_gemm_impl(wd_ctx* ctx, int32_t impl);
 
-/* Experimental (default off): let the GEMM CTA that completes an output tile also do the
- * consumer's element-wise work (1/rms scaling, RoPE + cache scatter, SwiGLU, residual add), which
- * shortens a block from nine kernels to five.  Only taken for bf16 with head_dim 128 and d_model,
- * d_ffn multiples of 128; same results within rounding.  Currently slower than separate kernels. */
-WD_API wd_status wd_set_fusion(wd_ctx* ctx, int32_t on);
+/* Where the element-wise consumers of the projections run (the 1/rms scaling of the normalised
+ * input, RoPE and the K/V cache write of Section 4.3, the residual adds, SwiGLU).  Every mode
+ * computes the same step (Sections 3.1 and 4.3) within rounding; they differ in kernel structure only.
+ *   WD_FUSION_AUTO     (default) the library's choice for the step's row count
+ *   WD_FUSION_NONE     separate kernels after each GEMM (nine kernels per block)
+ *   WD_FUSION_TILE     the GEMM CTA that completes an output tile finishes it (five kernels per block)
+ *   WD_FUSION_CLUSTER  few rows (<= 128): the K slices of a tile are summed inside a thread-block
+ *                      cluster through distributed shared memory and finished by the CTAs that own
+ *                      the result; other row counts fall back to WD_FUSION_NONE
+ *   WD_FUSION_CHAIN    few rows: the projections between two attention calls run as one persistent
+ *                      kernel that never stops streaming weights; other row counts fall back
+ * The fused modes need bf16, head_dim 128 and d_model, d_ffn multiples of 128 (else WD_FUSION_NONE).
+ * Errors: WD_ERR_NULL, WD_ERR_BAD_PARAM. */
+enum { WD_FUSION_AUTO = -1, WD_FUSION_NONE = 0, WD_FUSION_TILE = 1, WD_FUSION_CLUSTER = 2, WD_FUSION_CHAIN = 3 };
+WD_API wd_status wd_set_fusion(wd_ctx* ctx, int32_t mode);
 
 /* GEMM timing for benchmarks.  While enabled, wd_step brackets every GEMM launch
  * (one launch covers all weight matrices that share an input: q/k/v, gate/up)

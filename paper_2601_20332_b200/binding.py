@@ -17,6 +17,7 @@ WD_ERR_NULL, WD_ERR_INVALID_DIMS, WD_ERR_WORKSPACE_TOO_SMALL, WD_ERR_UNSUPPORTED
 WD_ERR_BAD_PARAM, WD_ERR_CAPACITY, WD_ERR_PENDING, WD_ERR_CUDA = -5, -6, -7, -8
 WD_ERR_DEVICE_TIMEOUT, WD_ERR_BOUNDS, WD_ERR_NOT_PENDING, WD_ERR_MISALIGNED, WD_ERR_INTERNAL = -9, -10, -11, -12, -13
 WD_ERR_POISONED = -14
+WD_FUSION_AUTO, WD_FUSION_NONE, WD_FUSION_TILE, WD_FUSION_CLUSTER, WD_FUSION_CHAIN = -1, 0, 1, 2, 3
 WD_F32, WD_BF16 = 0, 1
 WD_GEMM_AUTO, WD_GEMM_PLAIN, WD_GEMM_TCGEN05 = 0, 1, 2
 
@@ -219,8 +220,9 @@ class Context:
     def set_gemm_impl(self, impl: int):
         check(lib().wd_set_gemm_impl(self.handle, impl), "wd_set_gemm_impl")
 
-    def set_fusion(self, on: bool):
-        check(lib().wd_set_fusion(self.handle, 1 if on else 0), "wd_set_fusion")
+    def set_fusion(self, mode: int):
+        """A WD_FUSION_* mode: where the consumers of the GEMMs run (same results within rounding)."""
+        check(lib().wd_set_fusion(self.handle, int(mode)), "wd_set_fusion")
 
     def profile_enable(self, on: bool):
         check(lib().wd_profile_enable(self.handle, 1 if on else 0), "wd_profile_enable")

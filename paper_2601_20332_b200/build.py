@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libwd.so")
-SOURCES = ["api.cu", "planner.cpp", "kernels_plain.cu", "gemm_tc.cu", "attention_tc.cu"]
+SOURCES = ["api.cu", "planner.cpp", "kernels_plain.cu", "gemm_tc.cu", "gemm_ck.cu", "attention_tc.cu"]
 
 
 def _nvcc() -> str:
@@ -32,6 +32,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden", "-cudart", "static",
            "-Xptxas", "-v" if verbose else "-warn-spills"]
+    cmd += os.environ.get("WD_NVCC_FLAGS", "").split()          # e.g. -DWD_CK_TRACE for the development time stamps
     cmd += [os.path.join(CSRC, s) for s in SOURCES]
     cmd += ["-o", LIB]
     res = subprocess.run(cmd, capture_output=True, text=True)

@@ -80,7 +80,7 @@ struct wd_ctx {
     float* sumsq = nullptr;      // [d/128][max_rows] partial sums of squares of the residual rows
     int32_t* tile_counters = nullptr;  // arrival counters of the fused GEMM epilogues (kept zero)
     size_t n_tile_counters = 0;
-    bool fuse = false;           // fused GEMM epilogues (experimental: slower than separate kernels so far)
+    int fuse = WD_FUSION_AUTO;   // where the consumers of the GEMMs run (wd_set_fusion)
     int32_t* plan = nullptr;     // packed index lists of the step
     size_t plan_ints = 0;
     int32_t* result = nullptr;   // [status | n_sel[batch] | pos | tok | conf]
@@ -228,7 +228,7 @@ extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, v
     c->d = *dims;
     // debugging switches: WD_FUSE=1 moves the element-wise work into the GEMM epilogues,
     // WD_NO_PDL=1 launches every kernel fully serialised
-    if (const char* e = getenv("WD_FUSE")) c->fuse = (e[0] == '1');
+    if (const char* e = getenv("WD_FUSE")) c->fuse = atoi(e);       // a WD_FUSION_* value
     if (const char* e = getenv("WD_NO_PDL")) wd_pdl_enabled = !(e[0] == '1');
     c->sm_count = prop.multiProcessorCount;
     c->tok_embed = w->tok_embed;
@@ -371,9 +371,10 @@ extern "C" wd_status wd_set_gemm_impl(wd_ctx* ctx, int32_t impl) {
     return WD_OK;
 }
 
-extern "C" wd_status wd_set_fusion(wd_ctx* ctx, int32_t on) {
+extern "C" wd_status wd_set_fusion(wd_ctx* ctx, int32_t mode) {
     if (!ctx) return WD_ERR_NULL;
-    ctx->fuse = on != 0;
+    if (mode < WD_FUSION_AUTO || mode > WD_FUSION_CHAIN) return WD_ERR_BAD_PARAM;
+    ctx->fuse = mode;
     return WD_OK;
 }
 
@@ -836,7 +837,13 @@ static wd_status run_gemm(wd_ctx* c, const void* x, const WdTcX* x_map, const Wd
         c->prof_step_bytes += (double)ncol * K * elt + (double)rows * K * elt + (double)rows * ncol * 4;
         WD_CUDA_TRY(cudaEventRecord(e0, stream));
     }
-    if (use_tc(c)) {
+    if (use_tc(c) && !fp8 && fuse && fuse->cluster && wd_ck_usable(rows, K, segs, nseg, fuse)) {
+        // few rows: cluster split-K with the consumer in the epilogue; nothing goes to y
+        wd_status s = wd_ck_gemm(x_map, segs, nseg, rows, K, c->sm_count, status, stream, fuse);
+        if (s != WD_OK) return s;
+        if (c->prof_on) c->prof_step_bytes -= (double)rows * ncol * 4 - (double)rows * ncol * 2;   // bf16 results
+        *go = {1, (size_t)rows * ncol, 1, WD_GEMM_TCGEN05};
+    } else if (use_tc(c)) {
         int n_split = 1;
         wd_status s = wd_tc_gemm(x_map, segs, nseg, rows, K, y, y_floats, c->sm_count, status, stream, &n_split,
                                  single_split, fuse, fp8, sg);
@@ -1032,7 +1039,14 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     wd_status s;
 
     const int Sp = st->Sp;
-    const bool fused = use_tc(c) && c->fuse && dh == 128 && D % 128 == 0 && F % 128 == 0;
+    // Where the consumers of the GEMMs run (wd_set_fusion).  The fused forms need the tensor-core path,
+    // head_dim 128 and widths that are multiples of 128; a mode that cannot serve the step's row count
+    // falls back to the separate kernels.  The FP8 mode keeps its separate kernels.
+    const bool fusable = use_tc(c) && dh == 128 && D % 128 == 0 && F % 128 == 0 && !c->fp8_on;
+    int fuse_mode = fusable ? c->fuse : WD_FUSION_NONE;
+    if (fuse_mode == WD_FUSION_AUTO) fuse_mode = WD_FUSION_NONE;
+    if (fuse_mode == WD_FUSION_CLUSTER && !(R_ <= wd_ck_max_rows() && D >= 256 && F >= 256 && hq >= 256)) fuse_mode = WD_FUSION_NONE;
+    const bool fused = fuse_mode != WD_FUSION_NONE;
     const bool fp8 = c->fp8_on && use_tc(c) && !fused;      // FP8 projections (q/k/v, gate/up, down, LM head)
     auto attention = [&](int l, char* kc, char* vc) -> wd_status {
         float* attn_tap = st->taps.attn_out ? st->taps.attn_out + (size_t)l * R_ * hq : nullptr;
@@ -1053,6 +1067,8 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         WdTcFuse base;
         base.counters = c->tile_counters;
         base.rows_total = R_;
+        base.batch = batch;
+        base.cluster = fuse_mode == WD_FUSION_CLUSTER ? 1 : 0;
         base.n_prev_tiles = D / 128;
         base.inv_d = 1.f / (float)D;
         base.eps = d.rms_eps;

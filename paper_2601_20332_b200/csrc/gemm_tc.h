@@ -65,6 +65,8 @@ struct WdTcFuse {
     __nv_bfloat16* kcache = nullptr;
     __nv_bfloat16* vcache = nullptr;
     int Hq = 0, Hkv = 0, S = 0, Sp = 0;
+    int batch = 1;                    // sequences of the state (index check of row_seq)
+    int cluster = 0;                  // 1: take the cluster split-K kernel (gemm_ck.cu) where it can serve the shape
     // RESID: x += tile; xg = bf16(x * gain_next) for the next GEMM; partial sums of squares of the new x
     float* x = nullptr;
     const float* gain_next = nullptr; // null: no xg (after the last block)
@@ -108,6 +110,14 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
                      int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out,
                      bool force_single_split = false, const WdTcFuse* fuse = nullptr, const WdTcFp8* fp8 = nullptr,
                      const WdTcSwiglu* sg = nullptr);
+// Few tokens (rows <= 128), fused modes QKV / RESID / SWIGLU: split-K over the four CTAs of a thread-block
+// cluster, the partial tiles summed through distributed shared memory, the consumer's work done by the
+// CTAs that own the result (gemm_ck.cu).  Nothing is written to a partial-sum buffer.
+bool wd_ck_usable(int rows, int K, const WdTcSeg* segs, int nseg, const WdTcFuse* fuse);
+int wd_ck_max_rows();      // most rows for which every mode fits its buffers beside a ring deep enough to stream
+wd_status wd_ck_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, int K, int sm_count, int32_t* status,
+                     cudaStream_t stream, const WdTcFuse* fuse);
+
 // TMA descriptor of a [n_rows, K] byte matrix for the FP8 path (box 128 x box_rows)
 wd_status wd_tc_encode_fp8(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_rows);
 // TMA descriptor of a [n_rows, K] bf16 matrix (box 64 x box_rows, 128-byte swizzle)

@@ -20,7 +20,7 @@ def built():
 
 
 def run(cfg, n_steps, ids=None, decoded=None, impl=wd.WD_GEMM_AUTO, jitter=0.1, tol_layer=1e-2, tol_attn=2e-2,
-        oracle_seqs=None, weights=None, fusion=False, refresh_mode=0, fp8=False):
+        oracle_seqs=None, weights=None, fusion=wd.WD_FUSION_AUTO, refresh_mode=0, fp8=False):
     w = synth.make_weights(cfg, DEV, gain_jitter=jitter) if weights is None else weights
     ids = synth.make_prompts(cfg) if ids is None else ids
     p = Parity(cfg, w, ids, decoded, gemm_impl=impl, oracle_seqs=oracle_seqs, fusion=fusion, refresh_mode=refresh_mode,
@@ -73,11 +73,16 @@ def test_small_bf16_gqa_batch_two_tokens():
 DH128 = dict(L=2, d=512, Hq=4, Hkv=4, dh=128, F=1024, V=4000, P=200, G=150, A=16, B=40, R=3, T=2, k=2)
 
 
-@pytest.mark.parametrize("Hkv,batch,fusion", [(4, 1, False), (2, 2, False), (1, 1, False), (4, 1, True), (2, 2, True)])
+FUSIONS = [wd.WD_FUSION_NONE, wd.WD_FUSION_TILE, wd.WD_FUSION_CLUSTER, wd.WD_FUSION_CHAIN]
+
+
+@pytest.mark.parametrize("Hkv,batch,fusion", [(4, 1, wd.WD_FUSION_NONE), (2, 2, wd.WD_FUSION_NONE), (1, 1, wd.WD_FUSION_NONE)] +
+                         [(4, 1, f) for f in FUSIONS[1:]] + [(2, 2, f) for f in FUSIONS[1:]] + [(1, 3, f) for f in FUSIONS[2:]])
 def test_bf16_head_dim_128_tensor_core_attention(Hkv, batch, fusion):
     """head_dim 128 takes the tcgen05 attention: two query tiles at the refresh (256 visible
     rows), key tiles with a ragged tail split across CTAs, MHA and GQA, batch of independent
-    windows; with and without the fused GEMM epilogues."""
+    windows; with the consumers of the GEMMs as separate kernels and in every fused form (the
+    cluster and chain forms serve the normal steps: 18 to 54 rows here)."""
     cfg = synth.get_config("llada8b", **dict(DH128, Hkv=Hkv, batch=batch))
     logs = run(cfg, 7, fusion=fusion)
     assert [l["info"]["is_refresh"] for l in logs] == [1, 0, 0, 1, 0, 0, 1]

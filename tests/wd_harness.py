@@ -33,7 +33,7 @@ def max_rel(a, b):
 
 class Parity:
     def __init__(self, cfg, weights, ids, decoded=None, gemm_impl=wd.WD_GEMM_AUTO, oracle_seqs=None,
-                 max_rows=None, max_active=None, fusion=False, eos_id=None, refresh_mode=0, fp8=False,
+                 max_rows=None, max_active=None, fusion=wd.WD_FUSION_AUTO, eos_id=None, refresh_mode=0, fp8=False,
                  follow_rounded=False):
         """follow_rounded: a second oracle follower per sequence runs in the bfloat16 storage-points mode
         (the same teacher-forced trajectory); `step` then also records, per block, the GPU's distance to it
