@@ -304,6 +304,17 @@ WD_API wd_status wd_state_set_eos(wd_state* st, int32_t eos_id);
  * or WD_REFRESH_WINDOW (the variant described at the enum; no counterpart in the paper).
  * Kept across wd_state_reset.  Errors: WD_ERR_NULL, WD_ERR_PENDING, WD_ERR_BAD_PARAM. */
 WD_API wd_status wd_state_set_refresh_mode(wd_state* st, int32_t mode);
+/* Staggered refresh steps for a batch (no counterpart in the paper, which describes one sequence:
+ * Section 4.3 gives every phase one refresh step followed by normal steps, and with one phase clock
+ * per batch all sequences would run their compute-heavy refresh step in the same call).  With
+ * on != 0, sequence i of a batch of n shifts its phase clock by o = i * R / n steps (integer
+ * division): every sequence still refreshes at its first step (nothing is cached yet), a sequence
+ * with 0 < o < R refreshes again at step o, which makes its first phase o steps long, and all
+ * later phases have R steps.  Every phase is a phase of Section 4.3; only where the phases of
+ * different sequences begin differs, so that each call of wd_step carries about n / R refresh
+ * steps and the step time is flat.  Off by default.  Kept across wd_state_reset.
+ * Errors: WD_ERR_NULL, WD_ERR_PENDING. */
+WD_API wd_status wd_state_set_stagger(wd_state* st, int32_t on);
 
 /* ---- FP8 mode (no counterpart in the paper, which calls quantisation orthogonal to the method) ----
  * The projections q/k/v, gate/up, down and the LM head then take both operands in 8-bit floating
@@ -342,12 +353,14 @@ WD_API wd_status wd_plan(const wd_state* st, int32_t seq, int32_t A, int32_t B, 
  * eos_id for adaptive termination (see wd_state_set_eos; token_ids may be NULL
  * when eos_id < 0), step_index t, steps_since_refresh, and the external window
  * stored at the last refresh (ext_window[n_ext_window], ascending; empty before
- * the first step), and refresh_mode (WD_REFRESH_FULL or WD_REFRESH_WINDOW).
+ * the first step), refresh_mode (WD_REFRESH_FULL or WD_REFRESH_WINDOW), and the staggered-refresh
+ * identity of the sequence (stagger_i of stagger_n, see wd_state_set_stagger; stagger_n = 0: off).
  * Errors: as wd_plan, plus WD_ERR_BAD_PARAM for an index outside the sequence. */
 WD_API wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, const int32_t* token_ids,
                              int32_t eos_id, int32_t seq_len, int32_t step_index,
                              int32_t steps_since_refresh, const int32_t* ext_window, int32_t n_ext_window,
-                             int32_t A, int32_t B, int32_t R, int32_t T, int32_t refresh_mode, wd_index_sets* out);
+                             int32_t A, int32_t B, int32_t R, int32_t T, int32_t refresh_mode,
+                             int32_t stagger_i, int32_t stagger_n, wd_index_sets* out);
 
 /* Enqueue one step for every sequence of the state on `stream` and return
  * without waiting.  k = tokens unmasked per sequence (at most the number of

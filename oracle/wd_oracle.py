@@ -69,6 +69,7 @@ class SeqState:
     eos_id: int = None                    # adaptive termination (Section 4.2), None = off
     refresh_mode: int = 0                 # 0: the paper's refresh (Section 4.3); 1: window-only variant (see oracle_plan)
     bf16_points: bool = False             # activations rounded to bfloat16 where a bf16 pipeline stores them (see oracle_layer)
+    stagger: tuple = None                 # (i, n): sequence i of a batch of n with staggered refresh steps (see oracle_plan)
 
     def __post_init__(self):
         self.ids = np.array(self.ids, dtype=np.int64)
@@ -91,6 +92,14 @@ def oracle_plan(st: SeqState, A: int, B: int, R: int, T: int) -> dict:
     new external window and the tokens decoded during the phase that just ended; every other
     visible position (prompt, tokens of earlier phases) keeps the K/V it already has in the
     cache.  The first step of a state always computes everything (nothing is cached yet).
+
+    ``st.stagger = (i, n)`` selects a second VARIANT that is not in the paper, which never discusses
+    batches: sequence i of a batch of n shifts its phase clock by o = i * R // n steps, so that the
+    refresh steps of the batch's sequences fall on different steps instead of all on the same one.
+    Every sequence still refreshes at step 0 (nothing is cached yet); a sequence with 0 < o < R then
+    refreshes again at step o, which makes its first phase o steps long, and every later phase has
+    the paper's R steps (Section 4.3).  Each phase is a phase of the paper; only where the phases of
+    different sequences begin is new.
     """
     if A < 1 or B < 0 or R < 1 or T < 0:
         raise ValueError("bad window parameters")
@@ -112,6 +121,9 @@ def oracle_plan(st: SeqState, A: int, B: int, R: int, T: int) -> dict:
         return dict(done=True)
     Uset = set(U)
     refresh = (st.t == 0) or (st.since >= R) or not any(i in Uset for i in st.wex)
+    if st.stagger is not None:
+        offset = (st.stagger[0] * R) // st.stagger[1]
+        refresh = refresh or (0 < offset < R and st.t == offset)
     if refresh:
         wex = U[: min(A + B, len(U))]
         phase_start = st.t

@@ -82,13 +82,14 @@ SIGNATURES = {
     "wd_state_read": (C.c_int, [vp, i32, i32p, u8p, i32p, i32p, i32p]),
     "wd_debug_taps_set": (C.c_int, [vp, C.POINTER(wd_debug_taps)]),
     "wd_plan": (C.c_int, [vp, i32, i32, i32, i32, i32, C.POINTER(wd_index_sets)]),
-    "wd_plan_raw": (C.c_int, [u8p, i32p, i32p, i32, i32, i32, i32, i32p, i32, i32, i32, i32, i32, i32,
+    "wd_plan_raw": (C.c_int, [u8p, i32p, i32p, i32, i32, i32, i32, i32p, i32, i32, i32, i32, i32, i32, i32, i32,
                               C.POINTER(wd_index_sets)]),
     "wd_fp8_bytes": (C.c_size_t, [C.POINTER(wd_model_dims)]),
     "wd_fp8_enable": (C.c_int, [vp, vp, C.c_size_t, vp]),
     "wd_fp8_set": (C.c_int, [vp, i32]),
     "wd_state_set_eos": (C.c_int, [vp, i32]),
     "wd_state_set_refresh_mode": (C.c_int, [vp, i32]),
+    "wd_state_set_stagger": (C.c_int, [vp, i32]),
     "wd_step": (C.c_int, [vp, i32, i32, i32, i32, i32, vp, C.POINTER(wd_step_info)]),
     "wd_step_sync": (C.c_int, [vp, C.POINTER(wd_step_out)]),
     "wd_step_sync_all": (C.c_int, [vp, C.POINTER(wd_step_out), i32, i32p]),
@@ -180,7 +181,7 @@ WD_REFRESH_FULL, WD_REFRESH_WINDOW = 0, 1
 
 
 def plan_raw(decoded, dec_step, t: int, since: int, ext_window, A: int, B: int, R: int, T: int,
-             token_ids=None, eos_id: int = -1, refresh_mode: int = WD_REFRESH_FULL) -> dict:
+             token_ids=None, eos_id: int = -1, refresh_mode: int = WD_REFRESH_FULL, stagger=None) -> dict:
     """wd_plan_raw: the host planner on explicit state arrays (needs no GPU)."""
     dec = np.ascontiguousarray(decoded, dtype=np.uint8)
     ds = np.ascontiguousarray(dec_step, dtype=np.int32)
@@ -189,7 +190,7 @@ def plan_raw(decoded, dec_step, t: int, since: int, ext_window, A: int, B: int, 
     s, bufs = _index_sets(len(dec))
     check(lib().wd_plan_raw(dec.ctypes.data_as(u8p), _np_i32p(ds), None if ids is None else _np_i32p(ids), eos_id,
                             len(dec), t, since, _np_i32p(wex) if len(wex) else None, len(wex), A, B, R, T,
-                            refresh_mode, C.byref(s)), "wd_plan_raw")
+                            refresh_mode, stagger[0] if stagger else 0, stagger[1] if stagger else 0, C.byref(s)), "wd_plan_raw")
     return _index_sets_dict(s, bufs)
 
 
@@ -317,6 +318,10 @@ class State:
     def set_refresh_mode(self, mode: int):
         """WD_REFRESH_FULL (the paper's refresh) or WD_REFRESH_WINDOW (variant outside the paper)."""
         check(lib().wd_state_set_refresh_mode(self.handle, mode), "wd_state_set_refresh_mode")
+
+    def set_stagger(self, on: bool):
+        """Staggered refresh steps across the sequences of the batch (variant outside the paper)."""
+        check(lib().wd_state_set_stagger(self.handle, 1 if on else 0), "wd_state_set_stagger")
 
     def set_taps(self, layer_out=None, attn_out=None, logits=None):
         """Device float tensors that receive intermediates of later steps (None = off)."""

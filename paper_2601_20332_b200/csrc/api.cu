@@ -87,6 +87,8 @@ struct wd_ctx {
     size_t result_ints = 0;
 
     WdTcWeights tc;              // tensor maps of the weights (bf16 only)
+    WdTcChainState chain;        // counters of the chain kernel (WD_FUSION_CHAIN)
+    bool chain_dirty = false;    // a device-side error may have left them out of step: zero them before the next launch
 
     // FP8 mode (wd_fp8_enable): e4m3 copies of q/k/v, gate/up, down and the LM head with one scale
     // per weight row, FP8 activation buffers with one scale per row, and their tensor maps
@@ -174,7 +176,8 @@ static void carve_ctx(const wd_model_dims* d, Carve& c, size_t off[24]) {
     off[17] = c.take(((size_t)d->d_model / 128 + 1) * MR * 4);  // sumsq
     off[18] = c.take(((max_gemm_cols(d) + 127) / 128) * (MR / 256 + 2) * 4);   // tile counters
     off[19] = ((max_gemm_cols(d) + 127) / 128) * (MR / 256 + 2);
-    off[20] = off[21] = c.off;                                   // (unused)
+    off[20] = c.take(256);                                       // chain kernel counters
+    off[21] = c.off;
 }
 
 extern "C" size_t wd_workspace_bytes(const wd_model_dims* dims) {
@@ -267,6 +270,8 @@ extern "C" wd_status wd_create(const wd_model_dims* dims, const wd_weights* w, v
     c->tile_counters = (int32_t*)(base + off[18]);
     c->n_tile_counters = off[19];
     WD_CUDA_TRY(cudaMemset(c->tile_counters, 0, c->n_tile_counters * 4));
+    c->chain.ready_dev = (int32_t*)(base + off[20]);
+    WD_CUDA_TRY(cudaMemset(c->chain.ready_dev, 0, 256));
     WD_CUDA_TRY(cudaMemset(c->result, 0, 4));
 
     if (dims->dtype == WD_BF16) {
@@ -567,7 +572,7 @@ extern "C" wd_status wd_state_reset(wd_state* st, const int32_t* token_ids, cons
 // ---------------------------------------------------------------------------
 namespace {
 struct BlobHeader { uint32_t magic, version; int32_t batch, S; };
-struct BlobSeq { int32_t t, since, phase_start, eos_id, refresh_mode, n_wex; };
+struct BlobSeq { int32_t t, since, phase_start, eos_id, refresh_mode, n_wex, stagger_i, stagger_n; };
 constexpr uint32_t kBlobMagic = 0x57445354u;     // "WDST"
 }
 
@@ -588,7 +593,7 @@ extern "C" wd_status wd_state_export(const wd_state* st, void* buf, size_t bytes
     BlobHeader h = {kBlobMagic, 1u, st->batch, st->S};
     memcpy(p, &h, sizeof(h)); p += sizeof(h);
     for (const WdSeq& s : st->seqs) {
-        BlobSeq bs = {s.t, s.since, s.phase_start, s.eos_id, s.refresh_mode, (int32_t)s.wex.size()};
+        BlobSeq bs = {s.t, s.since, s.phase_start, s.eos_id, s.refresh_mode, (int32_t)s.wex.size(), s.stagger_i, s.stagger_n};
         memcpy(p, &bs, sizeof(bs)); p += sizeof(bs);
         memcpy(p, s.ids.data(), (size_t)st->S * 4); p += (size_t)st->S * 4;
         memcpy(p, s.dec_step.data(), (size_t)st->S * 4); p += (size_t)st->S * 4;
@@ -619,10 +624,12 @@ extern "C" wd_status wd_state_import(wd_state* st, const void* buf, size_t bytes
         const size_t need = (size_t)S * 8 + wd_align_up((size_t)S, 4);
         if (bs.n_wex < 0 || bs.n_wex > S || bs.t < 0 || bs.since < 0 || bs.phase_start < 0 || bs.phase_start > bs.t ||
             bs.eos_id >= vocab || (bs.refresh_mode != WD_REFRESH_FULL && bs.refresh_mode != WD_REFRESH_WINDOW) ||
+            bs.stagger_n < 0 || bs.stagger_i < 0 || (bs.stagger_n > 0 && bs.stagger_i >= bs.stagger_n) ||
             (size_t)(end - p) < need + (size_t)bs.n_wex * 4)
             return WD_ERR_BAD_PARAM;
         s.t = bs.t; s.since = bs.since; s.phase_start = bs.phase_start;
         s.eos_id = bs.eos_id < 0 ? -1 : bs.eos_id; s.refresh_mode = bs.refresh_mode;
+        s.stagger_i = bs.stagger_i; s.stagger_n = bs.stagger_n;
         s.ids.resize(S); s.dec_step.resize(S); s.decoded.resize(S); s.wex.resize((size_t)bs.n_wex);
         memcpy(s.ids.data(), p, (size_t)S * 4); p += (size_t)S * 4;
         memcpy(s.dec_step.data(), p, (size_t)S * 4); p += (size_t)S * 4;
@@ -727,6 +734,18 @@ extern "C" wd_status wd_state_set_refresh_mode(wd_state* st, int32_t mode) {
     return WD_OK;
 }
 
+extern "C" wd_status wd_state_set_stagger(wd_state* st, int32_t on) {
+    if (!st) return WD_ERR_NULL;
+    if (st->pending) return WD_ERR_PENDING;
+    for (int b = 0; b < st->batch; ++b) {
+        st->seqs[b].stagger_i = on ? b : 0;
+        st->seqs[b].stagger_n = on ? st->batch : 0;
+        st->counts[b].stagger_i = st->seqs[b].stagger_i;
+        st->counts[b].stagger_n = st->seqs[b].stagger_n;
+    }
+    return WD_OK;
+}
+
 extern "C" wd_status wd_debug_taps_set(wd_state* st, const wd_debug_taps* taps) {
     if (!st) return WD_ERR_NULL;
     if (st->pending) return WD_ERR_PENDING;
@@ -765,11 +784,12 @@ extern "C" wd_status wd_plan(const wd_state* st, int32_t seq, int32_t A, int32_t
 extern "C" wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step, const int32_t* token_ids,
                                  int32_t eos_id, int32_t seq_len, int32_t step_index, int32_t steps_since_refresh,
                                  const int32_t* ext_window, int32_t n_ext_window, int32_t A, int32_t B, int32_t R,
-                                 int32_t T, int32_t refresh_mode, wd_index_sets* out) {
+                                 int32_t T, int32_t refresh_mode, int32_t stagger_i, int32_t stagger_n, wd_index_sets* out) {
     if (!decoded || !dec_step || !out || (n_ext_window > 0 && !ext_window)) return WD_ERR_NULL;
     if (eos_id >= 0 && !token_ids) return WD_ERR_NULL;
     if (seq_len < 1 || n_ext_window < 0 || step_index < 0 || steps_since_refresh < 0) return WD_ERR_BAD_PARAM;
     if (refresh_mode != WD_REFRESH_FULL && refresh_mode != WD_REFRESH_WINDOW) return WD_ERR_BAD_PARAM;
+    if (stagger_n < 0 || stagger_i < 0 || (stagger_n > 0 && stagger_i >= stagger_n)) return WD_ERR_BAD_PARAM;
     WdSeq s;
     if (token_ids) s.ids.assign(token_ids, token_ids + seq_len);
     else s.ids.assign(seq_len, 0);
@@ -784,6 +804,8 @@ extern "C" wd_status wd_plan_raw(const uint8_t* decoded, const int32_t* dec_step
     s.since = steps_since_refresh;
     s.phase_start = step_index - steps_since_refresh;       // first step of the running phase
     s.refresh_mode = refresh_mode;
+    s.stagger_i = stagger_i;
+    s.stagger_n = stagger_n;
     WdSeqPlan p;
     wd_status r = wd_plan_seq(s, A, B, R, T, &p);
     if (r != WD_OK) return r;
@@ -1046,7 +1068,14 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     int fuse_mode = fusable ? c->fuse : WD_FUSION_NONE;
     if (fuse_mode == WD_FUSION_AUTO) fuse_mode = WD_FUSION_NONE;
     if (fuse_mode == WD_FUSION_CLUSTER && !(R_ <= wd_ck_max_rows() && D >= 256 && F >= 256 && hq >= 256)) fuse_mode = WD_FUSION_NONE;
+    if (fuse_mode == WD_FUSION_CHAIN && (!wd_tc_chain_rows_ok(R_) || c->prof_on)) fuse_mode = WD_FUSION_NONE;
     const bool fused = fuse_mode != WD_FUSION_NONE;
+    if (c->chain_dirty) {
+        WD_CUDA_TRY(cudaMemsetAsync(c->chain.ready_dev, 0, 256, stream));
+        WD_CUDA_TRY(cudaMemsetAsync(c->tile_counters, 0, c->n_tile_counters * 4, stream));
+        for (int i = 0; i < 4; ++i) c->chain.ready_host[i] = 0;
+        c->chain_dirty = false;
+    }
     const bool fp8 = c->fp8_on && use_tc(c) && !fused;      // FP8 projections (q/k/v, gate/up, down, LM head)
     auto attention = [&](int l, char* kc, char* vc) -> wd_status {
         float* attn_tap = st->taps.attn_out ? st->taps.attn_out + (size_t)l * R_ * hq : nullptr;
@@ -1072,6 +1101,34 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         base.n_prev_tiles = D / 128;
         base.inv_d = 1.f / (float)D;
         base.eps = d.rms_eps;
+        // The fused GEMMs between two attention calls: launched one by one, or (WD_FUSION_CHAIN) as one
+        // persistent launch.
+        WdTcChainItem items[4];
+        WdTcSeg segbuf[4][3];
+        int n_items = 0;
+        auto push = [&](const WdTcX* xm, const WdTcSeg* segs, int nseg, int K, const WdTcFuse& f) {
+            for (int i = 0; i < nseg; ++i) segbuf[n_items][i] = segs[i];
+            items[n_items].x = xm; items[n_items].segs = segbuf[n_items]; items[n_items].nseg = nseg; items[n_items].K = K;
+            items[n_items].fuse = f;
+            ++n_items;
+        };
+        auto flush = [&]() -> wd_status {
+            if (n_items == 0) return WD_OK;
+            bool chained = false;
+            if (fuse_mode == WD_FUSION_CHAIN && !c->prof_on && wd_tc_chain_rows_ok(R_)) {
+                const wd_status cs = wd_tc_chain(items, n_items, R_, c->part, c->part_floats, c->sm_count, status, &c->chain, stream);
+                if (cs == WD_OK) chained = true;
+                else if (cs != WD_ERR_CAPACITY && cs != WD_ERR_BAD_PARAM) return cs;     // shapes the chain cannot take: one by one
+            }
+            for (int i = 0; i < n_items && !chained; ++i) {
+                const wd_status gs = run_gemm(c, items[i].x->ptr, items[i].x, items[i].segs, items[i].nseg, R_, items[i].K, c->part,
+                                              c->part_floats, status, stream, &go, false, &items[i].fuse);
+                if (gs != WD_OK) return gs;
+            }
+            n_items = 0;
+            return WD_OK;
+        };
+        impl_used = WD_GEMM_TCGEN05;
         for (int l = 0; l < d.n_layers; ++l) {
             char* kc = st->kcache + (size_t)l * st->kv_layer_bytes;
             char* vc = st->vcache + (size_t)l * st->v_layer_bytes;
@@ -1083,35 +1140,32 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
             fq.Hq = Hq; fq.Hkv = Hkv; fq.S = S; fq.Sp = Sp;
             WdTcSeg qkv[3] = {{c->wq[l], hq, c->tc.get(WD_TC_WQ, l)}, {c->wk[l], hkv, c->tc.get(WD_TC_WK, l)},
                               {c->wv[l], hkv, c->tc.get(WD_TC_WV, l)}};
-            if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, qkv, 3, R_, D, c->part, c->part_floats, status, stream, &go, false,
-                              &fq)) != WD_OK)
-                return s;
-            impl_used = go.impl;
+            push(&c->tc.x_map_d, qkv, 3, D, fq);
+            if ((s = flush()) != WD_OK) return s;
             if ((s = attention(l, kc, vc)) != WD_OK) return s;
             WdTcFuse fo = base;
             fo.mode = WD_FUSE_RESID;
             fo.x = c->x; fo.gain_next = c->ffn_norm[l]; fo.xg = (__nv_bfloat16*)c->xn; fo.sumsq_out = c->sumsq;
             WdTcSeg wo[1] = {{c->wo[l], D, c->tc.get(WD_TC_WO, l)}};
-            if ((s = run_gemm(c, c->attn, &c->tc.x_map_attn, wo, 1, R_, hq, c->part, c->part_floats, status, stream, &go,
-                              false, &fo)) != WD_OK)
-                return s;
+            push(&c->tc.x_map_attn, wo, 1, hq, fo);
+            static const int chain_max = getenv("WD_CHAIN_MAX") ? atoi(getenv("WD_CHAIN_MAX")) : 4;    // tuning knob: GEMMs per chain launch
+            if (n_items >= chain_max && (s = flush()) != WD_OK) return s;
             WdTcFuse fg = base;
             fg.mode = WD_FUSE_SWIGLU;
             fg.sumsq_in = c->sumsq; fg.h = (__nv_bfloat16*)c->h; fg.F = F;
             WdTcSeg gu[2] = {{c->wg[l], F, c->tc.get(WD_TC_WG, l)}, {c->wu[l], F, c->tc.get(WD_TC_WU, l)}};
-            if ((s = run_gemm(c, c->xn, &c->tc.x_map_d, gu, 2, R_, D, c->part, c->part_floats, status, stream, &go, false,
-                              &fg)) != WD_OK)
-                return s;
+            push(&c->tc.x_map_d, gu, 2, D, fg);
+            if (n_items >= chain_max && (s = flush()) != WD_OK) return s;
             WdTcFuse fd = base;
             fd.mode = WD_FUSE_RESID;
             fd.x = c->x; fd.xg = (__nv_bfloat16*)c->xn; fd.sumsq_out = c->sumsq;
             fd.gain_next = l + 1 < d.n_layers ? c->attn_norm[l + 1] : nullptr;
             fd.tap = st->taps.layer_out ? st->taps.layer_out + (size_t)l * R_ * D : nullptr;
             WdTcSeg wdn[1] = {{c->wd[l], D, c->tc.get(WD_TC_WD, l)}};
-            if ((s = run_gemm(c, c->h, &c->tc.x_map_h, wdn, 1, R_, F, c->part, c->part_floats, status, stream, &go, false,
-                              &fd)) != WD_OK)
-                return s;
+            push(&c->tc.x_map_h, wdn, 1, F, fd);
+            if (n_items >= chain_max && (s = flush()) != WD_OK) return s;
         }
+        if ((s = flush()) != WD_OK) return s;
     } else {
     wd_launch_embed(d.dtype, c->tok_embed, st->ids_dev, row_seq, row_pos, c->x, c->rope_tab, R_, D, S, d.vocab, dh,
                     d.rope_theta, status, stream);
@@ -1304,6 +1358,7 @@ static wd_status drain_queue(wd_state* st, wd_step_out* outs, bool every_step, i
         // the state takes no more steps until wd_state_reset or wd_state_import gives it a consistent start.
         st->dev_mode = false;
         st->poisoned = true;
+        st->ctx->chain_dirty = true;
     }
     else if (host_planned)    // the count shadow did not follow host-planned steps: rebuild it from the mirror
         for (int b = 0; b < batch; ++b) wd_count_init(st->counts[b], st->seqs[b]);

@@ -691,6 +691,340 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
     }
 }
 
+// ------------------------------------------------------------------------------------------
+// Chain kernel: the projections between two attention calls as ONE persistent launch (few rows)
+// ------------------------------------------------------------------------------------------
+// A normal step of the windowed method computes a few dozen rows (Section 4.3), so a block is four
+// weight streams (q/k/v, output projection, gate/up, down) separated by work that touches a few
+// hundred KB: summing split-K partial tiles, the residual add, 1/rms, SwiGLU, RoPE and the cache
+// write.  As separate launches every one of those boundaries idles the memory system for several
+// microseconds (the last CTA's epilogue, the launch dependency, the first operand round trip),
+// which is where a third of the step went.  Here up to four consecutive GEMMs run inside one
+// launch of one CTA per SM, each with the persistent stream-K schedule of gemm_tc_kernel:
+//   * the TMA warp streams the weight boxes of GEMM g+1 straight after those of GEMM g: weights
+//     never depend on anything, so the ring keeps filling while GEMM g is still being finished;
+//     only the small activation box of a stage waits until GEMM g+1's input exists;
+//   * the CTA that completes an output tile of GEMM g finishes it (finalize_unit: the residual add
+//     and the next GEMM's bf16 input, SwiGLU, or RoPE and the cache rows) and counts it on a device
+//     counter; GEMM g+1's input exists when the counter has reached the number of tiles, which the
+//     TMA thread polls (bounded, with back-off);
+//   * the MMA warp and the epilogue warps run as in gemm_tc_kernel, on a stage and accumulator
+//     sequence that simply continues across GEMMs.
+// All CTAs are resident at the same time (one per SM, never more CTAs than SMs), so a CTA that
+// waits for the counter waits for CTAs that are running.  Every wait is bounded as elsewhere.
+constexpr int kChainMax = 4;
+
+struct ChainParams {
+    int n_gemm;
+    TcParams g[kChainMax];
+    int32_t* ready;                   // [kChainMax] tiles finished, counted up across launches (wraps)
+    int32_t target[kChainMax];        // counter value at which this launch's GEMM i is completely finished
+};
+struct ChainMaps {
+    CUtensorMap x[kChainMax];
+    CUtensorMap w[kChainMax][3];
+};
+
+__device__ __forceinline__ int32_t ld_acquire_gpu(const int32_t* p) {
+    int32_t v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+// orders this thread's generic-proxy accesses to global memory with accesses through the async proxy (TMA)
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+
+#ifdef WD_CK_TRACE
+// development aid (not compiled by default): globaltimer stamps of the last chain launch
+__device__ unsigned long long g_chain_trace[160][64];
+#define CH_STAMP(slot) do { if ((slot) < 64) g_chain_trace[blockIdx.x < 160 ? blockIdx.x : 159][(slot)] = global_ns(); } while (0)
+#else
+#define CH_STAMP(slot) do { } while (0)
+#endif
+
+__global__ void __launch_bounds__(kThreads)
+gemm_chain_kernel(const __grid_constant__ ChainMaps maps, const __grid_constant__ ChainParams cp) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const TcParams& p0 = cp.g[0];                          // rows, bn, ring and accumulator shape are common to the chain
+    const int NS = p0.n_stages;
+    const int stage_a = kStageA;
+    const int stage_bytes = stage_a + p0.bn * kBK * 2;
+    uint64_t* bars = (uint64_t*)(smem + (size_t)NS * stage_bytes);
+    // bars[0..NS) full | [NS..2NS) empty | [2NS, 2NS+1] accumulator full | [2NS+2, 2NS+3] accumulator empty
+    uint32_t* tmem_slot = (uint32_t*)(bars + 2 * NS + 4);
+    volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
+    int* last_flag = (int*)(tmem_slot + 2);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const long long G = gridDim.x, c = blockIdx.x;
+    // this CTA's share of every GEMM's line of K blocks
+    Sched sch[kChainMax];
+    int n_tot[kChainMax];
+    long long total = 0;
+#pragma unroll
+    for (int g = 0; g < kChainMax; ++g) {
+        n_tot[g] = 0;
+        if (g < cp.n_gemm) {
+            const long long gb = c * cp.g[g].W / G, ge = (c + 1) * cp.g[g].W / G;
+            sch[g].init(gb, ge, cp.g[g].kb_total);
+            n_tot[g] = (int)(ge - gb);
+            total += n_tot[g];
+        }
+    }
+
+    pdl_launch_dependents();
+    if (threadIdx.x == 0) {
+        CH_STAMP(60);
+        for (int s = 0; s < NS; ++s) {
+            mbar_init(smem_u32(&bars[s]), 1);
+            mbar_init(smem_u32(&bars[NS + s]), 1);
+        }
+        mbar_init(smem_u32(&bars[2 * NS]), 1);
+        mbar_init(smem_u32(&bars[2 * NS + 1]), 1);
+        mbar_init(smem_u32(&bars[2 * NS + 2]), 128);
+        mbar_init(smem_u32(&bars[2 * NS + 3]), 128);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(smem_u32(tmem_slot), 2u * (uint32_t)p0.buf_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        if (lane == 0 && total > 0) {
+            // ------------------------------------------------ TMA producer: a weight cursor and an activation cursor
+            uint64_t pol_stream;
+            asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol_stream));
+            struct Cur {
+                int g, piece, left, kb, n0, tok0;
+                const CUtensorMap* mw;
+                long long i;                               // stages issued so far
+                int s;                                     // ring slot of stage i, kept by increments (no division in the loop)
+                uint32_t ph;                               // (i / NS) & 1
+            };
+            auto enter = [&](Cur& w) {                     // first block of piece w.piece of GEMM w.g
+                while (w.g < cp.n_gemm && w.piece >= sch[w.g].n_pieces) { ++w.g; w.piece = 0; }
+                if (w.g >= cp.n_gemm) return;
+                const TcParams& p = cp.g[w.g];
+                long long gl;
+                int len;
+                sch[w.g].piece(w.piece, gl, len);
+                const int unit = (int)(gl / p.kb_total);
+                w.kb = (int)(gl - (long long)unit * p.kb_total);
+                w.left = len;
+                const UnitInfo u = decode_unit(p, unit, 0);
+                w.n0 = u.n0;
+                w.tok0 = u.tok0;
+                w.mw = &maps.w[w.g][u.seg];
+            };
+            auto advance = [&](Cur& w) {
+                ++w.i;
+                if (++w.s == NS) { w.s = 0; w.ph ^= 1u; }
+                ++w.kb;
+                if (--w.left == 0) { ++w.piece; enter(w); }
+            };
+            Cur cw, cx;
+            cw.g = 0; cw.piece = 0; cw.i = 0; cw.s = 0; cw.ph = 0;
+            enter(cw);
+            cx = cw;
+            bool rdy[kChainMax] = {false, false, false, false};
+            unsigned long long t_idle = 0;
+            bool ok = true;
+            auto issue_w = [&]() {
+                const int s = cw.s;
+                mbar_expect_tx(smem_u32(&bars[s]), (uint32_t)stage_bytes);
+                tma_load_2d_hint(smem_u32(smem + (size_t)s * stage_bytes), cw.mw, smem_u32(&bars[s]), cw.kb * kBK, cw.n0, pol_stream);
+                advance(cw);
+            };
+            while (cx.i < total && ok) {
+                // 1. an activation box that can go goes first (its weight box is already on the way)
+                if (cx.i < cw.i) {
+                    const int g = cx.g;
+                    if (!rdy[g] && g > 0 && (int32_t)(ld_acquire_gpu(cp.ready + (g - 1)) - cp.target[g - 1]) >= 0) {
+                        fence_proxy_async_global();            // the finishers' plain stores -> this thread's TMA loads
+                        rdy[g] = true;
+                        CH_STAMP(g * 14);
+                    }
+                    if (rdy[g]) {
+                        const int s = cx.s;
+                        tma_load_2d(smem_u32(smem + (size_t)s * stage_bytes) + stage_a, &maps.x[g], smem_u32(&bars[s]), cx.kb * kBK,
+                                    cx.tok0);
+                        advance(cx);
+                        t_idle = 0;
+                        continue;
+                    }
+                }
+                // 2. weights: as far ahead as the ring allows
+                if (cw.i < total) {
+                    const int s = cw.s;
+                    const uint32_t ph = cw.ph;
+                    if (cw.i < NS || mbar_try_wait(smem_u32(&bars[NS + s]), ph ^ 1u)) {
+                        issue_w();
+                        t_idle = 0;
+                        continue;
+                    }
+                    if (cx.i == cw.i) {
+                        // nothing else to do until this slot is free: the plain bounded wait
+                        if (!mbar_wait(smem_u32(&bars[NS + s]), ph ^ 1u, abort_flag)) { ok = false; break; }
+                        issue_w();
+                        t_idle = 0;
+                        continue;
+                    }
+                }
+                // 3. the ring is full of weights whose activations do not exist yet
+                if (!rdy[0]) {
+                    pdl_wait();                                // sit out the previous kernel
+                    rdy[0] = true;
+                    CH_STAMP(0);
+                    continue;
+                }
+                if (*abort_flag) ok = false;
+                const unsigned long long now = global_ns();
+                if (t_idle == 0) t_idle = now;
+                else if (now - t_idle > kWaitNs) ok = false;
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicCAS(p0.status, 0, WD_ERR_DEVICE_TIMEOUT);
+            }
+        }
+        __syncwarp();
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ------------------------------------------------ MMA issuer
+            bool ok = true;
+            int s = 0, pc = 0;
+            uint32_t ph = 0;
+            for (int g = 0; g < cp.n_gemm && ok; ++g) {
+                const uint32_t idesc = cp.g[g].idesc;
+                for (int piece = 0; piece < sch[g].n_pieces && ok; ++piece, ++pc) {
+                    long long gl;
+                    int len;
+                    sch[g].piece(piece, gl, len);
+                    const int buf = pc & 1;
+                    const uint32_t par = (uint32_t)(pc >> 1) & 1u;
+                    if (!(ok = mbar_wait(smem_u32(&bars[2 * NS + 2 + buf]), par ^ 1u, abort_flag))) break;
+                    tc_fence_after();
+                    const uint32_t acc = tmem_base + (uint32_t)(buf * p0.buf_cols);
+                    for (int j = 0; j < len; ++j) {
+                        if (!(ok = mbar_wait(smem_u32(&bars[s]), ph, abort_flag))) break;
+                        if (piece == 0 && j == 0) CH_STAMP(g * 14 + 1);
+                        tc_fence_after();
+                        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+                        const uint64_t adesc = make_sdesc(sa), bdesc = make_sdesc(sa + stage_a);
+#pragma unroll
+                        for (int kk = 0; kk < kBK / 16; ++kk)
+                            umma_bf16(acc, adesc + (uint64_t)(2 * kk), bdesc + (uint64_t)(2 * kk), idesc, (j > 0 || kk > 0) ? 1u : 0u);
+                        umma_commit(smem_u32(&bars[NS + s]));
+                        if (++s == NS) { s = 0; ph ^= 1u; }
+                    }
+                    if (ok) umma_commit(smem_u32(&bars[2 * NS + buf]));
+                    CH_STAMP(g * 14 + 2);
+                }
+            }
+            if (!ok) {
+                *abort_flag = 1;
+                atomicCAS(p0.status, 0, WD_ERR_DEVICE_TIMEOUT);
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------------------------------------------- epilogue (warps 2..5)
+        const int quarter = warp & 3;
+        const int n_local = quarter * 32 + lane;
+        const int e = (int)threadIdx.x - 64;
+        pdl_wait();
+        bool ok = true;
+        int pc = 0;
+        for (int g = 0; g < cp.n_gemm && ok; ++g) {
+            const TcParams& p = cp.g[g];
+            for (int piece = 0; piece < sch[g].n_pieces; ++piece, ++pc) {
+                long long gl;
+                int len;
+                sch[g].piece(piece, gl, len);
+                const int unit = (int)(gl / p.kb_total);
+                const UnitInfo u = decode_unit(p, unit, 0);
+                const int buf = pc & 1;
+                const uint32_t par = (uint32_t)(pc >> 1) & 1u;
+                const int n = u.n0 + n_local;
+                const int ord = (int)(c - (((long long)unit * p.kb_total + 1) * G - 1) / p.W);
+                ok = ok && mbar_wait(smem_u32(&bars[2 * NS + buf]), par, abort_flag);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                float* ys = p.y + p.seg_col[u.seg] + n + (size_t)ord * p.split_stride;
+                const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * p0.buf_cols);
+                for (int cc = 0; cc < p.bn; cc += 16) {
+                    if (u.tok0 + cc >= p.rows) break;
+                    uint32_t v[16];
+                    tmem_ld16(t_acc + (uint32_t)cc, v);
+#pragma unroll
+                    for (int t = 0; t < 16; ++t) {
+                        const int tok = u.tok0 + cc + t;
+                        if (tok < p.rows) ys[(size_t)tok * p.ncol] = __uint_as_float(v[t]);
+                    }
+                }
+                tc_fence_before();
+                mbar_arrive(smem_u32(&bars[2 * NS + 2 + buf]));       // accumulator may be overwritten
+                if (e == 0 && piece < 3) CH_STAMP(g * 14 + 3 + 3 * piece);
+                // count this piece's arrival at its tile; the CTA that arrives last finishes the tile
+                __threadfence();
+                epi_sync();
+                if (e == 0) {
+                    int idx = unit, expected;
+                    if (p.f.mode == WD_FUSE_SWIGLU) {
+                        const int tile = unit / p.tok_tiles, tokt = unit - tile * p.tok_tiles;
+                        const int t_in = tile - p.seg_tile0[u.seg];
+                        idx = t_in * p.tok_tiles + tokt;
+                        expected = n_contrib(p, G, (p.seg_tile0[0] + t_in) * p.tok_tiles + tokt) +
+                                   n_contrib(p, G, (p.seg_tile0[1] + t_in) * p.tok_tiles + tokt);
+                    } else {
+                        expected = n_contrib(p, G, unit);
+                    }
+                    const int old = atomicAdd(p.f.counters + idx, 1);
+                    const int last = (old + 1 == expected) ? 1 : 0;
+                    if (last) p.f.counters[idx] = 0;               // ready for the next GEMM that uses this counter
+                    *last_flag = last;
+                    __threadfence();
+                }
+                epi_sync();
+                if (e == 0 && piece < 3) CH_STAMP(g * 14 + 4 + 3 * piece);
+                if (*last_flag) {
+                    finalize_unit(p, G, unit, e);
+                    // the finished tile is the next GEMM's input (read by TMA) and the next finisher's x
+                    fence_proxy_async_global();
+                    __threadfence();
+                    epi_sync();
+                    if (e == 0) atomicAdd(cp.ready + g, 1);
+                    if (e == 0 && piece < 3) CH_STAMP(g * 14 + 5 + 3 * piece);
+                } else {
+                    epi_sync();
+                }
+            }
+        }
+        if (!ok && lane == 0) {
+            *abort_flag = 1;
+            atomicCAS(p0.status, 0, WD_ERR_DEVICE_TIMEOUT);
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) CH_STAMP(61);
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, 2u * (uint32_t)p0.buf_cols);
+    }
+}
+
+#ifdef WD_CK_TRACE
+extern "C" __attribute__((visibility("default"))) int wd_debug_chain_trace(unsigned long long* host /*[160][64]*/) {
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpyFromSymbol(host, g_chain_trace, sizeof(unsigned long long) * 160 * 64);
+}
+#endif
+
 // Two-CTA variant for many tokens (compute-bound shapes).  The CTA pair of a cluster works on one
 // [256 weight rows x BN tokens] tile with tcgen05.mma.cta_group::2: each CTA loads its own 128 weight
 // rows and HALF of the token rows of every K block (the tensor cores of both SMs read both halves),
@@ -1449,6 +1783,108 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     else if (p.f.mode == WD_FUSE_LMSTATS) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<false, true>, mx, m0, m1, m2, p));
     else WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_tc_kernel<false, false>, mx, m0, m1, m2, p));
     if (n_split_out) *n_split_out = p.n_slices;
+    return WD_OK;
+}
+
+// ---- chain launch -------------------------------------------------------------------------
+bool wd_tc_chain_rows_ok(int rows) { return rows >= 1 && rows <= 256; }
+
+wd_status wd_tc_chain(const WdTcChainItem* items, int n, int rows, float* y, size_t y_floats, int sm_count,
+                      int32_t* status, WdTcChainState* cs, cudaStream_t stream) {
+    if (!items || !y || !status || !cs || !cs->ready_dev) return WD_ERR_NULL;
+    if (n < 1 || n > kChainMax || !wd_tc_chain_rows_ok(rows)) return WD_ERR_BAD_PARAM;
+    const TcConfig cfg = pick_config(rows, false, false);
+    if (cfg.tok_tiles != 1 || cfg.ctas_per_sm != 1) return WD_ERR_BAD_PARAM;
+    static ChainParams cp;              // large: kept off the stack (host threads do not step one context concurrently)
+    static ChainMaps maps;
+    memset(&cp, 0, sizeof(cp));
+    cp.n_gemm = n;
+    cp.ready = cs->ready_dev;
+    const long long G = sm_count;
+    int32_t add[kChainMax] = {0, 0, 0, 0};
+    for (int g = 0; g < n; ++g) {
+        const WdTcChainItem& it = items[g];
+        if (!it.x || !it.segs || it.nseg < 1 || it.nseg > 3 || it.K < 8 || it.K % 8) return WD_ERR_BAD_PARAM;
+        const int mode = it.fuse.mode;
+        if (mode != WD_FUSE_QKV && mode != WD_FUSE_RESID && mode != WD_FUSE_SWIGLU) return WD_ERR_BAD_PARAM;
+        if (!it.fuse.counters) return WD_ERR_NULL;
+        TcParams& p = cp.g[g];
+        p.tile_rows = kBM;
+        int tiles = 0, col = 0;
+        for (int i = 0; i < it.nseg; ++i) {
+            if (!it.segs[i].map || it.segs[i].n % kBM) return WD_ERR_BAD_PARAM;      // whole tiles only
+            p.seg_tile0[i] = tiles;
+            p.seg_n[i] = it.segs[i].n;
+            p.seg_col[i] = col;
+            tiles += it.segs[i].n / kBM;
+            col += it.segs[i].n;
+            maps.w[g][i] = *it.segs[i].map;
+        }
+        for (int i = it.nseg; i < 3; ++i) maps.w[g][i] = *it.segs[0].map;
+        if (mode == WD_FUSE_SWIGLU && (it.nseg != 2 || it.segs[0].n != it.segs[1].n)) return WD_ERR_BAD_PARAM;
+        p.seg_tile0[it.nseg] = tiles;
+        p.nseg = it.nseg;
+        p.ncol = col;
+        p.rows = rows;
+        p.bn = cfg.bn;
+        p.kb_total = (it.K + kBK - 1) / kBK;
+        p.tok_tiles = 1;
+        p.tok_split = 1;
+        p.n_units = tiles;
+        p.W = (long long)tiles * p.kb_total;
+        p.n_stages = cfg.n_stages;
+        p.buf_cols = cfg.buf_cols;
+        if (G > p.W / 2) return WD_ERR_BAD_PARAM;                  // at least two K blocks per CTA and GEMM
+        const size_t slice = (size_t)rows * col;
+        const int n_slices = count_slices(p.n_units, p.kb_total, p.W, G);
+        if ((size_t)n_slices * slice > y_floats || n_slices > WD_TC_MAX_SPLIT) return WD_ERR_CAPACITY;
+        p.n_slices = n_slices;
+        p.y = y;
+        p.split_stride = slice;
+        p.status = status;
+        p.idesc = make_idesc(cfg.bn, kBM, false);
+        p.f = it.fuse;
+        // one count per finished tile (gate and up tile of the same columns finish together)
+        add[g] = mode == WD_FUSE_SWIGLU ? p.seg_tile0[1] : tiles;
+        bool hit = false;
+        for (const WdTcX::Entry& e : it.x->cache)
+            if (e.rows == rows && e.bn == cfg.bn) { maps.x[g] = e.map; hit = true; break; }
+        if (!hit) {
+            wd_status s = encode_2d(&maps.x[g], it.x->ptr, rows, it.K, cfg.bn);
+            if (s != WD_OK) return s;
+            if (it.x->keep) {
+                if (it.x->cache.size() >= 16) it.x->cache.erase(it.x->cache.begin());
+                it.x->cache.push_back({rows, cfg.bn, maps.x[g]});
+            }
+        }
+    }
+    for (int g = n; g < kChainMax; ++g) {
+        maps.x[g] = maps.x[0];
+        for (int i = 0; i < 3; ++i) maps.w[g][i] = maps.w[0][0];
+    }
+    for (int g = 0; g < n; ++g) {
+        cs->ready_host[g] = (int32_t)((uint32_t)cs->ready_host[g] + (uint32_t)add[g]);     // wraps; the kernel compares differences
+        cp.target[g] = cs->ready_host[g];
+    }
+    static bool attr_done[64] = {};
+    const int dev = current_device();
+    if (dev < 0) return WD_ERR_CUDA;
+    if (!attr_done[dev]) {
+        WD_CUDA_TRY(cudaFuncSetAttribute(gemm_chain_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 225 * 1024));
+        attr_done[dev] = true;
+    }
+    ++wd_launch_counter;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3((unsigned)G);
+    lc.blockDim = dim3(kThreads);
+    lc.dynamicSmemBytes = cfg.smem;
+    lc.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    lc.attrs = attr;
+    lc.numAttrs = wd_pdl_enabled ? 1 : 0;
+    WD_CUDA_TRY(cudaLaunchKernelEx(&lc, gemm_chain_kernel, maps, cp));
     return WD_OK;
 }
 

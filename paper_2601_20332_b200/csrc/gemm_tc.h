@@ -110,6 +110,25 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
                      int sm_count, int32_t* status, cudaStream_t stream, int* n_split_out,
                      bool force_single_split = false, const WdTcFuse* fuse = nullptr, const WdTcFp8* fp8 = nullptr,
                      const WdTcSwiglu* sg = nullptr);
+// Chain kernel (few rows): up to four consecutive fused GEMMs (modes QKV / RESID / SWIGLU) in one persistent
+// launch whose weight stream never stops; each GEMM's input is the previous one's finished tiles.
+struct WdTcChainItem {
+    const WdTcX* x;
+    const WdTcSeg* segs;
+    int nseg, K;
+    WdTcFuse fuse;
+};
+// Device counters of finished tiles (counted up across launches) and the host's running totals.  After a
+// device-side error the two may disagree: zero both before the next launch.
+struct WdTcChainState {
+    int32_t* ready_dev = nullptr;     // [4], zero-initialised
+    int32_t ready_host[4] = {0, 0, 0, 0};
+};
+bool wd_tc_chain_rows_ok(int rows);
+// WD_ERR_CAPACITY: the partial sums do not fit y (the caller launches the GEMMs one by one instead)
+wd_status wd_tc_chain(const WdTcChainItem* items, int n, int rows, float* y, size_t y_floats, int sm_count,
+                      int32_t* status, WdTcChainState* cs, cudaStream_t stream);
+
 // Few tokens (rows <= 128), fused modes QKV / RESID / SWIGLU: split-K over the four CTAs of a thread-block
 // cluster, the partial tiles summed through distributed shared memory, the consumer's work done by the
 // CTAs that own the result (gemm_ck.cu).  Nothing is written to a partial-sum buffer.

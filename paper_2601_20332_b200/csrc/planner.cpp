@@ -10,6 +10,8 @@
 // recently decoded tokens are computed).  Adaptive termination (Section 4.2): once an
 // end-of-sequence token has been generated, undecoded positions after it are never activated
 // again (they stay far-field) and the sequence is done when nothing undecoded precedes it.
+// Staggered refresh (a variant for batches, which the paper does not discuss): sequence i of n shifts its
+// phase clock by i * R / n steps, so that the batch's refresh steps do not all fall on the same step.
 #include <algorithm>
 #include <climits>
 
@@ -36,6 +38,11 @@ wd_status wd_plan_seq(const WdSeq& s, int32_t A, int32_t B, int32_t R, int32_t T
     bool window_alive = false;
     for (int32_t i : s.wex) if (!s.decoded[i] && i < limit) { window_alive = true; break; }
     p.refresh = (s.t == 0) || (s.since >= R) || !window_alive;
+    {
+        // staggered refresh (variant): this sequence's second refresh comes `offset` steps after the first
+        const int32_t offset = wd_stagger_offset(s.stagger_i, s.stagger_n, R);
+        if (offset > 0 && offset < R && s.t == offset) p.refresh = true;
+    }
 
     if (p.refresh) {
         // long arithmetic: A + B may exceed int32 for "window = everything" callers
@@ -111,6 +118,8 @@ void wd_count_init(WdCount& c, const WdSeq& s) {
     c.t = s.t;
     c.since = s.since;
     c.refresh_mode = s.refresh_mode;
+    c.stagger_i = s.stagger_i;
+    c.stagger_n = s.stagger_n;
     c.wex_size = (int32_t)s.wex.size();
     for (int32_t i : s.wex) c.w_alive += s.decoded[i] ? 0 : 1;
     // tokens unmasked at each step of the running phase, oldest first
@@ -128,6 +137,10 @@ wd_status wd_count_plan(const WdCount& c, int32_t A, int32_t B, int32_t R, int32
     p = WdCountPlan();
     if (c.undecoded == 0) { p.done = true; return WD_OK; }
     p.refresh = (c.t == 0) || (c.since >= R) || (c.w_alive == 0);
+    {
+        const int32_t offset = wd_stagger_offset(c.stagger_i, c.stagger_n, R);
+        if (offset > 0 && offset < R && c.t == offset) p.refresh = true;
+    }
     int32_t w_alive = c.w_alive;
     if (p.refresh) {
         p.n_wex = (int32_t)std::min<int64_t>((int64_t)A + (int64_t)B, c.undecoded);

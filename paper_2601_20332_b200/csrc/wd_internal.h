@@ -37,7 +37,13 @@ struct WdSeq {
     int32_t phase_start = 0;
     int32_t eos_id = -1;            // adaptive termination: id of the end-of-sequence token, -1 = off
     int32_t refresh_mode = 0;       // WD_REFRESH_FULL (the paper's refresh) or WD_REFRESH_WINDOW (variant)
+    int32_t stagger_i = 0, stagger_n = 0;   // staggered refresh (variant): sequence i of n, n = 0: off
 };
+
+// steps by which sequence i of n shifts its phase clock when refresh steps are staggered (0: not at all)
+static inline int32_t wd_stagger_offset(int32_t i, int32_t n, int32_t R) {
+    return n > 0 ? (int32_t)(((int64_t)i * R) / n) : 0;
+}
 
 struct WdSeqPlan {
     bool done = false, refresh = false, vis_contiguous = false;
@@ -59,6 +65,7 @@ struct WdCount {
     int32_t wex_size = 0, w_alive = 0;    // external window: size at phase start, still undecoded
     int32_t t = 0, since = 0;
     int32_t refresh_mode = 0;
+    int32_t stagger_i = 0, stagger_n = 0;
     std::vector<int32_t> hist;            // tokens unmasked at each step of the current phase
 };
 struct WdCountPlan {

@@ -20,11 +20,11 @@ def built():
 
 
 def run(cfg, n_steps, ids=None, decoded=None, impl=wd.WD_GEMM_AUTO, jitter=0.1, tol_layer=1e-2, tol_attn=2e-2,
-        oracle_seqs=None, weights=None, fusion=wd.WD_FUSION_AUTO, refresh_mode=0, fp8=False):
+        oracle_seqs=None, weights=None, fusion=wd.WD_FUSION_AUTO, refresh_mode=0, fp8=False, stagger=False):
     w = synth.make_weights(cfg, DEV, gain_jitter=jitter) if weights is None else weights
     ids = synth.make_prompts(cfg) if ids is None else ids
     p = Parity(cfg, w, ids, decoded, gemm_impl=impl, oracle_seqs=oracle_seqs, fusion=fusion, refresh_mode=refresh_mode,
-               fp8=fp8)
+               fp8=fp8, stagger=stagger)
     logs = []
     for _ in range(n_steps):
         r = p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"], tol_layer, tol_attn)
@@ -509,3 +509,41 @@ def test_state_export_import_resumes_the_trajectory():
     for s_ in (st, st2, st3):
         s_.close()
     ctx.close()
+
+
+@pytest.mark.parametrize("shape,batch,R", [(SMALL_BF16, 4, 4), (DH128, 3, 4), (DH128, 8, 3)])
+def test_staggered_refresh_variant_matches_its_oracle(shape, batch, R):
+    """wd_state_set_stagger (not in the paper): sequence i of the batch shifts its phase clock by i * R / n
+    steps, so one call of wd_step carries refresh steps of some sequences (hundreds of rows, all K/V written)
+    and normal steps of the others (a few rows, cached K/V read).  Index sets, layer outputs, logits and
+    unmask choices follow the oracle run in the same mode; the steps are planned on the device."""
+    cfg = synth.get_config("llada8b", **dict(shape, batch=batch, R=R))
+    logs = run(cfg, 3 * R + 2, stagger=True)
+    for t, l in enumerate(logs):
+        kinds = [p["refresh"] for p in l["plans"]]
+        want = [t == 0 or (t >= (i * R) // batch and (t - (i * R) // batch) % R == 0) for i in range(batch)]
+        assert kinds == want, (t, kinds)
+    mixed = [l for l in logs[1:] if any(p["refresh"] for p in l["plans"]) and not all(p["refresh"] for p in l["plans"])]
+    assert len(mixed) >= 2 * R                     # refresh and normal steps really share calls
+    # the rows of a mixed call: the visible positions of the refreshing sequences plus a few rows of the others
+    l = mixed[0]
+    assert l["info"]["n_rows"] == sum(len(p["vis"]) if p["refresh"] else len(p["active"]) + len(p["transient"]) for p in l["plans"])
+
+
+def test_staggered_refresh_queued_steps_match_stepwise_sync():
+    """Steps enqueued back to back (planned by the device kernel from counts that now differ per sequence in
+    kind) give the same tokens as stepping with a sync after every step."""
+    cfg = synth.get_config("llada8b", **dict(DH128, batch=4, R=4))
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    ctx, st = _small_state(cfg, w, ids)
+    st.set_stagger(True)
+    want = _steps(st, cfg, 12)
+    st.reset(ids)
+    got = []
+    for _ in range(12):
+        st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])
+    for r in st.sync_all(32):
+        got.append((r["positions"].tolist(), r["token_ids"].tolist(), r["confidence"].tolist()))
+    assert got == [(w_[2], w_[3], w_[4]) for w_ in want]
+    st.close(); ctx.close()

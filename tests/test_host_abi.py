@@ -54,13 +54,13 @@ def test_sizes_and_dims_validation():
     assert b"reset" in wd.lib().wd_status_string(wd.WD_ERR_POISONED)
 
 
-def _walk(seed, S, frac, A, B, R, T, k, prefix, eos_id=None, eos_prob=0.0, refresh_mode=0):
+def _walk(seed, S, frac, A, B, R, T, k, prefix, eos_id=None, eos_prob=0.0, refresh_mode=0, stagger=None):
     rng = np.random.default_rng(seed)
     dec = (np.arange(S) < int(S * frac)) if prefix else (rng.random(S) < frac)
     ids0 = np.where(dec, 3, 0)
     if eos_id is not None:
         ids0[: max(1, S // 8)] = np.where(dec[: max(1, S // 8)], eos_id, 0)     # eos ids among the GIVEN tokens
-    st = SeqState(ids=ids0.astype(np.int64), decoded=dec, eos_id=eos_id, refresh_mode=refresh_mode)
+    st = SeqState(ids=ids0.astype(np.int64), decoded=dec, eos_id=eos_id, refresh_mode=refresh_mode, stagger=stagger)
     # mirror of the state kept by the test for the raw planner
     m_dec = dec.astype(np.uint8).copy()
     m_ids = ids0.astype(np.int32).copy()
@@ -70,7 +70,7 @@ def _walk(seed, S, frac, A, B, R, T, k, prefix, eos_id=None, eos_prob=0.0, refre
     while True:
         want = oracle_plan(st, A, B, R, T)
         got = wd.plan_raw(m_dec, m_step, m_t, m_since, m_wex, A, B, R, T, token_ids=m_ids,
-                          eos_id=-1 if eos_id is None else eos_id, refresh_mode=refresh_mode)
+                          eos_id=-1 if eos_id is None else eos_id, refresh_mode=refresh_mode, stagger=stagger)
         assert got["done"] == want["done"]
         if want["done"]:
             break
@@ -125,6 +125,19 @@ def test_host_planner_matches_oracle_with_window_only_refresh(case):
     assert _walk(*case, eos_id=7, eos_prob=0.1, refresh_mode=1) > 0
 
 
+@pytest.mark.parametrize("case", [
+    (30, 96, 0.33, 8, 16, 4, 2, 1, True), (31, 70, 0.4, 3, 5, 5, 9, 2, False), (32, 300, 0.3, 32, 64, 8, 2, 1, True),
+    (33, 64, 0.5, 8, 0, 1, 0, 2, True), (34, 120, 0.2, 6, 10, 16, 3, 1, True),
+])
+def test_host_planner_matches_oracle_with_staggered_refresh(case):
+    """The batch variant outside the paper (wd_state_set_stagger): sequence i of n, for several i and n,
+    with the paper's refresh and with the window-only one."""
+    for stagger in ((0, 4), (1, 4), (3, 4), (5, 8), (7, 8), (2, 3)):
+        assert _walk(*case, stagger=stagger) > 0
+    assert _walk(*case, stagger=(3, 8), refresh_mode=1) > 0
+    assert _walk(*case, stagger=(1, 2), eos_id=7, eos_prob=0.1) > 0
+
+
 def test_plan_raw_errors():
     dec = np.zeros(8, np.uint8)
     ds = np.full(8, INT32_MIN, np.int32)
@@ -138,12 +151,15 @@ def test_plan_raw_errors():
     with pytest.raises(wd.WdError) as e:
         wd.plan_raw(dec, ds, 0, 0, [], 2, 2, 2, 1, refresh_mode=2)
     assert e.value.status == wd.WD_ERR_BAD_PARAM
+    with pytest.raises(wd.WdError) as e:
+        wd.plan_raw(dec, ds, 0, 0, [], 2, 2, 2, 1, stagger=(4, 4))      # sequence index outside the batch
+    assert e.value.status == wd.WD_ERR_BAD_PARAM
     # capacity too small for the lists
     import ctypes as C
     s, bufs = wd._index_sets(8)
     s.capacity = 2
     r = wd.lib().wd_plan_raw(dec.ctypes.data_as(wd.u8p), ds.ctypes.data_as(wd.i32p), None, -1, 8, 0, 0, None, 0, 4, 2,
-                             2, 1, 0, C.byref(s))
+                             2, 1, 0, 0, 0, C.byref(s))
     assert r == wd.WD_ERR_CAPACITY
     # huge window parameters must not overflow
     p = wd.plan_raw(dec, ds, 0, 0, [], 2**31 - 1, 2**31 - 1, 1, 0)

@@ -265,3 +265,57 @@ def test_window_refresh_rows_are_the_new_window_plus_the_previous_phase():
 def test_window_refresh_first_step_is_a_full_refresh():
     w = _walk(1, steps=1)[0]
     assert w["refresh"] and w["rows"] == w["vis"]
+
+
+# ---------------------------------------------------------------------------
+# staggered refresh steps across a batch (a variant outside the paper, flagged by SeqState.stagger)
+# ---------------------------------------------------------------------------
+
+def _walk_batch(n, R, stagger, S=200, P=20, A=4, B=12, T=2, k=1, steps=40, seed=5):
+    rng = np.random.default_rng(seed)
+    ids = np.where(np.arange(S) < P, 5, 99)
+    sts = [SeqState(ids=ids, decoded=np.arange(S) < P, stagger=(i, n) if stagger else None) for i in range(n)]
+    traces = [[] for _ in range(n)]
+    for _ in range(steps):
+        for i, st in enumerate(sts):
+            pl = oracle_plan(st, A, B, R, T)
+            assert not pl["done"]
+            traces[i].append(pl)
+            chosen = sorted(rng.choice(pl["active"], size=min(k, len(pl["active"])), replace=False).tolist())
+            oracle_commit(st, pl, chosen, [7] * len(chosen))
+    return traces
+
+
+@pytest.mark.parametrize("n,R", [(8, 4), (4, 8), (3, 5), (16, 4), (2, 2), (5, 1)])
+def test_staggered_refresh_spreads_the_refresh_steps_of_a_batch(n, R):
+    tr = _walk_batch(n, R, True)
+    base = _walk_batch(n, R, False)
+    for i in range(n):
+        o = (i * R) // n
+        got = [t for t, pl in enumerate(tr[i]) if pl["refresh"]]
+        # step 0 (nothing cached), then step o if 0 < o < R, then every R steps: each phase is a phase of Section 4.3
+        want = sorted({0} | {t for t in range(40) if t >= o and (t - o) % R == 0})
+        assert got == want, (i, got)
+        gaps = np.diff(got)
+        assert (gaps[1:] == R).all() and gaps[0] in (R, o)
+        # without the variant every sequence refreshes on the same steps
+        assert [t for t, pl in enumerate(base[i]) if pl["refresh"]] == list(range(0, 40, R))
+    # at most ceil(n / R) sequences refresh in any step after the first
+    per_step = [sum(tr[i][t]["refresh"] for i in range(n)) for t in range(40)]
+    assert per_step[0] == n and max(per_step[R:]) <= -(-n // R) and min(per_step[R:]) >= n // R
+    # sequence 0 is never shifted: identical to the unstaggered run
+    assert [pl for pl in tr[0]] == [pl for pl in base[0]]
+
+
+def test_staggered_refresh_keeps_the_set_identities():
+    """Only where the phases begin changes: the partition of Section 4.2 holds at every step."""
+    for pls in _walk_batch(4, 8, True, steps=60):
+        for pl in pls:
+            act, buf, far, dec = set(pl["active"]), set(pl["buffer"]), set(pl["far_field"]), set(pl["decoded"])
+            assert not (act & buf) and not (act & far) and not (buf & far) and not ((act | buf | far) & dec)
+            assert len(act | buf | far | dec) == 200
+            assert set(pl["transient"]) <= set(pl["in_phase_decoded"]) <= dec
+            assert set(pl["vis"]) == dec | act | buf
+            assert pl["rows"] == (pl["vis"] if pl["refresh"] else sorted(act | set(pl["transient"])))
+            if pl["refresh"]:
+                assert pl["transient"] == [] and pl["in_phase_decoded"] == []

@@ -34,7 +34,7 @@ def max_rel(a, b):
 class Parity:
     def __init__(self, cfg, weights, ids, decoded=None, gemm_impl=wd.WD_GEMM_AUTO, oracle_seqs=None,
                  max_rows=None, max_active=None, fusion=wd.WD_FUSION_AUTO, eos_id=None, refresh_mode=0, fp8=False,
-                 follow_rounded=False):
+                 follow_rounded=False, stagger=False):
         """follow_rounded: a second oracle follower per sequence runs in the bfloat16 storage-points mode
         (the same teacher-forced trajectory); `step` then also records, per block, the GPU's distance to it
         and its own distance to the plain float64 follower: what the storage format alone costs at that
@@ -54,6 +54,8 @@ class Parity:
             self.st.set_eos(eos_id)
         if refresh_mode:
             self.st.set_refresh_mode(refresh_mode)
+        if stagger:
+            self.st.set_stagger(True)
         L, d, hq, V = cfg["L"], cfg["d"], cfg["Hq"] * cfg["dh"], cfg["V"]
         self.t_layer = torch.zeros(L * max_rows * d, dtype=torch.float32, device=dev)
         self.t_attn = torch.zeros(L * max_rows * hq, dtype=torch.float32, device=dev)
@@ -64,12 +66,13 @@ class Parity:
             self.model.dims = dict(self.model.dims, fp8=True)
         self.oracle_seqs = list(range(self.batch)) if oracle_seqs is None else list(oracle_seqs)
         dec = (ids != cfg["mask_id"]) if decoded is None else decoded.astype(bool)
-        self.ost = [wo.SeqState(ids=ids[b], decoded=dec[b], eos_id=eos_id, refresh_mode=refresh_mode)
+        stg = (lambda b: (b, self.batch)) if stagger else (lambda b: None)
+        self.ost = [wo.SeqState(ids=ids[b], decoded=dec[b], eos_id=eos_id, refresh_mode=refresh_mode, stagger=stg(b))
                     for b in self.oracle_seqs]
         self.follow_rounded = follow_rounded
         if follow_rounded:      # followers n .. 2n-1: the same sequences with bfloat16 storage points
-            self.ost += [wo.SeqState(ids=ids[b], decoded=dec[b], eos_id=eos_id, refresh_mode=refresh_mode, bf16_points=True)
-                         for b in self.oracle_seqs]
+            self.ost += [wo.SeqState(ids=ids[b], decoded=dec[b], eos_id=eos_id, refresh_mode=refresh_mode, bf16_points=True,
+                                     stagger=stg(b)) for b in self.oracle_seqs]
         self.oc = [wo.KVCache.empty(self.model.dims, self.S) for _ in self.ost]
         self.log = []
 
