@@ -440,6 +440,16 @@ WD_API wd_status wd_op_gemm_fp8(const void* x, const void* w, float* y, int32_t 
                          void* scratch, size_t scratch_bytes, void* stream /*cudaStream_t*/);
 WD_API size_t wd_op_gemm_fp8_scratch_bytes(int32_t rows, int32_t n_out, int32_t k_in);
 
+/* The NVFP4 projection of the NVFP4 mode as a single operation (see wd_fp4_enable; no counterpart in the
+ * paper): both bf16 operands are quantised into `scratch` (4-bit e2m1 codes, one unsigned e4m3 scale per
+ * block of 16 elements along k, one float scale per row), multiplied on the block-scaled tensor-core
+ * path (tcgen05 kind::mxf4nvf4, block scales applied by the hardware from tensor memory, fp32
+ * accumulation) and scaled back by the row scales; y[rows, n_out] float.  k_in a multiple of 256;
+ * scratch 256-byte aligned, wd_op_gemm_fp4_scratch_bytes large.  Errors as wd_op_gemm. */
+WD_API wd_status wd_op_gemm_fp4(const void* x, const void* w, float* y, int32_t rows, int32_t n_out, int32_t k_in,
+                         void* scratch, size_t scratch_bytes, void* stream /*cudaStream_t*/);
+WD_API size_t wd_op_gemm_fp4_scratch_bytes(int32_t rows, int32_t n_out, int32_t k_in);
+
 /* (No counterpart in the paper: a packaging variant of wd_op_gemm.)
  * The same bf16 tensor-core GEMM, y[rows, n_out] (float) = x[rows, k_in] * w[n_out, k_in]^T,
  * for callers that cannot hand over scratch memory because they may not allocate

@@ -260,7 +260,70 @@ def fp8_matmul(x: np.ndarray, w: np.ndarray) -> np.ndarray:
     return (qx @ qw.T) * sx.astype(np.float64)[:, None] * sw.astype(np.float64)[None, :]
 
 
+# ---------------------------------------------------------------------------
+# NVFP4 mode (a second option outside the paper: 4-bit block-scaled operands)
+# ---------------------------------------------------------------------------
+# With dims["nvfp4"] set, the same projections take both operands in the NVFP4 format: elements are
+# 4-bit floats e2m1 (1 sign, 2 exponent, 1 mantissa bit: 0, 0.5, 1, 1.5, 2, 3, 4, 6 and their
+# negatives), every block of 16 consecutive elements along the reduction dimension shares one scale
+# stored as an unsigned e4m3 number, and every row has one float32 scale on top:
+#   g   = fl32(max|row| / (6 * 448))                 (1 for an all-zero row)
+#   s_b = e4m3(fl32(fl32(max|block| / 6) / g))       (round to nearest even; at most 448 by construction)
+#   q_i = e2m1(fl32(x_i / fl32(s_b * g)))            (round to nearest even, saturating at 6; 0 if s_b = 0)
+# and x_i is represented by q_i * s_b * g.  The value that is quantised is the bfloat16 rounding of the
+# activation (the pipeline stores its normalised rows as bfloat16 before quantising them); weights are
+# bfloat16 already.  The product is the exact sum over blocks of (s_a s_w) * sum_i q_a,i q_w,i, times the
+# two row scales.
+
+E2M1_GRID = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+
+
+def e2m1_round(v32: np.ndarray) -> np.ndarray:
+    """Nearest e2m1 value of each float32 (ties to the even code, saturating at +-6), as float64."""
+    v = np.asarray(v32, dtype=np.float32).astype(np.float64)
+    a = np.abs(v)
+    # midpoints between neighbours; a tie goes to the neighbour whose code (index in the grid) is even
+    out = np.zeros_like(a)
+    for i in range(1, 8):
+        mid = (E2M1_GRID[i - 1] + E2M1_GRID[i]) / 2.0
+        up = (a > mid) | ((a == mid) & (i % 2 == 0))
+        out = np.where(up, E2M1_GRID[i], out)
+    return np.copysign(out, v)
+
+
+def nvfp4_quant_rows(x: np.ndarray):
+    """NVFP4 quantisation of a [n, K] matrix, K a multiple of 16: (q on the e2m1 grid [n, K] as float64,
+    block scales [n, K / 16] as float64 on the e4m3 grid, row scales [n] float32)."""
+    x32 = bf16_round(np.asarray(x)).astype(np.float32)
+    n, K = x32.shape
+    blocks = x32.reshape(n, K // 16, 16)
+    amax = np.abs(x32).max(axis=1) if K else np.zeros(n, np.float32)
+    g = np.where(amax > 0, (amax / np.float32(6.0 * 448.0)).astype(np.float32), np.float32(1.0)).astype(np.float32)
+    bmax = np.abs(blocks).max(axis=2).astype(np.float32)
+    s = e4m3_round(((bmax / np.float32(6.0)).astype(np.float32) / g[:, None]).astype(np.float32))          # float64, on the grid
+    d = (s.astype(np.float32) * g[:, None]).astype(np.float32)                                             # fl32(s_b * g)
+    safe = np.where(d > 0, d, np.float32(1.0)).astype(np.float32)
+    q = e2m1_round((blocks / safe[:, :, None]).astype(np.float32))
+    q = np.where(d[:, :, None] > 0, q, 0.0)
+    return q.reshape(n, K), s, g
+
+
+def nvfp4_matmul(x: np.ndarray, w: np.ndarray) -> np.ndarray:
+    """x w^T with both operands in NVFP4 (see above)."""
+    qx, sx, gx = nvfp4_quant_rows(x)
+    qw, sw, gw = nvfp4_quant_rows(w)
+    n, K = qx.shape
+    m = qw.shape[0]
+    out = np.zeros((n, m))
+    for b in range(K // 16):
+        part = qx[:, 16 * b:16 * b + 16] @ qw[:, 16 * b:16 * b + 16].T
+        out += part * sx[:, b][:, None] * sw[:, b][None, :]
+    return out * gx.astype(np.float64)[:, None] * gw.astype(np.float64)[None, :]
+
+
 def _proj(dims: dict, x: np.ndarray, w: np.ndarray) -> np.ndarray:
+    if dims.get("nvfp4"):
+        return nvfp4_matmul(x, w)
     return fp8_matmul(x, w) if dims.get("fp8") else x @ w.T
 
 

@@ -98,6 +98,8 @@ SIGNATURES = {
     "wd_op_gemm_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
     "wd_op_gemm_fp8": (C.c_int, [vp, vp, vp, i32, i32, i32, vp, C.c_size_t, vp]),
     "wd_op_gemm_fp8_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
+    "wd_op_gemm_fp4": (C.c_int, [vp, vp, vp, i32, i32, i32, vp, C.c_size_t, vp]),
+    "wd_op_gemm_fp4_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
     "wd_op_gemm_noalloc": (C.c_int, [vp, vp, vp, i32, i32, i32, vp]),
     "wd_op_gemm_noalloc_max_floats": (C.c_size_t, []),
     "wd_op_attention": (C.c_int, [i32, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]),
@@ -413,6 +415,18 @@ def op_gemm_fp8(x, w, stream=None):
     nb = lib().wd_op_gemm_fp8_scratch_bytes(rows, n, k)
     scratch = torch.empty(max(nb, 256), dtype=torch.uint8, device=x.device)
     check(lib().wd_op_gemm_fp8(_ptr(x), _ptr(w), _ptr(y), rows, n, k, _ptr(scratch), nb, _stream_ptr(stream)), "wd_op_gemm_fp8")
+    return y
+
+
+def op_gemm_fp4(x, w, stream=None):
+    """y[rows, n] (float32) = NVFP4 product of the bf16 operands (e2m1 codes, e4m3 block scales, float row scales)."""
+    import torch
+    rows, k = x.shape
+    n = w.shape[0]
+    y = torch.empty(rows, n, dtype=torch.float32, device=x.device)
+    nb = lib().wd_op_gemm_fp4_scratch_bytes(rows, n, k)
+    scratch = torch.empty(max(nb, 256), dtype=torch.uint8, device=x.device)
+    check(lib().wd_op_gemm_fp4(_ptr(x), _ptr(w), _ptr(y), rows, n, k, _ptr(scratch), nb, _stream_ptr(stream)), "wd_op_gemm_fp4")
     return y
 
 

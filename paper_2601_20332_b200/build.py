@@ -8,7 +8,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libwd.so")
-SOURCES = ["api.cu", "planner.cpp", "kernels_plain.cu", "gemm_tc.cu", "gemm_ck.cu", "attention_tc.cu"]
+SOURCES = ["api.cu", "planner.cpp", "kernels_plain.cu", "gemm_tc.cu", "gemm_ck.cu", "gemm_fp4.cu", "attention_tc.cu"]
 
 
 def _nvcc() -> str:

@@ -1888,6 +1888,12 @@ wd_status wd_tc_chain(const WdTcChainItem* items, int n, int rows, float* y, siz
     return WD_OK;
 }
 
+void wd_launch_reduce_slices(const float* part, int n_split, size_t stride, float* y, size_t total, cudaStream_t st) {
+    const int blocks = (int)((total + 255) / 256 < 1184 ? (total + 255) / 256 : 1184);
+    ++wd_launch_counter;
+    reduce_slices_kernel<<<blocks, 256, 0, st>>>(part, n_split, stride, y, total);
+}
+
 wd_status wd_tc_encode_fp8(CUtensorMap* m, const void* ptr, int n_rows, int K, int box_rows) {
     return encode_2d8(m, ptr, n_rows, K, box_rows);
 }

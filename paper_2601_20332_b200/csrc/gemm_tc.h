@@ -147,3 +147,23 @@ wd_status wd_tc_gemm_standalone(const void* x, const void* w, float* y, int rows
                                 size_t scratch_bytes, cudaStream_t stream);
 wd_status wd_tc_gemm_standalone_fp8(const uint8_t* xq, const float* sx, const uint8_t* wq, const float* sw, float* y,
                                     int rows, int n_out, int k_in, float* slices, size_t slice_floats, cudaStream_t stream);
+
+// ---- NVFP4 (gemm_fp4.cu): e2m1 codes packed two per byte, one unsigned e4m3 scale per 16 elements along K,
+// one float scale per row
+struct WdFp4Operand {
+    uint8_t* codes = nullptr;    // [n_rows][K / 2]
+    uint8_t* sf = nullptr;       // [n_rows][K / 16]
+    float* g = nullptr;          // [n_rows]
+    int n_rows = 0, K = 0;
+};
+size_t wd_fp4_operand_bytes(int n_rows, int K);                       // device bytes of one quantised operand
+void wd_fp4_operand_split(void* mem, int n_rows, int K, WdFp4Operand* op);
+// quantises a [n_rows, K] matrix of `dtype` (taken as bfloat16), K a multiple of 16
+void wd_launch_quantize_nvfp4(int dtype, const void* x, int n_rows, int K, const WdFp4Operand* op, cudaStream_t st);
+// y[split][rows][n] = x * w^T on the block-scaled tensor-core path (K a multiple of 256); K slices side by side.
+// w_static: the weights were quantised before the previous kernel on the stream started, so the kernel may
+// fetch them ahead of its dependency wait.
+wd_status wd_fp4_gemm(const WdFp4Operand* x, const WdFp4Operand* w, float* y, size_t y_floats, int sm_count, int32_t* status,
+                      cudaStream_t stream, int* n_split_out, bool force_single_split, bool w_static);
+// adds the K slices of a GEMM result: y[i] = sum_s part[s * stride + i]
+void wd_launch_reduce_slices(const float* part, int n_split, size_t stride, float* y, size_t total, cudaStream_t st);

@@ -65,6 +65,24 @@ def test_gemm_fp8_vs_oracle(rows, n, k):
     assert 5e-3 < np.linalg.norm(got - exact) / np.linalg.norm(exact) < 8e-2      # it really is an 8-bit product
 
 
+@pytest.mark.parametrize("rows,n,k", [(1, 128, 256), (34, 384, 1024), (35, 640, 4096), (130, 200, 512), (300, 256, 1024),
+                                      (700, 384, 768), (34, 1000, 256), (48, 12288, 4096)])
+def test_gemm_nvfp4_vs_oracle(rows, n, k):
+    """Identical bf16 inputs on both sides, so the e2m1 codes, the e4m3 block scales and the row scales agree
+    exactly (both sides take every rounding decision in float32) and only the fp32 accumulation differs from
+    the oracle's float64 sum over the blocks."""
+    g = torch.Generator(device=DEV).manual_seed(rows * 1000 + n + k)
+    x = torch.randn(rows, k, device=DEV, generator=g).to(torch.bfloat16)
+    w = (torch.randn(n, k, device=DEV, generator=g) * 0.05).to(torch.bfloat16)
+    y = wd.op_gemm_fp4(x, w)
+    assert wd.op_status() == 0
+    ref = wo.nvfp4_matmul(x.float().cpu().numpy().astype(np.float64), w.float().cpu().numpy().astype(np.float64))
+    got = y.cpu().numpy().astype(np.float64)
+    assert np.abs(got - ref).max() <= 2e-5 * np.abs(ref).max()
+    exact = x.double().cpu().numpy() @ w.double().cpu().numpy().T
+    assert 3e-2 < np.linalg.norm(got - exact) / np.linalg.norm(exact) < 0.25        # it really is a 4-bit product
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("rows,n,k", [(1, 5, 3), (10, 70, 33), (34, 384, 256), (97, 130, 1000)])
 def test_gemm_plain_vs_oracle(dtype, rows, n, k):

@@ -533,3 +533,63 @@ def test_bf16_points_mode_rounds_the_stored_activations_and_nothing_else():
                            caches_for(cfg, model, 2), cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"])
     np.testing.assert_array_equal(mixed[0]["logits"], a["logits"])
     np.testing.assert_array_equal(mixed[1]["logits"], b["logits"])
+
+
+# ---------------------------------------------------------------- NVFP4 mode (option outside the paper)
+
+def test_e2m1_rounding_against_the_format_definition():
+    """e2m1 = sign, 2 exponent bits (bias 1), 1 mantissa bit; exponent 0 is subnormal (0 or 0.5)."""
+    vals = []
+    for e in range(4):
+        for m in range(2):
+            vals.append((m / 2.0) if e == 0 else (1.0 + m / 2.0) * 2.0 ** (e - 1))
+    assert vals == wo.E2M1_GRID.tolist() == [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]
+    np.testing.assert_array_equal(wo.e2m1_round(np.array(vals + [-v for v in vals], np.float32)), vals + [-v for v in vals])
+    rng = np.random.default_rng(7)
+    x = np.concatenate([rng.uniform(-8, 8, 4000), rng.normal(0, 1, 2000)]).astype(np.float32)
+    got = wo.e2m1_round(x)
+    for v, g in zip(x.astype(np.float64), got):
+        d = np.abs(wo.E2M1_GRID - abs(v))
+        best = np.flatnonzero(d == d.min())
+        assert abs(g) == wo.E2M1_GRID[best[0]] if len(best) == 1 else abs(g) in wo.E2M1_GRID[best]
+        assert g == 0 or np.sign(g) == np.sign(v)
+    # exact midpoints go to the even code: codes 0..7 = 0, .5, 1, 1.5, 2, 3, 4, 6
+    np.testing.assert_array_equal(wo.e2m1_round(np.array([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, -2.5, 100.0], np.float32)),
+                                  [0.0, 1.0, 1.0, 2.0, 2.0, 4.0, 4.0, -2.0, 6.0])
+
+
+def test_nvfp4_row_quantisation_and_product():
+    rng = np.random.default_rng(8)
+    x = rng.normal(0, 2, (5, 64))
+    q, s, g = wo.nvfp4_quant_rows(x)
+    assert q.shape == (5, 64) and s.shape == (5, 4) and g.dtype == np.float32
+    assert set(np.abs(q).ravel().tolist()) <= set(wo.E2M1_GRID.tolist())
+    np.testing.assert_array_equal(wo.e4m3_round(s.astype(np.float32)), s)               # block scales sit on the e4m3 grid
+    assert s.max() <= 448.0 and (s.max(axis=1) >= 416.0).all()                          # the largest block of a row uses the top of it
+    xb = wo.bf16_round(x)
+    rec = q * np.repeat(s, 16, axis=1) * g.astype(np.float64)[:, None]
+    # a block's elements are within half an e2m1 spacing (at most 1 of 6) of the block maximum's scale
+    bmax = np.abs(xb).reshape(5, 4, 16).max(axis=2)
+    assert (np.abs(rec - xb).reshape(5, 4, 16).max(axis=2) <= bmax * (1.0 / 6.0) * 1.07 + 1e-12).all()
+    zq, zs, zg = wo.nvfp4_quant_rows(np.zeros((2, 32)))
+    assert (zq == 0).all() and (zs == 0).all() and (zg == 1).all()
+    # operands that already are NVFP4 numbers multiply exactly: grid values, one block scale, row maximum 6 * 448 * 2^-9
+    a = rng.choice(wo.E2M1_GRID, size=(3, 32)) * rng.choice([-1.0, 1.0], size=(3, 32)); a[:, 0] = 6.0; a[:, 16] = 6.0
+    b = rng.choice(wo.E2M1_GRID, size=(4, 32)) * rng.choice([-1.0, 1.0], size=(4, 32)); b[:, 0] = 6.0; b[:, 16] = 6.0
+    np.testing.assert_allclose(wo.nvfp4_matmul(a * 448 * 2.0 ** -9, b * 448 * 2.0 ** -6), (a @ b.T) * 448 * 448 * 2.0 ** -15, rtol=1e-6)
+    # and a random product stays within the format's precision of the exact one
+    w = rng.normal(0, 0.02, (16, 256)); xx = rng.normal(0, 1, (7, 256))
+    err = np.linalg.norm(wo.nvfp4_matmul(xx, w) - xx @ w.T) / np.linalg.norm(xx @ w.T)
+    assert 2e-2 < err < 0.25
+
+
+def test_nvfp4_mode_changes_only_the_quantised_projections():
+    cfg = small_cfg(G=12)
+    model = make(cfg)
+    base, _, _ = run_traj(cfg, model, 2)
+    model.dims = dict(model.dims, nvfp4=True)
+    f4, _, _ = run_traj(cfg, model, 2)
+    a, b = base[0][0], f4[0][0]
+    assert a["plan"] == b["plan"]
+    rel = np.linalg.norm(a["logits"] - b["logits"]) / np.linalg.norm(a["logits"])
+    assert 1e-3 < rel < 0.6 and np.isfinite(b["logits"]).all()
