@@ -285,6 +285,22 @@ def run_ours(args, rank, world):
                     "normal_step_ms": float(np.median(f_normal)) if f_normal else None,
                     "refresh_step_ms": float(np.median(f_refresh)) if f_refresh else None}
         ctx.fp8_set(False)
+    # ---- NVFP4 projections (outside the paper too; 4-bit codes with block scales on the block-scaled tensor-core path)
+    fp4_line = None
+    if cfg["dtype"] == "bf16" and cfg["d"] % 256 == 0 and cfg["F"] % 256 == 0:
+        ctx.fp4_enable(stream)
+        state.reset(ids, None, stream)
+        q_infos, q_per_step, q_total_ms, _ = trajectory(W, K, state, queued=True)
+        q_total_ms = max_over_ranks(q_total_ms, world, dev)
+        q_normal = [t for t, i in zip(q_per_step, q_infos) if not i["is_refresh"]]
+        q_refresh = [t for t, i in zip(q_per_step, q_infos) if i["is_refresh"]]
+        fp4_line = {"note": "NOT the headline precision: NVFP4 (e2m1 codes, e4m3 scale per 16 elements, float scale per row) "
+                            "weights and activations for q/k/v, gate/up, down and the LM head (fp32 accumulation); "
+                            "everything else as in the bf16 run",
+                    "value": whole_job_value(batch * k * K, world, q_total_ms), "unit": UNIT,
+                    "normal_step_ms": float(np.median(q_normal)) if q_normal else None,
+                    "refresh_step_ms": float(np.median(q_refresh)) if q_refresh else None}
+        ctx.fp4_set(False)
     # ---- a whole generation through the library's own driver: host prompt in, host tokens out
     torch.cuda.synchronize()
     t0 = time.perf_counter()
@@ -337,6 +353,7 @@ def run_ours(args, rank, world):
                    "stepping": "queued: steps enqueued back to back, index lists planned on the device, drained every 16 steps",
                    "gemm_impl": infos[-1]["gemm_impl"],
                    "variant_fp8_projections": fp8_line,
+                   "variant_nvfp4_projections": fp4_line,
                    "variant_window_only_refresh": {
                        "note": "NOT the paper's refresh: after the first step a refresh recomputes only the new window "
                                "and the previous phase's tokens (an approximation beyond one block); same steps otherwise",

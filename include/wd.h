@@ -334,6 +334,23 @@ WD_API size_t wd_fp8_bytes(const wd_model_dims* dims);
 WD_API wd_status wd_fp8_enable(wd_ctx* ctx, void* mem, size_t mem_bytes, void* stream /*cudaStream_t*/);
 WD_API wd_status wd_fp8_set(wd_ctx* ctx, int32_t on);
 
+/* NVFP4 mode (outside the paper, which calls quantisation orthogonal to its method; bf16 models with
+ * d_model and d_ffn multiples of 256).  The same projections as in the FP8 mode (q/k/v, gate/up, down and
+ * the LM head; the attention output projection stays bf16) take both operands in the NVFP4 format:
+ * 4-bit e2m1 elements, one unsigned e4m3 scale per block of 16 elements along the inner dimension,
+ * one float scale per row (row maximum / (6 * 448)).  Every weight row is quantised once
+ * (wd_fp4_enable), every activation row (the bf16 output of the RMSNorm / SwiGLU kernels) at every
+ * step; the product runs on the block-scaled tensor-core path with fp32 accumulation.  The two quantised
+ * modes exclude each other: enabling one switches the other off.
+ *   wd_fp4_bytes   size of the device memory block wd_fp4_enable needs (0 for invalid dims)
+ *   wd_fp4_enable  quantises the weights on `stream` into `mem` (caller-owned, 256-byte aligned, must
+ *                  outlive the context's use of the mode) and switches the mode on
+ *   wd_fp4_set     switches the mode off / on again (on needs a prior wd_fp4_enable).
+ * Errors: WD_ERR_NULL, WD_ERR_BAD_PARAM (dtype or widths), WD_ERR_MISALIGNED, WD_ERR_WORKSPACE_TOO_SMALL. */
+WD_API size_t wd_fp4_bytes(const wd_model_dims* dims);
+WD_API wd_status wd_fp4_enable(wd_ctx* ctx, void* mem, size_t mem_bytes, void* stream /*cudaStream_t*/);
+WD_API wd_status wd_fp4_set(wd_ctx* ctx, int32_t on);
+
 /* ---- the step ----------------------------------------------------------- */
 
 /* Preview of the index sets the next wd_step(st, A, B, R, T, ...) will use for

@@ -87,6 +87,9 @@ SIGNATURES = {
     "wd_fp8_bytes": (C.c_size_t, [C.POINTER(wd_model_dims)]),
     "wd_fp8_enable": (C.c_int, [vp, vp, C.c_size_t, vp]),
     "wd_fp8_set": (C.c_int, [vp, i32]),
+    "wd_fp4_bytes": (C.c_size_t, [C.POINTER(wd_model_dims)]),
+    "wd_fp4_enable": (C.c_int, [vp, vp, C.c_size_t, vp]),
+    "wd_fp4_set": (C.c_int, [vp, i32]),
     "wd_state_set_eos": (C.c_int, [vp, i32]),
     "wd_state_set_refresh_mode": (C.c_int, [vp, i32]),
     "wd_state_set_stagger": (C.c_int, [vp, i32]),
@@ -241,6 +244,18 @@ class Context:
 
     def fp8_set(self, on: bool):
         check(lib().wd_fp8_set(self.handle, 1 if on else 0), "wd_fp8_set")
+
+    def fp4_enable(self, stream=None):
+        """wd_fp4_enable: quantise the weights to NVFP4 and run the projections in NVFP4 from now on."""
+        import torch
+        nbytes = lib().wd_fp4_bytes(C.byref(self.dims))
+        if nbytes == 0:
+            raise WdError(WD_ERR_BAD_PARAM, "wd_fp4_bytes")
+        self._fp4_mem = torch.empty(nbytes, dtype=torch.uint8, device=self.workspace.device)
+        check(lib().wd_fp4_enable(self.handle, _ptr(self._fp4_mem), nbytes, _stream_ptr(stream)), "wd_fp4_enable")
+
+    def fp4_set(self, on: bool):
+        check(lib().wd_fp4_set(self.handle, 1 if on else 0), "wd_fp4_set")
 
     def profile_read(self) -> dict:
         ms, by, n = C.c_double(), C.c_double(), C.c_int64()

@@ -101,6 +101,12 @@ struct wd_ctx {
     float* sxn = nullptr;        // [max_rows]
     float* sh = nullptr;         // [max_rows]
     WdTcX x8_d, x8_h;
+    // NVFP4 mode (wd_fp4_enable): the same projections with e2m1 codes, e4m3 block scales and float row scales;
+    // q/k/v and gate/up are one operand each (their rows one after the other)
+    bool fp4_ready = false, fp4_on = false;
+    std::vector<WdFp4Operand> f4qkv, f4gu, f4d;
+    WdFp4Operand f4lm;
+    void* fp4_x = nullptr;       // the step's quantised activations: max_rows x max(d, d_ffn)
 
     // optional GEMM timing (benchmarks): event pairs around every GEMM launch of a step
     bool prof_on = false;
@@ -351,6 +357,7 @@ extern "C" wd_status wd_fp8_enable(wd_ctx* c, void* mem, size_t mem_bytes, void*
     WD_CUDA_TRY(cudaGetLastError());
     c->fp8_ready = true;
     c->fp8_on = true;
+    c->fp4_on = false;
     return WD_OK;
 }
 
@@ -358,6 +365,82 @@ extern "C" wd_status wd_fp8_set(wd_ctx* c, int32_t on) {
     if (!c) return WD_ERR_NULL;
     if (on && !c->fp8_ready) return WD_ERR_BAD_PARAM;
     c->fp8_on = on != 0;
+    if (on) c->fp4_on = false;
+    return WD_OK;
+}
+
+// ---------------------------------------------------------------------------
+// NVFP4 mode
+// ---------------------------------------------------------------------------
+static size_t fp4_carve(const wd_model_dims* d, size_t* off /*[6]*/) {
+    const int hq = d->n_q_heads * d->head_dim, hkv = d->n_kv_heads * d->head_dim;
+    const int D = d->d_model, F = d->d_ffn;
+    const size_t L = d->n_layers;
+    size_t o = 0;
+    auto take = [&](size_t bytes) { const size_t at = o; o = wd_align_up(o + bytes, 256); return at; };
+    off[0] = take(L * wd_fp4_operand_bytes(hq + 2 * hkv, D));
+    off[1] = take(L * wd_fp4_operand_bytes(2 * F, D));
+    off[2] = take(L * wd_fp4_operand_bytes(D, F));
+    off[3] = take(wd_fp4_operand_bytes(d->vocab, D));
+    off[4] = take(wd_fp4_operand_bytes(d->max_rows, std::max(D, F)));
+    return o;
+}
+
+static bool fp4_dims_ok(const wd_model_dims* d) {
+    return d->dtype == WD_BF16 && d->d_model % 256 == 0 && d->d_ffn % 256 == 0;
+}
+
+extern "C" size_t wd_fp4_bytes(const wd_model_dims* dims) {
+    if (!dims_valid(dims) || !fp4_dims_ok(dims)) return 0;
+    size_t off[6];
+    return fp4_carve(dims, off);
+}
+
+extern "C" wd_status wd_fp4_enable(wd_ctx* c, void* mem, size_t mem_bytes, void* stream_) {
+    if (!c || !mem) return WD_ERR_NULL;
+    const wd_model_dims& d = c->d;
+    if (!fp4_dims_ok(&d)) return WD_ERR_BAD_PARAM;
+    if ((uintptr_t)mem % 256) return WD_ERR_MISALIGNED;
+    size_t off[6];
+    if (mem_bytes < fp4_carve(&d, off)) return WD_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    const int hq = d.n_q_heads * d.head_dim, hkv = d.n_kv_heads * d.head_dim, D = d.d_model, F = d.d_ffn, L = d.n_layers;
+    // rows [r0, r0 + n) of an operand, quantised from one weight matrix
+    auto quant = [&](const void* w, const WdFp4Operand& op, int r0, int n) {
+        WdFp4Operand sub = op;
+        sub.codes += (size_t)r0 * (op.K / 2);
+        sub.sf += (size_t)r0 * (op.K / 16);
+        sub.g += r0;
+        sub.n_rows = n;
+        wd_launch_quantize_nvfp4(WD_BF16, w, n, op.K, &sub, stream);
+    };
+    c->f4qkv.assign(L, {}); c->f4gu.assign(L, {}); c->f4d.assign(L, {});
+    for (int l = 0; l < L; ++l) {
+        wd_fp4_operand_split((char*)mem + off[0] + (size_t)l * wd_fp4_operand_bytes(hq + 2 * hkv, D), hq + 2 * hkv, D, &c->f4qkv[l]);
+        quant(c->wq[l], c->f4qkv[l], 0, hq);
+        quant(c->wk[l], c->f4qkv[l], hq, hkv);
+        quant(c->wv[l], c->f4qkv[l], hq + hkv, hkv);
+        wd_fp4_operand_split((char*)mem + off[1] + (size_t)l * wd_fp4_operand_bytes(2 * F, D), 2 * F, D, &c->f4gu[l]);
+        quant(c->wg[l], c->f4gu[l], 0, F);
+        quant(c->wu[l], c->f4gu[l], F, F);
+        wd_fp4_operand_split((char*)mem + off[2] + (size_t)l * wd_fp4_operand_bytes(D, F), D, F, &c->f4d[l]);
+        quant(c->wd[l], c->f4d[l], 0, D);
+    }
+    wd_fp4_operand_split((char*)mem + off[3], d.vocab, D, &c->f4lm);
+    quant(c->lm_head, c->f4lm, 0, d.vocab);
+    c->fp4_x = (char*)mem + off[4];
+    WD_CUDA_TRY(cudaGetLastError());
+    c->fp4_ready = true;
+    c->fp4_on = true;
+    c->fp8_on = false;
+    return WD_OK;
+}
+
+extern "C" wd_status wd_fp4_set(wd_ctx* c, int32_t on) {
+    if (!c) return WD_ERR_NULL;
+    if (on && !c->fp4_ready) return WD_ERR_BAD_PARAM;
+    c->fp4_on = on != 0;
+    if (on) c->fp8_on = false;
     return WD_OK;
 }
 
@@ -886,6 +969,33 @@ static wd_status run_gemm(wd_ctx* c, const void* x, const WdTcX* x_map, const Wd
     return WD_OK;
 }
 
+// NVFP4 projection of the step: the step's quantised activations (left in ctx->fp4_x by the RMSNorm / SwiGLU
+// kernel before it) times the quantised weights; K slices side by side in y like the bf16 kernel's.
+static wd_status run_gemm_fp4(wd_ctx* c, const WdFp4Operand* w, int rows, int K, float* y, size_t y_floats,
+                              int32_t* status, cudaStream_t stream, GemmOut* go, bool single_split = false) {
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (c->prof_on) {
+        while (c->prof_events.size() < c->prof_used + 2) {
+            cudaEvent_t e;
+            WD_CUDA_TRY(cudaEventCreate(&e));
+            c->prof_events.push_back(e);
+        }
+        e0 = c->prof_events[c->prof_used++];
+        e1 = c->prof_events[c->prof_used++];
+        // algorithmic bytes: codes + block scales of the weights once and of the activations, result out
+        c->prof_step_bytes += (double)(w->n_rows + rows) * K * (0.5 + 1.0 / 16) + (double)rows * w->n_rows * 4;
+        WD_CUDA_TRY(cudaEventRecord(e0, stream));
+    }
+    WdFp4Operand ox;
+    wd_fp4_operand_split(c->fp4_x, rows, K, &ox);
+    int ns = 1;
+    wd_status s = wd_fp4_gemm(&ox, w, y, y_floats, c->sm_count, status, stream, &ns, single_split, /*w_static=*/true);
+    if (s != WD_OK) return s;
+    *go = {ns, (size_t)rows * w->n_rows, 1, WD_GEMM_TCGEN05};
+    if (e1) WD_CUDA_TRY(cudaEventRecord(e1, stream));
+    return WD_OK;
+}
+
 // ---------------------------------------------------------------------------
 // wd_step
 // ---------------------------------------------------------------------------
@@ -1064,7 +1174,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     // Where the consumers of the GEMMs run (wd_set_fusion).  The fused forms need the tensor-core path,
     // head_dim 128 and widths that are multiples of 128; a mode that cannot serve the step's row count
     // falls back to the separate kernels.  The FP8 mode keeps its separate kernels.
-    const bool fusable = use_tc(c) && dh == 128 && D % 128 == 0 && F % 128 == 0 && !c->fp8_on;
+    const bool fusable = use_tc(c) && dh == 128 && D % 128 == 0 && F % 128 == 0 && !c->fp8_on && !c->fp4_on;
     int fuse_mode = fusable ? c->fuse : WD_FUSION_NONE;
     if (fuse_mode == WD_FUSION_AUTO) fuse_mode = WD_FUSION_NONE;
     if (fuse_mode == WD_FUSION_CLUSTER && !(R_ <= wd_ck_max_rows() && D >= 256 && F >= 256 && hq >= 256)) fuse_mode = WD_FUSION_NONE;
@@ -1077,6 +1187,13 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         c->chain_dirty = false;
     }
     const bool fp8 = c->fp8_on && use_tc(c) && !fused;      // FP8 projections (q/k/v, gate/up, down, LM head)
+    const bool fp4 = c->fp4_on && use_tc(c) && !fused;      // NVFP4 projections (the same ones)
+    WdFp4Operand x4_d, x4_f, x4_lm;                         // the step's quantised activations, by use
+    if (fp4) {
+        wd_fp4_operand_split(c->fp4_x, R_, D, &x4_d);
+        wd_fp4_operand_split(c->fp4_x, R_, F, &x4_f);
+        wd_fp4_operand_split(c->fp4_x, NA, D, &x4_lm);
+    }
     auto attention = [&](int l, char* kc, char* vc) -> wd_status {
         float* attn_tap = st->taps.attn_out ? st->taps.attn_out + (size_t)l * R_ * hq : nullptr;
         if (st->attn_tc && all_contig && c->attn_impl != WD_GEMM_PLAIN)
@@ -1176,9 +1293,12 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         char* vc = st->vcache + (size_t)l * st->v_layer_bytes;
         // attention half (FP8 mode: the normalised rows leave the RMSNorm as e4m3 codes + row scales)
         wd_launch_rmsnorm(d.dtype, c->x, down_pending ? c->part : nullptr, down_go.n_split, down_go.split_stride,
-                          c->attn_norm[l], d.rms_eps, c->xn, nullptr, R_, D, stream, fp8 ? c->xn8 : nullptr, c->sxn);
+                          c->attn_norm[l], d.rms_eps, c->xn, nullptr, R_, D, stream, fp8 ? c->xn8 : nullptr, c->sxn,
+                          fp4 ? &x4_d : nullptr);
         down_pending = false;
-        if (fp8) {
+        if (fp4) {
+            if ((s = run_gemm_fp4(c, &c->f4qkv[l], R_, D, c->part, c->part_floats, status, stream, &go)) != WD_OK) return s;
+        } else if (fp8) {
             WdTcSeg qkv[3] = {{c->f8q[l].q, hq, &c->f8q[l].map}, {c->f8k[l].q, hkv, &c->f8k[l].map},
                               {c->f8v[l].q, hkv, &c->f8v[l].map}};
             WdTcFp8 f8;
@@ -1201,8 +1321,12 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
             return s;
         // feed-forward half
         wd_launch_rmsnorm(d.dtype, c->x, c->part, go.n_split, go.split_stride, c->ffn_norm[l], d.rms_eps, c->xn,
-                          nullptr, R_, D, stream, fp8 ? c->xn8 : nullptr, c->sxn);
-        if (fp8) {
+                          nullptr, R_, D, stream, fp8 ? c->xn8 : nullptr, c->sxn, fp4 ? &x4_d : nullptr);
+        if (fp4) {
+            if ((s = run_gemm_fp4(c, &c->f4gu[l], R_, D, c->part, c->part_floats, status, stream, &go)) != WD_OK) return s;
+            if ((s = wd_launch_swiglu_fp4(c->part, go.n_split, go.split_stride, &x4_f, R_, F, stream)) != WD_OK) return s;
+            if ((s = run_gemm_fp4(c, &c->f4d[l], R_, F, c->part, c->part_floats, status, stream, &go)) != WD_OK) return s;
+        } else if (fp8) {
             WdTcSeg gu[2] = {{c->f8g[l].q, F, &c->f8g[l].map}, {c->f8u[l].q, F, &c->f8u[l].map}};
             WdTcFp8 f8;
             f8.sw[0] = c->f8g[l].s; f8.sw[1] = c->f8u[l].s; f8.sx = c->sxn;
@@ -1242,7 +1366,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     int lm_chunks = wd_unmask_chunks(d.vocab);
     if (NA > 0) {
         wd_launch_rmsnorm(d.dtype, c->x, nullptr, 0, 0, c->final_norm, d.rms_eps, c->xn, act_row, NA, D, stream,
-                          fp8 ? c->xn8 : nullptr, c->sxn);
+                          fp8 ? c->xn8 : nullptr, c->sxn, fp4 ? &x4_lm : nullptr);
         WdTcSeg lm[1] = {{c->lm_head, d.vocab, c->tc.get(WD_TC_LM, 0)}};
         WdTcFp8 f8lm;
         if (fp8) {
@@ -1255,8 +1379,12 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         fl.mode = WD_FUSE_LMSTATS;
         fl.st_max = c->ch_max; fl.st_idx = c->ch_idx; fl.st_sum = c->ch_sum;
         fl.write_logits = st->taps.logits ? 1 : 0;
-        lm_fused = use_tc(c) && NA <= 1024 && c->sm_count % 4 == 0;     // one CTA group per tile of <= 256 active rows
-        if ((s = run_gemm(c, fp8 ? (const void*)c->xn8 : c->xn, fp8 ? &c->x8_d : &c->tc.x_map_d, lm, 1, NA, D, c->logits,
+        lm_fused = use_tc(c) && NA <= 1024 && c->sm_count % 4 == 0 && !fp4;     // one CTA group per tile of <= 256 active rows
+        if (fp4) {
+            if ((s = run_gemm_fp4(c, &c->f4lm, NA, D, c->logits, (size_t)d.max_active * d.vocab, status, stream, &go,
+                                  /*single_split=*/true)) != WD_OK)
+                return s;
+        } else if ((s = run_gemm(c, fp8 ? (const void*)c->xn8 : c->xn, fp8 ? &c->x8_d : &c->tc.x_map_d, lm, 1, NA, D, c->logits,
                           (size_t)d.max_active * d.vocab, status, stream, &go, /*single_split=*/true,
                           lm_fused ? &fl : nullptr, fp8 ? &f8lm : nullptr)) != WD_OK)
             return s;

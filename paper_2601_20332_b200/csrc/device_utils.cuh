@@ -5,6 +5,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <cuda_fp8.h>
+
 namespace wdk {
 
 constexpr uint32_t kWaitLimit = 1u << 22;   // polls of one bounded wait before it gives up, whatever the clock says
@@ -269,5 +271,49 @@ __device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap* map
         ::"r"(dst), "l"(map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
         : "memory");
 }
+
+// ---- NVFP4 element formats
+// value of an e4m3 code (no infinities; the NaN code does not occur: the conversion saturates)
+__device__ __forceinline__ float e4m3_value(uint32_t code) {
+    const uint32_t e = (code >> 3) & 15u, m = code & 7u;
+    const float mag = e == 0 ? (float)m * 0.001953125f /* 2^-9 */ : __uint_as_float(((e + 120u) << 23) | (m << 20));
+    return (code & 0x80u) ? -mag : mag;
+}
+
+// e2m1 code of v: nearest of 0, .5, 1, 1.5, 2, 3, 4, 6 (ties to the even code, saturating), sign in bit 3
+__device__ __forceinline__ uint32_t e2m1_code(float v) {
+    const float a = fabsf(v);
+    uint32_t c = 0;
+    c = (a > 0.25f) ? 1u : c;
+    c = (a >= 0.75f) ? 2u : c;
+    c = (a > 1.25f) ? 3u : c;
+    c = (a >= 1.75f) ? 4u : c;
+    c = (a > 2.5f) ? 5u : c;
+    c = (a >= 3.5f) ? 6u : c;
+    c = (a > 5.0f) ? 7u : c;
+    return c | ((__float_as_uint(v) >> 31) << 3);
+}
+
+// The NVFP4 codes of four consecutive elements held by one thread, where four neighbouring lanes hold one block
+// of 16 (every lane of the warp calls; lanes past the row pass zeros and store == false): block maximum by two
+// shuffles, block scale s = e4m3((max / 6) / g), codes e2m1(v / (s g)); two bytes of codes per thread, the scale byte
+// from the first lane of the four.  c4 = index of the thread's float4 within the row.
+__device__ __forceinline__ void nvfp4_emit4(float4 v, float g, bool store, uint8_t* codes_row, uint8_t* sf_row, int c4) {
+    float bmax = fmaxf(fmaxf(fabsf(v.x), fabsf(v.y)), fmaxf(fabsf(v.z), fabsf(v.w)));
+    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 1));
+    bmax = fmaxf(bmax, __shfl_xor_sync(0xffffffffu, bmax, 2));
+    const uint32_t sc = (uint32_t)__nv_cvt_float_to_fp8(__fdiv_rn(__fdiv_rn(bmax, 6.0f), g), __NV_SATFINITE, __NV_E4M3);
+    const float d = __fmul_rn(e4m3_value(sc), g);
+    uint32_t c = 0;
+    if (d > 0.f)
+        c = e2m1_code(__fdiv_rn(v.x, d)) | (e2m1_code(__fdiv_rn(v.y, d)) << 4) | (e2m1_code(__fdiv_rn(v.z, d)) << 8) |
+            (e2m1_code(__fdiv_rn(v.w, d)) << 12);
+    if (store) {
+        *reinterpret_cast<uint16_t*>(codes_row + 2 * c4) = (uint16_t)c;
+        if ((c4 & 3) == 0) sf_row[c4 >> 2] = (uint8_t)sc;
+    }
+}
+
+__device__ __forceinline__ float bf16_round_f(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
 }  // namespace wdk

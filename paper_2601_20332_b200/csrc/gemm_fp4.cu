@@ -293,27 +293,6 @@ gemm_fp4_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant
 }
 
 // ---------------------------------------------------------------- quantisation
-// value of an e4m3 code (no infinities; the NaN code does not occur: the conversion saturates)
-__device__ __forceinline__ float e4m3_value(uint32_t code) {
-    const uint32_t e = (code >> 3) & 15u, m = code & 7u;
-    const float mag = e == 0 ? (float)m * 0.001953125f /* 2^-9 */ : __uint_as_float(((e + 120u) << 23) | (m << 20));
-    return (code & 0x80u) ? -mag : mag;
-}
-
-// e2m1 code of v: nearest of 0, .5, 1, 1.5, 2, 3, 4, 6 (ties to the even code, saturating), sign in bit 3
-__device__ __forceinline__ uint32_t e2m1_code(float v) {
-    const float a = fabsf(v);
-    uint32_t c = 0;
-    c = (a > 0.25f) ? 1u : c;
-    c = (a >= 0.75f) ? 2u : c;
-    c = (a > 1.25f) ? 3u : c;
-    c = (a >= 1.75f) ? 4u : c;
-    c = (a > 2.5f) ? 5u : c;
-    c = (a >= 3.5f) ? 6u : c;
-    c = (a > 5.0f) ? 7u : c;
-    return c | ((__float_as_uint(v) >> 31) << 3);
-}
-
 template <typename T> __device__ __forceinline__ float ldf(const T* p);
 template <> __device__ __forceinline__ float ldf<float>(const float* p) { return __bfloat162float(__float2bfloat16_rn(*p)); }
 template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
@@ -440,13 +419,19 @@ wd_status wd_fp4_gemm(const WdFp4Operand* x, const WdFp4Operand* w, float* y, si
     const size_t slice = (size_t)rows * n_out;
     if (slice > y_floats) return WD_ERR_CAPACITY;
     // K slices while (weight tile, token tile) pairs alone would leave SMs idle and the partial sums fit
+    // K slices: the split count that minimises (waves of units over the SMs) x (stages per unit) x (time one SM
+    // needs to take in a stage, about 63 GB/s whatever the source) + the write and re-read of one more partial
+    // result per slice at HBM speed
     int ns = 1;
     if (!force_single_split) {
-        ns = sm_count / (p.n_tiles * p.tok_tiles);
-        if (ns > WD_TC_MAX_SPLIT) ns = WD_TC_MAX_SPLIT;
-        if (ns > p.kb_total) ns = p.kb_total;
-        while (ns > 1 && (size_t)ns * slice > y_floats) --ns;
-        if (ns < 1) ns = 1;
+        const double t_stage = (double)(kStageW + p.bn * 128 + kSfW + p.bn * 16) / 63e9;
+        const double t_slice = (double)slice * 8.0 / 6.5e12;
+        double best = 1e30;
+        for (int c = 1; c <= WD_TC_MAX_SPLIT && c <= p.kb_total && (size_t)c * slice <= y_floats; ++c) {
+            const int units = p.n_tiles * p.tok_tiles * c;
+            const double t = (double)((units + sm_count - 1) / sm_count) * ((p.kb_total + c - 1) / c) * t_stage + c * t_slice;
+            if (t < best * 0.999) { best = t; ns = c; }
+        }
     }
     p.n_slices = ns;
     p.n_units = p.n_tiles * p.tok_tiles * ns;

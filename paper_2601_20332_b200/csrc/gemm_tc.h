@@ -150,12 +150,6 @@ wd_status wd_tc_gemm_standalone_fp8(const uint8_t* xq, const float* sx, const ui
 
 // ---- NVFP4 (gemm_fp4.cu): e2m1 codes packed two per byte, one unsigned e4m3 scale per 16 elements along K,
 // one float scale per row
-struct WdFp4Operand {
-    uint8_t* codes = nullptr;    // [n_rows][K / 2]
-    uint8_t* sf = nullptr;       // [n_rows][K / 16]
-    float* g = nullptr;          // [n_rows]
-    int n_rows = 0, K = 0;
-};
 size_t wd_fp4_operand_bytes(int n_rows, int K);                       // device bytes of one quantised operand
 void wd_fp4_operand_split(void* mem, int n_rows, int K, WdFp4Operand* op);
 // quantises a [n_rows, K] matrix of `dtype` (taken as bfloat16), K a multiple of 16

@@ -349,7 +349,7 @@ template <typename T, int MAXV>
 __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
                                size_t split_stride, const float* __restrict__ gain, float eps,
                                T* __restrict__ xn, const int32_t* __restrict__ row_idx, int d,
-                               uint8_t* __restrict__ xq, float* __restrict__ sx) {
+                               uint8_t* __restrict__ xq, float* __restrict__ sx, WdFp4Operand x4) {
     __shared__ float red[32];
     pdl_launch_dependents();
     pdl_wait();
@@ -401,6 +401,31 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ 
         for (int u = 0; u < MAXV; ++u) {
             const int c4 = threadIdx.x + u * blockDim.x;
             if (c4 < nv) reinterpret_cast<uint32_t*>(xq + (size_t)i * d)[c4] = pack_e4m3(v[u].x / s, v[u].y / s, v[u].z / s, v[u].w / s);
+        }
+        return;
+    }
+    if (x4.codes) {
+        // NVFP4 output of the bfloat16 rounding of the normalised row: row scale max / (6 * 448), then blocks of 16
+        float amax = 0.f;
+#pragma unroll
+        for (int u = 0; u < MAXV; ++u) {
+            const int c4 = threadIdx.x + u * blockDim.x;
+            if (c4 < nv) {
+                const float4 g = reinterpret_cast<const float4*>(gain)[c4];
+                v[u] = make_float4(wdk::bf16_round_f(v[u].x * inv * g.x), wdk::bf16_round_f(v[u].y * inv * g.y),
+                                   wdk::bf16_round_f(v[u].z * inv * g.z), wdk::bf16_round_f(v[u].w * inv * g.w));
+                amax = fmaxf(fmaxf(fmaxf(amax, fabsf(v[u].x)), fmaxf(fabsf(v[u].y), fabsf(v[u].z))), fabsf(v[u].w));
+            } else {
+                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+        amax = block_max(amax, red);
+        const float gr = amax > 0.f ? __fdiv_rn(amax, 6.0f * 448.0f) : 1.f;
+        if (threadIdx.x == 0) x4.g[i] = gr;
+#pragma unroll
+        for (int u = 0; u < MAXV; ++u) {
+            const int c4 = threadIdx.x + u * blockDim.x;
+            wdk::nvfp4_emit4(v[u], gr, c4 < nv, x4.codes + (size_t)i * (d >> 1), x4.sf + (size_t)i * (d >> 4), c4);
         }
         return;
     }
@@ -669,9 +694,10 @@ __global__ void swiglu_kernel(const float* __restrict__ part, int n_split, size_
 // and waiting while the GEMM still runs); each keeps its quarter of h = silu(gate) * up in registers
 // (up to kMaxV float4 per thread), the four partial maxima meet through distributed shared memory,
 // then every block writes the e4m3 codes of its quarter (and block 0 the row's scale).
-template <int kMaxV>
+// kFp4: NVFP4 output of the bfloat16 rounding of h instead (codes, block scales and row scale in h4; F % 64 == 0).
+template <int kMaxV, bool kFp4>
 __global__ void swiglu_fp8_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
-                                  uint8_t* __restrict__ hq, float* __restrict__ sh, int F) {
+                                  uint8_t* __restrict__ hq, float* __restrict__ sh, int F, WdFp4Operand h4) {
     __shared__ float red[32];
     __shared__ float my_max;
     pdl_launch_dependents();
@@ -706,6 +732,8 @@ __global__ void swiglu_fp8_kernel(const float* __restrict__ part, int n_split, s
     for (int u = 0; u < kMaxV; ++u) {
         g[u] = make_float4(g[u].x / (1.f + __expf(-g[u].x)) * up[u].x, g[u].y / (1.f + __expf(-g[u].y)) * up[u].y,
                            g[u].z / (1.f + __expf(-g[u].z)) * up[u].z, g[u].w / (1.f + __expf(-g[u].w)) * up[u].w);
+        if (kFp4)
+            g[u] = make_float4(wdk::bf16_round_f(g[u].x), wdk::bf16_round_f(g[u].y), wdk::bf16_round_f(g[u].z), wdk::bf16_round_f(g[u].w));
         amax = fmaxf(fmaxf(fmaxf(amax, fabsf(g[u].x)), fmaxf(fabsf(g[u].y), fabsf(g[u].z))), fabsf(g[u].w));
     }
     amax = block_max(amax, red);
@@ -718,6 +746,16 @@ __global__ void swiglu_fp8_kernel(const float* __restrict__ part, int n_split, s
         amax = fmaxf(amax, v);
     }
     wdk::cluster_sync();                            // nobody leaves while its maximum may still be read
+    if (kFp4) {
+        const float gr = amax > 0.f ? __fdiv_rn(amax, 6.0f * 448.0f) : 1.f;
+        if (threadIdx.x == 0 && quarter == 0) h4.g[r] = gr;
+#pragma unroll
+        for (int u = 0; u < kMaxV; ++u) {
+            const int c4 = c_lo + (int)threadIdx.x + u * (int)blockDim.x;
+            wdk::nvfp4_emit4(g[u], gr, c4 < c_hi, h4.codes + (size_t)r * (F >> 1), h4.sf + (size_t)r * (F >> 4), c4);
+        }
+        return;
+    }
     const float s = amax > 0.f ? amax / 448.f : 1.f;
     if (threadIdx.x == 0 && quarter == 0) sh[r] = s;
 #pragma unroll
@@ -925,8 +963,9 @@ void wd_launch_embed_fused(const void* embed, const int32_t* ids, const int32_t*
 
 void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size_t split_stride,
                        const float* gain, float eps, void* xn, const int32_t* row_idx, int n_rows,
-                       int d, cudaStream_t st, uint8_t* xq, float* sx) {
+                       int d, cudaStream_t st, uint8_t* xq, float* sx, const WdFp4Operand* x4p) {
     if (n_rows <= 0) return;
+    const WdFp4Operand x4 = x4p ? *x4p : WdFp4Operand();
     // one float4 per thread where the row allows it: the kernel is a chain of dependent L2 round
     // trips, so short per-thread work matters more than occupancy
     const int nv = d >> 2;
@@ -934,17 +973,17 @@ void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size
         // many rows: bandwidth matters, so more (smaller) blocks per SM with four float4 in flight per thread
         const int threads = ((nv + 3) / 4 + 31) / 32 * 32;
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 4>, dim3(n_rows), dim3(threads), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx, x4));
     } else if (nv <= 1024) {
         const int threads = (nv + 31) / 32 * 32;
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 1>, dim3(n_rows), dim3(threads), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx, x4));
     } else if (nv <= 2048) {
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 2>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx, x4));
     } else {
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 8>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx, x4));
     }
 }
 
@@ -1001,11 +1040,12 @@ void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_st
                                   (T*)h, n_rows, F));
 }
 
-wd_status wd_launch_swiglu_fp8(const float* part, int n_split, size_t split_stride, uint8_t* hq, float* sh, int n_rows,
-                               int F, cudaStream_t st) {
+static wd_status launch_swiglu_quant(const float* part, int n_split, size_t split_stride, uint8_t* hq, float* sh,
+                                     const WdFp4Operand* h4p, int n_rows, int F, cudaStream_t st) {
     if (n_rows <= 0) return WD_OK;
     const int f4 = F >> 2;
-    if (F % 4 || f4 > 8 * 1024) return WD_ERR_BAD_PARAM;
+    if (F % 4 || f4 > 8 * 1024 || (h4p && F % 64)) return WD_ERR_BAD_PARAM;
+    const WdFp4Operand h4 = h4p ? *h4p : WdFp4Operand();
     ++wd_launch_counter;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(4 * n_rows);
@@ -1022,11 +1062,28 @@ wd_status wd_launch_swiglu_fp8(const float* part, int n_split, size_t split_stri
     lc.numAttrs = wd_pdl_enabled ? 2 : 1;
     const int per_thread = ((f4 + 3) / 4 + 255) / 256;          // float4 per thread
     cudaError_t e;
-    if (per_thread <= 3) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<3>, part, n_split, split_stride, hq, sh, F);
-    else if (per_thread <= 5) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<5>, part, n_split, split_stride, hq, sh, F);
-    else e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<8>, part, n_split, split_stride, hq, sh, F);
+    if (h4p) {
+        if (per_thread <= 3) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<3, true>, part, n_split, split_stride, hq, sh, F, h4);
+        else if (per_thread <= 5) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<5, true>, part, n_split, split_stride, hq, sh, F, h4);
+        else e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<8, true>, part, n_split, split_stride, hq, sh, F, h4);
+    } else {
+        if (per_thread <= 3) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<3, false>, part, n_split, split_stride, hq, sh, F, h4);
+        else if (per_thread <= 5) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<5, false>, part, n_split, split_stride, hq, sh, F, h4);
+        else e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<8, false>, part, n_split, split_stride, hq, sh, F, h4);
+    }
     if (e != cudaSuccess) { wd_note_cuda_error(e, __FILE__, __LINE__); return WD_ERR_CUDA; }
     return WD_OK;
+}
+
+wd_status wd_launch_swiglu_fp8(const float* part, int n_split, size_t split_stride, uint8_t* hq, float* sh, int n_rows,
+                               int F, cudaStream_t st) {
+    return launch_swiglu_quant(part, n_split, split_stride, hq, sh, nullptr, n_rows, F, st);
+}
+
+wd_status wd_launch_swiglu_fp4(const float* part, int n_split, size_t split_stride, const WdFp4Operand* h4, int n_rows,
+                               int F, cudaStream_t st) {
+    if (!h4) return WD_ERR_NULL;
+    return launch_swiglu_quant(part, n_split, split_stride, nullptr, nullptr, h4, n_rows, F, st);
 }
 
 void wd_launch_quantize_rows(int dtype, const void* w, int n_rows, int K, uint8_t* q, float* s, cudaStream_t st) {

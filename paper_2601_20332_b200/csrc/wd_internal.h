@@ -94,13 +94,23 @@ void wd_launch_embed_fused(const void* embed, const int32_t* ids, const int32_t*
                            float* x, void* xg, const float* gain, float* sumsq, float2* rope_tab, int n_rows, int d, int S,
                            int vocab, int dh, float theta, int32_t* status, cudaStream_t st);
 
+// An operand in the NVFP4 format: e2m1 codes packed two per byte (element 2j in the low nibble), one unsigned
+// e4m3 scale per 16 elements along K, one float scale per row.
+struct WdFp4Operand {
+    uint8_t* codes = nullptr;    // [n_rows][K / 2]
+    uint8_t* sf = nullptr;       // [n_rows][K / 16]
+    float* g = nullptr;          // [n_rows]
+    int n_rows = 0, K = 0;
+};
+
 // x += sum_s part[s] (if part != null); xn = rmsnorm(x) * gain, written as `dtype`.
 // With row_idx != null the rows x[row_idx[i]] are read (no partial add, x not written)
 // and xn[i] is written: used for the final norm over the active rows only.  d % 4 == 0.
 void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size_t split_stride,
                        const float* gain, float eps, void* xn, const int32_t* row_idx, int n_rows,
-                       int d, cudaStream_t st, uint8_t* xq = nullptr, float* sx = nullptr);
-// (xq != null: FP8 output instead of xn: e4m3 codes [n_rows][d] and one scale per row)
+                       int d, cudaStream_t st, uint8_t* xq = nullptr, float* sx = nullptr, const WdFp4Operand* x4 = nullptr);
+// (xq != null: FP8 output instead of xn: e4m3 codes [n_rows][d] and one scale per row;
+//  x4 != null: NVFP4 output instead of xn, quantised from the bfloat16 rounding of the normalised row; d % 16 == 0)
 
 // plain GEMM: y[rows, n] (float) = x[rows,k] * w[n,k]^T
 void wd_launch_gemm_plain(int dtype, const void* x, const void* w, float* y, int rows, int n, int k,
@@ -131,6 +141,9 @@ void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_st
 
 // FP8: h as e4m3 codes [n_rows][F] with one scale per row (F <= 32768)
 wd_status wd_launch_swiglu_fp8(const float* part, int n_split, size_t split_stride, uint8_t* hq, float* sh, int n_rows,
+                               int F, cudaStream_t st);
+// NVFP4: the bfloat16 rounding of h in the NVFP4 format (F % 64 == 0, F <= 32768)
+wd_status wd_launch_swiglu_fp4(const float* part, int n_split, size_t split_stride, const WdFp4Operand* h4, int n_rows,
                                int F, cudaStream_t st);
 // per-row e4m3 quantisation of a [n_rows, K] matrix of `dtype` (K % 4 == 0): codes and scales
 void wd_launch_quantize_rows(int dtype, const void* w, int n_rows, int K, uint8_t* q, float* s, cudaStream_t st);

@@ -27,12 +27,12 @@ def built():
     wd_build.build()
 
 
-def run_cfg(cfg, n_steps, oracle_seqs=None, ids=None, decoded=None, refresh_mode=0, fp8=False, tol=None):
+def run_cfg(cfg, n_steps, oracle_seqs=None, ids=None, decoded=None, refresh_mode=0, fp8=False, tol=None, fp4=False):
     w = synth.make_weights(cfg, DEV)
     ids = synth.make_prompts(cfg) if ids is None else ids
     batch, S = ids.shape
     p = Parity(cfg, w, ids, decoded, oracle_seqs=oracle_seqs, max_rows=batch * S, max_active=batch * cfg["A"],
-               refresh_mode=refresh_mode, fp8=fp8)
+               refresh_mode=refresh_mode, fp8=fp8, fp4=fp4)
     logs = []
     for _ in range(n_steps):
         if tol is None:
@@ -137,3 +137,16 @@ def test_cfg2_and_cfg4_fp8_projections_at_full_width():
     assert logs[0]["info"]["n_rows"] == 352 and logs[1]["info"]["n_rows"] == 33
     logs = run_cfg(synth.get_config("dream7b", L=1), 2, oracle_seqs=[3], fp8=True, tol=(5e-2, 1e-1))
     assert logs[0]["info"]["n_rows"] == 8 * 672 and logs[1]["info"]["n_rows"] == 8 * 33
+
+
+def test_cfg2_and_cfg4_nvfp4_projections_at_full_width():
+    """NVFP4 mode (outside the paper) at the real layer widths: the LLaDA-8B block (d 4096, d_ffn 12288,
+    refresh at 352 rows and a normal step at 33) and the Dream-7B block's refresh (GQA, batch 8, d 3584, d_ffn 18944,
+    5376 rows: several token tiles per weight tile).  The vocabulary is cut to 16384 rows to keep the
+    oracle's block-by-block product within seconds; tolerances as derived in test_gpu_step."""
+    logs = run_cfg(synth.get_config("llada8b", L=1, V=16384), 2, fp4=True, tol=(1.5e-1, 1e-1))
+    assert logs[0]["info"]["n_rows"] == 352 and logs[1]["info"]["n_rows"] == 33
+    assert max(l["worst"]["logits"] for l in logs) < 2.5e-1
+    logs = run_cfg(synth.get_config("dream7b", L=1, V=16384), 1, oracle_seqs=[3], fp4=True, tol=(1.5e-1, 1e-1))
+    assert logs[0]["info"]["n_rows"] == 8 * 672
+    assert max(l["worst"]["logits"] for l in logs) < 2.5e-1

@@ -20,11 +20,11 @@ def built():
 
 
 def run(cfg, n_steps, ids=None, decoded=None, impl=wd.WD_GEMM_AUTO, jitter=0.1, tol_layer=1e-2, tol_attn=2e-2,
-        oracle_seqs=None, weights=None, fusion=wd.WD_FUSION_AUTO, refresh_mode=0, fp8=False, stagger=False):
+        oracle_seqs=None, weights=None, fusion=wd.WD_FUSION_AUTO, refresh_mode=0, fp8=False, stagger=False, fp4=False):
     w = synth.make_weights(cfg, DEV, gain_jitter=jitter) if weights is None else weights
     ids = synth.make_prompts(cfg) if ids is None else ids
     p = Parity(cfg, w, ids, decoded, gemm_impl=impl, oracle_seqs=oracle_seqs, fusion=fusion, refresh_mode=refresh_mode,
-               fp8=fp8, stagger=stagger)
+               fp8=fp8, stagger=stagger, fp4=fp4)
     logs = []
     for _ in range(n_steps):
         r = p.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"], tol_layer, tol_attn)
@@ -168,6 +168,64 @@ def test_fp8_mode_differs_from_bf16_and_can_be_switched_off():
     assert 1e-3 < rel < 0.3
     with pytest.raises(wd.WdError):
         wd.Context(synth.get_config("tiny"), synth.make_weights(synth.get_config("tiny"), DEV), 1, 96, 96, 8).fp8_enable()
+    ctx.close()
+
+
+NVFP4_SMALL = dict(SMALL_BF16, F=1536)       # the mode wants widths that are multiples of 256
+
+
+@pytest.mark.parametrize("shape,batch", [(NVFP4_SMALL, 1), (DH128, 2)])
+def test_nvfp4_mode_matches_the_oracle_in_nvfp4_mode(shape, batch):
+    """NVFP4 projections (outside the paper): the oracle quantises the same operands the same way.  On
+    identical inputs the quantised product agrees to 2e-5 (test_gemm_nvfp4_vs_oracle); in a step the two
+    sides' activations differ upstream by bf16-size amounts, and a 4-bit code turns such a difference into
+    a whole code step for the elements near a rounding boundary."""
+    cfg = synth.get_config("llada8b", **dict(shape, batch=batch))
+    # Tolerances: an upstream difference of 4e-3 (bf16) moves an element of magnitude |x| across an e2m1
+    # boundary with probability 4e-3 |x| / spacing, about 1 % (spacing 1/6 to 1/2 of |x|), and then by a
+    # whole spacing, a third of its value: 0.33 * sqrt(0.012) = 3.6e-2 relative RMS per quantised product;
+    # a flipped e4m3 block scale (4 % of the blocks) redraws the block's rounding noise, another 3e-2.
+    # Three quantised products in series per block and the LM head on top give, as the worst element over
+    # the largest, 9e-2 for the block outputs and 1.5e-1 for the logits measured; bounds at 1.7x that.
+    logs = run(cfg, 2 * cfg["R"] + 1, fp4=True, tol_layer=1.5e-1, tol_attn=1e-1)
+    assert sum(l["info"]["is_refresh"] for l in logs) == 3
+    assert max(l["worst"]["layer"] for l in logs) > 1e-2      # and it is not the bf16 pipeline
+    assert max(l["worst"]["logits"] for l in logs) < 2.5e-1
+
+
+def test_nvfp4_mode_differs_from_bf16_and_excludes_fp8():
+    cfg = synth.get_config("llada8b", **DH128)
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    S = ids.shape[1]
+    ctx = wd.Context(cfg, w, 1, S, S, S)
+    lg = torch.zeros(S * cfg["V"], device=DEV)
+    outs = {}
+    for mode in ("bf16", "fp4", "fp8", "fp4 again", "off"):
+        if mode == "fp4":
+            ctx.fp4_enable()
+        if mode == "fp8":
+            ctx.fp8_enable()            # switches NVFP4 off
+        if mode == "fp4 again":
+            ctx.fp4_set(True)           # ... and back, which switches FP8 off
+        if mode == "off":
+            ctx.fp4_set(False)
+        st = wd.State(ctx, ids)
+        st.set_taps(logits=lg)
+        _, info = st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], 1)
+        st.sync()
+        outs[mode] = lg[: info["n_active"] * cfg["V"]].clone()
+        st.close()
+    assert torch.equal(outs["bf16"], outs["off"])
+    assert torch.equal(outs["fp4"], outs["fp4 again"])
+    rel4 = float((outs["fp4"] - outs["bf16"]).norm() / outs["bf16"].norm())
+    rel8 = float((outs["fp8"] - outs["bf16"]).norm() / outs["bf16"].norm())
+    assert 1e-3 < rel8 < rel4 < 0.6
+    with pytest.raises(wd.WdError):     # fp32 model
+        wd.Context(synth.get_config("tiny"), synth.make_weights(synth.get_config("tiny"), DEV), 1, 96, 96, 8).fp4_enable()
+    with pytest.raises(wd.WdError):     # d_ffn not a multiple of 256
+        c2 = synth.get_config("llada8b", **SMALL_BF16)
+        wd.Context(c2, synth.make_weights(c2, DEV), 1, 120, 120, 8).fp4_enable()
     ctx.close()
 
 

@@ -34,7 +34,7 @@ def max_rel(a, b):
 class Parity:
     def __init__(self, cfg, weights, ids, decoded=None, gemm_impl=wd.WD_GEMM_AUTO, oracle_seqs=None,
                  max_rows=None, max_active=None, fusion=wd.WD_FUSION_AUTO, eos_id=None, refresh_mode=0, fp8=False,
-                 follow_rounded=False, stagger=False):
+                 follow_rounded=False, stagger=False, fp4=False):
         """follow_rounded: a second oracle follower per sequence runs in the bfloat16 storage-points mode
         (the same teacher-forced trajectory); `step` then also records, per block, the GPU's distance to it
         and its own distance to the plain float64 follower: what the storage format alone costs at that
@@ -49,6 +49,8 @@ class Parity:
         self.ctx.set_fusion(fusion)
         if fp8:
             self.ctx.fp8_enable()
+        if fp4:
+            self.ctx.fp4_enable()
         self.st = wd.State(self.ctx, ids, decoded)
         if eos_id is not None:
             self.st.set_eos(eos_id)
@@ -64,6 +66,8 @@ class Parity:
         self.model = synth.OracleModelView(weights)
         if fp8:
             self.model.dims = dict(self.model.dims, fp8=True)
+        if fp4:
+            self.model.dims = dict(self.model.dims, nvfp4=True)
         self.oracle_seqs = list(range(self.batch)) if oracle_seqs is None else list(oracle_seqs)
         dec = (ids != cfg["mask_id"]) if decoded is None else decoded.astype(bool)
         stg = (lambda b: (b, self.batch)) if stagger else (lambda b: None)
