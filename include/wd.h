@@ -467,6 +467,19 @@ WD_API wd_status wd_op_gemm_fp4(const void* x, const void* w, float* y, int32_t 
                          void* scratch, size_t scratch_bytes, void* stream /*cudaStream_t*/);
 WD_API size_t wd_op_gemm_fp4_scratch_bytes(int32_t rows, int32_t n_out, int32_t k_in);
 
+/* The two halves of wd_op_gemm_fp4 for callers that quantise an operand once and multiply it many times
+ * (no counterpart in the paper).  wd_op_nvfp4_quantize writes the NVFP4 form of the bf16 matrix
+ * x[rows, k_in] (k_in a multiple of 16) into `out` (device, 256-byte aligned, wd_op_nvfp4_bytes large:
+ * codes [rows][k_in / 2], then block scales [rows][k_in / 16], then float row scales [rows], each part
+ * starting on a 256-byte boundary).  wd_op_gemm_nvfp4 multiplies two such operands: y[rows, n_out] float;
+ * k_in a multiple of 256; scratch 256-byte aligned, wd_op_gemm_scratch_bytes(rows, n_out, k_in) large.
+ * Errors as wd_op_gemm. */
+WD_API size_t wd_op_nvfp4_bytes(int32_t rows, int32_t k_in);
+WD_API wd_status wd_op_nvfp4_quantize(const void* x, int32_t rows, int32_t k_in, void* out, size_t out_bytes,
+                               void* stream /*cudaStream_t*/);
+WD_API wd_status wd_op_gemm_nvfp4(const void* xq, const void* wq, float* y, int32_t rows, int32_t n_out, int32_t k_in,
+                           void* scratch, size_t scratch_bytes, void* stream /*cudaStream_t*/);
+
 /* (No counterpart in the paper: a packaging variant of wd_op_gemm.)
  * The same bf16 tensor-core GEMM, y[rows, n_out] (float) = x[rows, k_in] * w[n_out, k_in]^T,
  * for callers that cannot hand over scratch memory because they may not allocate

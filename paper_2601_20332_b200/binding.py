@@ -103,6 +103,9 @@ SIGNATURES = {
     "wd_op_gemm_fp8_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
     "wd_op_gemm_fp4": (C.c_int, [vp, vp, vp, i32, i32, i32, vp, C.c_size_t, vp]),
     "wd_op_gemm_fp4_scratch_bytes": (C.c_size_t, [i32, i32, i32]),
+    "wd_op_nvfp4_bytes": (C.c_size_t, [i32, i32]),
+    "wd_op_nvfp4_quantize": (C.c_int, [vp, i32, i32, vp, C.c_size_t, vp]),
+    "wd_op_gemm_nvfp4": (C.c_int, [vp, vp, vp, i32, i32, i32, vp, C.c_size_t, vp]),
     "wd_op_gemm_noalloc": (C.c_int, [vp, vp, vp, i32, i32, i32, vp]),
     "wd_op_gemm_noalloc_max_floats": (C.c_size_t, []),
     "wd_op_attention": (C.c_int, [i32, vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]),
@@ -442,6 +445,30 @@ def op_gemm_fp4(x, w, stream=None):
     nb = lib().wd_op_gemm_fp4_scratch_bytes(rows, n, k)
     scratch = torch.empty(max(nb, 256), dtype=torch.uint8, device=x.device)
     check(lib().wd_op_gemm_fp4(_ptr(x), _ptr(w), _ptr(y), rows, n, k, _ptr(scratch), nb, _stream_ptr(stream)), "wd_op_gemm_fp4")
+    return y
+
+
+def op_nvfp4_quantize(x, stream=None):
+    """The NVFP4 form of a bf16 matrix [rows, k] as one uint8 device tensor (codes | block scales | row scales)."""
+    import torch
+    rows, k = x.shape
+    nb = lib().wd_op_nvfp4_bytes(rows, k)
+    if nb == 0:
+        raise WdError(WD_ERR_BAD_PARAM, "wd_op_nvfp4_bytes")
+    out = torch.empty(nb, dtype=torch.uint8, device=x.device)
+    check(lib().wd_op_nvfp4_quantize(_ptr(x), rows, k, _ptr(out), nb, _stream_ptr(stream)), "wd_op_nvfp4_quantize")
+    return out
+
+
+def op_gemm_nvfp4(xq, wq, rows, n, k, scratch=None, stream=None):
+    """y[rows, n] (float32) from two operands quantised by op_nvfp4_quantize."""
+    import torch
+    y = torch.empty(rows, n, dtype=torch.float32, device=xq.device)
+    nb = lib().wd_op_gemm_scratch_bytes(rows, n, k)
+    if scratch is None:
+        scratch = torch.empty(max(nb, 256), dtype=torch.uint8, device=xq.device)
+    check(lib().wd_op_gemm_nvfp4(_ptr(xq), _ptr(wq), _ptr(y), rows, n, k, _ptr(scratch), scratch.numel(), _stream_ptr(stream)),
+          "wd_op_gemm_nvfp4")
     return y
 
 

@@ -1614,6 +1614,47 @@ extern "C" wd_status wd_op_gemm_fp4(const void* x, const void* w, float* y, int3
     return WD_OK;
 }
 
+extern "C" size_t wd_op_nvfp4_bytes(int32_t rows, int32_t k_in) {
+    if (rows < 1 || k_in < 16 || k_in % 16) return 0;
+    return wd_fp4_operand_bytes(rows, k_in);
+}
+
+extern "C" wd_status wd_op_nvfp4_quantize(const void* x, int32_t rows, int32_t k_in, void* out, size_t out_bytes, void* stream_) {
+    if (!x || !out) return WD_ERR_NULL;
+    if (rows < 1 || k_in < 16 || k_in % 16) return WD_ERR_BAD_PARAM;
+    if ((uintptr_t)out % 256) return WD_ERR_MISALIGNED;
+    if (out_bytes < wd_fp4_operand_bytes(rows, k_in)) return WD_ERR_WORKSPACE_TOO_SMALL;
+    WdFp4Operand op;
+    wd_fp4_operand_split(out, rows, k_in, &op);
+    wd_launch_quantize_nvfp4(WD_BF16, x, rows, k_in, &op, (cudaStream_t)stream_);
+    WD_CUDA_TRY(cudaGetLastError());
+    return WD_OK;
+}
+
+extern "C" wd_status wd_op_gemm_nvfp4(const void* xq, const void* wq, float* y, int32_t rows, int32_t n_out, int32_t k_in,
+                                      void* scratch, size_t scratch_bytes, void* stream_) {
+    if (!xq || !wq || !y || !scratch) return WD_ERR_NULL;
+    if (rows < 1 || n_out < 1 || k_in < 256 || k_in % 256) return WD_ERR_BAD_PARAM;
+    if ((uintptr_t)scratch % 256 || (uintptr_t)xq % 256 || (uintptr_t)wq % 256) return WD_ERR_MISALIGNED;
+    if (scratch_bytes < wd_tc_scratch_bytes(rows, n_out, k_in)) return WD_ERR_WORKSPACE_TOO_SMALL;
+    int32_t* status = wd_op_status_ptr();
+    if (!status) return WD_ERR_CUDA;
+    cudaStream_t stream = (cudaStream_t)stream_;
+    int sm = 148, dev = 0;
+    WD_CUDA_TRY(cudaGetDevice(&dev));
+    WD_CUDA_TRY(cudaDeviceGetAttribute(&sm, cudaDevAttrMultiProcessorCount, dev));
+    WdFp4Operand ox, ow;
+    wd_fp4_operand_split(const_cast<void*>(xq), rows, k_in, &ox);
+    wd_fp4_operand_split(const_cast<void*>(wq), n_out, k_in, &ow);
+    int ns = 1;
+    const size_t slice = (size_t)rows * n_out;
+    wd_status s = wd_fp4_gemm(&ox, &ow, (float*)scratch, scratch_bytes / 4, sm, status, stream, &ns, false, false);
+    if (s != WD_OK) return s;
+    wd_launch_reduce_slices((const float*)scratch, ns, slice, y, slice, stream);
+    WD_CUDA_TRY(cudaGetLastError());
+    return WD_OK;
+}
+
 extern "C" wd_status wd_op_gemm(int32_t dtype, int32_t impl, const void* x, const void* w, float* y, int32_t rows,
                                 int32_t n_out, int32_t k_in, void* scratch, size_t scratch_bytes, void* stream) {
     if (!x || !w || !y) return WD_ERR_NULL;

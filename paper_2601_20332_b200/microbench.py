@@ -1,6 +1,7 @@
 """Micro-benchmarks of single kernels through the C ABI (CUDA-event timing).
 
     python -m paper_2601_20332_b200.microbench gemm --rows 34 --n 24576 --k 4096 [--iters 20]
+    python -m paper_2601_20332_b200.microbench gemm-fp4 --rows 34 --n 24576 --k 4096 [--iters 20]
     python -m paper_2601_20332_b200.microbench gemm-suite [--rows 34]
     python -m paper_2601_20332_b200.microbench step --config llada8b --layers 4 [--steps 16]
     python -m paper_2601_20332_b200.microbench sweep [--A 16,32,64,128 --B 64,128,256 --R 1,4,16 --batch 1,16]
@@ -48,6 +49,38 @@ def time_gemm(rows, n, k, iters=20, impl=wd.WD_GEMM_TCGEN05, ring_bytes=600 << 2
     ts = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(iters)])
     by = wbytes + rows * k * 2 + rows * n * 4
     return dict(rows=rows, n=n, k=k, us_median=float(np.median(ts) * 1e3), us_min=float(ts.min() * 1e3),
+                algorithmic_bytes=by, gbs_median=by / (np.median(ts) * 1e-3) / 1e9,
+                tflops_median=2.0 * rows * n * k / (np.median(ts) * 1e-3) / 1e12,
+                note="includes the split-K reduce kernel of the single-op entry point")
+
+
+def time_gemm_fp4(rows, n, k, iters=20, ring_bytes=600 << 20):
+    """The NVFP4 GEMM alone on operands quantised beforehand (a ring of distinct weights keeps every launch cold)."""
+    dev = "cuda:0"
+    g = torch.Generator(device=dev).manual_seed(1)
+    wbytes = n * k * 9 // 16
+    n_ring = max(2, min(8, ring_bytes // wbytes + 1))
+    wqs = []
+    for _ in range(n_ring):
+        w = (torch.randn(n, k, device=dev, generator=g) * 0.02).to(torch.bfloat16)
+        wqs.append(wd.op_nvfp4_quantize(w))
+        del w
+    xq = wd.op_nvfp4_quantize(torch.randn(rows, k, device=dev, generator=g).to(torch.bfloat16))
+    nb = wd.lib().wd_op_gemm_scratch_bytes(rows, n, k)
+    scratch = torch.empty(max(nb, 256), dtype=torch.uint8, device=dev)
+    for i in range(3):
+        wd.op_gemm_nvfp4(xq, wqs[i % n_ring], rows, n, k, scratch=scratch)
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(iters + 1)]
+    ev[0].record()
+    for i in range(iters):
+        wd.op_gemm_nvfp4(xq, wqs[i % n_ring], rows, n, k, scratch=scratch)
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    assert wd.op_status() == 0
+    ts = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(iters)])
+    by = (n + rows) * k * 9 // 16 + rows * n * 4
+    return dict(kind="nvfp4", rows=rows, n=n, k=k, us_median=float(np.median(ts) * 1e3), us_min=float(ts.min() * 1e3),
                 algorithmic_bytes=by, gbs_median=by / (np.median(ts) * 1e-3) / 1e9,
                 tflops_median=2.0 * rows * n * k / (np.median(ts) * 1e-3) / 1e12,
                 note="includes the split-K reduce kernel of the single-op entry point")
@@ -140,7 +173,7 @@ def run_sweep(config, layers, A_list, B_list, R_list, batch_list, repeats, out_p
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("mode", choices=["gemm", "gemm-suite", "step", "sweep"])
+    ap.add_argument("mode", choices=["gemm", "gemm-fp4", "gemm-suite", "step", "sweep"])
     ap.add_argument("--rows", type=int, default=34)
     ap.add_argument("--n", type=int, default=24576)
     ap.add_argument("--k", type=int, default=4096)
@@ -161,6 +194,8 @@ def main():
     impl = wd.WD_GEMM_PLAIN if a.plain else wd.WD_GEMM_TCGEN05
     if a.mode == "gemm":
         print(json.dumps(time_gemm(a.rows, a.n, a.k, a.iters, impl)))
+    elif a.mode == "gemm-fp4":
+        print(json.dumps(time_gemm_fp4(a.rows, a.n, a.k, a.iters)))
     elif a.mode == "gemm-suite":
         for name, n, k in LLADA_GEMMS:
             r = time_gemm(a.rows, n, k, a.iters, impl)

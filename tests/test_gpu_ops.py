@@ -83,6 +83,38 @@ def test_gemm_nvfp4_vs_oracle(rows, n, k):
     assert 3e-2 < np.linalg.norm(got - exact) / np.linalg.norm(exact) < 0.25        # it really is a 4-bit product
 
 
+def test_nvfp4_quantise_once_multiply_many_and_the_stored_format():
+    """wd_op_nvfp4_quantize + wd_op_gemm_nvfp4 give the bits of wd_op_gemm_fp4, and the stored operand is the
+    oracle's quantisation: codes two per byte (even element in the low nibble), e4m3 block scales, float row scales."""
+    rows, n, k = 37, 300, 768
+    g = torch.Generator(device=DEV).manual_seed(5)
+    x = torch.randn(rows, k, device=DEV, generator=g).to(torch.bfloat16)
+    x[3] = 0                                                    # an all-zero row: row scale 1, every code 0
+    x[5, 32:48] = 0                                             # an all-zero block: block scale 0
+    w = (torch.randn(n, k, device=DEV, generator=g) * 0.05).to(torch.bfloat16)
+    xq, wq = wd.op_nvfp4_quantize(x), wd.op_nvfp4_quantize(w)
+    y1 = wd.op_gemm_nvfp4(xq, wq, rows, n, k)
+    y2 = wd.op_gemm_nvfp4(xq, wq, rows, n, k)
+    assert torch.equal(y1, y2) and torch.equal(y1, wd.op_gemm_fp4(x, w)) and wd.op_status() == 0
+    q, s, gr = wo.nvfp4_quant_rows(x.float().cpu().numpy().astype(np.float64))
+    raw = xq.cpu().numpy()
+    up = lambda v: (v + 255) // 256 * 256
+    codes = raw[: rows * k // 2].reshape(rows, k // 2)
+    sf = raw[up(rows * k // 2): up(rows * k // 2) + rows * k // 16].reshape(rows, k // 16)
+    g_off = up(rows * k // 2) + up(rows * k // 16)
+    gs = raw[g_off: g_off + 4 * rows].view(np.float32)
+    grid = np.array([0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0])
+    val = lambda c: np.where(c & 8, -1.0, 1.0) * grid[c & 7]
+    got = np.empty((rows, k))
+    got[:, 0::2] = val(codes & 15)
+    got[:, 1::2] = val(codes >> 4)
+    np.testing.assert_array_equal(np.abs(got), np.abs(q))       # (-0 and +0 are the same element)
+    np.testing.assert_array_equal(np.sign(got) * (got != 0), np.sign(q) * (q != 0))
+    np.testing.assert_array_equal(torch.from_numpy(sf.copy()).view(torch.float8_e4m3fn).double().numpy(), s)
+    np.testing.assert_array_equal(gs, gr)
+    assert gs[3] == 1.0 and not codes[3].any() and sf[5, 2] == 0
+
+
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 @pytest.mark.parametrize("rows,n,k", [(1, 5, 3), (10, 70, 33), (34, 384, 256), (97, 130, 1000)])
 def test_gemm_plain_vs_oracle(dtype, rows, n, k):
