@@ -1020,7 +1020,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     pend.cp.assign(batch, WdCountPlan());
     bool all_done = true, any_refresh = false, all_contig = true;
     size_t n_rows = 0, n_act = 0, n_vis = 0, n_qtiles = 0;
-    int max_vis = 0;
+    int max_vis = 0, max_tile_rows = 0;
     if (!dev_mode) {
         st->plans.assign(batch, WdSeqPlan());
         for (int b = 0; b < batch; ++b) {
@@ -1061,6 +1061,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         n_rows += cp.n_rows; n_act += cp.n_active; n_vis += cp.n_vis;
         n_qtiles += (cp.n_rows + 127) / 128;
         max_vis = std::max(max_vis, (int)cp.n_vis);
+        max_tile_rows = std::max(max_tile_rows, std::min(128, (int)cp.n_rows));
     }
     if (all_done) return WD_DONE;
     if (n_rows > (size_t)d.max_rows || n_act > (size_t)d.max_active ||
@@ -1199,7 +1200,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         if (st->attn_tc && all_contig && c->attn_impl != WD_GEMM_PLAIN)
             return wd_attn_tc_launch(c->q, R_, (int)n_qtiles, c->plan + o_qt_seq, c->plan + o_qt_row0, c->plan + o_qt_n,
                                      c->plan + o_nvis, &st->map_k, &st->map_vt, c->attn, attn_tap, Hq, Hkv, dh, l, max_vis,
-                                     c->sm_count, status, stream);
+                                     c->sm_count, status, stream, max_tile_rows);
         wd_launch_attention_plain(d.dtype, c->q, kc, vc, row_seq, vis_idx, vis_off, c->attn, attn_tap, R_, max_vis, Hq,
                                   Hkv, dh, S, Sp, batch, status, stream);
         return WD_OK;
@@ -1719,7 +1720,8 @@ extern "C" wd_status wd_op_attention_tc(const void* q, const void* kcache, const
     wd_launch_fill_qtiles(lists, n_rows, n_vis, stream);
     WD_CUDA_TRY(cudaGetLastError());
     return wd_attn_tc_launch(q, n_rows, n_tiles, lists, lists + n_tiles, lists + 2 * n_tiles, lists + 3 * n_tiles, &map_k,
-                             &map_vt, out, nullptr, n_q_heads, n_kv_heads, 128, 0, max_vis, sm, status, stream);
+                             &map_vt, out, nullptr, n_q_heads, n_kv_heads, 128, 0, max_vis, sm, status, stream,
+                             std::min(n_rows, 128));
 }
 
 extern "C" size_t wd_op_lm_unmask_scratch_bytes(int32_t n, int32_t vocab) {

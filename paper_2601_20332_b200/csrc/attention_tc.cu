@@ -28,6 +28,8 @@
 // Every wait is bounded; on expiry the CTA records WD_ERR_DEVICE_TIMEOUT and leaves.
 #include <cstring>
 
+#include <cstdlib>
+
 #include "attention_tc.h"
 #include "device_utils.cuh"
 
@@ -57,6 +59,9 @@ struct AttnParams {
     // split over the keys: CTA z of (tile, head) takes key tiles [z * tiles_per_split, ...); the
     // max_parts CTAs of a (tile, head) pair form one cluster
     int tiles_per_split, max_parts;
+    // head packing (grouped-query attention with few rows): a 128-row query tile holds `pack` slots of `slot`
+    // rows, one query head of the same KV head each (slot >= the tile's valid rows); grid.y = Hkv * tiles_per_kv
+    int pack, slot, slot_shift, tiles_per_kv;      // slot = 128 / pack = 1 << slot_shift
 };
 
 __device__ __forceinline__ void cluster_sync_all() {
@@ -124,9 +129,12 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     float* part_ml = (float*)(sK + 2 * kOperand);          // [128 rows][2] running maximum, sum
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile = blockIdx.x, h = blockIdx.y;
+    const int tile = blockIdx.x;
     const int b = p.qtile_seq[tile], row0 = p.qtile_row0[tile], n_valid = p.qtile_n[tile];
-    const int kvh = h / (p.Hq / p.Hkv);
+    const int group = p.Hq / p.Hkv;
+    const int kvh = (int)blockIdx.y / p.tiles_per_kv, hg = (int)blockIdx.y % p.tiles_per_kv;
+    const int h = kvh * group + hg * p.pack;              // query head of slot 0; slot j holds head h + j
+    const int n_slots = min(p.pack, group - hg * p.pack);  // slots of this tile that hold a head
 
     pdl_launch_dependents();
     // The index lists are complete before this kernel can start: a host-planned step copies them in
@@ -161,9 +169,14 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (lane == 0) {
             // ---------------------------------------------------- TMA producer
             const uint32_t qf = smem_u32(&bars[kQFull]);
-            mbar_expect_tx(qf, kOperand);
-            tma_load_2d(smem_u32(sQ), &map_q, qf, h * kTile, row0);
-            tma_load_2d(smem_u32(sQ) + kAtom, &map_q, qf, h * kTile + 64, row0);
+            // slot j: rows [row0, row0 + slot) of head h + j at tile rows [j * slot, ...); slots without a head
+            // stay unwritten (their rows of S and O are never read)
+            mbar_expect_tx(qf, (uint32_t)(n_slots * p.slot * 256));
+            for (int j = 0; j < n_slots; ++j) {
+                const uint32_t dst = smem_u32(sQ) + (uint32_t)(j * p.slot * 128);
+                tma_load_2d(dst, &map_q, qf, (h + j) * kTile, row0);
+                tma_load_2d(dst + kAtom, &map_q, qf, (h + j) * kTile + 64, row0);
+            }
             const int bh = b * p.Hkv + kvh;
             auto load_k = [&](int j) -> bool {
                 const int ks = j % kStages;
@@ -252,8 +265,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         const int r = quarter * 32 + lane;                 // query row of the tile = TMEM lane
         // warps whose 32 rows are all beyond the valid ones only keep the barrier counts right.
         // The test is per warp, not per row: tcgen05.ld is warp-collective and must not diverge.
-        const bool live = quarter * 32 < n_valid;
-        const bool valid = r < n_valid;
+        const int sj = r >> p.slot_shift, rr_ = r & (p.slot - 1);       // slot (head h + sj) and row within the slot
+        const bool live = ((quarter * 32) >> p.slot_shift) < n_slots && ((quarter * 32) & (p.slot - 1)) < n_valid;
+        const bool valid = sj < n_slots && rr_ < n_valid;
         const int c_off = 64 * hf;
         const uint32_t t_row = tmem_base + ((uint32_t)(quarter * 32) << 16);
         float* xch = (float*)(tmem_slot + 4);              // [2][128] exchange between the two halves (row sums)
@@ -380,7 +394,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         if (n_parts == 1) {
             if (ok && valid) {
                 const float inv = 1.f / l;
-                const size_t base = ((size_t)(row0 + r) * p.Hq + h) * kTile + c_off;
+                const size_t base = ((size_t)(row0 + rr_) * p.Hq + h + sj) * kTile + c_off;
                 uint4* dst = reinterpret_cast<uint4*>(p.out + base);
 #pragma unroll
                 for (int g = 0; g < 8; ++g) {
@@ -413,8 +427,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             // CTA z merges rows [z * per, (z + 1) * per).  An item = (row, group of 4 columns); a
             // thread takes items t, t + 256, ... and keeps kItems x kParts remote loads in flight.
             constexpr int kItems = 2, kParts = 4;
-            const int per = (n_valid + n_parts - 1) / n_parts;
-            const int r_lo = min((int)blockIdx.z * per, n_valid), r_hi = min(r_lo + per, n_valid);
+            // (rows are counted over the valid rows of all slots: index q = slot * n_valid + row within the slot)
+            const int n_tot = n_slots * n_valid;
+            const int per = (n_tot + n_parts - 1) / n_parts;
+            const int r_lo = min((int)blockIdx.z * per, n_tot), r_hi = min(r_lo + per, n_tot);
             const int t = (int)threadIdx.x - 64, n_items = (r_hi - r_lo) * 32;
             const uint32_t lo = smem_u32(part_o), lml = smem_u32(part_ml);
             for (int it0 = t; it0 < n_items; it0 += 256 * kItems) {
@@ -431,7 +447,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                     float4 v[kItems][kParts];
 #pragma unroll
                     for (int u = 0; u < kItems; ++u) {
-                        const int item = it0 + u * 256, rr = r_lo + (item >> 5), cg = item & 31;
+                        const int item = it0 + u * 256, qq = r_lo + (item >> 5), cg = item & 31;
+                        const int rr = (qq / n_valid) * p.slot + qq % n_valid;         // tile row
 #pragma unroll
                         for (int zz = 0; zz < kParts; ++zz) {
                             ml[u][zz] = make_float2(-INFINITY, 0.f);
@@ -464,10 +481,10 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
                 }
 #pragma unroll
                 for (int u = 0; u < kItems; ++u) {
-                    const int item = it0 + u * 256, rr = r_lo + (item >> 5), cg = item & 31;
+                    const int item = it0 + u * 256, qq = r_lo + (item >> 5), cg = item & 31;
                     if (item >= n_items) continue;
                     const float inv = 1.f / lsum[u];
-                    const size_t base = ((size_t)(row0 + rr) * p.Hq + h) * kTile + 4 * cg;
+                    const size_t base = ((size_t)(row0 + qq % n_valid) * p.Hq + h + qq / n_valid) * kTile + 4 * cg;
                     uint2 w2;
                     w2.x = pack_bf16(acc[u].x * inv, acc[u].y * inv);
                     w2.y = pack_bf16(acc[u].z * inv, acc[u].w * inv);
@@ -541,7 +558,7 @@ wd_status wd_attn_tc_encode_cache(CUtensorMap* map_k, CUtensorMap* map_vt, const
 wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_t* qtile_seq, const int32_t* qtile_row0,
                             const int32_t* qtile_n, const int32_t* seq_nvis, const CUtensorMap* map_k,
                             const CUtensorMap* map_vt, void* out, float* tap, int Hq, int Hkv, int dh, int layer,
-                            int max_vis, int sm_count, int32_t* status, cudaStream_t stream) {
+                            int max_vis, int sm_count, int32_t* status, cudaStream_t stream, int max_tile_rows) {
     if (dh != kTile) return WD_ERR_BAD_PARAM;
     if (n_tiles <= 0) return WD_OK;
     EncodeTiledFn enc = get_encode();
@@ -549,19 +566,31 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     // the query descriptor depends only on (buffer, rows, heads): the same for every layer of a step
     static CUtensorMap mq;
     static const void* mq_ptr = nullptr;
-    static int mq_rows = -1, mq_hq = -1, mq_dev = -1;
+    static int mq_rows = -1, mq_hq = -1, mq_dev = -1, mq_slot = -1;
     int dev = 0;
     WD_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return WD_ERR_CUDA;
-    if (mq_ptr != q || mq_rows != n_rows || mq_hq != Hq || mq_dev != dev) {
+    // Grouped-query attention with few rows per tile: 2 or 4 query heads of one KV head share a 128-row tile
+    // (slots of 64 or 32 rows), so their K/V tiles are loaded once and the grid shrinks by that factor
+    const int group = Hq / Hkv;
+    static const int pack_max = getenv("WD_ATTN_PACK") ? atoi(getenv("WD_ATTN_PACK")) : 4;     // 1 switches packing off
+    int pack = 1;
+    if (max_tile_rows > 0 && group > 1) {
+        if (max_tile_rows <= 32 && group >= 4) pack = 4;
+        else if (max_tile_rows <= 64) pack = 2;
+        if (pack > pack_max) pack = pack_max >= 2 ? 2 : 1;
+        if (pack == 2 && max_tile_rows > 64) pack = 1;
+    }
+    const int slot = kTile / pack;
+    if (mq_ptr != q || mq_rows != n_rows || mq_hq != Hq || mq_dev != dev || mq_slot != slot) {
         cuuint64_t dims[2] = {(cuuint64_t)Hq * dh, (cuuint64_t)n_rows};
         cuuint64_t strides[1] = {(cuuint64_t)Hq * dh * 2};
-        cuuint32_t box[2] = {64, 128}, estr[2] = {1, 1};
+        cuuint32_t box[2] = {64, (cuuint32_t)slot}, estr[2] = {1, 1};
         if (enc(&mq, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(q), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return WD_ERR_CUDA;
-        mq_ptr = q; mq_rows = n_rows; mq_hq = Hq; mq_dev = dev;
+        mq_ptr = q; mq_rows = n_rows; mq_hq = Hq; mq_dev = dev; mq_slot = slot;
     }
     AttnParams p;
     memset(&p, 0, sizeof(p));
@@ -573,7 +602,12 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     p.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(kTile >> 3) << 17) | ((uint32_t)(kTile >> 4) << 24);
     // split the keys across the CTAs of a cluster while (tile, head) pairs alone would leave SMs idle
     const int max_kt = (max_vis + kTile - 1) / kTile;
-    int want = sm_count / (n_tiles * Hq);
+    p.pack = pack;
+    p.slot = slot;
+    p.slot_shift = pack == 1 ? 7 : (pack == 2 ? 6 : 5);
+    p.tiles_per_kv = (group + pack - 1) / pack;
+    const int grid_y = Hkv * p.tiles_per_kv;
+    int want = sm_count / (n_tiles * grid_y);
     if (want < 1) want = 1;
     if (want > kMaxCluster) want = kMaxCluster;
     if (want > max_kt) want = max_kt;
@@ -586,7 +620,7 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
         attr_done[dev] = true;
     }
     cudaLaunchConfig_t lc = {};
-    lc.gridDim = dim3(n_tiles, Hq, p.max_parts);
+    lc.gridDim = dim3(n_tiles, grid_y, p.max_parts);
     lc.blockDim = dim3(kThreads);
     lc.dynamicSmemBytes = smem;
     lc.stream = stream;

@@ -177,6 +177,10 @@ ATTN_TC_CASES = [  # rows, n_vis, Hq, Hkv, S, q scale, max_vis (0 = n_vis)
     (35, 3072, 7, 1, 3072, 8.0, 0), (129, 1025, 14, 2, 1040, 1.5, 0), (5, 3072, 1, 1, 3072, 1.5, 0),
     # max_vis > n_vis: the split is sized for 8 or 24 key tiles, this sequence has 1, 2 or 3
     (34, 129, 1, 1, 1024, 8.0, 1024), (1, 1, 7, 1, 3072, 1.5, 3072), (130, 300, 2, 2, 1024, 1.5, 1000),
+    # grouped-query heads with few rows: 4 heads per tile (<= 32 rows, slots of 32), 2 heads per tile (<= 64 rows),
+    # groups that leave the last tile with an empty slot (7 = 4 + 3, 3 = 2 + 1), 65 rows (no packing)
+    (32, 700, 8, 2, 704, 8.0, 0), (33, 500, 8, 2, 512, 1.5, 0), (64, 260, 4, 2, 264, 8.0, 0), (65, 260, 4, 2, 264, 1.5, 0),
+    (20, 129, 12, 4, 136, 8.0, 1024), (7, 1300, 28, 4, 1304, 1.5, 0),
 ]
 
 
