@@ -76,18 +76,19 @@ __device__ __forceinline__ float block_max(float v, float* red) {
     return warp_max(t);
 }
 
-// Sum of n_split partial-sum slices at one float4 position.  Slices are loaded four at a time
-// before the first add so that their L2 round trips overlap; the adds keep slice order.
+// Sum of n_split partial-sum slices at one float4 position.  Slices are loaded eight at a time
+// before the first add so that their L2 round trips overlap (the narrow GEMMs of a few-row step leave up
+// to six); the adds keep slice order.
 __device__ __forceinline__ float4 sum_slices4(const float* __restrict__ p, int n_split, size_t stride) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s0 = 0; s0 < n_split; s0 += 4) {
-        float4 t[4];
+    for (int s0 = 0; s0 < n_split; s0 += 8) {
+        float4 t[8];
 #pragma unroll
-        for (int k = 0; k < 4; ++k)
+        for (int k = 0; k < 8; ++k)
             t[k] = s0 + k < n_split ? *reinterpret_cast<const float4*>(p + (size_t)(s0 + k) * stride)
                                     : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) { acc.x += t[k].x; acc.y += t[k].y; acc.z += t[k].z; acc.w += t[k].w; }
+        for (int k = 0; k < 8; ++k) { acc.x += t[k].x; acc.y += t[k].y; acc.z += t[k].z; acc.w += t[k].w; }
     }
     return acc;
 }
@@ -345,26 +346,22 @@ __device__ __forceinline__ uint32_t pack_e4m3(float a, float b, float c, float d
            ((uint32_t)__nv_cvt_float_to_fp8(d, __NV_SATFINITE, __NV_E4M3) << 24);
 }
 
-template <typename T, int MAXV>
-__global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
-                               size_t split_stride, const float* __restrict__ gain, float eps,
-                               T* __restrict__ xn, const int32_t* __restrict__ row_idx, int d,
-                               uint8_t* __restrict__ xq, float* __restrict__ sx, WdFp4Operand x4) {
-    __shared__ float red[32];
-    pdl_launch_dependents();
-    pdl_wait();
-    const int i = blockIdx.x;
-    const int r = row_idx ? row_idx[i] : i;
-    float* xr = x + (size_t)r * d;
-    const int nv = d >> 2;
-    float4 v[MAXV], add[MAXV];
+// The front of the RMSNorm kernels: x += sum of the partial slices (if any), v = the row's float4 of this
+// thread, returns 1 / rms of the row.
+template <int MAXV>
+__device__ __forceinline__ float rmsnorm_front(float* __restrict__ xr, const float* __restrict__ part, int n_split,
+                                               size_t split_stride, size_t row_off, int nv, int d, float eps,
+                                               const float* __restrict__ gain, float4 (&v)[MAXV], float4 (&gv)[MAXV],
+                                               float* red) {
+    float4 add[MAXV];
     float ss = 0.f;
 #pragma unroll
-    for (int u = 0; u < MAXV; ++u) {             // all loads first: x and every slice of every group
+    for (int u = 0; u < MAXV; ++u) {             // all loads first: x, the gains and every slice of every group
         const int c4 = threadIdx.x + u * blockDim.x;
         if (c4 < nv) {
             v[u] = reinterpret_cast<const float4*>(xr)[c4];
-            if (part) add[u] = sum_slices4(part + (size_t)r * d + 4 * c4, n_split, split_stride);
+            gv[u] = reinterpret_cast<const float4*>(gain)[c4];       // not needed before the reduction, but no round trip after it
+            if (part) add[u] = sum_slices4(part + row_off + 4 * c4, n_split, split_stride);
         }
     }
 #pragma unroll
@@ -381,7 +378,22 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ 
         }
     }
     ss = block_sum(ss, red);
-    const float inv = rsqrtf(ss / (float)d + eps);
+    return rsqrtf(ss / (float)d + eps);
+}
+
+template <typename T, int MAXV>
+__global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
+                               size_t split_stride, const float* __restrict__ gain, float eps,
+                               T* __restrict__ xn, const int32_t* __restrict__ row_idx, int d,
+                               uint8_t* __restrict__ xq, float* __restrict__ sx) {
+    __shared__ float red[32];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int i = blockIdx.x;
+    const int r = row_idx ? row_idx[i] : i;
+    const int nv = d >> 2;
+    float4 v[MAXV], gv[MAXV];
+    const float inv = rmsnorm_front<MAXV>(x + (size_t)r * d, part, n_split, split_stride, (size_t)r * d, nv, d, eps, gain, v, gv, red);
     if (xq) {
         // FP8 output: e4m3 codes of (value / s) with s = max |value| / 448 of this row (1 for a zero row)
         float amax = 0.f;
@@ -389,7 +401,7 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ 
         for (int u = 0; u < MAXV; ++u) {
             const int c4 = threadIdx.x + u * blockDim.x;
             if (c4 < nv) {
-                const float4 g = reinterpret_cast<const float4*>(gain)[c4];
+                const float4 g = gv[u];
                 v[u] = make_float4(v[u].x * inv * g.x, v[u].y * inv * g.y, v[u].z * inv * g.z, v[u].w * inv * g.w);
                 amax = fmaxf(fmaxf(fmaxf(amax, fabsf(v[u].x)), fmaxf(fabsf(v[u].y), fabsf(v[u].z))), fabsf(v[u].w));
             }
@@ -404,39 +416,52 @@ __global__ void rmsnorm_kernel(float* __restrict__ x, const float* __restrict__ 
         }
         return;
     }
-    if (x4.codes) {
-        // NVFP4 output of the bfloat16 rounding of the normalised row: row scale max / (6 * 448), then blocks of 16
-        float amax = 0.f;
-#pragma unroll
-        for (int u = 0; u < MAXV; ++u) {
-            const int c4 = threadIdx.x + u * blockDim.x;
-            if (c4 < nv) {
-                const float4 g = reinterpret_cast<const float4*>(gain)[c4];
-                v[u] = make_float4(wdk::bf16_round_f(v[u].x * inv * g.x), wdk::bf16_round_f(v[u].y * inv * g.y),
-                                   wdk::bf16_round_f(v[u].z * inv * g.z), wdk::bf16_round_f(v[u].w * inv * g.w));
-                amax = fmaxf(fmaxf(fmaxf(amax, fabsf(v[u].x)), fmaxf(fabsf(v[u].y), fabsf(v[u].z))), fabsf(v[u].w));
-            } else {
-                v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-        }
-        amax = block_max(amax, red);
-        const float gr = amax > 0.f ? __fdiv_rn(amax, 6.0f * 448.0f) : 1.f;
-        if (threadIdx.x == 0) x4.g[i] = gr;
-#pragma unroll
-        for (int u = 0; u < MAXV; ++u) {
-            const int c4 = threadIdx.x + u * blockDim.x;
-            wdk::nvfp4_emit4(v[u], gr, c4 < nv, x4.codes + (size_t)i * (d >> 1), x4.sf + (size_t)i * (d >> 4), c4);
-        }
-        return;
-    }
 #pragma unroll
     for (int u = 0; u < MAXV; ++u) {
         const int c4 = threadIdx.x + u * blockDim.x;
         if (c4 < nv) {
-            const float4 g = reinterpret_cast<const float4*>(gain)[c4];
+            const float4 g = gv[u];
             Vec4<T>::store(xn + (size_t)i * d + 4 * c4, v[u].x * inv * g.x, v[u].y * inv * g.y, v[u].z * inv * g.z,
                            v[u].w * inv * g.w);
         }
+    }
+}
+
+// The same with NVFP4 output of the bfloat16 rounding of the normalised row (a kernel of its own, so that the
+// bf16 path's kernel carries neither its arguments nor its code): row scale max / (6 * 448), then blocks of 16
+// elements held by four neighbouring lanes.  d % 16 == 0.
+template <int MAXV>
+__global__ void __launch_bounds__(1024) rmsnorm_fp4_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
+                                   size_t split_stride, const float* __restrict__ gain, float eps,
+                                   const int32_t* __restrict__ row_idx, int d, WdFp4Operand x4) {
+    __shared__ float red[32];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int i = blockIdx.x;
+    const int r = row_idx ? row_idx[i] : i;
+    const int nv = d >> 2;
+    float4 v[MAXV], gv[MAXV];
+    const float inv = rmsnorm_front<MAXV>(x + (size_t)r * d, part, n_split, split_stride, (size_t)r * d, nv, d, eps, gain, v, gv, red);
+    float amax = 0.f;
+#pragma unroll
+    for (int u = 0; u < MAXV; ++u) {
+        const int c4 = threadIdx.x + u * blockDim.x;
+        if (c4 < nv) {
+            const float4 g = gv[u];
+            v[u] = make_float4(wdk::bf16_round_f(v[u].x * inv * g.x), wdk::bf16_round_f(v[u].y * inv * g.y),
+                               wdk::bf16_round_f(v[u].z * inv * g.z), wdk::bf16_round_f(v[u].w * inv * g.w));
+            amax = fmaxf(fmaxf(fmaxf(amax, fabsf(v[u].x)), fmaxf(fabsf(v[u].y), fabsf(v[u].z))), fabsf(v[u].w));
+        } else {
+            v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+    }
+    amax = block_max(amax, red);
+    const float gr = amax > 0.f ? __fdiv_rn(amax, 6.0f * 448.0f) : 1.f;
+    if (threadIdx.x == 0) x4.g[i] = gr;
+#pragma unroll
+    for (int u = 0; u < MAXV; ++u) {
+        const int c4 = threadIdx.x + u * blockDim.x;
+        wdk::nvfp4_emit4(v[u], gr, c4 < nv, x4.codes + (size_t)i * (d >> 1), x4.sf + (size_t)i * (d >> 4), c4);
     }
 }
 
@@ -521,11 +546,13 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
                 // four rotation pairs per thread (float4 loads, 8-byte bf16 stores): half/4 threads per head
                 const int tph = half >> 2, hpb = blockDim.x / tph;
                 const int h = grp * hpb + (int)threadIdx.x / tph, j = ((int)threadIdx.x % tph) * 4;
-                if ((int)threadIdx.x < hpb * tph && h < Hq + Hkv && (h < Hq || in_range)) {
+                // (the loads do not wait for the index check: only the store of a cache row does)
+                if ((int)threadIdx.x < hpb * tph && h < Hq + Hkv) {
                     const float4 a = sum_slices4(pr + h * dh + j, n_split, split_stride);
                     const float4 bb = sum_slices4(pr + h * dh + half + j, n_split, split_stride);
                     const float4 c01 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j);       // (cos, sin) x 2
                     const float4 c23 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j + 2);
+                    if (h >= Hq && !in_range) continue;
                     T* dst = h < Hq ? q + ((size_t)r * Hq + h) * dh : kcache + (((size_t)b * Hkv + (h - Hq)) * S + pos) * dh;
                     Vec4<T>::store(dst + j, a.x * c01.x - bb.x * c01.y, a.y * c01.z - bb.y * c01.w, a.z * c23.x - bb.z * c23.y,
                                    a.w * c23.z - bb.w * c23.w);
@@ -556,6 +583,8 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
     const int d0 = (rem / rchunks) * 32, r0 = (rem % rchunks) * 32;
     const int lx = threadIdx.x & 31, ly = threadIdx.x >> 5;
     const int vcol = (Hq + Hkv) * dh + kh * dh + d0;
+    const int r_out = r0 + lx;                                   // the row this thread writes after the transpose
+    const int pos_out = r_out < n_rows ? row_pos[r_out] : 0, b_out = r_out < n_rows ? row_seq[r_out] : 0;
     if ((dh & 3) == 0) {
         // one float4 (four head dims of one row) per thread
         const int rr = threadIdx.x >> 3, d4 = (threadIdx.x & 7) * 4, r = r0 + rr;
@@ -570,9 +599,9 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
         }
     }
     __syncthreads();
-    const int r = r0 + lx;
+    const int r = r_out;
     if (r < n_rows) {
-        const int pos = row_pos[r], b = row_seq[r];
+        const int pos = pos_out, b = b_out;
         if ((unsigned)pos < (unsigned)S && (unsigned)b < (unsigned)batch) {
             T* dst = vcache + ((size_t)b * Hkv + kh) * dh * Sp + pos;
             for (int dd = ly; dd < 32 && d0 + dd < dh; dd += 8) dst[(size_t)(d0 + dd) * Sp] = from_f<T>(tile[lx][dd]);
@@ -694,19 +723,14 @@ __global__ void swiglu_kernel(const float* __restrict__ part, int n_split, size_
 // and waiting while the GEMM still runs); each keeps its quarter of h = silu(gate) * up in registers
 // (up to kMaxV float4 per thread), the four partial maxima meet through distributed shared memory,
 // then every block writes the e4m3 codes of its quarter (and block 0 the row's scale).
-// kFp4: NVFP4 output of the bfloat16 rounding of h instead (codes, block scales and row scale in h4; F % 64 == 0).
-template <int kMaxV, bool kFp4>
-__global__ void swiglu_fp8_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
-                                  uint8_t* __restrict__ hq, float* __restrict__ sh, int F, WdFp4Operand h4) {
-    __shared__ float red[32];
-    __shared__ float my_max;
-    pdl_launch_dependents();
-    pdl_wait();
-    const int r = blockIdx.x >> 2, quarter = blockIdx.x & 3, f4 = F >> 2;
-    const int q4 = (f4 + 3) >> 2, c_lo = quarter * q4, c_hi = min(f4, c_lo + q4);     // this block's float4 columns
+// The front of the quantising SwiGLU kernels: this block's quarter of h = silu(gate) * up of row r in g[] (fp32,
+// or rounded to bfloat16 when kRound), returns the row's maximum |h| (over the four blocks of the cluster).
+template <int kMaxV, bool kRound>
+__device__ __forceinline__ float swiglu_quarter(const float* __restrict__ part, int n_split, size_t split_stride, int F,
+                                                int r, int c_lo, int c_hi, float4 (&g)[kMaxV], float* red, float* my_max) {
     const float* pr = part + (size_t)r * 2 * F;
     // slice by slice, all of this thread's positions at once: 2 * kMaxV loads in flight per round trip
-    float4 g[kMaxV], up[kMaxV];
+    float4 up[kMaxV];
 #pragma unroll
     for (int u = 0; u < kMaxV; ++u) g[u] = up[u] = make_float4(0.f, 0.f, 0.f, 0.f);
     for (int sl = 0; sl < n_split; ++sl) {
@@ -732,36 +756,61 @@ __global__ void swiglu_fp8_kernel(const float* __restrict__ part, int n_split, s
     for (int u = 0; u < kMaxV; ++u) {
         g[u] = make_float4(g[u].x / (1.f + __expf(-g[u].x)) * up[u].x, g[u].y / (1.f + __expf(-g[u].y)) * up[u].y,
                            g[u].z / (1.f + __expf(-g[u].z)) * up[u].z, g[u].w / (1.f + __expf(-g[u].w)) * up[u].w);
-        if (kFp4)
+        if (kRound)
             g[u] = make_float4(wdk::bf16_round_f(g[u].x), wdk::bf16_round_f(g[u].y), wdk::bf16_round_f(g[u].z), wdk::bf16_round_f(g[u].w));
         amax = fmaxf(fmaxf(fmaxf(amax, fabsf(g[u].x)), fmaxf(fabsf(g[u].y), fabsf(g[u].z))), fabsf(g[u].w));
     }
     amax = block_max(amax, red);
-    if (threadIdx.x == 0) my_max = amax;
+    if (threadIdx.x == 0) *my_max = amax;
     wdk::cluster_sync();                            // the four partial maxima are in place
-    const uint32_t local = wdk::smem_u32(&my_max);
+    const uint32_t local = wdk::smem_u32(my_max);
     for (uint32_t k = 0; k < 4; ++k) {
         float v;
         asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(wdk::cluster_map(local, k)));
         amax = fmaxf(amax, v);
     }
     wdk::cluster_sync();                            // nobody leaves while its maximum may still be read
-    if (kFp4) {
-        const float gr = amax > 0.f ? __fdiv_rn(amax, 6.0f * 448.0f) : 1.f;
-        if (threadIdx.x == 0 && quarter == 0) h4.g[r] = gr;
-#pragma unroll
-        for (int u = 0; u < kMaxV; ++u) {
-            const int c4 = c_lo + (int)threadIdx.x + u * (int)blockDim.x;
-            wdk::nvfp4_emit4(g[u], gr, c4 < c_hi, h4.codes + (size_t)r * (F >> 1), h4.sf + (size_t)r * (F >> 4), c4);
-        }
-        return;
-    }
+    return amax;
+}
+
+template <int kMaxV>
+__global__ void swiglu_fp8_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
+                                  uint8_t* __restrict__ hq, float* __restrict__ sh, int F) {
+    __shared__ float red[32];
+    __shared__ float my_max;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int r = blockIdx.x >> 2, quarter = blockIdx.x & 3, f4 = F >> 2;
+    const int q4 = (f4 + 3) >> 2, c_lo = quarter * q4, c_hi = min(f4, c_lo + q4);     // this block's float4 columns
+    float4 g[kMaxV];
+    const float amax = swiglu_quarter<kMaxV, false>(part, n_split, split_stride, F, r, c_lo, c_hi, g, red, &my_max);
     const float s = amax > 0.f ? amax / 448.f : 1.f;
     if (threadIdx.x == 0 && quarter == 0) sh[r] = s;
 #pragma unroll
     for (int u = 0; u < kMaxV; ++u) {
         const int c4 = c_lo + (int)threadIdx.x + u * (int)blockDim.x;
         if (c4 < c_hi) reinterpret_cast<uint32_t*>(hq + (size_t)r * F)[c4] = pack_e4m3(g[u].x / s, g[u].y / s, g[u].z / s, g[u].w / s);
+    }
+}
+
+// NVFP4 variant: the bfloat16 rounding of h as codes, block scales and row scale (F % 64 == 0, so that every
+// block's quarter is a whole number of 16-element blocks held by four neighbouring lanes).
+template <int kMaxV>
+__global__ void swiglu_fp4_kernel(const float* __restrict__ part, int n_split, size_t split_stride, int F, WdFp4Operand h4) {
+    __shared__ float red[32];
+    __shared__ float my_max;
+    pdl_launch_dependents();
+    pdl_wait();
+    const int r = blockIdx.x >> 2, quarter = blockIdx.x & 3, f4 = F >> 2;
+    const int q4 = (f4 + 3) >> 2, c_lo = quarter * q4, c_hi = min(f4, c_lo + q4);
+    float4 g[kMaxV];
+    const float amax = swiglu_quarter<kMaxV, true>(part, n_split, split_stride, F, r, c_lo, c_hi, g, red, &my_max);
+    const float gr = amax > 0.f ? __fdiv_rn(amax, 6.0f * 448.0f) : 1.f;
+    if (threadIdx.x == 0 && quarter == 0) h4.g[r] = gr;
+#pragma unroll
+    for (int u = 0; u < kMaxV; ++u) {
+        const int c4 = c_lo + (int)threadIdx.x + u * (int)blockDim.x;
+        wdk::nvfp4_emit4(g[u], gr, c4 < c_hi, h4.codes + (size_t)r * (F >> 1), h4.sf + (size_t)r * (F >> 4), c4);
     }
 }
 
@@ -965,25 +1014,40 @@ void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size
                        const float* gain, float eps, void* xn, const int32_t* row_idx, int n_rows,
                        int d, cudaStream_t st, uint8_t* xq, float* sx, const WdFp4Operand* x4p) {
     if (n_rows <= 0) return;
-    const WdFp4Operand x4 = x4p ? *x4p : WdFp4Operand();
     // one float4 per thread where the row allows it: the kernel is a chain of dependent L2 round
     // trips, so short per-thread work matters more than occupancy
     const int nv = d >> 2;
+    if (x4p) {
+        const WdFp4Operand x4 = *x4p;
+        if (n_rows >= 512 && nv >= 256 && nv <= 4096)
+            launch_pdl(rmsnorm_fp4_kernel<4>, dim3(n_rows), dim3(((nv + 3) / 4 + 31) / 32 * 32), 0, st, x, part, n_split,
+                       split_stride, gain, eps, row_idx, d, x4);
+        else if (nv <= 1024)
+            launch_pdl(rmsnorm_fp4_kernel<1>, dim3(n_rows), dim3((nv + 31) / 32 * 32), 0, st, x, part, n_split, split_stride,
+                       gain, eps, row_idx, d, x4);
+        else if (nv <= 2048)
+            launch_pdl(rmsnorm_fp4_kernel<2>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split, split_stride, gain, eps,
+                       row_idx, d, x4);
+        else
+            launch_pdl(rmsnorm_fp4_kernel<8>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split, split_stride, gain, eps,
+                       row_idx, d, x4);
+        return;
+    }
     if (n_rows >= 512 && nv >= 256 && nv <= 4096) {
         // many rows: bandwidth matters, so more (smaller) blocks per SM with four float4 in flight per thread
         const int threads = ((nv + 3) / 4 + 31) / 32 * 32;
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 4>, dim3(n_rows), dim3(threads), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx, x4));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
     } else if (nv <= 1024) {
         const int threads = (nv + 31) / 32 * 32;
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 1>, dim3(n_rows), dim3(threads), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx, x4));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
     } else if (nv <= 2048) {
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 2>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx, x4));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
     } else {
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_kernel<T, 8>, dim3(n_rows), dim3(1024), 0, st, x, part, n_split,
-                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx, x4));
+                                      split_stride, gain, eps, (T*)xn, row_idx, d, xq, sx));
     }
 }
 
@@ -1063,13 +1127,13 @@ static wd_status launch_swiglu_quant(const float* part, int n_split, size_t spli
     const int per_thread = ((f4 + 3) / 4 + 255) / 256;          // float4 per thread
     cudaError_t e;
     if (h4p) {
-        if (per_thread <= 3) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<3, true>, part, n_split, split_stride, hq, sh, F, h4);
-        else if (per_thread <= 5) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<5, true>, part, n_split, split_stride, hq, sh, F, h4);
-        else e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<8, true>, part, n_split, split_stride, hq, sh, F, h4);
+        if (per_thread <= 3) e = cudaLaunchKernelEx(&lc, swiglu_fp4_kernel<3>, part, n_split, split_stride, F, h4);
+        else if (per_thread <= 5) e = cudaLaunchKernelEx(&lc, swiglu_fp4_kernel<5>, part, n_split, split_stride, F, h4);
+        else e = cudaLaunchKernelEx(&lc, swiglu_fp4_kernel<8>, part, n_split, split_stride, F, h4);
     } else {
-        if (per_thread <= 3) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<3, false>, part, n_split, split_stride, hq, sh, F, h4);
-        else if (per_thread <= 5) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<5, false>, part, n_split, split_stride, hq, sh, F, h4);
-        else e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<8, false>, part, n_split, split_stride, hq, sh, F, h4);
+        if (per_thread <= 3) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<3>, part, n_split, split_stride, hq, sh, F);
+        else if (per_thread <= 5) e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<5>, part, n_split, split_stride, hq, sh, F);
+        else e = cudaLaunchKernelEx(&lc, swiglu_fp8_kernel<8>, part, n_split, split_stride, hq, sh, F);
     }
     if (e != cudaSuccess) { wd_note_cuda_error(e, __FILE__, __LINE__); return WD_ERR_CUDA; }
     return WD_OK;
