@@ -84,6 +84,8 @@ SIGNATURES = {
     "wd_plan": (C.c_int, [vp, i32, i32, i32, i32, i32, C.POINTER(wd_index_sets)]),
     "wd_plan_raw": (C.c_int, [u8p, i32p, i32p, i32, i32, i32, i32, i32p, i32, i32, i32, i32, i32, i32, i32, i32,
                               C.POINTER(wd_index_sets)]),
+    "wd_set_graphs": (C.c_int, [vp, i32]),
+    "wd_debug_graph_stats": (C.c_int, [vp, C.POINTER(i32), C.POINTER(i32)]),
     "wd_fp8_bytes": (C.c_size_t, [C.POINTER(wd_model_dims)]),
     "wd_fp8_enable": (C.c_int, [vp, vp, C.c_size_t, vp]),
     "wd_fp8_set": (C.c_int, [vp, i32]),
@@ -235,6 +237,15 @@ class Context:
 
     def profile_enable(self, on: bool):
         check(lib().wd_profile_enable(self.handle, 1 if on else 0), "wd_profile_enable")
+
+    def set_graphs(self, on: bool):
+        check(lib().wd_set_graphs(self.handle, 1 if on else 0), "wd_set_graphs")
+
+    def graph_stats(self):
+        """(graphs recorded, steps replayed) since the context was created."""
+        a, b = i32(0), i32(0)
+        check(lib().wd_debug_graph_stats(self.handle, C.byref(a), C.byref(b)), "wd_debug_graph_stats")
+        return a.value, b.value
 
     def fp8_enable(self, stream=None):
         """wd_fp8_enable: quantise the weights to e4m3 and run the projections in FP8 from now on."""

@@ -229,6 +229,50 @@ def test_nvfp4_mode_differs_from_bf16_and_excludes_fp8():
     ctx.close()
 
 
+@pytest.mark.parametrize("mode", ["bf16", "fp8", "fp4"])
+def test_step_graphs_replay_gives_the_same_generation(mode):
+    """Steps replayed from a CUDA graph (wd_set_graphs, the default) run the same kernels with the same
+    arguments as steps launched directly: token ids, confidences, per-step launch counts and step shapes of a
+    whole generation are identical, graphs really are recorded and replayed, and a context with graphs off
+    records none."""
+    cfg = synth.get_config("llada8b", **dict(DH128, batch=2, G=96))
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    S = ids.shape[1]
+    runs = []
+    stream = torch.cuda.Stream(device=DEV)         # (the legacy default stream cannot record graphs)
+    for on in (False, True):
+        ctx = wd.Context(cfg, w, 2, S, 2 * S, 2 * cfg["A"])
+        ctx.set_graphs(on)
+        if mode == "fp8":
+            ctx.fp8_enable()
+        if mode == "fp4":
+            ctx.fp4_enable()
+        st = wd.State(ctx, ids)
+        infos, outs = [], []
+        for i in range(200):
+            status, info = st.step(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"], stream)
+            if status == wd.WD_DONE:
+                break
+            infos.append((info["is_refresh"], info["n_rows"], info["n_active"], info["n_vis"], info["n_launches"]))
+            if i % 5 == 4:                 # a few steps queue up between syncs
+                outs += st.sync_all()
+        outs += st.sync_all()
+        final = [st.read(b)["ids"].copy() for b in range(2)]
+        runs.append((infos, outs, final, ctx.graph_stats()))
+        st.close()
+        ctx.close()
+    (i0, o0, f0, g0), (i1, o1, f1, g1) = runs
+    assert i0 == i1 and len(i0) == 96 // cfg["k"]
+    assert all(np.array_equal(a, b) for a, b in zip(f0, f1)) and all((f != cfg["mask_id"]).all() for f in f0)
+    assert len(o0) == len(o1)
+    for x, y in zip(o0, o1):
+        assert np.array_equal(x["positions"], y["positions"]) and np.array_equal(x["token_ids"], y["token_ids"])
+        assert np.array_equal(x["confidence"], y["confidence"])
+    assert g0 == (0, 0)
+    assert g1[0] >= 1 and g1[1] >= len(i1) // 3          # most normal steps are replays
+
+
 def test_plain_and_tensor_core_paths_agree():
     """The CUDA-core kernels and the tensor-core kernels compute the same step."""
     cfg = synth.get_config("llada8b", **DH128)
