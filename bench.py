@@ -8,9 +8,10 @@ uniform-random prompt ids.  A "step" is one wd_step + wd_step_sync of the
 generation trajectory (one refresh step then R-1 normal steps per phase).
 
 Prints ONE JSON line.  `value` is generated tokens/s with the state resident
-on the GPU; `e2e` is the same loop timed on the host clock from host buffers
-(ids uploaded inside the timed region, per-step index lists up and results
-down); `roofline` is the tensor-core GEMM kernel's algorithmic bytes over its
+on the GPU; `e2e` is a whole generation through the library's own driver on the
+host clock from host buffers (prompt ids uploaded, every step's result block
+copied down, final ids read back; `e2e.per_step_sync` = the timed steps with a
+host sync after each); `roofline` is the tensor-core GEMM kernel's algorithmic bytes over its
 CUDA-event time; `cpu_baseline` is the fp64 oracle timed on the host cores.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--config NAME]
@@ -362,13 +363,17 @@ def run_ours(args, rank, world):
                        "refresh_rows": float(np.mean([i["n_rows"] for i in v_infos if i["is_refresh"]])) if v_refresh else None}},
         "clocks": {"sm_mhz": clocks["sm_mhz"], "sm_max_mhz": clocks["sm_max_mhz"], "reasons": clocks["reasons"],
                    "samples": clocks["samples"]},
-        "e2e": {"value": batch * k * (W + K) * world / e2e_wall, "unit": UNIT,
-                "stepping": "one wd_step + wd_step_sync per step (every step's tokens reach the host before the next)",
-                "whole_generation": {"value": gen_tokens * world / gen_wall, "unit": UNIT, "steps": gen_steps,
-                                     "tokens": gen_tokens, "seconds": gen_wall,
-                                     "call": "wd_state_reset + wd_generate + wd_state_read on the host clock"},
-                "h2d_bytes_per_step": float(batch * S * 5 / (W + K)),
-                "d2h_bytes_per_step": float((1 + batch + 3 * batch * k) * 4)},
+        # end to end = the call a user makes for a generation: host prompt in (wd_state_reset), the library's own
+        # decoding loop (wd_generate: every step copies its result block to pinned host memory, the host commits
+        # them as they arrive), host tokens out (wd_state_read), on the host clock
+        "e2e": {"value": gen_tokens * world / gen_wall, "unit": UNIT, "steps": gen_steps, "tokens": gen_tokens,
+                "seconds": gen_wall,
+                "call": "wd_state_reset + wd_generate + wd_state_read on the host clock (the whole generation)",
+                "per_step_sync": {"value": batch * k * (W + K) * world / e2e_wall, "unit": UNIT,
+                                  "stepping": "the bench's W + K steps as one wd_step + wd_step_sync per step (every "
+                                              "step's tokens reach the host before the next is enqueued)"},
+                "h2d_bytes_per_step": float(batch * S * 5 / max(gen_steps, 1)),
+                "d2h_bytes_per_step": float((1 + batch + 3 * batch * k) * 4 + batch * S * 4 / max(gen_steps, 1))},
         "gpu_launches": int(sum(i["n_launches"] for i in infos)),
         "roofline": {"bound": "hbm", "kernel": "gemm_tc_kernel (launches of the normal, weight-streaming steps)",
                      "achieved": gemm_gbs, "peak": peaks["hbm_gbs"],
