@@ -1474,7 +1474,10 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     // graph.  With an empty queue (a caller that syncs after every step) direct launches win, because the GPU
     // starts on the first kernels while the host is still launching the later ones (measured: 230 against 227
     // tokens/s end to end).
-    if (c->graphs_on && dev_mode && !c->prof_on && !taps_on && !fused && !stream_capturing && use_tc(c) && all_contig &&
+    // The tensor-core attention only: the index-list kernel sizes its shared memory by the exact visible count,
+    // which a recorded launch would keep while the count grows.
+    const bool attn_by_tc = st->attn_tc && all_contig && c->attn_impl != WD_GEMM_PLAIN;
+    if (c->graphs_on && dev_mode && !c->prof_on && !taps_on && !fused && !stream_capturing && use_tc(c) && attn_by_tc &&
         !st->queue.empty()) {
         wd_ctx::StepKey key;
         key.state_uid = st->uid; key.batch = batch; key.rows = R_; key.n_act = NA; key.n_qtiles = (int)n_qtiles;

@@ -273,6 +273,23 @@ def test_step_graphs_replay_gives_the_same_generation(mode):
     assert g1[0] >= 1 and g1[1] >= len(i1) // 3          # most normal steps are replays
 
 
+def test_step_graphs_stay_off_without_the_tensor_core_attention():
+    """head_dim 64 runs the index-list attention kernel, whose launch depends on the exact visible count: such
+    steps are never recorded (and the generation still completes, queued steps and all)."""
+    cfg = synth.get_config("llada8b", **dict(SMALL_BF16, G=40))
+    w = synth.make_weights(cfg, DEV)
+    ids = synth.make_prompts(cfg)
+    S = ids.shape[1]
+    ctx = wd.Context(cfg, w, 1, S, S, cfg["A"])
+    st = wd.State(ctx, ids)
+    stream = torch.cuda.Stream(device=DEV)
+    status, steps, tokens = st.generate(cfg["A"], cfg["B"], cfg["R"], cfg["T"], cfg["k"], 0, stream)
+    assert tokens == 40 and (st.read(0)["ids"] != cfg["mask_id"]).all()
+    assert ctx.graph_stats() == (0, 0)
+    st.close()
+    ctx.close()
+
+
 def test_plain_and_tensor_core_paths_agree():
     """The CUDA-core kernels and the tensor-core kernels compute the same step."""
     cfg = synth.get_config("llada8b", **DH128)
