@@ -1246,12 +1246,13 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         wd_fp4_operand_split(c->fp4_x, R_, F, &x4_f);
         wd_fp4_operand_split(c->fp4_x, NA, D, &x4_lm);
     }
+    size_t attn_smem = 0;               // shared memory of an attention CTA (tensor-core form), for the projection after it
     auto attention = [&](int l, char* kc, char* vc) -> wd_status {
         float* attn_tap = st->taps.attn_out ? st->taps.attn_out + (size_t)l * R_ * hq : nullptr;
         if (st->attn_tc && all_contig && c->attn_impl != WD_GEMM_PLAIN)
             return wd_attn_tc_launch(c->q, R_, (int)n_qtiles, c->plan + o_qt_seq, c->plan + o_qt_row0, c->plan + o_qt_n,
                                      c->plan + o_nvis, &st->map_k, &st->map_vt, c->attn, attn_tap, Hq, Hkv, dh, l, max_vis,
-                                     c->sm_count, status, stream, max_tile_rows);
+                                     c->sm_count, status, stream, max_tile_rows, &attn_smem);
         wd_launch_attention_plain(d.dtype, c->q, kc, vc, row_seq, vis_idx, vis_off, c->attn, attn_tap, R_, max_vis, Hq,
                                   Hkv, dh, S, Sp, batch, status, stream);
         return WD_OK;
@@ -1371,6 +1372,11 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         wd_launch_rope_scatter(d.dtype, c->part, go.n_split, go.split_stride, row_seq, row_pos, c->rope_tab, c->q, kc,
                                vc, R_, Hq, Hkv, dh, S, Sp, batch, status, stream);
         if ((s = attention(l, kc, vc)) != WD_OK) return s;
+        // the output projection's CTAs beside the attention's (when those take less than half an SM's shared
+        // memory): a shorter ring, but its weights are on their way while the attention still runs
+        // (measured: 215 KB for the two CTAs together still fits an SM, 222 KB does not)
+        c->tc.x_map_attn.smem_cap = (attn_smem > 0 && attn_smem <= 110 * 1024 && R_ <= 128) ? (int)(223232 - attn_smem) : 0;
+        if (getenv("WD_WO_CAP")) c->tc.x_map_attn.smem_cap = atoi(getenv("WD_WO_CAP"));
         WdTcSeg wo[1] = {{c->wo[l], D, c->tc.get(WD_TC_WO, l)}};
         if ((s = run_gemm(c, c->attn, &c->tc.x_map_attn, wo, 1, R_, hq, c->part, c->part_floats, status, stream, &go)) != WD_OK)
             return s;

@@ -102,16 +102,27 @@ constexpr int kQFull = 0, kKFull = 1, kKEmpty = 4, kVFull = 7, kVEmpty = 10, kSF
               kOEmpty = 19;
 constexpr int kStages = 3;                 // K stages and V stages
 
-__global__ void __launch_bounds__(kThreads, 1)
-attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                    const __grid_constant__ CUtensorMap map_vt, const AttnParams p) {
+// kSingle: every CTA has at most one key tile (few keys, or keys split finely over the cluster): one K and one
+// V stage, one S and one O buffer (256 tensor-memory columns), no running rescale — 97 KB of shared memory
+// instead of 225 KB and fewer registers, so that the CTAs of the next kernel (the output projection, with a
+// ring cut to fit) can be resident beside it and fetch their weights while the attention runs.
+#ifdef WD_GEMM_TRACE
+__device__ unsigned long long g_attn_end[64];       // latest CTA exit per layer
+#endif
+
+template <bool kSingle>
+__device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_q, const CUtensorMap& map_k, const CUtensorMap& map_vt,
+                                                  const AttnParams& p) {
+    constexpr int NS = kSingle ? 1 : kStages;
+    constexpr uint32_t kCols = kSingle ? 256u : (uint32_t)kTmemCols;
+    constexpr uint32_t kOBase = kSingle ? (uint32_t)kTile : (uint32_t)(2 * kTile);     // first column of the O buffers
     extern __shared__ uint8_t smem_raw[];
     // the same offset in every CTA of the cluster (the dynamic window starts at the same address)
     uint8_t* smem = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
     uint8_t* sQ = smem;                          // 32 KB
     uint8_t* sK = smem + kOperand;               // 3 stages x 32 KB
-    uint8_t* sV = sK + kStages * kOperand;       // 3 stages x 32 KB (transposed V tiles)
-    uint64_t* bars = (uint64_t*)(sV + kStages * kOperand);
+    uint8_t* sV = sK + NS * kOperand;       // 3 stages x 32 KB (transposed V tiles)
+    uint64_t* bars = (uint64_t*)(sV + NS * kOperand);
     // q_full | k_full[3] | k_empty[3] | v_full[3] | v_empty[3] | s_full[2] | p_full[2] | o_full[2] | o_empty[2].
     // p_full and o_empty count the 256 softmax threads.  p_full is one barrier per S buffer, not one for all
     // tiles: the softmax threads can finish P(i+1) before the MMA thread has looked at P(i)'s barrier (it waits
@@ -126,7 +137,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
     volatile int* abort_flag = (volatile int*)(tmem_slot + 1);
     // after the last P V the K/V ring is free: this CTA's part of a split lives there
     float* part_o = (float*)sK;                            // [128 rows][128], 16-byte chunks XOR-swizzled by row
-    float* part_ml = (float*)(sK + 2 * kOperand);          // [128 rows][2] running maximum, sum
+    // [128 rows][2] running maximum, sum: behind the part's 64 KB; with one stage each that is the end of the
+    // ring, so it goes where Q was (every Q K^T has completed by then)
+    float* part_ml = kSingle ? (float*)sQ : (float*)(sK + 2 * kOperand);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int tile = blockIdx.x;
@@ -155,7 +168,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             *abort_flag = 0;
             asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         }
-        if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kTmemCols);
+        if (warp == 1) tmem_alloc(smem_u32(tmem_slot), kCols);
         tc_fence_before();
         __syncthreads();
         tc_fence_after();
@@ -179,8 +192,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             }
             const int bh = b * p.Hkv + kvh;
             auto load_k = [&](int j) -> bool {
-                const int ks = j % kStages;
-                const uint32_t ph = (uint32_t)(j / kStages) & 1u;
+                const int ks = j % NS;
+                const uint32_t ph = (uint32_t)(j / NS) & 1u;
                 const uint32_t kfull = smem_u32(&bars[kKFull + ks]);
                 if (!mbar_wait(smem_u32(&bars[kKEmpty + ks]), ph ^ 1u, abort_flag)) return false;   // stage free
                 const uint32_t sk = smem_u32(sK + (size_t)ks * kOperand);
@@ -194,8 +207,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             bool ok = load_k(0);
             for (int i = 0; i < n_kt && ok; ++i) {
                 if (i + 1 < n_kt && !(ok = load_k(i + 1))) break;
-                const int vs = i % kStages;
-                const uint32_t ph = (uint32_t)(i / kStages) & 1u;
+                const int vs = i % NS;
+                const uint32_t ph = (uint32_t)(i / NS) & 1u;
                 const uint32_t vfull = smem_u32(&bars[kVFull + vs]);
                 const uint32_t sv = smem_u32(sV + (size_t)vs * kOperand);
                 const int kv0 = (kt_begin + i) * kTile;
@@ -217,8 +230,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             bool ok = mbar_wait(smem_u32(&bars[kQFull]), 0, abort_flag);
             const uint64_t qd0 = make_sdesc(smem_u32(sQ)), qd1 = make_sdesc(smem_u32(sQ) + kAtom);
             auto issue_qk = [&](int j) -> bool {           // S[j&1] = Q K(j)^T
-                const int s = j & 1, ks = j % kStages;
-                if (!mbar_wait(smem_u32(&bars[kKFull + ks]), (uint32_t)(j / kStages) & 1u, abort_flag)) return false;   // K(j) landed
+                const int s = j & 1, ks = j % NS;
+                if (!mbar_wait(smem_u32(&bars[kKFull + ks]), (uint32_t)(j / NS) & 1u, abort_flag)) return false;   // K(j) landed
                 tc_fence_after();
                 const uint32_t sk = smem_u32(sK + (size_t)ks * kOperand);
                 const uint64_t kd0 = make_sdesc(sk), kd1 = make_sdesc(sk + kAtom);
@@ -233,16 +246,16 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             };
             ok = ok && issue_qk(0);
             for (int i = 0; i < n_kt && ok; ++i) {
-                const int s = i & 1, vs = i % kStages;
+                const int s = i & 1, vs = i % NS;
                 const uint32_t ph = (uint32_t)(i >> 1) & 1u;
                 if (i + 1 < n_kt && !(ok = issue_qk(i + 1))) break;                           // runs ahead of the softmax
-                if (!(ok = mbar_wait(smem_u32(&bars[kVFull + vs]), (uint32_t)(i / kStages) & 1u, abort_flag))) break;   // V(i) landed
+                if (!(ok = mbar_wait(smem_u32(&bars[kVFull + vs]), (uint32_t)(i / NS) & 1u, abort_flag))) break;   // V(i) landed
                 if (!(ok = mbar_wait(smem_u32(&bars[kPFull + s]), ph, abort_flag))) break;              // P(i) written
                 if (!(ok = mbar_wait(smem_u32(&bars[kOEmpty + s]), ph ^ 1u, abort_flag))) break;        // O_tile(i-2) folded
                 tc_fence_after();
                 const uint32_t sv = smem_u32(sV + (size_t)vs * kOperand);
                 const uint64_t vd0 = make_sdesc(sv), vd1 = make_sdesc(sv + kAtom);
-                const uint32_t acc = tmem_base + (uint32_t)(2 * kTile + s * kTile);
+                const uint32_t acc = tmem_base + kOBase + (uint32_t)(s * kTile);
                 const uint32_t pa = tmem_base + (uint32_t)(s * kTile);       // P(i): 64 columns over S(i)
                 // O_tile = P V: reduction over the 128 keys of the tile, 16 keys = 8 columns of P per MMA
 #pragma unroll
@@ -287,9 +300,9 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
 #pragma unroll
                 for (int c0 = 0; c0 < 64; c0 += 32) {
                     uint32_t v[32];
-                    tmem_ld32(t_row + (uint32_t)(2 * kTile + s * kTile + c_off + c0), v);
+                    tmem_ld32(t_row + kOBase + (uint32_t)(s * kTile + c_off + c0), v);
 #pragma unroll
-                    for (int c = 0; c < 32; ++c) o[c0 + c] = o[c0 + c] * alpha + __uint_as_float(v[c]);
+                    for (int c = 0; c < 32; ++c) o[c0 + c] = kSingle ? __uint_as_float(v[c]) : o[c0 + c] * alpha + __uint_as_float(v[c]);
                 }
             }
             tc_fence_before();
@@ -306,8 +319,8 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             // keys past n_vis may hold anything: zero their V columns so that 0 * garbage stays 0.
             // Thread (r, hf) owns row r (a head dim) of atom hf (keys 64*hf..) of the transposed V tile.
             if (n_keys < c_off + 64) {
-                if (!mbar_wait(smem_u32(&bars[kVFull + i % kStages]), (uint32_t)(i / kStages) & 1u, abort_flag)) *abort_flag = 1;   // V landed
-                uint8_t* vt = sV + (size_t)(i % kStages) * kOperand + hf * kAtom + r * 128;
+                if (!mbar_wait(smem_u32(&bars[kVFull + i % NS]), (uint32_t)(i / NS) & 1u, abort_flag)) *abort_flag = 1;   // V landed
+                uint8_t* vt = sV + (size_t)(i % NS) * kOperand + hf * kAtom + r * 128;
                 for (int kv = max(n_keys - c_off, 0); kv < 64; ++kv)
                     *reinterpret_cast<uint16_t*>(vt + (((kv >> 3) ^ (r & 7)) << 4) + (kv & 7) * 2) = 0;
             }
@@ -378,7 +391,7 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
             fence_proxy_async_smem();                      // the zeroed V columns -> visible to the MMA
             tc_fence_before();
             mbar_arrive(smem_u32(&bars[kPFull + s]));
-            if (i > 0) fold(i - 1, alpha_prev);
+            if (!kSingle && i > 0) fold(i - 1, alpha_prev);
             alpha_prev = alpha;
         }
         if (ok && n_kt > 0) fold(n_kt - 1, alpha_prev);
@@ -502,10 +515,33 @@ attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_cons
         __syncthreads();
         if (warp == 1) {
             tc_fence_after();
-            tmem_dealloc(tmem_base, kTmemCols);
+            tmem_dealloc(tmem_base, kCols);
         }
     }
+#ifdef WD_GEMM_TRACE
+    if (threadIdx.x == 0) atomicMax(&g_attn_end[p.layer & 63], global_ns());
+#endif
 }
+
+__global__ void __launch_bounds__(kThreads, 1)
+attention_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                    const __grid_constant__ CUtensorMap map_vt, const AttnParams p) {
+    attention_tc_body<false>(map_q, map_k, map_vt, p);
+}
+
+// (128 registers: 320 threads of this kernel and the 192 of a GEMM CTA fit the register file together)
+__global__ void __maxnreg__(128)
+attention_tc_single_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                           const __grid_constant__ CUtensorMap map_vt, const AttnParams p) {
+    attention_tc_body<true>(map_q, map_k, map_vt, p);
+}
+
+#ifdef WD_GEMM_TRACE
+extern "C" __attribute__((visibility("default"))) int wd_debug_attn_trace(unsigned long long* host /*[64]*/) {
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpyFromSymbol(host, g_attn_end, sizeof(unsigned long long) * 64);
+}
+#endif
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
@@ -558,7 +594,8 @@ wd_status wd_attn_tc_encode_cache(CUtensorMap* map_k, CUtensorMap* map_vt, const
 wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_t* qtile_seq, const int32_t* qtile_row0,
                             const int32_t* qtile_n, const int32_t* seq_nvis, const CUtensorMap* map_k,
                             const CUtensorMap* map_vt, void* out, float* tap, int Hq, int Hkv, int dh, int layer,
-                            int max_vis, int sm_count, int32_t* status, cudaStream_t stream, int max_tile_rows) {
+                            int max_vis, int sm_count, int32_t* status, cudaStream_t stream, int max_tile_rows,
+                            size_t* smem_used) {
     if (dh != kTile) return WD_ERR_BAD_PARAM;
     if (n_tiles <= 0) return WD_OK;
     EncodeTiledFn enc = get_encode();
@@ -613,10 +650,21 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     if (want > max_kt) want = max_kt;
     p.tiles_per_split = (max_kt + want - 1) / want;
     p.max_parts = (max_kt + p.tiles_per_split - 1) / p.tiles_per_split;
-    const size_t smem = (1 + 2 * kStages) * (size_t)kOperand + (kBars + 1) * 8 + 16 + 2 * kTile * 4 + 1024;
+    static const int single_on = getenv("WD_ATTN_SINGLE") ? atoi(getenv("WD_ATTN_SINGLE")) : 1;
+    const bool single = single_on && p.tiles_per_split == 1;
+    const size_t smem_of[2] = {(1 + 2 * kStages) * (size_t)kOperand + (kBars + 1) * 8 + 16 + 2 * kTile * 4 + 1024,
+                               (1 + 2) * (size_t)kOperand + (kBars + 1) * 8 + 16 + 2 * kTile * 4 + 1024};
+    const size_t smem = smem_of[single ? 1 : 0];
+    if (smem_used) *smem_used = smem;
     static bool attr_done[64] = {};     // the attribute is per device
     if (!attr_done[dev]) {
-        WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_of[0]));
+        WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_single_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_of[1]));
+        // the whole SM's shared memory although the kernel takes less than half: the output projection's CTAs are
+        // to be resident beside it, and an SM keeps its carve-out while blocks are resident
+        if (!(getenv("WD_NO_CARVEOUT") && atoi(getenv("WD_NO_CARVEOUT"))))
+            WD_CUDA_TRY(cudaFuncSetAttribute(attention_tc_single_kernel, cudaFuncAttributePreferredSharedMemoryCarveout,
+                                             cudaSharedmemCarveoutMaxShared));
         attr_done[dev] = true;
     }
     cudaLaunchConfig_t lc = {};
@@ -641,6 +689,7 @@ wd_status wd_attn_tc_launch(const void* q, int n_rows, int n_tiles, const int32_
     lc.attrs = attr;
     lc.numAttrs = n_attr;
     ++wd_launch_counter;
-    WD_CUDA_TRY(cudaLaunchKernelEx(&lc, attention_tc_kernel, mq, *map_k, *map_vt, p));
+    if (single) WD_CUDA_TRY(cudaLaunchKernelEx(&lc, attention_tc_single_kernel, mq, *map_k, *map_vt, p));
+    else WD_CUDA_TRY(cudaLaunchKernelEx(&lc, attention_tc_kernel, mq, *map_k, *map_vt, p));
     return WD_OK;
 }

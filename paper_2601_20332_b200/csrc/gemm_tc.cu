@@ -38,6 +38,7 @@ constexpr int kThreadsPair = 320;     // two-CTA kernel: 8 epilogue warps, two p
 
 struct TcParams {
     int rows, bn, kb_total, tok_tiles, n_units, n_stages, buf_cols, n_slices, aligned;
+    int trace_slot;                  // -DWD_GEMM_TRACE builds: which trace table this launch stamps
     int wide;                       // 1: a tile is 256 weight rows = two MMA halves sharing each activation box
     int tile_rows;                  // 128, or 256 when wide
     // > 1: the grid is tok_split groups of CTAs, group t working on token tile t only; the K-block
@@ -341,6 +342,14 @@ __device__ void finalize_unit(const TcParams& p, long long G, int unit, int e) {
 // kWide: two weight halves per CTA (many tokens).  kLmStats: the LM-head epilogue that reduces
 // the logits to per-row statistics.  Separate instantiations keep the plain weight-streaming
 // kernel free of the other variants' code (its issue loops are sensitive to it).
+#ifdef WD_GEMM_TRACE
+// clock stamps of the last launch per slot (q/k/v, o, gate/up, down, other): [slot][CTA][event]
+__device__ unsigned long long g_gemm_trace[8][160][8];
+#define G_STAMP(k) do { g_gemm_trace[p.trace_slot & 7][blockIdx.x < 160 ? blockIdx.x : 159][k] = global_ns(); } while (0)
+#else
+#define G_STAMP(k) do { } while (0)
+#endif
+
 template <bool kWide, bool kLmStats, bool kFp8 = false>
 __global__ void __launch_bounds__(kWide ? kThreadsWide : kThreads)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant__ CUtensorMap map_w0,
@@ -377,6 +386,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
 
     pdl_launch_dependents();      // the next kernel may start its own prologue / weight prefetch
     if (threadIdx.x == 0) {
+        G_STAMP(0);
         for (int s = 0; s < NS; ++s) {
             mbar_init(smem_u32(&bars[s]), 1);
             mbar_init(smem_u32(&bars[NS + s]), 1);
@@ -437,7 +447,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                     tma_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes) + kStageA, w.mw, smem_u32(&bars[i]),
                                      w.kb * kKE, w.n0 + kBM, pol_stream);
             }
+            G_STAMP(1);
             pdl_wait();
+            G_STAMP(2);
             Walk wx = w0;
             for (int i = 0; i < n_pre; ++i, advance(wx))
                 tma_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + stage_a, &map_x, smem_u32(&bars[i]), wx.kb * kKE,
@@ -480,6 +492,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 for (int j = 0; j < len; ++j) {
                     if (!(ok = mbar_wait(smem_u32(&bars[s]), ph, abort_flag))) break;
                     tc_fence_after();
+                    if (piece == 0 && j == 0) G_STAMP(3);
                     const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
                     const uint64_t adesc = make_sdesc(sa);
                     const uint64_t bdesc = make_sdesc(sa + stage_a);
@@ -502,6 +515,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 }
                 if (ok) umma_commit(smem_u32(&bars[2 * NS + buf]));  // this piece's accumulator complete
             }
+            G_STAMP(4);
             if (!ok) {
                 *abort_flag = 1;
                 atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
@@ -539,6 +553,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
+            if (threadIdx.x == 64 && piece == sch.n_pieces - 1) G_STAMP(5);
             float* yb = p.y + p.seg_col[u.seg] + n;
             const float sw_n = (kFp8 && n_ok) ? p.sw[u.seg][n] : 1.f;      // FP8: scale of this weight row
             const uint32_t t_acc = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)((buf + half_sel) * p.buf_cols);
@@ -664,6 +679,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
                 }
             }
         }
+        if (threadIdx.x == 64) G_STAMP(6);
         if (!ok && lane == 0) {
             *abort_flag = 1;
             atomicCAS(p.status, 0, WD_ERR_DEVICE_TIMEOUT);
@@ -685,11 +701,19 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_constant_
         tc_fence_before();
     }
     __syncthreads();
+    if (threadIdx.x == 0) G_STAMP(7);
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_base, 2u * (uint32_t)p.buf_cols);
     }
 }
+
+#ifdef WD_GEMM_TRACE
+extern "C" __attribute__((visibility("default"))) int wd_debug_gemm_trace(unsigned long long* host /*[8][160][8]*/) {
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpyFromSymbol(host, g_gemm_trace, sizeof(unsigned long long) * 8 * 160 * 8);
+}
+#endif
 
 // ------------------------------------------------------------------------------------------
 // Chain kernel: the projections between two attention calls as ONE persistent launch (few rows)
@@ -1678,8 +1702,18 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     for (int i = 0; i < nseg; ++i) wide_units += (segs[i].n + 2 * kBM - 1) / (2 * kBM);
     wide_units *= (rows + 255) / 256;
     static const int wide_min_units = env_int("WD_GEMM_WIDE_MIN_UNITS", 0);     // tuning knob; 0 = one unit per SM
-    const TcConfig cfg = pick_config(rows, !fused && !fp8 && wide_units >= (wide_min_units > 0 ? wide_min_units : sm_count),
-                                     fuse && fuse->mode == WD_FUSE_LMSTATS);
+    TcConfig cfg = pick_config(rows, !fused && !fp8 && wide_units >= (wide_min_units > 0 ? wide_min_units : sm_count),
+                               fuse && fuse->mode == WD_FUSE_LMSTATS);
+    if (x->smem_cap > 0 && cfg.smem > (size_t)x->smem_cap) {
+        // a shorter ring, so that the CTA fits beside the producer kernel's (see WdTcX::smem_cap); the plain
+        // bf16 form does not use the epilogue scratch either
+        if (!fused && !fp8) cfg.smem -= 7168;
+        const size_t per_stage = (size_t)cfg.tile_rows * kBK * 2 + (size_t)cfg.bn * kBK * 2 + 16;
+        while (cfg.n_stages > 3 && cfg.smem > (size_t)x->smem_cap) {
+            --cfg.n_stages;
+            cfg.smem -= per_stage;
+        }
+    }
     p.wide = cfg.wide;
     p.tile_rows = cfg.tile_rows;
     int tiles = 0, col = 0;
@@ -1710,6 +1744,8 @@ wd_status wd_tc_gemm(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, in
     p.W = (long long)p.n_units * p.kb_total;
     p.n_stages = cfg.n_stages;
     p.buf_cols = cfg.buf_cols;
+    // (trace builds) q/k/v, o, gate/up, down of a block by their shape; everything else in slot 4
+    p.trace_slot = nseg == 3 ? 0 : (nseg == 2 ? 2 : (lm ? 4 : (K == col ? 1 : (K > col ? 3 : 4))));
     const size_t slice = (size_t)rows * col;
     if (slice > y_floats) return WD_ERR_CAPACITY;
     // stream-K over all SMs when the partial sums fit, whole tiles per CTA otherwise

@@ -27,6 +27,9 @@ struct WdTcX {
     struct Entry { int rows, bn; CUtensorMap map; };
     mutable std::vector<Entry> cache;
     bool keep = true;        // false: one-off operand (single operations): encode on the stack, remember nothing
+    // > 0: most dynamic shared memory a CTA of the GEMM over this operand may take (fewer ring stages), so that it
+    // fits on an SM beside a CTA of the kernel that produces the operand and can fetch weights while that runs
+    mutable int smem_cap = 0;
 };
 
 struct WdTcWeights {

@@ -5,8 +5,10 @@
 // plus CUDA-core versions of the GEMM and of attention that work for any dtype
 // and any index list; the fp32 configuration runs on them entirely and the
 // bf16 tensor-core kernels are cross-checked against them.
+#include <cstdlib>
 #include <cstring>
 #include <utility>
+#include <vector>
 
 #include <cuda_fp8.h>
 
@@ -22,8 +24,24 @@ using wdk::pdl_wait;
 
 // Launch with programmatic stream serialization: the kernel may start while its predecessor
 // is still draining; it calls pdl_wait() before touching anything the predecessor wrote.
+// Every small kernel asks for the largest shared-memory carve-out although it uses next to none: an SM keeps its
+// carve-out while blocks are resident, and the next GEMM's blocks (some 200 KB each, launched early under
+// programmatic dependent launch so that they can fetch weights ahead of their dependency) become resident
+// beside a small kernel's blocks only if the SM is already configured for that much shared memory.
+static void prefer_max_shared(const void* kernel) {
+    static std::vector<std::pair<const void*, int>> done;      // (kernel, device) pairs already configured
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return; }
+    for (const auto& e : done) if (e.first == kernel && e.second == dev) return;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared) != cudaSuccess)
+        cudaGetLastError();
+    done.emplace_back(kernel, dev);
+}
+
 template <typename... KArgs, typename... Args>
 void launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st, Args&&... args) {
+    static const bool carve = !(getenv("WD_NO_CARVEOUT") && atoi(getenv("WD_NO_CARVEOUT")));
+    if (carve) prefer_max_shared((const void*)kernel);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
     cfg.blockDim = block;
@@ -79,16 +97,17 @@ __device__ __forceinline__ float block_max(float v, float* red) {
 // Sum of n_split partial-sum slices at one float4 position.  Slices are loaded eight at a time
 // before the first add so that their L2 round trips overlap (the narrow GEMMs of a few-row step leave up
 // to six); the adds keep slice order.
+template <int kWidth = 8>
 __device__ __forceinline__ float4 sum_slices4(const float* __restrict__ p, int n_split, size_t stride) {
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int s0 = 0; s0 < n_split; s0 += 8) {
-        float4 t[8];
+    for (int s0 = 0; s0 < n_split; s0 += kWidth) {
+        float4 t[kWidth];
 #pragma unroll
-        for (int k = 0; k < 8; ++k)
+        for (int k = 0; k < kWidth; ++k)
             t[k] = s0 + k < n_split ? *reinterpret_cast<const float4*>(p + (size_t)(s0 + k) * stride)
                                     : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int k = 0; k < 8; ++k) { acc.x += t[k].x; acc.y += t[k].y; acc.z += t[k].z; acc.w += t[k].w; }
+        for (int k = 0; k < kWidth; ++k) { acc.x += t[k].x; acc.y += t[k].y; acc.z += t[k].z; acc.w += t[k].w; }
     }
     return acc;
 }
@@ -685,9 +704,11 @@ __global__ void attention_plain_kernel(const T* __restrict__ q, const T* __restr
 
 // ---------------------------------------------------------------- SwiGLU
 // four columns per thread; F must be a multiple of 4
+// (Registers capped at 51: three of its blocks and a CTA of the down-projection GEMM, launched early to fetch
+// its weights, then fit an SM's register file together; the gate/up launch leaves at most four K slices.)
 template <typename T>
-__global__ void swiglu_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
-                              T* __restrict__ h, int n_rows, int F) {
+__global__ void __launch_bounds__(256, 5) swiglu_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
+                                                        T* __restrict__ h, int n_rows, int F) {
     pdl_launch_dependents();
     pdl_wait();
     const int f4 = F >> 2;
@@ -706,10 +727,10 @@ __global__ void swiglu_kernel(const float* __restrict__ part, int n_split, size_
             gb = *reinterpret_cast<const float4*>(pb);
             ub = *reinterpret_cast<const float4*>(pb + F);
         } else {
-            ga = sum_slices4(pa, n_split, split_stride);
-            ua = sum_slices4(pa + F, n_split, split_stride);
-            gb = sum_slices4(pb, n_split, split_stride);
-            ub = sum_slices4(pb + F, n_split, split_stride);
+            ga = sum_slices4<4>(pa, n_split, split_stride);
+            ua = sum_slices4<4>(pa + F, n_split, split_stride);
+            gb = sum_slices4<4>(pb, n_split, split_stride);
+            ub = sum_slices4<4>(pb + F, n_split, split_stride);
         }
         Vec4<T>::store(h + ra * F + 4 * ca, ga.x / (1.f + __expf(-ga.x)) * ua.x, ga.y / (1.f + __expf(-ga.y)) * ua.y,
                        ga.z / (1.f + __expf(-ga.z)) * ua.z, ga.w / (1.f + __expf(-ga.w)) * ua.w);
@@ -1126,6 +1147,14 @@ static wd_status launch_swiglu_quant(const float* part, int n_split, size_t spli
     lc.numAttrs = wd_pdl_enabled ? 2 : 1;
     const int per_thread = ((f4 + 3) / 4 + 255) / 256;          // float4 per thread
     cudaError_t e;
+    {
+        static const bool carve = !(getenv("WD_NO_CARVEOUT") && atoi(getenv("WD_NO_CARVEOUT")));
+        if (carve) {
+            prefer_max_shared((const void*)swiglu_fp4_kernel<3>); prefer_max_shared((const void*)swiglu_fp4_kernel<5>);
+            prefer_max_shared((const void*)swiglu_fp4_kernel<8>); prefer_max_shared((const void*)swiglu_fp8_kernel<3>);
+            prefer_max_shared((const void*)swiglu_fp8_kernel<5>); prefer_max_shared((const void*)swiglu_fp8_kernel<8>);
+        }
+    }
     if (h4p) {
         if (per_thread <= 3) e = cudaLaunchKernelEx(&lc, swiglu_fp4_kernel<3>, part, n_split, split_stride, F, h4);
         else if (per_thread <= 5) e = cudaLaunchKernelEx(&lc, swiglu_fp4_kernel<5>, part, n_split, split_stride, F, h4);
