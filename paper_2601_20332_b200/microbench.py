@@ -5,6 +5,7 @@
     python -m paper_2601_20332_b200.microbench gemm-suite [--rows 34]
     python -m paper_2601_20332_b200.microbench step --config llada8b --layers 4 [--steps 16]
     python -m paper_2601_20332_b200.microbench sweep [--A 16,32,64,128 --B 64,128,256 --R 1,4,16 --batch 1,16]
+    python -m paper_2601_20332_b200.microbench stamps --layers 4 --steps 6      (a -DWD_GEMM_TRACE build)
 
 `gemm` times y = x w^T for one shape (weights larger than L2 unless the shape is
 small; a ring of distinct weight buffers keeps every launch cold).  `step` runs
@@ -114,6 +115,46 @@ def run_step(config, layers, steps, warmup, impl):
                 rows=out[-1][0]["n_rows"])
 
 
+def run_stamps(config, layers, steps):
+    """Clock stamps of the last block's GEMM launches (a library built with -DWD_GEMM_TRACE: `WD_NVCC_FLAGS=-DWD_GEMM_TRACE
+    python -m paper_2601_20332_b200.build`): per launch and event the minimum, median and maximum over the CTAs, in
+    nanoseconds after the first CTA's dependency wait returned (output projection: after the attention kernel's last
+    CTA left)."""
+    import ctypes as C
+    lib = wd.lib()
+    if not hasattr(lib, "wd_debug_gemm_trace"):
+        raise SystemExit("this libwd.so was built without -DWD_GEMM_TRACE")
+    dev = "cuda:0"
+    cfg = synth.get_config(config, L=layers)
+    A, B, R, T, k, batch = (cfg[x] for x in ("A", "B", "R", "T", "k", "batch"))
+    S = cfg["P"] + cfg["G"]
+    w = synth.make_weights(cfg, dev)
+    ctx = wd.Context(cfg, w, batch, S, batch * S, batch * A)
+    st = wd.State(ctx, synth.make_prompts(cfg))
+    stream = torch.cuda.Stream(device=dev)
+    for _ in range(steps):
+        st.step(A, B, R, T, k, stream)
+        st.sync()
+    torch.cuda.synchronize()
+    buf = np.zeros((8, 160, 8), np.uint64)
+    lib.wd_debug_gemm_trace(buf.ctypes.data_as(C.c_void_p))
+    ab = np.zeros(64, np.uint64)
+    lib.wd_debug_attn_trace(ab.ctypes.data_as(C.c_void_p))
+    names = ["qkv", "o", "gate_up", "down"]
+    events = ["entry", "ring filled (before the wait)", "wait returned", "first stage complete", "last MMA issued",
+              "last accumulator ready", "epilogue done", "exit"]
+    out = {}
+    for slot, name in enumerate(names):
+        t = buf[slot, :148, :].astype(np.int64)
+        t = t[t[:, 0] > 0]
+        if not len(t):
+            continue
+        ref = int(ab[layers - 1]) if name == "o" and ab[layers - 1] else int(t[:, 2].min())
+        out[name] = {e: [int((t[:, i] - ref).min()), int(np.median(t[:, i] - ref)), int((t[:, i] - ref).max())]
+                     for i, e in enumerate(events)}
+    return dict(config=config, layers=layers, ctas=148, ns_min_median_max=out)
+
+
 def run_sweep(config, layers, A_list, B_list, R_list, batch_list, repeats, out_path):
     """Window sweep (benchmark configuration 5): for every (A, B, R, batch) one full phase
     (R steps) from three fast-forwarded states (0 %, 50 %, ~100 % of the masks decoded), with the
@@ -173,7 +214,7 @@ def run_sweep(config, layers, A_list, B_list, R_list, batch_list, repeats, out_p
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("mode", choices=["gemm", "gemm-fp4", "gemm-suite", "step", "sweep"])
+    ap.add_argument("mode", choices=["gemm", "gemm-fp4", "gemm-suite", "step", "sweep", "stamps"])
     ap.add_argument("--rows", type=int, default=34)
     ap.add_argument("--n", type=int, default=24576)
     ap.add_argument("--k", type=int, default=4096)
@@ -194,6 +235,8 @@ def main():
     impl = wd.WD_GEMM_PLAIN if a.plain else wd.WD_GEMM_TCGEN05
     if a.mode == "gemm":
         print(json.dumps(time_gemm(a.rows, a.n, a.k, a.iters, impl)))
+    elif a.mode == "stamps":
+        print(json.dumps(run_stamps(a.config, a.layers, a.steps)))
     elif a.mode == "gemm-fp4":
         print(json.dumps(time_gemm_fp4(a.rows, a.n, a.k, a.iters)))
     elif a.mode == "gemm-suite":
