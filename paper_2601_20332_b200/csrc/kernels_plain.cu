@@ -22,6 +22,37 @@ namespace {
 using wdk::pdl_launch_dependents;
 using wdk::pdl_wait;
 
+#ifdef WD_GEMM_TRACE
+// development clock stamps of the small kernels: every block appends (kind, wait returned, exit) to a ring
+__device__ unsigned long long g_small_trace[16384][4];
+__device__ unsigned int g_small_idx;
+struct SmallStamp {
+    unsigned long long t0, tm;
+    int kind;
+    __device__ SmallStamp(int k) : t0(0), tm(0), kind(k) { if (threadIdx.x == 0) t0 = wdk::global_ns(); }
+    __device__ void mid() { if (threadIdx.x == 0) tm = wdk::global_ns(); }
+    __device__ ~SmallStamp() {
+        if (threadIdx.x == 0) {
+            const unsigned int i = atomicAdd(&g_small_idx, 1u) & 16383u;
+            g_small_trace[i][0] = (unsigned long long)kind;
+            g_small_trace[i][1] = t0;
+            g_small_trace[i][2] = wdk::global_ns();
+            g_small_trace[i][3] = tm;
+        }
+    }
+};
+#define S_STAMP(kind) SmallStamp small_stamp_(kind)
+#define S_MID() small_stamp_.mid()
+extern "C" __attribute__((visibility("default"))) int wd_debug_small_trace(unsigned long long* host /*[16384][4]*/, unsigned int* idx) {
+    cudaDeviceSynchronize();
+    cudaMemcpyFromSymbol(idx, g_small_idx, sizeof(unsigned int));
+    return (int)cudaMemcpyFromSymbol(host, g_small_trace, sizeof(unsigned long long) * 16384 * 4);
+}
+#else
+#define S_STAMP(kind) do { } while (0)
+#define S_MID() do { } while (0)
+#endif
+
 // Launch with programmatic stream serialization: the kernel may start while its predecessor
 // is still draining; it calls pdl_wait() before touching anything the predecessor wrote.
 // Every small kernel asks for the largest shared-memory carve-out although it uses next to none: an SM keeps its
@@ -108,6 +139,27 @@ __device__ __forceinline__ float4 sum_slices4(const float* __restrict__ p, int n
                                     : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int k = 0; k < kWidth; ++k) { acc.x += t[k].x; acc.y += t[k].y; acc.z += t[k].z; acc.w += t[k].w; }
+    }
+    return acc;
+}
+// The same with the loads pinned in program order (volatile), so that up to eight of them are in flight before the
+// first add whatever the compiler would rather do with its registers: for kernels that are one L2 round trip long.
+__device__ __forceinline__ float4 ld_f4_pinned(const float* p) {
+    float4 v;
+    asm volatile("ld.global.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ float4 sum_slices4_pinned(const float* __restrict__ p, int n_split, size_t stride) {
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s0 = 0; s0 < n_split; s0 += 8) {
+        float4 t[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            t[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (s0 + k < n_split) t[k] = ld_f4_pinned(p + (size_t)(s0 + k) * stride);
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) { acc.x += t[k].x; acc.y += t[k].y; acc.z += t[k].z; acc.w += t[k].w; }
     }
     return acc;
 }
@@ -367,7 +419,7 @@ __device__ __forceinline__ uint32_t pack_e4m3(float a, float b, float c, float d
 
 // The front of the RMSNorm kernels: x += sum of the partial slices (if any), v = the row's float4 of this
 // thread, returns 1 / rms of the row.
-template <int MAXV>
+template <int MAXV, bool kPinned = false>
 __device__ __forceinline__ float rmsnorm_front(float* __restrict__ xr, const float* __restrict__ part, int n_split,
                                                size_t split_stride, size_t row_off, int nv, int d, float eps,
                                                const float* __restrict__ gain, float4 (&v)[MAXV], float4 (&gv)[MAXV],
@@ -378,9 +430,16 @@ __device__ __forceinline__ float rmsnorm_front(float* __restrict__ xr, const flo
     for (int u = 0; u < MAXV; ++u) {             // all loads first: x, the gains and every slice of every group
         const int c4 = threadIdx.x + u * blockDim.x;
         if (c4 < nv) {
-            v[u] = reinterpret_cast<const float4*>(xr)[c4];
-            gv[u] = reinterpret_cast<const float4*>(gain)[c4];       // not needed before the reduction, but no round trip after it
-            if (part) add[u] = sum_slices4(part + row_off + 4 * c4, n_split, split_stride);
+            if (kPinned) {
+                // few rows: row, gains and every slice in flight together
+                v[u] = ld_f4_pinned(xr + 4 * c4);
+                gv[u] = ld_f4_pinned(gain + 4 * c4);
+                if (part) add[u] = sum_slices4_pinned(part + row_off + 4 * c4, n_split, split_stride);
+            } else {
+                v[u] = reinterpret_cast<const float4*>(xr)[c4];
+                gv[u] = reinterpret_cast<const float4*>(gain)[c4];   // not needed before the reduction, but no round trip after it
+                if (part) add[u] = sum_slices4(part + row_off + 4 * c4, n_split, split_stride);
+            }
         }
     }
 #pragma unroll
@@ -408,11 +467,13 @@ __global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ x, co
     __shared__ float red[32];
     pdl_launch_dependents();
     pdl_wait();
+    S_STAMP(1);
     const int i = blockIdx.x;
     const int r = row_idx ? row_idx[i] : i;
     const int nv = d >> 2;
     float4 v[MAXV], gv[MAXV];
     const float inv = rmsnorm_front<MAXV>(x + (size_t)r * d, part, n_split, split_stride, (size_t)r * d, nv, d, eps, gain, v, gv, red);
+    S_MID();
     if (xq) {
         // FP8 output: e4m3 codes of (value / s) with s = max |value| / 448 of this row (1 for a zero row)
         float amax = 0.f;
@@ -446,11 +507,39 @@ __global__ void __launch_bounds__(1024) rmsnorm_kernel(float* __restrict__ x, co
     }
 }
 
+// Few rows (one block per row cannot fill the machine, so the kernel is as long as its loads): 512 threads with two
+// float4 each and all their loads — row, gains, up to eight K slices — in flight at once, which takes 80 registers;
+// capped at 88 so that such a block (45 K registers) and a CTA of the next GEMM (18 K), launched early to fetch its
+// weights, fit an SM's register file together.  With 1024 threads that budget is 40 registers, too few for the loads.
+template <typename T>
+__global__ void __maxnreg__(88) rmsnorm_rows_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
+                                                    size_t split_stride, const float* __restrict__ gain, float eps,
+                                                    T* __restrict__ xn, const int32_t* __restrict__ row_idx, int d) {
+    __shared__ float red[32];
+    pdl_launch_dependents();
+    pdl_wait();
+    S_STAMP(1);
+    const int i = blockIdx.x;
+    const int r = row_idx ? row_idx[i] : i;
+    const int nv = d >> 2;
+    float4 v[2], gv[2];
+    const float inv = rmsnorm_front<2, true>(x + (size_t)r * d, part, n_split, split_stride, (size_t)r * d, nv, d, eps, gain, v, gv, red);
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int c4 = threadIdx.x + u * blockDim.x;
+        if (c4 < nv) {
+            const float4 g = gv[u];
+            Vec4<T>::store(xn + (size_t)i * d + 4 * c4, v[u].x * inv * g.x, v[u].y * inv * g.y, v[u].z * inv * g.z,
+                           v[u].w * inv * g.w);
+        }
+    }
+}
+
 // The same with NVFP4 output of the bfloat16 rounding of the normalised row (a kernel of its own, so that the
 // bf16 path's kernel carries neither its arguments nor its code): row scale max / (6 * 448), then blocks of 16
 // elements held by four neighbouring lanes.  d % 16 == 0.
 template <int MAXV>
-__global__ void __launch_bounds__(1024) rmsnorm_fp4_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
+__global__ void __launch_bounds__(1024, 1) rmsnorm_fp4_kernel(float* __restrict__ x, const float* __restrict__ part, int n_split,
                                    size_t split_stride, const float* __restrict__ gain, float eps,
                                    const int32_t* __restrict__ row_idx, int d, WdFp4Operand x4) {
     __shared__ float red[32];
@@ -541,7 +630,7 @@ __global__ void gemm_plain_kernel(const T* __restrict__ x, const T* __restrict__
 //                      transposed through shared memory and written with the rows (normally
 //                      consecutive positions) contiguous, so neighbouring lanes share sectors
 template <typename T>
-__global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
+__global__ void __launch_bounds__(256, 4) rope_scatter_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
                                     const int32_t* __restrict__ row_seq, const int32_t* __restrict__ row_pos,
                                     const float2* __restrict__ rope_tab, T* __restrict__ q, T* __restrict__ kcache,
                                     T* __restrict__ vcache, int n_rows, int Hq, int Hkv, int dh, int S, int Sp,
@@ -549,6 +638,7 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
     __shared__ float tile[32][33];
     pdl_launch_dependents();
     pdl_wait();
+    S_STAMP(2);
     const int half = dh >> 1;
     const int ncol = (Hq + 2 * Hkv) * dh;
     if ((int)blockIdx.x < n_qk_blocks) {
@@ -567,10 +657,32 @@ __global__ void rope_scatter_kernel(const float* __restrict__ part, int n_split,
                 const int h = grp * hpb + (int)threadIdx.x / tph, j = ((int)threadIdx.x % tph) * 4;
                 // (the loads do not wait for the index check: only the store of a cache row does)
                 if ((int)threadIdx.x < hpb * tph && h < Hq + Hkv) {
-                    const float4 a = sum_slices4(pr + h * dh + j, n_split, split_stride);
-                    const float4 bb = sum_slices4(pr + h * dh + half + j, n_split, split_stride);
-                    const float4 c01 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j);       // (cos, sin) x 2
-                    const float4 c23 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j + 2);
+                    float4 a, bb, c01, c23;
+                    if (n_split <= 4) {
+                        // few slices (the usual case): the table and both halves' slices in flight together
+                        float4 ta[4], tb[4];
+                        c01 = ld_f4_pinned(reinterpret_cast<const float*>(rope_tab + (size_t)r * half + j));   // (cos, sin) x 2
+                        c23 = ld_f4_pinned(reinterpret_cast<const float*>(rope_tab + (size_t)r * half + j + 2));
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            ta[k] = tb[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+                            if (k < n_split) {
+                                ta[k] = ld_f4_pinned(pr + h * dh + j + (size_t)k * split_stride);
+                                tb[k] = ld_f4_pinned(pr + h * dh + half + j + (size_t)k * split_stride);
+                            }
+                        }
+                        a = bb = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            a.x += ta[k].x; a.y += ta[k].y; a.z += ta[k].z; a.w += ta[k].w;
+                            bb.x += tb[k].x; bb.y += tb[k].y; bb.z += tb[k].z; bb.w += tb[k].w;
+                        }
+                    } else {
+                        a = sum_slices4(pr + h * dh + j, n_split, split_stride);
+                        bb = sum_slices4(pr + h * dh + half + j, n_split, split_stride);
+                        c01 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j);
+                        c23 = *reinterpret_cast<const float4*>(rope_tab + (size_t)r * half + j + 2);
+                    }
                     if (h >= Hq && !in_range) continue;
                     T* dst = h < Hq ? q + ((size_t)r * Hq + h) * dh : kcache + (((size_t)b * Hkv + (h - Hq)) * S + pos) * dh;
                     Vec4<T>::store(dst + j, a.x * c01.x - bb.x * c01.y, a.y * c01.z - bb.y * c01.w, a.z * c23.x - bb.z * c23.y,
@@ -711,6 +823,7 @@ __global__ void __launch_bounds__(256, 5) swiglu_kernel(const float* __restrict_
                                                         T* __restrict__ h, int n_rows, int F) {
     pdl_launch_dependents();
     pdl_wait();
+    S_STAMP(3);
     const int f4 = F >> 2;
     const size_t total = (size_t)n_rows * f4, stride = (size_t)gridDim.x * blockDim.x;
     // two positions per iteration so that four (or more) loads are in flight per thread
@@ -738,6 +851,44 @@ __global__ void __launch_bounds__(256, 5) swiglu_kernel(const float* __restrict_
             Vec4<T>::store(h + rb * F + 4 * cb, gb.x / (1.f + __expf(-gb.x)) * ub.x, gb.y / (1.f + __expf(-gb.y)) * ub.y,
                            gb.z / (1.f + __expf(-gb.z)) * ub.z, gb.w / (1.f + __expf(-gb.w)) * ub.w);
     }
+}
+
+// Few rows: one position per thread, 32-bit index arithmetic, all of a thread's loads (gate and up, up to four K
+// slices each) in flight together; registers capped like the kernel above, for the same reason.
+template <typename T>
+__global__ void __launch_bounds__(256, 5) swiglu_rows_kernel(const float* __restrict__ part, int n_split, size_t split_stride,
+                                                             T* __restrict__ h, int n_rows, int F) {
+    pdl_launch_dependents();
+    pdl_wait();
+    S_STAMP(3);
+    const int f4 = F >> 2;
+    const int i = (int)(blockIdx.x * blockDim.x + threadIdx.x);
+    if (i >= n_rows * f4) return;
+    const int r = i / f4, c = i - r * f4;
+    const float* pg = part + (size_t)r * 2 * F + 4 * c;
+    float4 tg[4], tu[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        tg[k] = tu[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (k < n_split) {
+            tg[k] = ld_f4_pinned(pg + (size_t)k * split_stride);
+            tu[k] = ld_f4_pinned(pg + (size_t)k * split_stride + F);
+        }
+    }
+    float4 g = make_float4(0.f, 0.f, 0.f, 0.f), u = g;
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        g.x += tg[k].x; g.y += tg[k].y; g.z += tg[k].z; g.w += tg[k].w;
+        u.x += tu[k].x; u.y += tu[k].y; u.z += tu[k].z; u.w += tu[k].w;
+    }
+    for (int s0 = 4; s0 < n_split; ++s0) {          // (more than four slices: not on this path's shapes, kept correct)
+        const float4 a = *reinterpret_cast<const float4*>(pg + (size_t)s0 * split_stride);
+        const float4 b = *reinterpret_cast<const float4*>(pg + (size_t)s0 * split_stride + F);
+        g.x += a.x; g.y += a.y; g.z += a.z; g.w += a.w;
+        u.x += b.x; u.y += b.y; u.z += b.z; u.w += b.w;
+    }
+    Vec4<T>::store(h + (size_t)r * F + 4 * c, g.x / (1.f + __expf(-g.x)) * u.x, g.y / (1.f + __expf(-g.y)) * u.y,
+                   g.z / (1.f + __expf(-g.z)) * u.z, g.w / (1.f + __expf(-g.w)) * u.w);
 }
 
 // FP8 variant: a cluster of four 256-thread blocks per row (light blocks, so that they are resident
@@ -1054,6 +1205,12 @@ void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size
                        row_idx, d, x4);
         return;
     }
+    static const int rms_rows = getenv("WD_RMS_ROWS") ? atoi(getenv("WD_RMS_ROWS")) : 1;
+    if (rms_rows && !xq && n_rows <= 128 && nv >= 512 && nv <= 1024 && nv % 2 == 0) {
+        WD_DISPATCH(dtype, launch_pdl(rmsnorm_rows_kernel<T>, dim3(n_rows), dim3((nv / 2 + 31) / 32 * 32), 0, st, x, part, n_split,
+                                      split_stride, gain, eps, (T*)xn, row_idx, d));
+        return;
+    }
     if (n_rows >= 512 && nv >= 256 && nv <= 4096) {
         // many rows: bandwidth matters, so more (smaller) blocks per SM with four float4 in flight per thread
         const int threads = ((nv + 3) / 4 + 31) / 32 * 32;
@@ -1120,6 +1277,12 @@ void wd_launch_swiglu(int dtype, const float* part, int n_split, size_t split_st
                       int n_rows, int F, cudaStream_t st) {
     if (n_rows <= 0) return;
     const size_t total = (size_t)n_rows * (F >> 2);
+    static const int sw_rows = getenv("WD_SWIGLU_ROWS") ? atoi(getenv("WD_SWIGLU_ROWS")) : 1;
+    if (sw_rows && total <= (size_t)148 * 3 * 256) {       // everything resident at once: one position per thread
+        WD_DISPATCH(dtype, launch_pdl(swiglu_rows_kernel<T>, dim3((unsigned)((total + 255) / 256)), dim3(256), 0, st, part, n_split,
+                                      split_stride, (T*)h, n_rows, F));
+        return;
+    }
     const int blocks = (int)((total + 255) / 256 < 148 * 16 ? (total + 255) / 256 : 148 * 16);
     WD_DISPATCH(dtype, launch_pdl(swiglu_kernel<T>, dim3(blocks), dim3(256), 0, st, part, n_split, split_stride,
                                   (T*)h, n_rows, F));
