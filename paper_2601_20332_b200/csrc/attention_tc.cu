@@ -108,6 +108,10 @@ constexpr int kStages = 3;                 // K stages and V stages
 // ring cut to fit) can be resident beside it and fetch their weights while the attention runs.
 #ifdef WD_GEMM_TRACE
 __device__ unsigned long long g_attn_end[64];       // latest CTA exit per layer
+__device__ unsigned long long g_attn_trace[160][8]; // per CTA (last launch): entry, wait returned, S ready, P written, O ready, part written, merged, exit
+#define A_STAMP(k) do { const unsigned int b_ = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); g_attn_trace[b_ < 160 ? b_ : 159][k] = global_ns(); } while (0)
+#else
+#define A_STAMP(k) do { } while (0)
 #endif
 
 template <bool kSingle>
@@ -174,7 +178,9 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_q, cons
         tc_fence_after();
         tmem_base = *tmem_slot;
     }
+    if (threadIdx.x == 64) A_STAMP(0);
     pdl_wait();                                   // q and the cache rows come from the previous kernel
+    if (threadIdx.x == 64) A_STAMP(1);
 
     if (!has_work) {
         // nothing to compute
@@ -315,6 +321,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_q, cons
             // reaches the barrier, and all of them leave together right after it.
             if (!mbar_wait(smem_u32(&bars[kSFull + s]), (uint32_t)(i >> 1) & 1u, abort_flag)) *abort_flag = 1;
             tc_fence_after();
+            if (threadIdx.x == 64 && i == 0) A_STAMP(2);
             const int n_keys = min(kTile, n_vis - (kt_begin + i) * kTile);   // valid keys in this tile
             // keys past n_vis may hold anything: zero their V columns so that 0 * garbage stays 0.
             // Thread (r, hf) owns row r (a head dim) of atom hf (keys 64*hf..) of the transposed V tile.
@@ -391,10 +398,12 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_q, cons
             fence_proxy_async_smem();                      // the zeroed V columns -> visible to the MMA
             tc_fence_before();
             mbar_arrive(smem_u32(&bars[kPFull + s]));
+            if (threadIdx.x == 64 && i == n_kt - 1) A_STAMP(3);
             if (!kSingle && i > 0) fold(i - 1, alpha_prev);
             alpha_prev = alpha;
         }
         if (ok && n_kt > 0) fold(n_kt - 1, alpha_prev);
+        if (threadIdx.x == 64) A_STAMP(4);
         // row sum = sum of the two halves (same running maximum on both sides)
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (*abort_flag) {
@@ -435,6 +444,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_q, cons
     }
     if (p.max_parts > 1) {
         // ------------------------------------------------------------ merge across the cluster
+        if (threadIdx.x == 64) A_STAMP(5);
         cluster_sync_all();                                // every part is in place and visible
         if (has_work && n_parts > 1 && warp >= 2) {
             // CTA z merges rows [z * per, (z + 1) * per).  An item = (row, group of 4 columns); a
@@ -508,6 +518,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_q, cons
                 }
             }
         }
+        if (threadIdx.x == 64) A_STAMP(6);
         cluster_sync_all();                                // no CTA leaves while its part may still be read
     }
     if (has_work) {
@@ -520,6 +531,7 @@ __device__ __forceinline__ void attention_tc_body(const CUtensorMap& map_q, cons
     }
 #ifdef WD_GEMM_TRACE
     if (threadIdx.x == 0) atomicMax(&g_attn_end[p.layer & 63], global_ns());
+    if (threadIdx.x == 64) A_STAMP(7);
 #endif
 }
 
@@ -537,6 +549,10 @@ attention_tc_single_kernel(const __grid_constant__ CUtensorMap map_q, const __gr
 }
 
 #ifdef WD_GEMM_TRACE
+extern "C" __attribute__((visibility("default"))) int wd_debug_attn_stamps(unsigned long long* host /*[160][8]*/) {
+    cudaDeviceSynchronize();
+    return (int)cudaMemcpyFromSymbol(host, g_attn_trace, sizeof(unsigned long long) * 160 * 8);
+}
 extern "C" __attribute__((visibility("default"))) int wd_debug_attn_trace(unsigned long long* host /*[64]*/) {
     cudaDeviceSynchronize();
     return (int)cudaMemcpyFromSymbol(host, g_attn_end, sizeof(unsigned long long) * 64);

@@ -524,6 +524,7 @@ __global__ void __maxnreg__(88) rmsnorm_rows_kernel(float* __restrict__ x, const
     const int nv = d >> 2;
     float4 v[2], gv[2];
     const float inv = rmsnorm_front<2, true>(x + (size_t)r * d, part, n_split, split_stride, (size_t)r * d, nv, d, eps, gain, v, gv, red);
+    S_MID();
 #pragma unroll
     for (int u = 0; u < 2; ++u) {
         const int c4 = threadIdx.x + u * blockDim.x;
