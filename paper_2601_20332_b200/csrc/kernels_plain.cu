@@ -1207,7 +1207,8 @@ void wd_launch_rmsnorm(int dtype, float* x, const float* part, int n_split, size
         return;
     }
     static const int rms_rows = getenv("WD_RMS_ROWS") ? atoi(getenv("WD_RMS_ROWS")) : 1;
-    if (rms_rows && !xq && n_rows <= 128 && nv >= 512 && nv <= 1024 && nv % 2 == 0) {
+    static const int rms_rows_max = getenv("WD_RMS_ROWS_MAX") ? atoi(getenv("WD_RMS_ROWS_MAX")) : 128;
+    if (rms_rows && !xq && n_rows <= rms_rows_max && nv >= 512 && nv <= 1024 && nv % 2 == 0) {
         WD_DISPATCH(dtype, launch_pdl(rmsnorm_rows_kernel<T>, dim3(n_rows), dim3((nv / 2 + 31) / 32 * 32), 0, st, x, part, n_split,
                                       split_stride, gain, eps, (T*)xn, row_idx, d));
         return;
