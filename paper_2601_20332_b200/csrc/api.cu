@@ -1376,7 +1376,6 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
         // memory): a shorter ring, but its weights are on their way while the attention still runs
         // (measured: 215 KB for the two CTAs together still fits an SM, 222 KB does not)
         c->tc.x_map_attn.smem_cap = (attn_smem > 0 && attn_smem <= 110 * 1024 && R_ <= 128) ? (int)(223232 - attn_smem) : 0;
-        if (getenv("WD_WO_CAP")) c->tc.x_map_attn.smem_cap = atoi(getenv("WD_WO_CAP"));
         WdTcSeg wo[1] = {{c->wo[l], D, c->tc.get(WD_TC_WO, l)}};
         if ((s = run_gemm(c, c->attn, &c->tc.x_map_attn, wo, 1, R_, hq, c->part, c->part_floats, status, stream, &go)) != WD_OK)
             return s;
