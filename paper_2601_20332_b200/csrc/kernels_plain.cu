@@ -1089,7 +1089,7 @@ __global__ void rowstats_kernel(const float* __restrict__ logits, int V, int chu
 // over chunks, then a fixed shuffle tree, so identical rows give identical bits); then
 // rank(i) = #{j : s_j < s_i or (s_j == s_i and pos_j < pos_i)}; positions are ascending inside a
 // sequence, so "pos_j < pos_i" is "j < i".
-__global__ void select_kernel(const float* __restrict__ ch_max, const int32_t* __restrict__ ch_idx,
+__global__ void __launch_bounds__(1024) select_kernel(const float* __restrict__ ch_max, const int32_t* __restrict__ ch_idx,
                               const double* __restrict__ ch_sum, int n_chunks, int32_t* __restrict__ row_token,
                               double* __restrict__ row_sumexp, const int32_t* __restrict__ act_pos,
                               const int32_t* __restrict__ act_off, int n_single, int k, int32_t* __restrict__ ids,
@@ -1381,7 +1381,8 @@ void wd_launch_select(const float* ch_max, const int32_t* ch_idx, const double* 
                       int32_t* sel_token, float* sel_conf, float* row_conf, uint8_t* decoded, int32_t* dec_step,
                       const int32_t* step_of_seq, cudaStream_t st) {
     if (batch <= 0) return;
-    launch_pdl(select_kernel, dim3(batch), dim3(256), 0, st, ch_max, ch_idx, ch_sum, n_chunks, row_token, row_sumexp,
+    // one warp per active row where the block allows it (a row is two dependent passes over its chunk statistics)
+    launch_pdl(select_kernel, dim3(batch), dim3(1024), 0, st, ch_max, ch_idx, ch_sum, n_chunks, row_token, row_sumexp,
                act_pos, act_off, n_single, k, ids, S, n_sel, sel_pos, sel_token, sel_conf, row_conf, decoded, dec_step,
                step_of_seq);
 }
