@@ -1093,6 +1093,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_ctarank();              // 0: issues the MMAs
+    if (threadIdx.x == 0) G_STAMP(0);
     // pairs per token group, this pair's index in its group, its token group (see TcParams::tok_split)
     const long long G = (gridDim.x >> 1) / (p.tok_split > 1 ? p.tok_split : 1), c = (blockIdx.x >> 1) % G;
     const int tok_group = (int)((blockIdx.x >> 1) / G);
@@ -1179,7 +1180,9 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
                     tma2_load_2d_hint(smem_u32(smem + (size_t)i * stage_bytes) + kStageA, &map_w1,
                                       cluster_map(smem_u32(&bars[i]), 0), w.kb * kKE, w.n0, pol_stream);
             }
+            G_STAMP(1);
             pdl_wait();
+            G_STAMP(2);
             Walk wx = w0;
             for (int i = 0; i < n_pre; ++i, advance(wx))
                 tma2_load_2d(smem_u32(smem + (size_t)i * stage_bytes) + stage_a, &map_x,
@@ -1359,6 +1362,7 @@ gemm_tc_pair_kernel(const __grid_constant__ CUtensorMap map_x, const __grid_cons
     }
     __syncthreads();
     cluster_sync();               // neither CTA frees tensor memory or leaves while the other may still signal it
+    if (threadIdx.x == 0) G_STAMP(7);
     if (warp == 1) {
         tc_fence_after();
         tmem2_dealloc(tmem_base, (uint32_t)(n_sets * set_cols));
@@ -1597,6 +1601,7 @@ wd_status tc_gemm_pair(const WdTcX* x, const WdTcSeg* segs, int nseg, int rows, 
     p.y = y;
     p.split_stride = slice;
     p.status = status;
+    p.trace_slot = nseg == 3 ? 0 : ((nseg == 2 || p.dual == 2) ? 2 : (K == col ? 1 : (K > col ? 3 : 4)));
     p.idesc = make_idesc(p.bn, 2 * kBM, fp8 != nullptr);
 
     CUtensorMap mx;
