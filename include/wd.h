@@ -231,7 +231,8 @@ WD_API wd_status wd_set_fusion(wd_ctx* ctx, int32_t mode);
 /* CUDA graphs for the kernels of a step (Section 4.3: the normal steps of a phase repeat the same
  * launch configuration).  On by default.  A step that the device plans (see wd_step) and whose launch
  * configuration — batch, computed rows, active rows, query tiles, key tiles, projection mode — recurs is
- * recorded into a graph (a normal step at once, a refresh step the second time it occurs) and replayed
+ * recorded into a graph (a normal step with full active windows at once, any other step the second time its
+ * configuration occurs) and replayed
  * from then on (at most 8 graphs per context, least recently used replaced); the planner kernel and the
  * copy of the result block stay ordinary launches on the caller's stream.  Graphs need the tensor-core
  * kernels (bf16, head_dim 128) and are used only while earlier steps are still queued: a caller that calls

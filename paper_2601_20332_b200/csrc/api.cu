@@ -1499,9 +1499,13 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
             ++c->graphs_replayed;
             graphed = true;
         } else {
-            // a refresh step's configuration rarely comes back (its rows grow with every phase): record it only
-            // when it does; a normal step's configuration recurs for many phases: record it at once
-            bool seen = !any_refresh;
+            // a refresh step's configuration rarely comes back (its rows grow with every phase), and neither does
+            // that of a step near the end of a generation, whose active window shrinks by the tokens unmasked every
+            // step: record those only when they do come back; a normal step with full windows recurs for many
+            // phases: record it at once
+            int live = 0;
+            for (int b = 0; b < batch; ++b) live += pend.cp[b].done ? 0 : 1;
+            bool seen = !any_refresh && NA == A * live;
             for (const wd_ctx::StepKey& k2 : c->seen) if (k2 == key) { seen = true; break; }
             if (!seen) {
                 if (c->seen.size() >= 32) c->seen.erase(c->seen.begin());
