@@ -1260,6 +1260,7 @@ extern "C" wd_status wd_step(wd_state* st, int32_t A, int32_t B, int32_t R, int3
     // ---- the kernels of the step, from the embedding to the selection (everything after the planner and
     // before the copy of the result block); launched directly, or recorded into a CUDA graph and replayed
     auto run_kernels = [&]() -> wd_status {
+    c->tc.x_map_attn.smem_cap = 0;          // set per block below, and only beside the single-key-tile attention
     if (fused) {
         // Five kernels per block.  The GEMM input is bf16(x * gain) without the 1/rms factor; the CTA
         // that completes an output tile applies it (from per-block sums of squares written by the
